@@ -1,0 +1,164 @@
+/*
+ * vsa2.h -- C ABI of the B200 (sm_100a) library for VSA2 routed block-sparse attention.
+ *
+ * The operator (paper Sec. 2.2) works on the tokens of a video latent grid (T, H, W), tiled
+ * into cubes of B = Bt*Bh*Bw tokens (N = Nt*Nh*Nw cubes after padding each dimension up to a
+ * whole number of cubes):
+ *
+ *   coarse branch  Q_c,K_c,V_c = MeanPool_B(Q,K,V); P_c = softmax(Q_c K_c^T * scale);
+ *                  O_c = Repeat_B(P_c V_c)                                       (Eq. 1-4)
+ *   router         Q_r,K_r = MeanPool_R(Q,K); P^_r = softmax(Q_r K_r^T * scale);
+ *                  P_r = MeanPool_{GxG}(P^_r), G = B/R                           (Eq. 5-7)
+ *   selection      keep the N*K largest of the N*N entries of P_r                (Eq. 8-9)
+ *   fine branch    O_f = BlockSparseAttn(Q,K,V; M)                               (Eq. 12)
+ *   merge          O = gate * O_c + O_f                                          (Eq. 14)
+ *
+ * Conventions shared by every entry point
+ *   - All tensor pointers are DEVICE pointers on the current CUDA device unless a comment says
+ *     "host".  Structs (params, map, saved, sizes) live in HOST memory and are read during
+ *     the call only.  The library never allocates or frees device memory in the four entry
+ *     points vsa2_route / vsa2_attn_fwd / vsa2_attn_bwd / vsa2_device_status: every buffer
+ *     is caller-owned.
+ *   - Q is [batch, heads_q, L, D], K and V are [batch, heads_kv, L, D], bf16, contiguous,
+ *     tokens in raster order l = (t*H + h)*W + w of the VALID grid (padding is never
+ *     materialised), L = T*H*W.  Query head hq uses KV head hq / (heads_q / heads_kv).
+ *   - Tensor base pointers must be 16-byte aligned (workspaces 256-byte aligned).
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream);
+ *     no entry point synchronises the stream except vsa2_device_status.
+ *   - Return value: VSA2_OK or a negative vsa2 error code; nothing is enqueued when an
+ *     argument check fails.  There is no CPU fallback.
+ */
+#ifndef VSA2_H_
+#define VSA2_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  VSA2_OK = 0,
+  VSA2_ERR_INVALID_ARG = -1,          /* null pointer, non-positive size, bad enum, heads_q % heads_kv != 0 ... */
+  VSA2_ERR_UNSUPPORTED = -2,          /* shape outside what the kernels implement, or device is not sm_100 */
+  VSA2_ERR_WORKSPACE_TOO_SMALL = -3,
+  VSA2_ERR_MISALIGNED = -4,
+  VSA2_ERR_CUDA = -5,                 /* a CUDA runtime/driver call or a launch failed */
+  VSA2_ERR_DEVICE_TIMEOUT = -6,       /* a bounded device-side wait ran out (reported by vsa2_device_status) */
+  VSA2_ERR_MAP_OVERFLOW = -7          /* more selected blocks than nnz_cap (reported by vsa2_device_status) */
+};
+
+enum { VSA2_PER_SEQUENCE = 0,         /* Eq. 8-9: the N*K largest entries of the flattened P_r per (batch, query head) */
+       VSA2_PER_QUERY = 1,            /* Sec. 2.1 (VSA form): the K largest per query block */
+       VSA2_PER_QUERY_BUDGET = 2 };   /* query block i keeps its own k_i largest (k_i from `budgets`) */
+
+enum { VSA2_BF16 = 0, VSA2_F32 = 1 };
+
+enum { VSA2_FLAG_NO_COARSE = 1 };     /* skip the coarse branch: O = O_f (the gate = 0 case, Sec. 2.3) */
+
+/* Problem statement (host struct). */
+typedef struct vsa2_params {
+  int32_t batch, heads_q, heads_kv, head_dim;  /* head_dim in {64, 128}; heads_q % heads_kv == 0 */
+  int32_t grid_t, grid_h, grid_w;              /* valid latent grid */
+  int32_t cube_t, cube_h, cube_w;              /* cube (block) shape, product must be 64 */
+  int32_t rpool_t, rpool_h, rpool_w;           /* router pooling R, each divides the cube dimension */
+  int32_t select_mode;                         /* VSA2_PER_* */
+  int32_t topk;                                /* K in blocks (clamped to N); if 0, K = max(1, round(keep_fraction*N)) */
+  float   keep_fraction;                       /* 1 - block sparsity, used only when topk == 0 */
+  float   softmax_scale;                       /* 0 => 1/sqrt(head_dim); used by coarse, router and fine alike */
+  int32_t out_dtype;                           /* VSA2_BF16 or VSA2_F32: dtype of O, dQ, dK, dV */
+  int32_t flags;                               /* VSA2_FLAG_* */
+  int64_t nnz_cap;                             /* capacity of col_idx/row_idx per (batch, query head); 0 => N*K.
+                                                  PER_QUERY_BUDGET requires it (>= sum_i min(k_i, N)). */
+} vsa2_params;
+
+/* Derived sizes (host struct, filled by vsa2_query_sizes).  Element counts are totals over batch and heads. */
+typedef struct vsa2_sizes {
+  int32_t n_cubes;            /* N */
+  int32_t n_subcubes;         /* G */
+  int32_t block_tokens;       /* B */
+  int32_t topk_eff;           /* K after clamping / keep_fraction */
+  int64_t seq_len;            /* L */
+  int64_t nnz_cap;            /* per (batch, query head) */
+  int64_t ptr_elems;          /* int32 elements of row_ptr and of col_ptr: batch*heads_q*(N+1) */
+  int64_t idx_elems;          /* int32 elements of col_idx and of row_idx: batch*heads_q*nnz_cap */
+  int64_t pooled_q_elems;     /* float elements of saved.qc and saved.oc_hat: batch*heads_q*N*D */
+  int64_t pooled_kv_elems;    /* float elements of saved.kc and of saved.vc: batch*heads_kv*N*D */
+  int64_t lse_c_elems;        /* float elements of saved.lse_c: batch*heads_q*N */
+  size_t  route_workspace_bytes;
+  size_t  fwd_workspace_bytes;
+  size_t  bwd_workspace_bytes;
+} vsa2_sizes;
+
+/* Block map of the selected (query block, KV block) pairs (host struct of device pointers).
+ * CSR: query block i of (b, hq) owns col_idx[(b*Hq+hq)*nnz_cap + row_ptr[(b*Hq+hq)*(N+1) + i ...+ i+1)],
+ * KV block indices ascending.  CSC is the transpose (KV block j -> ascending query blocks), used by
+ * the dK/dV pass. */
+typedef struct vsa2_map {
+  int32_t* row_ptr;   /* [batch, heads_q, N+1] */
+  int32_t* col_idx;   /* [batch, heads_q, nnz_cap] */
+  int32_t* col_ptr;   /* [batch, heads_q, N+1] */
+  int32_t* row_idx;   /* [batch, heads_q, nnz_cap] */
+} vsa2_map;
+
+/* State the forward pass leaves for the backward pass (host struct of device pointers, fp32). */
+typedef struct vsa2_saved {
+  float* qc;       /* [batch, heads_q,  N, D]  Eq. 1 */
+  float* kc;       /* [batch, heads_kv, N, D] */
+  float* vc;       /* [batch, heads_kv, N, D] */
+  float* oc_hat;   /* [batch, heads_q,  N, D]  Eq. 3 */
+  float* lse_c;    /* [batch, heads_q,  N]     log-sum-exp of the coarse scores */
+} vsa2_saved;
+
+/* Validates `p` and fills `out`.  Pure host arithmetic; no CUDA call. */
+int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out);
+
+/* Router + selection (Eq. 5-9).  Reads q, k; writes the CSR and CSC maps.
+ *   budgets: device int32 [batch, heads_q, N], only for VSA2_PER_QUERY_BUDGET (else may be NULL).
+ *   workspace: >= sizes.route_workspace_bytes; holds the pooled bf16 operands, the router
+ *   log-sum-exp, P_r [batch, heads_q, N, N] fp32 and selection scratch.  Its first word is the
+ *   device status word read by vsa2_device_status.
+ * Pooled router operands are the bf16 rounding of the fp32 mean (sum taken along w, then h, then
+ * t; valid tokens only).  Ties in the TopK go to the lower flat index i*N + j.  No gradient is
+ * defined through this call (Sec. 2.1). */
+int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t* budgets,
+               const vsa2_map* map_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Read-only access to the block scores P_r [batch, heads_q, N, N] (fp32) that the last vsa2_route
+ * call on `workspace` left there; valid until the workspace is reused.  Returns NULL on bad input. */
+const float* vsa2_route_scores(const vsa2_params* p, const void* workspace);
+
+/* Coarse branch (Eq. 1-4), fine branch (Eq. 12) and merge (Eq. 14).
+ *   gate: fp32 [batch, heads_q, L] (the caller's tanh(X W_g), Eq. 13); NULL means gate = 0.
+ *   o:    [batch, heads_q, L, D] in p->out_dtype;  lse: fp32 [batch, heads_q, L], natural log of the
+ *         fine branch's softmax denominator (scaled scores); -inf and O_f = 0 for a query block
+ *         with no selected KV block.
+ *   saved: filled for vsa2_attn_bwd (ignored, may be NULL, with VSA2_FLAG_NO_COARSE).
+ *   workspace: >= sizes.fwd_workspace_bytes. */
+int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
+                  const vsa2_map* map, void* o, float* lse, const vsa2_saved* saved,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward of vsa2_attn_fwd for a fixed map (the map carries no gradient, Sec. 2.1).
+ *   o, lse, saved: as written by the forward call;  d_o: bf16 [batch, heads_q, L, D].
+ *   dq [batch, heads_q, L, D], dk, dv [batch, heads_kv, L, D] in p->out_dtype (dk, dv summed over the
+ *   query heads of a group); dgate fp32 [batch, heads_q, L] (may be NULL).
+ *   workspace: >= sizes.bwd_workspace_bytes.  No floating-point atomics are used: results are
+ *   bitwise reproducible run to run. */
+int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
+                  const vsa2_map* map, const void* o, const float* lse, const vsa2_saved* saved,
+                  const void* d_o, void* dq, void* dk, void* dv, float* dgate,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the status word at the start of `workspace` and stores it in
+ * *status_out (host): VSA2_OK, VSA2_ERR_DEVICE_TIMEOUT or VSA2_ERR_MAP_OVERFLOW. */
+int vsa2_device_status(const void* workspace, void* cuda_stream, int32_t* status_out);
+
+/* Static string for an error code. */
+const char* vsa2_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VSA2_H_ */

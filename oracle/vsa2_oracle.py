@@ -282,20 +282,14 @@ def head_forward(Q, K, V, gate, mask, geo: Geometry, scale):
     return dict(O=O, O_f=O_f, lse=lse, Oc_hat=Oc_hat, lse_c=lse_c, Qc=Qc, Kc=Kc, Vc=Vc)
 
 
-def head_backward(Q, K, V, gate, mask, geo: Geometry, scale, dO, fwd=None):
-    """Gradients of sum(O * dO) for one (batch, query head) given the block mask.
+def coarse_path_backward(Q, K, V, gate, geo: Geometry, scale, dO, fwd):
+    """Backward of the merge, repeat, coarse attention and cube pooling (Eq. 14, 4, 3, 2, 1).
 
-    Chain rule on Eq. 14, 4, 3, 2, 1 (coarse path) and on Eq. 12 (fine path).
-    The mask is a constant: nothing flows through Eq. 5-9.
-    Returns dQ, dK, dV [L, D] (dK, dV are this query head's contribution) and dGate [L].
+    Returns dGate [L] and the coarse branch's contribution to dQ, dK, dV [L, D].
     """
-    if fwd is None:
-        fwd = head_forward(Q, K, V, gate, mask, geo, scale)
-    L, D = Q.shape
     Oc_hat, Qc, Kc, Vc = fwd["Oc_hat"], fwd["Qc"], fwd["Kc"], fwd["Vc"]
     # merge (Eq. 14) and repeat (Eq. 4)
     dGate = (dO * Oc_hat[geo.cube_of]).sum(axis=1)
-    dO_f = dO
     dOc_hat = np.zeros_like(Oc_hat)
     np.add.at(dOc_hat, geo.cube_of, gate[:, None] * dO)
     # coarse attention backward (Eq. 2-3): dense softmax attention on N tokens
@@ -309,25 +303,73 @@ def head_backward(Q, K, V, gate, mask, geo: Geometry, scale, dO, fwd=None):
     dKc = (dSc.T @ Qc) * scale
     # mean-pool backward (Eq. 1): every valid token gets grad / count of its cube
     inv = 1.0 / geo.cube_count[geo.cube_of][:, None]
-    dQ = dQc[geo.cube_of] * inv
-    dK = dKc[geo.cube_of] * inv
-    dV = dVc[geo.cube_of] * inv
-    # fine branch backward (Eq. 12)
-    delta = (dO_f * fwd["O_f"]).sum(axis=1)
-    for i in range(geo.N):
+    return dict(dGate=dGate, dQ=dQc[geo.cube_of] * inv, dK=dKc[geo.cube_of] * inv, dV=dVc[geo.cube_of] * inv)
+
+
+def fine_backward(Q, K, V, mask, geo: Geometry, scale, dO, lse, O_f, rows=None):
+    """Backward of Eq. 12 for the query cubes in `rows` (all if None).
+
+    With P = exp(S - lse), delta = rowsum(dO * O_f), dP = dO V^T, dS = P * (dP - delta):
+    dQ = dS K * scale, dK = dS^T Q * scale, dV = P^T dO.  Returns the three [L, D] arrays
+    (dK and dV hold only the contributions of the visited query cubes).
+    """
+    dQ, dK, dV = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)
+    delta = (dO * O_f).sum(axis=1)
+    for i in (range(geo.N) if rows is None else rows):
         cols = np.nonzero(mask[i])[0]
         if cols.size == 0:
             continue
         qt = geo.cube_tokens[i]
         kt = np.concatenate([geo.cube_tokens[j] for j in cols])
         s = (Q[qt] @ K[kt].T) * scale
-        P = np.exp(s - fwd["lse"][qt][:, None])
-        dV[kt] += P.T @ dO_f[qt]
-        dP = dO_f[qt] @ V[kt].T
+        P = np.exp(s - lse[qt][:, None])
+        dV[kt] += P.T @ dO[qt]
+        dP = dO[qt] @ V[kt].T
         dS = P * (dP - delta[qt][:, None])
         dQ[qt] += (dS @ K[kt]) * scale
         dK[kt] += (dS.T @ Q[qt]) * scale
-    return dict(dQ=dQ, dK=dK, dV=dV, dGate=dGate)
+    return dQ, dK, dV
+
+
+def fine_backward_kv_cubes(Q, K, V, mask, geo: Geometry, scale, dO, kv_cubes):
+    """Fine-branch dK, dV restricted to the tokens of the KV cubes in `kv_cubes`.
+
+    Visits every query cube that keeps one of those KV cubes, runs its forward (over all of its
+    kept blocks, to get lse and delta) and adds its gradient contribution to the requested
+    cubes only.  Same formulas as fine_backward; used where the full backward is too slow.
+    """
+    dK, dV = np.zeros_like(K), np.zeros_like(V)
+    kv_cubes = list(kv_cubes)
+    rows = np.nonzero(mask[:, kv_cubes].any(axis=1))[0]
+    O_f, lse = fine_attention(Q, K, V, mask, geo, scale, rows=rows)
+    delta = (dO * O_f).sum(axis=1)
+    for i in rows:
+        qt = geo.cube_tokens[i]
+        for j in kv_cubes:
+            if not mask[i, j]:
+                continue
+            kt = geo.cube_tokens[j]
+            s = (Q[qt] @ K[kt].T) * scale
+            P = np.exp(s - lse[qt][:, None])
+            dV[kt] += P.T @ dO[qt]
+            dP = dO[qt] @ V[kt].T
+            dS = P * (dP - delta[qt][:, None])
+            dK[kt] += (dS.T @ Q[qt]) * scale
+    return dK, dV
+
+
+def head_backward(Q, K, V, gate, mask, geo: Geometry, scale, dO, fwd=None):
+    """Gradients of sum(O * dO) for one (batch, query head) given the block mask.
+
+    Chain rule on Eq. 14, 4, 3, 2, 1 (coarse path) and on Eq. 12 (fine path).
+    The mask is a constant: nothing flows through Eq. 5-9.
+    Returns dQ, dK, dV [L, D] (dK, dV are this query head's contribution) and dGate [L].
+    """
+    if fwd is None:
+        fwd = head_forward(Q, K, V, gate, mask, geo, scale)
+    c = coarse_path_backward(Q, K, V, gate, geo, scale, dO, fwd)
+    fq, fk, fv = fine_backward(Q, K, V, mask, geo, scale, dO, fwd["lse"], fwd["O_f"])
+    return dict(dQ=c["dQ"] + fq, dK=c["dK"] + fk, dV=c["dV"] + fv, dGate=c["dGate"])
 
 
 # ----------------------------------------------------------------------------

@@ -1,0 +1,301 @@
+// C ABI of the VSA2 library: argument checks, workspace layout, kernel sequencing.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace vsa2;
+
+namespace {
+
+struct RouteLayout {
+  size_t status, qr, kr, lse_r, pr, hist, state, row_tau, row_eq_take, row_cnt, row_gt, row_eq, bitmap, total;
+  int words;
+};
+struct BwdLayout {
+  size_t status, delta, d_oc_hat, delta_c, dqc, dkc, dvc, total;
+};
+
+struct Carver {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  }
+};
+
+int fill_geo(const vsa2_params* p, Geo* g) {
+  if (p == nullptr) return VSA2_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->heads_q <= 0 || p->heads_kv <= 0 || p->grid_t <= 0 || p->grid_h <= 0 || p->grid_w <= 0 ||
+      p->cube_t <= 0 || p->cube_h <= 0 || p->cube_w <= 0 || p->rpool_t <= 0 || p->rpool_h <= 0 || p->rpool_w <= 0)
+    return VSA2_ERR_INVALID_ARG;
+  if (p->heads_q % p->heads_kv) return VSA2_ERR_INVALID_ARG;
+  if (p->select_mode < VSA2_PER_SEQUENCE || p->select_mode > VSA2_PER_QUERY_BUDGET) return VSA2_ERR_INVALID_ARG;
+  if (p->out_dtype != VSA2_BF16 && p->out_dtype != VSA2_F32) return VSA2_ERR_INVALID_ARG;
+  if (p->topk < 0 || p->nnz_cap < 0 || !(p->softmax_scale >= 0.f)) return VSA2_ERR_INVALID_ARG;
+  if (p->cube_t % p->rpool_t || p->cube_h % p->rpool_h || p->cube_w % p->rpool_w) return VSA2_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return VSA2_ERR_UNSUPPORTED;
+  if ((long long)p->cube_t * p->cube_h * p->cube_w != kBlockTokens) return VSA2_ERR_UNSUPPORTED;
+  if (p->batch > 65535 || p->heads_q > 65535) return VSA2_ERR_UNSUPPORTED;
+  g->batch = p->batch; g->Hq = p->heads_q; g->Hkv = p->heads_kv; g->rep = p->heads_q / p->heads_kv; g->D = p->head_dim;
+  g->T = p->grid_t; g->H = p->grid_h; g->W = p->grid_w;
+  long long L = (long long)g->T * g->H * g->W;
+  if (L > 0x7fffffffLL / 128) return VSA2_ERR_UNSUPPORTED;
+  g->L = (int)L;
+  g->Bt = p->cube_t; g->Bh = p->cube_h; g->Bw = p->cube_w;
+  g->Nt = (g->T + g->Bt - 1) / g->Bt; g->Nh = (g->H + g->Bh - 1) / g->Bh; g->Nw = (g->W + g->Bw - 1) / g->Bw;
+  g->N = g->Nt * g->Nh * g->Nw;
+  g->Rt = p->rpool_t; g->Rh = p->rpool_h; g->Rw = p->rpool_w;
+  g->Gt = g->Bt / g->Rt; g->Gh = g->Bh / g->Rh; g->Gw = g->Bw / g->Rw;
+  g->G = g->Gt * g->Gh * g->Gw;
+  if (128 % g->G) return VSA2_ERR_UNSUPPORTED;
+  int K = p->topk;
+  if (K == 0) {
+    if (!(p->keep_fraction > 0.f) || p->keep_fraction > 1.f) {
+      if (p->select_mode != VSA2_PER_QUERY_BUDGET) return VSA2_ERR_INVALID_ARG;
+      K = 1;
+    } else {
+      K = (int)lroundf(p->keep_fraction * (float)g->N);
+      if (K < 1) K = 1;
+    }
+  }
+  if (K > g->N) K = g->N;
+  g->K = K;
+  g->mode = p->select_mode;
+  g->out_f32 = p->out_dtype == VSA2_F32;
+  g->flags = p->flags;
+  g->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)g->D);
+  if (p->nnz_cap > 0) g->nnz_cap = p->nnz_cap;
+  else if (p->select_mode == VSA2_PER_QUERY_BUDGET) return VSA2_ERR_INVALID_ARG;
+  else g->nnz_cap = (long long)g->N * K;
+  return VSA2_OK;
+}
+
+RouteLayout route_layout(const Geo& g) {
+  RouteLayout r;
+  Carver c;
+  const size_t BHq = (size_t)g.batch * g.Hq, BHk = (size_t)g.batch * g.Hkv, NG = (size_t)g.N * g.G;
+  r.words = (g.N + 31) / 32;
+  r.status = c.take(sizeof(StatusBlock));
+  r.qr = c.take(BHq * NG * g.D * sizeof(bf16));
+  r.kr = c.take(BHk * NG * g.D * sizeof(bf16));
+  r.lse_r = c.take(BHq * NG * sizeof(float));
+  r.pr = c.take(BHq * (size_t)g.N * g.N * sizeof(float));
+  r.hist = c.take(BHq * 3 * 2048 * sizeof(unsigned));
+  r.state = c.take(BHq * 8 * sizeof(unsigned));
+  r.row_tau = c.take(BHq * g.N * sizeof(float));
+  r.row_eq_take = c.take(BHq * g.N * sizeof(int));
+  r.row_cnt = c.take(BHq * g.N * sizeof(int));
+  r.row_gt = c.take(BHq * g.N * sizeof(int));
+  r.row_eq = c.take(BHq * g.N * sizeof(int));
+  r.bitmap = c.take(BHq * (size_t)g.N * r.words * sizeof(unsigned));
+  r.total = c.off;
+  return r;
+}
+
+BwdLayout bwd_layout(const Geo& g) {
+  BwdLayout r;
+  Carver c;
+  const size_t BHq = (size_t)g.batch * g.Hq;
+  r.status = c.take(sizeof(StatusBlock));
+  r.delta = c.take(BHq * g.L * sizeof(float));
+  r.d_oc_hat = c.take(BHq * g.N * g.D * sizeof(float));
+  r.delta_c = c.take(BHq * g.N * sizeof(float));
+  r.dqc = c.take(BHq * g.N * g.D * sizeof(float));
+  r.dkc = c.take(BHq * g.N * g.D * sizeof(float));
+  r.dvc = c.take(BHq * g.N * g.D * sizeof(float));
+  r.total = c.off;
+  return r;
+}
+
+size_t fwd_workspace_bytes(const Geo&) { return align_up(sizeof(StatusBlock), 256); }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+// The kernels are built for sm_100a only.
+int check_device() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return VSA2_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return VSA2_ERR_CUDA;
+  return major == 10 ? VSA2_OK : VSA2_ERR_UNSUPPORTED;
+}
+
+template <typename T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(reinterpret_cast<unsigned char*>(ws) + off); }
+
+#define VSA2_CUDA(call)                              \
+  do {                                               \
+    cudaError_t e_ = (call);                         \
+    if (e_ != cudaSuccess) return VSA2_ERR_CUDA;     \
+  } while (0)
+
+}  // namespace
+
+extern "C" {
+
+int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
+  if (out == nullptr) return VSA2_ERR_INVALID_ARG;
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  memset(out, 0, sizeof(*out));
+  out->n_cubes = g.N;
+  out->n_subcubes = g.G;
+  out->block_tokens = kBlockTokens;
+  out->topk_eff = g.K;
+  out->seq_len = g.L;
+  out->nnz_cap = g.nnz_cap;
+  const long long BHq = (long long)g.batch * g.Hq, BHk = (long long)g.batch * g.Hkv;
+  out->ptr_elems = BHq * (g.N + 1);
+  out->idx_elems = BHq * g.nnz_cap;
+  out->pooled_q_elems = BHq * g.N * g.D;
+  out->pooled_kv_elems = BHk * g.N * g.D;
+  out->lse_c_elems = BHq * g.N;
+  out->route_workspace_bytes = route_layout(g).total;
+  out->fwd_workspace_bytes = fwd_workspace_bytes(g);
+  out->bwd_workspace_bytes = bwd_layout(g).total;
+  return VSA2_OK;
+}
+
+int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t* budgets, const vsa2_map* map,
+               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  if (!q || !k || !map || !workspace || !map->row_ptr || !map->col_idx || !map->col_ptr || !map->row_idx)
+    return VSA2_ERR_INVALID_ARG;
+  if (g.mode == VSA2_PER_QUERY_BUDGET && budgets == nullptr) return VSA2_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned256(workspace)) return VSA2_ERR_MISALIGNED;
+  const RouteLayout lay = route_layout(g);
+  if (workspace_bytes < lay.total) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if ((rc = check_device()) != VSA2_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  StatusBlock* status = at<StatusBlock>(workspace, lay.status);
+  VSA2_CUDA(cudaMemsetAsync(status, 0, sizeof(StatusBlock), st));
+  bf16* qr = at<bf16>(workspace, lay.qr);
+  bf16* kr = at<bf16>(workspace, lay.kr);
+  VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(q), g.Hq, qr, nullptr, st));
+  VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(k), g.Hkv, kr, nullptr, st));
+  float* pr = at<float>(workspace, lay.pr);
+  VSA2_CUDA(launch_router_scores(g, qr, kr, at<float>(workspace, lay.lse_r), pr, st));
+  SelectScratch s;
+  s.hist = at<unsigned>(workspace, lay.hist);
+  s.state = at<unsigned>(workspace, lay.state);
+  s.row_tau = at<float>(workspace, lay.row_tau);
+  s.row_eq_take = at<int>(workspace, lay.row_eq_take);
+  s.row_cnt = at<int>(workspace, lay.row_cnt);
+  s.row_gt = at<int>(workspace, lay.row_gt);
+  s.row_eq = at<int>(workspace, lay.row_eq);
+  s.bitmap = at<unsigned>(workspace, lay.bitmap);
+  s.words = lay.words;
+  VSA2_CUDA(launch_select(g, pr, budgets, s, map->row_ptr, map->col_idx, map->col_ptr, map->row_idx, status, st));
+  return VSA2_OK;
+}
+
+const float* vsa2_route_scores(const vsa2_params* p, const void* workspace) {
+  Geo g;
+  if (workspace == nullptr || fill_geo(p, &g) != VSA2_OK) return nullptr;
+  return reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(workspace) + route_layout(g).pr);
+}
+
+int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
+                  const vsa2_map* map, void* o, float* lse, const vsa2_saved* saved, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream) {
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  if (!q || !k || !v || !map || !o || !lse || !workspace || !map->row_ptr || !map->col_idx) return VSA2_ERR_INVALID_ARG;
+  const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE);
+  if (coarse && (!saved || !saved->qc || !saved->kc || !saved->vc || !saved->oc_hat || !saved->lse_c))
+    return VSA2_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned256(workspace))
+    return VSA2_ERR_MISALIGNED;
+  if (workspace_bytes < fwd_workspace_bytes(g)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if ((rc = check_device()) != VSA2_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  VSA2_CUDA(cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), st));
+  const bf16* qb = reinterpret_cast<const bf16*>(q);
+  const bf16* kb = reinterpret_cast<const bf16*>(k);
+  const bf16* vb = reinterpret_cast<const bf16*>(v);
+  if (coarse) {
+    VSA2_CUDA(launch_pool(g, qb, g.Hq, nullptr, saved->qc, st));
+    VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
+    VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
+    VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+  }
+  VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
+                            coarse ? saved->oc_hat : nullptr, o, lse, st));
+  return VSA2_OK;
+}
+
+int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
+                  const vsa2_map* map, const void* o, const float* lse, const vsa2_saved* saved, const void* d_o,
+                  void* dq, void* dk, void* dv, float* dgate, void* workspace, size_t workspace_bytes,
+                  void* cuda_stream) {
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  if (!q || !k || !v || !map || !o || !lse || !d_o || !dq || !dk || !dv || !workspace || !map->row_ptr ||
+      !map->col_idx || !map->col_ptr || !map->row_idx)
+    return VSA2_ERR_INVALID_ARG;
+  const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr;
+  if (coarse && (!saved || !saved->qc || !saved->kc || !saved->vc || !saved->oc_hat || !saved->lse_c))
+    return VSA2_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
+      !aligned16(dk) || !aligned16(dv) || !aligned256(workspace))
+    return VSA2_ERR_MISALIGNED;
+  const BwdLayout lay = bwd_layout(g);
+  if (workspace_bytes < lay.total) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if ((rc = check_device()) != VSA2_OK) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  VSA2_CUDA(cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), st));
+  const bf16* qb = reinterpret_cast<const bf16*>(q);
+  const bf16* kb = reinterpret_cast<const bf16*>(k);
+  const bf16* vb = reinterpret_cast<const bf16*>(v);
+  const bf16* dob = reinterpret_cast<const bf16*>(d_o);
+  float* delta = at<float>(workspace, lay.delta);
+  float* d_oc_hat = at<float>(workspace, lay.d_oc_hat);
+  float* dqc = at<float>(workspace, lay.dqc);
+  float* dkc = at<float>(workspace, lay.dkc);
+  float* dvc = at<float>(workspace, lay.dvc);
+  if (!coarse && dgate != nullptr)
+    VSA2_CUDA(cudaMemsetAsync(dgate, 0, (size_t)g.batch * g.Hq * g.L * sizeof(float), st));
+  VSA2_CUDA(launch_bwd_preprocess(g, dob, o, coarse ? gate : nullptr, coarse ? saved->oc_hat : nullptr, delta,
+                                  coarse ? dgate : nullptr, d_oc_hat, st));
+  if (coarse)
+    VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
+                                at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
+  VSA2_CUDA(launch_fine_bwd_dq(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx, coarse ? dqc : nullptr, dq,
+                               st));
+  VSA2_CUDA(launch_fine_bwd_dkv(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx, coarse ? dkc : nullptr,
+                                coarse ? dvc : nullptr, dk, dv, st));
+  return VSA2_OK;
+}
+
+int vsa2_device_status(const void* workspace, void* cuda_stream, int32_t* status_out) {
+  if (workspace == nullptr || status_out == nullptr) return VSA2_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  VSA2_CUDA(cudaStreamSynchronize(st));
+  int s = 0;
+  VSA2_CUDA(cudaMemcpy(&s, workspace, sizeof(int), cudaMemcpyDeviceToHost));
+  *status_out = s;
+  return VSA2_OK;
+}
+
+const char* vsa2_strerror(int code) {
+  switch (code) {
+    case VSA2_OK: return "ok";
+    case VSA2_ERR_INVALID_ARG: return "invalid argument";
+    case VSA2_ERR_UNSUPPORTED: return "unsupported shape, dtype or device (needs sm_100)";
+    case VSA2_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case VSA2_ERR_MISALIGNED: return "pointer not aligned (16 bytes for tensors, 256 bytes for workspaces)";
+    case VSA2_ERR_CUDA: return "CUDA call or kernel launch failed";
+    case VSA2_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case VSA2_ERR_MAP_OVERFLOW: return "more selected blocks than nnz_cap";
+    default: return "unknown vsa2 error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,142 @@
+// Shared device/host definitions of the VSA2 library: geometry of the latent grid, index
+// maps between raster tokens and cubes (paper Sec. 2.2 "Permutation"), workspace layout.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vsa2.h"
+
+namespace vsa2 {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kBlockTokens = 64;   // B: tokens per cube handled by the kernels
+
+// Everything a kernel needs to know about the problem; passed by value.
+struct Geo {
+  int batch, Hq, Hkv, rep, D;
+  int T, H, W, L;
+  int Bt, Bh, Bw, Nt, Nh, Nw, N;
+  int Rt, Rh, Rw, Gt, Gh, Gw, G;
+  int K;            // TopK after clamping
+  int mode;         // VSA2_PER_*
+  int out_f32;      // 1: outputs are fp32, 0: bf16
+  int flags;
+  float scale;      // softmax scale
+  long long nnz_cap;
+};
+
+// Status block at the start of every workspace.
+struct StatusBlock {
+  int status;       // VSA2_OK / VSA2_ERR_DEVICE_TIMEOUT / VSA2_ERR_MAP_OVERFLOW
+  int detail;
+  int pad[62];
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// cube n -> (nt, nh, nw);  n = (nt*Nh + nh)*Nw + nw
+__device__ __forceinline__ void cube_coords(const Geo& g, int n, int& nt, int& nh, int& nw) {
+  nw = n % g.Nw;
+  int r = n / g.Nw;
+  nh = r % g.Nh;
+  nt = r / g.Nh;
+}
+
+// position p in [0, B) inside a cube, ordered (bt, bh, bw) -> raster token index, or -1 if padding
+__device__ __forceinline__ int cube_token(const Geo& g, int nt, int nh, int nw, int p) {
+  int bw = p % g.Bw;
+  int r = p / g.Bw;
+  int bh = r % g.Bh;
+  int bt = r / g.Bh;
+  int t = nt * g.Bt + bt, h = nh * g.Bh + bh, w = nw * g.Bw + bw;
+  if (t >= g.T || h >= g.H || w >= g.W) return -1;
+  return (t * g.H + h) * g.W + w;
+}
+
+// 64-bit mask of the valid positions of cube n
+__device__ __forceinline__ unsigned long long cube_valid_mask(const Geo& g, int n) {
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  unsigned long long m = 0ull;
+  for (int p = 0; p < kBlockTokens; ++p)
+    if (cube_token(g, nt, nh, nw, p) >= 0) m |= 1ull << p;
+  return m;
+}
+
+// number of valid tokens of cube n
+__device__ __forceinline__ int cube_count(const Geo& g, int n) {
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  int ct = min(g.Bt, g.T - nt * g.Bt), ch = min(g.Bh, g.H - nh * g.Bh), cw = min(g.Bw, g.W - nw * g.Bw);
+  return ct * ch * cw;
+}
+
+// router sub-cube gsub of cube n: number of valid tokens (0 = the sub-cube is padding only)
+__device__ __forceinline__ int subcube_count(const Geo& g, int n, int gsub) {
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  int gw = gsub % g.Gw;
+  int r = gsub / g.Gw;
+  int gh = r % g.Gh;
+  int gt = r / g.Gh;
+  int t0 = nt * g.Bt + gt * g.Rt, h0 = nh * g.Bh + gh * g.Rh, w0 = nw * g.Bw + gw * g.Rw;
+  int ct = max(0, min(g.Rt, g.T - t0)), ch = max(0, min(g.Rh, g.H - h0)), cw = max(0, min(g.Rw, g.W - w0));
+  return ct * ch * cw;
+}
+
+__device__ __forceinline__ void store_out(void* base, size_t idx, float v, int out_f32) {
+  if (out_f32) reinterpret_cast<float*>(base)[idx] = v;
+  else reinterpret_cast<bf16*>(base)[idx] = __float2bfloat16_rn(v);
+}
+
+__device__ __forceinline__ float load_out(const void* base, size_t idx, int out_f32) {
+  return out_f32 ? reinterpret_cast<const float*>(base)[idx]
+                 : __bfloat162float(reinterpret_cast<const bf16*>(base)[idx]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// launchers implemented in the .cu files (all enqueue on `st`, return cudaGetLastError())
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_pool(const Geo& g, const bf16* x, int heads, bf16* xr, float* xc, cudaStream_t st);
+
+cudaError_t launch_router_scores(const Geo& g, const bf16* qr, const bf16* kr, float* lse_r, float* pr,
+                                 cudaStream_t st);
+
+struct SelectScratch {
+  unsigned* hist;        // [BH][3][2048]
+  unsigned* state;       // [BH][8]
+  float* row_tau;        // [BH][N]
+  int* row_eq_take;      // [BH][N]
+  int* row_cnt;          // [BH][N]
+  int* row_gt;           // [BH][N]
+  int* row_eq;           // [BH][N]
+  unsigned* bitmap;      // [BH][N][words]
+  int words;             // ceil(N/32)
+};
+cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, const SelectScratch& s,
+                          int* row_ptr, int* col_idx, int* col_ptr, int* row_idx, StatusBlock* status,
+                          cudaStream_t st);
+
+cudaError_t launch_coarse_fwd(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
+                              float* lse_c, cudaStream_t st);
+cudaError_t launch_coarse_bwd(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
+                              const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
+                              float* dvc, cudaStream_t st);
+
+cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                            const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, float* lse,
+                            cudaStream_t st);
+
+cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const float* gate,
+                                  const float* oc_hat, float* delta, float* dgate, float* d_oc_hat,
+                                  cudaStream_t st);
+cudaError_t launch_fine_bwd_dq(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                               const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
+                               const float* dqc, void* dq, cudaStream_t st);
+cudaError_t launch_fine_bwd_dkv(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                                const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
+                                const float* dkc, const float* dvc, void* dk, void* dv, cudaStream_t st);
+
+}  // namespace vsa2

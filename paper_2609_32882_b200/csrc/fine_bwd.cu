@@ -1,0 +1,297 @@
+// Backward of the fine branch (gradient of paper Eq. 12) and of the gated merge (Eq. 14).
+//   preprocess: delta = rowsum(dO * O_f), dGate = rowsum(dO * O_c), dO_c_hat[n] = sum_{l in n} gate_l dO_l
+//   dQ pass   : query-block stationary, driven by the CSR map
+//   dK/dV pass: KV-block stationary, driven by the CSC map (transpose), summing the query heads of a
+//               GQA group; no floating-point atomics anywhere.
+// With P = exp(S*scale - lse), dP = dO V^T, dS = P * (dP - delta):
+//   dQ = dS K * scale,  dK = dS^T Q * scale,  dV = P^T dO.
+// The pooling backward of the coarse branch (Eq. 1) is added in the epilogues:
+//   dX[l] += dX_c[cube(l)] / count(cube(l)).
+#include "wmma_tile.cuh"
+
+namespace vsa2 {
+
+// ------------------------------------------------------------------------------------------
+// preprocess: grid (N, Hq, batch), 256 threads
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restrict__ d_o, const void* __restrict__ o,
+                                                             const float* __restrict__ gate,
+                                                             const float* __restrict__ oc_hat, Geo g,
+                                                             float* __restrict__ delta, float* __restrict__ dgate,
+                                                             float* __restrict__ d_oc_hat) {
+  __shared__ float gdo[64][D];   // gate_l * dO_l
+  const int i = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
+  const size_t bhq = (size_t)b * g.Hq + hq;
+  const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr;
+  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  constexpr int OC = D / 4;
+  int nt, nh, nw;
+  cube_coords(g, i, nt, nh, nw);
+  const int l = cube_token(g, nt, nh, nw, r);
+  float s_oo = 0.f, s_oc = 0.f;
+  const float gt = (coarse && l >= 0) ? gate[bhq * g.L + l] : 0.f;
+  const float* oc = oc_hat + (bhq * g.N + i) * D;
+  for (int c = 0; c < OC; ++c) {
+    int d = qd * OC + c;
+    float dov = 0.f;
+    if (l >= 0) {
+      size_t idx = (bhq * g.L + l) * D + d;
+      dov = __bfloat162float(d_o[idx]);
+      s_oo = fmaf(dov, load_out(o, idx, g.out_f32), s_oo);
+      if (coarse) s_oc = fmaf(dov, oc[d], s_oc);
+    }
+    gdo[r][d] = gt * dov;
+  }
+  s_oo += __shfl_xor_sync(0xffffffffu, s_oo, 1);
+  s_oo += __shfl_xor_sync(0xffffffffu, s_oo, 2);
+  s_oc += __shfl_xor_sync(0xffffffffu, s_oc, 1);
+  s_oc += __shfl_xor_sync(0xffffffffu, s_oc, 2);
+  if (qd == 0 && l >= 0) {
+    delta[bhq * g.L + l] = s_oo - gt * s_oc;     // rowsum(dO * (O - gate*O_c)) = rowsum(dO * O_f)
+    if (dgate != nullptr) dgate[bhq * g.L + l] = s_oc;
+  }
+  if (coarse) {
+    __syncthreads();
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+      float acc = 0.f;
+#pragma unroll 8
+      for (int p = 0; p < 64; ++p) acc += gdo[p][d];
+      d_oc_hat[(bhq * g.N + i) * D + d] = acc;
+    }
+  }
+}
+
+cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const float* gate,
+                                  const float* oc_hat, float* delta, float* dgate, float* d_oc_hat, cudaStream_t st) {
+  dim3 grid(g.N, g.Hq, g.batch);
+  if (g.D == 128) bwd_preprocess_kernel<128><<<grid, 256, 0, st>>>(d_o, o, gate, oc_hat, g, delta, dgate, d_oc_hat);
+  else bwd_preprocess_kernel<64><<<grid, 256, 0, st>>>(d_o, o, gate, oc_hat, g, delta, dgate, d_oc_hat);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// dQ pass: grid (N, Hq, batch), 256 threads
+// ------------------------------------------------------------------------------------------
+template <int D>
+struct BwdSmem {
+  static constexpr int LDX = D + 8;
+  static constexpr int LDS = 64 + 4;
+  static constexpr int LDP = 64 + 8;
+  static constexpr int LDO = D + 4;
+  static constexpr size_t tile = 64 * LDX * sizeof(bf16);
+  static constexpr size_t sc = 64 * LDS * sizeof(float);
+  static constexpr size_t pb = 64 * LDP * sizeof(bf16);
+  static constexpr size_t acc = 64 * LDO * sizeof(float);
+  static constexpr size_t dq_bytes = 4 * tile + 2 * sc + pb + acc + 2 * 64 * sizeof(float) + 64;
+  static constexpr size_t dkv_bytes = 4 * tile + 2 * sc + 2 * pb + 2 * acc + 2 * 64 * sizeof(float) + 128;
+};
+
+template <int D>
+__global__ void __launch_bounds__(256) fine_bwd_dq_kernel(const bf16* __restrict__ q, const bf16* __restrict__ k,
+                                                          const bf16* __restrict__ v, const bf16* __restrict__ d_o,
+                                                          const float* __restrict__ lse, const float* __restrict__ delta,
+                                                          const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
+                                                          const float* __restrict__ dqc, Geo g, void* __restrict__ dq) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  using SM = BwdSmem<D>;
+  bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
+  bf16* dOs = Qs + 64 * SM::LDX;
+  bf16* Ks = dOs + 64 * SM::LDX;
+  bf16* Vs = Ks + 64 * SM::LDX;
+  float* S = reinterpret_cast<float*>(Vs + 64 * SM::LDX);
+  float* dP = S + 64 * SM::LDS;
+  bf16* dS = reinterpret_cast<bf16*>(dP + 64 * SM::LDS);
+  float* A = reinterpret_cast<float*>(dS + 64 * SM::LDP);
+  float* row_lse = A + 64 * SM::LDO;
+  float* row_delta = row_lse + 64;
+  unsigned char* kvalid = reinterpret_cast<unsigned char*>(row_delta + 64);
+
+  const int i = blockIdx.x, hq = blockIdx.y, b = blockIdx.z, hk = hq / g.rep;
+  const size_t bhq = (size_t)b * g.Hq + hq, bhk = (size_t)b * g.Hkv + hk;
+  const bf16* kh = k + bhk * g.L * D;
+  const bf16* vh = v + bhk * g.L * D;
+  const int* cols = col_idx + bhq * g.nnz_cap;
+  const int beg = row_ptr[bhq * (g.N + 1) + i], end = row_ptr[bhq * (g.N + 1) + i + 1];
+  int nt, nh, nw;
+  cube_coords(g, i, nt, nh, nw);
+
+  load_cube_tile<D>(Qs, SM::LDX, q + bhq * g.L * D, g, i);
+  load_cube_tile<D>(dOs, SM::LDX, d_o + bhq * g.L * D, g, i);
+  for (int e = threadIdx.x; e < 64 * SM::LDO; e += blockDim.x) A[e] = 0.f;
+  if (threadIdx.x < 64) {
+    int l = cube_token(g, nt, nh, nw, threadIdx.x);
+    row_lse[threadIdx.x] = l >= 0 ? lse[bhq * g.L + l] : INFINITY;   // +inf => P = 0 for padding rows
+    row_delta[threadIdx.x] = l >= 0 ? delta[bhq * g.L + l] : 0.f;
+  }
+  for (int it = beg; it < end; ++it) {
+    const int j = cols[it];
+    __syncthreads();
+    load_cube_tile<D>(Ks, SM::LDX, kh, g, j);
+    load_cube_tile<D>(Vs, SM::LDX, vh, g, j);
+    if (threadIdx.x < 64) {
+      int jt, jh, jw;
+      cube_coords(g, j, jt, jh, jw);
+      kvalid[threadIdx.x] = cube_token(g, jt, jh, jw, threadIdx.x) >= 0;
+    }
+    __syncthreads();
+    tile_gemm<64, 64, D, false, true, false>(Qs, SM::LDX, Ks, SM::LDX, S, SM::LDS);
+    tile_gemm<64, 64, D, false, true, false>(dOs, SM::LDX, Vs, SM::LDX, dP, SM::LDS);
+    __syncthreads();
+    for (int e = threadIdx.x; e < 64 * 64; e += blockDim.x) {
+      int r = e >> 6, c = e & 63;
+      float p = kvalid[c] ? __expf(S[r * SM::LDS + c] * g.scale - row_lse[r]) : 0.f;
+      float ds = p * (dP[r * SM::LDS + c] - row_delta[r]) * g.scale;
+      dS[r * SM::LDP + c] = __float2bfloat16_rn(ds);
+    }
+    __syncthreads();
+    tile_gemm<64, D, 64, false, false, true>(dS, SM::LDP, Ks, SM::LDX, A, SM::LDO);
+  }
+  __syncthreads();
+  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  constexpr int OC = D / 4;
+  const int l = cube_token(g, nt, nh, nw, r);
+  if (l >= 0) {
+    const bool coarse = dqc != nullptr;
+    const float inv_cnt = 1.f / (float)cube_count(g, i);
+    const float* qc_g = coarse ? dqc + (bhq * g.N + i) * D : nullptr;
+    const size_t obase = (bhq * g.L + l) * D;
+    for (int c = 0; c < OC; ++c) {
+      int d = qd * OC + c;
+      float val = A[r * SM::LDO + d];
+      if (coarse) val = fmaf(qc_g[d], inv_cnt, val);
+      store_out(dq, obase + d, val, g.out_f32);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// dK/dV pass: grid (N, Hkv, batch), 256 threads
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) fine_bwd_dkv_kernel(const bf16* __restrict__ q, const bf16* __restrict__ k,
+                                                           const bf16* __restrict__ v, const bf16* __restrict__ d_o,
+                                                           const float* __restrict__ lse, const float* __restrict__ delta,
+                                                           const int* __restrict__ col_ptr, const int* __restrict__ row_idx,
+                                                           const float* __restrict__ dkc, const float* __restrict__ dvc,
+                                                           Geo g, void* __restrict__ dk, void* __restrict__ dv) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  using SM = BwdSmem<D>;
+  bf16* Ks = reinterpret_cast<bf16*>(smem_raw);
+  bf16* Vs = Ks + 64 * SM::LDX;
+  bf16* Qs = Vs + 64 * SM::LDX;
+  bf16* dOs = Qs + 64 * SM::LDX;
+  float* S = reinterpret_cast<float*>(dOs + 64 * SM::LDX);
+  float* dP = S + 64 * SM::LDS;
+  bf16* P = reinterpret_cast<bf16*>(dP + 64 * SM::LDS);
+  bf16* dS = P + 64 * SM::LDP;
+  float* AK = reinterpret_cast<float*>(dS + 64 * SM::LDP);
+  float* AV = AK + 64 * SM::LDO;
+  float* row_lse = AV + 64 * SM::LDO;
+  float* row_delta = row_lse + 64;
+  unsigned char* kvalid = reinterpret_cast<unsigned char*>(row_delta + 64);
+
+  const int j = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const size_t bhk = (size_t)b * g.Hkv + hk;
+  int jt, jh, jw;
+  cube_coords(g, j, jt, jh, jw);
+  load_cube_tile<D>(Ks, SM::LDX, k + bhk * g.L * D, g, j);
+  load_cube_tile<D>(Vs, SM::LDX, v + bhk * g.L * D, g, j);
+  for (int e = threadIdx.x; e < 64 * SM::LDO; e += blockDim.x) { AK[e] = 0.f; AV[e] = 0.f; }
+  if (threadIdx.x < 64) kvalid[threadIdx.x] = cube_token(g, jt, jh, jw, threadIdx.x) >= 0;
+
+  for (int hh = 0; hh < g.rep; ++hh) {
+    const int hq = hk * g.rep + hh;
+    const size_t bhq = (size_t)b * g.Hq + hq;
+    const int* rows = row_idx + bhq * g.nnz_cap;
+    const int beg = col_ptr[bhq * (g.N + 1) + j], end = col_ptr[bhq * (g.N + 1) + j + 1];
+    for (int it = beg; it < end; ++it) {
+      const int i = rows[it];
+      __syncthreads();
+      load_cube_tile<D>(Qs, SM::LDX, q + bhq * g.L * D, g, i);
+      load_cube_tile<D>(dOs, SM::LDX, d_o + bhq * g.L * D, g, i);
+      if (threadIdx.x < 64) {
+        int it_, ih_, iw_;
+        cube_coords(g, i, it_, ih_, iw_);
+        int l = cube_token(g, it_, ih_, iw_, threadIdx.x);
+        row_lse[threadIdx.x] = l >= 0 ? lse[bhq * g.L + l] : INFINITY;
+        row_delta[threadIdx.x] = l >= 0 ? delta[bhq * g.L + l] : 0.f;
+      }
+      __syncthreads();
+      tile_gemm<64, 64, D, false, true, false>(Qs, SM::LDX, Ks, SM::LDX, S, SM::LDS);
+      tile_gemm<64, 64, D, false, true, false>(dOs, SM::LDX, Vs, SM::LDX, dP, SM::LDS);
+      __syncthreads();
+      for (int e = threadIdx.x; e < 64 * 64; e += blockDim.x) {
+        int r = e >> 6, c = e & 63;
+        float p = kvalid[c] ? __expf(S[r * SM::LDS + c] * g.scale - row_lse[r]) : 0.f;
+        float ds = p * (dP[r * SM::LDS + c] - row_delta[r]) * g.scale;
+        P[r * SM::LDP + c] = __float2bfloat16_rn(p);
+        dS[r * SM::LDP + c] = __float2bfloat16_rn(ds);
+      }
+      __syncthreads();
+      tile_gemm<64, D, 64, true, false, true>(P, SM::LDP, dOs, SM::LDX, AV, SM::LDO);    // dV += P^T dO
+      tile_gemm<64, D, 64, true, false, true>(dS, SM::LDP, Qs, SM::LDX, AK, SM::LDO);    // dK += dS^T Q
+    }
+  }
+  __syncthreads();
+  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  constexpr int OC = D / 4;
+  const int l = cube_token(g, jt, jh, jw, r);
+  if (l >= 0) {
+    const bool coarse = dkc != nullptr;
+    const float inv_cnt = 1.f / (float)cube_count(g, j);
+    const size_t obase = (bhk * g.L + l) * D;
+    for (int c = 0; c < OC; ++c) {
+      int d = qd * OC + c;
+      float vk = AK[r * SM::LDO + d], vv = AV[r * SM::LDO + d];
+      if (coarse) {
+        float ck = 0.f, cv = 0.f;
+        for (int hh = 0; hh < g.rep; ++hh) {
+          size_t cidx = (((size_t)b * g.Hq + hk * g.rep + hh) * g.N + j) * D + d;
+          ck += dkc[cidx];
+          cv += dvc[cidx];
+        }
+        vk = fmaf(ck, inv_cnt, vk);
+        vv = fmaf(cv, inv_cnt, vv);
+      }
+      store_out(dk, obase + d, vk, g.out_f32);
+      store_out(dv, obase + d, vv, g.out_f32);
+    }
+  }
+}
+
+cudaError_t launch_fine_bwd_dq(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                               const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
+                               const float* dqc, void* dq, cudaStream_t st) {
+  dim3 grid(g.N, g.Hq, g.batch);
+  cudaError_t e;
+  if (g.D == 128) {
+    size_t smb = BwdSmem<128>::dq_bytes;
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_bwd_dq_kernel<128><<<grid, 256, smb, st>>>(q, k, v, d_o, lse, delta, row_ptr, col_idx, dqc, g, dq);
+  } else {
+    size_t smb = BwdSmem<64>::dq_bytes;
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_bwd_dq_kernel<64><<<grid, 256, smb, st>>>(q, k, v, d_o, lse, delta, row_ptr, col_idx, dqc, g, dq);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fine_bwd_dkv(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                                const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
+                                const float* dkc, const float* dvc, void* dk, void* dv, cudaStream_t st) {
+  dim3 grid(g.N, g.Hkv, g.batch);
+  cudaError_t e;
+  if (g.D == 128) {
+    size_t smb = BwdSmem<128>::dkv_bytes;
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_bwd_dkv_kernel<128><<<grid, 256, smb, st>>>(q, k, v, d_o, lse, delta, col_ptr, row_idx, dkc, dvc, g, dk, dv);
+  } else {
+    size_t smb = BwdSmem<64>::dkv_bytes;
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_bwd_dkv_kernel<64><<<grid, 256, smb, st>>>(q, k, v, d_o, lse, delta, col_ptr, row_idx, dkc, dvc, g, dk, dv);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace vsa2

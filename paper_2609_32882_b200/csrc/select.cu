@@ -1,0 +1,321 @@
+// TopK selection on the router block scores and construction of the block map
+// (paper Eq. 8-9: the N*K largest of the flattened N*N scores; Sec. 2.1 for the per-row form).
+// Scores are non-negative floats, so their bit patterns order like unsigned integers: the
+// K-th largest value is found by a most-significant-digit radix select, ties at the threshold
+// go to the lower flat index, and rows/columns are emitted in ascending order (deterministic,
+// integer work only).
+#include "common.cuh"
+
+namespace vsa2 {
+
+constexpr int kHistBins = 2048;
+// digit positions of the three per-sequence passes: bits [31:21], [20:10], [9:0]
+__device__ __forceinline__ int seq_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
+__device__ __forceinline__ unsigned seq_mask(int pass) { return pass == 2 ? 0x3FFu : 0x7FFu; }
+
+// state[bh*8 + ..]: 0 prefix bits, 1 prefix mask, 2 remaining k, 3 tau bits, 4 eq_take
+__global__ void sel_init_kernel(unsigned* state, unsigned* hist, int BH, unsigned keep) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < BH * 3 * kHistBins) hist[i] = 0u;
+  if (i < BH) {
+    state[i * 8 + 0] = 0u;
+    state[i * 8 + 1] = 0u;
+    state[i * 8 + 2] = keep;
+    state[i * 8 + 3] = 0u;
+    state[i * 8 + 4] = 0u;
+  }
+}
+
+__global__ void __launch_bounds__(256) sel_hist_kernel(const float* __restrict__ pr, long long n_elems,
+                                                       const unsigned* __restrict__ state, unsigned* hist, int pass) {
+  __shared__ unsigned sh[kHistBins];
+  const int bh = blockIdx.y;
+  for (int i = threadIdx.x; i < kHistBins; i += blockDim.x) sh[i] = 0u;
+  __syncthreads();
+  const unsigned prefix = state[bh * 8 + 0], pmask = state[bh * 8 + 1];
+  const int shift = seq_shift(pass);
+  const unsigned dmask = seq_mask(pass);
+  const unsigned* src = reinterpret_cast<const unsigned*>(pr) + (size_t)bh * n_elems;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_elems;
+       i += (long long)gridDim.x * blockDim.x) {
+    unsigned v = __ldg(src + i);
+    if ((v & pmask) == prefix) atomicAdd(&sh[(v >> shift) & dmask], 1u);
+  }
+  __syncthreads();
+  unsigned* dst = hist + ((size_t)bh * 3 + pass) * kHistBins;
+  for (int i = threadIdx.x; i < kHistBins; i += blockDim.x)
+    if (sh[i]) atomicAdd(&dst[i], sh[i]);
+}
+
+__global__ void sel_pick_kernel(unsigned* state, const unsigned* hist, int pass) {
+  const int bh = blockIdx.x;
+  if (threadIdx.x != 0) return;
+  const unsigned* hsrc = hist + ((size_t)bh * 3 + pass) * kHistBins;
+  unsigned remaining = state[bh * 8 + 2];
+  const int nb = (int)seq_mask(pass) + 1;
+  int bin = 0;
+  for (int d = nb - 1; d >= 0; --d) {
+    unsigned c = hsrc[d];
+    if (c >= remaining) { bin = d; break; }
+    remaining -= c;
+  }
+  const int shift = seq_shift(pass);
+  unsigned prefix = state[bh * 8 + 0] | ((unsigned)bin << shift);
+  state[bh * 8 + 0] = prefix;
+  state[bh * 8 + 1] |= seq_mask(pass) << shift;
+  state[bh * 8 + 2] = remaining;
+  if (pass == 2) {
+    state[bh * 8 + 3] = prefix;      // tau: the smallest kept value
+    state[bh * 8 + 4] = remaining;   // how many entries equal to tau are kept
+  }
+}
+
+// per-sequence: count entries above / equal to tau in every row.  grid (N, BH), 128 threads
+__global__ void __launch_bounds__(128) sel_row_stats_kernel(const float* __restrict__ pr, int N,
+                                                            const unsigned* __restrict__ state, int* row_gt, int* row_eq) {
+  const int i = blockIdx.x, bh = blockIdx.y;
+  const unsigned tau = state[bh * 8 + 3];
+  const unsigned* src = reinterpret_cast<const unsigned*>(pr) + ((size_t)bh * N + i) * N;
+  int gt = 0, eq = 0;
+  for (int j = threadIdx.x; j < N; j += blockDim.x) {
+    unsigned v = __ldg(src + j);
+    gt += v > tau;
+    eq += v == tau;
+  }
+  __shared__ int sg[4], se[4];
+  for (int o = 16; o; o >>= 1) {
+    gt += __shfl_xor_sync(0xffffffffu, gt, o);
+    eq += __shfl_xor_sync(0xffffffffu, eq, o);
+  }
+  if ((threadIdx.x & 31) == 0) { sg[threadIdx.x >> 5] = gt; se[threadIdx.x >> 5] = eq; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    row_gt[(size_t)bh * N + i] = sg[0] + sg[1] + sg[2] + sg[3];
+    row_eq[(size_t)bh * N + i] = se[0] + se[1] + se[2] + se[3];
+  }
+}
+
+// per-row modes: radix select of the k_i-th largest of row i.  grid (N, BH), 256 threads
+__global__ void __launch_bounds__(256) sel_row_topk_kernel(const float* __restrict__ pr, int N, int K,
+                                                           const int* __restrict__ budgets, float* row_tau,
+                                                           int* row_eq_take, int* row_cnt) {
+  __shared__ unsigned sh[256];
+  __shared__ unsigned s_prefix, s_mask, s_remaining;
+  const int i = blockIdx.x, bh = blockIdx.y;
+  const unsigned* src = reinterpret_cast<const unsigned*>(pr) + ((size_t)bh * N + i) * N;
+  int k = budgets ? budgets[(size_t)bh * N + i] : K;
+  k = max(0, min(k, N));
+  const size_t o = (size_t)bh * N + i;
+  if (k == 0) {
+    if (threadIdx.x == 0) { row_tau[o] = INFINITY; row_eq_take[o] = 0; row_cnt[o] = 0; }
+    return;
+  }
+  if (threadIdx.x == 0) { s_prefix = 0u; s_mask = 0u; s_remaining = (unsigned)k; }
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    sh[threadIdx.x] = 0u;
+    __syncthreads();
+    const unsigned prefix = s_prefix, pmask = s_mask;
+    for (int j = threadIdx.x; j < N; j += blockDim.x) {
+      unsigned v = __ldg(src + j);
+      if ((v & pmask) == prefix) atomicAdd(&sh[(v >> shift) & 0xFFu], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned remaining = s_remaining;
+      int bin = 0;
+      for (int d = 255; d >= 0; --d) {
+        unsigned c = sh[d];
+        if (c >= remaining) { bin = d; break; }
+        remaining -= c;
+      }
+      s_prefix = prefix | ((unsigned)bin << shift);
+      s_mask = pmask | (0xFFu << shift);
+      s_remaining = remaining;
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    row_tau[o] = __uint_as_float(s_prefix);
+    row_eq_take[o] = (int)s_remaining;
+    row_cnt[o] = k;
+  }
+}
+
+// exclusive scan of v over the block (1024 threads); returns the prefix, total in `total`
+__device__ __forceinline__ int block_excl_scan(int v, int* warp_sums, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane];
+    int wi = w;
+    for (int o = 1; o < 32; o <<= 1) {
+      int t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
+    }
+    warp_sums[lane] = wi - w;        // exclusive prefix of the warp sums
+    if (lane == 31) warp_sums[32] = wi;
+  }
+  __syncthreads();
+  int res = warp_sums[warp] + incl - v;
+  total = warp_sums[32];
+  __syncthreads();
+  return res;
+}
+
+// one block per (batch, head): per-sequence tie quota per row, then row_ptr = exclusive scan of counts
+__global__ void __launch_bounds__(1024) sel_scan_rows_kernel(int N, int per_sequence, const unsigned* __restrict__ state,
+                                                             const int* __restrict__ row_gt, const int* __restrict__ row_eq,
+                                                             float* row_tau, int* row_eq_take, int* row_cnt, int* row_ptr,
+                                                             long long nnz_cap, StatusBlock* status) {
+  __shared__ int ws[33];
+  const int bh = blockIdx.x;
+  const size_t base = (size_t)bh * N;
+  if (per_sequence) {
+    const unsigned tau = state[bh * 8 + 3];
+    const int quota = (int)state[bh * 8 + 4];
+    int carry = 0;
+    for (int i0 = 0; i0 < N; i0 += blockDim.x) {
+      int i = i0 + threadIdx.x;
+      int eq = i < N ? row_eq[base + i] : 0;
+      int tot;
+      int before = carry + block_excl_scan(eq, ws, tot);
+      if (i < N) {
+        int take = max(0, min(eq, quota - before));
+        row_eq_take[base + i] = take;
+        row_cnt[base + i] = row_gt[base + i] + take;
+        row_tau[base + i] = __uint_as_float(tau);
+      }
+      carry += tot;
+    }
+    __syncthreads();
+  }
+  int carry = 0;
+  for (int i0 = 0; i0 < N; i0 += blockDim.x) {
+    int i = i0 + threadIdx.x;
+    int c = i < N ? row_cnt[base + i] : 0;
+    int tot;
+    int pre = carry + block_excl_scan(c, ws, tot);
+    if (i < N) row_ptr[(size_t)bh * (N + 1) + i] = pre;
+    carry += tot;
+  }
+  if (threadIdx.x == 0) {
+    row_ptr[(size_t)bh * (N + 1) + N] = carry;
+    if ((long long)carry > nnz_cap) atomicExch(&status->status, VSA2_ERR_MAP_OVERFLOW);
+  }
+}
+
+// one warp per row: ordered emission of the kept columns and of the row's bitmap words
+__global__ void __launch_bounds__(256) sel_emit_rows_kernel(const float* __restrict__ pr, int N, int words,
+                                                            const float* __restrict__ row_tau,
+                                                            const int* __restrict__ row_eq_take,
+                                                            const int* __restrict__ row_ptr, int* col_idx,
+                                                            unsigned* bitmap, long long nnz_cap) {
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int bh = blockIdx.y;
+  if (i >= N) return;
+  const unsigned* src = reinterpret_cast<const unsigned*>(pr) + ((size_t)bh * N + i) * N;
+  const unsigned tau = __float_as_uint(row_tau[(size_t)bh * N + i]);
+  const int take = row_eq_take[(size_t)bh * N + i];
+  int pos = row_ptr[(size_t)bh * (N + 1) + i];
+  int eq_seen = 0;
+  int* out = col_idx + (size_t)bh * nnz_cap;
+  const unsigned lt = (1u << lane) - 1u;
+  for (int w = 0; w < words; ++w) {
+    int j = w * 32 + lane;
+    unsigned v = j < N ? __ldg(src + j) : 0u;
+    bool gt = j < N && v > tau;
+    bool eq = j < N && v == tau;
+    unsigned eqb = __ballot_sync(0xffffffffu, eq);
+    bool sel = gt || (eq && (eq_seen + __popc(eqb & lt)) < take);
+    unsigned selb = __ballot_sync(0xffffffffu, sel);
+    if (sel) {
+      int p = pos + __popc(selb & lt);
+      if (p < nnz_cap) out[p] = j;
+    }
+    pos += __popc(selb);
+    eq_seen += __popc(eqb);
+    if (lane == 0) bitmap[((size_t)bh * N + i) * words + w] = selb;
+  }
+}
+
+// thread per column: count set bits down the rows.  grid (ceil(N/256), BH)
+__global__ void __launch_bounds__(256) sel_col_count_kernel(const unsigned* __restrict__ bitmap, int N, int words,
+                                                            int* col_cnt) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x, bh = blockIdx.y;
+  if (j >= N) return;
+  const unsigned* bm = bitmap + (size_t)bh * N * words + (j >> 5);
+  int c = 0;
+  for (int i = 0; i < N; ++i) c += (__ldg(bm + (size_t)i * words) >> (j & 31)) & 1u;
+  col_cnt[(size_t)bh * N + j] = c;
+}
+
+__global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* __restrict__ col_cnt, int* col_ptr) {
+  __shared__ int ws[33];
+  const int bh = blockIdx.x;
+  int carry = 0;
+  for (int j0 = 0; j0 < N; j0 += blockDim.x) {
+    int j = j0 + threadIdx.x;
+    int c = j < N ? col_cnt[(size_t)bh * N + j] : 0;
+    int tot;
+    int pre = carry + block_excl_scan(c, ws, tot);
+    if (j < N) col_ptr[(size_t)bh * (N + 1) + j] = pre;
+    carry += tot;
+  }
+  if (threadIdx.x == 0) col_ptr[(size_t)bh * (N + 1) + N] = carry;
+}
+
+__global__ void __launch_bounds__(256) sel_emit_cols_kernel(const unsigned* __restrict__ bitmap, int N, int words,
+                                                            const int* __restrict__ col_ptr, int* row_idx,
+                                                            long long nnz_cap) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x, bh = blockIdx.y;
+  if (j >= N) return;
+  const unsigned* bm = bitmap + (size_t)bh * N * words + (j >> 5);
+  int pos = col_ptr[(size_t)bh * (N + 1) + j];
+  int* out = row_idx + (size_t)bh * nnz_cap;
+  for (int i = 0; i < N; ++i) {
+    if ((__ldg(bm + (size_t)i * words) >> (j & 31)) & 1u) {
+      if (pos < nnz_cap) out[pos] = i;
+      ++pos;
+    }
+  }
+}
+
+cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, const SelectScratch& s, int* row_ptr,
+                          int* col_idx, int* col_ptr, int* row_idx, StatusBlock* status, cudaStream_t st) {
+  const int BH = g.batch * g.Hq, N = g.N;
+  const long long n_elems = (long long)N * N;
+  if (g.mode == VSA2_PER_SEQUENCE) {
+    const unsigned keep = (unsigned)((long long)N * g.K);
+    int init_n = BH * 3 * kHistBins;
+    sel_init_kernel<<<(init_n + 255) / 256, 256, 0, st>>>(s.state, s.hist, BH, keep);
+    int chunks = (int)((n_elems + 256 * 16 - 1) / (256 * 16));
+    if (chunks > 256) chunks = 256;
+    for (int pass = 0; pass < 3; ++pass) {
+      sel_hist_kernel<<<dim3(chunks, BH), 256, 0, st>>>(pr, n_elems, s.state, s.hist, pass);
+      sel_pick_kernel<<<BH, 32, 0, st>>>(s.state, s.hist, pass);
+    }
+    sel_row_stats_kernel<<<dim3(N, BH), 128, 0, st>>>(pr, N, s.state, s.row_gt, s.row_eq);
+  } else {
+    sel_row_topk_kernel<<<dim3(N, BH), 256, 0, st>>>(pr, N, g.K, g.mode == VSA2_PER_QUERY_BUDGET ? budgets : nullptr,
+                                                     s.row_tau, s.row_eq_take, s.row_cnt);
+  }
+  sel_scan_rows_kernel<<<BH, 1024, 0, st>>>(N, g.mode == VSA2_PER_SEQUENCE, s.state, s.row_gt, s.row_eq, s.row_tau,
+                                            s.row_eq_take, s.row_cnt, row_ptr, g.nnz_cap, status);
+  sel_emit_rows_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(pr, N, s.words, s.row_tau, s.row_eq_take, row_ptr,
+                                                              col_idx, s.bitmap, g.nnz_cap);
+  // the column counts reuse row_gt as scratch
+  sel_col_count_kernel<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(s.bitmap, N, s.words, s.row_gt);
+  sel_scan_cols_kernel<<<BH, 1024, 0, st>>>(N, s.row_gt, col_ptr);
+  sel_emit_cols_kernel<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(s.bitmap, N, s.words, col_ptr, row_idx, g.nnz_cap);
+  return cudaGetLastError();
+}
+
+}  // namespace vsa2

@@ -1,0 +1,153 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vsa2_oracle as orc
+from paper_2609_32882_b200 import binding as vb
+from paper_2609_32882_b200 import inputs as syn
+from vsa2_testlib import (GpuRun, assert_close, assert_lse_close, check_routing, dev_bf16, oracle_arrays, to_f64)
+
+pytestmark = pytest.mark.gpu
+
+# small workloads that span several tiles, a ragged (padded) grid and GQA
+MINI_PADDED = syn.Workload("mini_padded_gqa", 1, 4, 2, 128, (5, 6, 9), select_mode=syn.PER_QUERY, topk=3, seed=21)
+MINI_SEQ = syn.Workload("mini_per_sequence", 2, 3, 3, 64, (6, 9, 10), select_mode=syn.PER_SEQUENCE, topk=4, seed=22)
+MINI_BUDGET = syn.Workload("mini_budget", 1, 2, 1, 128, (8, 8, 12), select_mode=syn.PER_QUERY_BUDGET, seed=23)
+
+
+def full_parity(wl, data, out_dtype=vb.BF16, nnz_cap=0, check_route=True):
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    run = GpuRun(wl, data, out_dtype=out_dtype, nnz_cap=nnz_cap)
+    a = oracle_arrays(data)
+    gmask = run.route()
+    if check_route:
+        omask, P_r = orc.route(a["q"], a["k"], geo, scale, wl.select_mode, wl.topk, data.get("budgets"), return_scores=True)
+        for b in range(wl.batch):
+            for h in range(wl.heads_q):
+                check_routing(gmask[b, h], omask[b, h], P_r[b, h], wl.select_mode)
+        # the GPU's own block scores
+        pr_gpu = to_f64(run.attn.scores())
+        assert np.abs(pr_gpu - P_r).max() <= 1e-4 * P_r.max()
+    # attention parity for the GPU's map
+    O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale)
+    O, lse = run.forward()
+    assert_close("O", O, O_ref)
+    assert_lse_close(lse, lse_ref)
+    dQ_ref, dK_ref, dV_ref, dG_ref = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
+    dQ, dK, dV, dG = run.backward()
+    assert_close("dQ", dQ, dQ_ref)
+    assert_close("dK", dK, dK_ref)
+    assert_close("dV", dV, dV_ref)
+    assert_close("dGate", dG, dG_ref, tol_abs=5e-2)
+    return run
+
+
+def test_config0_tiny_full_parity():
+    wl = syn.CONFIGS[0]
+    full_parity(wl, syn.make_inputs(wl))
+
+
+def test_config0_fp32_outputs():
+    wl = syn.CONFIGS[0]
+    full_parity(wl, syn.make_inputs(wl), out_dtype=vb.F32, check_route=False)
+
+
+def test_config1_small_video_full_parity():
+    wl = syn.CONFIGS[1]
+    full_parity(wl, syn.make_inputs(wl))
+
+
+def test_padded_grid_gqa_full_parity():
+    full_parity(MINI_PADDED, syn.make_inputs(MINI_PADDED))
+
+
+def test_per_sequence_batch2_d64_full_parity():
+    run = full_parity(MINI_SEQ, syn.make_inputs(MINI_SEQ))
+    rows = run.mask.sum(axis=-1)
+    assert (run.mask.sum(axis=(-1, -2)) == run.N * 4).all()          # exactly N*K per (batch, head)
+    assert rows.min() != rows.max()                                    # per-sequence TopK gives variable rows
+
+
+def test_per_query_budget_full_parity():
+    wl = MINI_BUDGET
+    data = syn.make_inputs(wl)
+    N = wl.n_cubes
+    rng = np.random.default_rng(5)
+    data["budgets"] = rng.integers(0, N + 3, size=(1, 2, N), dtype=np.int32)   # includes 0 (empty rows) and > N
+    cap = int(np.minimum(data["budgets"], N).sum(axis=-1).max())
+    run = full_parity(wl, data, nnz_cap=cap)
+    assert np.array_equal(run.mask.sum(axis=-1), np.minimum(data["budgets"], N))
+
+
+def test_all_blocks_kept_equals_dense_attention():
+    wl = syn.CONFIGS[1].replace(heads_q=2, heads_kv=2, select_mode=syn.PER_SEQUENCE, topk=32)
+    data = syn.make_inputs(wl)
+    run = GpuRun(wl, data, flags=vb.FLAG_NO_COARSE)
+    assert run.route().all()
+    O, lse = run.forward()
+    q, k, v = (t.float() for t in (run.q, run.k, run.v))
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v)
+    assert_close("O vs dense SDPA", O, to_f64(ref))
+
+
+def test_gate_none_and_no_coarse_flag_give_fine_only():
+    wl = MINI_PADDED
+    data = syn.make_inputs(wl)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    a = oracle_arrays(data)
+    run = GpuRun(wl, data, flags=vb.FLAG_NO_COARSE)
+    gmask = run.route()
+    O, lse = run.forward()
+    zero = np.zeros_like(a["gate"])
+    O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], zero, gmask, geo, 1 / np.sqrt(wl.head_dim))
+    assert_close("O_f", O, O_ref)
+    dQ, dK, dV, dG = run.backward()
+    dQ_ref, dK_ref, dV_ref, _ = orc.backward(a["q"], a["k"], a["v"], zero, gmask, geo, 1 / np.sqrt(wl.head_dim), a["do"])
+    assert_close("dQ", dQ, dQ_ref)
+    assert_close("dK", dK, dK_ref)
+    assert_close("dV", dV, dV_ref)
+    assert (dG == 0).all()
+
+
+def test_results_are_bitwise_reproducible():
+    wl = MINI_PADDED
+    data = syn.make_inputs(wl)
+    outs = []
+    for _ in range(2):
+        run = GpuRun(wl, data)
+        run.route()
+        run.forward()
+        run.backward()
+        outs.append([t.clone() for t in (run.o, run.lse, run.dq, run.dk, run.dv, run.dgate, run.attn.col_idx, run.attn.row_idx)])
+    for x, y in zip(*outs):
+        assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
+
+
+def test_router_pool_is_bit_exact():
+    """Q_r of the GPU equals the oracle's bf16 pooled operands bit for bit (same summation order)."""
+    wl = MINI_PADDED
+    data = syn.make_inputs(wl)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    run = GpuRun(wl, data)
+    run.route()
+    s = run.attn.sizes
+    n = wl.batch * wl.heads_q * s.n_cubes * s.n_subcubes * wl.head_dim
+    qr = run.attn.ws_route[256:256 + 2 * n].view(torch.bfloat16).view(wl.batch, wl.heads_q, s.n_cubes, s.n_subcubes, wl.head_dim)
+    for h in range(wl.heads_q):
+        ref, valid = orc.mean_pool_router(orc.bf16_bits_to_f64(data["q"][0, h]), geo)
+        got = to_f64(qr[0, h])
+        assert np.array_equal(got[valid], ref[valid])
+
+
+def test_bad_arguments_are_rejected_on_the_gpu_box_too():
+    wl = syn.CONFIGS[0]
+    data = syn.make_inputs(wl)
+    run = GpuRun(wl, data)
+    with pytest.raises(vb.Vsa2Error) as e:
+        vb.vsa2_route(run.p, run.q, run.k, None, run.attn.map, run.attn.ws_route, workspace_bytes=1024)
+    assert e.value.code == vb.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(vb.Vsa2Error) as e:
+        vb.vsa2_route(run.p, run.q.data_ptr() + 2, run.k, None, run.attn.map, run.attn.ws_route)
+    assert e.value.code == vb.ERR_MISALIGNED

@@ -1,0 +1,110 @@
+"""CPU-only checks of the C ABI: the library builds and loads, exports every symbol the header
+declares, and its host-side argument logic behaves as documented (no kernel is launched here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_32882_b200 import binding as vb
+from paper_2609_32882_b200 import build as vbuild
+from paper_2609_32882_b200 import inputs as syn
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    vbuild.build_library()
+    return ctypes.CDLL(vb.LIB_PATH)
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "vsa2.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vsa2_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_functions_are_exported(lib):
+    names = declared_functions()
+    assert {"vsa2_query_sizes", "vsa2_route", "vsa2_attn_fwd", "vsa2_attn_bwd", "vsa2_device_status",
+            "vsa2_strerror"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/vsa2.h but not exported"
+    for n in vb.EXPORTS:
+        assert n in names
+
+
+def test_query_sizes_matches_the_geometry_of_the_five_configs():
+    expect = {0: (4, 256, 2), 1: (32, 2048, 8), 2: (624, 32760, 78), 3: (1440, 75600, 64)}
+    for c, (N, L, K) in expect.items():
+        wl = syn.CONFIGS[c]
+        s = vb.vsa2_query_sizes(vb.params_from_workload(wl))
+        assert (s.n_cubes, s.seq_len, s.topk_eff, s.n_subcubes, s.block_tokens) == (N, L, K, 8, 64)
+        assert s.nnz_cap == N * K
+        assert s.ptr_elems == wl.batch * wl.heads_q * (N + 1)
+        assert s.idx_elems == wl.batch * wl.heads_q * N * K
+        assert s.pooled_q_elems == wl.batch * wl.heads_q * N * wl.head_dim
+        assert s.pooled_kv_elems == wl.batch * wl.heads_kv * N * wl.head_dim
+        assert s.route_workspace_bytes > wl.batch * wl.heads_q * N * N * 4
+        assert s.route_workspace_bytes % 256 == 0 and s.bwd_workspace_bytes % 256 == 0
+
+
+def test_topk_is_clamped_and_keep_fraction_is_honoured():
+    wl = syn.CONFIGS[1]
+    assert vb.vsa2_query_sizes(vb.params_from_workload(wl, topk=1000)).topk_eff == 32
+    s = vb.vsa2_query_sizes(vb.params_from_workload(wl, topk=0, keep_fraction=0.125))
+    assert s.topk_eff == 4
+    assert vb.vsa2_query_sizes(vb.params_from_workload(wl, topk=0, keep_fraction=0.001)).topk_eff == 1
+    s = vb.vsa2_query_sizes(vb.params_from_workload(syn.CONFIGS[2], topk=0, keep_fraction=0.125))
+    assert s.topk_eff == 78                                     # 87.5 % block sparsity of 624 cubes
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(heads_kv=5), vb.ERR_INVALID_ARG),                       # heads_q % heads_kv
+    (dict(head_dim=96), vb.ERR_UNSUPPORTED),
+    (dict(cube=(4, 4, 8)), vb.ERR_UNSUPPORTED),                   # B = 128 not built yet
+    (dict(rpool=(3, 2, 2)), vb.ERR_INVALID_ARG),                  # must divide the cube
+    (dict(select_mode=7), vb.ERR_INVALID_ARG),
+    (dict(topk=0, keep_fraction=0.0), vb.ERR_INVALID_ARG),
+    (dict(topk=-1), vb.ERR_INVALID_ARG),
+    (dict(grid=(0, 4, 4)), vb.ERR_INVALID_ARG),
+    (dict(out_dtype=3), vb.ERR_INVALID_ARG),
+    (dict(select_mode=vb.PER_QUERY_BUDGET, nnz_cap=0), vb.ERR_INVALID_ARG),
+])
+def test_bad_params_are_rejected(kw, code):
+    base = dict(batch=1, heads_q=12, heads_kv=12, head_dim=128, grid=(8, 16, 16), topk=8)
+    base.update(kw)
+    with pytest.raises(vb.Vsa2Error) as e:
+        vb.vsa2_query_sizes(vb.make_params(**base))
+    assert e.value.code == code
+
+
+def test_null_pointers_are_rejected_before_any_cuda_call(lib):
+    p = vb.params_from_workload(syn.CONFIGS[0])
+    m = vb.Map(0, 0, 0, 0)
+    rc = vb._lib().vsa2_route(ctypes.byref(p), None, None, None, ctypes.byref(m), None, 0, None)
+    assert rc == vb.ERR_INVALID_ARG
+    rc = vb._lib().vsa2_attn_fwd(ctypes.byref(p), None, None, None, None, ctypes.byref(m), None, None, None, None, 0, None)
+    assert rc == vb.ERR_INVALID_ARG
+    rc = vb._lib().vsa2_attn_bwd(ctypes.byref(p), None, None, None, None, ctypes.byref(m), None, None, None, None,
+                                 None, None, None, None, None, 0, None)
+    assert rc == vb.ERR_INVALID_ARG
+    assert vb._lib().vsa2_device_status(None, None, None) == vb.ERR_INVALID_ARG
+    assert vb._lib().vsa2_query_sizes(None, None) == vb.ERR_INVALID_ARG
+
+
+def test_strerror_covers_every_code():
+    seen = set()
+    for code in range(0, -8, -1):
+        msg = vb._lib().vsa2_strerror(code).decode()
+        assert msg and "unknown" not in msg
+        seen.add(msg)
+    assert len(seen) == 8
+    assert "unknown" in vb._lib().vsa2_strerror(-99).decode()
+
+
+def test_binding_refuses_host_tensors():
+    import torch
+    with pytest.raises(ValueError):
+        vb._ptr(torch.zeros(4))

@@ -1,0 +1,124 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C ABI, run the oracle
+on the same seeded inputs, compare with the tolerances the build's target states.
+
+Tolerances (fp32 comparison against the fp64 oracle):
+  outputs and gradients: max abs err <= 2e-2 and mean rel err <= 5e-3, where
+                         mean rel err = mean|a - b| / mean|b| over the tensor;
+  lse:                   max abs err <= 1e-3 where finite, -inf must match -inf;
+  routing:               the map must equal the oracle's except at entries whose oracle score lies
+                         within 1e-3 * tau (relative) of the threshold tau = smallest kept score of
+                         that (batch, head) [per-sequence] or row [per-query]; counts must be exact.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import vsa2_oracle as orc
+from paper_2609_32882_b200 import binding as vb
+from paper_2609_32882_b200 import inputs as syn
+
+TOL_ABS, TOL_REL, TOL_LSE, TOL_ROUTE = 2e-2, 5e-3, 1e-3, 1e-3
+
+
+def dev_bf16(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def err(a: np.ndarray, b: np.ndarray):
+    """(max abs err, mean rel err) of a against the reference b."""
+    d = np.abs(a - b)
+    return float(d.max()) if d.size else 0.0, float(d.mean() / max(np.abs(b).mean(), 1e-30)) if d.size else 0.0
+
+
+def assert_close(name, a, b, tol_abs=TOL_ABS, tol_rel=TOL_REL):
+    mx, rel = err(a, b)
+    assert mx <= tol_abs and rel <= tol_rel, f"{name}: max abs err {mx:.3e} (tol {tol_abs}), mean rel err {rel:.3e} (tol {tol_rel})"
+    return mx, rel
+
+
+def assert_lse_close(a, b):
+    fin = np.isfinite(b)
+    assert np.array_equal(np.isneginf(a), np.isneginf(b)), "lse: -inf pattern differs"
+    if fin.any():
+        mx = float(np.abs(a[fin] - b[fin]).max())
+        assert mx <= TOL_LSE, f"lse: max abs err {mx:.3e}"
+
+
+def csr_to_mask(row_ptr, col_idx, N):
+    """row_ptr [..., N+1], col_idx [..., cap] (numpy) -> bool [..., N, N]; also checks ordering."""
+    lead = row_ptr.shape[:-1]
+    rp = row_ptr.reshape(-1, N + 1)
+    ci = col_idx.reshape(rp.shape[0], -1)
+    mask = np.zeros((rp.shape[0], N, N), dtype=bool)
+    for h in range(rp.shape[0]):
+        assert rp[h, 0] == 0 and np.all(np.diff(rp[h]) >= 0)
+        for i in range(N):
+            cols = ci[h, rp[h, i]:rp[h, i + 1]]
+            if cols.size:
+                assert np.all(np.diff(cols) > 0), "indices not strictly ascending"
+                assert cols[0] >= 0 and cols[-1] < N
+            mask[h, i, cols] = True
+    return mask.reshape(lead + (N, N))
+
+
+def check_routing(gpu_mask, oracle_mask, P_r, mode):
+    """T1 rule on one (batch, head): gpu_mask, oracle_mask bool [N, N], P_r oracle scores."""
+    N = P_r.shape[0]
+    p32 = P_r.astype(np.float32).astype(np.float64)
+    diff = gpu_mask != oracle_mask
+    if mode == orc.PER_SEQUENCE:
+        assert gpu_mask.sum() == oracle_mask.sum()
+        if diff.any():
+            tau = p32[oracle_mask].min()
+            assert np.all(np.abs(p32[diff] - tau) <= TOL_ROUTE * tau), "routing differs away from the threshold"
+    else:
+        assert np.array_equal(gpu_mask.sum(axis=1), oracle_mask.sum(axis=1))
+        for i in np.nonzero(diff.any(axis=1))[0]:
+            tau = p32[i][oracle_mask[i]].min()
+            assert np.all(np.abs(p32[i][diff[i]] - tau) <= TOL_ROUTE * tau), "routing differs away from the row threshold"
+    return int(diff.sum())
+
+
+class GpuRun:
+    """Uploads a workload's tensors and drives the library through the binding."""
+
+    def __init__(self, wl, data, out_dtype=vb.BF16, flags=0, nnz_cap=0, **param_overrides):
+        self.wl = wl
+        self.p = vb.params_from_workload(wl, out_dtype=out_dtype, flags=flags, nnz_cap=nnz_cap, **param_overrides)
+        self.attn = vb.Vsa2Attention(self.p)
+        self.q, self.k, self.v = dev_bf16(data["q"]), dev_bf16(data["k"]), dev_bf16(data["v"])
+        self.gate = torch.from_numpy(data["gate"]).cuda()
+        self.do = dev_bf16(data["do"]) if "do" in data else None
+        self.budgets = torch.from_numpy(data["budgets"]).cuda() if "budgets" in data else None
+        self.N = self.attn.sizes.n_cubes
+
+    def route(self):
+        self.attn.route(self.q, self.k, self.budgets)
+        self.attn.check_status()
+        rp, ci, cp, ri = (t.cpu().numpy() for t in self.attn.map_views())
+        self.mask = csr_to_mask(rp, ci, self.N)
+        mask_t = csr_to_mask(cp, ri, self.N)
+        assert np.array_equal(self.mask, np.swapaxes(mask_t, -1, -2)), "CSR and CSC disagree"
+        assert np.array_equal(rp[..., -1], cp[..., -1])
+        return self.mask
+
+    def forward(self):
+        self.o, self.lse = self.attn.forward(self.q, self.k, self.v, self.gate)
+        self.attn.check_status()
+        return to_f64(self.o), to_f64(self.lse)
+
+    def backward(self):
+        self.dq, self.dk, self.dv, self.dgate = self.attn.backward(self.q, self.k, self.v, self.gate, self.o, self.lse, self.do)
+        self.attn.check_status()
+        return tuple(to_f64(t) for t in (self.dq, self.dk, self.dv, self.dgate))
+
+
+def oracle_arrays(data):
+    out = {k: orc.bf16_bits_to_f64(data[k]) for k in ("q", "k", "v", "do") if k in data}
+    out["gate"] = data["gate"].astype(np.float64)
+    return out
