@@ -86,6 +86,7 @@ typedef struct vsa2_sizes {
   int64_t pooled_q_elems;     /* float elements of saved.qc and saved.oc_hat: batch*heads_q*N*D */
   int64_t pooled_kv_elems;    /* float elements of saved.kc and of saved.vc: batch*heads_kv*N*D */
   int64_t lse_c_elems;        /* float elements of saved.lse_c: batch*heads_q*N */
+  int64_t o_res_elems;        /* bf16 elements of saved.o_res: batch*heads_q*L*D (0 when out_dtype is fp32) */
   size_t  route_workspace_bytes;
   size_t  fwd_workspace_bytes;
   size_t  bwd_workspace_bytes;
@@ -109,6 +110,10 @@ typedef struct vsa2_saved {
   float* vc;       /* [batch, heads_kv, N, D] */
   float* oc_hat;   /* [batch, heads_q,  N, D]  Eq. 3 */
   float* lse_c;    /* [batch, heads_q,  N]     log-sum-exp of the coarse scores */
+  void*  o_res;    /* bf16 [batch, heads_q, L, D], optional (may be NULL), used only when out_dtype is bf16:
+                      the rounding residual bf16(O_fp32 - O_bf16) of the forward output.  The backward adds it
+                      back to O when it forms delta = rowsum(dO * O_f), which removes the bf16 storage noise of O
+                      from dQ and dK. */
 } vsa2_saved;
 
 /* Validates `p` and fills `out`.  Pure host arithmetic; no CUDA call. */

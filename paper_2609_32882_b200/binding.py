@@ -48,7 +48,7 @@ class Sizes(C.Structure):
     _fields_ = [("n_cubes", C.c_int32), ("n_subcubes", C.c_int32), ("block_tokens", C.c_int32),
                 ("topk_eff", C.c_int32), ("seq_len", C.c_int64), ("nnz_cap", C.c_int64),
                 ("ptr_elems", C.c_int64), ("idx_elems", C.c_int64), ("pooled_q_elems", C.c_int64),
-                ("pooled_kv_elems", C.c_int64), ("lse_c_elems", C.c_int64),
+                ("pooled_kv_elems", C.c_int64), ("lse_c_elems", C.c_int64), ("o_res_elems", C.c_int64),
                 ("route_workspace_bytes", C.c_size_t), ("fwd_workspace_bytes", C.c_size_t),
                 ("bwd_workspace_bytes", C.c_size_t)]
 
@@ -59,7 +59,7 @@ class Map(C.Structure):
 
 class Saved(C.Structure):
     _fields_ = [("qc", C.c_void_p), ("kc", C.c_void_p), ("vc", C.c_void_p), ("oc_hat", C.c_void_p),
-                ("lse_c", C.c_void_p)]
+                ("lse_c", C.c_void_p), ("o_res", C.c_void_p)]
 
 
 _LIB = None
@@ -195,8 +195,9 @@ class Vsa2Attention:
         self.vc = torch.empty(s.pooled_kv_elems, **f32)
         self.oc_hat = torch.empty(s.pooled_q_elems, **f32)
         self.lse_c = torch.empty(s.lse_c_elems, **f32)
+        self.o_res = torch.empty(s.o_res_elems, dtype=torch.bfloat16, device=dev) if s.o_res_elems else None
         self.saved = Saved(self.qc.data_ptr(), self.kc.data_ptr(), self.vc.data_ptr(), self.oc_hat.data_ptr(),
-                           self.lse_c.data_ptr())
+                           self.lse_c.data_ptr(), self.o_res.data_ptr() if s.o_res_elems else None)
         u8 = dict(dtype=torch.uint8, device=dev)
         self.ws_route = torch.empty(s.route_workspace_bytes, **u8)
         self.ws_fwd = torch.empty(s.fwd_workspace_bytes, **u8)

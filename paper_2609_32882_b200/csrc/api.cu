@@ -153,6 +153,7 @@ int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
   out->pooled_q_elems = BHq * g.N * g.D;
   out->pooled_kv_elems = BHk * g.N * g.D;
   out->lse_c_elems = BHq * g.N;
+  out->o_res_elems = g.out_f32 ? 0 : BHq * (long long)g.L * g.D;
   out->route_workspace_bytes = route_layout(g).total;
   out->fwd_workspace_bytes = fwd_workspace_bytes(g);
   out->bwd_workspace_bytes = bwd_layout(g).total;
@@ -225,8 +226,10 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
     VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
   }
+  bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
+  if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
   VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
-                            coarse ? saved->oc_hat : nullptr, o, lse, st));
+                            coarse ? saved->oc_hat : nullptr, o, o_res, lse, st));
   return VSA2_OK;
 }
 
@@ -262,7 +265,8 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   float* dvc = at<float>(workspace, lay.dvc);
   if (!coarse && dgate != nullptr)
     VSA2_CUDA(cudaMemsetAsync(dgate, 0, (size_t)g.batch * g.Hq * g.L * sizeof(float), st));
-  VSA2_CUDA(launch_bwd_preprocess(g, dob, o, coarse ? gate : nullptr, coarse ? saved->oc_hat : nullptr, delta,
+  const bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<const bf16*>(saved->o_res) : nullptr;
+  VSA2_CUDA(launch_bwd_preprocess(g, dob, o, o_res, coarse ? gate : nullptr, coarse ? saved->oc_hat : nullptr, delta,
                                   coarse ? dgate : nullptr, d_oc_hat, st));
   if (coarse)
     VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,

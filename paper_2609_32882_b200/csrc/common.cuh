@@ -126,10 +126,10 @@ cudaError_t launch_coarse_bwd(const Geo& g, const float* qc, const float* kc, co
                               float* dvc, cudaStream_t st);
 
 cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
-                            const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, float* lse,
-                            cudaStream_t st);
+                            const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                            float* lse, cudaStream_t st);
 
-cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const float* gate,
+cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,
                                   const float* oc_hat, float* delta, float* dgate, float* d_oc_hat,
                                   cudaStream_t st);
 cudaError_t launch_fine_bwd_dq(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,

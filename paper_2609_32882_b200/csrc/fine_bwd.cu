@@ -16,6 +16,7 @@ namespace vsa2 {
 // ------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restrict__ d_o, const void* __restrict__ o,
+                                                             const bf16* __restrict__ o_res,
                                                              const float* __restrict__ gate,
                                                              const float* __restrict__ oc_hat, Geo g,
                                                              float* __restrict__ delta, float* __restrict__ dgate,
@@ -38,7 +39,9 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restr
     if (l >= 0) {
       size_t idx = (bhq * g.L + l) * D + d;
       dov = __bfloat162float(d_o[idx]);
-      s_oo = fmaf(dov, load_out(o, idx, g.out_f32), s_oo);
+      float ov = load_out(o, idx, g.out_f32);
+      if (o_res != nullptr) ov += __bfloat162float(o_res[idx]);
+      s_oo = fmaf(dov, ov, s_oo);
       if (coarse) s_oc = fmaf(dov, oc[d], s_oc);
     }
     gdo[r][d] = gt * dov;
@@ -62,11 +65,11 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restr
   }
 }
 
-cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const float* gate,
+cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,
                                   const float* oc_hat, float* delta, float* dgate, float* d_oc_hat, cudaStream_t st) {
   dim3 grid(g.N, g.Hq, g.batch);
-  if (g.D == 128) bwd_preprocess_kernel<128><<<grid, 256, 0, st>>>(d_o, o, gate, oc_hat, g, delta, dgate, d_oc_hat);
-  else bwd_preprocess_kernel<64><<<grid, 256, 0, st>>>(d_o, o, gate, oc_hat, g, delta, dgate, d_oc_hat);
+  if (g.D == 128) bwd_preprocess_kernel<128><<<grid, 256, 0, st>>>(d_o, o, o_res, gate, oc_hat, g, delta, dgate, d_oc_hat);
+  else bwd_preprocess_kernel<64><<<grid, 256, 0, st>>>(d_o, o, o_res, gate, oc_hat, g, delta, dgate, d_oc_hat);
   return cudaGetLastError();
 }
 

@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ 
                                                        const bf16* __restrict__ v, const float* __restrict__ gate,
                                                        const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                                                        const float* __restrict__ oc_hat, Geo g, void* __restrict__ o,
-                                                       float* __restrict__ lse) {
+                                                       bf16* __restrict__ o_res, float* __restrict__ lse) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   using SM = FineFwdSmem<D>;
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ 
         float p = __expf(x[c] - m_new);
         bf16 pb = __float2bfloat16_rn(p);
         P[r * SM::LDP + qd * 16 + c] = pb;
-        ps += __bfloat162float(pb);
+        ps += p;
       }
       ps += __shfl_xor_sync(0xffffffffu, ps, 1);
       ps += __shfl_xor_sync(0xffffffffu, ps, 2);
@@ -115,24 +115,29 @@ __global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ 
       float val = O[r * SM::LDO + d] * inv;
       if (coarse) val = fmaf(gt, oc[d], val);
       store_out(o, obase + d, val, g.out_f32);
+      if (o_res != nullptr) {
+        // what the bf16 rounding of O dropped, for the backward's delta
+        float rounded = __bfloat162float(__float2bfloat16_rn(val));
+        o_res[obase + d] = __float2bfloat16_rn(val - rounded);
+      }
     }
     if (qd == 0) lse[bhq * g.L + l] = denom > 0.f ? row_m[r] + __logf(denom) : -INFINITY;
   }
 }
 
 cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
-                            const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, float* lse,
-                            cudaStream_t st) {
+                            const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                            float* lse, cudaStream_t st) {
   dim3 grid(g.N, g.Hq, g.batch);
   cudaError_t e;
   if (g.D == 128) {
     size_t smb = FineFwdSmem<128>::bytes;
     if ((e = cudaFuncSetAttribute(fine_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    fine_fwd_kernel<128><<<grid, 256, smb, st>>>(q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, lse);
+    fine_fwd_kernel<128><<<grid, 256, smb, st>>>(q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
   } else {
     size_t smb = FineFwdSmem<64>::bytes;
     if ((e = cudaFuncSetAttribute(fine_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    fine_fwd_kernel<64><<<grid, 256, smb, st>>>(q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, lse);
+    fine_fwd_kernel<64><<<grid, 256, smb, st>>>(q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
   }
   return cudaGetLastError();
 }
