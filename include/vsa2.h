@@ -160,6 +160,30 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
  * *status_out (host): VSA2_OK, VSA2_ERR_DEVICE_TIMEOUT or VSA2_ERR_MAP_OVERFLOW. */
 int vsa2_device_status(const void* workspace, void* cuda_stream, int32_t* status_out);
 
+/* Kernel groups, for timing from outside (e.g. a benchmark) without a profiler. */
+enum {
+  VSA2_KERNEL_POOL = 0,         /* mean pooling (Eq. 1, Eq. 5) */
+  VSA2_KERNEL_ROUTER_LSE = 1,   /* router pass 1: row log-sum-exp (Eq. 6) */
+  VSA2_KERNEL_ROUTER_POOL = 2,  /* router pass 2: softmax + G x G pooling (Eq. 6-7) */
+  VSA2_KERNEL_SELECT = 3,       /* TopK + CSR/CSC (Eq. 8-9) */
+  VSA2_KERNEL_COARSE_FWD = 4,   /* Eq. 2-3 */
+  VSA2_KERNEL_FINE_FWD = 5,     /* Eq. 12 + Eq. 14 */
+  VSA2_KERNEL_BWD_PRE = 6,      /* delta, dGate, dO_c_hat */
+  VSA2_KERNEL_COARSE_BWD = 7,
+  VSA2_KERNEL_FINE_BWD_DQ = 8,
+  VSA2_KERNEL_FINE_BWD_DKV = 9,
+  VSA2_KERNEL_COUNT = 10
+};
+
+/* Asks the library to record `start_event` before and `stop_event` after the launches of one kernel
+ * group (cudaEvent_t handles passed as void*, recorded on the stream of the call that launches them) in
+ * every later call, until cleared by passing NULL events.  The paper has no counterpart: this is a
+ * measurement hook.  Process-global and not thread-safe. */
+int vsa2_profile_events(int32_t kernel_id, void* start_event, void* stop_event);
+
+/* Number of kernels this library has launched in this process so far. */
+int64_t vsa2_launch_count(void);
+
 /* Static string for an error code. */
 const char* vsa2_strerror(int code);
 

@@ -24,7 +24,10 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, 
 ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_MAP_OVERFLOW = -5, -6, -7
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
-           "vsa2_device_status", "vsa2_strerror")
+           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count")
+
+KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
+           "fine_bwd_dq", "fine_bwd_dkv")
 
 
 class Vsa2Error(RuntimeError):
@@ -84,8 +87,11 @@ def _lib():
         lib.vsa2_device_status.argtypes = [vp, vp, i32p]
         lib.vsa2_strerror.argtypes = [C.c_int]
         lib.vsa2_strerror.restype = C.c_char_p
+        lib.vsa2_profile_events.argtypes = [C.c_int32, vp, vp]
+        lib.vsa2_launch_count.argtypes = []
+        lib.vsa2_launch_count.restype = C.c_int64
         for name in EXPORTS:
-            if name not in ("vsa2_strerror", "vsa2_route_scores"):
+            if name not in ("vsa2_strerror", "vsa2_route_scores", "vsa2_launch_count"):
                 getattr(lib, name).restype = C.c_int
         _LIB = lib
     return _LIB
@@ -162,6 +168,17 @@ def vsa2_attn_bwd(p, q, k, v, gate, vmap: Map, o, lse, saved, d_o, dq, dk, dv, d
     _check(_lib().vsa2_attn_bwd(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate), C.byref(vmap), _ptr(o), _ptr(lse),
                                 C.byref(saved) if saved is not None else None, _ptr(d_o), _ptr(dq), _ptr(dk),
                                 _ptr(dv), _ptr(dgate), _ptr(workspace), nbytes, _stream(stream)), "vsa2_attn_bwd")
+
+
+def vsa2_profile_events(kernel_id: int, start_event, stop_event):
+    """start/stop: torch.cuda.Event objects (already recorded once, so that their handles exist) or None."""
+    a = None if start_event is None else start_event.cuda_event
+    b = None if stop_event is None else stop_event.cuda_event
+    _check(_lib().vsa2_profile_events(kernel_id, a, b), "vsa2_profile_events")
+
+
+def vsa2_launch_count() -> int:
+    return int(_lib().vsa2_launch_count())
 
 
 def vsa2_device_status(workspace, stream=None) -> int:

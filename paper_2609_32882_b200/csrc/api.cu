@@ -8,6 +8,10 @@ using namespace vsa2;
 
 namespace {
 
+cudaEvent_t g_prof_start[VSA2_KERNEL_COUNT];
+cudaEvent_t g_prof_stop[VSA2_KERNEL_COUNT];
+long long g_launches = 0;
+
 struct RouteLayout {
   size_t status, qr, kr, lse_r, pr, hist, state, row_tau, row_eq_take, row_cnt, row_gt, row_eq, bitmap, total;
   int words;
@@ -133,7 +137,26 @@ T* at(void* ws, size_t off) { return reinterpret_cast<T*>(reinterpret_cast<unsig
 
 }  // namespace
 
+namespace vsa2 {
+ProfScope::ProfScope(int kernel_id, cudaStream_t stream, int launches) : id(kernel_id), st(stream) {
+  g_launches += launches;
+  if (g_prof_start[id] != nullptr) cudaEventRecord(g_prof_start[id], st);
+}
+ProfScope::~ProfScope() {
+  if (g_prof_stop[id] != nullptr) cudaEventRecord(g_prof_stop[id], st);
+}
+}  // namespace vsa2
+
 extern "C" {
+
+int vsa2_profile_events(int32_t kernel_id, void* start_event, void* stop_event) {
+  if (kernel_id < 0 || kernel_id >= VSA2_KERNEL_COUNT) return VSA2_ERR_INVALID_ARG;
+  g_prof_start[kernel_id] = reinterpret_cast<cudaEvent_t>(start_event);
+  g_prof_stop[kernel_id] = reinterpret_cast<cudaEvent_t>(stop_event);
+  return VSA2_OK;
+}
+
+int64_t vsa2_launch_count(void) { return g_launches; }
 
 int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
   if (out == nullptr) return VSA2_ERR_INVALID_ARG;
@@ -177,8 +200,11 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
   VSA2_CUDA(cudaMemsetAsync(status, 0, sizeof(StatusBlock), st));
   bf16* qr = at<bf16>(workspace, lay.qr);
   bf16* kr = at<bf16>(workspace, lay.kr);
-  VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(q), g.Hq, qr, nullptr, st));
-  VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(k), g.Hkv, kr, nullptr, st));
+  {
+    ProfScope ps(VSA2_KERNEL_POOL, st, 2);
+    VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(q), g.Hq, qr, nullptr, st));
+    VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(k), g.Hkv, kr, nullptr, st));
+  }
   float* pr = at<float>(workspace, lay.pr);
   VSA2_CUDA(launch_router_scores(g, qr, kr, at<float>(workspace, lay.lse_r), pr, st));
   SelectScratch s;
@@ -191,7 +217,10 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
   s.row_eq = at<int>(workspace, lay.row_eq);
   s.bitmap = at<unsigned>(workspace, lay.bitmap);
   s.words = lay.words;
-  VSA2_CUDA(launch_select(g, pr, budgets, s, map->row_ptr, map->col_idx, map->col_ptr, map->row_idx, status, st));
+  {
+    ProfScope ps(VSA2_KERNEL_SELECT, st, g.mode == VSA2_PER_SEQUENCE ? 13 : 6);
+    VSA2_CUDA(launch_select(g, pr, budgets, s, map->row_ptr, map->col_idx, map->col_ptr, map->row_idx, status, st));
+  }
   return VSA2_OK;
 }
 
@@ -221,15 +250,22 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
   const bf16* kb = reinterpret_cast<const bf16*>(k);
   const bf16* vb = reinterpret_cast<const bf16*>(v);
   if (coarse) {
-    VSA2_CUDA(launch_pool(g, qb, g.Hq, nullptr, saved->qc, st));
-    VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
-    VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
+    {
+      ProfScope ps(VSA2_KERNEL_POOL, st, 3);
+      VSA2_CUDA(launch_pool(g, qb, g.Hq, nullptr, saved->qc, st));
+      VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
+      VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
+    }
+    ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, 1);
     VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
   }
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
   if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
-  VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
-                            coarse ? saved->oc_hat : nullptr, o, o_res, lse, st));
+  {
+    ProfScope ps(VSA2_KERNEL_FINE_FWD, st, 1);
+    VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
+                              coarse ? saved->oc_hat : nullptr, o, o_res, lse, st));
+  }
   return VSA2_OK;
 }
 
@@ -266,15 +302,26 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   if (!coarse && dgate != nullptr)
     VSA2_CUDA(cudaMemsetAsync(dgate, 0, (size_t)g.batch * g.Hq * g.L * sizeof(float), st));
   const bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<const bf16*>(saved->o_res) : nullptr;
-  VSA2_CUDA(launch_bwd_preprocess(g, dob, o, o_res, coarse ? gate : nullptr, coarse ? saved->oc_hat : nullptr, delta,
-                                  coarse ? dgate : nullptr, d_oc_hat, st));
-  if (coarse)
+  {
+    ProfScope ps(VSA2_KERNEL_BWD_PRE, st, 1);
+    VSA2_CUDA(launch_bwd_preprocess(g, dob, o, o_res, coarse ? gate : nullptr, coarse ? saved->oc_hat : nullptr,
+                                    delta, coarse ? dgate : nullptr, d_oc_hat, st));
+  }
+  if (coarse) {
+    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, 2);
     VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
                                 at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
-  VSA2_CUDA(launch_fine_bwd_dq(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx, coarse ? dqc : nullptr, dq,
-                               st));
-  VSA2_CUDA(launch_fine_bwd_dkv(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx, coarse ? dkc : nullptr,
-                                coarse ? dvc : nullptr, dk, dv, st));
+  }
+  {
+    ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
+    VSA2_CUDA(launch_fine_bwd_dq(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx, coarse ? dqc : nullptr,
+                                 dq, st));
+  }
+  {
+    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
+    VSA2_CUDA(launch_fine_bwd_dkv(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx,
+                                  coarse ? dkc : nullptr, coarse ? dvc : nullptr, dk, dv, st));
+  }
   return VSA2_OK;
 }
 

@@ -34,6 +34,14 @@ struct StatusBlock {
   int pad[62];
 };
 
+// Brackets the launches of one kernel group: counts them and records the caller's timing events.
+struct ProfScope {
+  int id;
+  cudaStream_t st;
+  ProfScope(int kernel_id, cudaStream_t stream, int launches);
+  ~ProfScope();
+};
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // cube n -> (nt, nh, nw);  n = (nt*Nh + nh)*Nw + nw

@@ -128,13 +128,21 @@ cudaError_t launch_router_scores(const Geo& g, const bf16* qr, const bf16* kr, f
     size_t sm = RouterSmem<128>::bytes;
     if ((e = cudaFuncSetAttribute(router_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm))) return e;
     if ((e = cudaFuncSetAttribute(router_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm))) return e;
-    router_kernel<128, 1><<<grid, 256, sm, st>>>(qr, kr, g, lse_r, pr);
+    {
+      ProfScope ps(VSA2_KERNEL_ROUTER_LSE, st, 1);
+      router_kernel<128, 1><<<grid, 256, sm, st>>>(qr, kr, g, lse_r, pr);
+    }
+    ProfScope ps(VSA2_KERNEL_ROUTER_POOL, st, 1);
     router_kernel<128, 2><<<grid, 256, sm, st>>>(qr, kr, g, lse_r, pr);
   } else {
     size_t sm = RouterSmem<64>::bytes;
     if ((e = cudaFuncSetAttribute(router_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm))) return e;
     if ((e = cudaFuncSetAttribute(router_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm))) return e;
-    router_kernel<64, 1><<<grid, 256, sm, st>>>(qr, kr, g, lse_r, pr);
+    {
+      ProfScope ps(VSA2_KERNEL_ROUTER_LSE, st, 1);
+      router_kernel<64, 1><<<grid, 256, sm, st>>>(qr, kr, g, lse_r, pr);
+    }
+    ProfScope ps(VSA2_KERNEL_ROUTER_POOL, st, 1);
     router_kernel<64, 2><<<grid, 256, sm, st>>>(qr, kr, g, lse_r, pr);
   }
   return cudaGetLastError();
