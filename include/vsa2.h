@@ -184,6 +184,16 @@ int vsa2_profile_events(int32_t kernel_id, void* start_event, void* stop_event);
 /* Number of kernels this library has launched in this process so far. */
 int64_t vsa2_launch_count(void);
 
+/* Diagnostic: runs, in one CTA, the two tensor-core products the attention kernels are built from, on
+ * real cube tiles of batch 0 / head 0 fetched by TMA: S^T = K_pair Q^T (fp32 [128, 64]; K_pair = the 64-token
+ * tiles of cubes cube_a and cube_b stacked) and O^T = V_pair^T P^T (fp32 [128, 64]; rows are head channels, with
+ * head_dim 64 rows 64..127 repeat rows 0..63), where p_t is a bf16 [128, 64] matrix supplied by the caller.
+ * k_tile_dump receives the raw shared-memory image of the K pair (2 * head_dim/64 * 8 KB).  `status` is a device
+ * int32 set to VSA2_ERR_DEVICE_TIMEOUT if a bounded wait ran out.  The paper has no counterpart. */
+int vsa2_selftest_umma(const vsa2_params* p, const void* q, const void* k, const void* v, int32_t cube_q,
+                       int32_t cube_a, int32_t cube_b, const void* p_t, float* s_t_out, float* o_t_out,
+                       void* k_tile_dump, int32_t* status, void* cuda_stream);
+
 /* Static string for an error code. */
 const char* vsa2_strerror(int code);
 

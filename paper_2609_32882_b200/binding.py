@@ -24,7 +24,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, 
 ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_MAP_OVERFLOW = -5, -6, -7
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
-           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count")
+           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv")
@@ -88,6 +88,7 @@ def _lib():
         lib.vsa2_strerror.argtypes = [C.c_int]
         lib.vsa2_strerror.restype = C.c_char_p
         lib.vsa2_profile_events.argtypes = [C.c_int32, vp, vp]
+        lib.vsa2_selftest_umma.argtypes = [C.POINTER(Params), vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
         lib.vsa2_launch_count.argtypes = []
         lib.vsa2_launch_count.restype = C.c_int64
         for name in EXPORTS:
@@ -175,6 +176,12 @@ def vsa2_profile_events(kernel_id: int, start_event, stop_event):
     a = None if start_event is None else start_event.cuda_event
     b = None if stop_event is None else stop_event.cuda_event
     _check(_lib().vsa2_profile_events(kernel_id, a, b), "vsa2_profile_events")
+
+
+def vsa2_selftest_umma(p, q, k, v, cube_q, cube_a, cube_b, p_t, s_t_out, o_t_out, k_tile_dump, status, stream=None):
+    _check(_lib().vsa2_selftest_umma(C.byref(p), _ptr(q), _ptr(k), _ptr(v), cube_q, cube_a, cube_b, _ptr(p_t),
+                                     _ptr(s_t_out), _ptr(o_t_out), _ptr(k_tile_dump), _ptr(status), _stream(stream)),
+           "vsa2_selftest_umma")
 
 
 def vsa2_launch_count() -> int:
