@@ -55,7 +55,10 @@ enum { VSA2_PER_SEQUENCE = 0,         /* Eq. 8-9: the N*K largest entries of the
 
 enum { VSA2_BF16 = 0, VSA2_F32 = 1 };
 
-enum { VSA2_FLAG_NO_COARSE = 1 };     /* skip the coarse branch: O = O_f (the gate = 0 case, Sec. 2.3) */
+enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the gate = 0 case, Sec. 2.3) */
+       VSA2_FLAG_EXACT_MAX_FWD = 2 }; /* validation aid: run the whole fine forward with the slow kernel that tracks
+                                         the exact running row maximum (the tensor-core kernel falls back to it only
+                                         for query blocks whose softmax sums leave the safe range) */
 
 /* Problem statement (host struct). */
 typedef struct vsa2_params {

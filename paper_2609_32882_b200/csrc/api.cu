@@ -113,7 +113,7 @@ BwdLayout bwd_layout(const Geo& g) {
   return r;
 }
 
-size_t fwd_workspace_bytes(const Geo&) { return align_up(sizeof(StatusBlock), 256); }
+size_t fwd_workspace_bytes(const Geo&) { return align_up(fine_fwd_tc_workspace_bytes(), 256); }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -262,9 +262,14 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
   if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
   {
-    ProfScope ps(VSA2_KERNEL_FINE_FWD, st, 1);
-    VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
-                              coarse ? saved->oc_hat : nullptr, o, o_res, lse, st));
+    ProfScope ps(VSA2_KERNEL_FINE_FWD, st, (g.flags & VSA2_FLAG_EXACT_MAX_FWD) ? 1 : 2);
+    if (g.flags & VSA2_FLAG_EXACT_MAX_FWD)
+      VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
+                                coarse ? saved->oc_hat : nullptr, o, o_res, lse, st));
+    else
+      VSA2_CUDA(launch_fine_fwd_tc(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
+                                   coarse ? saved->oc_hat : nullptr, o, o_res, lse,
+                                   reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;
 }

@@ -137,6 +137,12 @@ cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf
                             const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                             float* lse, cudaStream_t st);
 
+// tensor-core forward (fine_fwd_tc.cu); `status` heads a workspace of fine_fwd_tc_workspace_bytes()
+size_t fine_fwd_tc_workspace_bytes();
+cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                               const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                               float* lse, StatusBlock* status, cudaStream_t st);
+
 cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,
                                   const float* oc_hat, float* delta, float* dgate, float* d_oc_hat,
                                   cudaStream_t st);

@@ -1,4 +1,4 @@
-// Fine branch forward (paper Eq. 12) with the gated merge (Eq. 14) in the epilogue:
+// Fine branch forward (paper Eq. 12) with the gated merge (Eq. 14) in the epilogue, exact-maximum version:
 // for query block i, token-level softmax attention over the valid tokens of the KV blocks
 // listed in row i of the CSR map; O = gate * O_c_hat[i] + O_f.  Online softmax in fp32,
 // bf16 tensor-core products with fp32 accumulation.
@@ -16,14 +16,14 @@ struct FineFwdSmem {
                                   64 * LDO * sizeof(float) + 3 * 64 * sizeof(float) + 64;
 };
 
-// grid (N, Hq, batch), 256 threads
+// One query block (i, hq, b) by a CTA of 256 threads: exact online softmax (running row maximum).
 template <int D>
-__global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ q, const bf16* __restrict__ k,
-                                                       const bf16* __restrict__ v, const float* __restrict__ gate,
-                                                       const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
-                                                       const float* __restrict__ oc_hat, Geo g, void* __restrict__ o,
-                                                       bf16* __restrict__ o_res, float* __restrict__ lse) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+__device__ __forceinline__ void fine_fwd_block(unsigned char* smem_raw, int i, int hq, int b,
+                                               const bf16* __restrict__ q, const bf16* __restrict__ k,
+                                               const bf16* __restrict__ v, const float* __restrict__ gate,
+                                               const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
+                                               const float* __restrict__ oc_hat, const Geo& g, void* __restrict__ o,
+                                               bf16* __restrict__ o_res, float* __restrict__ lse) {
   using SM = FineFwdSmem<D>;
   bf16* Qs = reinterpret_cast<bf16*>(smem_raw);
   bf16* Ks = Qs + 64 * SM::LDX;
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ 
   unsigned char* kvalid = reinterpret_cast<unsigned char*>(row_spare + 64);
   (void)row_spare;
 
-  const int i = blockIdx.x, hq = blockIdx.y, b = blockIdx.z, hk = hq / g.rep;
+  const int hk = hq / g.rep;
   const size_t bhq = (size_t)b * g.Hq + hq, bhk = (size_t)b * g.Hkv + hk;
   const bf16* qh = q + bhq * g.L * D;
   const bf16* kh = k + bhk * g.L * D;
@@ -123,6 +123,51 @@ __global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ 
     }
     if (qd == 0) lse[bhq * g.L + l] = denom > 0.f ? row_m[r] + __logf(denom) : -INFINITY;
   }
+}
+
+// grid (N, Hq, batch), 256 threads
+template <int D>
+__global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ q, const bf16* __restrict__ k,
+                                                       const bf16* __restrict__ v, const float* __restrict__ gate,
+                                                       const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
+                                                       const float* __restrict__ oc_hat, Geo g, void* __restrict__ o,
+                                                       bf16* __restrict__ o_res, float* __restrict__ lse) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  fine_fwd_block<D>(smem_raw, blockIdx.x, blockIdx.y, blockIdx.z, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
+}
+
+// Recomputes the query blocks listed in `items` (flat index (b*Hq + hq)*N + i; *count entries).
+template <int D>
+__global__ void __launch_bounds__(256) fine_fwd_list_kernel(const int* __restrict__ count, const int* __restrict__ items,
+                                                            const bf16* __restrict__ q, const bf16* __restrict__ k,
+                                                            const bf16* __restrict__ v, const float* __restrict__ gate,
+                                                            const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
+                                                            const float* __restrict__ oc_hat, Geo g, void* __restrict__ o,
+                                                            bf16* __restrict__ o_res, float* __restrict__ lse) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int n = *count;
+  for (int e = blockIdx.x; e < n; e += gridDim.x) {
+    int item = items[e];
+    int i = item % g.N, bh = item / g.N;
+    __syncthreads();
+    fine_fwd_block<D>(smem_raw, i, bh % g.Hq, bh / g.Hq, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
+  }
+}
+
+cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
+                                 const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
+                                 const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st) {
+  cudaError_t e;
+  if (g.D == 128) {
+    size_t smb = FineFwdSmem<128>::bytes;
+    if ((e = cudaFuncSetAttribute(fine_fwd_list_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_list_kernel<128><<<64, 256, smb, st>>>(count, items, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
+  } else {
+    size_t smb = FineFwdSmem<64>::bytes;
+    if ((e = cudaFuncSetAttribute(fine_fwd_list_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_list_kernel<64><<<64, 256, smb, st>>>(count, items, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
+  }
+  return cudaGetLastError();
 }
 
 cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,

@@ -5,6 +5,9 @@ Tolerances (fp32 comparison against the fp64 oracle):
   outputs and gradients: max abs err <= 2e-2 and mean rel err <= 5e-3, where
                          mean rel err = mean|a - b| / mean|b| over the tensor;
   lse:                   max abs err <= 1e-3 where finite, -inf must match -inf;
+                         When the library stores a tensor in bf16 (out_dtype BF16) the storage rounding,
+                         up to 2^-8 |x| per element (half an ulp at the bottom of a binade), comes on top: the
+                         elementwise bound is then 2e-2 + 2^-8 |ref|; runs with fp32 outputs are held to the plain 2e-2.
   routing:               the map must equal the oracle's except at entries whose oracle score lies
                          within 1e-3 * tau (relative) of the threshold tau = smallest kept score of
                          that (batch, head) [per-sequence] or row [per-query]; counts must be exact.
@@ -35,9 +38,15 @@ def err(a: np.ndarray, b: np.ndarray):
     return float(d.max()) if d.size else 0.0, float(d.mean() / max(np.abs(b).mean(), 1e-30)) if d.size else 0.0
 
 
-def assert_close(name, a, b, tol_abs=TOL_ABS, tol_rel=TOL_REL):
+def assert_close(name, a, b, tol_abs=TOL_ABS, tol_rel=TOL_REL, bf16_storage=False):
     mx, rel = err(a, b)
-    assert mx <= tol_abs and rel <= tol_rel, f"{name}: max abs err {mx:.3e} (tol {tol_abs}), mean rel err {rel:.3e} (tol {tol_rel})"
+    if bf16_storage:
+        excess = float((np.abs(a - b) - 2.0 ** -8 * np.abs(b)).max()) if a.size else 0.0
+        ok_abs = excess <= tol_abs
+    else:
+        ok_abs = mx <= tol_abs
+    assert ok_abs and rel <= tol_rel, (f"{name}: max abs err {mx:.3e} (tol {tol_abs}"
+                                       f"{' + bf16 storage rounding' if bf16_storage else ''}), mean rel err {rel:.3e} (tol {tol_rel})")
     return mx, rel
 
 
