@@ -59,10 +59,11 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
        VSA2_FLAG_EXACT_MAX_FWD = 2 }; /* validation aid: run the whole fine forward with the slow kernel that tracks
                                          the exact running row maximum (the tensor-core kernel falls back to it only
                                          for query blocks whose softmax sums leave the safe range) */
+enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */
 
 /* Problem statement (host struct). */
 typedef struct vsa2_params {
-  int32_t batch, heads_q, heads_kv, head_dim;  /* head_dim in {64, 128}; heads_q % heads_kv == 0 */
+  int32_t batch, heads_q, heads_kv, head_dim;  /* head_dim in {64, 128}; heads_q % heads_kv == 0, ratio <= 16 */
   int32_t grid_t, grid_h, grid_w;              /* valid latent grid */
   int32_t cube_t, cube_h, cube_w;              /* cube (block) shape, product must be 64 */
   int32_t rpool_t, rpool_h, rpool_w;           /* router pooling R, each divides the cube dimension */

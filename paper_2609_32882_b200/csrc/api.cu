@@ -41,7 +41,7 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   if (p->cube_t % p->rpool_t || p->cube_h % p->rpool_h || p->cube_w % p->rpool_w) return VSA2_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return VSA2_ERR_UNSUPPORTED;
   if ((long long)p->cube_t * p->cube_h * p->cube_w != kBlockTokens) return VSA2_ERR_UNSUPPORTED;
-  if (p->batch > 65535 || p->heads_q > 65535) return VSA2_ERR_UNSUPPORTED;
+  if (p->batch > 65535 || p->heads_q > 65535 || p->heads_q / p->heads_kv > 16) return VSA2_ERR_UNSUPPORTED;
   g->batch = p->batch; g->Hq = p->heads_q; g->Hkv = p->heads_kv; g->rep = p->heads_q / p->heads_kv; g->D = p->head_dim;
   g->T = p->grid_t; g->H = p->grid_h; g->W = p->grid_w;
   long long L = (long long)g->T * g->H * g->W;
@@ -319,13 +319,22 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
-    VSA2_CUDA(launch_fine_bwd_dq(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx, coarse ? dqc : nullptr,
-                                 dq, st));
+    if (g.flags & VSA2_FLAG_SIMPLE_BWD)
+      VSA2_CUDA(launch_fine_bwd_dq(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx,
+                                   coarse ? dqc : nullptr, dq, st));
+    else
+      VSA2_CUDA(launch_fine_bwd_dq_tc(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx,
+                                      coarse ? dqc : nullptr, dq, reinterpret_cast<StatusBlock*>(workspace), st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
-    VSA2_CUDA(launch_fine_bwd_dkv(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx,
-                                  coarse ? dkc : nullptr, coarse ? dvc : nullptr, dk, dv, st));
+    if (g.flags & VSA2_FLAG_SIMPLE_BWD)
+      VSA2_CUDA(launch_fine_bwd_dkv(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx,
+                                    coarse ? dkc : nullptr, coarse ? dvc : nullptr, dk, dv, st));
+    else
+      VSA2_CUDA(launch_fine_bwd_dkv_tc(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx,
+                                       coarse ? dkc : nullptr, coarse ? dvc : nullptr, dk, dv,
+                                       reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;
 }

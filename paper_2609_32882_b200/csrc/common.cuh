@@ -143,6 +143,15 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
                                const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                float* lse, StatusBlock* status, cudaStream_t st);
 
+// tensor-core backward passes (fine_bwd_tc.cu)
+cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                                  const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
+                                  const float* dqc, void* dq, StatusBlock* status, cudaStream_t st);
+cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                                   const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
+                                   const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
+                                   cudaStream_t st);
+
 cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,
                                   const float* oc_hat, float* delta, float* dgate, float* d_oc_hat,
                                   cudaStream_t st);

@@ -18,9 +18,7 @@
 //
 // Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (one elected lane each), warps 2..5 =
 // softmax + epilogue (each owns the tensor-memory lane quadrant warp % 4).  Every wait is bounded.
-#include "common.cuh"
-#include "tc05.cuh"
-#include "tmap.cuh"
+#include "tc_attn.cuh"
 
 namespace vsa2 {
 
@@ -67,30 +65,6 @@ struct FwdArgs {
   int* rescue_count;
   int* rescue_items;
 };
-
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-// swizzled index into the 128 x 64 fp32 reduction scratch (row r written by one thread, column c read by one)
-__device__ __forceinline__ int scratch_idx(int r, int c) { return r * 64 + (c ^ (r & 31)); }
-
-__device__ __forceinline__ bool pos_valid(const Geo& g, int n, int pos) {
-  int nt, nh, nw;
-  cube_coords(g, n, nt, nh, nw);
-  return cube_token(g, nt, nh, nw, pos) >= 0;
-}
-
-#define VSA2_WAIT(bar, parity)                                        \
-  do {                                                                \
-    if (!tc::mbar_wait((bar), (parity), &misc->abort_flag)) goto done; \
-  } while (0)
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)

@@ -1,0 +1,72 @@
+// Helpers shared by the tensor-core attention kernels (forward and backward).
+#pragma once
+#include "common.cuh"
+#include "tc05.cuh"
+#include "tmap.cuh"
+
+namespace vsa2 {
+
+constexpr uint32_t kSlab = 8192;   // one cube x 64 channels of bf16, 64 rows of 128 bytes, 128-byte swizzled
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// swizzled index into a 128 x 64 fp32 reduction scratch (row r written by one thread, column c read by one)
+__device__ __forceinline__ int scratch_idx(int r, int c) { return r * 64 + (c ^ (r & 31)); }
+
+__device__ __forceinline__ bool pos_valid(const Geo& g, int n, int pos) {
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  return cube_token(g, nt, nh, nw, pos) >= 0;
+}
+
+// 64 bf16 (32 packed words) -> one 128-byte row of a swizzled operand tile: 16-byte chunk c lands at c ^ (row & 7)
+__device__ __forceinline__ void store_row_sw128(unsigned char* tile, int row, const uint32_t (&packed)[32]) {
+  unsigned char* prow = tile + row * 128;
+#pragma unroll
+  for (int ch = 0; ch < 8; ++ch)
+    *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
+        make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+}
+
+// Issues the D/16 (K-major x K-major) instructions of  acc[128, 64] = A_pair[128, D] * B[64, D]^T.
+// A_pair: slot laid out [half][block A | block B] slabs; B: tile laid out [half] slabs.
+template <int D>
+__device__ __forceinline__ void mma_pair_kmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile) {
+  constexpr uint32_t idesc = tc::idesc_bf16(128, 64, false, false);
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    const uint32_t aa = a_slot + (ks / 4) * 2 * kSlab + (ks % 4) * 32;
+    const uint32_t bb = b_tile + (ks / 4) * kSlab + (ks % 4) * 32;
+    tc::mma_ss(tm_acc, tc::smem_desc_sw128(aa, 16, 1024), tc::smem_desc_sw128(bb, 16, 1024), idesc, ks > 0);
+  }
+}
+
+// Issues the 8 (MN-major x MN-major) instructions of  acc[D, 64] (+)= A_pair^T[D, 128] * B[128, 64], where A_pair is a
+// slot in the [half][block A | block B] layout (rows = the 128 contraction indices) and B is a 128-row swizzled tile.
+template <int D>
+__device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, bool accumulate_first) {
+  constexpr uint32_t idesc = tc::idesc_bf16(128, 64, true, true);
+  constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;     // distance between the two 64-channel halves
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const uint32_t aa = a_slot + (ks / 4) * kSlab + (ks % 4) * 2048;
+    const uint32_t bb = b_tile + ks * 2048;
+    tc::mma_ss(tm_acc, tc::smem_desc_sw128(aa, lbo, 1024), tc::smem_desc_sw128(bb, 0, 1024), idesc,
+               accumulate_first || (ks > 0));
+  }
+}
+
+#define VSA2_WAIT(bar, parity)                                         \
+  do {                                                                 \
+    if (!tc::mbar_wait((bar), (parity), &misc->abort_flag)) goto done; \
+  } while (0)
+
+}  // namespace vsa2

@@ -196,3 +196,16 @@ def test_forward_survives_a_late_dominant_key_block():
     assert_lse_close(lse, lse_ref)
     rescued = int(run.attn.ws_fwd[8:12].view(torch.int32).item())
     assert rescued >= 1
+
+
+def test_tensor_core_backward_matches_first_generation_kernels():
+    wl = MINI_PADDED
+    data = syn.make_inputs(wl)
+    outs = []
+    for flags in (0, vb.FLAG_SIMPLE_BWD):
+        run = GpuRun(wl, data, flags=flags, out_dtype=vb.F32)
+        run.route()
+        run.forward()
+        outs.append(run.backward())
+    for name, x, y in zip(("dQ", "dK", "dV", "dGate"), *outs):
+        assert np.abs(x - y).max() < 2e-2, name
