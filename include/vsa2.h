@@ -59,6 +59,7 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
        VSA2_FLAG_EXACT_MAX_FWD = 2 }; /* validation aid: run the whole fine forward with the slow kernel that tracks
                                          the exact running row maximum (the tensor-core kernel falls back to it only
                                          for query blocks whose softmax sums leave the safe range) */
+enum { VSA2_FLAG_SIMPLE_ROUTER = 8 }; /* validation aid: router scores with the slow first-generation kernel */
 enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */
 
 /* Problem statement (host struct). */

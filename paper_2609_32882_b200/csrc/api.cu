@@ -206,7 +206,10 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
     VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(k), g.Hkv, kr, nullptr, st));
   }
   float* pr = at<float>(workspace, lay.pr);
-  VSA2_CUDA(launch_router_scores(g, qr, kr, at<float>(workspace, lay.lse_r), pr, st));
+  if (router_tc_supported(g) && !(g.flags & VSA2_FLAG_SIMPLE_ROUTER))
+    VSA2_CUDA(launch_router_scores_tc(g, qr, kr, at<float>(workspace, lay.lse_r), pr, status, st));
+  else
+    VSA2_CUDA(launch_router_scores(g, qr, kr, at<float>(workspace, lay.lse_r), pr, st));
   SelectScratch s;
   s.hist = at<unsigned>(workspace, lay.hist);
   s.state = at<unsigned>(workspace, lay.state);

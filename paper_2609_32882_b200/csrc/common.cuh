@@ -112,6 +112,11 @@ cudaError_t launch_pool(const Geo& g, const bf16* x, int heads, bf16* xr, float*
 cudaError_t launch_router_scores(const Geo& g, const bf16* qr, const bf16* kr, float* lse_r, float* pr,
                                  cudaStream_t st);
 
+// tensor-core router (router_tc.cu): lse_r holds log2-domain row statistics between its two passes
+bool router_tc_supported(const Geo& g);
+cudaError_t launch_router_scores_tc(const Geo& g, const bf16* qr, const bf16* kr, float* lse_r, float* pr,
+                                    StatusBlock* status, cudaStream_t st);
+
 struct SelectScratch {
   unsigned* hist;        // [BH][3][2048]
   unsigned* state;       // [BH][8]

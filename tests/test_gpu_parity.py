@@ -209,3 +209,15 @@ def test_tensor_core_backward_matches_first_generation_kernels():
         outs.append(run.backward())
     for name, x, y in zip(("dQ", "dK", "dV", "dGate"), *outs):
         assert np.abs(x - y).max() < 2e-2, name
+
+
+def test_tensor_core_router_matches_first_generation_kernel():
+    wl = MINI_PADDED
+    data = syn.make_inputs(wl)
+    scores = []
+    for flags in (0, vb.FLAG_SIMPLE_ROUTER):
+        run = GpuRun(wl, data, flags=flags)
+        run.route()
+        scores.append(to_f64(run.attn.scores()))
+    assert np.abs(scores[0] - scores[1]).max() <= 1e-5 * scores[1].max()
+    assert np.allclose(scores[0].sum(axis=-1), 1.0 / 8, atol=1e-5)      # rows of P_r sum to 1/G
