@@ -206,6 +206,7 @@ def run_ours(args):
 
     from paper_2609_32882_b200 import binding as vb
     from paper_2609_32882_b200 import build as vbuild
+    from paper_2609_32882_b200 import replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -223,7 +224,7 @@ def run_ours(args):
 
     # every rank runs its own replica of the workload (heads are independent: no data-path collective)
     wl = workload(args.config)
-    wl = wl.replace(seed=wl.seed + 1000 * rank)
+    wl = wl.replace(seed=replicas.replica_seed(wl.seed, rank))
     t_gen = time.time()
     data = syn.make_inputs(wl, threads=max(1, min(32, cpu_cores() // max(1, world))))
     t_gen = time.time() - t_gen
@@ -314,10 +315,7 @@ def run_ours(args):
     barrier()
     ms_e2e = e_start.elapsed_time(e_stop)
 
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = t.tolist()
+    ms_total, ms_e2e = replicas.max_over_ranks([ms_total, ms_e2e], device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -326,8 +324,8 @@ def run_ours(args):
     flops = flop_counts(wl, nnz_total)
     ms_step = ms_total / args.steps
     ms_step_e2e = ms_e2e / args.steps
-    value = world * flops["dense_equiv_fwd_bwd"] / (ms_step * 1e-3) / 1e12
-    value_e2e = world * flops["dense_equiv_fwd_bwd"] / (ms_step_e2e * 1e-3) / 1e12
+    value = replicas.whole_job_throughput(flops["dense_equiv_fwd_bwd"], world, ms_step * 1e-3) / 1e12
+    value_e2e = replicas.whole_job_throughput(flops["dense_equiv_fwd_bwd"], world, ms_step_e2e * 1e-3) / 1e12
     pk, pk_kind = peaks()
     executed = flops["fine_fwd"] + flops["fine_bwd_dq_executed"] + flops["fine_bwd_dkv_executed"] + 2 * flops["router_per_pass"]
     kernel_flops = {"fine_fwd": flops["fine_fwd"], "fine_bwd_dq": flops["fine_bwd_dq_executed"],
