@@ -46,7 +46,8 @@ enum {
   VSA2_ERR_MISALIGNED = -4,
   VSA2_ERR_CUDA = -5,                 /* a CUDA runtime/driver call or a launch failed */
   VSA2_ERR_DEVICE_TIMEOUT = -6,       /* a bounded device-side wait ran out (reported by vsa2_device_status) */
-  VSA2_ERR_MAP_OVERFLOW = -7          /* more selected blocks than nnz_cap (reported by vsa2_device_status) */
+  VSA2_ERR_MAP_OVERFLOW = -7,         /* more selected blocks than nnz_cap (reported by vsa2_device_status) */
+  VSA2_ERR_STATIC_SCRATCH = -8        /* vsa2_route_noalloc: the problem needs more scratch than the built-in buffer */
 };
 
 enum { VSA2_PER_SEQUENCE = 0,         /* Eq. 8-9: the N*K largest entries of the flattened P_r per (batch, query head) */
@@ -134,6 +135,26 @@ int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out);
  * defined through this call (Sec. 2.1). */
 int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t* budgets,
                const vsa2_map* map_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Allocation-free variant of vsa2_route (the paper has no counterpart).
+ *
+ * For callers that cannot allocate device memory where they need a block map: code running where cudaMalloc is
+ * forbidden or would stall (an allocator lock is held, a latency-critical loop sized up front, a plug-in that is
+ * handed no allocator) or a process whose memory budget is fixed at start-up.  Same inputs, outputs, readings and
+ * error codes as vsa2_route, but the workspace is a device array built into the library: 8 MiB
+ * (VSA2_ROUTE_NOALLOC_MAX_BYTES) that every GPU loading the library holds until the process exits.
+ *   - A problem whose sizes.route_workspace_bytes exceeds 8 MiB is rejected with VSA2_ERR_STATIC_SCRATCH before
+ *     anything is enqueued (roughly: up to ~2k tokens x 12 heads fits; the 480p and 720p shapes do not).
+ *   - device_status: optional device int32; if not NULL the status word of this call (VSA2_OK,
+ *     VSA2_ERR_MAP_OVERFLOW, VSA2_ERR_DEVICE_TIMEOUT) is copied there on the stream, after the kernels.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *     current); make that first call outside any stream capture.  No call allocates or frees device memory.
+ *   - All calls on one device share the one array, and it keeps the last call's contents: the call clears what
+ *     must start at zero itself, but two calls that overlap on the GPU (different streams, no ordering) race;
+ *     order them on one stream or with events.  Host-side it is safe to call from several threads. */
+#define VSA2_ROUTE_NOALLOC_MAX_BYTES (8u << 20)
+int vsa2_route_noalloc(const vsa2_params* p, const void* q, const void* k, const int32_t* budgets,
+                       const vsa2_map* map_out, int32_t* device_status, void* cuda_stream);
 
 /* Read-only access to the block scores P_r [batch, heads_q, N, N] (fp32) that the last vsa2_route
  * call on `workspace` left there; valid until the workspace is reused.  Returns NULL on bad input. */

@@ -25,9 +25,10 @@ FLAG_SIMPLE_ROUTER = 8
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
 ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_MAP_OVERFLOW = -5, -6, -7
+ERR_STATIC_SCRATCH = -8
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
-           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma")
+           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv")
@@ -82,6 +83,7 @@ def _lib():
         vp, sz, i32p = C.c_void_p, C.c_size_t, C.POINTER(C.c_int32)
         lib.vsa2_query_sizes.argtypes = [C.POINTER(Params), C.POINTER(Sizes)]
         lib.vsa2_route.argtypes = [C.POINTER(Params), vp, vp, vp, C.POINTER(Map), vp, sz, vp]
+        lib.vsa2_route_noalloc.argtypes = [C.POINTER(Params), vp, vp, vp, C.POINTER(Map), vp, vp]
         lib.vsa2_route_scores.argtypes = [C.POINTER(Params), vp]
         lib.vsa2_route_scores.restype = vp
         lib.vsa2_attn_fwd.argtypes = [C.POINTER(Params), vp, vp, vp, vp, C.POINTER(Map), vp, vp, C.POINTER(Saved), vp, sz, vp]
@@ -153,6 +155,15 @@ def vsa2_route(p, q, k, budgets, vmap: Map, workspace, workspace_bytes=None, str
     nbytes = workspace_bytes if workspace_bytes is not None else workspace.numel() * workspace.element_size()
     _check(_lib().vsa2_route(C.byref(p), _ptr(q), _ptr(k), _ptr(budgets), C.byref(vmap), _ptr(workspace), nbytes,
                              _stream(stream)), "vsa2_route")
+
+
+def vsa2_route_noalloc(p, q, k, budgets, vmap: Map, device_status=None, stream=None):
+    """Router + selection without a caller workspace (scratch is a fixed 8 MiB array inside the library).
+
+    For callers that cannot allocate device memory at this point; problems needing more scratch raise
+    Vsa2Error(ERR_STATIC_SCRATCH).  `device_status`: optional int32 CUDA tensor receiving the status word."""
+    _check(_lib().vsa2_route_noalloc(C.byref(p), _ptr(q), _ptr(k), _ptr(budgets), C.byref(vmap), _ptr(device_status),
+                                     _stream(stream)), "vsa2_route_noalloc")
 
 
 def vsa2_route_scores(p, workspace) -> int:

@@ -362,6 +362,7 @@ const char* vsa2_strerror(int code) {
     case VSA2_ERR_CUDA: return "CUDA call or kernel launch failed";
     case VSA2_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
     case VSA2_ERR_MAP_OVERFLOW: return "more selected blocks than nnz_cap";
+    case VSA2_ERR_STATIC_SCRATCH: return "problem needs more scratch than the library's built-in 8 MiB buffer (use vsa2_route)";
     default: return "unknown vsa2 error";
   }
 }

@@ -96,11 +96,11 @@ def test_null_pointers_are_rejected_before_any_cuda_call(lib):
 
 def test_strerror_covers_every_code():
     seen = set()
-    for code in range(0, -8, -1):
+    for code in range(0, -9, -1):
         msg = vb._lib().vsa2_strerror(code).decode()
         assert msg and "unknown" not in msg
         seen.add(msg)
-    assert len(seen) == 8
+    assert len(seen) == 9
     assert "unknown" in vb._lib().vsa2_strerror(-99).decode()
 
 
