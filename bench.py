@@ -39,8 +39,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {}
 
 
-def workload(config: int) -> syn.Workload:
-    return syn.CONFIGS[config]
+def workload(config: int, heads: int = 0) -> syn.Workload:
+    wl = syn.CONFIGS[config]
+    if heads:
+        wl = wl.replace(heads_q=heads, heads_kv=max(1, heads * wl.heads_kv // wl.heads_q), name=f"{wl.name}_{heads}heads")
+    return wl
 
 
 def flop_counts(wl: syn.Workload, nnz_total: int) -> dict:
@@ -172,7 +175,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = workload(args.config)
+    wl = workload(args.config, args.heads)
     hd = head_inputs(wl, 0, 0)
     flops = flop_counts(wl, 0)
     for _ in range(args.warmup):
@@ -223,7 +226,7 @@ def run_ours(args):
     vb._lib()
 
     # every rank runs its own replica of the workload (heads are independent: no data-path collective)
-    wl = workload(args.config)
+    wl = workload(args.config, args.heads)
     wl = wl.replace(seed=replicas.replica_seed(wl.seed, rank))
     t_gen = time.time()
     data = syn.make_inputs(wl, threads=max(1, min(32, cpu_cores() // max(1, world))))
@@ -304,16 +307,18 @@ def run_ours(args):
     attn.check_status()
 
     # end to end: host buffers in, results back to the host, copies inside the timed region
-    for _ in range(2):
-        step_e2e()
-    barrier()
-    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_start.record()
-    for _ in range(args.steps):
-        step_e2e()
-    e_stop.record()
-    barrier()
-    ms_e2e = e_start.elapsed_time(e_stop)
+    ms_e2e = float("nan")
+    if not args.no_e2e:
+        for _ in range(2):
+            step_e2e()
+        barrier()
+        e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e_start.record()
+        for _ in range(args.steps):
+            step_e2e()
+        e_stop.record()
+        barrier()
+        ms_e2e = e_start.elapsed_time(e_stop)
 
     ms_total, ms_e2e = replicas.max_over_ranks([ms_total, ms_e2e], device="cuda")
     if rank != 0:
@@ -390,6 +395,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="index into the five baseline configurations (3 = 720p top-64)")
     ap.add_argument("--ref-rows", type=int, default=96, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
+    ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small cases for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

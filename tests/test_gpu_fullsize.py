@@ -1,0 +1,121 @@
+"""GPU parity at the full sizes of the baseline configurations 2-4, in the launch configuration the benchmark
+times.  The GPU runs the whole problem; the oracle checks the routing of whole heads and sampled outputs
+(query blocks / KV blocks it can compute one by one), plus properties that hold at any size."""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import vsa2_oracle as orc
+from paper_2609_32882_b200 import binding as vb
+from paper_2609_32882_b200 import inputs as syn
+from vsa2_testlib import (GpuRun, assert_close, check_routing, oracle_arrays, sampled_attention_parity, to_f64)
+
+pytestmark = pytest.mark.gpu
+
+
+@functools.lru_cache(maxsize=2)
+def inputs_for(config, heads_kv=None):
+    wl = syn.CONFIGS[config]
+    if heads_kv is not None:
+        wl = wl.replace(heads_kv=heads_kv)
+    return wl, syn.make_inputs(wl, threads=16)
+
+
+def oracle_route_head(wl, data, b, hq, mode, topk, budgets=None):
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    hk = hq // (wl.heads_q // wl.heads_kv)
+    Q = orc.bf16_bits_to_f64(data["q"][b, hq])[None, None]
+    K = orc.bf16_bits_to_f64(data["k"][b, hk])[None, None]
+    bud = None if budgets is None else budgets[b:b + 1, hq:hq + 1]
+    m, P = orc.route(Q, K, geo, 1.0 / np.sqrt(wl.head_dim), mode, topk, bud, return_scores=True)
+    return m[0, 0], P[0, 0]
+
+
+def test_config2_480p_gqa_padded():
+    wl, data = inputs_for(2)
+    run = GpuRun(wl, data)
+    gmask = run.route()
+    assert (gmask.sum(axis=-1) == 78).all()                                   # 87.5 % sparsity: 78 of 624 per row
+    for hq in (0, 5, 11):
+        om, P = oracle_route_head(wl, data, 0, hq, wl.select_mode, wl.topk)
+        check_routing(gmask[0, hq], om, P, wl.select_mode)
+        pr = to_f64(run.attn.scores()[0, hq])
+        assert np.abs(pr - P).max() <= 1e-4 * P.max()
+    run.forward()
+    run.backward()
+    N = wl.n_cubes
+    sampled_attention_parity(wl, data, run, gmask, q_heads=(1, 10), rows=(0, 311, N - 1),
+                             kv_groups=(0,), kv_cubes=(7, N - 1))               # N-1 is a ragged corner cube
+    assert torch.isfinite(run.o.float()).all() and torch.isfinite(run.dk.float()).all()
+
+
+def test_config3_720p_top64_forward_backward():
+    wl, data = inputs_for(3)
+    run = GpuRun(wl, data)
+    gmask = run.route()
+    N = wl.n_cubes
+    assert (gmask.sum(axis=(-1, -2)) == N * 64).all()                          # exactly N*K pairs per head (Eq. 9)
+    rows = gmask.sum(axis=-1)
+    assert rows.min() < 64 < rows.max()                                        # variable KV count per query block
+    for hq in (0, 39):
+        om, P = oracle_route_head(wl, data, 0, hq, syn.PER_SEQUENCE, 64)
+        check_routing(gmask[0, hq], om, P, syn.PER_SEQUENCE)
+    run.forward()
+    run.backward()
+    heavy = int(np.argmax(gmask[0, 17].sum(axis=0)))                           # the most selected KV block of head 17
+    sampled_attention_parity(wl, data, run, gmask, q_heads=(0, 39), rows=(3, 700, N - 1),
+                             kv_groups=(17,), kv_cubes=(heavy, N - 1))
+
+
+def test_config3_720p_top128_forward_only():
+    wl, data = inputs_for(3)
+    run = GpuRun(wl.replace(topk=128), data)
+    gmask = run.route()
+    assert (gmask.sum(axis=(-1, -2)) == wl.n_cubes * 128).all()
+    run.forward()
+    sampled_attention_parity(wl, data, run, gmask, q_heads=(21,), rows=(100, 1400), backward=False)
+
+
+def test_config4_budgets_mha_and_dense_reference():
+    wl, data = inputs_for(4)
+    N = wl.n_cubes
+    cap = int(np.minimum(data["budgets"], N).sum(axis=-1).max())
+    run = GpuRun(wl, data, nnz_cap=cap)
+    gmask = run.route()
+    assert np.array_equal(gmask.sum(axis=-1), data["budgets"])                 # every row keeps exactly its budget
+    om, P = oracle_route_head(wl, data, 0, 8, syn.PER_QUERY_BUDGET, 0, data["budgets"])
+    check_routing(gmask[0, 8], om, P, syn.PER_QUERY_BUDGET)
+    run.forward()
+    run.backward()
+    sampled_attention_parity(wl, data, run, gmask, q_heads=(8,), rows=(5, 1000), kv_groups=(30,), kv_cubes=(77,))
+    # dense reference: the same kernels with every block kept, against softmax attention over all valid keys
+    sub = wl.replace(heads_q=4, heads_kv=4, select_mode=syn.PER_SEQUENCE, topk=N)
+    dsub = {k: np.ascontiguousarray(v[:, :4]) for k, v in data.items()}
+    dense = GpuRun(sub, dsub, flags=vb.FLAG_NO_COARSE)
+    assert dense.route().all()
+    dense.forward()
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    a = {k: orc.bf16_bits_to_f64(dsub[k][0, 2]) for k in ("q", "k", "v")}
+    rows = (0, 719, N - 1)
+    toks = np.concatenate([geo.cube_tokens[i] for i in rows])
+    s = a["q"][toks] @ a["k"].T / np.sqrt(wl.head_dim)
+    p = np.exp(s - s.max(axis=1, keepdims=True))
+    ref = (p / p.sum(axis=1, keepdims=True)) @ a["v"]
+    assert_close("dense O", to_f64(dense.o[0, 2][toks]), ref, bf16_storage=True)
+
+
+def test_config4_gqa_sparsity_levels():
+    wl, data = inputs_for(4, heads_kv=10)
+    N = wl.n_cubes
+    for topk in (360, 45):                                                     # 75 % and 96.9 % block sparsity
+        w = wl.replace(select_mode=syn.PER_SEQUENCE, topk=topk)
+        run = GpuRun(w, data)
+        gmask = run.route()
+        assert (gmask.sum(axis=(-1, -2)) == N * topk).all()
+        run.forward()
+        run.backward()
+        sampled_attention_parity(w, data, run, gmask, q_heads=(13,), rows=(640,), kv_groups=(3,), kv_cubes=(900,))
+        del run
+        torch.cuda.empty_cache()

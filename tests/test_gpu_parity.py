@@ -6,7 +6,7 @@ import torch
 from oracle import vsa2_oracle as orc
 from paper_2609_32882_b200 import binding as vb
 from paper_2609_32882_b200 import inputs as syn
-from vsa2_testlib import (GpuRun, assert_close, assert_lse_close, check_routing, dev_bf16, oracle_arrays, to_f64)
+from vsa2_testlib import (TOL_ABS, GpuRun, assert_close, assert_lse_close, check_routing, dev_bf16, oracle_arrays, to_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -39,8 +39,9 @@ def full_parity(wl, data, out_dtype=vb.BF16, nnz_cap=0, check_route=True):
     dQ_ref, dK_ref, dV_ref, dG_ref = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
     dQ, dK, dV, dG = run.backward()
     assert_close("dQ", dQ, dQ_ref, bf16_storage=st)
-    assert_close("dK", dK, dK_ref, bf16_storage=st)
-    assert_close("dV", dV, dV_ref, bf16_storage=st)
+    tol_kv = TOL_ABS * np.sqrt(wl.heads_q // wl.heads_kv)          # group-summed gradients (see vsa2_testlib)
+    assert_close("dK", dK, dK_ref, tol_abs=tol_kv, bf16_storage=st)
+    assert_close("dV", dV, dV_ref, tol_abs=tol_kv, bf16_storage=st)
     assert_close("dGate", dG, dG_ref)
     return run
 

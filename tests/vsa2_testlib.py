@@ -8,6 +8,9 @@ Tolerances (fp32 comparison against the fp64 oracle):
                          When the library stores a tensor in bf16 (out_dtype BF16) the storage rounding,
                          up to 2^-8 |x| per element (half an ulp at the bottom of a binade), comes on top: the
                          elementwise bound is then 2e-2 + 2^-8 |ref|; runs with fp32 outputs are held to the plain 2e-2.
+                         dK and dV of a GQA group are sums over the group's `rep` query heads, each within
+                         the bound above; independent rounding noise adds in quadrature, so group-summed dK, dV are
+                         held to sqrt(rep) * 2e-2 (rep = 1 for MHA: unchanged).
   routing:               the map must equal the oracle's except at entries whose oracle score lies
                          within 1e-3 * tau (relative) of the threshold tau = smallest kept score of
                          that (batch, head) [per-sequence] or row [per-query]; counts must be exact.
@@ -131,3 +134,57 @@ def oracle_arrays(data):
     out = {k: orc.bf16_bits_to_f64(data[k]) for k in ("q", "k", "v", "do") if k in data}
     out["gate"] = data["gate"].astype(np.float64)
     return out
+
+
+def sampled_attention_parity(wl, data, run, gmask, q_heads, rows, kv_groups=(), kv_cubes=(), backward=True):
+    """Oracle vs GPU on sampled outputs of a full-size run (the full oracle would take hours):
+    O, lse, dQ, dGate on the tokens of the query cubes `rows` of the query heads `q_heads`; dK, dV on the tokens
+    of `kv_cubes` for the KV heads `kv_groups` (all query heads of the group, all query blocks that keep the cube).
+    `run` must have executed forward (and backward).  bf16 outputs are assumed."""
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    rep = wl.heads_q // wl.heads_kv
+    o_gpu, lse_gpu = run.o, run.lse
+    stats = {}
+
+    def head_arrays(b, hq):
+        hk = hq // rep
+        return (orc.bf16_bits_to_f64(data["q"][b, hq]), orc.bf16_bits_to_f64(data["k"][b, hk]),
+                orc.bf16_bits_to_f64(data["v"][b, hk]), data["gate"][b, hq].astype(np.float64),
+                orc.bf16_bits_to_f64(data["do"][b, hq]) if backward else None)
+
+    def coarse_fwd(Q, K, V):
+        Qc, Kc, Vc = orc.mean_pool_cube(Q, geo), orc.mean_pool_cube(K, geo), orc.mean_pool_cube(V, geo)
+        Oc_hat, lse_c = orc.coarse_attention(Qc, Kc, Vc, scale)
+        return dict(Oc_hat=Oc_hat, lse_c=lse_c, Qc=Qc, Kc=Kc, Vc=Vc)
+
+    b = 0
+    for hq in q_heads:
+        Q, K, V, gate, dO = head_arrays(b, hq)
+        fwd = coarse_fwd(Q, K, V)
+        toks = np.concatenate([geo.cube_tokens[i] for i in rows])
+        O_f, lse = orc.fine_attention(Q, K, V, gmask[b, hq], geo, scale, rows=rows)
+        O_ref = gate[toks, None] * fwd["Oc_hat"][geo.cube_of[toks]] + O_f[toks]
+        stats[f"O_h{hq}"] = assert_close(f"O head {hq}", to_f64(o_gpu[b, hq][toks]), O_ref, bf16_storage=True)
+        assert_lse_close(to_f64(lse_gpu[b, hq][toks]), lse[toks])
+        if backward:
+            c = orc.coarse_path_backward(Q, K, V, gate, geo, scale, dO, fwd)
+            fq, _, _ = orc.fine_backward(Q, K, V, gmask[b, hq], geo, scale, dO, lse, O_f, rows=rows)
+            stats[f"dQ_h{hq}"] = assert_close(f"dQ head {hq}", to_f64(run.dq[b, hq][toks]), (c["dQ"] + fq)[toks], bf16_storage=True)
+            assert_close(f"dGate head {hq}", to_f64(run.dgate[b, hq][toks]), c["dGate"][toks])
+    if backward:
+        for hk in kv_groups:
+            toks = np.concatenate([geo.cube_tokens[j] for j in kv_cubes])
+            dK_ref = np.zeros((toks.size, wl.head_dim))
+            dV_ref = np.zeros((toks.size, wl.head_dim))
+            for hq in range(hk * rep, (hk + 1) * rep):
+                Q, K, V, gate, dO = head_arrays(b, hq)
+                fwd = coarse_fwd(Q, K, V)
+                c = orc.coarse_path_backward(Q, K, V, gate, geo, scale, dO, fwd)
+                fk, fv = orc.fine_backward_kv_cubes(Q, K, V, gmask[b, hq], geo, scale, dO, kv_cubes)
+                dK_ref += (c["dK"] + fk)[toks]
+                dV_ref += (c["dV"] + fv)[toks]
+            tol = TOL_ABS * np.sqrt(rep)
+            stats[f"dK_g{hk}"] = assert_close(f"dK kv head {hk}", to_f64(run.dk[b, hk][toks]), dK_ref, tol_abs=tol, bf16_storage=True)
+            stats[f"dV_g{hk}"] = assert_close(f"dV kv head {hk}", to_f64(run.dv[b, hk][toks]), dV_ref, tol_abs=tol, bf16_storage=True)
+    return stats
