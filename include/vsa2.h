@@ -220,6 +220,9 @@ int vsa2_selftest_umma(const vsa2_params* p, const void* q, const void* k, const
                        int32_t cube_a, int32_t cube_b, const void* p_t, float* s_t_out, float* o_t_out,
                        void* k_tile_dump, int32_t* status, void* cuda_stream);
 
+/* Text of the CUDA error behind the most recent VSA2_ERR_CUDA returned in this process ("no error" if none). */
+const char* vsa2_last_cuda_error(void);
+
 /* Static string for an error code. */
 const char* vsa2_strerror(int code);
 

@@ -28,7 +28,7 @@ ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_MAP_OVERFLOW = -5, -6, -7
 ERR_STATIC_SCRATCH = -8
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
-           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc")
+           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc", "vsa2_last_cuda_error")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv")
@@ -38,6 +38,8 @@ class Vsa2Error(RuntimeError):
     def __init__(self, code, where):
         self.code = code
         msg = _lib().vsa2_strerror(code).decode() if _LIB is not None else "library not loaded"
+        if code == ERR_CUDA and _LIB is not None:
+            msg += ": " + _lib().vsa2_last_cuda_error().decode()
         super().__init__(f"{where}: {msg} (code {code})")
 
 
@@ -90,6 +92,8 @@ def _lib():
         lib.vsa2_attn_bwd.argtypes = [C.POINTER(Params), vp, vp, vp, vp, C.POINTER(Map), vp, vp, C.POINTER(Saved), vp,
                                       vp, vp, vp, vp, vp, sz, vp]
         lib.vsa2_device_status.argtypes = [vp, vp, i32p]
+        lib.vsa2_last_cuda_error.argtypes = []
+        lib.vsa2_last_cuda_error.restype = C.c_char_p
         lib.vsa2_strerror.argtypes = [C.c_int]
         lib.vsa2_strerror.restype = C.c_char_p
         lib.vsa2_profile_events.argtypes = [C.c_int32, vp, vp]
@@ -97,7 +101,7 @@ def _lib():
         lib.vsa2_launch_count.argtypes = []
         lib.vsa2_launch_count.restype = C.c_int64
         for name in EXPORTS:
-            if name not in ("vsa2_strerror", "vsa2_route_scores", "vsa2_launch_count"):
+            if name not in ("vsa2_strerror", "vsa2_route_scores", "vsa2_launch_count", "vsa2_last_cuda_error"):
                 getattr(lib, name).restype = C.c_int
         _LIB = lib
     return _LIB

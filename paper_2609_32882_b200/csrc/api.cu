@@ -129,10 +129,15 @@ int check_device() {
 template <typename T>
 T* at(void* ws, size_t off) { return reinterpret_cast<T*>(reinterpret_cast<unsigned char*>(ws) + off); }
 
+cudaError_t g_last_cuda_error = cudaSuccess;
+
 #define VSA2_CUDA(call)                              \
   do {                                               \
     cudaError_t e_ = (call);                         \
-    if (e_ != cudaSuccess) return VSA2_ERR_CUDA;     \
+    if (e_ != cudaSuccess) {                         \
+      g_last_cuda_error = e_;                        \
+      return VSA2_ERR_CUDA;                          \
+    }                                                \
   } while (0)
 
 }  // namespace
@@ -157,6 +162,8 @@ int vsa2_profile_events(int32_t kernel_id, void* start_event, void* stop_event) 
 }
 
 int64_t vsa2_launch_count(void) { return g_launches; }
+
+const char* vsa2_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
   if (out == nullptr) return VSA2_ERR_INVALID_ARG;

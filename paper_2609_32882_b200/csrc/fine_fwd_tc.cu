@@ -22,33 +22,39 @@
 
 namespace vsa2 {
 
-constexpr int kFwdThreads = 192;
-constexpr int kFwdSlots = 5;
+constexpr int kFwdThreads = 384;
+constexpr int kFwdKSlots = 3;   // ring of K pairs: filled by warp 0, drained by the S^T issuer
+constexpr int kFwdVSlots = 2;   // ring of V pairs: filled by warp 3, drained by the O^T issuer
+constexpr int kFwdSlots = kFwdKSlots + kFwdVSlots;
+constexpr int kFwdSBufs = 4;
 constexpr int kRescueCap = 16384;
+constexpr int kFwdMaxCubes = 12288;   // edge-flag table in shared memory: one byte per cube
 
 template <int D>
 struct FwdTc {
   static constexpr int DH = D / 64;
-  static constexpr uint32_t SLAB = 8192;             // one cube x 64 channels
-  static constexpr uint32_t SLOT = 2 * DH * SLAB;    // a K pair or a V pair
+  static constexpr uint32_t SLAB = kSlab;            // one cube x 64 channels
+  static constexpr uint32_t SLOT = 2 * DH * SLAB;    // a K pair or a V pair, [half][A | B]
   static constexpr uint32_t QBYTES = DH * SLAB;
   static constexpr uint32_t PBYTES = 128 * 128;      // P^T: 128 key rows x 64 queries bf16
   static constexpr uint32_t OFF_Q = kFwdSlots * SLOT;
   static constexpr uint32_t OFF_P = OFF_Q + QBYTES;
   static constexpr uint32_t OFF_MISC = OFF_P + 2 * PBYTES;
-  static constexpr uint32_t MISC_BYTES = 4096;
-  static constexpr size_t smem_bytes = OFF_MISC + MISC_BYTES + 1024;
+  static constexpr uint32_t MISC_BYTES = 2048;
+  static size_t smem_bytes(int n_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_cubes + 15) / 16 * 16 + 1024; }
 };
 
 struct FwdMisc {
   uint64_t q_full, q_empty, o_full, o_empty;
-  uint64_t kv_full[kFwdSlots], kv_empty[kFwdSlots];
-  uint64_t s_full[2], p_ready[2], p_free[2];
+  uint64_t k_full[kFwdKSlots], k_empty[kFwdKSlots];
+  uint64_t v_full[kFwdVSlots], v_empty[kFwdVSlots];
+  uint64_t s_full[kFwdSBufs], s_free[kFwdSBufs];
+  uint64_t p_ready[2], p_free[2];
   uint32_t tmem_base;
   int abort_flag;
   int rescue_flag;
-  float m_ref[64];          // per query column: reference exponent (log2 units)
-  float l_inv[64];
+  alignas(16) float m_ref[64];   // per query column: reference exponent (log2 units); read as float4
+  alignas(16) float l_inv[64];
   int tok[2][64];           // raster token of each query position (-1 = padding), by item parity
   float gate[2][64];
 };
@@ -66,6 +72,13 @@ struct FwdArgs {
   int* rescue_items;
 };
 
+// Roles (384 threads = 3 warpgroups):
+//   warpgroup 0: warps 0 and 3 = TMA producers (K pairs + Q tile, V pairs), warp 1 = issuer of the S^T products,
+//                warp 2 = issuer of the O^T products (one elected lane each; the work is split because one thread
+//                cannot issue a tile's 8 copies, 16 MMAs, commits and waits fast enough).  Gives most of its
+//                registers away.
+//   warpgroups 1, 2: softmax + epilogue; warpgroup w handles the tiles with (global tile index & 1) == w - 1, so two
+//                tiles are in the exponential unit at any time.  A warp owns tensor-memory lane quadrant warp % 4.
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -76,24 +89,33 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   unsigned char* q_tile = smem + C::OFF_Q;
   unsigned char* p_tile = smem + C::OFF_P;
   FwdMisc* misc = reinterpret_cast<FwdMisc*>(smem + C::OFF_MISC);
-  float* scratch = reinterpret_cast<float*>(p_tile);     // 32 KB, reused for the cross-row reductions
+  unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;      // edge flags of every cube
+  float* scratch = reinterpret_cast<float*>(p_tile);             // 32 KB, reused for the cross-row reductions
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_items = g.batch * g.Hq * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
 
+  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
   if (tid == 0) {
     misc->abort_flag = 0;
     tc::mbar_init(&misc->q_full, 1);
     tc::mbar_init(&misc->q_empty, 1);
     tc::mbar_init(&misc->o_full, 1);
-    tc::mbar_init(&misc->o_empty, 128);
-    for (int s = 0; s < kFwdSlots; ++s) {
-      tc::mbar_init(&misc->kv_full[s], 1);
-      tc::mbar_init(&misc->kv_empty[s], 1);
+    tc::mbar_init(&misc->o_empty, 256);
+    for (int s = 0; s < kFwdKSlots; ++s) {
+      tc::mbar_init(&misc->k_full[s], 1);
+      tc::mbar_init(&misc->k_empty[s], 1);
+    }
+    for (int s = 0; s < kFwdVSlots; ++s) {
+      tc::mbar_init(&misc->v_full[s], 1);
+      tc::mbar_init(&misc->v_empty[s], 1);
+    }
+    for (int s = 0; s < kFwdSBufs; ++s) {
+      tc::mbar_init(&misc->s_full[s], 1);
+      tc::mbar_init(&misc->s_free[s], 128);
     }
     for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(&misc->s_full[s], 1);
       tc::mbar_init(&misc->p_ready[s], 128);
       tc::mbar_init(&misc->p_free[s], 1);
     }
@@ -103,18 +125,31 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc::prefetch_tmap(&tm_v);
   }
   if (warp == 1) {
-    tc::tmem_alloc(&misc->tmem_base, 256);
+    tc::tmem_alloc(&misc->tmem_base, 512);
     tc::tmem_relinquish();
   }
   tc::tc_fence_before();
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
+  // tensor-memory columns: S^T buffers 0, 64, 128, 192; O^T 256
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t seq = 0, n_items = 0;
+  if (warp < 4) {
+    // (no register rebalancing)
+    if (warp == 0 || warp == 3) {
+      // ---------------------------------------------------------------- TMA producers: warp 0 streams the K pairs
+      // (and the Q tile), warp 3 the V pairs.  Lane 0 owns the barrier traffic; lanes 0 .. 2*DH-1 each issue one
+      // box (half h = lane / 2 of block lane & 1), so a pair costs one warp instruction instead of 2*DH.
+      // Each ring has one producer and one consumer, so a barrier's phase can never be two ahead of a waiter.
+      const int which = warp == 0 ? 0 : 1;                  // 0: K ring, 1: V ring
+      const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+      const uint32_t nslots = which == 0 ? kFwdKSlots : kFwdVSlots;
+      uint64_t* full = which == 0 ? misc->k_full : misc->v_full;
+      uint64_t* empty = which == 0 ? misc->k_empty : misc->v_empty;
+      unsigned char* ring = smem + (which == 0 ? 0 : kFwdKSlots * C::SLOT);
+      const int my_h = lane >> 1, my_blk = lane & 1;
+      const bool issuer = lane < 2 * C::DH;
+      uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         const int i = item % g.N, bhq = item / g.N;
         const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
@@ -122,118 +157,107 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int k = end - beg;
         if (k == 0) continue;
         const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
-        int it_, ih_, iw_;
-        cube_coords(g, i, it_, ih_, iw_);
-        VSA2_WAIT(&misc->q_empty, (n_items & 1) ^ 1);
-        tc::mbar_expect_tx(&misc->q_full, C::QBYTES);
-        for (int h = 0; h < C::DH; ++h)
-          tc::tma_load_5d(q_tile + h * C::SLAB, &tm_q, &misc->q_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+        if (which == 0) {
+          int it_, ih_, iw_;
+          cube_coords(g, i, it_, ih_, iw_);
+          int ok = 1;
+          if (lane == 0) {
+            ok = tc::mbar_wait(&misc->q_empty, (n_items & 1) ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&misc->q_full, C::QBYTES);
+          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+          if (lane < C::DH)
+            tc::tma_load_5d(q_tile + lane * C::SLAB, &tm_q, &misc->q_full, lane * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+        }
         ++n_items;
         const int nt = (k + 1) >> 1;
-        for (int t = 0; t < nt; ++t) {
-          const int ja = cols[2 * t], jb = (2 * t + 1 < k) ? cols[2 * t + 1] : ja;
-          int at, ah, aw, bt, bh_, bw;
-          cube_coords(g, ja, at, ah, aw);
-          cube_coords(g, jb, bt, bh_, bw);
-          {  // K pair: [half][A | B]
-            const uint32_t slot = seq % kFwdSlots, par = (seq / kFwdSlots) & 1;
-            unsigned char* dst = smem + slot * C::SLOT;
-            VSA2_WAIT(&misc->kv_empty[slot], par ^ 1);
-            tc::mbar_expect_tx(&misc->kv_full[slot], C::SLOT);
-            for (int h = 0; h < C::DH; ++h) {
-              tc::tma_load_5d(dst + (2 * h + 0) * C::SLAB, &tm_k, &misc->kv_full[slot], h * 64, aw * g.Bw, ah * g.Bh, at * g.Bt, bhk);
-              tc::tma_load_5d(dst + (2 * h + 1) * C::SLAB, &tm_k, &misc->kv_full[slot], h * 64, bw * g.Bw, bh_ * g.Bh, bt * g.Bt, bhk);
-            }
-            ++seq;
+        int j = cols[(my_blk == 1 && k > 1) ? 1 : 0];           // this lane's KV block of tile 0
+        for (int t = 0; t < nt; ++t, ++tg) {
+          int jt, jh, jw;
+          cube_coords(g, j, jt, jh, jw);
+          if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];   // next tile, fetched early
+          const uint32_t slot = tg % nslots, par = (tg / nslots) & 1;
+          int ok = 1;
+          if (lane == 0) {
+            ok = tc::mbar_wait(&empty[slot], par ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&full[slot], C::SLOT);
           }
-          {  // V pair: [A half0 .. | B half0 ..]
-            const uint32_t slot = seq % kFwdSlots, par = (seq / kFwdSlots) & 1;
-            unsigned char* dst = smem + slot * C::SLOT;
-            VSA2_WAIT(&misc->kv_empty[slot], par ^ 1);
-            tc::mbar_expect_tx(&misc->kv_full[slot], C::SLOT);
-            for (int h = 0; h < C::DH; ++h) {
-              tc::tma_load_5d(dst + (0 * C::DH + h) * C::SLAB, &tm_v, &misc->kv_full[slot], h * 64, aw * g.Bw, ah * g.Bh, at * g.Bt, bhk);
-              tc::tma_load_5d(dst + (1 * C::DH + h) * C::SLAB, &tm_v, &misc->kv_full[slot], h * 64, bw * g.Bw, bh_ * g.Bh, bt * g.Bt, bhk);
-            }
-            ++seq;
-          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+          if (issuer)
+            tc::tma_load_5d(ring + slot * C::SLOT + (2 * my_h + my_blk) * C::SLAB, tm, &full[slot], my_h * 64,
+                            jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
         }
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = tc::idesc_bf16(128, 64, false, false);
-      constexpr uint32_t idesc_o = tc::idesc_bf16(128, 64, true, true);
-      const uint32_t q_addr = tc::smem_u32(q_tile), p_addr = tc::smem_u32(p_tile), slot0 = tc::smem_u32(smem);
-      const uint32_t tm_o = tmem_base + 128;
-      uint32_t seq_k = 0;       // ring sequence number of the next K pair (its V pair is seq_k + 1)
-      uint32_t tt = 0;          // tiles issued so far (S buffer = tt & 1)
-      uint32_t n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
-        const int i = item % g.N, bhq = item / g.N;
-        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
-        const int k = end - beg;
-        if (k == 0) continue;
-        const int nt = (k + 1) >> 1;
-        VSA2_WAIT(&misc->q_full, n_items & 1);
-        tc::tc_fence_after();
-        for (int t = 0; t <= nt; ++t) {
-          if (t < nt) {   // S^T(t) = K_pair * Q^T
-            const uint32_t seq = seq_k + 2 * t, slot = seq % kFwdSlots, par = (seq / kFwdSlots) & 1;
-            VSA2_WAIT(&misc->kv_full[slot], par);
+    } else if (warp == 1) {
+      // ---------------------------------------------------------------- issuer of S^T(t) = K_pair * Q^T
+      if (lane == 0) {
+        const uint32_t q_addr = tc::smem_u32(q_tile), slot0 = tc::smem_u32(smem);
+        uint32_t tg = 0, n_items = 0;     // tg: tiles issued so far
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+          const int i = item % g.N, bhq = item / g.N;
+          const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+          if (k == 0) continue;
+          const int nt = (k + 1) >> 1;
+          VSA2_WAIT(&misc->q_full, n_items & 1);
+          for (int t = 0; t < nt; ++t, ++tg) {
+            const uint32_t slot = tg % kFwdKSlots, buf = tg % kFwdSBufs;
+            VSA2_WAIT(&misc->k_full[slot], (tg / kFwdKSlots) & 1);
+            VSA2_WAIT(&misc->s_free[buf], ((tg / kFwdSBufs) & 1) ^ 1);
             tc::tc_fence_after();
-            const uint32_t k_addr = slot0 + slot * C::SLOT, tm_s = tmem_base + ((tt + t) & 1) * 64;
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-              const uint32_t aa = k_addr + (ks / 4) * 2 * C::SLAB + (ks % 4) * 32;
-              const uint32_t bb = q_addr + (ks / 4) * C::SLAB + (ks % 4) * 32;
-              tc::mma_ss(tm_s, tc::smem_desc_sw128(aa, 16, 1024), tc::smem_desc_sw128(bb, 16, 1024), idesc_s, ks > 0);
-            }
-            tc::mma_commit(&misc->s_full[(tt + t) & 1]);
-            tc::mma_commit(&misc->kv_empty[slot]);
+            mma_pair_kmajor<D>(tmem_base + buf * 64, slot0 + slot * C::SLOT, q_addr);
+            tc::mma_commit(&misc->s_full[buf]);
+            tc::mma_commit(&misc->k_empty[slot]);
             if (t == nt - 1) tc::mma_commit(&misc->q_empty);
           }
-          if (t >= 1) {   // O^T += V_pair^T * P^T for tile t - 1
-            const uint32_t tp = tt + t - 1, buf = tp & 1;
-            const uint32_t seq = seq_k + 2 * (t - 1) + 1, slot = seq % kFwdSlots, par = (seq / kFwdSlots) & 1;
-            VSA2_WAIT(&misc->p_ready[buf], (tp >> 1) & 1);
-            VSA2_WAIT(&misc->kv_full[slot], par);
-            if (t == 1) VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
-            tc::tc_fence_after();
-            const uint32_t v_addr = slot0 + slot * C::SLOT;
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              const uint32_t aa = v_addr + (ks / 4) * C::DH * C::SLAB + (ks % 4) * 2048;
-              const uint32_t bb = p_addr + buf * C::PBYTES + ks * 2048;
-              tc::mma_ss(tm_o, tc::smem_desc_sw128(aa, C::DH == 2 ? C::SLAB : 0, 1024), tc::smem_desc_sw128(bb, 0, 1024),
-                         idesc_o, (t > 1) || (ks > 0));
-            }
-            tc::mma_commit(&misc->kv_empty[slot]);
-            tc::mma_commit(&misc->p_free[buf]);
-            if (t == nt) tc::mma_commit(&misc->o_full);
-          }
+          ++n_items;
         }
-        seq_k += 2 * nt;
-        tt += nt;
-        ++n_items;
+      }
+    } else if (warp == 2) {
+      // ---------------------------------------------------------------- issuer of O^T += V_pair^T * P^T
+      if (lane == 0) {
+        const uint32_t p_addr = tc::smem_u32(p_tile), slot0 = tc::smem_u32(smem);
+        uint32_t tg = 0, n_items = 0;
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+          const int i = item % g.N, bhq = item / g.N;
+          const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+          if (k == 0) continue;
+          const int nt = (k + 1) >> 1;
+          for (int t = 0; t < nt; ++t, ++tg) {
+            const uint32_t slot = tg % kFwdVSlots, buf = tg & 1;
+            VSA2_WAIT(&misc->v_full[slot], (tg / kFwdVSlots) & 1);
+            VSA2_WAIT(&misc->p_ready[buf], (tg >> 1) & 1);
+            if (t == 0) VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
+            tc::tc_fence_after();
+            mma_pairT_mnmajor<D>(tmem_base + 256, slot0 + (kFwdKSlots + slot) * C::SLOT, p_addr + buf * C::PBYTES, t > 0);
+            tc::mma_commit(&misc->v_empty[slot]);
+            tc::mma_commit(&misc->p_free[buf]);
+            if (t == nt - 1) tc::mma_commit(&misc->o_full);
+          }
+          ++n_items;
+        }
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax + epilogue (128 threads)
+    // ------------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
+    // (no register rebalancing)
+    const int wg = (warp >> 2) - 1;              // 0 or 1
     const int quad = warp & 3;
     const int row = (quad << 5) | lane;          // tensor-memory lane: key row in S^T, channel in O^T
-    const int sm_tid = tid - 64;                 // 0..127 inside this group
+    const int sm_tid = (tid - 128) & 127;        // 0..127 inside this warpgroup
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
-    uint32_t tt = 0, n_items = 0, n_all = 0;
+    unsigned char* my_p = p_tile + wg * C::PBYTES;
+    CubePos cpos;
+    cpos.init(g, row & 63);
+    const int blk = row >> 6;
+    uint32_t tg = 0, n_items = 0, n_all = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
       const int i = item % g.N, bhq = item / g.N;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
       const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
       const int tb = n_all & 1;
-      if (sm_tid < 64) {
+      if (wg == 0 && sm_tid < 64) {
         int it_, ih_, iw_;
         cube_coords(g, i, it_, ih_, iw_);
         const int l = cube_token(g, it_, ih_, iw_, sm_tid);
@@ -241,13 +265,14 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         misc->gate[tb][sm_tid] = (coarse && l >= 0) ? a.gate[(size_t)bhq * g.L + l] : 0.f;
       }
       const float oc_d = (coarse && row < D) ? a.oc_hat[((size_t)bhq * g.N + i) * D + row] : 0.f;
-      if (sm_tid == 0) misc->rescue_flag = 0;
-      tc::named_bar_sync(1, 128);
+      if (wg == 0 && sm_tid == 0) misc->rescue_flag = 0;
+      tc::named_bar_sync(3, 256);
+      const int q0 = wg * 32;                    // this warpgroup writes query columns q0 .. q0 + 31 in the epilogue
 
       if (k == 0) {
         // no selected block: O = gate * O_c, lse = -inf
         if (row < D) {
-          for (int qi = 0; qi < 64; ++qi) {
+          for (int qi = q0; qi < q0 + 32; ++qi) {
             const int l = misc->tok[tb][qi];
             if (l < 0) continue;
             const size_t idx = ((size_t)bhq * g.L + l) * D + row;
@@ -256,7 +281,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (a.o_res != nullptr) a.o_res[idx] = __float2bfloat16_rn(val - __bfloat162float(__float2bfloat16_rn(val)));
           }
         }
-        if (sm_tid < 64 && misc->tok[tb][sm_tid] >= 0) a.lse[(size_t)bhq * g.L + misc->tok[tb][sm_tid]] = -INFINITY;
+        if (wg == 0 && sm_tid < 64 && misc->tok[tb][sm_tid] >= 0) a.lse[(size_t)bhq * g.L + misc->tok[tb][sm_tid]] = -INFINITY;
         continue;
       }
 
@@ -264,75 +289,98 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #pragma unroll
       for (int c = 0; c < 64; ++c) l_part[c] = 0.f;
       const int nt = (k + 1) >> 1;
-      for (int t = 0; t < nt; ++t, ++tt) {
-        const uint32_t buf = tt & 1, use = (tt >> 1) & 1;
-        // validity of this thread's key row
-        const int blk = row >> 6;
-        const bool dup = (blk == 1) && (2 * t + 1 >= k);
-        const int j = cols[dup ? 2 * t : 2 * t + blk];
-        const bool valid = !dup && pos_valid(g, j, row & 63);
-        VSA2_WAIT(&misc->s_full[buf], use);
+      const int first_wg = tg & 1;               // warpgroup that owns tile 0 of this query block
+      if (wg == first_wg) {
+        // reference exponent of every query column = exact column maximum of the first tile
+        const uint32_t buf = tg % kFwdSBufs;
+        const bool valid = !((blk == 1) && k < 2) && cpos.valid(edge[cols[(blk == 1 && k > 1) ? 1 : 0]]);
+        VSA2_WAIT(&misc->s_full[buf], (tg / kFwdSBufs) & 1);
         tc::tc_fence_after();
         uint32_t s0[32], s1[32];
         tc::tmem_ld32(lane_addr + buf * 64, s0);
         tc::tmem_ld32(lane_addr + buf * 64 + 32, s1);
         tc::tmem_ld_wait();
-        if (t == 0) {
-          // reference exponent of every query column = exact column maximum of the first tile
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            scratch[scratch_idx(sm_tid, c)] = valid ? __uint_as_float(s0[c]) : -INFINITY;
-            scratch[scratch_idx(sm_tid, c + 32)] = valid ? __uint_as_float(s1[c]) : -INFINITY;
-          }
-          tc::named_bar_sync(1, 128);
-          if (sm_tid < 64) {
-            float mx = -INFINITY;
-            for (int r = 0; r < 128; ++r) mx = fmaxf(mx, scratch[scratch_idx(r, sm_tid)]);
-            misc->m_ref[sm_tid] = (mx > -INFINITY) ? mx * c2 : 0.f;
-          }
-          tc::named_bar_sync(1, 128);
+        for (int c = 0; c < 32; ++c) {
+          scratch[scratch_idx(sm_tid, c)] = valid ? __uint_as_float(s0[c]) : -INFINITY;
+          scratch[scratch_idx(sm_tid, c + 32)] = valid ? __uint_as_float(s1[c]) : -INFINITY;
         }
-        VSA2_WAIT(&misc->p_free[buf], use ^ 1);
-        uint32_t packed[32];
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float m0 = misc->m_ref[c], m1 = misc->m_ref[c + 1];
-          float p0 = ex2_approx(fmaf(__uint_as_float(s0[c]), c2, -m0));
-          float p1 = ex2_approx(fmaf(__uint_as_float(s0[c + 1]), c2, -m1));
-          p0 = valid ? p0 : 0.f;
-          p1 = valid ? p1 : 0.f;
-          l_part[c] += p0;
-          l_part[c + 1] += p1;
-          packed[c >> 1] = pack_bf16x2(p0, p1);
+        tc::named_bar_sync(1 + wg, 128);
+        if (sm_tid < 64) {
+          float mx = -INFINITY;
+          for (int r = 0; r < 128; ++r) mx = fmaxf(mx, scratch[scratch_idx(r, sm_tid)]);
+          misc->m_ref[sm_tid] = (mx > -INFINITY) ? mx * c2 : 0.f;
         }
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float m0 = misc->m_ref[32 + c], m1 = misc->m_ref[33 + c];
-          float p0 = ex2_approx(fmaf(__uint_as_float(s1[c]), c2, -m0));
-          float p1 = ex2_approx(fmaf(__uint_as_float(s1[c + 1]), c2, -m1));
-          p0 = valid ? p0 : 0.f;
-          p1 = valid ? p1 : 0.f;
-          l_part[32 + c] += p0;
-          l_part[33 + c] += p1;
-          packed[16 + (c >> 1)] = pack_bf16x2(p0, p1);
-        }
-        unsigned char* prow = p_tile + buf * C::PBYTES + row * 128;
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-          *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
-              make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
-        tc::fence_proxy_async_smem();
+      }
+      tc::named_bar_sync(3, 256);
+
+      for (int t = 0; t < nt; ++t, ++tg) {
+        if ((int)(tg & 1) != wg) continue;
+        const uint32_t buf = tg % kFwdSBufs;
+        const bool dup = (blk == 1) && (2 * t + 1 >= k);
+        const int j = cols[(blk == 1 && !dup) ? 2 * t + 1 : 2 * t];
+        const bool valid = !dup && cpos.valid(edge[j]);
+        const bool all_valid = __all_sync(0xffffffffu, valid);
+        VSA2_WAIT(&misc->s_full[buf], (tg / kFwdSBufs) & 1);
+        tc::tc_fence_after();
+        uint32_t sa[32], sb[32];
+        tc::tmem_ld32(lane_addr + buf * 64, sa);
+        tc::tmem_ld32(lane_addr + buf * 64 + 32, sb);
+        tc::tmem_ld_wait();
         tc::tc_fence_before();
-        tc::mbar_arrive(&misc->p_ready[buf]);
+        tc::mbar_arrive(&misc->s_free[buf]);
+        uint32_t packed[32];
+        const float4* mref4 = reinterpret_cast<const float4*>(misc->m_ref);
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 m = mref4[c4];
+          float p0 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 0]), c2, -m.x));
+          float p1 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 1]), c2, -m.y));
+          float p2 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 2]), c2, -m.z));
+          float p3 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 3]), c2, -m.w));
+          if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
+          l_part[4 * c4 + 0] += p0;
+          l_part[4 * c4 + 1] += p1;
+          l_part[4 * c4 + 2] += p2;
+          l_part[4 * c4 + 3] += p3;
+          packed[2 * c4] = pack_bf16x2(p0, p1);
+          packed[2 * c4 + 1] = pack_bf16x2(p2, p3);
+        }
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const float4 m = mref4[8 + c4];
+          float p0 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 0]), c2, -m.x));
+          float p1 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 1]), c2, -m.y));
+          float p2 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 2]), c2, -m.z));
+          float p3 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 3]), c2, -m.w));
+          if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
+          l_part[32 + 4 * c4 + 0] += p0;
+          l_part[32 + 4 * c4 + 1] += p1;
+          l_part[32 + 4 * c4 + 2] += p2;
+          l_part[32 + 4 * c4 + 3] += p3;
+          packed[16 + 2 * c4] = pack_bf16x2(p0, p1);
+          packed[16 + 2 * c4 + 1] = pack_bf16x2(p2, p3);
+        }
+        VSA2_WAIT(&misc->p_free[wg], ((tg >> 1) & 1) ^ 1);
+        store_row_sw128(my_p, row, packed);
+        tc::fence_proxy_async_smem();
+        tc::mbar_arrive(&misc->p_ready[wg]);
       }
 
-      // ---- epilogue of the query block
+      // ---- epilogue of the query block (both warpgroups)
       VSA2_WAIT(&misc->o_full, n_items & 1);
       tc::tc_fence_after();
+      if (wg == 0) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) scratch[scratch_idx(sm_tid, c)] = l_part[c];
-      tc::named_bar_sync(1, 128);
-      if (sm_tid < 64) {
+        for (int c = 0; c < 64; ++c) scratch[scratch_idx(sm_tid, c)] = l_part[c];
+      }
+      tc::named_bar_sync(3, 256);
+      if (wg == 1) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) scratch[scratch_idx(sm_tid, c)] += l_part[c];
+      }
+      tc::named_bar_sync(3, 256);
+      if (wg == 0 && sm_tid < 64) {
         float l = 0.f;
         for (int r = 0; r < 128; ++r) l += scratch[scratch_idx(r, sm_tid)];
         // sums outside the safe range (overflow, NaN or total underflow): hand the block to the exact kernel
@@ -341,28 +389,27 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int tk = misc->tok[tb][sm_tid];
         if (tk >= 0) a.lse[(size_t)bhq * g.L + tk] = (misc->m_ref[sm_tid] + __log2f(l)) * 0.6931471805599453f;
       }
-      tc::named_bar_sync(1, 128);
+      tc::named_bar_sync(3, 256);
       {
-        uint32_t o0[32], o1[32];
-        tc::tmem_ld32(lane_addr + 128, o0);
-        tc::tmem_ld32(lane_addr + 128 + 32, o1);
+        uint32_t o0[32];
+        tc::tmem_ld32(lane_addr + 256 + q0, o0);
         tc::tmem_ld_wait();
         tc::tc_fence_before();
         tc::mbar_arrive(&misc->o_empty);
         if (row < D) {
 #pragma unroll
-          for (int qi = 0; qi < 64; ++qi) {
+          for (int qq = 0; qq < 32; ++qq) {
+            const int qi = q0 + qq;
             const int l = misc->tok[tb][qi];
             if (l < 0) continue;
-            const float acc = __uint_as_float(qi < 32 ? o0[qi & 31] : o1[qi & 31]);
-            const float val = fmaf(misc->gate[tb][qi], oc_d, acc * misc->l_inv[qi]);
+            const float val = fmaf(misc->gate[tb][qi], oc_d, __uint_as_float(o0[qq]) * misc->l_inv[qi]);
             const size_t idx = ((size_t)bhq * g.L + l) * D + row;
             store_out(a.o, idx, val, g.out_f32);
             if (a.o_res != nullptr) a.o_res[idx] = __float2bfloat16_rn(val - __bfloat162float(__float2bfloat16_rn(val)));
           }
         }
       }
-      if (sm_tid == 0 && misc->rescue_flag) {
+      if (wg == 0 && sm_tid == 0 && misc->rescue_flag) {
         int slot = atomicAdd(a.rescue_count, 1);
         if (slot < kRescueCap) a.rescue_items[slot] = item;
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
@@ -384,7 +431,7 @@ done:
     }
     __syncthreads();
   }
-  if (warp == 1) tc::tmem_dealloc(tmem_base, 256);
+  if (warp == 1) tc::tmem_dealloc(tmem_base, 512);
 }
 
 cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
@@ -411,12 +458,15 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
   a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
+  if (g.N > kFwdMaxCubes) return cudaErrorInvalidValue;
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdTc<128>::smem_bytes))) return e;
-    fine_fwd_tc_kernel<128><<<grid, kFwdThreads, FwdTc<128>::smem_bytes, st>>>(tq, tk, tv, g, a);
+    const size_t smb = FwdTc<128>::smem_bytes(g.N);
+    if ((e = cudaFuncSetAttribute(fine_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_tc_kernel<128><<<grid, kFwdThreads, smb, st>>>(tq, tk, tv, g, a);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FwdTc<64>::smem_bytes))) return e;
-    fine_fwd_tc_kernel<64><<<grid, kFwdThreads, FwdTc<64>::smem_bytes, st>>>(tq, tk, tv, g, a);
+    const size_t smb = FwdTc<64>::smem_bytes(g.N);
+    if ((e = cudaFuncSetAttribute(fine_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_tc_kernel<64><<<grid, kFwdThreads, smb, st>>>(tq, tk, tv, g, a);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // query blocks whose row sums left the safe range are redone with the exact running maximum

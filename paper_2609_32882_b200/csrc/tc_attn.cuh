@@ -38,14 +38,16 @@ __device__ __forceinline__ void store_row_sw128(unsigned char* tile, int row, co
 
 // Issues the D/16 (K-major x K-major) instructions of  acc[128, 64] = A_pair[128, D] * B[64, D]^T.
 // A_pair: slot laid out [half][block A | block B] slabs; B: tile laid out [half] slabs.
+// The descriptors are built once and advanced by adding the (16-byte-unit) offset to the address field.
 template <int D>
 __device__ __forceinline__ void mma_pair_kmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile) {
   constexpr uint32_t idesc = tc::idesc_bf16(128, 64, false, false);
+  const uint64_t da = tc::smem_desc_sw128(a_slot, 16, 1024), db = tc::smem_desc_sw128(b_tile, 16, 1024);
 #pragma unroll
   for (int ks = 0; ks < D / 16; ++ks) {
-    const uint32_t aa = a_slot + (ks / 4) * 2 * kSlab + (ks % 4) * 32;
-    const uint32_t bb = b_tile + (ks / 4) * kSlab + (ks % 4) * 32;
-    tc::mma_ss(tm_acc, tc::smem_desc_sw128(aa, 16, 1024), tc::smem_desc_sw128(bb, 16, 1024), idesc, ks > 0);
+    const uint64_t oa = (uint64_t)(((ks / 4) * 2 * kSlab + (ks % 4) * 32) >> 4);
+    const uint64_t ob = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 32) >> 4);
+    tc::mma_ss(tm_acc, da + oa, db + ob, idesc, ks > 0);
   }
 }
 
@@ -55,14 +57,42 @@ template <int D>
 __device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, bool accumulate_first) {
   constexpr uint32_t idesc = tc::idesc_bf16(128, 64, true, true);
   constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;     // distance between the two 64-channel halves
+  const uint64_t da = tc::smem_desc_sw128(a_slot, lbo, 1024), db = tc::smem_desc_sw128(b_tile, 0, 1024);
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) {
-    const uint32_t aa = a_slot + (ks / 4) * kSlab + (ks % 4) * 2048;
-    const uint32_t bb = b_tile + ks * 2048;
-    tc::mma_ss(tm_acc, tc::smem_desc_sw128(aa, lbo, 1024), tc::smem_desc_sw128(bb, 0, 1024), idesc,
-               accumulate_first || (ks > 0));
+    const uint64_t oa = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 2048) >> 4);
+    const uint64_t ob = (uint64_t)((ks * 2048) >> 4);
+    tc::mma_ss(tm_acc, da + oa, db + ob, idesc, accumulate_first || (ks > 0));
   }
 }
+
+// Which cubes are cut by the grid boundary: bit 0 / 1 / 2 = last cube along t / h / w with a partial extent.
+__device__ __forceinline__ unsigned cube_edge_flags(const Geo& g, int n) {
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  unsigned f = 0;
+  if (nt == g.Nt - 1 && g.T % g.Bt) f |= 1u;
+  if (nh == g.Nh - 1 && g.H % g.Bh) f |= 2u;
+  if (nw == g.Nw - 1 && g.W % g.Bw) f |= 4u;
+  return f;
+}
+
+// Position of a token inside its cube and the test "is this position inside the valid grid for a cube with edge flags f".
+struct CubePos {
+  int bt, bh, bw, lt, lh, lw;   // coordinates of the position; valid extents of the last cube along each axis
+  __device__ __forceinline__ void init(const Geo& g, int pos) {
+    bw = pos % g.Bw;
+    int r = pos / g.Bw;
+    bh = r % g.Bh;
+    bt = r / g.Bh;
+    lt = g.T - (g.Nt - 1) * g.Bt;
+    lh = g.H - (g.Nh - 1) * g.Bh;
+    lw = g.W - (g.Nw - 1) * g.Bw;
+  }
+  __device__ __forceinline__ bool valid(unsigned f) const {
+    return (!(f & 1u) || bt < lt) && (!(f & 2u) || bh < lh) && (!(f & 4u) || bw < lw);
+  }
+};
 
 #define VSA2_WAIT(bar, parity)                                         \
   do {                                                                 \
