@@ -22,10 +22,9 @@
 
 namespace vsa2 {
 
-constexpr int kFwdThreads = 384;
-constexpr int kFwdKSlots = 3;   // ring of K pairs: filled by warp 0, drained by the S^T issuer
-constexpr int kFwdVSlots = 2;   // ring of V pairs: filled by warp 3, drained by the O^T issuer
-constexpr int kFwdSlots = kFwdKSlots + kFwdVSlots;
+constexpr int kFwdThreads = 512;
+constexpr int kFwdKSlots = 3;   // ring of K pairs: filled by warp 0, drained by the S^T issuers
+constexpr int kFwdVSlots = 2;   // ring of V pairs: filled by warp 1, drained by the O^T issuers
 constexpr int kFwdSBufs = 4;
 constexpr int kRescueCap = 16384;
 constexpr int kFwdMaxCubes = 12288;   // edge-flag table in shared memory: one byte per cube
@@ -37,10 +36,10 @@ struct FwdTc {
   static constexpr uint32_t SLOT = 2 * DH * SLAB;    // a K pair or a V pair, [half][A | B]
   static constexpr uint32_t QBYTES = DH * SLAB;
   static constexpr uint32_t PBYTES = 128 * 128;      // P^T: 128 key rows x 64 queries bf16
-  static constexpr uint32_t OFF_Q = kFwdSlots * SLOT;
+  static constexpr uint32_t OFF_Q = (kFwdKSlots + kFwdVSlots) * SLOT;
   static constexpr uint32_t OFF_P = OFF_Q + QBYTES;
   static constexpr uint32_t OFF_MISC = OFF_P + 2 * PBYTES;
-  static constexpr uint32_t MISC_BYTES = 2048;
+  static constexpr uint32_t MISC_BYTES = 5120;
   static size_t smem_bytes(int n_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_cubes + 15) / 16 * 16 + 1024; }
 };
 
@@ -53,11 +52,13 @@ struct FwdMisc {
   uint32_t tmem_base;
   int abort_flag;
   int rescue_flag;
-  alignas(16) float m_ref[64];   // per query column: reference exponent (log2 units); read as float4
+  alignas(16) float m_ref[64];     // per query column: reference exponent (log2 units); read as float4
   alignas(16) float l_inv[64];
-  int tok[2][64];           // raster token of each query position (-1 = padding), by item parity
+  alignas(16) float red[8][64];    // per-warp partial column reductions
+  int tok[2][64];                  // raster token of each query position (-1 = padding), by item parity
   float gate[2][64];
 };
+static_assert(sizeof(FwdMisc) <= 5120, "misc region too small");
 
 struct FwdArgs {
   const float* gate;
@@ -72,13 +73,16 @@ struct FwdArgs {
   int* rescue_items;
 };
 
-// Roles (384 threads = 3 warpgroups):
-//   warpgroup 0: warps 0 and 3 = TMA producers (K pairs + Q tile, V pairs), warp 1 = issuer of the S^T products,
-//                warp 2 = issuer of the O^T products (one elected lane each; the work is split because one thread
-//                cannot issue a tile's 8 copies, 16 MMAs, commits and waits fast enough).  Gives most of its
-//                registers away.
-//   warpgroups 1, 2: softmax + epilogue; warpgroup w handles the tiles with (global tile index & 1) == w - 1, so two
-//                tiles are in the exponential unit at any time.  A warp owns tensor-memory lane quadrant warp % 4.
+// Roles (512 threads = 4 warpgroups).  An issuing thread needs ~60 cycles per MMA plus ~100-200 per barrier
+// operation, more than the 48 cycles an N = 64 MMA takes to execute, so issue and copy work is spread:
+//   warpgroups 0, 1 (few registers): warp 0 = TMA producer of the K pairs and the Q tile, warp 1 = TMA producer of the
+//       V pairs (lane 0 owns the barriers, lanes 0 .. 2*D/64-1 each issue one box), warps 2, 3 = issuers of the S^T
+//       products of the even / odd tiles, warps 4, 5 = issuers of the O^T products of the even / odd tiles (each
+//       into its own accumulator, summed in the epilogue), warps 6, 7 idle.
+//   warpgroups 2, 3: softmax + epilogue; warpgroup w handles the tiles with (global tile index & 1) == w - 2, so two
+//       tiles are in the exponential unit at any time.  A warp owns tensor-memory lane quadrant warp % 4.
+// Every mbarrier has one producing role and one consuming role (or all consumers see every phase), so a phase can
+// never run two ahead of a waiter.
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -90,7 +94,6 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   unsigned char* p_tile = smem + C::OFF_P;
   FwdMisc* misc = reinterpret_cast<FwdMisc*>(smem + C::OFF_MISC);
   unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;      // edge flags of every cube
-  float* scratch = reinterpret_cast<float*>(p_tile);             // 32 KB, reused for the cross-row reductions
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_items = g.batch * g.Hq * g.N;
@@ -100,8 +103,8 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   if (tid == 0) {
     misc->abort_flag = 0;
     tc::mbar_init(&misc->q_full, 1);
-    tc::mbar_init(&misc->q_empty, 1);
-    tc::mbar_init(&misc->o_full, 1);
+    tc::mbar_init(&misc->q_empty, 2);      // both S^T issuers
+    tc::mbar_init(&misc->o_full, 2);       // both O^T issuers
     tc::mbar_init(&misc->o_empty, 256);
     for (int s = 0; s < kFwdKSlots; ++s) {
       tc::mbar_init(&misc->k_full[s], 1);
@@ -124,7 +127,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc::prefetch_tmap(&tm_k);
     tc::prefetch_tmap(&tm_v);
   }
-  if (warp == 1) {
+  if (warp == 2) {
     tc::tmem_alloc(&misc->tmem_base, 512);
     tc::tmem_relinquish();
   }
@@ -132,16 +135,13 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
-  // tensor-memory columns: S^T buffers 0, 64, 128, 192; O^T 256
+  // tensor-memory columns: S^T buffers 0, 64, 128, 192; O^T of the even tiles 256, of the odd tiles 320
 
-  if (warp < 4) {
-    // (no register rebalancing)
-    if (warp == 0 || warp == 3) {
-      // ---------------------------------------------------------------- TMA producers: warp 0 streams the K pairs
-      // (and the Q tile), warp 3 the V pairs.  Lane 0 owns the barrier traffic; lanes 0 .. 2*DH-1 each issue one
-      // box (half h = lane / 2 of block lane & 1), so a pair costs one warp instruction instead of 2*DH.
-      // Each ring has one producer and one consumer, so a barrier's phase can never be two ahead of a waiter.
-      const int which = warp == 0 ? 0 : 1;                  // 0: K ring, 1: V ring
+  if (warp < 8) {
+    tc::reg_dec<56>();
+    if (warp < 2) {
+      // ---------------------------------------------------------------- TMA producers
+      const int which = warp;                               // 0: K ring (+ Q tile), 1: V ring
       const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
       const uint32_t nslots = which == 0 ? kFwdKSlots : kFwdVSlots;
       uint64_t* full = which == 0 ? misc->k_full : misc->v_full;
@@ -188,18 +188,21 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                             jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
         }
       }
-    } else if (warp == 1) {
-      // ---------------------------------------------------------------- issuer of S^T(t) = K_pair * Q^T
+    } else if (warp < 4) {
+      // ---------------------------------------------------------------- issuers of S^T(t) = K_pair * Q^T
       if (lane == 0) {
+        const uint32_t mine = warp - 2;            // parity of the tiles this warp issues
         const uint32_t q_addr = tc::smem_u32(q_tile), slot0 = tc::smem_u32(smem);
-        uint32_t tg = 0, n_items = 0;     // tg: tiles issued so far
+        uint32_t tg = 0, n_items = 0;
         for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
           const int i = item % g.N, bhq = item / g.N;
           const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
           if (k == 0) continue;
           const int nt = (k + 1) >> 1;
           VSA2_WAIT(&misc->q_full, n_items & 1);
+          bool issued = false;
           for (int t = 0; t < nt; ++t, ++tg) {
+            if ((tg & 1) != mine) continue;
             const uint32_t slot = tg % kFwdKSlots, buf = tg % kFwdSBufs;
             VSA2_WAIT(&misc->k_full[slot], (tg / kFwdKSlots) & 1);
             VSA2_WAIT(&misc->s_free[buf], ((tg / kFwdSBufs) & 1) ^ 1);
@@ -207,43 +210,53 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             mma_pair_kmajor<D>(tmem_base + buf * 64, slot0 + slot * C::SLOT, q_addr);
             tc::mma_commit(&misc->s_full[buf]);
             tc::mma_commit(&misc->k_empty[slot]);
-            if (t == nt - 1) tc::mma_commit(&misc->q_empty);
+            issued = true;
           }
+          // the Q tile may be replaced once both issuers are through with it
+          if (issued) tc::mma_commit(&misc->q_empty);
+          else tc::mbar_arrive(&misc->q_empty);
           ++n_items;
         }
       }
-    } else if (warp == 2) {
-      // ---------------------------------------------------------------- issuer of O^T += V_pair^T * P^T
+    } else if (warp < 6) {
+      // ---------------------------------------------------------------- issuers of O^T += V_pair^T * P^T
       if (lane == 0) {
+        const uint32_t mine = warp - 4;
         const uint32_t p_addr = tc::smem_u32(p_tile), slot0 = tc::smem_u32(smem);
+        const uint32_t tm_o = tmem_base + 256 + mine * 64;
         uint32_t tg = 0, n_items = 0;
         for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
           const int i = item % g.N, bhq = item / g.N;
           const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
           if (k == 0) continue;
           const int nt = (k + 1) >> 1;
+          VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous query block's accumulators were read out
+          bool issued = false;
           for (int t = 0; t < nt; ++t, ++tg) {
-            const uint32_t slot = tg % kFwdVSlots, buf = tg & 1;
+            if ((tg & 1) != mine) continue;
+            const uint32_t slot = tg % kFwdVSlots;
             VSA2_WAIT(&misc->v_full[slot], (tg / kFwdVSlots) & 1);
-            VSA2_WAIT(&misc->p_ready[buf], (tg >> 1) & 1);
-            if (t == 0) VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
+            VSA2_WAIT(&misc->p_ready[mine], (tg >> 1) & 1);
             tc::tc_fence_after();
-            mma_pairT_mnmajor<D>(tmem_base + 256, slot0 + (kFwdKSlots + slot) * C::SLOT, p_addr + buf * C::PBYTES, t > 0);
+            mma_pairT_mnmajor<D>(tm_o, slot0 + (kFwdKSlots + slot) * C::SLOT, p_addr + mine * C::PBYTES, issued);
             tc::mma_commit(&misc->v_empty[slot]);
-            tc::mma_commit(&misc->p_free[buf]);
-            if (t == nt - 1) tc::mma_commit(&misc->o_full);
+            tc::mma_commit(&misc->p_free[mine]);
+            issued = true;
           }
+          if (issued) tc::mma_commit(&misc->o_full);
+          else tc::mbar_arrive(&misc->o_full);
           ++n_items;
         }
       }
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
-    // (no register rebalancing)
-    const int wg = (warp >> 2) - 1;              // 0 or 1
+    tc::reg_inc<200>();
+    const int wg = (warp >> 2) - 2;              // 0 or 1
     const int quad = warp & 3;
     const int row = (quad << 5) | lane;          // tensor-memory lane: key row in S^T, channel in O^T
-    const int sm_tid = (tid - 128) & 127;        // 0..127 inside this warpgroup
+    const int sm_tid = tid & 127;                // 0..127 inside this warpgroup
+    const int sm_warp = warp - 8;                // 0..7 over both warpgroups
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
     unsigned char* my_p = p_tile + wg * C::PBYTES;
@@ -266,155 +279,196 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       }
       const float oc_d = (coarse && row < D) ? a.oc_hat[((size_t)bhq * g.N + i) * D + row] : 0.f;
       if (wg == 0 && sm_tid == 0) misc->rescue_flag = 0;
-      tc::named_bar_sync(3, 256);
       const int q0 = wg * 32;                    // this warpgroup writes query columns q0 .. q0 + 31 in the epilogue
-
-      if (k == 0) {
-        // no selected block: O = gate * O_c, lse = -inf
-        if (row < D) {
-          for (int qi = q0; qi < q0 + 32; ++qi) {
-            const int l = misc->tok[tb][qi];
-            if (l < 0) continue;
-            const size_t idx = ((size_t)bhq * g.L + l) * D + row;
-            const float val = misc->gate[tb][qi] * oc_d;
-            store_out(a.o, idx, val, g.out_f32);
-            if (a.o_res != nullptr) a.o_res[idx] = __float2bfloat16_rn(val - __bfloat162float(__float2bfloat16_rn(val)));
-          }
-        }
-        if (wg == 0 && sm_tid < 64 && misc->tok[tb][sm_tid] >= 0) a.lse[(size_t)bhq * g.L + misc->tok[tb][sm_tid]] = -INFINITY;
-        continue;
-      }
 
       float l_part[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) l_part[c] = 0.f;
       const int nt = (k + 1) >> 1;
-      const int first_wg = tg & 1;               // warpgroup that owns tile 0 of this query block
-      if (wg == first_wg) {
-        // reference exponent of every query column = exact column maximum of the first tile
-        const uint32_t buf = tg % kFwdSBufs;
-        const bool valid = !((blk == 1) && k < 2) && cpos.valid(edge[cols[(blk == 1 && k > 1) ? 1 : 0]]);
-        VSA2_WAIT(&misc->s_full[buf], (tg / kFwdSBufs) & 1);
-        tc::tc_fence_after();
-        uint32_t s0[32], s1[32];
-        tc::tmem_ld32(lane_addr + buf * 64, s0);
-        tc::tmem_ld32(lane_addr + buf * 64 + 32, s1);
-        tc::tmem_ld_wait();
+      const uint32_t tg0 = tg;
+      if (k > 0) {
+        const int first_wg = tg & 1;               // warpgroup that owns tile 0 of this query block
+        if (wg == first_wg) {
+          // reference exponent of every query column = exact column maximum of the first tile
+          const uint32_t buf = tg % kFwdSBufs;
+          const bool valid = !((blk == 1) && k < 2) && cpos.valid(edge[cols[(blk == 1 && k > 1) ? 1 : 0]]);
+          VSA2_WAIT(&misc->s_full[buf], (tg / kFwdSBufs) & 1);
+          tc::tc_fence_after();
+          uint32_t s0[32], s1[32];
+          tc::tmem_ld32(lane_addr + buf * 64, s0);
+          tc::tmem_ld32(lane_addr + buf * 64 + 32, s1);
+          tc::tmem_ld_wait();
+          float mx[64];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          scratch[scratch_idx(sm_tid, c)] = valid ? __uint_as_float(s0[c]) : -INFINITY;
-          scratch[scratch_idx(sm_tid, c + 32)] = valid ? __uint_as_float(s1[c]) : -INFINITY;
-        }
-        tc::named_bar_sync(1 + wg, 128);
-        if (sm_tid < 64) {
-          float mx = -INFINITY;
-          for (int r = 0; r < 128; ++r) mx = fmaxf(mx, scratch[scratch_idx(r, sm_tid)]);
-          misc->m_ref[sm_tid] = (mx > -INFINITY) ? mx * c2 : 0.f;
-        }
-      }
-      tc::named_bar_sync(3, 256);
-
-      for (int t = 0; t < nt; ++t, ++tg) {
-        if ((int)(tg & 1) != wg) continue;
-        const uint32_t buf = tg % kFwdSBufs;
-        const bool dup = (blk == 1) && (2 * t + 1 >= k);
-        const int j = cols[(blk == 1 && !dup) ? 2 * t + 1 : 2 * t];
-        const bool valid = !dup && cpos.valid(edge[j]);
-        const bool all_valid = __all_sync(0xffffffffu, valid);
-        VSA2_WAIT(&misc->s_full[buf], (tg / kFwdSBufs) & 1);
-        tc::tc_fence_after();
-        uint32_t sa[32], sb[32];
-        tc::tmem_ld32(lane_addr + buf * 64, sa);
-        tc::tmem_ld32(lane_addr + buf * 64 + 32, sb);
-        tc::tmem_ld_wait();
-        tc::tc_fence_before();
-        tc::mbar_arrive(&misc->s_free[buf]);
-        uint32_t packed[32];
-        const float4* mref4 = reinterpret_cast<const float4*>(misc->m_ref);
-#pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4) {
-          const float4 m = mref4[c4];
-          float p0 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 0]), c2, -m.x));
-          float p1 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 1]), c2, -m.y));
-          float p2 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 2]), c2, -m.z));
-          float p3 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 3]), c2, -m.w));
-          if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
-          l_part[4 * c4 + 0] += p0;
-          l_part[4 * c4 + 1] += p1;
-          l_part[4 * c4 + 2] += p2;
-          l_part[4 * c4 + 3] += p3;
-          packed[2 * c4] = pack_bf16x2(p0, p1);
-          packed[2 * c4 + 1] = pack_bf16x2(p2, p3);
-        }
-#pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4) {
-          const float4 m = mref4[8 + c4];
-          float p0 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 0]), c2, -m.x));
-          float p1 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 1]), c2, -m.y));
-          float p2 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 2]), c2, -m.z));
-          float p3 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 3]), c2, -m.w));
-          if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
-          l_part[32 + 4 * c4 + 0] += p0;
-          l_part[32 + 4 * c4 + 1] += p1;
-          l_part[32 + 4 * c4 + 2] += p2;
-          l_part[32 + 4 * c4 + 3] += p3;
-          packed[16 + 2 * c4] = pack_bf16x2(p0, p1);
-          packed[16 + 2 * c4 + 1] = pack_bf16x2(p2, p3);
-        }
-        VSA2_WAIT(&misc->p_free[wg], ((tg >> 1) & 1) ^ 1);
-        store_row_sw128(my_p, row, packed);
-        tc::fence_proxy_async_smem();
-        tc::mbar_arrive(&misc->p_ready[wg]);
-      }
-
-      // ---- epilogue of the query block (both warpgroups)
-      VSA2_WAIT(&misc->o_full, n_items & 1);
-      tc::tc_fence_after();
-      if (wg == 0) {
-#pragma unroll
-        for (int c = 0; c < 64; ++c) scratch[scratch_idx(sm_tid, c)] = l_part[c];
-      }
-      tc::named_bar_sync(3, 256);
-      if (wg == 1) {
-#pragma unroll
-        for (int c = 0; c < 64; ++c) scratch[scratch_idx(sm_tid, c)] += l_part[c];
-      }
-      tc::named_bar_sync(3, 256);
-      if (wg == 0 && sm_tid < 64) {
-        float l = 0.f;
-        for (int r = 0; r < 128; ++r) l += scratch[scratch_idx(r, sm_tid)];
-        // sums outside the safe range (overflow, NaN or total underflow): hand the block to the exact kernel
-        if (!(l > 1e-30f && l < 1e30f)) misc->rescue_flag = 1;
-        misc->l_inv[sm_tid] = 1.f / l;
-        const int tk = misc->tok[tb][sm_tid];
-        if (tk >= 0) a.lse[(size_t)bhq * g.L + tk] = (misc->m_ref[sm_tid] + __log2f(l)) * 0.6931471805599453f;
-      }
-      tc::named_bar_sync(3, 256);
-      {
-        uint32_t o0[32];
-        tc::tmem_ld32(lane_addr + 256 + q0, o0);
-        tc::tmem_ld_wait();
-        tc::tc_fence_before();
-        tc::mbar_arrive(&misc->o_empty);
-        if (row < D) {
-#pragma unroll
-          for (int qq = 0; qq < 32; ++qq) {
-            const int qi = q0 + qq;
-            const int l = misc->tok[tb][qi];
-            if (l < 0) continue;
-            const float val = fmaf(misc->gate[tb][qi], oc_d, __uint_as_float(o0[qq]) * misc->l_inv[qi]);
-            const size_t idx = ((size_t)bhq * g.L + l) * D + row;
-            store_out(a.o, idx, val, g.out_f32);
-            if (a.o_res != nullptr) a.o_res[idx] = __float2bfloat16_rn(val - __bfloat162float(__float2bfloat16_rn(val)));
+          for (int c = 0; c < 32; ++c) {
+            mx[c] = valid ? __uint_as_float(s0[c]) : -INFINITY;
+            mx[c + 32] = valid ? __uint_as_float(s1[c]) : -INFINITY;
+          }
+          warp_reduce_cols64<true>(mx, lane);
+          const int cb = warp_reduce_col(lane);
+          misc->red[quad][cb] = mx[0];
+          misc->red[quad][cb + 1] = mx[1];
+          tc::named_bar_sync(1 + wg, 128);
+          if (sm_tid < 64) {
+            const float m4 = fmaxf(fmaxf(misc->red[0][sm_tid], misc->red[1][sm_tid]), fmaxf(misc->red[2][sm_tid], misc->red[3][sm_tid]));
+            misc->m_ref[sm_tid] = (m4 > -INFINITY) ? m4 * c2 : 0.f;
           }
         }
       }
-      if (wg == 0 && sm_tid == 0 && misc->rescue_flag) {
+      tc::named_bar_sync(3, 256);       // tables and reference exponents visible to both warpgroups
+
+      if (k > 0) {
+        // first own tile of this query block and the KV block of this thread's key row in it
+        int t_own = ((tg & 1) == (uint32_t)wg) ? 0 : 1;
+        int j_next = 0;
+        if (t_own < nt) j_next = cols[(blk == 1 && 2 * t_own + 1 < k) ? 2 * t_own + 1 : 2 * t_own];
+        for (int t = t_own; t < nt; t += 2) {
+          const uint32_t tgt = tg0 + t, buf = tgt % kFwdSBufs;
+          const bool dup = (blk == 1) && (2 * t + 1 >= k);
+          const bool valid = !dup && cpos.valid(edge[j_next]);
+          if (t + 2 < nt) j_next = cols[(blk == 1 && 2 * t + 5 < k) ? 2 * t + 5 : 2 * t + 4];   // next own tile, fetched early
+          const bool all_valid = __all_sync(0xffffffffu, valid);
+          VSA2_WAIT(&misc->s_full[buf], (tgt / kFwdSBufs) & 1);
+          tc::tc_fence_after();
+          uint32_t sa[32], sb[32];
+          tc::tmem_ld32(lane_addr + buf * 64, sa);
+          tc::tmem_ld32(lane_addr + buf * 64 + 32, sb);
+          tc::tmem_ld_wait();
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->s_free[buf]);
+          uint32_t packed[32];
+          const float4* mref4 = reinterpret_cast<const float4*>(misc->m_ref);
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 m = mref4[c4];
+            float p0 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 0]), c2, -m.x));
+            float p1 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 1]), c2, -m.y));
+            float p2 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 2]), c2, -m.z));
+            float p3 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 3]), c2, -m.w));
+            if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
+            l_part[4 * c4 + 0] += p0;
+            l_part[4 * c4 + 1] += p1;
+            l_part[4 * c4 + 2] += p2;
+            l_part[4 * c4 + 3] += p3;
+            packed[2 * c4] = pack_bf16x2(p0, p1);
+            packed[2 * c4 + 1] = pack_bf16x2(p2, p3);
+          }
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 m = mref4[8 + c4];
+            float p0 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 0]), c2, -m.x));
+            float p1 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 1]), c2, -m.y));
+            float p2 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 2]), c2, -m.z));
+            float p3 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 3]), c2, -m.w));
+            if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
+            l_part[32 + 4 * c4 + 0] += p0;
+            l_part[32 + 4 * c4 + 1] += p1;
+            l_part[32 + 4 * c4 + 2] += p2;
+            l_part[32 + 4 * c4 + 3] += p3;
+            packed[16 + 2 * c4] = pack_bf16x2(p0, p1);
+            packed[16 + 2 * c4 + 1] = pack_bf16x2(p2, p3);
+          }
+          VSA2_WAIT(&misc->p_free[wg], ((tgt >> 1) & 1) ^ 1);
+          store_row_sw128(my_p, row, packed);
+          tc::fence_proxy_async_smem();
+          tc::mbar_arrive(&misc->p_ready[wg]);
+        }
+        tg += nt;
+
+        // ---- epilogue of the query block (both warpgroups): row sums over all 256 key rows x tiles
+        warp_reduce_cols64<false>(l_part, lane);
+        {
+          const int cb = warp_reduce_col(lane);
+          misc->red[sm_warp][cb] = l_part[0];
+          misc->red[sm_warp][cb + 1] = l_part[1];
+        }
+        tc::named_bar_sync(3, 256);
+        if (wg == 0 && sm_tid < 64) {
+          float l = 0.f;
+#pragma unroll
+          for (int w = 0; w < 8; ++w) l += misc->red[w][sm_tid];
+          // sums outside the safe range (overflow, NaN or total underflow): hand the block to the exact kernel
+          if (!(l > 1e-30f && l < 1e30f)) misc->rescue_flag = 1;
+          misc->l_inv[sm_tid] = 1.f / l;
+          const int tk = misc->tok[tb][sm_tid];
+          if (tk >= 0) a.lse[(size_t)bhq * g.L + tk] = (misc->m_ref[sm_tid] + __log2f(l)) * 0.6931471805599453f;
+        }
+        VSA2_WAIT(&misc->o_full, n_items & 1);
+        tc::tc_fence_after();
+        tc::named_bar_sync(3, 256);
+      }
+
+      // O[l, d] = (O_even^T + O_odd^T)[d, q] / l[q] + gate[q] * O_c[d]; this warpgroup owns 32 query columns
+      {
+        float acc[32];
+        if (k > 0) {
+          uint32_t o0[32];
+          tc::tmem_ld32(lane_addr + 256 + (tg0 & 1) * 64 + q0, o0);       // accumulator of the parity that saw tile 0
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) acc[c] = __uint_as_float(o0[c]);
+          if (nt > 1) {
+            tc::tmem_ld32(lane_addr + 256 + ((tg0 & 1) ^ 1) * 64 + q0, o0);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) acc[c] += __uint_as_float(o0[c]);
+          }
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->o_empty);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) acc[c] = 0.f;
+        }
+        if (g.out_f32 || a.o_res == nullptr) {
+          // plain stores (validation paths): one element per thread and query
+          if (row < D) {
+#pragma unroll
+            for (int qq = 0; qq < 32; ++qq) {
+              const int qi = q0 + qq;
+              const int l = misc->tok[tb][qi];
+              if (l < 0) continue;
+              const float val = fmaf(misc->gate[tb][qi], oc_d, k > 0 ? acc[qq] * misc->l_inv[qi] : 0.f);
+              const size_t idx = ((size_t)bhq * g.L + l) * D + row;
+              store_out(a.o, idx, val, g.out_f32);
+              if (a.o_res != nullptr) a.o_res[idx] = __float2bfloat16_rn(val - __bfloat162float(__float2bfloat16_rn(val)));
+            }
+          }
+        } else {
+          // bf16 output and residual: transpose through shared memory (the P^T buffers are idle now), then 16-byte stores
+          bf16* st_o = reinterpret_cast<bf16*>(p_tile);                 // [64 q][D]
+          bf16* st_r = reinterpret_cast<bf16*>(p_tile + C::PBYTES);     // [64 q][D]
+          if (row < D) {
+#pragma unroll
+            for (int qq = 0; qq < 32; ++qq) {
+              const int qi = q0 + qq;
+              const float val = fmaf(misc->gate[tb][qi], oc_d, k > 0 ? acc[qq] * misc->l_inv[qi] : 0.f);
+              const bf16 vb = __float2bfloat16_rn(val);
+              st_o[qi * D + row] = vb;
+              st_r[qi * D + row] = __float2bfloat16_rn(val - __bfloat162float(vb));
+            }
+          }
+          tc::named_bar_sync(3, 256);
+          constexpr int CH = D / 8;                                      // 16-byte chunks per token row
+          const int t256 = tid - 256;
+          for (int e = t256; e < 64 * CH; e += 256) {
+            const int qi = e / CH, ch = e % CH;
+            const int l = misc->tok[tb][qi];
+            if (l < 0) continue;
+            const size_t idx = ((size_t)bhq * g.L + l) * D + ch * 8;
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.o) + idx) = *reinterpret_cast<const uint4*>(st_o + qi * D + ch * 8);
+            *reinterpret_cast<uint4*>(a.o_res + idx) = *reinterpret_cast<const uint4*>(st_r + qi * D + ch * 8);
+          }
+          tc::named_bar_sync(3, 256);        // staging buffers free before the next query block writes P^T
+        }
+      }
+      if (k == 0 && wg == 0 && sm_tid < 64 && misc->tok[tb][sm_tid] >= 0)
+        a.lse[(size_t)bhq * g.L + misc->tok[tb][sm_tid]] = -INFINITY;
+      if (k > 0 && wg == 0 && sm_tid == 0 && misc->rescue_flag) {
         int slot = atomicAdd(a.rescue_count, 1);
         if (slot < kRescueCap) a.rescue_items[slot] = item;
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
       }
-      ++n_items;
+      if (k > 0) ++n_items;
     }
   }
 
@@ -431,7 +485,7 @@ done:
     }
     __syncthreads();
   }
-  if (warp == 1) tc::tmem_dealloc(tmem_base, 512);
+  if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
 }
 
 cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
