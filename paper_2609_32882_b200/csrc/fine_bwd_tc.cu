@@ -24,32 +24,53 @@
 
 namespace vsa2 {
 
-constexpr int kBwdThreads = 192;
-constexpr int kBwdSlots = 4;
+constexpr int kBwdThreads = 256;
+constexpr int kBwdMaxCubes = 12288;   // edge-flag table in shared memory: one byte per cube
 
+// Shared-memory plan of both passes (D = 128: 4 x 32 KB ring slots, 2 x 16 KB stationary tiles, 2 x 16 KB operand
+// buffers): ring A = 2 slots, ring B = 2 slots, each with one producing warp and fixed consuming roles.
 template <int D>
 struct BwdTc {
   static constexpr int DH = D / 64;
   static constexpr uint32_t SLOT = 2 * DH * kSlab;   // a pair of cube tiles, [half][A | B]
   static constexpr uint32_t TILE = DH * kSlab;       // one cube tile, [half]
   static constexpr uint32_t PBYTES = 128 * 128;      // 128 rows x 64 bf16
-  static constexpr uint32_t OFF_ST0 = kBwdSlots * SLOT;        // stationary tile 0 (Q or K)
+  static constexpr uint32_t OFF_RING_B = 2 * SLOT;
+  static constexpr uint32_t OFF_ST0 = 4 * SLOT;                // stationary tile 0 (Q or K)
   static constexpr uint32_t OFF_ST1 = OFF_ST0 + TILE;          // stationary tile 1 (dO or V)
   static constexpr uint32_t OFF_P = OFF_ST1 + TILE;            // two 16 KB operand buffers
   static constexpr uint32_t OFF_MISC = OFF_P + 2 * PBYTES;
-  static constexpr size_t smem_bytes = OFF_MISC + 4096 + 1024;
+  static constexpr uint32_t MISC_BYTES = 3072;
+  static size_t smem_bytes(int n_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_cubes + 15) / 16 * 16 + 1024; }
 };
 
 struct BwdMisc {
   uint64_t st_full, st_empty, o_full, o_empty;
-  uint64_t ring_full[kBwdSlots], ring_empty[kBwdSlots];
-  uint64_t sdp_full[2], ds_ready[2], ds_free[2];
+  uint64_t a_full[2], a_empty[2], b_full[2], b_empty[2];      // the two rings
+  uint64_t sdp_full[2], sdp_free[2], ds_ready[2], ds_free[2];
   uint32_t tmem_base;
   int abort_flag;
-  float lse2[2][64];     // dQ pass: per query column, lse * log2(e) (+inf for padding), by item parity
-  float delta[2][64];
+  alignas(16) float lse2[2][64];   // dQ pass: per query column, lse * log2(e) (+inf for padding), by item parity
+  alignas(16) float delta[2][64];
   int tok[2][64];
 };
+static_assert(sizeof(BwdMisc) <= 3072, "misc region too small");
+
+// One warp streams pairs of cube tiles into a two-slot ring: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one box
+// each (half h = lane / 2 of block lane & 1).  `coord_*`: cube coordinates of this lane's block, `bh`: its head index.
+#define VSA2_RING_LOAD(FULL, EMPTY, RING_BASE, TMAP, SEQ, CT, CH, CW, BH)                                         \
+  do {                                                                                                            \
+    const uint32_t slot_ = (SEQ) & 1, par_ = ((SEQ) >> 1) & 1;                                                    \
+    int ok_ = 1;                                                                                                  \
+    if (lane == 0) {                                                                                              \
+      ok_ = tc::mbar_wait(&(EMPTY)[slot_], par_ ^ 1, &misc->abort_flag);                                          \
+      if (ok_) tc::mbar_expect_tx(&(FULL)[slot_], C::SLOT);                                                       \
+    }                                                                                                             \
+    if (!__shfl_sync(0xffffffffu, ok_, 0)) goto done;                                                             \
+    if (lane < 2 * C::DH)                                                                                         \
+      tc::tma_load_5d((RING_BASE) + slot_ * C::SLOT + (2 * (lane >> 1) + (lane & 1)) * kSlab, (TMAP), &(FULL)[slot_], \
+                      (lane >> 1) * 64, (CW) * g.Bw, (CH) * g.Bh, (CT) * g.Bt, (BH));                             \
+  } while (0)
 
 // ================================================================================================
 // dQ pass
@@ -64,6 +85,9 @@ struct DqArgs {
   StatusBlock* status;
 };
 
+// Roles (256 threads): warp 0 = TMA producer of the K pairs (ring A; held until the dQ^T product of the tile is done)
+// and of the stationary Q and dO tiles, warp 1 = TMA producer of the V pairs (ring B), warp 2 = issuer of S^T and dP^T,
+// warp 3 = issuer of dQ^T += K_pair^T dS^T, warps 4..7 = elementwise stage + epilogue.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -76,23 +100,26 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   unsigned char* do_tile = smem + C::OFF_ST1;
   unsigned char* ds_tile = smem + C::OFF_P;      // two buffers
   BwdMisc* misc = reinterpret_cast<BwdMisc*>(smem + C::OFF_MISC);
+  unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_items = g.batch * g.Hq * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
 
+  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
   if (tid == 0) {
     misc->abort_flag = 0;
     tc::mbar_init(&misc->st_full, 1);
     tc::mbar_init(&misc->st_empty, 1);
     tc::mbar_init(&misc->o_full, 1);
     tc::mbar_init(&misc->o_empty, 128);
-    for (int s = 0; s < kBwdSlots; ++s) {
-      tc::mbar_init(&misc->ring_full[s], 1);
-      tc::mbar_init(&misc->ring_empty[s], 1);
-    }
     for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(&misc->a_full[s], 1);
+      tc::mbar_init(&misc->a_empty[s], 1);
+      tc::mbar_init(&misc->b_full[s], 1);
+      tc::mbar_init(&misc->b_empty[s], 1);
       tc::mbar_init(&misc->sdp_full[s], 1);
+      tc::mbar_init(&misc->sdp_free[s], 128);
       tc::mbar_init(&misc->ds_ready[s], 128);
       tc::mbar_init(&misc->ds_free[s], 1);
     }
@@ -102,7 +129,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     tc::prefetch_tmap(&tm_v);
     tc::prefetch_tmap(&tm_do);
   }
-  if (warp == 1) {
+  if (warp == 2) {
     tc::tmem_alloc(&misc->tmem_base, 512);
     tc::tmem_relinquish();
   }
@@ -112,94 +139,106 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const uint32_t tmem_base = misc->tmem_base;
   // tensor-memory columns: S^T buffers 0, 64; dP^T buffers 128, 192; dQ^T 256
 
-  if (warp == 0) {
-    if (lane == 0) {
-      uint32_t seq = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
-        const int i = item % g.N, bhq = item / g.N;
-        const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
-        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
-        const int k = end - beg;
-        if (k == 0) continue;
-        const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+  if (warp < 2) {
+    // ------------------------------------------------------------------ TMA producers
+    const int which = warp;                               // 0: K pairs (ring A) + Q, dO tiles; 1: V pairs (ring B)
+    const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+    uint64_t* full = which == 0 ? misc->a_full : misc->b_full;
+    uint64_t* empty = which == 0 ? misc->a_empty : misc->b_empty;
+    unsigned char* ring = smem + (which == 0 ? 0 : C::OFF_RING_B);
+    const int my_blk = lane & 1;
+    uint32_t tg = 0, n_items = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      const int i = item % g.N, bhq = item / g.N;
+      const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
+      const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
+      const int k = end - beg;
+      if (k == 0) continue;
+      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+      if (which == 0) {
         int it_, ih_, iw_;
         cube_coords(g, i, it_, ih_, iw_);
-        VSA2_WAIT(&misc->st_empty, (n_items & 1) ^ 1);
-        tc::mbar_expect_tx(&misc->st_full, 2 * C::TILE);
-        for (int h = 0; h < C::DH; ++h) {
-          tc::tma_load_5d(q_tile + h * kSlab, &tm_q, &misc->st_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
-          tc::tma_load_5d(do_tile + h * kSlab, &tm_do, &misc->st_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+        int ok = 1;
+        if (lane == 0) {
+          ok = tc::mbar_wait(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
+          if (ok) tc::mbar_expect_tx(&misc->st_full, 2 * C::TILE);
         }
-        ++n_items;
-        const int nt = (k + 1) >> 1;
-        for (int t = 0; t < nt; ++t) {
-          const int ja = cols[2 * t], jb = (2 * t + 1 < k) ? cols[2 * t + 1] : ja;
-          int at, ah, aw, bt, bh_, bw;
-          cube_coords(g, ja, at, ah, aw);
-          cube_coords(g, jb, bt, bh_, bw);
-          for (int which = 0; which < 2; ++which, ++seq) {   // K pair, then V pair
-            const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
-            const uint32_t slot = seq % kBwdSlots, par = (seq / kBwdSlots) & 1;
-            unsigned char* dst = smem + slot * C::SLOT;
-            VSA2_WAIT(&misc->ring_empty[slot], par ^ 1);
-            tc::mbar_expect_tx(&misc->ring_full[slot], C::SLOT);
-            for (int h = 0; h < C::DH; ++h) {
-              tc::tma_load_5d(dst + (2 * h + 0) * kSlab, tm, &misc->ring_full[slot], h * 64, aw * g.Bw, ah * g.Bh, at * g.Bt, bhk);
-              tc::tma_load_5d(dst + (2 * h + 1) * kSlab, tm, &misc->ring_full[slot], h * 64, bw * g.Bw, bh_ * g.Bh, bt * g.Bt, bhk);
-            }
-          }
+        if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+        if (lane < 2 * C::DH) {
+          const int h = lane >> 1;
+          if (lane & 1) tc::tma_load_5d(do_tile + h * kSlab, &tm_do, &misc->st_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+          else tc::tma_load_5d(q_tile + h * kSlab, &tm_q, &misc->st_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
         }
       }
+      ++n_items;
+      const int nt = (k + 1) >> 1;
+      int j = cols[(my_blk == 1 && k > 1) ? 1 : 0];
+      for (int t = 0; t < nt; ++t, ++tg) {
+        int jt, jh, jw;
+        cube_coords(g, j, jt, jh, jw);
+        if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
+        VSA2_RING_LOAD(full, empty, ring, tm, tg, jt, jh, jw, bhk);
+      }
     }
-  } else if (warp == 1) {
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ issuer of S^T = K_pair Q^T and dP^T = V_pair dO^T
     if (lane == 0) {
-      const uint32_t q_addr = tc::smem_u32(q_tile), do_addr = tc::smem_u32(do_tile), ds_addr = tc::smem_u32(ds_tile);
-      const uint32_t slot0 = tc::smem_u32(smem);
-      uint32_t seq0 = 0, tt = 0, n_items = 0;
+      const uint32_t q_addr = tc::smem_u32(q_tile), do_addr = tc::smem_u32(do_tile), base = tc::smem_u32(smem);
+      uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         const int i = item % g.N, bhq = item / g.N;
-        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
-        const int k = end - beg;
+        const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->st_full, n_items & 1);
-        tc::tc_fence_after();
-        for (int t = 0; t <= nt; ++t) {
-          if (t < nt) {
-            const uint32_t sk = seq0 + 2 * t, sv = sk + 1;
-            const uint32_t slot_k = sk % kBwdSlots, slot_v = sv % kBwdSlots, buf = (tt + t) & 1;
-            VSA2_WAIT(&misc->ring_full[slot_k], (sk / kBwdSlots) & 1);
-            VSA2_WAIT(&misc->ring_full[slot_v], (sv / kBwdSlots) & 1);
-            tc::tc_fence_after();
-            mma_pair_kmajor<D>(tmem_base + buf * 64, slot0 + slot_k * C::SLOT, q_addr);
-            mma_pair_kmajor<D>(tmem_base + 128 + buf * 64, slot0 + slot_v * C::SLOT, do_addr);
-            tc::mma_commit(&misc->sdp_full[buf]);
-            tc::mma_commit(&misc->ring_empty[slot_v]);
-            if (t == nt - 1) tc::mma_commit(&misc->st_empty);
-          }
-          if (t >= 1) {
-            const uint32_t tp = tt + t - 1, buf = tp & 1;
-            const uint32_t sk = seq0 + 2 * (t - 1), slot_k = sk % kBwdSlots;
-            VSA2_WAIT(&misc->ds_ready[buf], (tp >> 1) & 1);
-            if (t == 1) VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
-            tc::tc_fence_after();
-            mma_pairT_mnmajor<D>(tmem_base + 256, slot0 + slot_k * C::SLOT, ds_addr + buf * C::PBYTES, t > 1);
-            tc::mma_commit(&misc->ring_empty[slot_k]);
-            tc::mma_commit(&misc->ds_free[buf]);
-            if (t == nt) tc::mma_commit(&misc->o_full);
-          }
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
+          VSA2_WAIT(&misc->a_full[s], par);
+          VSA2_WAIT(&misc->b_full[s], par);
+          VSA2_WAIT(&misc->sdp_free[s], par ^ 1);
+          tc::tc_fence_after();
+          mma_pair_kmajor<D>(tmem_base + s * 64, base + s * C::SLOT, q_addr);
+          mma_pair_kmajor<D>(tmem_base + 128 + s * 64, base + C::OFF_RING_B + s * C::SLOT, do_addr);
+          tc::mma_commit(&misc->sdp_full[s]);
+          tc::mma_commit(&misc->b_empty[s]);
         }
-        seq0 += 2 * nt;
-        tt += nt;
+        tc::mma_commit(&misc->st_empty);
+        ++n_items;
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ issuer of dQ^T += K_pair^T dS^T
+    if (lane == 0) {
+      const uint32_t ds_addr = tc::smem_u32(ds_tile), base = tc::smem_u32(smem);
+      uint32_t tg = 0, n_items = 0;
+      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        const int i = item % g.N, bhq = item / g.N;
+        const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+        if (k == 0) continue;
+        const int nt = (k + 1) >> 1;
+        VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
+          VSA2_WAIT(&misc->ds_ready[s], par);
+          tc::tc_fence_after();
+          mma_pairT_mnmajor<D>(tmem_base + 256, base + s * C::SLOT, ds_addr + s * C::PBYTES, t > 0);
+          tc::mma_commit(&misc->a_empty[s]);
+          tc::mma_commit(&misc->ds_free[s]);
+        }
+        tc::mma_commit(&misc->o_full);
         ++n_items;
       }
     }
   } else {
+    // ------------------------------------------------------------------ elementwise stage + epilogue (128 threads)
     const int quad = warp & 3;
-    const int row = (quad << 5) | lane;
-    const int sm_tid = tid - 64;
+    const int row = (quad << 5) | lane;          // key row of the tile (S^T, dP^T) / channel (dQ^T)
+    const int sm_tid = tid - 128;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t tt = 0, n_items = 0, n_all = 0;
+    CubePos cpos;
+    cpos.init(g, row & 63);
+    const int blk = row >> 6;
+    uint32_t tg = 0, n_items = 0, n_all = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
       const int i = item % g.N, bhq = item / g.N;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
@@ -219,36 +258,46 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       tc::named_bar_sync(1, 128);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
-        for (int t = 0; t < nt; ++t, ++tt) {
-          const uint32_t buf = tt & 1, use = (tt >> 1) & 1;
-          const int blk = row >> 6;
+        const float4* lse4 = reinterpret_cast<const float4*>(misc->lse2[tb]);
+        const float4* del4 = reinterpret_cast<const float4*>(misc->delta[tb]);
+        int j_next = cols[(blk == 1 && k > 1) ? 1 : 0];
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
           const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          const int j = cols[dup ? 2 * t : 2 * t + blk];
-          const bool valid = !dup && pos_valid(g, j, row & 63);
-          VSA2_WAIT(&misc->sdp_full[buf], use);
+          const bool valid = !dup && cpos.valid(edge[j_next]);
+          if (t + 1 < nt) j_next = cols[(blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
+          VSA2_WAIT(&misc->sdp_full[s], par);
           tc::tc_fence_after();
           uint32_t packed[32];
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            uint32_t s[32], dp[32];
-            tc::tmem_ld32(lane_addr + buf * 64 + half * 32, s);
-            tc::tmem_ld32(lane_addr + 128 + buf * 64 + half * 32, dp);
+            uint32_t sv[32], dp[32];
+            tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
+            tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
             tc::tmem_ld_wait();
+            if (half == 1) {
+              tc::tc_fence_before();
+              tc::mbar_arrive(&misc->sdp_free[s]);
+            }
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              const int q0 = half * 32 + c;
-              float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), c2, -misc->lse2[tb][q0]));
-              float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), c2, -misc->lse2[tb][q0 + 1]));
-              float d0 = p0 * (__uint_as_float(dp[c]) - misc->delta[tb][q0]) * g.scale;
-              float d1 = p1 * (__uint_as_float(dp[c + 1]) - misc->delta[tb][q0 + 1]) * g.scale;
-              packed[half * 16 + (c >> 1)] = valid ? pack_bf16x2(d0, d1) : 0u;
+            for (int c4 = 0; c4 < 8; ++c4) {
+              const float4 ls = lse4[half * 8 + c4], dl = del4[half * 8 + c4];
+              const float p0 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 0]), c2, -ls.x));
+              const float p1 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 1]), c2, -ls.y));
+              const float p2 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 2]), c2, -ls.z));
+              const float p3 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 3]), c2, -ls.w));
+              const float d0 = p0 * (__uint_as_float(dp[4 * c4 + 0]) - dl.x) * g.scale;
+              const float d1 = p1 * (__uint_as_float(dp[4 * c4 + 1]) - dl.y) * g.scale;
+              const float d2 = p2 * (__uint_as_float(dp[4 * c4 + 2]) - dl.z) * g.scale;
+              const float d3 = p3 * (__uint_as_float(dp[4 * c4 + 3]) - dl.w) * g.scale;
+              packed[half * 16 + 2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
+              packed[half * 16 + 2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
             }
           }
-          VSA2_WAIT(&misc->ds_free[buf], use ^ 1);
-          store_row_sw128(ds_tile + buf * C::PBYTES, row, packed);
+          VSA2_WAIT(&misc->ds_free[s], par ^ 1);
+          store_row_sw128(ds_tile + s * C::PBYTES, row, packed);
           tc::fence_proxy_async_smem();
-          tc::tc_fence_before();
-          tc::mbar_arrive(&misc->ds_ready[buf]);
+          tc::mbar_arrive(&misc->ds_ready[s]);
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
@@ -266,14 +315,34 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 #pragma unroll
           for (int c = 0; c < 32; ++c) { o0[c] = 0u; o1[c] = 0u; }
         }
-        if (row < D) {
+        if (g.out_f32) {
+          if (row < D) {
 #pragma unroll
-          for (int qi = 0; qi < 64; ++qi) {
+            for (int qi = 0; qi < 64; ++qi) {
+              const int l = misc->tok[tb][qi];
+              if (l < 0) continue;
+              const float acc = __uint_as_float(qi < 32 ? o0[qi & 31] : o1[qi & 31]);
+              store_out(a.dq, ((size_t)bhq * g.L + l) * D + row, acc + coarse_d, 1);
+            }
+          }
+        } else {
+          // bf16: transpose through shared memory (the dS^T buffers are idle now), then 16-byte stores
+          bf16* st = reinterpret_cast<bf16*>(ds_tile);                  // [64 q][D]
+          if (row < D) {
+#pragma unroll
+            for (int qi = 0; qi < 64; ++qi)
+              st[qi * D + row] = __float2bfloat16_rn(__uint_as_float(qi < 32 ? o0[qi & 31] : o1[qi & 31]) + coarse_d);
+          }
+          tc::named_bar_sync(1, 128);
+          constexpr int CH = D / 8;
+          for (int e = sm_tid; e < 64 * CH; e += 128) {
+            const int qi = e / CH, ch = e % CH;
             const int l = misc->tok[tb][qi];
             if (l < 0) continue;
-            const float acc = __uint_as_float(qi < 32 ? o0[qi & 31] : o1[qi & 31]);
-            store_out(a.dq, ((size_t)bhq * g.L + l) * D + row, acc + coarse_d, g.out_f32);
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dq) + ((size_t)bhq * g.L + l) * D + ch * 8) =
+                *reinterpret_cast<const uint4*>(st + qi * D + ch * 8);
           }
+          tc::named_bar_sync(1, 128);
         }
       }
       if (k > 0) ++n_items;
@@ -292,7 +361,7 @@ done:
     }
     __syncthreads();
   }
-  if (warp == 1) tc::tmem_dealloc(tmem_base, 512);
+  if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
 }
 
 // ================================================================================================
@@ -322,6 +391,10 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b,
   i = a.row_idx[(size_t)bhq * g.nnz_cap + beg + (e - cnt_prefix[hh])];
 }
 
+// Roles (256 threads): warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA
+// producer of the dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T and dP = dO_pair V^T, warp 3 = issuer of
+// dV^T += dO_pair^T P and dK^T += Q_pair^T dS (both rings are held until these are done), warps 4..7 = elementwise
+// stage + epilogue.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -346,12 +419,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tc::mbar_init(&misc->st_empty, 1);
     tc::mbar_init(&misc->o_full, 1);
     tc::mbar_init(&misc->o_empty, 128);
-    for (int s = 0; s < kBwdSlots; ++s) {
-      tc::mbar_init(&misc->ring_full[s], 1);
-      tc::mbar_init(&misc->ring_empty[s], 1);
-    }
     for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(&misc->a_full[s], 1);
+      tc::mbar_init(&misc->a_empty[s], 1);
+      tc::mbar_init(&misc->b_full[s], 1);
+      tc::mbar_init(&misc->b_empty[s], 1);
       tc::mbar_init(&misc->sdp_full[s], 1);
+      tc::mbar_init(&misc->sdp_free[s], 128);
       tc::mbar_init(&misc->ds_ready[s], 128);
       tc::mbar_init(&misc->ds_free[s], 1);
     }
@@ -361,7 +435,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tc::prefetch_tmap(&tm_v);
     tc::prefetch_tmap(&tm_do);
   }
-  if (warp == 1) {
+  if (warp == 2) {
     tc::tmem_alloc(&misc->tmem_base, 512);
     tc::tmem_relinquish();
   }
@@ -378,108 +452,118 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   int cnt_prefix[kMaxRep + 1];                                                           \
   cnt_prefix[0] = 0;                                                                     \
   for (int hh = 0; hh < g.rep; ++hh) {                                                   \
-    const size_t base = (size_t)(b * g.Hq + hk * g.rep + hh) * (g.N + 1) + j;            \
-    cnt_prefix[hh + 1] = cnt_prefix[hh] + (a.col_ptr[base + 1] - a.col_ptr[base]);       \
+    const size_t base_ = (size_t)(b * g.Hq + hk * g.rep + hh) * (g.N + 1) + j;           \
+    cnt_prefix[hh + 1] = cnt_prefix[hh] + (a.col_ptr[base_ + 1] - a.col_ptr[base_]);     \
   }                                                                                      \
   const int k = cnt_prefix[g.rep];
 
-  if (warp == 0) {
-    if (lane == 0) {
-      uint32_t seq = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
-        VSA2_DKV_ITEM_SETUP();
-        if (k == 0) continue;
+  if (warp < 2) {
+    // ------------------------------------------------------------------ TMA producers
+    const int which = warp;                               // 0: Q pairs (ring A) + K, V tiles; 1: dO pairs (ring B)
+    const CUtensorMap* tm = which == 0 ? &tm_q : &tm_do;
+    uint64_t* full = which == 0 ? misc->a_full : misc->b_full;
+    uint64_t* empty = which == 0 ? misc->a_empty : misc->b_empty;
+    unsigned char* ring = smem + (which == 0 ? 0 : C::OFF_RING_B);
+    const int my_blk = lane & 1;
+    uint32_t tg = 0, n_items = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      VSA2_DKV_ITEM_SETUP();
+      if (k == 0) continue;
+      if (which == 0) {
         int jt, jh, jw;
         cube_coords(g, j, jt, jh, jw);
-        VSA2_WAIT(&misc->st_empty, (n_items & 1) ^ 1);
-        tc::mbar_expect_tx(&misc->st_full, 2 * C::TILE);
-        for (int h = 0; h < C::DH; ++h) {
-          tc::tma_load_5d(k_tile + h * kSlab, &tm_k, &misc->st_full, h * 64, jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
-          tc::tma_load_5d(v_tile + h * kSlab, &tm_v, &misc->st_full, h * 64, jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
+        int ok = 1;
+        if (lane == 0) {
+          ok = tc::mbar_wait(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
+          if (ok) tc::mbar_expect_tx(&misc->st_full, 2 * C::TILE);
         }
-        ++n_items;
-        const int nt = (k + 1) >> 1;
-        for (int t = 0; t < nt; ++t) {
-          int bhq_a, ia, bhq_b, ib;
-          dkv_entry(g, a, b, hk, j, cnt_prefix, 2 * t, bhq_a, ia);
-          if (2 * t + 1 < k) dkv_entry(g, a, b, hk, j, cnt_prefix, 2 * t + 1, bhq_b, ib);
-          else { bhq_b = bhq_a; ib = ia; }
-          int at, ah, aw, bt, bh_, bw;
-          cube_coords(g, ia, at, ah, aw);
-          cube_coords(g, ib, bt, bh_, bw);
-          for (int which = 0; which < 2; ++which, ++seq) {   // Q pair, then dO pair
-            const CUtensorMap* tm = which == 0 ? &tm_q : &tm_do;
-            const uint32_t slot = seq % kBwdSlots, par = (seq / kBwdSlots) & 1;
-            unsigned char* dst = smem + slot * C::SLOT;
-            VSA2_WAIT(&misc->ring_empty[slot], par ^ 1);
-            tc::mbar_expect_tx(&misc->ring_full[slot], C::SLOT);
-            for (int h = 0; h < C::DH; ++h) {
-              tc::tma_load_5d(dst + (2 * h + 0) * kSlab, tm, &misc->ring_full[slot], h * 64, aw * g.Bw, ah * g.Bh, at * g.Bt, bhq_a);
-              tc::tma_load_5d(dst + (2 * h + 1) * kSlab, tm, &misc->ring_full[slot], h * 64, bw * g.Bw, bh_ * g.Bh, bt * g.Bt, bhq_b);
-            }
-          }
+        if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+        if (lane < 2 * C::DH) {
+          const int h = lane >> 1;
+          if (lane & 1) tc::tma_load_5d(v_tile + h * kSlab, &tm_v, &misc->st_full, h * 64, jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
+          else tc::tma_load_5d(k_tile + h * kSlab, &tm_k, &misc->st_full, h * 64, jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
         }
       }
+      ++n_items;
+      const int nt = (k + 1) >> 1;
+      for (int t = 0; t < nt; ++t, ++tg) {
+        int bhq_l, i_l;
+        dkv_entry(g, a, b, hk, j, cnt_prefix, (my_blk == 1 && 2 * t + 1 < k) ? 2 * t + 1 : 2 * t, bhq_l, i_l);
+        int it_, ih_, iw_;
+        cube_coords(g, i_l, it_, ih_, iw_);
+        VSA2_RING_LOAD(full, empty, ring, tm, tg, it_, ih_, iw_, bhq_l);
+      }
     }
-  } else if (warp == 1) {
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ issuer of S = Q_pair K^T and dP = dO_pair V^T
     if (lane == 0) {
-      const uint32_t k_addr = tc::smem_u32(k_tile), v_addr = tc::smem_u32(v_tile);
-      const uint32_t p_addr = tc::smem_u32(p_tile), ds_addr = tc::smem_u32(ds_tile), slot0 = tc::smem_u32(smem);
-      uint32_t seq0 = 0, tt = 0, n_items = 0;
+      const uint32_t k_addr = tc::smem_u32(k_tile), v_addr = tc::smem_u32(v_tile), base = tc::smem_u32(smem);
+      uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         VSA2_DKV_ITEM_SETUP();
-        (void)b; (void)hk;
+        (void)b; (void)hk; (void)j; (void)bhk;
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->st_full, n_items & 1);
-        tc::tc_fence_after();
-        for (int t = 0; t <= nt; ++t) {
-          if (t < nt) {
-            const uint32_t sq = seq0 + 2 * t, sd = sq + 1;
-            const uint32_t slot_q = sq % kBwdSlots, slot_d = sd % kBwdSlots, buf = (tt + t) & 1;
-            VSA2_WAIT(&misc->ring_full[slot_q], (sq / kBwdSlots) & 1);
-            VSA2_WAIT(&misc->ring_full[slot_d], (sd / kBwdSlots) & 1);
-            tc::tc_fence_after();
-            mma_pair_kmajor<D>(tmem_base + buf * 64, slot0 + slot_q * C::SLOT, k_addr);
-            mma_pair_kmajor<D>(tmem_base + 128 + buf * 64, slot0 + slot_d * C::SLOT, v_addr);
-            tc::mma_commit(&misc->sdp_full[buf]);
-            if (t == nt - 1) tc::mma_commit(&misc->st_empty);
-          }
-          if (t >= 1) {
-            const uint32_t tp = tt + t - 1;
-            const uint32_t sq = seq0 + 2 * (t - 1), slot_q = sq % kBwdSlots, slot_d = (sq + 1) % kBwdSlots;
-            VSA2_WAIT(&misc->ds_ready[0], tp & 1);
-            if (t == 1) VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
-            tc::tc_fence_after();
-            mma_pairT_mnmajor<D>(tmem_base + 320, slot0 + slot_d * C::SLOT, p_addr, t > 1);    // dV^T += dO^T P
-            mma_pairT_mnmajor<D>(tmem_base + 256, slot0 + slot_q * C::SLOT, ds_addr, t > 1);   // dK^T += Q^T dS
-            tc::mma_commit(&misc->ring_empty[slot_q]);
-            tc::mma_commit(&misc->ring_empty[slot_d]);
-            tc::mma_commit(&misc->ds_free[0]);
-            if (t == nt) tc::mma_commit(&misc->o_full);
-          }
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
+          VSA2_WAIT(&misc->a_full[s], par);
+          VSA2_WAIT(&misc->b_full[s], par);
+          VSA2_WAIT(&misc->sdp_free[s], par ^ 1);
+          tc::tc_fence_after();
+          mma_pair_kmajor<D>(tmem_base + s * 64, base + s * C::SLOT, k_addr);
+          mma_pair_kmajor<D>(tmem_base + 128 + s * 64, base + C::OFF_RING_B + s * C::SLOT, v_addr);
+          tc::mma_commit(&misc->sdp_full[s]);
         }
-        seq0 += 2 * nt;
-        tt += nt;
+        tc::mma_commit(&misc->st_empty);
+        ++n_items;
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ issuer of dV^T += dO_pair^T P and dK^T += Q_pair^T dS
+    if (lane == 0) {
+      const uint32_t p_addr = tc::smem_u32(p_tile), ds_addr = tc::smem_u32(ds_tile), base = tc::smem_u32(smem);
+      uint32_t tg = 0, n_items = 0;
+      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        VSA2_DKV_ITEM_SETUP();
+        (void)b; (void)hk; (void)j; (void)bhk;
+        if (k == 0) continue;
+        const int nt = (k + 1) >> 1;
+        VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t s = tg & 1;
+          VSA2_WAIT(&misc->ds_ready[0], tg & 1);
+          tc::tc_fence_after();
+          mma_pairT_mnmajor<D>(tmem_base + 320, base + C::OFF_RING_B + s * C::SLOT, p_addr, t > 0);    // dV^T += dO^T P
+          mma_pairT_mnmajor<D>(tmem_base + 256, base + s * C::SLOT, ds_addr, t > 0);                  // dK^T += Q^T dS
+          tc::mma_commit(&misc->a_empty[s]);
+          tc::mma_commit(&misc->b_empty[s]);
+          tc::mma_commit(&misc->ds_free[0]);
+        }
+        tc::mma_commit(&misc->o_full);
         ++n_items;
       }
     }
   } else {
+    // ------------------------------------------------------------------ elementwise stage + epilogue (128 threads)
     const int quad = warp & 3;
     const int row = (quad << 5) | lane;      // query row of the tile (S, dP) / channel (dK^T, dV^T)
-    const int sm_tid = tid - 64;
+    const int sm_tid = tid - 128;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t tt = 0, n_items = 0, n_all = 0;
+    const int blk = row >> 6;
+    uint32_t tg = 0, n_items = 0, n_all = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
       VSA2_DKV_ITEM_SETUP();
       const int tb = n_all & 1;
       int jt, jh, jw;
       cube_coords(g, j, jt, jh, jw);
       if (sm_tid < 64) misc->tok[tb][sm_tid] = cube_token(g, jt, jh, jw, sm_tid);
-      unsigned long long kvmask = 0ull;
-      if (k > 0)
+      unsigned long long kvmask = ~0ull;
+      if (k > 0 && cube_edge_flags(g, j) != 0) {
+        kvmask = 0ull;
         for (int p = 0; p < 64; ++p)
           if (cube_token(g, jt, jh, jw, p) >= 0) kvmask |= 1ull << p;
+      }
       float coarse_k = 0.f, coarse_v = 0.f;
       if (a.dkc != nullptr && row < D) {
         for (int hh = 0; hh < g.rep; ++hh) {
@@ -494,73 +578,104 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       tc::named_bar_sync(1, 128);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
-        for (int t = 0; t < nt; ++t, ++tt) {
-          const uint32_t buf = tt & 1, use = (tt >> 1) & 1;
-          // this thread's query row: which (head, block, token)
-          const int blk = row >> 6;
+        // (head, block, token) of this thread's query row in tile 0, then one tile ahead
+        int bhq_n, i_n;
+        dkv_entry(g, a, b, hk, j, cnt_prefix, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
           const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          int bhq, i;
-          dkv_entry(g, a, b, hk, j, cnt_prefix, dup ? 2 * t : 2 * t + blk, bhq, i);
           int it_, ih_, iw_;
-          cube_coords(g, i, it_, ih_, iw_);
+          cube_coords(g, i_n, it_, ih_, iw_);
           const int l = dup ? -1 : cube_token(g, it_, ih_, iw_, row & 63);
-          const float lse2 = l >= 0 ? a.lse[(size_t)bhq * g.L + l] * 1.4426950408889634f : INFINITY;
-          const float dlt = l >= 0 ? a.delta[(size_t)bhq * g.L + l] : 0.f;
-          VSA2_WAIT(&misc->sdp_full[buf], use);
+          const float lse2 = l >= 0 ? a.lse[(size_t)bhq_n * g.L + l] * 1.4426950408889634f : INFINITY;
+          const float dlt = l >= 0 ? a.delta[(size_t)bhq_n * g.L + l] : 0.f;
+          if (t + 1 < nt) dkv_entry(g, a, b, hk, j, cnt_prefix, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
+          VSA2_WAIT(&misc->sdp_full[s], par);
           tc::tc_fence_after();
           uint32_t pp[32], pd[32];
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            uint32_t s[32], dp[32];
-            tc::tmem_ld32(lane_addr + buf * 64 + half * 32, s);
-            tc::tmem_ld32(lane_addr + 128 + buf * 64 + half * 32, dp);
+            uint32_t sv[32], dp[32];
+            tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
+            tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
             tc::tmem_ld_wait();
+            if (half == 1) {
+              tc::tc_fence_before();
+              tc::mbar_arrive(&misc->sdp_free[s]);
+            }
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
               const int c0 = half * 32 + c;
-              float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), c2, -lse2));
-              float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), c2, -lse2));
-              p0 = ((kvmask >> c0) & 1ull) ? p0 : 0.f;
-              p1 = ((kvmask >> (c0 + 1)) & 1ull) ? p1 : 0.f;
+              float p0 = ex2_approx(fmaf(__uint_as_float(sv[c]), c2, -lse2));
+              float p1 = ex2_approx(fmaf(__uint_as_float(sv[c + 1]), c2, -lse2));
+              if (kvmask != ~0ull) {
+                p0 = ((kvmask >> c0) & 1ull) ? p0 : 0.f;
+                p1 = ((kvmask >> (c0 + 1)) & 1ull) ? p1 : 0.f;
+              }
               const float d0 = p0 * (__uint_as_float(dp[c]) - dlt) * g.scale;
               const float d1 = p1 * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
               pp[half * 16 + (c >> 1)] = pack_bf16x2(p0, p1);
               pd[half * 16 + (c >> 1)] = pack_bf16x2(d0, d1);
             }
           }
-          VSA2_WAIT(&misc->ds_free[0], (tt & 1) ^ 1);
+          VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
           store_row_sw128(p_tile, row, pp);
           store_row_sw128(ds_tile, row, pd);
           tc::fence_proxy_async_smem();
-          tc::tc_fence_before();
           tc::mbar_arrive(&misc->ds_ready[0]);
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
       }
-      {
-        uint32_t k0[32], k1[32], v0[32], v1[32];
+      // epilogue: dK[l, d] = dK^T[d, kv] + sum_heads dK_c[j, d] / count(j), same for dV; 32 key columns at a time
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        uint32_t kk[32], vv[32];
         if (k > 0) {
-          tc::tmem_ld32(lane_addr + 256, k0);
-          tc::tmem_ld32(lane_addr + 256 + 32, k1);
-          tc::tmem_ld32(lane_addr + 320, v0);
-          tc::tmem_ld32(lane_addr + 320 + 32, v1);
+          tc::tmem_ld32(lane_addr + 256 + half * 32, kk);
+          tc::tmem_ld32(lane_addr + 320 + half * 32, vv);
           tc::tmem_ld_wait();
-          tc::tc_fence_before();
-          tc::mbar_arrive(&misc->o_empty);
+          if (half == 1) {
+            tc::tc_fence_before();
+            tc::mbar_arrive(&misc->o_empty);
+          }
         } else {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) { k0[c] = 0u; k1[c] = 0u; v0[c] = 0u; v1[c] = 0u; }
+          for (int c = 0; c < 32; ++c) { kk[c] = 0u; vv[c] = 0u; }
         }
-        if (row < D) {
+        if (g.out_f32) {
+          if (row < D) {
 #pragma unroll
-          for (int ki = 0; ki < 64; ++ki) {
-            const int l = misc->tok[tb][ki];
-            if (l < 0) continue;
-            const size_t idx = ((size_t)bhk * g.L + l) * D + row;
-            store_out(a.dk, idx, __uint_as_float(ki < 32 ? k0[ki & 31] : k1[ki & 31]) + coarse_k, g.out_f32);
-            store_out(a.dv, idx, __uint_as_float(ki < 32 ? v0[ki & 31] : v1[ki & 31]) + coarse_v, g.out_f32);
+            for (int c = 0; c < 32; ++c) {
+              const int l = misc->tok[tb][half * 32 + c];
+              if (l < 0) continue;
+              const size_t idx = ((size_t)bhk * g.L + l) * D + row;
+              store_out(a.dk, idx, __uint_as_float(kk[c]) + coarse_k, 1);
+              store_out(a.dv, idx, __uint_as_float(vv[c]) + coarse_v, 1);
+            }
           }
+        } else {
+          // bf16: transpose 32 key rows through shared memory (P and dS buffers are idle), then 16-byte stores
+          bf16* st_k = reinterpret_cast<bf16*>(p_tile);       // [32 kv][D]
+          bf16* st_v = reinterpret_cast<bf16*>(ds_tile);      // [32 kv][D]
+          if (row < D) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              st_k[c * D + row] = __float2bfloat16_rn(__uint_as_float(kk[c]) + coarse_k);
+              st_v[c * D + row] = __float2bfloat16_rn(__uint_as_float(vv[c]) + coarse_v);
+            }
+          }
+          tc::named_bar_sync(1, 128);
+          constexpr int CH = D / 8;
+          for (int e = sm_tid; e < 32 * CH; e += 128) {
+            const int c = e / CH, ch = e % CH;
+            const int l = misc->tok[tb][half * 32 + c];
+            if (l < 0) continue;
+            const size_t idx = ((size_t)bhk * g.L + l) * D + ch * 8;
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dk) + idx) = *reinterpret_cast<const uint4*>(st_k + c * D + ch * 8);
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dv) + idx) = *reinterpret_cast<const uint4*>(st_v + c * D + ch * 8);
+          }
+          tc::named_bar_sync(1, 128);
         }
       }
       if (k > 0) ++n_items;
@@ -579,7 +694,7 @@ done:
     }
     __syncthreads();
   }
-  if (warp == 1) tc::tmem_dealloc(tmem_base, 512);
+  if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
 }
 
 // ================================================================================================
@@ -605,12 +720,13 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
   DqArgs a{lse, delta, row_ptr, col_idx, dqc, dq, status};
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
+  if (g.N > kBwdMaxCubes) return cudaErrorInvalidValue;
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
-    fine_bwd_dq_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes(g.N)))) return e;
+    fine_bwd_dq_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
-    fine_bwd_dq_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes(g.N)))) return e;
+    fine_bwd_dq_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
   }
   return cudaGetLastError();
 }
@@ -631,11 +747,11 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
-    fine_bwd_dkv_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes(g.N)))) return e;
+    fine_bwd_dkv_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
-    fine_bwd_dkv_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes(g.N)))) return e;
+    fine_bwd_dkv_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
   }
   return cudaGetLastError();
 }
