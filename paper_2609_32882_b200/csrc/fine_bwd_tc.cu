@@ -24,7 +24,7 @@
 
 namespace vsa2 {
 
-constexpr int kBwdThreads = 256;
+constexpr int kBwdThreads = 384;   // 4 service warps + 2 x 4 elementwise warps
 constexpr int kBwdMaxCubes = 12288;   // edge-flag table in shared memory: one byte per cube
 
 // Shared-memory plan of both passes (D = 128: 4 x 32 KB ring slots, 2 x 16 KB stationary tiles, 2 x 16 KB operand
@@ -85,9 +85,9 @@ struct DqArgs {
   StatusBlock* status;
 };
 
-// Roles (256 threads): warp 0 = TMA producer of the K pairs (ring A; held until the dQ^T product of the tile is done)
+// Roles (384 threads): warp 0 = TMA producer of the K pairs (ring A; held until the dQ^T product of the tile is done)
 // and of the stationary Q and dO tiles, warp 1 = TMA producer of the V pairs (ring B), warp 2 = issuer of S^T and dP^T,
-// warp 3 = issuer of dQ^T += K_pair^T dS^T, warps 4..7 = elementwise stage + epilogue.
+// warp 3 = issuer of dQ^T += K_pair^T dS^T, warps 4..11 = elementwise stage + epilogue (each half of the query columns).
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -112,15 +112,15 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     tc::mbar_init(&misc->st_full, 1);
     tc::mbar_init(&misc->st_empty, 1);
     tc::mbar_init(&misc->o_full, 1);
-    tc::mbar_init(&misc->o_empty, 128);
+    tc::mbar_init(&misc->o_empty, 256);
     for (int s = 0; s < 2; ++s) {
       tc::mbar_init(&misc->a_full[s], 1);
       tc::mbar_init(&misc->a_empty[s], 1);
       tc::mbar_init(&misc->b_full[s], 1);
       tc::mbar_init(&misc->b_empty[s], 1);
       tc::mbar_init(&misc->sdp_full[s], 1);
-      tc::mbar_init(&misc->sdp_free[s], 128);
-      tc::mbar_init(&misc->ds_ready[s], 128);
+      tc::mbar_init(&misc->sdp_free[s], 256);
+      tc::mbar_init(&misc->ds_ready[s], 256);
       tc::mbar_init(&misc->ds_free[s], 1);
     }
     tc::fence_barrier_init();
@@ -230,10 +230,12 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       }
     }
   } else {
-    // ------------------------------------------------------------------ elementwise stage + epilogue (128 threads)
+    // ------------------------------------------------------------------ elementwise stage + epilogue (256 threads):
+    // warps 4..7 take query columns 0..31 of every tile, warps 8..11 columns 32..63
     const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;            // which 32 query columns
     const int row = (quad << 5) | lane;          // key row of the tile (S^T, dP^T) / channel (dQ^T)
-    const int sm_tid = tid - 128;
+    const int sm_tid = tid - 128;                // 0..255
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     CubePos cpos;
     cpos.init(g, row & 63);
@@ -255,11 +257,11 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       }
       const float coarse_d = (a.dqc != nullptr && row < D)
                                  ? a.dqc[((size_t)bhq * g.N + i) * D + row] / (float)cube_count(g, i) : 0.f;
-      tc::named_bar_sync(1, 128);
+      tc::named_bar_sync(1, 256);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
-        const float4* lse4 = reinterpret_cast<const float4*>(misc->lse2[tb]);
-        const float4* del4 = reinterpret_cast<const float4*>(misc->delta[tb]);
+        const float4* lse4 = reinterpret_cast<const float4*>(misc->lse2[tb]) + half * 8;
+        const float4* del4 = reinterpret_cast<const float4*>(misc->delta[tb]) + half * 8;
         int j_next = cols[(blk == 1 && k > 1) ? 1 : 0];
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t s = tg & 1, par = (tg >> 1) & 1;
@@ -268,20 +270,17 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           if (t + 1 < nt) j_next = cols[(blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
           VSA2_WAIT(&misc->sdp_full[s], par);
           tc::tc_fence_after();
-          uint32_t packed[32];
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
+          uint32_t packed[16];
+          {
             uint32_t sv[32], dp[32];
             tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
             tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
             tc::tmem_ld_wait();
-            if (half == 1) {
-              tc::tc_fence_before();
-              tc::mbar_arrive(&misc->sdp_free[s]);
-            }
+            tc::tc_fence_before();
+            tc::mbar_arrive(&misc->sdp_free[s]);
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
-              const float4 ls = lse4[half * 8 + c4], dl = del4[half * 8 + c4];
+              const float4 ls = lse4[c4], dl = del4[c4];
               const float p0 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 0]), c2, -ls.x));
               const float p1 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 1]), c2, -ls.y));
               const float p2 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 2]), c2, -ls.z));
@@ -290,39 +289,43 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
               const float d1 = p1 * (__uint_as_float(dp[4 * c4 + 1]) - dl.y) * g.scale;
               const float d2 = p2 * (__uint_as_float(dp[4 * c4 + 2]) - dl.z) * g.scale;
               const float d3 = p3 * (__uint_as_float(dp[4 * c4 + 3]) - dl.w) * g.scale;
-              packed[half * 16 + 2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
-              packed[half * 16 + 2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
+              packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
+              packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
             }
           }
           VSA2_WAIT(&misc->ds_free[s], par ^ 1);
-          store_row_sw128(ds_tile + s * C::PBYTES, row, packed);
+          {
+            unsigned char* prow = ds_tile + s * C::PBYTES + row * 128;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch)
+              *reinterpret_cast<uint4*>(prow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
+                  make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+          }
           tc::fence_proxy_async_smem();
           tc::mbar_arrive(&misc->ds_ready[s]);
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
       }
-      // epilogue: dQ[l, d] = dQ^T[d, q] + dQ_c[i, d] / count(i)
+      // epilogue: dQ[l, d] = dQ^T[d, q] + dQ_c[i, d] / count(i); this thread owns 32 query columns of channel `row`
       {
-        uint32_t o0[32], o1[32];
+        uint32_t o0[32];
         if (k > 0) {
-          tc::tmem_ld32(lane_addr + 256, o0);
-          tc::tmem_ld32(lane_addr + 256 + 32, o1);
+          tc::tmem_ld32(lane_addr + 256 + half * 32, o0);
           tc::tmem_ld_wait();
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->o_empty);
         } else {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) { o0[c] = 0u; o1[c] = 0u; }
+          for (int c = 0; c < 32; ++c) o0[c] = 0u;
         }
         if (g.out_f32) {
           if (row < D) {
 #pragma unroll
-            for (int qi = 0; qi < 64; ++qi) {
-              const int l = misc->tok[tb][qi];
+            for (int c = 0; c < 32; ++c) {
+              const int l = misc->tok[tb][half * 32 + c];
               if (l < 0) continue;
-              const float acc = __uint_as_float(qi < 32 ? o0[qi & 31] : o1[qi & 31]);
-              store_out(a.dq, ((size_t)bhq * g.L + l) * D + row, acc + coarse_d, 1);
+              store_out(a.dq, ((size_t)bhq * g.L + l) * D + row, __uint_as_float(o0[c]) + coarse_d, 1);
             }
           }
         } else {
@@ -330,19 +333,19 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           bf16* st = reinterpret_cast<bf16*>(ds_tile);                  // [64 q][D]
           if (row < D) {
 #pragma unroll
-            for (int qi = 0; qi < 64; ++qi)
-              st[qi * D + row] = __float2bfloat16_rn(__uint_as_float(qi < 32 ? o0[qi & 31] : o1[qi & 31]) + coarse_d);
+            for (int c = 0; c < 32; ++c)
+              st[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(o0[c]) + coarse_d);
           }
-          tc::named_bar_sync(1, 128);
+          tc::named_bar_sync(1, 256);
           constexpr int CH = D / 8;
-          for (int e = sm_tid; e < 64 * CH; e += 128) {
+          for (int e = sm_tid; e < 64 * CH; e += 256) {
             const int qi = e / CH, ch = e % CH;
             const int l = misc->tok[tb][qi];
             if (l < 0) continue;
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dq) + ((size_t)bhq * g.L + l) * D + ch * 8) =
                 *reinterpret_cast<const uint4*>(st + qi * D + ch * 8);
           }
-          tc::named_bar_sync(1, 128);
+          tc::named_bar_sync(1, 256);
         }
       }
       if (k > 0) ++n_items;
@@ -391,10 +394,10 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b,
   i = a.row_idx[(size_t)bhq * g.nnz_cap + beg + (e - cnt_prefix[hh])];
 }
 
-// Roles (256 threads): warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA
+// Roles (384 threads): warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA
 // producer of the dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T and dP = dO_pair V^T, warp 3 = issuer of
-// dV^T += dO_pair^T P and dK^T += Q_pair^T dS (both rings are held until these are done), warps 4..7 = elementwise
-// stage + epilogue.
+// dV^T += dO_pair^T P and dK^T += Q_pair^T dS (both rings are held until these are done), warps 4..11 = elementwise
+// stage + epilogue (each half of the key columns).
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -418,15 +421,15 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     tc::mbar_init(&misc->st_full, 1);
     tc::mbar_init(&misc->st_empty, 1);
     tc::mbar_init(&misc->o_full, 1);
-    tc::mbar_init(&misc->o_empty, 128);
+    tc::mbar_init(&misc->o_empty, 256);
     for (int s = 0; s < 2; ++s) {
       tc::mbar_init(&misc->a_full[s], 1);
       tc::mbar_init(&misc->a_empty[s], 1);
       tc::mbar_init(&misc->b_full[s], 1);
       tc::mbar_init(&misc->b_empty[s], 1);
       tc::mbar_init(&misc->sdp_full[s], 1);
-      tc::mbar_init(&misc->sdp_free[s], 128);
-      tc::mbar_init(&misc->ds_ready[s], 128);
+      tc::mbar_init(&misc->sdp_free[s], 256);
+      tc::mbar_init(&misc->ds_ready[s], 256);
       tc::mbar_init(&misc->ds_free[s], 1);
     }
     tc::fence_barrier_init();
@@ -545,10 +548,12 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
     }
   } else {
-    // ------------------------------------------------------------------ elementwise stage + epilogue (128 threads)
+    // ------------------------------------------------------------------ elementwise stage + epilogue (256 threads):
+    // warps 4..7 take key columns 0..31 of every tile, warps 8..11 columns 32..63
     const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
     const int row = (quad << 5) | lane;      // query row of the tile (S, dP) / channel (dK^T, dV^T)
-    const int sm_tid = tid - 128;
+    const int sm_tid = tid - 128;            // 0..255
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const int blk = row >> 6;
     uint32_t tg = 0, n_items = 0, n_all = 0;
@@ -558,11 +563,11 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       int jt, jh, jw;
       cube_coords(g, j, jt, jh, jw);
       if (sm_tid < 64) misc->tok[tb][sm_tid] = cube_token(g, jt, jh, jw, sm_tid);
-      unsigned long long kvmask = ~0ull;
+      uint32_t kvmask = 0xffffffffu;           // validity of this thread's 32 key columns
       if (k > 0 && cube_edge_flags(g, j) != 0) {
-        kvmask = 0ull;
-        for (int p = 0; p < 64; ++p)
-          if (cube_token(g, jt, jh, jw, p) >= 0) kvmask |= 1ull << p;
+        kvmask = 0u;
+        for (int p = 0; p < 32; ++p)
+          if (cube_token(g, jt, jh, jw, half * 32 + p) >= 0) kvmask |= 1u << p;
       }
       float coarse_k = 0.f, coarse_v = 0.f;
       if (a.dkc != nullptr && row < D) {
@@ -575,7 +580,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         coarse_k *= inv_cnt;
         coarse_v *= inv_cnt;
       }
-      tc::named_bar_sync(1, 128);
+      tc::named_bar_sync(1, 256);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
         // (head, block, token) of this thread's query row in tile 0, then one tile ahead
@@ -592,53 +597,54 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (t + 1 < nt) dkv_entry(g, a, b, hk, j, cnt_prefix, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
           VSA2_WAIT(&misc->sdp_full[s], par);
           tc::tc_fence_after();
-          uint32_t pp[32], pd[32];
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
+          uint32_t pp[16], pd[16];
+          {
             uint32_t sv[32], dp[32];
             tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
             tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
             tc::tmem_ld_wait();
-            if (half == 1) {
-              tc::tc_fence_before();
-              tc::mbar_arrive(&misc->sdp_free[s]);
-            }
+            tc::tc_fence_before();
+            tc::mbar_arrive(&misc->sdp_free[s]);
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
-              const int c0 = half * 32 + c;
               float p0 = ex2_approx(fmaf(__uint_as_float(sv[c]), c2, -lse2));
               float p1 = ex2_approx(fmaf(__uint_as_float(sv[c + 1]), c2, -lse2));
-              if (kvmask != ~0ull) {
-                p0 = ((kvmask >> c0) & 1ull) ? p0 : 0.f;
-                p1 = ((kvmask >> (c0 + 1)) & 1ull) ? p1 : 0.f;
+              if (kvmask != 0xffffffffu) {
+                p0 = ((kvmask >> c) & 1u) ? p0 : 0.f;
+                p1 = ((kvmask >> (c + 1)) & 1u) ? p1 : 0.f;
               }
               const float d0 = p0 * (__uint_as_float(dp[c]) - dlt) * g.scale;
               const float d1 = p1 * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
-              pp[half * 16 + (c >> 1)] = pack_bf16x2(p0, p1);
-              pd[half * 16 + (c >> 1)] = pack_bf16x2(d0, d1);
+              pp[c >> 1] = pack_bf16x2(p0, p1);
+              pd[c >> 1] = pack_bf16x2(d0, d1);
             }
           }
           VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
-          store_row_sw128(p_tile, row, pp);
-          store_row_sw128(ds_tile, row, pd);
+          {
+            unsigned char* prow = p_tile + row * 128;
+            unsigned char* drow = ds_tile + row * 128;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+              const int off = ((half * 4 + ch) ^ (row & 7)) << 4;
+              *reinterpret_cast<uint4*>(prow + off) = make_uint4(pp[4 * ch], pp[4 * ch + 1], pp[4 * ch + 2], pp[4 * ch + 3]);
+              *reinterpret_cast<uint4*>(drow + off) = make_uint4(pd[4 * ch], pd[4 * ch + 1], pd[4 * ch + 2], pd[4 * ch + 3]);
+            }
+          }
           tc::fence_proxy_async_smem();
           tc::mbar_arrive(&misc->ds_ready[0]);
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
       }
-      // epilogue: dK[l, d] = dK^T[d, kv] + sum_heads dK_c[j, d] / count(j), same for dV; 32 key columns at a time
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
+      // epilogue: dK[l, d] = dK^T[d, kv] + sum_heads dK_c[j, d] / count(j), same for dV; this thread owns 32 key columns
+      {
         uint32_t kk[32], vv[32];
         if (k > 0) {
           tc::tmem_ld32(lane_addr + 256 + half * 32, kk);
           tc::tmem_ld32(lane_addr + 320 + half * 32, vv);
           tc::tmem_ld_wait();
-          if (half == 1) {
-            tc::tc_fence_before();
-            tc::mbar_arrive(&misc->o_empty);
-          }
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->o_empty);
         } else {
 #pragma unroll
           for (int c = 0; c < 32; ++c) { kk[c] = 0u; vv[c] = 0u; }
@@ -655,27 +661,27 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
           }
         } else {
-          // bf16: transpose 32 key rows through shared memory (P and dS buffers are idle), then 16-byte stores
-          bf16* st_k = reinterpret_cast<bf16*>(p_tile);       // [32 kv][D]
-          bf16* st_v = reinterpret_cast<bf16*>(ds_tile);      // [32 kv][D]
+          // bf16: transpose through shared memory (the P and dS buffers are idle now), then 16-byte stores
+          bf16* st_k = reinterpret_cast<bf16*>(p_tile);       // [64 kv][D]
+          bf16* st_v = reinterpret_cast<bf16*>(ds_tile);      // [64 kv][D]
           if (row < D) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
-              st_k[c * D + row] = __float2bfloat16_rn(__uint_as_float(kk[c]) + coarse_k);
-              st_v[c * D + row] = __float2bfloat16_rn(__uint_as_float(vv[c]) + coarse_v);
+              st_k[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(kk[c]) + coarse_k);
+              st_v[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(vv[c]) + coarse_v);
             }
           }
-          tc::named_bar_sync(1, 128);
+          tc::named_bar_sync(1, 256);
           constexpr int CH = D / 8;
-          for (int e = sm_tid; e < 32 * CH; e += 128) {
+          for (int e = sm_tid; e < 64 * CH; e += 256) {
             const int c = e / CH, ch = e % CH;
-            const int l = misc->tok[tb][half * 32 + c];
+            const int l = misc->tok[tb][c];
             if (l < 0) continue;
             const size_t idx = ((size_t)bhk * g.L + l) * D + ch * 8;
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dk) + idx) = *reinterpret_cast<const uint4*>(st_k + c * D + ch * 8);
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dv) + idx) = *reinterpret_cast<const uint4*>(st_v + c * D + ch * 8);
           }
-          tc::named_bar_sync(1, 128);
+          tc::named_bar_sync(1, 256);
         }
       }
       if (k > 0) ++n_items;
