@@ -61,6 +61,8 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
                                          the exact running row maximum (the tensor-core kernel falls back to it only
                                          for query blocks whose softmax sums leave the safe range) */
 enum { VSA2_FLAG_SIMPLE_ROUTER = 8 }; /* validation aid: router scores with the slow first-generation kernel */
+enum { VSA2_FLAG_SIMPLE_COARSE = 16 };/* validation aid: coarse branch (forward and backward) with the fp32 SIMT kernels
+                                         instead of the TF32 tensor-core ones */
 enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */
 
 /* Problem statement (host struct). */

@@ -21,6 +21,7 @@ FLAG_NO_COARSE = 1
 FLAG_EXACT_MAX_FWD = 2
 FLAG_SIMPLE_BWD = 4
 FLAG_SIMPLE_ROUTER = 8
+FLAG_SIMPLE_COARSE = 16
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4

@@ -267,7 +267,10 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
       VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
     }
     ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, 1);
-    VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+    if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
+      VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+    else
+      VSA2_CUDA(launch_coarse_fwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
   }
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
   if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
@@ -324,8 +327,12 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   }
   if (coarse) {
     ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, 2);
-    VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
-                                at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
+    if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
+      VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
+                                  at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
+    else
+      VSA2_CUDA(launch_coarse_bwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
+                                     at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);

@@ -1,0 +1,343 @@
+// Coarse branch on the pooled tokens (paper Eq. 2-3) and its backward with TF32 tensor-core tiles.
+// The pooled tensors are fp32 means of 64 tokens; the products run as TF32 (10-bit mantissa) with fp32
+// accumulation, softmax statistics in fp32.  Dense attention over N cubes: 1/B^2 of the dense FLOPs.
+#include <mma.h>
+
+#include "common.cuh"
+
+namespace vsa2 {
+
+using namespace nvcuda;
+
+constexpr int kCT = 64;    // rows per tile (queries and keys)
+
+template <int D>
+struct CoarseTc {
+  static constexpr int LDX = D + 4;     // fp32 operand tiles
+  static constexpr int LDS = kCT + 4;   // fp32 score tiles
+  static constexpr size_t tile = (size_t)kCT * LDX * sizeof(float);
+  static constexpr size_t score = (size_t)kCT * LDS * sizeof(float);
+  static constexpr size_t fwd_bytes = 4 * tile + score + 3 * kCT * sizeof(float);          // Q, K, V, O, S
+  static constexpr size_t bwd_bytes = 4 * tile + 2 * score + 4 * kCT * sizeof(float);      // 4 operand tiles, S, dP
+};
+
+typedef wmma::fragment<wmma::matrix_a, 16, 16, 8, wmma::precision::tf32, wmma::row_major> FragA;
+typedef wmma::fragment<wmma::matrix_a, 16, 16, 8, wmma::precision::tf32, wmma::col_major> FragAT;
+typedef wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::row_major> FragB;
+typedef wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::col_major> FragBT;
+typedef wmma::fragment<wmma::accumulator, 16, 16, 8, float> FragC;
+
+template <typename F>
+__device__ __forceinline__ void to_tf32(F& f) {
+#pragma unroll
+  for (int i = 0; i < f.num_elements; ++i) f.x[i] = wmma::__float_to_tf32(f.x[i]);
+}
+
+// C[64 x 64] = A[64 x D] * B[64 x D]^T  (both row-major in shared memory), 8 warps, 2 output tiles each
+template <int D>
+__device__ __forceinline__ void scores_64x64(const float* A, const float* B, float* C) {
+  constexpr int LDX = D + 4, LDS = kCT + 4;
+  const int warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int t = warp * 2 + i, tm = t >> 2, tn = t & 3;
+    FragC acc;
+    wmma::fill_fragment(acc, 0.f);
+#pragma unroll 4
+    for (int k = 0; k < D; k += 8) {
+      FragA a;
+      FragBT b;
+      wmma::load_matrix_sync(a, A + tm * 16 * LDX + k, LDX);
+      wmma::load_matrix_sync(b, B + tn * 16 * LDX + k, LDX);
+      to_tf32(a);
+      to_tf32(b);
+      wmma::mma_sync(acc, a, b, acc);
+    }
+    wmma::store_matrix_sync(C + tm * 16 * LDS + tn * 16, acc, LDS, wmma::mem_row_major);
+  }
+}
+
+// acc tiles (this warp owns output tiles warp*4 .. warp*4+3 of a [64 x D] result, tile = (tm, tn) with tn fastest)
+//   TRANS_W = false: out += W[64 x 64] * X[64 x D];   TRANS_W = true: out += W^T * X
+template <int D, bool TRANS_W>
+__device__ __forceinline__ void accumulate_64xD(FragC (&acc)[D / 32], const float* W, const float* X) {
+  constexpr int LDX = D + 4, LDS = kCT + 4, TN = D / 16;
+  const int warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < D / 32; ++i) {
+    const int t = warp * (D / 32) + i, tm = t / TN, tn = t % TN;
+#pragma unroll
+    for (int k = 0; k < kCT; k += 8) {
+      FragB b;
+      wmma::load_matrix_sync(b, X + k * LDX + tn * 16, LDX);
+      to_tf32(b);
+      if constexpr (TRANS_W) {
+        FragAT a;
+        wmma::load_matrix_sync(a, W + k * LDS + tm * 16, LDS);
+        to_tf32(a);
+        wmma::mma_sync(acc[i], a, b, acc[i]);
+      } else {
+        FragA a;
+        wmma::load_matrix_sync(a, W + tm * 16 * LDS + k, LDS);
+        to_tf32(a);
+        wmma::mma_sync(acc[i], a, b, acc[i]);
+      }
+    }
+  }
+}
+
+template <int D>
+__device__ __forceinline__ void load_tile(float* dst, const float* src, int row0, int limit) {
+  constexpr int LDX = D + 4, CH = D / 4;
+  for (int e = threadIdx.x; e < kCT * CH; e += blockDim.x) {
+    const int r = e / CH, c = e % CH;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row0 + r < limit) v = __ldg(reinterpret_cast<const float4*>(src + (size_t)(row0 + r) * D + c * 4));
+    *reinterpret_cast<float4*>(dst + r * LDX + c * 4) = v;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- forward
+// grid (ceil(N/64), Hq, batch), 256 threads
+template <int D>
+__global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restrict__ qc, const float* __restrict__ kc,
+                                                            const float* __restrict__ vc, Geo g,
+                                                            float* __restrict__ oc_hat, float* __restrict__ lse_c) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  using C = CoarseTc<D>;
+  float* Qs = reinterpret_cast<float*>(smem_raw);
+  float* Ks = Qs + kCT * C::LDX;
+  float* Vs = Ks + kCT * C::LDX;
+  float* Os = Vs + kCT * C::LDX;
+  float* S = Os + kCT * C::LDX;
+  float* row_m = S + kCT * C::LDS;
+  float* row_l = row_m + kCT;
+  const int hq = blockIdx.y, b = blockIdx.z, hk = hq / g.rep;
+  const int i0 = blockIdx.x * kCT;
+  const size_t qoff = (size_t)(b * g.Hq + hq) * g.N * D, koff = (size_t)(b * g.Hkv + hk) * g.N * D;
+  load_tile<D>(Qs, qc + qoff, i0, g.N);
+  for (int e = threadIdx.x; e < kCT * C::LDX; e += blockDim.x) Os[e] = 0.f;
+  if (threadIdx.x < kCT) { row_m[threadIdx.x] = -INFINITY; row_l[threadIdx.x] = 0.f; }
+  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  for (int j0 = 0; j0 < g.N; j0 += kCT) {
+    __syncthreads();
+    load_tile<D>(Ks, kc + koff, j0, g.N);
+    load_tile<D>(Vs, vc + koff, j0, g.N);
+    __syncthreads();
+    scores_64x64<D>(Qs, Ks, S);
+    __syncthreads();
+    {
+      float x[16];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const int col = qd * 16 + c;
+        x[c] = (j0 + col < g.N) ? S[r * C::LDS + col] * g.scale : -INFINITY;
+        mx = fmaxf(mx, x[c]);
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_old = row_m[r], m_new = fmaxf(m_old, mx);
+      float ps = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const float p = __expf(x[c] - m_new);
+        S[r * C::LDS + qd * 16 + c] = p;
+        ps += p;
+      }
+      ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+      const float alpha = __expf(m_old - m_new);
+      for (int c = 0; c < D / 4; ++c) Os[r * C::LDX + qd * (D / 4) + c] *= alpha;
+      __syncwarp();
+      if (qd == 0) { row_m[r] = m_new; row_l[r] = row_l[r] * alpha + ps; }
+    }
+    __syncthreads();
+    {
+      // O += P V with the accumulator round-tripping through shared memory (rows were just rescaled there)
+      constexpr int TN = D / 16;
+      const int warp = threadIdx.x >> 5;
+#pragma unroll
+      for (int i = 0; i < D / 32; ++i) {
+        const int t = warp * (D / 32) + i, tm = t / TN, tn = t % TN;
+        FragC acc;
+        wmma::load_matrix_sync(acc, Os + tm * 16 * C::LDX + tn * 16, C::LDX, wmma::mem_row_major);
+#pragma unroll
+        for (int k = 0; k < kCT; k += 8) {
+          FragA a;
+          FragB bfr;
+          wmma::load_matrix_sync(a, S + tm * 16 * C::LDS + k, C::LDS);
+          wmma::load_matrix_sync(bfr, Vs + k * C::LDX + tn * 16, C::LDX);
+          to_tf32(a);
+          to_tf32(bfr);
+          wmma::mma_sync(acc, a, bfr, acc);
+        }
+        wmma::store_matrix_sync(Os + tm * 16 * C::LDX + tn * 16, acc, C::LDX, wmma::mem_row_major);
+      }
+    }
+  }
+  __syncthreads();
+  const int i = i0 + r;
+  if (i < g.N) {
+    const float inv = 1.f / row_l[r];
+    for (int c = 0; c < D / 4; ++c) {
+      const int d = qd * (D / 4) + c;
+      oc_hat[qoff + (size_t)i * D + d] = Os[r * C::LDX + d] * inv;
+    }
+    if (qd == 0) lse_c[(size_t)(b * g.Hq + hq) * g.N + i] = row_m[r] + __logf(row_l[r]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- backward
+// ROWS = true : 64 query cubes stationary; streams key tiles; writes dQ_c and delta_c.
+// ROWS = false: 64 key cubes stationary; streams query tiles; writes dK_c, dV_c (per query head).
+// dS = P * (dP - delta_c) * scale, P = exp(S*scale - lse_c), dP = dO_c_hat V_c^T, delta_c = rowsum(dO_c_hat * O_c_hat).
+template <int D, bool ROWS>
+__global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restrict__ qc, const float* __restrict__ kc,
+                                                            const float* __restrict__ vc, const float* __restrict__ oc_hat,
+                                                            const float* __restrict__ lse_c, const float* __restrict__ d_oc,
+                                                            Geo g, float* __restrict__ delta_c, float* __restrict__ out0,
+                                                            float* __restrict__ out1) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  using C = CoarseTc<D>;
+  float* X0 = reinterpret_cast<float*>(smem_raw);   // stationary operand of the score product (Q or K)
+  float* X1 = X0 + kCT * C::LDX;                    // stationary operand of the dP product (dO_c or V)
+  float* Y0 = X1 + kCT * C::LDX;                    // streamed operand of the score product (K or Q)
+  float* Y1 = Y0 + kCT * C::LDX;                    // streamed operand of the dP product (V or dO_c)
+  float* S = Y1 + kCT * C::LDX;                     // scores -> P   [query][key]
+  float* dP = S + kCT * C::LDS;                     // dP -> dS      [query][key]
+  float* q_lse = dP + kCT * C::LDS;                 // per query row of the current (query) tile
+  float* q_delta = q_lse + kCT;
+  const int hq = blockIdx.y, b = blockIdx.z, hk = hq / g.rep;
+  const int s0 = blockIdx.x * kCT;
+  const size_t qoff = (size_t)(b * g.Hq + hq) * g.N * D, koff = (size_t)(b * g.Hkv + hk) * g.N * D;
+  const size_t roff = (size_t)(b * g.Hq + hq) * g.N;
+  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  if (ROWS) {
+    load_tile<D>(X0, qc + qoff, s0, g.N);
+    load_tile<D>(X1, d_oc + qoff, s0, g.N);
+    __syncthreads();
+    // delta_c of the stationary query rows
+    float acc = 0.f;
+    const int i = s0 + r;
+    if (i < g.N)
+      for (int c = 0; c < D / 4; ++c) {
+        const int d = qd * (D / 4) + c;
+        acc = fmaf(X1[r * C::LDX + d], __ldg(oc_hat + qoff + (size_t)i * D + d), acc);
+      }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    if (qd == 0) {
+      q_delta[r] = acc;
+      q_lse[r] = i < g.N ? lse_c[roff + i] : INFINITY;
+      if (i < g.N) delta_c[roff + i] = acc;
+    }
+  } else {
+    load_tile<D>(X0, kc + koff, s0, g.N);
+    load_tile<D>(X1, vc + koff, s0, g.N);
+  }
+  FragC acc0[D / 32], acc1[D / 32];
+#pragma unroll
+  for (int i = 0; i < D / 32; ++i) { wmma::fill_fragment(acc0[i], 0.f); wmma::fill_fragment(acc1[i], 0.f); }
+
+  for (int j0 = 0; j0 < g.N; j0 += kCT) {
+    __syncthreads();
+    if (ROWS) {
+      load_tile<D>(Y0, kc + koff, j0, g.N);
+      load_tile<D>(Y1, vc + koff, j0, g.N);
+    } else {
+      load_tile<D>(Y0, qc + qoff, j0, g.N);
+      load_tile<D>(Y1, d_oc + qoff, j0, g.N);
+      if (threadIdx.x < kCT) {
+        const int i = j0 + threadIdx.x;
+        q_lse[threadIdx.x] = i < g.N ? lse_c[roff + i] : INFINITY;
+        q_delta[threadIdx.x] = i < g.N ? delta_c[roff + i] : 0.f;
+      }
+    }
+    __syncthreads();
+    // S[query][key], dP[query][key]
+    if (ROWS) {
+      scores_64x64<D>(X0, Y0, S);
+      scores_64x64<D>(X1, Y1, dP);
+    } else {
+      scores_64x64<D>(Y0, X0, S);
+      scores_64x64<D>(Y1, X1, dP);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < kCT * kCT; e += blockDim.x) {
+      const int qi = e >> 6, ki = e & 63;
+      const bool ok = ROWS ? (j0 + ki < g.N) : (s0 + ki < g.N);     // the key must exist (missing queries carry lse = +inf)
+      const float p = ok ? __expf(S[qi * C::LDS + ki] * g.scale - q_lse[qi]) : 0.f;
+      const float ds = p * (dP[qi * C::LDS + ki] - q_delta[qi]) * g.scale;
+      S[qi * C::LDS + ki] = p;
+      dP[qi * C::LDS + ki] = ds;
+    }
+    __syncthreads();
+    if (ROWS) {
+      accumulate_64xD<D, false>(acc0, dP, Y0);        // dQ_c += dS K_c
+    } else {
+      accumulate_64xD<D, true>(acc0, dP, Y0);         // dK_c += dS^T Q_c
+      accumulate_64xD<D, true>(acc1, S, Y1);          // dV_c += P^T dO_c_hat
+    }
+  }
+  // accumulators -> shared memory (operand tiles are idle) -> global
+  __syncthreads();
+  {
+    constexpr int TN = D / 16;
+    const int warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) {
+      const int t = warp * (D / 32) + i, tm = t / TN, tn = t % TN;
+      wmma::store_matrix_sync(Y0 + tm * 16 * C::LDX + tn * 16, acc0[i], C::LDX, wmma::mem_row_major);
+      if (!ROWS) wmma::store_matrix_sync(Y1 + tm * 16 * C::LDX + tn * 16, acc1[i], C::LDX, wmma::mem_row_major);
+    }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < kCT * (D / 4); e += blockDim.x) {
+    const int rr = e / (D / 4), c = e % (D / 4);
+    const int i = s0 + rr;
+    if (i >= g.N) continue;
+    *reinterpret_cast<float4*>(out0 + qoff + (size_t)i * D + c * 4) = *reinterpret_cast<const float4*>(Y0 + rr * C::LDX + c * 4);
+    if (!ROWS)
+      *reinterpret_cast<float4*>(out1 + qoff + (size_t)i * D + c * 4) = *reinterpret_cast<const float4*>(Y1 + rr * C::LDX + c * 4);
+  }
+}
+
+cudaError_t launch_coarse_fwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
+                                 float* lse_c, cudaStream_t st) {
+  dim3 grid((g.N + kCT - 1) / kCT, g.Hq, g.batch);
+  cudaError_t e;
+  if (g.D == 128) {
+    const size_t smb = CoarseTc<128>::fwd_bytes;
+    if ((e = cudaFuncSetAttribute(coarse_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    coarse_fwd_tc_kernel<128><<<grid, 256, smb, st>>>(qc, kc, vc, g, oc_hat, lse_c);
+  } else {
+    const size_t smb = CoarseTc<64>::fwd_bytes;
+    if ((e = cudaFuncSetAttribute(coarse_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    coarse_fwd_tc_kernel<64><<<grid, 256, smb, st>>>(qc, kc, vc, g, oc_hat, lse_c);
+  }
+  return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t coarse_bwd_tc_t(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
+                                   const float* lse_c, const float* d_oc, float* delta_c, float* dqc, float* dkc,
+                                   float* dvc, cudaStream_t st) {
+  dim3 grid((g.N + kCT - 1) / kCT, g.Hq, g.batch);
+  const size_t smb = CoarseTc<D>::bwd_bytes;
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(coarse_bwd_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+  if ((e = cudaFuncSetAttribute(coarse_bwd_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+  coarse_bwd_tc_kernel<D, true><<<grid, 256, smb, st>>>(qc, kc, vc, oc_hat, lse_c, d_oc, g, delta_c, dqc, nullptr);
+  coarse_bwd_tc_kernel<D, false><<<grid, 256, smb, st>>>(qc, kc, vc, oc_hat, lse_c, d_oc, g, delta_c, dkc, dvc);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_coarse_bwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
+                                 const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
+                                 float* dvc, cudaStream_t st) {
+  if (g.D == 128) return coarse_bwd_tc_t<128>(g, qc, kc, vc, oc_hat, lse_c, d_oc_hat, delta_c, dqc, dkc, dvc, st);
+  return coarse_bwd_tc_t<64>(g, qc, kc, vc, oc_hat, lse_c, d_oc_hat, delta_c, dqc, dkc, dvc, st);
+}
+
+}  // namespace vsa2

@@ -137,6 +137,11 @@ cudaError_t launch_coarse_fwd(const Geo& g, const float* qc, const float* kc, co
 cudaError_t launch_coarse_bwd(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
                               const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
                               float* dvc, cudaStream_t st);
+cudaError_t launch_coarse_fwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
+                                 float* lse_c, cudaStream_t st);
+cudaError_t launch_coarse_bwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
+                                 const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
+                                 float* dvc, cudaStream_t st);
 
 cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
                             const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,

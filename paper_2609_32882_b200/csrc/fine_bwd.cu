@@ -21,30 +21,68 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restr
                                                              const float* __restrict__ oc_hat, Geo g,
                                                              float* __restrict__ delta, float* __restrict__ dgate,
                                                              float* __restrict__ d_oc_hat) {
-  __shared__ float gdo[64][D];   // gate_l * dO_l
+  // HBM-bound: one pass over dO and O (and the bf16 residual of O) with 16-byte loads; 4 threads per token row.
+  __shared__ float gdo[64][D + 4];   // gate_l * dO_l
+  __shared__ float ocs[D];
   const int i = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const size_t bhq = (size_t)b * g.Hq + hq;
   const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr;
   const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
-  constexpr int OC = D / 4;
+  constexpr int OC = D / 4;            // channels per thread
   int nt, nh, nw;
   cube_coords(g, i, nt, nh, nw);
   const int l = cube_token(g, nt, nh, nw, r);
+  if (coarse)
+    for (int d = threadIdx.x; d < D; d += blockDim.x) ocs[d] = oc_hat[(bhq * g.N + i) * D + d];
+  __syncthreads();
   float s_oo = 0.f, s_oc = 0.f;
   const float gt = (coarse && l >= 0) ? gate[bhq * g.L + l] : 0.f;
-  const float* oc = oc_hat + (bhq * g.N + i) * D;
-  for (int c = 0; c < OC; ++c) {
-    int d = qd * OC + c;
-    float dov = 0.f;
-    if (l >= 0) {
-      size_t idx = (bhq * g.L + l) * D + d;
-      dov = __bfloat162float(d_o[idx]);
-      float ov = load_out(o, idx, g.out_f32);
-      if (o_res != nullptr) ov += __bfloat162float(o_res[idx]);
-      s_oo = fmaf(dov, ov, s_oo);
-      if (coarse) s_oc = fmaf(dov, oc[d], s_oc);
+  if (l >= 0) {
+    const size_t base = (bhq * g.L + l) * D + qd * OC;
+#pragma unroll
+    for (int c = 0; c < OC; c += 8) {
+      const uint4 dv = __ldg(reinterpret_cast<const uint4*>(d_o + base + c));
+      const __nv_bfloat162* d2 = reinterpret_cast<const __nv_bfloat162*>(&dv);
+      float ov[8];
+      if (g.out_f32) {
+        const float4 a0 = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(o) + base + c));
+        const float4 a1 = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(o) + base + c + 4));
+        ov[0] = a0.x; ov[1] = a0.y; ov[2] = a0.z; ov[3] = a0.w; ov[4] = a1.x; ov[5] = a1.y; ov[6] = a1.z; ov[7] = a1.w;
+      } else {
+        const uint4 ob = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(o) + base + c));
+        const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&ob);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(o2[e]);
+          ov[2 * e] = f.x; ov[2 * e + 1] = f.y;
+        }
+        if (o_res != nullptr) {
+          const uint4 rb = __ldg(reinterpret_cast<const uint4*>(o_res + base + c));
+          const __nv_bfloat162* r2 = reinterpret_cast<const __nv_bfloat162*>(&rb);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(r2[e]);
+            ov[2 * e] += f.x; ov[2 * e + 1] += f.y;
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 dd = __bfloat1622float2(d2[e]);
+        const int d = qd * OC + c + 2 * e;
+        s_oo = fmaf(dd.x, ov[2 * e], s_oo);
+        s_oo = fmaf(dd.y, ov[2 * e + 1], s_oo);
+        if (coarse) {
+          s_oc = fmaf(dd.x, ocs[d], s_oc);
+          s_oc = fmaf(dd.y, ocs[d + 1], s_oc);
+          gdo[r][d] = gt * dd.x;
+          gdo[r][d + 1] = gt * dd.y;
+        }
+      }
     }
-    gdo[r][d] = gt * dov;
+  } else if (coarse) {
+#pragma unroll 4
+    for (int c = 0; c < OC; ++c) gdo[r][qd * OC + c] = 0.f;
   }
   s_oo += __shfl_xor_sync(0xffffffffu, s_oo, 1);
   s_oo += __shfl_xor_sync(0xffffffffu, s_oo, 2);

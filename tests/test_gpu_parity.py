@@ -13,6 +13,7 @@ pytestmark = pytest.mark.gpu
 # small workloads that span several tiles, a ragged (padded) grid and GQA
 MINI_PADDED = syn.Workload("mini_padded_gqa", 1, 4, 2, 128, (5, 6, 9), select_mode=syn.PER_QUERY, topk=3, seed=21)
 MINI_SEQ = syn.Workload("mini_per_sequence", 2, 3, 3, 64, (6, 9, 10), select_mode=syn.PER_SEQUENCE, topk=4, seed=22)
+MINI_COARSE = syn.Workload("mini_two_coarse_tiles", 1, 2, 1, 128, (8, 24, 28), select_mode=syn.PER_QUERY, topk=16, seed=24)
 MINI_BUDGET = syn.Workload("mini_budget", 1, 2, 1, 128, (8, 8, 12), select_mode=syn.PER_QUERY_BUDGET, seed=23)
 
 
@@ -222,3 +223,22 @@ def test_tensor_core_router_matches_first_generation_kernel():
         scores.append(to_f64(run.attn.scores()))
     assert np.abs(scores[0] - scores[1]).max() <= 1e-5 * scores[1].max()
     assert np.allclose(scores[0].sum(axis=-1), 1.0 / 8, atol=1e-5)      # rows of P_r sum to 1/G
+
+
+def test_coarse_branch_spanning_two_tiles_with_a_ragged_tail():
+    # 84 cubes: the coarse kernels' 64-row tiles see one full and one partial tile on both operands
+    full_parity(MINI_COARSE, syn.make_inputs(MINI_COARSE), out_dtype=vb.F32, check_route=False)
+
+
+def test_tensor_core_coarse_branch_matches_fp32_kernels():
+    wl = MINI_COARSE
+    data = syn.make_inputs(wl)
+    outs = []
+    for flags in (0, vb.FLAG_SIMPLE_COARSE):
+        run = GpuRun(wl, data, flags=flags, out_dtype=vb.F32)
+        run.route()
+        O, lse = run.forward()
+        outs.append((O,) + tuple(run.backward()))
+    for name, x, y in zip(("O", "dQ", "dK", "dV", "dGate"), *outs):
+        # TF32 operands carry 2^-11 relative rounding; dGate sums 128 such products of magnitude up to ~4
+        assert np.abs(x - y).max() < 5e-3, name
