@@ -24,43 +24,74 @@
 
 namespace vsa2 {
 
-constexpr int kBwdThreads = 384;   // 4 service warps + 2 x 4 elementwise warps
-constexpr int kBwdMaxCubes = 12288;   // edge-flag table in shared memory: one byte per cube
+constexpr int kBwdThreads = 448;   // 4 service warps, 2 x 4 elementwise warps, 2 more issuer warps
+constexpr int kRingA = 3;          // slots of the ring whose tiles are also an operand of the last product of a tile
+constexpr int kRingB = 2;          // (the ring-B slot of a tile is also the index of its tensor-memory buffers)
+static_assert(kRingB == 2, "ring B shares its slot index with the two accumulator buffers");
 
-// Shared-memory plan of both passes (D = 128: 4 x 32 KB ring slots, 2 x 16 KB stationary tiles, 2 x 16 KB operand
-// buffers): ring A = 2 slots, ring B = 2 slots, each with one producing warp and fixed consuming roles.
+// Shared-memory plan of both passes (D = 128: 5 x 32 KB ring slots, 2 x 16 KB stationary tiles, 2 x 16 KB operand
+// buffers, 2 KB of barriers and per-block vectors: exactly the 227 KB a block may use).  Ring A has 3 slots, ring B 2;
+// each ring has one producing warp and fixed consuming roles.
 template <int D>
 struct BwdTc {
   static constexpr int DH = D / 64;
   static constexpr uint32_t SLOT = 2 * DH * kSlab;   // a pair of cube tiles, [half][A | B]
   static constexpr uint32_t TILE = DH * kSlab;       // one cube tile, [half]
   static constexpr uint32_t PBYTES = 128 * 128;      // 128 rows x 64 bf16
-  static constexpr uint32_t OFF_RING_B = 2 * SLOT;
-  static constexpr uint32_t OFF_ST0 = 4 * SLOT;                // stationary tile 0 (Q or K)
-  static constexpr uint32_t OFF_ST1 = OFF_ST0 + TILE;          // stationary tile 1 (dO or V)
-  static constexpr uint32_t OFF_P = OFF_ST1 + TILE;            // two 16 KB operand buffers
+  static constexpr uint32_t OFF_RING_B = kRingA * SLOT;
+  static constexpr uint32_t OFF_ST0 = (kRingA + kRingB) * SLOT;   // stationary tile 0 (Q or K)
+  static constexpr uint32_t OFF_ST1 = OFF_ST0 + TILE;             // stationary tile 1 (dO or V)
+  static constexpr uint32_t OFF_P = OFF_ST1 + TILE;               // two 16 KB operand buffers
   static constexpr uint32_t OFF_MISC = OFF_P + 2 * PBYTES;
-  static constexpr uint32_t MISC_BYTES = 3072;
-  static size_t smem_bytes(int n_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_cubes + 15) / 16 * 16 + 1024; }
+  static constexpr uint32_t MISC_BYTES = 2048;
+  static constexpr size_t smem_bytes = OFF_MISC + MISC_BYTES + 1024;
 };
 
 struct BwdMisc {
   uint64_t st_full, st_empty, o_full, o_empty;
-  uint64_t a_full[2], a_empty[2], b_full[2], b_empty[2];      // the two rings
-  uint64_t sdp_full[2], sdp_free[2], ds_ready[2], ds_free[2];
+  uint64_t a_full[kRingA], a_empty[kRingA], b_full[kRingB], b_empty[kRingB];
+  uint64_t s_full[2], s_free[2], dp_full[2], dp_free[2];   // the two score / dP accumulators in tensor memory
+  uint64_t p_ready, p_free;                                 // dK/dV pass: the P operand buffer
+  uint64_t ds_ready[2], ds_free[2];                         // dS operand buffers (the dK/dV pass has one)
   uint32_t tmem_base;
   int abort_flag;
   alignas(16) float lse2[2][64];   // dQ pass: per query column, lse * log2(e) (+inf for padding), by item parity
   alignas(16) float delta[2][64];
   int tok[2][64];
 };
-static_assert(sizeof(BwdMisc) <= 3072, "misc region too small");
+static_assert(sizeof(BwdMisc) <= 2048, "misc region too small");
 
-// One warp streams pairs of cube tiles into a two-slot ring: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one box
-// each (half h = lane / 2 of block lane & 1).  `coord_*`: cube coordinates of this lane's block, `bh`: its head index.
-#define VSA2_RING_LOAD(FULL, EMPTY, RING_BASE, TMAP, SEQ, CT, CH, CW, BH)                                         \
+__device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
+  misc->abort_flag = 0;
+  tc::mbar_init(&misc->st_full, 1);
+  tc::mbar_init(&misc->st_empty, 2);     // both first-stage issuers
+  tc::mbar_init(&misc->o_full, 1);       // re-initialised to 2 by the dK/dV pass (two last-stage issuers)
+  tc::mbar_init(&misc->o_empty, 256);
+  for (int s = 0; s < kRingA; ++s) {
+    tc::mbar_init(&misc->a_full[s], 1);
+    tc::mbar_init(&misc->a_empty[s], 1);
+  }
+  for (int s = 0; s < kRingB; ++s) {
+    tc::mbar_init(&misc->b_full[s], 1);
+    tc::mbar_init(&misc->b_empty[s], 1);
+  }
+  for (int s = 0; s < 2; ++s) {
+    tc::mbar_init(&misc->s_full[s], 1);
+    tc::mbar_init(&misc->s_free[s], 256);
+    tc::mbar_init(&misc->dp_full[s], 1);
+    tc::mbar_init(&misc->dp_free[s], 256);
+    tc::mbar_init(&misc->ds_ready[s], 256);
+    tc::mbar_init(&misc->ds_free[s], 1);
+  }
+  tc::mbar_init(&misc->p_ready, 256);
+  tc::mbar_init(&misc->p_free, 1);
+}
+
+// One warp streams pairs of cube tiles into a ring of NS slots: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one
+// box each (half h = lane / 2 of block lane & 1).  `coord_*`: cube coordinates of this lane's block, `bh`: its head.
+#define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH)                                     \
   do {                                                                                                            \
-    const uint32_t slot_ = (SEQ) & 1, par_ = ((SEQ) >> 1) & 1;                                                    \
+    const uint32_t slot_ = (SEQ) % (NS), par_ = ((SEQ) / (NS)) & 1;                                               \
     int ok_ = 1;                                                                                                  \
     if (lane == 0) {                                                                                              \
       ok_ = tc::mbar_wait(&(EMPTY)[slot_], par_ ^ 1, &misc->abort_flag);                                          \
@@ -85,9 +116,10 @@ struct DqArgs {
   StatusBlock* status;
 };
 
-// Roles (384 threads): warp 0 = TMA producer of the K pairs (ring A; held until the dQ^T product of the tile is done)
-// and of the stationary Q and dO tiles, warp 1 = TMA producer of the V pairs (ring B), warp 2 = issuer of S^T and dP^T,
-// warp 3 = issuer of dQ^T += K_pair^T dS^T, warps 4..11 = elementwise stage + epilogue (each half of the query columns).
+// Roles: warp 0 = TMA producer of the K pairs (ring A; a slot is held until the dQ^T product of its tile is done) and of
+// the stationary Q and dO tiles, warp 1 = TMA producer of the V pairs (ring B), warp 2 = issuer of S^T, warp 3 = issuer
+// of dP^T, warp 12 = issuer of dQ^T += K_pair^T dS^T, warps 4..11 = elementwise stage + epilogue (each half of the query
+// columns): P is formed from S^T while dP^T is still being computed.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -100,29 +132,13 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   unsigned char* do_tile = smem + C::OFF_ST1;
   unsigned char* ds_tile = smem + C::OFF_P;      // two buffers
   BwdMisc* misc = reinterpret_cast<BwdMisc*>(smem + C::OFF_MISC);
-  unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_items = g.batch * g.Hq * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
 
-  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
   if (tid == 0) {
-    misc->abort_flag = 0;
-    tc::mbar_init(&misc->st_full, 1);
-    tc::mbar_init(&misc->st_empty, 1);
-    tc::mbar_init(&misc->o_full, 1);
-    tc::mbar_init(&misc->o_empty, 256);
-    for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(&misc->a_full[s], 1);
-      tc::mbar_init(&misc->a_empty[s], 1);
-      tc::mbar_init(&misc->b_full[s], 1);
-      tc::mbar_init(&misc->b_empty[s], 1);
-      tc::mbar_init(&misc->sdp_full[s], 1);
-      tc::mbar_init(&misc->sdp_free[s], 256);
-      tc::mbar_init(&misc->ds_ready[s], 256);
-      tc::mbar_init(&misc->ds_free[s], 1);
-    }
+    bwd_init_barriers(misc);
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -143,9 +159,6 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     // ------------------------------------------------------------------ TMA producers
     const int which = warp;                               // 0: K pairs (ring A) + Q, dO tiles; 1: V pairs (ring B)
     const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
-    uint64_t* full = which == 0 ? misc->a_full : misc->b_full;
-    uint64_t* empty = which == 0 ? misc->a_empty : misc->b_empty;
-    unsigned char* ring = smem + (which == 0 ? 0 : C::OFF_RING_B);
     const int my_blk = lane & 1;
     uint32_t tg = 0, n_items = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
@@ -177,13 +190,16 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         int jt, jh, jw;
         cube_coords(g, j, jt, jh, jw);
         if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
-        VSA2_RING_LOAD(full, empty, ring, tm, tg, jt, jh, jw, bhk);
+        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, jt, jh, jw, bhk);
+        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, jt, jh, jw, bhk);
       }
     }
-  } else if (warp == 2) {
-    // ------------------------------------------------------------------ issuer of S^T = K_pair Q^T and dP^T = V_pair dO^T
+  } else if (warp == 2 || warp == 3) {
+    // ------------------------------------------------------------------ issuers of S^T = K_pair Q^T (warp 2) and
+    // dP^T = V_pair dO^T (warp 3)
     if (lane == 0) {
-      const uint32_t q_addr = tc::smem_u32(q_tile), do_addr = tc::smem_u32(do_tile), base = tc::smem_u32(smem);
+      const bool is_s = warp == 2;
+      const uint32_t b_addr = tc::smem_u32(is_s ? q_tile : do_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         const int i = item % g.N, bhq = item / g.N;
@@ -192,21 +208,28 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->st_full, n_items & 1);
         for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
-          VSA2_WAIT(&misc->a_full[s], par);
-          VSA2_WAIT(&misc->b_full[s], par);
-          VSA2_WAIT(&misc->sdp_free[s], par ^ 1);
-          tc::tc_fence_after();
-          mma_pair_kmajor<D>(tmem_base + s * 64, base + s * C::SLOT, q_addr);
-          mma_pair_kmajor<D>(tmem_base + 128 + s * 64, base + C::OFF_RING_B + s * C::SLOT, do_addr);
-          tc::mma_commit(&misc->sdp_full[s]);
-          tc::mma_commit(&misc->b_empty[s]);
+          const uint32_t sb = tg & 1, pb = (tg >> 1) & 1;
+          if (is_s) {
+            const uint32_t sa = tg % kRingA, pa = (tg / kRingA) & 1;
+            VSA2_WAIT(&misc->a_full[sa], pa);
+            VSA2_WAIT(&misc->s_free[sb], pb ^ 1);
+            tc::tc_fence_after();
+            mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+            tc::mma_commit(&misc->s_full[sb]);
+          } else {
+            VSA2_WAIT(&misc->b_full[sb], pb);
+            VSA2_WAIT(&misc->dp_free[sb], pb ^ 1);
+            tc::tc_fence_after();
+            mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
+            tc::mma_commit(&misc->dp_full[sb]);
+            tc::mma_commit(&misc->b_empty[sb]);
+          }
         }
         tc::mma_commit(&misc->st_empty);
         ++n_items;
       }
     }
-  } else if (warp == 3) {
+  } else if (warp == 12) {
     // ------------------------------------------------------------------ issuer of dQ^T += K_pair^T dS^T
     if (lane == 0) {
       const uint32_t ds_addr = tc::smem_u32(ds_tile), base = tc::smem_u32(smem);
@@ -218,18 +241,18 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
         for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
-          VSA2_WAIT(&misc->ds_ready[s], par);
+          const uint32_t sd = tg & 1, pd = (tg >> 1) & 1, sa = tg % kRingA;
+          VSA2_WAIT(&misc->ds_ready[sd], pd);
           tc::tc_fence_after();
-          mma_pairT_mnmajor<D>(tmem_base + 256, base + s * C::SLOT, ds_addr + s * C::PBYTES, t > 0);
-          tc::mma_commit(&misc->a_empty[s]);
-          tc::mma_commit(&misc->ds_free[s]);
+          mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
+          tc::mma_commit(&misc->a_empty[sa]);
+          tc::mma_commit(&misc->ds_free[sd]);
         }
         tc::mma_commit(&misc->o_full);
         ++n_items;
       }
     }
-  } else {
+  } else if (warp >= 4 && warp < 12) {
     // ------------------------------------------------------------------ elementwise stage + epilogue (256 threads):
     // warps 4..7 take query columns 0..31 of every tile, warps 8..11 columns 32..63
     const int quad = warp & 3;
@@ -266,29 +289,39 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t s = tg & 1, par = (tg >> 1) & 1;
           const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          const bool valid = !dup && cpos.valid(edge[j_next]);
+          const bool valid = !dup && cpos.valid(cube_edge_flags(g, j_next));
           if (t + 1 < nt) j_next = cols[(blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
-          VSA2_WAIT(&misc->sdp_full[s], par);
-          tc::tc_fence_after();
           uint32_t packed[16];
           {
-            uint32_t sv[32], dp[32];
+            uint32_t sv[32];      // S^T, then P^T
+            VSA2_WAIT(&misc->s_full[s], par);
+            tc::tc_fence_after();
             tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
+            tc::tmem_ld_wait();
+            tc::tc_fence_before();
+            tc::mbar_arrive(&misc->s_free[s]);
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) {
+              const float4 ls = lse4[c4];
+              sv[4 * c4 + 0] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 0]), c2, -ls.x)));
+              sv[4 * c4 + 1] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 1]), c2, -ls.y)));
+              sv[4 * c4 + 2] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 2]), c2, -ls.z)));
+              sv[4 * c4 + 3] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 3]), c2, -ls.w)));
+            }
+            uint32_t dp[32];
+            VSA2_WAIT(&misc->dp_full[s], par);
+            tc::tc_fence_after();
             tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
             tc::tmem_ld_wait();
             tc::tc_fence_before();
-            tc::mbar_arrive(&misc->sdp_free[s]);
+            tc::mbar_arrive(&misc->dp_free[s]);
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
-              const float4 ls = lse4[c4], dl = del4[c4];
-              const float p0 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 0]), c2, -ls.x));
-              const float p1 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 1]), c2, -ls.y));
-              const float p2 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 2]), c2, -ls.z));
-              const float p3 = ex2_approx(fmaf(__uint_as_float(sv[4 * c4 + 3]), c2, -ls.w));
-              const float d0 = p0 * (__uint_as_float(dp[4 * c4 + 0]) - dl.x) * g.scale;
-              const float d1 = p1 * (__uint_as_float(dp[4 * c4 + 1]) - dl.y) * g.scale;
-              const float d2 = p2 * (__uint_as_float(dp[4 * c4 + 2]) - dl.z) * g.scale;
-              const float d3 = p3 * (__uint_as_float(dp[4 * c4 + 3]) - dl.w) * g.scale;
+              const float4 dl = del4[c4];
+              const float d0 = __uint_as_float(sv[4 * c4 + 0]) * (__uint_as_float(dp[4 * c4 + 0]) - dl.x) * g.scale;
+              const float d1 = __uint_as_float(sv[4 * c4 + 1]) * (__uint_as_float(dp[4 * c4 + 1]) - dl.y) * g.scale;
+              const float d2 = __uint_as_float(sv[4 * c4 + 2]) * (__uint_as_float(dp[4 * c4 + 2]) - dl.z) * g.scale;
+              const float d3 = __uint_as_float(sv[4 * c4 + 3]) * (__uint_as_float(dp[4 * c4 + 3]) - dl.w) * g.scale;
               packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
               packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
             }
@@ -385,19 +418,20 @@ struct DkvArgs {
 constexpr int kMaxRep = 16;   // query heads per KV head the dK/dV pass supports
 
 // entry e of the concatenated column lists of the group's query heads -> (query head, query block)
-__device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b, int hk, int j, const int* cnt_prefix,
-                                          int e, int& bhq, int& i) {
+// (`cnt_prefix`, `col_beg`: per-head counts prefix and list starts of the item, read once per item so that this lookup
+// costs a single global load)
+__device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b, int hk, const int* cnt_prefix,
+                                          const int* col_beg, int e, int& bhq, int& i) {
   int hh = 0;
   while (hh + 1 < g.rep && e >= cnt_prefix[hh + 1]) ++hh;
   bhq = b * g.Hq + hk * g.rep + hh;
-  const int beg = a.col_ptr[(size_t)bhq * (g.N + 1) + j];
-  i = a.row_idx[(size_t)bhq * g.nnz_cap + beg + (e - cnt_prefix[hh])];
+  i = a.row_idx[(size_t)bhq * g.nnz_cap + col_beg[hh] + (e - cnt_prefix[hh])];
 }
 
-// Roles (384 threads): warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA
-// producer of the dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T and dP = dO_pair V^T, warp 3 = issuer of
-// dV^T += dO_pair^T P and dK^T += Q_pair^T dS (both rings are held until these are done), warps 4..11 = elementwise
-// stage + epilogue (each half of the key columns).
+// Roles: warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA producer of the
+// dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T, warp 3 = issuer of dP = dO_pair V^T, warp 12 = issuer of
+// dV^T += dO_pair^T P (frees the dO slot), warp 13 = issuer of dK^T += Q_pair^T dS (frees the Q slot), warps 4..11 =
+// elementwise stage + epilogue (each half of the key columns): P is handed to the dV^T product before dS is formed.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -417,21 +451,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const float c2 = g.scale * 1.4426950408889634f;
 
   if (tid == 0) {
-    misc->abort_flag = 0;
-    tc::mbar_init(&misc->st_full, 1);
-    tc::mbar_init(&misc->st_empty, 1);
-    tc::mbar_init(&misc->o_full, 1);
-    tc::mbar_init(&misc->o_empty, 256);
-    for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(&misc->a_full[s], 1);
-      tc::mbar_init(&misc->a_empty[s], 1);
-      tc::mbar_init(&misc->b_full[s], 1);
-      tc::mbar_init(&misc->b_empty[s], 1);
-      tc::mbar_init(&misc->sdp_full[s], 1);
-      tc::mbar_init(&misc->sdp_free[s], 256);
-      tc::mbar_init(&misc->ds_ready[s], 256);
-      tc::mbar_init(&misc->ds_free[s], 1);
-    }
+    bwd_init_barriers(misc);
+    tc::mbar_init(&misc->o_full, 2);
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -448,15 +469,16 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const uint32_t tmem_base = misc->tmem_base;
   // tensor-memory columns: S buffers 0, 64; dP buffers 128, 192; dK^T 256; dV^T 320
 
-  // per item: prefix of the per-head column counts (every role recomputes it)
+  // per item: prefix of the per-head column counts and the list starts (every role recomputes them)
 #define VSA2_DKV_ITEM_SETUP()                                                            \
   const int j = item % g.N, bhk = item / g.N;                                            \
   const int b = bhk / g.Hkv, hk = bhk % g.Hkv;                                           \
-  int cnt_prefix[kMaxRep + 1];                                                           \
+  int cnt_prefix[kMaxRep + 1], col_beg[kMaxRep];                                         \
   cnt_prefix[0] = 0;                                                                     \
   for (int hh = 0; hh < g.rep; ++hh) {                                                   \
     const size_t base_ = (size_t)(b * g.Hq + hk * g.rep + hh) * (g.N + 1) + j;           \
-    cnt_prefix[hh + 1] = cnt_prefix[hh] + (a.col_ptr[base_ + 1] - a.col_ptr[base_]);     \
+    col_beg[hh] = a.col_ptr[base_];                                                      \
+    cnt_prefix[hh + 1] = cnt_prefix[hh] + (a.col_ptr[base_ + 1] - col_beg[hh]);          \
   }                                                                                      \
   const int k = cnt_prefix[g.rep];
 
@@ -464,9 +486,6 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // ------------------------------------------------------------------ TMA producers
     const int which = warp;                               // 0: Q pairs (ring A) + K, V tiles; 1: dO pairs (ring B)
     const CUtensorMap* tm = which == 0 ? &tm_q : &tm_do;
-    uint64_t* full = which == 0 ? misc->a_full : misc->b_full;
-    uint64_t* empty = which == 0 ? misc->a_empty : misc->b_empty;
-    unsigned char* ring = smem + (which == 0 ? 0 : C::OFF_RING_B);
     const int my_blk = lane & 1;
     uint32_t tg = 0, n_items = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
@@ -489,59 +508,80 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
       ++n_items;
       const int nt = (k + 1) >> 1;
+      int bhq_l, i_l;           // this lane's entry of the tile, fetched one tile ahead of the slot wait
+      dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && k > 1) ? 1 : 0, bhq_l, i_l);
       for (int t = 0; t < nt; ++t, ++tg) {
-        int bhq_l, i_l;
-        dkv_entry(g, a, b, hk, j, cnt_prefix, (my_blk == 1 && 2 * t + 1 < k) ? 2 * t + 1 : 2 * t, bhq_l, i_l);
         int it_, ih_, iw_;
         cube_coords(g, i_l, it_, ih_, iw_);
-        VSA2_RING_LOAD(full, empty, ring, tm, tg, it_, ih_, iw_, bhq_l);
+        const int bhq_t = bhq_l;
+        if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
+        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, it_, ih_, iw_, bhq_t);
+        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t);
       }
     }
-  } else if (warp == 2) {
-    // ------------------------------------------------------------------ issuer of S = Q_pair K^T and dP = dO_pair V^T
+  } else if (warp == 2 || warp == 3) {
+    // ------------------------------------------------------------------ issuers of S = Q_pair K^T (warp 2) and
+    // dP = dO_pair V^T (warp 3)
     if (lane == 0) {
-      const uint32_t k_addr = tc::smem_u32(k_tile), v_addr = tc::smem_u32(v_tile), base = tc::smem_u32(smem);
+      const bool is_s = warp == 2;
+      const uint32_t b_addr = tc::smem_u32(is_s ? k_tile : v_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         VSA2_DKV_ITEM_SETUP();
-        (void)b; (void)hk; (void)j; (void)bhk;
+        (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->st_full, n_items & 1);
         for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
-          VSA2_WAIT(&misc->a_full[s], par);
-          VSA2_WAIT(&misc->b_full[s], par);
-          VSA2_WAIT(&misc->sdp_free[s], par ^ 1);
-          tc::tc_fence_after();
-          mma_pair_kmajor<D>(tmem_base + s * 64, base + s * C::SLOT, k_addr);
-          mma_pair_kmajor<D>(tmem_base + 128 + s * 64, base + C::OFF_RING_B + s * C::SLOT, v_addr);
-          tc::mma_commit(&misc->sdp_full[s]);
+          const uint32_t sb = tg & 1, pb = (tg >> 1) & 1;
+          if (is_s) {
+            const uint32_t sa = tg % kRingA, pa = (tg / kRingA) & 1;
+            VSA2_WAIT(&misc->a_full[sa], pa);
+            VSA2_WAIT(&misc->s_free[sb], pb ^ 1);
+            tc::tc_fence_after();
+            mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+            tc::mma_commit(&misc->s_full[sb]);
+          } else {
+            VSA2_WAIT(&misc->b_full[sb], pb);
+            VSA2_WAIT(&misc->dp_free[sb], pb ^ 1);
+            tc::tc_fence_after();
+            mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
+            tc::mma_commit(&misc->dp_full[sb]);
+          }
         }
         tc::mma_commit(&misc->st_empty);
         ++n_items;
       }
     }
-  } else if (warp == 3) {
-    // ------------------------------------------------------------------ issuer of dV^T += dO_pair^T P and dK^T += Q_pair^T dS
+  } else if (warp == 12 || warp == 13) {
+    // ------------------------------------------------------------------ issuers of dV^T += dO_pair^T P (warp 12) and
+    // dK^T += Q_pair^T dS (warp 13)
     if (lane == 0) {
-      const uint32_t p_addr = tc::smem_u32(p_tile), ds_addr = tc::smem_u32(ds_tile), base = tc::smem_u32(smem);
+      const bool is_v = warp == 12;
+      const uint32_t b_addr = tc::smem_u32(is_v ? p_tile : ds_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
         VSA2_DKV_ITEM_SETUP();
-        (void)b; (void)hk; (void)j; (void)bhk;
+        (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
         for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t s = tg & 1;
-          VSA2_WAIT(&misc->ds_ready[0], tg & 1);
-          tc::tc_fence_after();
-          mma_pairT_mnmajor<D>(tmem_base + 320, base + C::OFF_RING_B + s * C::SLOT, p_addr, t > 0);    // dV^T += dO^T P
-          mma_pairT_mnmajor<D>(tmem_base + 256, base + s * C::SLOT, ds_addr, t > 0);                  // dK^T += Q^T dS
-          tc::mma_commit(&misc->a_empty[s]);
-          tc::mma_commit(&misc->b_empty[s]);
-          tc::mma_commit(&misc->ds_free[0]);
+          if (is_v) {
+            const uint32_t sv = tg & 1;
+            VSA2_WAIT(&misc->p_ready, tg & 1);
+            tc::tc_fence_after();
+            mma_pairT_mnmajor<D>(tmem_base + 320, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
+            tc::mma_commit(&misc->b_empty[sv]);
+            tc::mma_commit(&misc->p_free);
+          } else {
+            const uint32_t sa = tg % kRingA;
+            VSA2_WAIT(&misc->ds_ready[0], tg & 1);
+            tc::tc_fence_after();
+            mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, b_addr, t > 0);
+            tc::mma_commit(&misc->a_empty[sa]);
+            tc::mma_commit(&misc->ds_free[0]);
+          }
         }
         tc::mma_commit(&misc->o_full);
         ++n_items;
@@ -583,28 +623,39 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       tc::named_bar_sync(1, 256);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
-        // (head, block, token) of this thread's query row in tile 0, then one tile ahead
+        // Software pipeline over the tiles: the (head, block) entry of this thread's query row is fetched two tiles
+        // ahead and its lse / delta one tile ahead, so no global-memory latency sits between two tiles.
+        // (the loaded values are not touched before the tile's wait: an arithmetic use would stall the warp on the load)
+        auto row_stats = [&](int bhq_r, int i_r, int t_r, float& lse_r, float& dlt_r) -> bool {
+          int it_, ih_, iw_;
+          cube_coords(g, i_r, it_, ih_, iw_);
+          const bool dup = (blk == 1) && (2 * t_r + 1 >= k);
+          const int l = dup ? -1 : cube_token(g, it_, ih_, iw_, row & 63);
+          const size_t idx = l >= 0 ? (size_t)bhq_r * g.L + l : 0;
+          lse_r = a.lse[idx];
+          dlt_r = a.delta[idx];
+          return l >= 0;
+        };
         int bhq_n, i_n;
-        dkv_entry(g, a, b, hk, j, cnt_prefix, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
+        float lse_raw, dlt_raw, lse_raw_next = 0.f, dlt_raw_next = 0.f;
+        dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
+        bool row_ok = row_stats(bhq_n, i_n, 0, lse_raw, dlt_raw), row_ok_next = false;
+        if (nt > 1) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 3 < k) ? 3 : 2, bhq_n, i_n);
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t s = tg & 1, par = (tg >> 1) & 1;
-          const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          int it_, ih_, iw_;
-          cube_coords(g, i_n, it_, ih_, iw_);
-          const int l = dup ? -1 : cube_token(g, it_, ih_, iw_, row & 63);
-          const float lse2 = l >= 0 ? a.lse[(size_t)bhq_n * g.L + l] * 1.4426950408889634f : INFINITY;
-          const float dlt = l >= 0 ? a.delta[(size_t)bhq_n * g.L + l] : 0.f;
-          if (t + 1 < nt) dkv_entry(g, a, b, hk, j, cnt_prefix, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
-          VSA2_WAIT(&misc->sdp_full[s], par);
+          if (t + 1 < nt) row_ok_next = row_stats(bhq_n, i_n, t + 1, lse_raw_next, dlt_raw_next);
+          if (t + 2 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 5 < k) ? 2 * t + 5 : 2 * t + 4, bhq_n, i_n);
+          uint32_t sv[32];      // S, then P
+          VSA2_WAIT(&misc->s_full[s], par);
           tc::tc_fence_after();
-          uint32_t pp[16], pd[16];
+          tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
+          tc::tmem_ld_wait();
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->s_free[s]);
+          const float lse2 = row_ok ? lse_raw * 1.4426950408889634f : INFINITY;
+          const float dlt = row_ok ? dlt_raw : 0.f;
           {
-            uint32_t sv[32], dp[32];
-            tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
-            tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
-            tc::tmem_ld_wait();
-            tc::tc_fence_before();
-            tc::mbar_arrive(&misc->sdp_free[s]);
+            uint32_t pp[16];
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
               float p0 = ex2_approx(fmaf(__uint_as_float(sv[c]), c2, -lse2));
@@ -613,25 +664,45 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 p0 = ((kvmask >> c) & 1u) ? p0 : 0.f;
                 p1 = ((kvmask >> (c + 1)) & 1u) ? p1 : 0.f;
               }
-              const float d0 = p0 * (__uint_as_float(dp[c]) - dlt) * g.scale;
-              const float d1 = p1 * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
+              sv[c] = __float_as_uint(p0);
+              sv[c + 1] = __float_as_uint(p1);
               pp[c >> 1] = pack_bf16x2(p0, p1);
+            }
+            VSA2_WAIT(&misc->p_free, (tg & 1) ^ 1);
+            unsigned char* prow = p_tile + row * 128;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch)
+              *reinterpret_cast<uint4*>(prow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
+                  make_uint4(pp[4 * ch], pp[4 * ch + 1], pp[4 * ch + 2], pp[4 * ch + 3]);
+            tc::fence_proxy_async_smem();
+            tc::mbar_arrive(&misc->p_ready);
+          }
+          {
+            uint32_t dp[32], pd[16];
+            VSA2_WAIT(&misc->dp_full[s], par);
+            tc::tc_fence_after();
+            tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
+            tc::tmem_ld_wait();
+            tc::tc_fence_before();
+            tc::mbar_arrive(&misc->dp_free[s]);
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              const float d0 = __uint_as_float(sv[c]) * (__uint_as_float(dp[c]) - dlt) * g.scale;
+              const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
               pd[c >> 1] = pack_bf16x2(d0, d1);
             }
-          }
-          VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
-          {
-            unsigned char* prow = p_tile + row * 128;
+            VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
             unsigned char* drow = ds_tile + row * 128;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              const int off = ((half * 4 + ch) ^ (row & 7)) << 4;
-              *reinterpret_cast<uint4*>(prow + off) = make_uint4(pp[4 * ch], pp[4 * ch + 1], pp[4 * ch + 2], pp[4 * ch + 3]);
-              *reinterpret_cast<uint4*>(drow + off) = make_uint4(pd[4 * ch], pd[4 * ch + 1], pd[4 * ch + 2], pd[4 * ch + 3]);
-            }
+            for (int ch = 0; ch < 4; ++ch)
+              *reinterpret_cast<uint4*>(drow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
+                  make_uint4(pd[4 * ch], pd[4 * ch + 1], pd[4 * ch + 2], pd[4 * ch + 3]);
+            tc::fence_proxy_async_smem();
+            tc::mbar_arrive(&misc->ds_ready[0]);
           }
-          tc::fence_proxy_async_smem();
-          tc::mbar_arrive(&misc->ds_ready[0]);
+          lse_raw = lse_raw_next;
+          dlt_raw = dlt_raw_next;
+          row_ok = row_ok_next;
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
@@ -726,13 +797,12 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
   DqArgs a{lse, delta, row_ptr, col_idx, dqc, dq, status};
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
-  if (g.N > kBwdMaxCubes) return cudaErrorInvalidValue;
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes(g.N)))) return e;
-    fine_bwd_dq_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
+    fine_bwd_dq_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes(g.N)))) return e;
-    fine_bwd_dq_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
+    fine_bwd_dq_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   }
   return cudaGetLastError();
 }
@@ -753,11 +823,11 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes(g.N)))) return e;
-    fine_bwd_dkv_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
+    fine_bwd_dkv_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes(g.N)))) return e;
-    fine_bwd_dkv_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes(g.N), st>>>(tq, tk, tv, tdo, g, a);
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
+    fine_bwd_dkv_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   }
   return cudaGetLastError();
 }
