@@ -44,23 +44,40 @@ struct ProfScope {
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// q = n / d, r = n % d for 0 <= n < 2^22 and 0 < d, through one reciprocal and a fix-up (exact).  The tensor-core
+// kernels decode cube and token indices several times per tile, and a 32-bit integer division costs tens of instructions.
+__device__ __forceinline__ void fast_divmod(int n, int d, int& q, int& r) {
+  q = __float2int_rz(__fdividef((float)n, (float)d));
+  r = n - q * d;
+  if (r < 0) {
+    --q;
+    r += d;
+  } else if (r >= d) {
+    ++q;
+    r -= d;
+  }
+}
+
 // cube n -> (nt, nh, nw);  n = (nt*Nh + nh)*Nw + nw
 __device__ __forceinline__ void cube_coords(const Geo& g, int n, int& nt, int& nh, int& nw) {
-  nw = n % g.Nw;
-  int r = n / g.Nw;
-  nh = r % g.Nh;
-  nt = r / g.Nh;
+  int r;
+  fast_divmod(n, g.Nw, r, nw);
+  fast_divmod(r, g.Nh, nt, nh);
+}
+
+// position (bt, bh, bw) inside cube (nt, nh, nw) -> raster token index, or -1 if padding
+__device__ __forceinline__ int cube_token_at(const Geo& g, int nt, int nh, int nw, int bt, int bh, int bw) {
+  int t = nt * g.Bt + bt, h = nh * g.Bh + bh, w = nw * g.Bw + bw;
+  if (t >= g.T || h >= g.H || w >= g.W) return -1;
+  return (t * g.H + h) * g.W + w;
 }
 
 // position p in [0, B) inside a cube, ordered (bt, bh, bw) -> raster token index, or -1 if padding
 __device__ __forceinline__ int cube_token(const Geo& g, int nt, int nh, int nw, int p) {
-  int bw = p % g.Bw;
-  int r = p / g.Bw;
-  int bh = r % g.Bh;
-  int bt = r / g.Bh;
-  int t = nt * g.Bt + bt, h = nh * g.Bh + bh, w = nw * g.Bw + bw;
-  if (t >= g.T || h >= g.H || w >= g.W) return -1;
-  return (t * g.H + h) * g.W + w;
+  int bw, bh, bt, r;
+  fast_divmod(p, g.Bw, r, bw);
+  fast_divmod(r, g.Bh, bt, bh);
+  return cube_token_at(g, nt, nh, nw, bt, bh, bw);
 }
 
 // 64-bit mask of the valid positions of cube n

@@ -596,6 +596,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int sm_tid = tid - 128;            // 0..255
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const int blk = row >> 6;
+    CubePos cpos;
+    cpos.init(g, row & 63);
     uint32_t tg = 0, n_items = 0, n_all = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
       VSA2_DKV_ITEM_SETUP();
@@ -630,7 +632,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           int it_, ih_, iw_;
           cube_coords(g, i_r, it_, ih_, iw_);
           const bool dup = (blk == 1) && (2 * t_r + 1 >= k);
-          const int l = dup ? -1 : cube_token(g, it_, ih_, iw_, row & 63);
+          const int l = dup ? -1 : cube_token_at(g, it_, ih_, iw_, cpos.bt, cpos.bh, cpos.bw);
           const size_t idx = l >= 0 ? (size_t)bhq_r * g.L + l : 0;
           lse_r = a.lse[idx];
           dlt_r = a.delta[idx];
