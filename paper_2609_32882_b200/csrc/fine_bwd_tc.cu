@@ -24,7 +24,8 @@
 
 namespace vsa2 {
 
-constexpr int kBwdThreads = 448;   // 4 service warps, 2 x 4 elementwise warps, 2 more issuer warps
+constexpr int kDqThreads = 416;    // dQ pass: 4 service warps, 2 x 4 elementwise warps, 1 more issuer warp
+constexpr int kDkvThreads = 576;   // dK/dV pass: 4 service warps, 2 x 4 elementwise warps, 4 row-statistics warps, 2 issuer warps
 constexpr int kRingA = 3;          // slots of the ring whose tiles are also an operand of the last product of a tile
 constexpr int kRingB = 2;          // (the ring-B slot of a tile is also the index of its tensor-memory buffers)
 static_assert(kRingB == 2, "ring B shares its slot index with the two accumulator buffers");
@@ -53,10 +54,14 @@ struct BwdMisc {
   uint64_t s_full[2], s_free[2], dp_full[2], dp_free[2];   // the two score / dP accumulators in tensor memory
   uint64_t p_ready, p_free;                                 // dK/dV pass: the P operand buffer
   uint64_t ds_ready[2], ds_free[2];                         // dS operand buffers (the dK/dV pass has one)
+  uint64_t stat_full, stat_free;                            // dK/dV pass: the per-row statistics of a tile
   uint32_t tmem_base;
   int abort_flag;
-  alignas(16) float lse2[2][64];   // dQ pass: per query column, lse * log2(e) (+inf for padding), by item parity
-  alignas(16) float delta[2][64];
+  unsigned char edge[kRingA][2];   // dQ pass: edge flags of the two key cubes in each ring-A slot (written by its producer)
+  // dQ pass: lse2[tb][c] = stats[tb * 64 + c], delta[tb][c] = stats[128 + tb * 64 + c]: per query column of the item with
+  // parity tb, lse * log2(e) (+inf for padding) and delta.  dK/dV pass: (lse * log2(e), delta) of the 128 query rows of
+  // the current tile, interleaved.
+  alignas(16) float stats[256];
   int tok[2][64];
 };
 static_assert(sizeof(BwdMisc) <= 2048, "misc region too small");
@@ -85,17 +90,23 @@ __device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
   }
   tc::mbar_init(&misc->p_ready, 256);
   tc::mbar_init(&misc->p_free, 1);
+  tc::mbar_init(&misc->stat_full, 128);
+  tc::mbar_init(&misc->stat_free, 256);
 }
 
 // One warp streams pairs of cube tiles into a ring of NS slots: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one
 // box each (half h = lane / 2 of block lane & 1).  `coord_*`: cube coordinates of this lane's block, `bh`: its head.
-#define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH)                                     \
+// `LANE0_PRE`: statement lane 0 runs once the slot is free, before the loads are armed (may use slot_).
+#define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH, LANE0_PRE)                          \
   do {                                                                                                            \
     const uint32_t slot_ = (SEQ) % (NS), par_ = ((SEQ) / (NS)) & 1;                                               \
     int ok_ = 1;                                                                                                  \
     if (lane == 0) {                                                                                              \
       ok_ = tc::mbar_wait(&(EMPTY)[slot_], par_ ^ 1, &misc->abort_flag);                                          \
-      if (ok_) tc::mbar_expect_tx(&(FULL)[slot_], C::SLOT);                                                       \
+      if (ok_) {                                                                                                  \
+        LANE0_PRE;                                                                                                \
+        tc::mbar_expect_tx(&(FULL)[slot_], C::SLOT);                                                              \
+      }                                                                                                           \
     }                                                                                                             \
     if (!__shfl_sync(0xffffffffu, ok_, 0)) goto done;                                                             \
     if (lane < 2 * C::DH)                                                                                         \
@@ -121,7 +132,7 @@ struct DqArgs {
 // of dP^T, warp 12 = issuer of dQ^T += K_pair^T dS^T, warps 4..11 = elementwise stage + epilogue (each half of the query
 // columns): P is formed from S^T while dP^T is still being computed.
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, Geo g,
                       DqArgs a) {
@@ -190,8 +201,13 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         int jt, jh, jw;
         cube_coords(g, j, jt, jh, jw);
         if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
-        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, jt, jh, jw, bhk);
-        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, jt, jh, jw, bhk);
+        if (which == 0) {
+          const unsigned ef0 = cube_edge_flags_at(g, jt, jh, jw), ef1 = __shfl_sync(0xffffffffu, ef0, 1);
+          VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, jt, jh, jw, bhk,
+                         { misc->edge[slot_][0] = (unsigned char)ef0; misc->edge[slot_][1] = (unsigned char)ef1; });
+        } else {
+          VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, jt, jh, jw, bhk, {});
+        }
       }
     }
   } else if (warp == 2 || warp == 3) {
@@ -268,34 +284,32 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       const int i = item % g.N, bhq = item / g.N;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
-      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
       const int tb = n_all & 1;
       if (sm_tid < 64) {
         int it_, ih_, iw_;
         cube_coords(g, i, it_, ih_, iw_);
         const int l = cube_token(g, it_, ih_, iw_, sm_tid);
         misc->tok[tb][sm_tid] = l;
-        misc->lse2[tb][sm_tid] = l >= 0 ? a.lse[(size_t)bhq * g.L + l] * 1.4426950408889634f : INFINITY;
-        misc->delta[tb][sm_tid] = l >= 0 ? a.delta[(size_t)bhq * g.L + l] : 0.f;
+        misc->stats[tb * 64 + sm_tid] = l >= 0 ? a.lse[(size_t)bhq * g.L + l] * 1.4426950408889634f : INFINITY;
+        misc->stats[128 + tb * 64 + sm_tid] = l >= 0 ? a.delta[(size_t)bhq * g.L + l] : 0.f;
       }
       const float coarse_d = (a.dqc != nullptr && row < D)
                                  ? a.dqc[((size_t)bhq * g.N + i) * D + row] / (float)cube_count(g, i) : 0.f;
       tc::named_bar_sync(1, 256);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
-        const float4* lse4 = reinterpret_cast<const float4*>(misc->lse2[tb]) + half * 8;
-        const float4* del4 = reinterpret_cast<const float4*>(misc->delta[tb]) + half * 8;
-        int j_next = cols[(blk == 1 && k > 1) ? 1 : 0];
+        const float4* lse4 = reinterpret_cast<const float4*>(misc->stats + tb * 64) + half * 8;
+        const float4* del4 = reinterpret_cast<const float4*>(misc->stats + 128 + tb * 64) + half * 8;
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t s = tg & 1, par = (tg >> 1) & 1;
           const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          const bool valid = !dup && cpos.valid(cube_edge_flags(g, j_next));
-          if (t + 1 < nt) j_next = cols[(blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
           uint32_t packed[16];
           {
             uint32_t sv[32];      // S^T, then P^T
             VSA2_WAIT(&misc->s_full[s], par);
             tc::tc_fence_after();
+            // (the K slot of the tile, and with it its edge flags, stays until the tile's dQ^T product is done)
+            const bool valid = !dup && cpos.valid(misc->edge[tg % kRingA][blk]);
             tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
             tc::tmem_ld_wait();
             tc::tc_fence_before();
@@ -429,11 +443,13 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b,
 }
 
 // Roles: warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA producer of the
-// dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T, warp 3 = issuer of dP = dO_pair V^T, warp 12 = issuer of
-// dV^T += dO_pair^T P (frees the dO slot), warp 13 = issuer of dK^T += Q_pair^T dS (frees the Q slot), warps 4..11 =
-// elementwise stage + epilogue (each half of the key columns): P is handed to the dV^T product before dS is formed.
+// dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T, warp 3 = issuer of dP = dO_pair V^T, warp 16 = issuer of
+// dV^T += dO_pair^T P (frees the dO slot), warp 17 = issuer of dK^T += Q_pair^T dS (frees the Q slot), warps 4..11 =
+// elementwise stage + epilogue (each half of the key columns): P is handed to the dV^T product before dS is formed;
+// warps 12..15 = one thread per query row of the tile: they look up the row's (head, block, token) and fetch its lse and
+// delta one tile ahead, so that the elementwise warps, which bound the pass, touch no global memory inside a tile.
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(kDkvThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, Geo g,
                        DkvArgs a) {
@@ -452,7 +468,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
   if (tid == 0) {
     bwd_init_barriers(misc);
-    tc::mbar_init(&misc->o_full, 2);
+    tc::mbar_init(&misc->o_full, 2);                                          // two last-stage issuers
+    for (int s = 0; s < kRingB; ++s) tc::mbar_init(&misc->b_empty[s], 2);     // a dO slot is read by dP and by dV^T
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -515,8 +532,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         cube_coords(g, i_l, it_, ih_, iw_);
         const int bhq_t = bhq_l;
         if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
-        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, it_, ih_, iw_, bhq_t);
-        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t);
+        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, it_, ih_, iw_, bhq_t, {});
+        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t, {});
       }
     }
   } else if (warp == 2 || warp == 3) {
@@ -547,17 +564,18 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc::tc_fence_after();
             mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
             tc::mma_commit(&misc->dp_full[sb]);
+            tc::mma_commit(&misc->b_empty[sb]);
           }
         }
         tc::mma_commit(&misc->st_empty);
         ++n_items;
       }
     }
-  } else if (warp == 12 || warp == 13) {
-    // ------------------------------------------------------------------ issuers of dV^T += dO_pair^T P (warp 12) and
-    // dK^T += Q_pair^T dS (warp 13)
+  } else if (warp == 16 || warp == 17) {
+    // ------------------------------------------------------------------ issuers of dV^T += dO_pair^T P (warp 16) and
+    // dK^T += Q_pair^T dS (warp 17)
     if (lane == 0) {
-      const bool is_v = warp == 12;
+      const bool is_v = warp == 16;
       const uint32_t b_addr = tc::smem_u32(is_v ? p_tile : ds_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
@@ -568,7 +586,9 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
         for (int t = 0; t < nt; ++t, ++tg) {
           if (is_v) {
+            // P depends on S only, so it can be ready before the dO pair of the tile has landed: wait for that too
             const uint32_t sv = tg & 1;
+            VSA2_WAIT(&misc->b_full[sv], (tg >> 1) & 1);
             VSA2_WAIT(&misc->p_ready, tg & 1);
             tc::tc_fence_after();
             mma_pairT_mnmajor<D>(tmem_base + 320, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
@@ -587,7 +607,35 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         ++n_items;
       }
     }
-  } else {
+  } else if (warp >= 12 && warp < 16) {
+    // ------------------------------------------------------------------ row statistics of the tiles (128 threads)
+    const int r = tid - 384;                 // query row of the tile
+    const int blk = r >> 6;
+    CubePos cpos;
+    cpos.init(g, r & 63);
+    float2* rowstat = reinterpret_cast<float2*>(misc->stats);
+    uint32_t tg = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      VSA2_DKV_ITEM_SETUP();
+      (void)j; (void)bhk;
+      if (k == 0) continue;
+      const int nt = (k + 1) >> 1;
+      int bhq_n, i_n;
+      dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
+      for (int t = 0; t < nt; ++t, ++tg) {
+        int it_, ih_, iw_;
+        cube_coords(g, i_n, it_, ih_, iw_);
+        const bool dup = (blk == 1) && (2 * t + 1 >= k);
+        const int l = dup ? -1 : cube_token_at(g, it_, ih_, iw_, cpos.bt, cpos.bh, cpos.bw);
+        const size_t idx = l >= 0 ? (size_t)bhq_n * g.L + l : 0;
+        const float lse_raw = a.lse[idx], dlt_raw = a.delta[idx];
+        if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
+        VSA2_WAIT(&misc->stat_free, (tg & 1) ^ 1);
+        rowstat[r] = make_float2(l >= 0 ? lse_raw * 1.4426950408889634f : INFINITY, l >= 0 ? dlt_raw : 0.f);
+        tc::mbar_arrive(&misc->stat_full);
+      }
+    }
+  } else if (warp >= 4 && warp < 12) {
     // ------------------------------------------------------------------ elementwise stage + epilogue (256 threads):
     // warps 4..7 take key columns 0..31 of every tile, warps 8..11 columns 32..63
     const int quad = warp & 3;
@@ -595,12 +643,10 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int row = (quad << 5) | lane;      // query row of the tile (S, dP) / channel (dK^T, dV^T)
     const int sm_tid = tid - 128;            // 0..255
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    const int blk = row >> 6;
-    CubePos cpos;
-    cpos.init(g, row & 63);
     uint32_t tg = 0, n_items = 0, n_all = 0;
     for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
       VSA2_DKV_ITEM_SETUP();
+      (void)col_beg;
       const int tb = n_all & 1;
       int jt, jh, jw;
       cube_coords(g, j, jt, jh, jw);
@@ -625,28 +671,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       tc::named_bar_sync(1, 256);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
-        // Software pipeline over the tiles: the (head, block) entry of this thread's query row is fetched two tiles
-        // ahead and its lse / delta one tile ahead, so no global-memory latency sits between two tiles.
-        // (the loaded values are not touched before the tile's wait: an arithmetic use would stall the warp on the load)
-        auto row_stats = [&](int bhq_r, int i_r, int t_r, float& lse_r, float& dlt_r) -> bool {
-          int it_, ih_, iw_;
-          cube_coords(g, i_r, it_, ih_, iw_);
-          const bool dup = (blk == 1) && (2 * t_r + 1 >= k);
-          const int l = dup ? -1 : cube_token_at(g, it_, ih_, iw_, cpos.bt, cpos.bh, cpos.bw);
-          const size_t idx = l >= 0 ? (size_t)bhq_r * g.L + l : 0;
-          lse_r = a.lse[idx];
-          dlt_r = a.delta[idx];
-          return l >= 0;
-        };
-        int bhq_n, i_n;
-        float lse_raw, dlt_raw, lse_raw_next = 0.f, dlt_raw_next = 0.f;
-        dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
-        bool row_ok = row_stats(bhq_n, i_n, 0, lse_raw, dlt_raw), row_ok_next = false;
-        if (nt > 1) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 3 < k) ? 3 : 2, bhq_n, i_n);
+        const float2* rowstat = reinterpret_cast<const float2*>(misc->stats);
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t s = tg & 1, par = (tg >> 1) & 1;
-          if (t + 1 < nt) row_ok_next = row_stats(bhq_n, i_n, t + 1, lse_raw_next, dlt_raw_next);
-          if (t + 2 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 5 < k) ? 2 * t + 5 : 2 * t + 4, bhq_n, i_n);
+          VSA2_WAIT(&misc->stat_full, tg & 1);
+          const float2 rs = rowstat[row];
+          tc::mbar_arrive(&misc->stat_free);
+          const float lse2 = rs.x, dlt = rs.y;
           uint32_t sv[32];      // S, then P
           VSA2_WAIT(&misc->s_full[s], par);
           tc::tc_fence_after();
@@ -654,8 +685,6 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           tc::tmem_ld_wait();
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->s_free[s]);
-          const float lse2 = row_ok ? lse_raw * 1.4426950408889634f : INFINITY;
-          const float dlt = row_ok ? dlt_raw : 0.f;
           {
             uint32_t pp[16];
 #pragma unroll
@@ -702,9 +731,6 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&misc->ds_ready[0]);
           }
-          lse_raw = lse_raw_next;
-          dlt_raw = dlt_raw_next;
-          row_ok = row_ok_next;
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
@@ -801,10 +827,10 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
   const int grid = total < sms ? total : sms;
   if (g.D == 128) {
     if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
-    fine_bwd_dq_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    fine_bwd_dq_tc_kernel<128><<<grid, kDqThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   } else {
     if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
-    fine_bwd_dq_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    fine_bwd_dq_tc_kernel<64><<<grid, kDqThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   }
   return cudaGetLastError();
 }
@@ -826,10 +852,10 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   const int grid = total < sms ? total : sms;
   if (g.D == 128) {
     if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
-    fine_bwd_dkv_tc_kernel<128><<<grid, kBwdThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    fine_bwd_dkv_tc_kernel<128><<<grid, kDkvThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   } else {
     if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
-    fine_bwd_dkv_tc_kernel<64><<<grid, kBwdThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    fine_bwd_dkv_tc_kernel<64><<<grid, kDkvThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
   }
   return cudaGetLastError();
 }

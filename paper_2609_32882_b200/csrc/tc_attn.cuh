@@ -67,14 +67,17 @@ __device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_sl
 }
 
 // Which cubes are cut by the grid boundary: bit 0 / 1 / 2 = last cube along t / h / w with a partial extent.
-__device__ __forceinline__ unsigned cube_edge_flags(const Geo& g, int n) {
-  int nt, nh, nw;
-  cube_coords(g, n, nt, nh, nw);
+__device__ __forceinline__ unsigned cube_edge_flags_at(const Geo& g, int nt, int nh, int nw) {
   unsigned f = 0;
   if (nt == g.Nt - 1 && g.T % g.Bt) f |= 1u;
   if (nh == g.Nh - 1 && g.H % g.Bh) f |= 2u;
   if (nw == g.Nw - 1 && g.W % g.Bw) f |= 4u;
   return f;
+}
+__device__ __forceinline__ unsigned cube_edge_flags(const Geo& g, int n) {
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  return cube_edge_flags_at(g, nt, nh, nw);
 }
 
 // Position of a token inside its cube and the test "is this position inside the valid grid for a cube with edge flags f".
