@@ -1,6 +1,9 @@
 // Coarse branch on the pooled tokens (paper Eq. 2-3) and its backward with TF32 tensor-core tiles.
 // The pooled tensors are fp32 means of 64 tokens; the products run as TF32 (10-bit mantissa) with fp32
 // accumulation, softmax statistics in fp32.  Dense attention over N cubes: 1/B^2 of the dense FLOPs.
+// Operands are rounded to TF32 once, when they are written to shared memory (tile loads, P and dS), so the
+// fragment loads need no conversion; the k loop is the outer one so that the output tiles of a warp share
+// the fragment of their common operand and their accumulation chains interleave.
 #include <mma.h>
 
 #include "common.cuh"
@@ -27,61 +30,51 @@ typedef wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::r
 typedef wmma::fragment<wmma::matrix_b, 16, 16, 8, wmma::precision::tf32, wmma::col_major> FragBT;
 typedef wmma::fragment<wmma::accumulator, 16, 16, 8, float> FragC;
 
-template <typename F>
-__device__ __forceinline__ void to_tf32(F& f) {
-#pragma unroll
-  for (int i = 0; i < f.num_elements; ++i) f.x[i] = wmma::__float_to_tf32(f.x[i]);
-}
+__device__ __forceinline__ float tf32(float x) { return wmma::__float_to_tf32(x); }
 
-// C[64 x 64] = A[64 x D] * B[64 x D]^T  (both row-major in shared memory), 8 warps, 2 output tiles each
+// C[64 x 64] = A[64 x D] * B[64 x D]^T  (both row-major in shared memory, already TF32), 8 warps; a warp owns the two
+// output tiles (tm, tn0) and (tm, tn0 + 1), which share the A fragment
 template <int D>
 __device__ __forceinline__ void scores_64x64(const float* A, const float* B, float* C) {
   constexpr int LDX = D + 4, LDS = kCT + 4;
   const int warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    const int t = warp * 2 + i, tm = t >> 2, tn = t & 3;
-    FragC acc;
-    wmma::fill_fragment(acc, 0.f);
+  const int tm = warp >> 1, tn0 = (warp & 1) * 2;
+  FragC acc0, acc1;
+  wmma::fill_fragment(acc0, 0.f);
+  wmma::fill_fragment(acc1, 0.f);
 #pragma unroll 4
-    for (int k = 0; k < D; k += 8) {
-      FragA a;
-      FragBT b;
-      wmma::load_matrix_sync(a, A + tm * 16 * LDX + k, LDX);
-      wmma::load_matrix_sync(b, B + tn * 16 * LDX + k, LDX);
-      to_tf32(a);
-      to_tf32(b);
-      wmma::mma_sync(acc, a, b, acc);
-    }
-    wmma::store_matrix_sync(C + tm * 16 * LDS + tn * 16, acc, LDS, wmma::mem_row_major);
+  for (int k = 0; k < D; k += 8) {
+    FragA a;
+    FragBT b0, b1;
+    wmma::load_matrix_sync(a, A + tm * 16 * LDX + k, LDX);
+    wmma::load_matrix_sync(b0, B + tn0 * 16 * LDX + k, LDX);
+    wmma::load_matrix_sync(b1, B + (tn0 + 1) * 16 * LDX + k, LDX);
+    wmma::mma_sync(acc0, a, b0, acc0);
+    wmma::mma_sync(acc1, a, b1, acc1);
   }
+  wmma::store_matrix_sync(C + tm * 16 * LDS + tn0 * 16, acc0, LDS, wmma::mem_row_major);
+  wmma::store_matrix_sync(C + tm * 16 * LDS + (tn0 + 1) * 16, acc1, LDS, wmma::mem_row_major);
 }
 
-// acc tiles (this warp owns output tiles warp*4 .. warp*4+3 of a [64 x D] result, tile = (tm, tn) with tn fastest)
-//   TRANS_W = false: out += W[64 x 64] * X[64 x D];   TRANS_W = true: out += W^T * X
+// acc tiles: this warp owns the D/32 consecutive output tiles (tm, tn0 .. tn0 + D/32 - 1) of a [64 x D] result, which
+// share the W fragment.   TRANS_W = false: out += W[64 x 64] * X[64 x D];   TRANS_W = true: out += W^T * X
 template <int D, bool TRANS_W>
 __device__ __forceinline__ void accumulate_64xD(FragC (&acc)[D / 32], const float* W, const float* X) {
-  constexpr int LDX = D + 4, LDS = kCT + 4, TN = D / 16;
+  constexpr int LDX = D + 4, LDS = kCT + 4, TN = D / 16, PER = D / 32;
   const int warp = threadIdx.x >> 5;
+  const int tm = (warp * PER) / TN, tn0 = (warp * PER) % TN;
 #pragma unroll
-  for (int i = 0; i < D / 32; ++i) {
-    const int t = warp * (D / 32) + i, tm = t / TN, tn = t % TN;
+  for (int k = 0; k < kCT; k += 8) {
+    FragA a;
+    FragAT at;
+    if constexpr (TRANS_W) wmma::load_matrix_sync(at, W + k * LDS + tm * 16, LDS);
+    else wmma::load_matrix_sync(a, W + tm * 16 * LDS + k, LDS);
 #pragma unroll
-    for (int k = 0; k < kCT; k += 8) {
+    for (int i = 0; i < PER; ++i) {
       FragB b;
-      wmma::load_matrix_sync(b, X + k * LDX + tn * 16, LDX);
-      to_tf32(b);
-      if constexpr (TRANS_W) {
-        FragAT a;
-        wmma::load_matrix_sync(a, W + k * LDS + tm * 16, LDS);
-        to_tf32(a);
-        wmma::mma_sync(acc[i], a, b, acc[i]);
-      } else {
-        FragA a;
-        wmma::load_matrix_sync(a, W + tm * 16 * LDS + k, LDS);
-        to_tf32(a);
-        wmma::mma_sync(acc[i], a, b, acc[i]);
-      }
+      wmma::load_matrix_sync(b, X + k * LDX + (tn0 + i) * 16, LDX);
+      if constexpr (TRANS_W) wmma::mma_sync(acc[i], at, b, acc[i]);
+      else wmma::mma_sync(acc[i], a, b, acc[i]);
     }
   }
 }
@@ -93,7 +86,7 @@ __device__ __forceinline__ void load_tile(float* dst, const float* src, int row0
     const int r = e / CH, c = e % CH;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (row0 + r < limit) v = __ldg(reinterpret_cast<const float4*>(src + (size_t)(row0 + r) * D + c * 4));
-    *reinterpret_cast<float4*>(dst + r * LDX + c * 4) = v;
+    *reinterpret_cast<float4*>(dst + r * LDX + c * 4) = make_float4(tf32(v.x), tf32(v.y), tf32(v.z), tf32(v.w));
   }
 }
 
@@ -142,7 +135,7 @@ __global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restr
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
         const float p = __expf(x[c] - m_new);
-        S[r * C::LDS + qd * 16 + c] = p;
+        S[r * C::LDS + qd * 16 + c] = tf32(p);
         ps += p;
       }
       ps += __shfl_xor_sync(0xffffffffu, ps, 1);
@@ -154,26 +147,18 @@ __global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restr
     }
     __syncthreads();
     {
-      // O += P V with the accumulator round-tripping through shared memory (rows were just rescaled there)
-      constexpr int TN = D / 16;
+      // O += P V with the accumulators round-tripping through shared memory (rows were just rescaled there)
+      constexpr int TN = D / 16, PER = D / 32;
       const int warp = threadIdx.x >> 5;
+      const int tm = (warp * PER) / TN, tn0 = (warp * PER) % TN;
+      FragC acc[PER];
 #pragma unroll
-      for (int i = 0; i < D / 32; ++i) {
-        const int t = warp * (D / 32) + i, tm = t / TN, tn = t % TN;
-        FragC acc;
-        wmma::load_matrix_sync(acc, Os + tm * 16 * C::LDX + tn * 16, C::LDX, wmma::mem_row_major);
+      for (int i = 0; i < PER; ++i)
+        wmma::load_matrix_sync(acc[i], Os + tm * 16 * C::LDX + (tn0 + i) * 16, C::LDX, wmma::mem_row_major);
+      accumulate_64xD<D, false>(acc, S, Vs);
 #pragma unroll
-        for (int k = 0; k < kCT; k += 8) {
-          FragA a;
-          FragB bfr;
-          wmma::load_matrix_sync(a, S + tm * 16 * C::LDS + k, C::LDS);
-          wmma::load_matrix_sync(bfr, Vs + k * C::LDX + tn * 16, C::LDX);
-          to_tf32(a);
-          to_tf32(bfr);
-          wmma::mma_sync(acc, a, bfr, acc);
-        }
-        wmma::store_matrix_sync(Os + tm * 16 * C::LDX + tn * 16, acc, C::LDX, wmma::mem_row_major);
-      }
+      for (int i = 0; i < PER; ++i)
+        wmma::store_matrix_sync(Os + tm * 16 * C::LDX + (tn0 + i) * 16, acc[i], C::LDX, wmma::mem_row_major);
     }
   }
   __syncthreads();
@@ -269,8 +254,8 @@ __global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restr
       const bool ok = ROWS ? (j0 + ki < g.N) : (s0 + ki < g.N);     // the key must exist (missing queries carry lse = +inf)
       const float p = ok ? __expf(S[qi * C::LDS + ki] * g.scale - q_lse[qi]) : 0.f;
       const float ds = p * (dP[qi * C::LDS + ki] - q_delta[qi]) * g.scale;
-      S[qi * C::LDS + ki] = p;
-      dP[qi * C::LDS + ki] = ds;
+      S[qi * C::LDS + ki] = tf32(p);
+      dP[qi * C::LDS + ki] = tf32(ds);
     }
     __syncthreads();
     if (ROWS) {
@@ -283,13 +268,13 @@ __global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restr
   // accumulators -> shared memory (operand tiles are idle) -> global
   __syncthreads();
   {
-    constexpr int TN = D / 16;
+    constexpr int TN = D / 16, PER = D / 32;
     const int warp = threadIdx.x >> 5;
+    const int tm = (warp * PER) / TN, tn0 = (warp * PER) % TN;
 #pragma unroll
-    for (int i = 0; i < D / 32; ++i) {
-      const int t = warp * (D / 32) + i, tm = t / TN, tn = t % TN;
-      wmma::store_matrix_sync(Y0 + tm * 16 * C::LDX + tn * 16, acc0[i], C::LDX, wmma::mem_row_major);
-      if (!ROWS) wmma::store_matrix_sync(Y1 + tm * 16 * C::LDX + tn * 16, acc1[i], C::LDX, wmma::mem_row_major);
+    for (int i = 0; i < PER; ++i) {
+      wmma::store_matrix_sync(Y0 + tm * 16 * C::LDX + (tn0 + i) * 16, acc0[i], C::LDX, wmma::mem_row_major);
+      if (!ROWS) wmma::store_matrix_sync(Y1 + tm * 16 * C::LDX + (tn0 + i) * 16, acc1[i], C::LDX, wmma::mem_row_major);
     }
   }
   __syncthreads();
