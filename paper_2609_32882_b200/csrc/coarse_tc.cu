@@ -13,6 +13,7 @@ namespace vsa2 {
 using namespace nvcuda;
 
 constexpr int kCT = 64;    // rows per tile (queries and keys)
+constexpr int kCoarseThreads = 512;   // 16 warps: one score tile, D/64 output tiles each
 
 template <int D>
 struct CoarseTc {
@@ -32,35 +33,37 @@ typedef wmma::fragment<wmma::accumulator, 16, 16, 8, float> FragC;
 
 __device__ __forceinline__ float tf32(float x) { return wmma::__float_to_tf32(x); }
 
-// C[64 x 64] = A[64 x D] * B[64 x D]^T  (both row-major in shared memory, already TF32), 8 warps; a warp owns the two
-// output tiles (tm, tn0) and (tm, tn0 + 1), which share the A fragment
+// C[64 x 64] = A[64 x D] * B[64 x D]^T  (both row-major in shared memory, already TF32), 16 warps, one output tile
+// each; the contraction is split into two halves with their own accumulators so that two dependent chains interleave
 template <int D>
 __device__ __forceinline__ void scores_64x64(const float* A, const float* B, float* C) {
   constexpr int LDX = D + 4, LDS = kCT + 4;
   const int warp = threadIdx.x >> 5;
-  const int tm = warp >> 1, tn0 = (warp & 1) * 2;
+  const int tm = warp >> 2, tn = warp & 3;
   FragC acc0, acc1;
   wmma::fill_fragment(acc0, 0.f);
   wmma::fill_fragment(acc1, 0.f);
 #pragma unroll 4
-  for (int k = 0; k < D; k += 8) {
-    FragA a;
+  for (int k = 0; k < D / 2; k += 8) {
+    FragA a0, a1;
     FragBT b0, b1;
-    wmma::load_matrix_sync(a, A + tm * 16 * LDX + k, LDX);
-    wmma::load_matrix_sync(b0, B + tn0 * 16 * LDX + k, LDX);
-    wmma::load_matrix_sync(b1, B + (tn0 + 1) * 16 * LDX + k, LDX);
-    wmma::mma_sync(acc0, a, b0, acc0);
-    wmma::mma_sync(acc1, a, b1, acc1);
+    wmma::load_matrix_sync(a0, A + tm * 16 * LDX + k, LDX);
+    wmma::load_matrix_sync(b0, B + tn * 16 * LDX + k, LDX);
+    wmma::load_matrix_sync(a1, A + tm * 16 * LDX + D / 2 + k, LDX);
+    wmma::load_matrix_sync(b1, B + tn * 16 * LDX + D / 2 + k, LDX);
+    wmma::mma_sync(acc0, a0, b0, acc0);
+    wmma::mma_sync(acc1, a1, b1, acc1);
   }
-  wmma::store_matrix_sync(C + tm * 16 * LDS + tn0 * 16, acc0, LDS, wmma::mem_row_major);
-  wmma::store_matrix_sync(C + tm * 16 * LDS + (tn0 + 1) * 16, acc1, LDS, wmma::mem_row_major);
+#pragma unroll
+  for (int i = 0; i < acc0.num_elements; ++i) acc0.x[i] += acc1.x[i];
+  wmma::store_matrix_sync(C + tm * 16 * LDS + tn * 16, acc0, LDS, wmma::mem_row_major);
 }
 
-// acc tiles: this warp owns the D/32 consecutive output tiles (tm, tn0 .. tn0 + D/32 - 1) of a [64 x D] result, which
+// acc tiles: this warp owns the D/64 consecutive output tiles (tm, tn0 .. tn0 + D/64 - 1) of a [64 x D] result, which
 // share the W fragment.   TRANS_W = false: out += W[64 x 64] * X[64 x D];   TRANS_W = true: out += W^T * X
 template <int D, bool TRANS_W>
-__device__ __forceinline__ void accumulate_64xD(FragC (&acc)[D / 32], const float* W, const float* X) {
-  constexpr int LDX = D + 4, LDS = kCT + 4, TN = D / 16, PER = D / 32;
+__device__ __forceinline__ void accumulate_64xD(FragC (&acc)[D / 64], const float* W, const float* X) {
+  constexpr int LDX = D + 4, LDS = kCT + 4, TN = D / 16, PER = D / 64;
   const int warp = threadIdx.x >> 5;
   const int tm = (warp * PER) / TN, tn0 = (warp * PER) % TN;
 #pragma unroll
@@ -91,9 +94,9 @@ __device__ __forceinline__ void load_tile(float* dst, const float* src, int row0
 }
 
 // ---------------------------------------------------------------------------------------------- forward
-// grid (ceil(N/64), Hq, batch), 256 threads
+// grid (ceil(N/64), Hq, batch), 512 threads
 template <int D>
-__global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restrict__ qc, const float* __restrict__ kc,
+__global__ void __launch_bounds__(kCoarseThreads) coarse_fwd_tc_kernel(const float* __restrict__ qc, const float* __restrict__ kc,
                                                             const float* __restrict__ vc, Geo g,
                                                             float* __restrict__ oc_hat, float* __restrict__ lse_c) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -111,7 +114,7 @@ __global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restr
   load_tile<D>(Qs, qc + qoff, i0, g.N);
   for (int e = threadIdx.x; e < kCT * C::LDX; e += blockDim.x) Os[e] = 0.f;
   if (threadIdx.x < kCT) { row_m[threadIdx.x] = -INFINITY; row_l[threadIdx.x] = 0.f; }
-  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  const int r = threadIdx.x >> 3, qd = threadIdx.x & 7;   // 8 threads per row, 8 columns / D/8 channels each
   for (int j0 = 0; j0 < g.N; j0 += kCT) {
     __syncthreads();
     load_tile<D>(Ks, kc + koff, j0, g.N);
@@ -120,35 +123,37 @@ __global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restr
     scores_64x64<D>(Qs, Ks, S);
     __syncthreads();
     {
-      float x[16];
+      float x[8];
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const int col = qd * 16 + c;
+      for (int c = 0; c < 8; ++c) {
+        const int col = qd * 8 + c;
         x[c] = (j0 + col < g.N) ? S[r * C::LDS + col] * g.scale : -INFINITY;
         mx = fmaxf(mx, x[c]);
       }
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
       const float m_old = row_m[r], m_new = fmaxf(m_old, mx);
       float ps = 0.f;
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
+      for (int c = 0; c < 8; ++c) {
         const float p = __expf(x[c] - m_new);
-        S[r * C::LDS + qd * 16 + c] = tf32(p);
+        S[r * C::LDS + qd * 8 + c] = tf32(p);
         ps += p;
       }
       ps += __shfl_xor_sync(0xffffffffu, ps, 1);
       ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 4);
       const float alpha = __expf(m_old - m_new);
-      for (int c = 0; c < D / 4; ++c) Os[r * C::LDX + qd * (D / 4) + c] *= alpha;
+      for (int c = 0; c < D / 8; ++c) Os[r * C::LDX + qd * (D / 8) + c] *= alpha;
       __syncwarp();
       if (qd == 0) { row_m[r] = m_new; row_l[r] = row_l[r] * alpha + ps; }
     }
     __syncthreads();
     {
       // O += P V with the accumulators round-tripping through shared memory (rows were just rescaled there)
-      constexpr int TN = D / 16, PER = D / 32;
+      constexpr int TN = D / 16, PER = D / 64;
       const int warp = threadIdx.x >> 5;
       const int tm = (warp * PER) / TN, tn0 = (warp * PER) % TN;
       FragC acc[PER];
@@ -165,8 +170,8 @@ __global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restr
   const int i = i0 + r;
   if (i < g.N) {
     const float inv = 1.f / row_l[r];
-    for (int c = 0; c < D / 4; ++c) {
-      const int d = qd * (D / 4) + c;
+    for (int c = 0; c < D / 8; ++c) {
+      const int d = qd * (D / 8) + c;
       oc_hat[qoff + (size_t)i * D + d] = Os[r * C::LDX + d] * inv;
     }
     if (qd == 0) lse_c[(size_t)(b * g.Hq + hq) * g.N + i] = row_m[r] + __logf(row_l[r]);
@@ -178,7 +183,7 @@ __global__ void __launch_bounds__(256) coarse_fwd_tc_kernel(const float* __restr
 // ROWS = false: 64 key cubes stationary; streams query tiles; writes dK_c, dV_c (per query head).
 // dS = P * (dP - delta_c) * scale, P = exp(S*scale - lse_c), dP = dO_c_hat V_c^T, delta_c = rowsum(dO_c_hat * O_c_hat).
 template <int D, bool ROWS>
-__global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restrict__ qc, const float* __restrict__ kc,
+__global__ void __launch_bounds__(kCoarseThreads) coarse_bwd_tc_kernel(const float* __restrict__ qc, const float* __restrict__ kc,
                                                             const float* __restrict__ vc, const float* __restrict__ oc_hat,
                                                             const float* __restrict__ lse_c, const float* __restrict__ d_oc,
                                                             Geo g, float* __restrict__ delta_c, float* __restrict__ out0,
@@ -197,7 +202,7 @@ __global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restr
   const int s0 = blockIdx.x * kCT;
   const size_t qoff = (size_t)(b * g.Hq + hq) * g.N * D, koff = (size_t)(b * g.Hkv + hk) * g.N * D;
   const size_t roff = (size_t)(b * g.Hq + hq) * g.N;
-  const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
+  const int r = threadIdx.x >> 3, qd = threadIdx.x & 7;
   if (ROWS) {
     load_tile<D>(X0, qc + qoff, s0, g.N);
     load_tile<D>(X1, d_oc + qoff, s0, g.N);
@@ -206,12 +211,13 @@ __global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restr
     float acc = 0.f;
     const int i = s0 + r;
     if (i < g.N)
-      for (int c = 0; c < D / 4; ++c) {
-        const int d = qd * (D / 4) + c;
+      for (int c = 0; c < D / 8; ++c) {
+        const int d = qd * (D / 8) + c;
         acc = fmaf(X1[r * C::LDX + d], __ldg(oc_hat + qoff + (size_t)i * D + d), acc);
       }
     acc += __shfl_xor_sync(0xffffffffu, acc, 1);
     acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
     if (qd == 0) {
       q_delta[r] = acc;
       q_lse[r] = i < g.N ? lse_c[roff + i] : INFINITY;
@@ -221,9 +227,9 @@ __global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restr
     load_tile<D>(X0, kc + koff, s0, g.N);
     load_tile<D>(X1, vc + koff, s0, g.N);
   }
-  FragC acc0[D / 32], acc1[D / 32];
+  FragC acc0[D / 64], acc1[D / 64];
 #pragma unroll
-  for (int i = 0; i < D / 32; ++i) { wmma::fill_fragment(acc0[i], 0.f); wmma::fill_fragment(acc1[i], 0.f); }
+  for (int i = 0; i < D / 64; ++i) { wmma::fill_fragment(acc0[i], 0.f); wmma::fill_fragment(acc1[i], 0.f); }
 
   for (int j0 = 0; j0 < g.N; j0 += kCT) {
     __syncthreads();
@@ -268,7 +274,7 @@ __global__ void __launch_bounds__(256) coarse_bwd_tc_kernel(const float* __restr
   // accumulators -> shared memory (operand tiles are idle) -> global
   __syncthreads();
   {
-    constexpr int TN = D / 16, PER = D / 32;
+    constexpr int TN = D / 16, PER = D / 64;
     const int warp = threadIdx.x >> 5;
     const int tm = (warp * PER) / TN, tn0 = (warp * PER) % TN;
 #pragma unroll
@@ -295,11 +301,11 @@ cudaError_t launch_coarse_fwd_tc(const Geo& g, const float* qc, const float* kc,
   if (g.D == 128) {
     const size_t smb = CoarseTc<128>::fwd_bytes;
     if ((e = cudaFuncSetAttribute(coarse_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    coarse_fwd_tc_kernel<128><<<grid, 256, smb, st>>>(qc, kc, vc, g, oc_hat, lse_c);
+    coarse_fwd_tc_kernel<128><<<grid, kCoarseThreads, smb, st>>>(qc, kc, vc, g, oc_hat, lse_c);
   } else {
     const size_t smb = CoarseTc<64>::fwd_bytes;
     if ((e = cudaFuncSetAttribute(coarse_fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    coarse_fwd_tc_kernel<64><<<grid, 256, smb, st>>>(qc, kc, vc, g, oc_hat, lse_c);
+    coarse_fwd_tc_kernel<64><<<grid, kCoarseThreads, smb, st>>>(qc, kc, vc, g, oc_hat, lse_c);
   }
   return cudaGetLastError();
 }
@@ -313,8 +319,8 @@ static cudaError_t coarse_bwd_tc_t(const Geo& g, const float* qc, const float* k
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(coarse_bwd_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
   if ((e = cudaFuncSetAttribute(coarse_bwd_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-  coarse_bwd_tc_kernel<D, true><<<grid, 256, smb, st>>>(qc, kc, vc, oc_hat, lse_c, d_oc, g, delta_c, dqc, nullptr);
-  coarse_bwd_tc_kernel<D, false><<<grid, 256, smb, st>>>(qc, kc, vc, oc_hat, lse_c, d_oc, g, delta_c, dkc, dvc);
+  coarse_bwd_tc_kernel<D, true><<<grid, kCoarseThreads, smb, st>>>(qc, kc, vc, oc_hat, lse_c, d_oc, g, delta_c, dqc, nullptr);
+  coarse_bwd_tc_kernel<D, false><<<grid, kCoarseThreads, smb, st>>>(qc, kc, vc, oc_hat, lse_c, d_oc, g, delta_c, dkc, dvc);
   return cudaGetLastError();
 }
 
