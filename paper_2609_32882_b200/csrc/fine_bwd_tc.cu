@@ -97,12 +97,12 @@ __device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
 // One warp streams pairs of cube tiles into a ring of NS slots: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one
 // box each (half h = lane / 2 of block lane & 1).  `coord_*`: cube coordinates of this lane's block, `bh`: its head.
 // `LANE0_PRE`: statement lane 0 runs once the slot is free, before the loads are armed (may use slot_).
-#define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH, LANE0_PRE)                          \
+#define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH, LANE0_PRE, WAITFN)                  \
   do {                                                                                                            \
     const uint32_t slot_ = (SEQ) % (NS), par_ = ((SEQ) / (NS)) & 1;                                               \
     int ok_ = 1;                                                                                                  \
     if (lane == 0) {                                                                                              \
-      ok_ = tc::mbar_wait(&(EMPTY)[slot_], par_ ^ 1, &misc->abort_flag);                                          \
+      ok_ = tc::WAITFN(&(EMPTY)[slot_], par_ ^ 1, &misc->abort_flag);                                             \
       if (ok_) {                                                                                                  \
         LANE0_PRE;                                                                                                \
         tc::mbar_expect_tx(&(FULL)[slot_], C::SLOT);                                                              \
@@ -204,9 +204,9 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         if (which == 0) {
           const unsigned ef0 = cube_edge_flags_at(g, jt, jh, jw), ef1 = __shfl_sync(0xffffffffu, ef0, 1);
           VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, jt, jh, jw, bhk,
-                         { misc->edge[slot_][0] = (unsigned char)ef0; misc->edge[slot_][1] = (unsigned char)ef1; });
+                         { misc->edge[slot_][0] = (unsigned char)ef0; misc->edge[slot_][1] = (unsigned char)ef1; }, mbar_wait);
         } else {
-          VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, jt, jh, jw, bhk, {});
+          VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, jt, jh, jw, bhk, {}, mbar_wait);
         }
       }
     }
@@ -513,7 +513,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         cube_coords(g, j, jt, jh, jw);
         int ok = 1;
         if (lane == 0) {
-          ok = tc::mbar_wait(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
+          ok = tc::mbar_wait_parked(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
           if (ok) tc::mbar_expect_tx(&misc->st_full, 2 * C::TILE);
         }
         if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
@@ -532,8 +532,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         cube_coords(g, i_l, it_, ih_, iw_);
         const int bhq_t = bhq_l;
         if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
-        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, it_, ih_, iw_, bhq_t, {});
-        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t, {});
+        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
+        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
       }
     }
   } else if (warp == 2 || warp == 3) {
@@ -548,19 +548,19 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
-        VSA2_WAIT(&misc->st_full, n_items & 1);
+        VSA2_WAIT_PARKED(&misc->st_full, n_items & 1);
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t sb = tg & 1, pb = (tg >> 1) & 1;
           if (is_s) {
             const uint32_t sa = tg % kRingA, pa = (tg / kRingA) & 1;
-            VSA2_WAIT(&misc->a_full[sa], pa);
-            VSA2_WAIT(&misc->s_free[sb], pb ^ 1);
+            VSA2_WAIT_PARKED(&misc->a_full[sa], pa);
+            VSA2_WAIT_PARKED(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
             mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
             tc::mma_commit(&misc->s_full[sb]);
           } else {
-            VSA2_WAIT(&misc->b_full[sb], pb);
-            VSA2_WAIT(&misc->dp_free[sb], pb ^ 1);
+            VSA2_WAIT_PARKED(&misc->b_full[sb], pb);
+            VSA2_WAIT_PARKED(&misc->dp_free[sb], pb ^ 1);
             tc::tc_fence_after();
             mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
             tc::mma_commit(&misc->dp_full[sb]);
@@ -583,20 +583,20 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
-        VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
+        VSA2_WAIT_PARKED(&misc->o_empty, (n_items & 1) ^ 1);
         for (int t = 0; t < nt; ++t, ++tg) {
           if (is_v) {
             // P depends on S only, so it can be ready before the dO pair of the tile has landed: wait for that too
             const uint32_t sv = tg & 1;
-            VSA2_WAIT(&misc->b_full[sv], (tg >> 1) & 1);
-            VSA2_WAIT(&misc->p_ready, tg & 1);
+            VSA2_WAIT_PARKED(&misc->b_full[sv], (tg >> 1) & 1);
+            VSA2_WAIT_PARKED(&misc->p_ready, tg & 1);
             tc::tc_fence_after();
             mma_pairT_mnmajor<D>(tmem_base + 320, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
             tc::mma_commit(&misc->b_empty[sv]);
             tc::mma_commit(&misc->p_free);
           } else {
             const uint32_t sa = tg % kRingA;
-            VSA2_WAIT(&misc->ds_ready[0], tg & 1);
+            VSA2_WAIT_PARKED(&misc->ds_ready[0], tg & 1);
             tc::tc_fence_after();
             mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, b_addr, t > 0);
             tc::mma_commit(&misc->a_empty[sa]);
@@ -630,7 +630,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const size_t idx = l >= 0 ? (size_t)bhq_n * g.L + l : 0;
         const float lse_raw = a.lse[idx], dlt_raw = a.delta[idx];
         if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
-        VSA2_WAIT(&misc->stat_free, (tg & 1) ^ 1);
+        VSA2_WAIT_PARKED(&misc->stat_free, (tg & 1) ^ 1);
         rowstat[r] = make_float2(l >= 0 ? lse_raw * 1.4426950408889634f : INFINITY, l >= 0 ? dlt_raw : 0.f);
         tc::mbar_arrive(&misc->stat_full);
       }

@@ -43,6 +43,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint (ns): the hardware parks the thread until the phase completes or the time is up,
+// so a waiting role does not spend issue slots that the working warps of its scheduler need.
+constexpr uint32_t kSuspendHintNs = 100000u;
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait: gives up after about `kWaitLimitNs` of wall time, or as soon as another thread of the CTA
 // has raised *abort_flag.  Returns false on failure, after raising the flag itself.
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -60,6 +74,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) break;
     }
+  }
+  *abort_flag = 1;
+  return false;
+}
+// The same for roles with slack: parked between polls (a slightly later wake-up, no issue slots spent spinning).
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (;;) {
+    if (mbar_try_wait_parked(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   return false;

@@ -122,5 +122,9 @@ __device__ __forceinline__ int warp_reduce_col(int lane) {
   do {                                                                 \
     if (!tc::mbar_wait((bar), (parity), &misc->abort_flag)) goto done; \
   } while (0)
+#define VSA2_WAIT_PARKED(bar, parity)                                         \
+  do {                                                                        \
+    if (!tc::mbar_wait_parked((bar), (parity), &misc->abort_flag)) goto done; \
+  } while (0)
 
 }  // namespace vsa2
