@@ -3,15 +3,16 @@
 // Q_r K_r^T * scale, pass 2 recomputes the scores, applies the softmax and pools G x G sub-blocks on chip.
 //
 // A CTA owns 128 consecutive pooled queries (128/G query cubes) of one head and streams the head's pooled
-// keys in tiles of 128 through a TMA ring; S [128 q, 128 keys] lands in tensor memory (two buffers) and
-// each of the 128 compute threads owns one query row, so the softmax statistics are thread-local.  The G
+// keys in tiles of 128 through a TMA ring; S [128 q, 128 keys] lands in tensor memory (two buffers).  Two
+// compute threads own each query row, 64 key columns of every tile each (a single warp per scheduler keeps
+// the exponential unit only half busy); pass 1 merges their running (max, sum) pairs once per item.  The G
 // rows of a query cube sit in G adjacent lanes: their pooled sums are combined with warp shuffles.
 // Both passes are bound by the exponential unit (one ex2 per score), not by the tensor pipe.
 #include "tc_attn.cuh"
 
 namespace vsa2 {
 
-constexpr int kRtThreads = 192;
+constexpr int kRtThreads = 320;    // TMA warp, MMA warp, 8 compute warps
 constexpr int kRtSlots = 4;
 constexpr int kRtTile = 128;
 
@@ -22,7 +23,7 @@ struct RouterTc {
   static constexpr uint32_t TILE = DH * HALF;
   static constexpr uint32_t OFF_Q = kRtSlots * TILE;
   static constexpr uint32_t OFF_MISC = OFF_Q + TILE;
-  static constexpr uint32_t MISC_BYTES = 1024;
+  static constexpr uint32_t MISC_BYTES = 2048;
   static size_t smem_bytes(int valid_words) { return OFF_MISC + MISC_BYTES + (size_t)valid_words * 4 + 1024; }
 };
 
@@ -30,8 +31,10 @@ struct RouterMisc {
   uint64_t q_full, q_empty;
   uint64_t k_full[kRtSlots], k_empty[kRtSlots];
   uint64_t s_full[2], s_free[2];
+  uint64_t part_ready, part_free;   // pass 1: hand-over of part_stats
   uint32_t tmem_base;
   int abort_flag;
+  float2 part_stats[128];   // pass 1: (running max, running sum) of the threads that own key columns 64..127
 };
 
 // tensor map over pooled operands [BH, N*G, D] bf16: box = 64 channels x 128 rows x 1
@@ -92,8 +95,10 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     for (int s = 0; s < 2; ++s) {
       tc::mbar_init(&misc->s_full[s], 1);
-      tc::mbar_init(&misc->s_free[s], 128);
+      tc::mbar_init(&misc->s_free[s], 256);
     }
+    tc::mbar_init(&misc->part_ready, 128);
+    tc::mbar_init(&misc->part_free, 128);
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -152,11 +157,12 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
   } else {
-    const int quad = warp & 3;
+    const int quad = warp & 3;                   // tensor-memory lane quadrant of this warp
+    const int part = (warp - 2) >> 2;            // 0: key columns 0..63 of every tile, 1: columns 64..127
     const int row = (quad << 5) | lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t seq = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+    uint32_t seq = 0, n_items = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_items) {
       const int rt = item % row_tiles, bhq = item / row_tiles;
       const int r = rt * kRtTile + row;                          // pooled query index inside the head
       const bool q_valid = (valid_bits[r >> 5] >> (r & 31)) & 1u;
@@ -174,7 +180,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         VSA2_WAIT(&misc->s_full[buf], (seq >> 1) & 1);
         tc::tc_fence_after();
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int ch = part * 2; ch < part * 2 + 2; ++ch) {
           uint32_t s[32];
           tc::tmem_ld32(lane_addr + buf * 128 + ch * 32, s);
           tc::tmem_ld_wait();
@@ -220,7 +226,21 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         tc::tc_fence_before();
         tc::mbar_arrive(&misc->s_free[buf]);
       }
-      if (PASS == 1 && r < NG) lse2[(size_t)bhq * NG + r] = (l_run > 0.f) ? m_run + __log2f(l_run) : 0.f;
+      if (PASS == 1) {
+        // merge the two column halves of the row
+        if (part == 1) {
+          VSA2_WAIT(&misc->part_free, (n_items & 1) ^ 1);
+          misc->part_stats[row] = make_float2(m_run, l_run);
+          tc::mbar_arrive(&misc->part_ready);
+        } else {
+          VSA2_WAIT(&misc->part_ready, n_items & 1);
+          const float2 o = misc->part_stats[row];
+          tc::mbar_arrive(&misc->part_free);
+          const float m_new = fmaxf(m_run, o.x);
+          if (m_new > -INFINITY) l_run = l_run * ex2_approx(m_run - m_new) + o.y * ex2_approx(o.x - m_new);
+          if (r < NG) lse2[(size_t)bhq * NG + r] = (l_run > 0.f) ? m_new + __log2f(l_run) : 0.f;
+        }
+      }
     }
   }
 
