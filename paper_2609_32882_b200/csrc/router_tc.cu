@@ -3,8 +3,8 @@
 // Q_r K_r^T * scale, pass 2 recomputes the scores, applies the softmax and pools G x G sub-blocks on chip.
 //
 // A CTA owns 128 consecutive pooled queries (128/G query cubes) of one head and streams the head's pooled
-// keys in tiles of 128 through a TMA ring; S [128 q, 128 keys] lands in tensor memory (two buffers).  Two
-// compute threads own each query row, 64 key columns of every tile each (a single warp per scheduler keeps
+// keys in tiles of 128 through a TMA ring; S [128 q, 128 keys] lands in tensor memory (two buffers).
+// Four compute threads own each query row, 32 key columns of every tile each (a single warp per scheduler keeps
 // the exponential unit only half busy); pass 1 merges their running (max, sum) pairs once per item.  The G
 // rows of a query cube sit in G adjacent lanes: their pooled sums are combined with warp shuffles.
 // Both passes are bound by the exponential unit (one ex2 per score), not by the tensor pipe.
@@ -12,7 +12,8 @@
 
 namespace vsa2 {
 
-constexpr int kRtThreads = 320;    // TMA warp, MMA warp, 8 compute warps
+constexpr int kRtParts = 4;        // compute threads per pooled query row (each owns 128 / kRtParts key columns of a tile)
+constexpr int kRtThreads = 64 + 128 * kRtParts;    // TMA warp, MMA warp, 4 * kRtParts compute warps
 constexpr int kRtSlots = 4;
 constexpr int kRtTile = 128;
 
@@ -23,7 +24,7 @@ struct RouterTc {
   static constexpr uint32_t TILE = DH * HALF;
   static constexpr uint32_t OFF_Q = kRtSlots * TILE;
   static constexpr uint32_t OFF_MISC = OFF_Q + TILE;
-  static constexpr uint32_t MISC_BYTES = 2048;
+  static constexpr uint32_t MISC_BYTES = 4096;
   static size_t smem_bytes(int valid_words) { return OFF_MISC + MISC_BYTES + (size_t)valid_words * 4 + 1024; }
 };
 
@@ -34,7 +35,7 @@ struct RouterMisc {
   uint64_t part_ready, part_free;   // pass 1: hand-over of part_stats
   uint32_t tmem_base;
   int abort_flag;
-  float2 part_stats[128];   // pass 1: (running max, running sum) of the threads that own key columns 64..127
+  float2 part_stats[kRtParts - 1][128];   // pass 1: (running max, running sum) of the threads of parts 1 .. kRtParts-1
 };
 
 // tensor map over pooled operands [BH, N*G, D] bf16: box = 64 channels x 128 rows x 1
@@ -95,9 +96,9 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     for (int s = 0; s < 2; ++s) {
       tc::mbar_init(&misc->s_full[s], 1);
-      tc::mbar_init(&misc->s_free[s], 256);
+      tc::mbar_init(&misc->s_free[s], 128 * kRtParts);
     }
-    tc::mbar_init(&misc->part_ready, 128);
+    tc::mbar_init(&misc->part_ready, 128 * (kRtParts - 1));
     tc::mbar_init(&misc->part_free, 128);
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
@@ -158,7 +159,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
   } else {
     const int quad = warp & 3;                   // tensor-memory lane quadrant of this warp
-    const int part = (warp - 2) >> 2;            // 0: key columns 0..63 of every tile, 1: columns 64..127
+    const int part = (warp - 2) >> 2;            // which 128 / kRtParts key columns of every tile
     const int row = (quad << 5) | lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint32_t seq = 0, n_items = 0;
@@ -180,7 +181,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         VSA2_WAIT(&misc->s_full[buf], (seq >> 1) & 1);
         tc::tc_fence_after();
 #pragma unroll
-        for (int ch = part * 2; ch < part * 2 + 2; ++ch) {
+        for (int ch = part * (4 / kRtParts); ch < (part + 1) * (4 / kRtParts); ++ch) {
           uint32_t s[32];
           tc::tmem_ld32(lane_addr + buf * 128 + ch * 32, s);
           tc::tmem_ld_wait();
@@ -228,16 +229,25 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       if (PASS == 1) {
         // merge the two column halves of the row
-        if (part == 1) {
+        if (part > 0) {
           VSA2_WAIT(&misc->part_free, (n_items & 1) ^ 1);
-          misc->part_stats[row] = make_float2(m_run, l_run);
+          misc->part_stats[part - 1][row] = make_float2(m_run, l_run);
           tc::mbar_arrive(&misc->part_ready);
         } else {
           VSA2_WAIT(&misc->part_ready, n_items & 1);
-          const float2 o = misc->part_stats[row];
+          float2 o[kRtParts - 1];
+          float m_new = m_run;
+#pragma unroll
+          for (int pp = 0; pp < kRtParts - 1; ++pp) {
+            o[pp] = misc->part_stats[pp][row];
+            m_new = fmaxf(m_new, o[pp].x);
+          }
           tc::mbar_arrive(&misc->part_free);
-          const float m_new = fmaxf(m_run, o.x);
-          if (m_new > -INFINITY) l_run = l_run * ex2_approx(m_run - m_new) + o.y * ex2_approx(o.x - m_new);
+          if (m_new > -INFINITY) {
+            l_run *= ex2_approx(m_run - m_new);
+#pragma unroll
+            for (int pp = 0; pp < kRtParts - 1; ++pp) l_run += o[pp].y * ex2_approx(o[pp].x - m_new);
+          }
           if (r < NG) lse2[(size_t)bhq * NG + r] = (l_run > 0.f) ? m_new + __log2f(l_run) : 0.f;
         }
       }
