@@ -31,7 +31,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2609_32882_b200 import inputs as syn  # noqa: E402
 
-METRIC = "720p routed sparse attn fwd+bwd dense-equivalent TFLOPS (ms and actual TFLOPS alongside)"
+METRIC = "720p routed sparse attn fwd+bwd ms and TFLOPS (actual & dense-equiv) vs B200 BF16 peak"
 UNIT = "TFLOP/s dense-equivalent"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch of the kernels named below, from the ncu captures summarised under profiles/
