@@ -34,9 +34,11 @@ from paper_2609_32882_b200 import inputs as syn  # noqa: E402
 METRIC = "720p routed sparse attn fwd+bwd ms and TFLOPS (actual & dense-equiv) vs B200 BF16 peak"
 UNIT = "TFLOP/s dense-equivalent"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch of the kernels named below, from the ncu captures summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the 720p top-64 launch with 40 heads: the
+# 8-head ncu capture summarised in profiles/kernels_720p_8heads_ncu_full.md times 5 (every head streams its own
+# tensors, so the traffic grows in proportion to the heads; the 40-head launch is too large for a full-set capture).
+NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.691206e9 + 0.297706e9), "fine_bwd_dq": 5 * (0.928855e9 + 0.152408e9),
+                                "fine_bwd_dkv": 5 * (2.848521e9 + 0.323660e9)}
 
 
 def workload(config: int, heads: int = 0) -> syn.Workload:
@@ -341,7 +343,9 @@ def run_ours(args):
     peak_tf = pk["bf16_tflops_sustained"]
     achieved = kernel_flops[dominant] / (kernel_ms[dominant] * 1e-3) / 1e12
     roofline = {"kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": achieved / peak_tf, "traffic": NCU_TRAFFIC_BYTES.get(dominant), "peak_kind": pk_kind + " sustained bf16",
+                "frac": achieved / peak_tf,
+                "traffic": NCU_TRAFFIC_BYTES_720P_TOP64.get(dominant) if (args.config == 3 and not args.heads) else None,
+                "peak_kind": pk_kind + " sustained bf16",
                 "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant]}
     fine_fwd_tf = flops["fine_fwd"] / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
     bytes_in = sum(host[k].numel() * host[k].element_size() for k in host)
@@ -393,7 +397,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, help="index into the five baseline configurations (3 = 720p top-64)")
-    ap.add_argument("--ref-rows", type=int, default=96, help="query blocks the CPU oracle computes in its sample")
+    ap.add_argument("--ref-rows", type=int, default=480, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small cases for ncu captures)")

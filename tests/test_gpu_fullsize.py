@@ -10,7 +10,7 @@ import torch
 from oracle import vsa2_oracle as orc
 from paper_2609_32882_b200 import binding as vb
 from paper_2609_32882_b200 import inputs as syn
-from vsa2_testlib import (GpuRun, assert_close, check_routing, oracle_arrays, sampled_attention_parity, to_f64)
+from vsa2_testlib import (CudaPath, assert_close, check_routing, oracle_arrays, sampled_attention_parity, to_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -35,7 +35,7 @@ def oracle_route_head(wl, data, b, hq, mode, topk, budgets=None):
 
 def test_config2_480p_gqa_padded():
     wl, data = inputs_for(2)
-    run = GpuRun(wl, data)
+    run = CudaPath(wl, data)
     gmask = run.route()
     assert (gmask.sum(axis=-1) == 78).all()                                   # 87.5 % sparsity: 78 of 624 per row
     for hq in (0, 5, 11):
@@ -53,7 +53,7 @@ def test_config2_480p_gqa_padded():
 
 def test_config3_720p_top64_forward_backward():
     wl, data = inputs_for(3)
-    run = GpuRun(wl, data)
+    run = CudaPath(wl, data)
     gmask = run.route()
     N = wl.n_cubes
     assert (gmask.sum(axis=(-1, -2)) == N * 64).all()                          # exactly N*K pairs per head (Eq. 9)
@@ -71,7 +71,7 @@ def test_config3_720p_top64_forward_backward():
 
 def test_config3_720p_top128_forward_only():
     wl, data = inputs_for(3)
-    run = GpuRun(wl.replace(topk=128), data)
+    run = CudaPath(wl.replace(topk=128), data)
     gmask = run.route()
     assert (gmask.sum(axis=(-1, -2)) == wl.n_cubes * 128).all()
     run.forward()
@@ -82,7 +82,7 @@ def test_config4_budgets_mha_and_dense_reference():
     wl, data = inputs_for(4)
     N = wl.n_cubes
     cap = int(np.minimum(data["budgets"], N).sum(axis=-1).max())
-    run = GpuRun(wl, data, nnz_cap=cap)
+    run = CudaPath(wl, data, nnz_cap=cap)
     gmask = run.route()
     assert np.array_equal(gmask.sum(axis=-1), data["budgets"])                 # every row keeps exactly its budget
     om, P = oracle_route_head(wl, data, 0, 8, syn.PER_QUERY_BUDGET, 0, data["budgets"])
@@ -93,7 +93,7 @@ def test_config4_budgets_mha_and_dense_reference():
     # dense reference: the same kernels with every block kept, against softmax attention over all valid keys
     sub = wl.replace(heads_q=4, heads_kv=4, select_mode=syn.PER_SEQUENCE, topk=N)
     dsub = {k: np.ascontiguousarray(v[:, :4]) for k, v in data.items()}
-    dense = GpuRun(sub, dsub, flags=vb.FLAG_NO_COARSE)
+    dense = CudaPath(sub, dsub, flags=vb.FLAG_NO_COARSE)
     assert dense.route().all()
     dense.forward()
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
@@ -111,7 +111,7 @@ def test_config4_gqa_sparsity_levels():
     N = wl.n_cubes
     for topk in (360, 45):                                                     # 75 % and 96.9 % block sparsity
         w = wl.replace(select_mode=syn.PER_SEQUENCE, topk=topk)
-        run = GpuRun(w, data)
+        run = CudaPath(w, data)
         gmask = run.route()
         assert (gmask.sum(axis=(-1, -2)) == N * topk).all()
         run.forward()

@@ -6,7 +6,7 @@ import torch
 from oracle import vsa2_oracle as orc
 from paper_2609_32882_b200 import binding as vb
 from paper_2609_32882_b200 import inputs as syn
-from vsa2_testlib import (TOL_ABS, GpuRun, assert_close, assert_lse_close, check_routing, dev_bf16, oracle_arrays, to_f64)
+from vsa2_testlib import (TOL_ABS, CudaPath, assert_close, assert_lse_close, check_routing, dev_bf16, oracle_arrays, to_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -20,7 +20,7 @@ MINI_BUDGET = syn.Workload("mini_budget", 1, 2, 1, 128, (8, 8, 12), select_mode=
 def full_parity(wl, data, out_dtype=vb.BF16, nnz_cap=0, check_route=True):
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
     scale = 1.0 / np.sqrt(wl.head_dim)
-    run = GpuRun(wl, data, out_dtype=out_dtype, nnz_cap=nnz_cap)
+    run = CudaPath(wl, data, out_dtype=out_dtype, nnz_cap=nnz_cap)
     a = oracle_arrays(data)
     gmask = run.route()
     if check_route:
@@ -92,7 +92,7 @@ def test_per_query_budget_full_parity():
 def test_all_blocks_kept_equals_dense_attention():
     wl = syn.CONFIGS[1].replace(heads_q=2, heads_kv=2, select_mode=syn.PER_SEQUENCE, topk=32)
     data = syn.make_inputs(wl)
-    run = GpuRun(wl, data, flags=vb.FLAG_NO_COARSE)
+    run = CudaPath(wl, data, flags=vb.FLAG_NO_COARSE)
     assert run.route().all()
     O, lse = run.forward()
     q, k, v = (t.float() for t in (run.q, run.k, run.v))
@@ -105,7 +105,7 @@ def test_gate_none_and_no_coarse_flag_give_fine_only():
     data = syn.make_inputs(wl)
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
     a = oracle_arrays(data)
-    run = GpuRun(wl, data, flags=vb.FLAG_NO_COARSE)
+    run = CudaPath(wl, data, flags=vb.FLAG_NO_COARSE)
     gmask = run.route()
     O, lse = run.forward()
     zero = np.zeros_like(a["gate"])
@@ -124,7 +124,7 @@ def test_results_are_bitwise_reproducible():
     data = syn.make_inputs(wl)
     outs = []
     for _ in range(2):
-        run = GpuRun(wl, data)
+        run = CudaPath(wl, data)
         run.route()
         run.forward()
         run.backward()
@@ -138,7 +138,7 @@ def test_router_pool_is_bit_exact():
     wl = MINI_PADDED
     data = syn.make_inputs(wl)
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
-    run = GpuRun(wl, data)
+    run = CudaPath(wl, data)
     run.route()
     s = run.attn.sizes
     n = wl.batch * wl.heads_q * s.n_cubes * s.n_subcubes * wl.head_dim
@@ -152,7 +152,7 @@ def test_router_pool_is_bit_exact():
 def test_bad_arguments_are_rejected_on_the_gpu_box_too():
     wl = syn.CONFIGS[0]
     data = syn.make_inputs(wl)
-    run = GpuRun(wl, data)
+    run = CudaPath(wl, data)
     with pytest.raises(vb.Vsa2Error) as e:
         vb.vsa2_route(run.p, run.q, run.k, None, run.attn.map, run.attn.ws_route, workspace_bytes=1024)
     assert e.value.code == vb.ERR_WORKSPACE_TOO_SMALL
@@ -166,7 +166,7 @@ def test_tensor_core_forward_matches_exact_maximum_kernel():
     data = syn.make_inputs(wl)
     outs = []
     for flags in (0, vb.FLAG_EXACT_MAX_FWD):
-        run = GpuRun(wl, data, flags=flags, out_dtype=vb.F32)
+        run = CudaPath(wl, data, flags=flags, out_dtype=vb.F32)
         run.route()
         outs.append(run.forward())
     assert np.abs(outs[0][0] - outs[1][0]).max() < 2e-2
@@ -188,7 +188,7 @@ def test_forward_survives_a_late_dominant_key_block():
     q[0, 0, geo.cube_tokens[2]] = 8.0 * np.sign(q[0, 0, big[0]])   # one query block points at them
     data["q"], data["k"] = syn.f32_to_bf16_bits(q), syn.f32_to_bf16_bits(k)
     a = oracle_arrays(data)
-    run = GpuRun(wl, data, flags=vb.FLAG_NO_COARSE, out_dtype=vb.F32)
+    run = CudaPath(wl, data, flags=vb.FLAG_NO_COARSE, out_dtype=vb.F32)
     gmask = run.route()
     assert gmask.all()
     O, lse = run.forward()
@@ -205,7 +205,7 @@ def test_tensor_core_backward_matches_first_generation_kernels():
     data = syn.make_inputs(wl)
     outs = []
     for flags in (0, vb.FLAG_SIMPLE_BWD):
-        run = GpuRun(wl, data, flags=flags, out_dtype=vb.F32)
+        run = CudaPath(wl, data, flags=flags, out_dtype=vb.F32)
         run.route()
         run.forward()
         outs.append(run.backward())
@@ -218,7 +218,7 @@ def test_tensor_core_router_matches_first_generation_kernel():
     data = syn.make_inputs(wl)
     scores = []
     for flags in (0, vb.FLAG_SIMPLE_ROUTER):
-        run = GpuRun(wl, data, flags=flags)
+        run = CudaPath(wl, data, flags=flags)
         run.route()
         scores.append(to_f64(run.attn.scores()))
     assert np.abs(scores[0] - scores[1]).max() <= 1e-5 * scores[1].max()
@@ -235,7 +235,7 @@ def test_tensor_core_coarse_branch_matches_fp32_kernels():
     data = syn.make_inputs(wl)
     outs = []
     for flags in (0, vb.FLAG_SIMPLE_COARSE):
-        run = GpuRun(wl, data, flags=flags, out_dtype=vb.F32)
+        run = CudaPath(wl, data, flags=flags, out_dtype=vb.F32)
         run.route()
         O, lse = run.forward()
         outs.append((O,) + tuple(run.backward()))

@@ -96,7 +96,7 @@ def check_routing(gpu_mask, oracle_mask, P_r, mode):
     return int(diff.sum())
 
 
-class GpuRun:
+class CudaPath:
     """Uploads a workload's tensors and drives the library through the binding."""
 
     def __init__(self, wl, data, out_dtype=vb.BF16, flags=0, nnz_cap=0, **param_overrides):
