@@ -108,7 +108,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc::mbar_init(&misc->o_empty, 256);
     for (int s = 0; s < kFwdKSlots; ++s) {
       tc::mbar_init(&misc->k_full[s], 1);
-      tc::mbar_init(&misc->k_empty[s], 1);
+      tc::mbar_init(&misc->k_empty[s], 2);   // the issuing S^T warp (on completion) and the observing one
     }
     for (int s = 0; s < kFwdVSlots; ++s) {
       tc::mbar_init(&misc->v_full[s], 1);
@@ -202,9 +202,14 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           VSA2_WAIT(&misc->q_full, n_items & 1);
           bool issued = false;
           for (int t = 0; t < nt; ++t, ++tg) {
-            if ((tg & 1) != mine) continue;
+            // Both issuers pass through every phase of the K ring (a slot alternates between them): the issuer that
+            // does not own the tile only observes the load and adds its arrival to the slot's release.
             const uint32_t slot = tg % kFwdKSlots, buf = tg % kFwdSBufs;
             VSA2_WAIT(&misc->k_full[slot], (tg / kFwdKSlots) & 1);
+            if ((tg & 1) != mine) {
+              tc::mbar_arrive(&misc->k_empty[slot]);
+              continue;
+            }
             VSA2_WAIT(&misc->s_free[buf], ((tg / kFwdSBufs) & 1) ^ 1);
             tc::tc_fence_after();
             mma_pair_kmajor<D>(tmem_base + buf * 64, slot0 + slot * C::SLOT, q_addr);
