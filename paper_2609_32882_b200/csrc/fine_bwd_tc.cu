@@ -55,6 +55,7 @@ struct BwdMisc {
   uint64_t p_ready, p_free;                                 // dK/dV pass: the P operand buffer
   uint64_t ds_ready[2], ds_free[2];                         // dS operand buffers (the dK/dV pass has one)
   uint64_t stat_full, stat_free;                            // dK/dV pass: the per-row statistics of a tile
+  ItemQueue items;                                          // work items of this CTA (see tc_attn.cuh)
   uint32_t tmem_base;
   int abort_flag;
   unsigned char edge[kRingA][2];   // dQ pass: edge flags of the two key cubes in each ring-A slot (written by its producer)
@@ -418,6 +419,7 @@ done:
 // dK/dV pass
 // ================================================================================================
 struct DkvArgs {
+  int* item_counter;    // global, zero before the launch
   const float* lse;
   const float* delta;
   const int* col_ptr;
@@ -469,6 +471,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   if (tid == 0) {
     bwd_init_barriers(misc);
     tc::mbar_init(&misc->o_full, 2);                                          // two last-stage issuers
+    item_queue_init(&misc->items, 2 + 4 + 256 + 128);
     for (int s = 0; s < kRingB; ++s) tc::mbar_init(&misc->b_empty[s], 2);     // a dO slot is read by dP and by dV^T
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
@@ -504,8 +507,17 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int which = warp;                               // 0: Q pairs (ring A) + K, V tiles; 1: dO pairs (ring B)
     const CUtensorMap* tm = which == 0 ? &tm_q : &tm_do;
     const int my_blk = lane & 1;
-    uint32_t tg = 0, n_items = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+    uint32_t tg = 0, n_items = 0, published = 0;
+    for (uint32_t seq = 0;; ++seq) {
+      // warp 0, lane 0 is the CTA's scheduler
+      int item = 0;
+      if (lane == 0) {
+        if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
+        else item = item_get(&misc->items, seq, &misc->abort_flag);
+      }
+      item = __shfl_sync(0xffffffffu, item, 0);
+      if (item == -2) goto done;
+      if (item < 0) break;
       VSA2_DKV_ITEM_SETUP();
       if (k == 0) continue;
       if (which == 0) {
@@ -543,7 +555,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const bool is_s = warp == 2;
       const uint32_t b_addr = tc::smem_u32(is_s ? k_tile : v_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      for (uint32_t seq = 0;; ++seq) {
+        VSA2_NEXT_ITEM(item, seq);
         VSA2_DKV_ITEM_SETUP();
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
@@ -578,7 +591,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const bool is_v = warp == 16;
       const uint32_t b_addr = tc::smem_u32(is_v ? p_tile : ds_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      for (uint32_t seq = 0;; ++seq) {
+        VSA2_NEXT_ITEM(item, seq);
         VSA2_DKV_ITEM_SETUP();
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
@@ -615,7 +629,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     cpos.init(g, r & 63);
     float2* rowstat = reinterpret_cast<float2*>(misc->stats);
     uint32_t tg = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+    for (uint32_t seq = 0;; ++seq) {
+      VSA2_NEXT_ITEM(item, seq);
       VSA2_DKV_ITEM_SETUP();
       (void)j; (void)bhk;
       if (k == 0) continue;
@@ -643,8 +658,9 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int row = (quad << 5) | lane;      // query row of the tile (S, dP) / channel (dK^T, dV^T)
     const int sm_tid = tid - 128;            // 0..255
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t tg = 0, n_items = 0, n_all = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
+    uint32_t tg = 0, n_items = 0;
+    for (uint32_t n_all = 0;; ++n_all) {
+      VSA2_NEXT_ITEM(item, n_all);
       VSA2_DKV_ITEM_SETUP();
       (void)col_beg;
       const int tb = n_all & 1;
@@ -847,7 +863,7 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   int sms = 0;
   cudaError_t e;
   if ((e = sm_count(&sms)) != cudaSuccess) return e;
-  DkvArgs a{lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
+  DkvArgs a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
   if (g.D == 128) {

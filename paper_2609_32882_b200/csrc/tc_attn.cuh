@@ -118,6 +118,52 @@ __device__ __forceinline__ int warp_reduce_col(int lane) {
   return ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Work queue of a persistent CTA.  Work items (query blocks or KV blocks) have very different list lengths, so a static
+// round-robin split leaves some CTAs with up to 15 % more tiles than the average.  One thread of the CTA (the
+// scheduler) draws item numbers from a global counter, a few items ahead, and publishes them through a small ring in
+// shared memory; every role of the CTA reads the same sequence from the ring.  All CTAs therefore advance through the
+// item sequence together (neighbouring items share operand tiles in L2) and finish together.  Item -1 ends the CTA.
+constexpr int kItemSlots = 4;       // ring depth
+constexpr int kItemAhead = 2;       // items published ahead of the scheduler's own position
+struct ItemQueue {
+  uint64_t full[kItemSlots], empty[kItemSlots];
+  int item[kItemSlots];
+};
+// `consumers`: threads that call item_get for every sequence number (the scheduler thread included)
+__device__ __forceinline__ void item_queue_init(ItemQueue* q, int consumers) {
+  for (int s = 0; s < kItemSlots; ++s) {
+    tc::mbar_init(&q->full[s], 1);
+    tc::mbar_init(&q->empty[s], consumers);
+  }
+}
+// scheduler: publishes every sequence number up to seq + kItemAhead that is not out yet; false on a timed-out wait
+__device__ __forceinline__ bool item_publish_ahead(ItemQueue* q, uint32_t seq, uint32_t& published, int* counter, int total,
+                                                   volatile int* abort_flag) {
+  while (published <= seq + kItemAhead) {
+    const uint32_t slot = published % kItemSlots, par = ((published / kItemSlots) & 1) ^ 1;
+    if (!tc::mbar_wait_parked(&q->empty[slot], par, abort_flag)) return false;
+    const int it = atomicAdd(counter, 1);
+    q->item[slot] = it < total ? it : -1;
+    tc::mbar_arrive(&q->full[slot]);
+    ++published;
+  }
+  return true;
+}
+// consumer: item of sequence number seq, or -2 if the wait timed out
+__device__ __forceinline__ int item_get(ItemQueue* q, uint32_t seq, volatile int* abort_flag) {
+  const uint32_t slot = seq % kItemSlots, par = (seq / kItemSlots) & 1;
+  if (!tc::mbar_wait_parked(&q->full[slot], par, abort_flag)) return -2;
+  const int it = q->item[slot];
+  tc::mbar_arrive(&q->empty[slot]);
+  return it;
+}
+// loop header of a role whose threads all call it: `for (uint32_t seq = 0;; ++seq) { VSA2_NEXT_ITEM(item, seq); ... }`
+#define VSA2_NEXT_ITEM(ITEM, SEQ)                                  \
+  const int ITEM = item_get(&misc->items, (SEQ), &misc->abort_flag); \
+  if (ITEM == -2) goto done;                                       \
+  if (ITEM < 0) break
+
 #define VSA2_WAIT(bar, parity)                                         \
   do {                                                                 \
     if (!tc::mbar_wait((bar), (parity), &misc->abort_flag)) goto done; \
