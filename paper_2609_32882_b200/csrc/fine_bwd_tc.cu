@@ -119,6 +119,7 @@ __device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
 // dQ pass
 // ================================================================================================
 struct DqArgs {
+  int* item_counter;    // global, zero before the launch
   const float* lse;
   const float* delta;
   const int* row_ptr;
@@ -151,6 +152,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
   if (tid == 0) {
     bwd_init_barriers(misc);
+    item_queue_init(&misc->items, 2 + 3 + 256);     // lane 0 of the producers, three issuers, the elementwise threads
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -172,8 +174,17 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const int which = warp;                               // 0: K pairs (ring A) + Q, dO tiles; 1: V pairs (ring B)
     const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
     const int my_blk = lane & 1;
-    uint32_t tg = 0, n_items = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+    uint32_t tg = 0, n_items = 0, published = 0;
+    for (uint32_t seq = 0;; ++seq) {
+      // warp 0, lane 0 is the CTA's scheduler
+      int item = 0;
+      if (lane == 0) {
+        if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
+        else item = item_get(&misc->items, seq, &misc->abort_flag);
+      }
+      item = __shfl_sync(0xffffffffu, item, 0);
+      if (item == -2) goto done;
+      if (item < 0) break;
       const int i = item % g.N, bhq = item / g.N;
       const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
@@ -218,7 +229,8 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       const bool is_s = warp == 2;
       const uint32_t b_addr = tc::smem_u32(is_s ? q_tile : do_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      for (uint32_t seq = 0;; ++seq) {
+        VSA2_NEXT_ITEM(item, seq);
         const int i = item % g.N, bhq = item / g.N;
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
@@ -251,7 +263,8 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     if (lane == 0) {
       const uint32_t ds_addr = tc::smem_u32(ds_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      for (uint32_t seq = 0;; ++seq) {
+        VSA2_NEXT_ITEM(item, seq);
         const int i = item % g.N, bhq = item / g.N;
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
@@ -280,8 +293,9 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     CubePos cpos;
     cpos.init(g, row & 63);
     const int blk = row >> 6;
-    uint32_t tg = 0, n_items = 0, n_all = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
+    uint32_t tg = 0, n_items = 0;
+    for (uint32_t n_all = 0;; ++n_all) {
+      VSA2_NEXT_ITEM(item, n_all);
       const int i = item % g.N, bhq = item / g.N;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
@@ -838,7 +852,7 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
   int sms = 0;
   cudaError_t e;
   if ((e = sm_count(&sms)) != cudaSuccess) return e;
-  DqArgs a{lse, delta, row_ptr, col_idx, dqc, dq, status};
+  DqArgs a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, dq, status};
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
   if (g.D == 128) {

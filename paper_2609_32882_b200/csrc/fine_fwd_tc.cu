@@ -49,6 +49,7 @@ struct FwdMisc {
   uint64_t v_full[kFwdVSlots], v_empty[kFwdVSlots];
   uint64_t s_full[kFwdSBufs], s_free[kFwdSBufs];
   uint64_t p_ready[2], p_free[2];
+  ItemQueue items;                 // work items of this CTA (see tc_attn.cuh)
   uint32_t tmem_base;
   int abort_flag;
   int rescue_flag;
@@ -61,6 +62,7 @@ struct FwdMisc {
 static_assert(sizeof(FwdMisc) <= 5120, "misc region too small");
 
 struct FwdArgs {
+  int* item_counter;    // global, zero before the launch
   const float* gate;
   const int* row_ptr;
   const int* col_idx;
@@ -122,6 +124,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       tc::mbar_init(&misc->p_ready[s], 128);
       tc::mbar_init(&misc->p_free[s], 1);
     }
+    item_queue_init(&misc->items, 2 + 4 + 256);     // lane 0 of the producers, four issuers, the softmax threads
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -149,8 +152,17 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       unsigned char* ring = smem + (which == 0 ? 0 : kFwdKSlots * C::SLOT);
       const int my_h = lane >> 1, my_blk = lane & 1;
       const bool issuer = lane < 2 * C::DH;
-      uint32_t tg = 0, n_items = 0;
-      for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+      uint32_t tg = 0, n_items = 0, published = 0;
+      for (uint32_t seq = 0;; ++seq) {
+        // warp 0, lane 0 is the CTA's scheduler
+        int item = 0;
+        if (lane == 0) {
+          if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
+          else item = item_get(&misc->items, seq, &misc->abort_flag);
+        }
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item == -2) goto done;
+        if (item < 0) break;
         const int i = item % g.N, bhq = item / g.N;
         const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
         const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
@@ -194,7 +206,8 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t mine = warp - 2;            // parity of the tiles this warp issues
         const uint32_t q_addr = tc::smem_u32(q_tile), slot0 = tc::smem_u32(smem);
         uint32_t tg = 0, n_items = 0;
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        for (uint32_t seq = 0;; ++seq) {
+          VSA2_NEXT_ITEM(item, seq);
           const int i = item % g.N, bhq = item / g.N;
           const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
           if (k == 0) continue;
@@ -230,7 +243,8 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t p_addr = tc::smem_u32(p_tile), slot0 = tc::smem_u32(smem);
         const uint32_t tm_o = tmem_base + 256 + mine * 64;
         uint32_t tg = 0, n_items = 0;
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
+        for (uint32_t seq = 0;; ++seq) {
+          VSA2_NEXT_ITEM(item, seq);
           const int i = item % g.N, bhq = item / g.N;
           const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
           if (k == 0) continue;
@@ -269,7 +283,8 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     cpos.init(g, row & 63);
     const int blk = row >> 6;
     uint32_t tg = 0, n_items = 0, n_all = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_all) {
+    for (;; ++n_all) {
+      VSA2_NEXT_ITEM(item, n_all);
       const int i = item % g.N, bhq = item / g.N;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
@@ -514,6 +529,7 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
   a.gate = gate; a.row_ptr = row_ptr; a.col_idx = col_idx; a.oc_hat = oc_hat; a.o = o; a.o_res = o_res; a.lse = lse;
   a.status = status;
   a.rescue_count = &status->pad[0];
+  a.item_counter = &status->pad[1];
   a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
