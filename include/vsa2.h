@@ -61,6 +61,14 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
                                          the exact running row maximum (the tensor-core kernel falls back to it only
                                          for query blocks whose softmax sums leave the safe range) */
 enum { VSA2_FLAG_SIMPLE_ROUTER = 8 }; /* validation aid: router scores with the slow first-generation kernel */
+/* Coarse branch (Eq. 2-3).  Default: forward with TF32 tensor-core tiles on the fp32 cube means (O_c feeds dGate, which
+ * needs that precision); backward by running the tcgen05 fine-branch kernels on the pooled grid with the means rounded
+ * to bf16 (its results enter dQ, dK, dV divided by the cube size, where bf16 operand rounding is far below the error
+ * bounds). */
+enum { VSA2_FLAG_TF32_COARSE = 32 };  /* validation aid: coarse backward with the TF32 kernels too */
+enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
+                                         (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
+                                         output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
 enum { VSA2_FLAG_SIMPLE_COARSE = 16 };/* validation aid: coarse branch (forward and backward) with the fp32 SIMT kernels
                                          instead of the TF32 tensor-core ones */
 enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */

@@ -22,6 +22,8 @@ FLAG_EXACT_MAX_FWD = 2
 FLAG_SIMPLE_BWD = 4
 FLAG_SIMPLE_ROUTER = 8
 FLAG_SIMPLE_COARSE = 16
+FLAG_TF32_COARSE = 32
+FLAG_BF16_COARSE_FWD = 64
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4

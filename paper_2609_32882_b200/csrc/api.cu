@@ -17,7 +17,7 @@ struct RouteLayout {
   int words;
 };
 struct BwdLayout {
-  size_t status, delta, d_oc_hat, delta_c, dqc, dkc, dvc, total;
+  size_t status, delta, d_oc_hat, delta_c, dqc, dkc, dvc, pooled, total;
 };
 
 struct Carver {
@@ -109,11 +109,14 @@ BwdLayout bwd_layout(const Geo& g) {
   r.dqc = c.take(BHq * g.N * g.D * sizeof(float));
   r.dkc = c.take(BHq * g.N * g.D * sizeof(float));
   r.dvc = c.take(BHq * g.N * g.D * sizeof(float));
+  r.pooled = c.take(pooled_layout(g, true).total);
   r.total = c.off;
   return r;
 }
 
-size_t fwd_workspace_bytes(const Geo&) { return align_up(fine_fwd_tc_workspace_bytes(), 256); }
+// [StatusBlock + rescue list of the fine forward][scratch of the coarse branch on the pooled grid]
+size_t fwd_pooled_offset() { return align_up(fine_fwd_tc_workspace_bytes(), 256); }
+size_t fwd_workspace_bytes(const Geo& g) { return fwd_pooled_offset() + pooled_layout(g, false).total; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -269,8 +272,11 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, 1);
     if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
       VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
-    else
+    else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
       VSA2_CUDA(launch_coarse_fwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+    else
+      VSA2_CUDA(launch_coarse_fwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c,
+                                         at<unsigned char>(workspace, fwd_pooled_offset()), st));
   }
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
   if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
@@ -330,9 +336,12 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
     if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
       VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
                                   at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
-    else
+    else if (g.flags & VSA2_FLAG_TF32_COARSE)
       VSA2_CUDA(launch_coarse_bwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
                                      at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
+    else
+      VSA2_CUDA(launch_coarse_bwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat, dqc,
+                                         dkc, dvc, at<unsigned char>(workspace, lay.pooled), st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);

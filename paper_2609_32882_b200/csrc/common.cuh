@@ -164,6 +164,18 @@ cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf
                             const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                             float* lse, cudaStream_t st);
 
+// coarse branch through the fine-branch kernels on the pooled grid (coarse_pooled.cu); offsets into a scratch region
+struct PooledLayout {
+  size_t status, q16, k16, v16, ptr, idx, do16, delta, dk_kv, dv_kv, total;
+};
+Geo pooled_geo(const Geo& g);
+PooledLayout pooled_layout(const Geo& g, bool backward);
+cudaError_t launch_coarse_fwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
+                                     float* lse_c, void* workspace, cudaStream_t st);
+cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
+                                     const float* lse_c, const float* d_oc_hat, float* dqc, float* dkc, float* dvc,
+                                     void* workspace, cudaStream_t st);
+
 // tensor-core forward (fine_fwd_tc.cu); `status` heads a workspace of fine_fwd_tc_workspace_bytes()
 size_t fine_fwd_tc_workspace_bytes();
 cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,

@@ -242,3 +242,18 @@ def test_tensor_core_coarse_branch_matches_fp32_kernels():
     for name, x, y in zip(("O", "dQ", "dK", "dV", "dGate"), *outs):
         # TF32 operands carry 2^-11 relative rounding; dGate sums 128 such products of magnitude up to ~4
         assert np.abs(x - y).max() < 5e-3, name
+
+
+def test_bf16_coarse_forward_flag_keeps_the_output_bound():
+    # the optional forward of the coarse branch on the pooled grid (bf16 operands): O and LSE within the stated bounds
+    for wl in (syn.CONFIGS[1], MINI_COARSE):
+        data = syn.make_inputs(wl)
+        geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+        scale = 1.0 / np.sqrt(wl.head_dim)
+        run = CudaPath(wl, data, flags=vb.FLAG_BF16_COARSE_FWD, out_dtype=vb.F32)
+        gmask = run.route()
+        a = oracle_arrays(data)
+        O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale)
+        O, lse = run.forward()
+        assert_close("O", O, O_ref)
+        assert_lse_close(lse, lse_ref)
