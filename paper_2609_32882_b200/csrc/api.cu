@@ -269,7 +269,7 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
       VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
       VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
     }
-    ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, 1);
+    ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, (g.flags & VSA2_FLAG_BF16_COARSE_FWD) && !(g.flags & VSA2_FLAG_SIMPLE_COARSE) ? 6 : 1);
     if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
       VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
     else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
@@ -332,7 +332,9 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
                                     delta, coarse ? dgate : nullptr, d_oc_hat, st));
   }
   if (coarse) {
-    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, 2);
+    // SIMT / TF32: two kernels; pooled grid: four casts, the dense map, the pooled preprocess, dQ, dK/dV (+ two group spreads)
+    const bool pooled_bwd = !(g.flags & (VSA2_FLAG_SIMPLE_COARSE | VSA2_FLAG_TF32_COARSE));
+    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, pooled_bwd ? 8 + (g.rep > 1 ? 2 : 0) : 2);
     if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
       VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
                                   at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
