@@ -397,7 +397,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, help="index into the five baseline configurations (3 = 720p top-64)")
-    ap.add_argument("--ref-rows", type=int, default=480, help="query blocks the CPU oracle computes in its sample")
+    ap.add_argument("--ref-rows", type=int, default=1440, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small cases for ncu captures)")

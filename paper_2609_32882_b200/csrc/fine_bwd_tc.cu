@@ -56,6 +56,7 @@ struct BwdMisc {
   uint64_t ds_ready[2], ds_free[2];                         // dS operand buffers (the dK/dV pass has one)
   uint64_t stat_full, stat_free;                            // dK/dV pass: the per-row statistics of a tile
   ItemQueue items;                                          // work items of this CTA (see tc_attn.cuh)
+  uint64_t e_sync;                                          // group barrier of the 256 elementwise threads
   uint32_t tmem_base;
   int abort_flag;
   unsigned char edge[kRingA][2];   // dQ pass: edge flags of the two key cubes in each ring-A slot (written by its producer)
@@ -90,6 +91,7 @@ __device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
     tc::mbar_init(&misc->ds_free[s], 1);
   }
   tc::mbar_init(&misc->p_ready, 256);
+  tc::mbar_init(&misc->e_sync, 256);
   tc::mbar_init(&misc->p_free, 1);
   tc::mbar_init(&misc->stat_full, 128);
   tc::mbar_init(&misc->stat_free, 256);
@@ -300,6 +302,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
       const int tb = n_all & 1;
+      const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
       if (sm_tid < 64) {
         int it_, ih_, iw_;
         cube_coords(g, i, it_, ih_, iw_);
@@ -310,7 +313,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       }
       const float coarse_d = (a.dqc != nullptr && row < D)
                                  ? a.dqc[((size_t)bhq * g.N + i) * D + row] / (float)cube_count(g, i) : 0.f;
-      tc::named_bar_sync(1, 256);
+      VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
         const float4* lse4 = reinterpret_cast<const float4*>(misc->stats + tb * 64) + half * 8;
@@ -398,7 +401,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int c = 0; c < 32; ++c)
               st[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(o0[c]) + coarse_d);
           }
-          tc::named_bar_sync(1, 256);
+          VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 1);
           constexpr int CH = D / 8;
           for (int e = sm_tid; e < 64 * CH; e += 256) {
             const int qi = e / CH, ch = e % CH;
@@ -407,7 +410,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dq) + ((size_t)bhq * g.L + l) * D + ch * 8) =
                 *reinterpret_cast<const uint4*>(st + qi * D + ch * 8);
           }
-          tc::named_bar_sync(1, 256);
+          VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 2);
         }
       }
       if (k > 0) ++n_items;
@@ -678,6 +681,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       VSA2_DKV_ITEM_SETUP();
       (void)col_beg;
       const int tb = n_all & 1;
+      const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
       int jt, jh, jw;
       cube_coords(g, j, jt, jh, jw);
       if (sm_tid < 64) misc->tok[tb][sm_tid] = cube_token(g, jt, jh, jw, sm_tid);
@@ -698,7 +702,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         coarse_k *= inv_cnt;
         coarse_v *= inv_cnt;
       }
-      tc::named_bar_sync(1, 256);
+      VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
         const float2* rowstat = reinterpret_cast<const float2*>(misc->stats);
@@ -800,7 +804,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               st_v[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(vv[c]) + coarse_v);
             }
           }
-          tc::named_bar_sync(1, 256);
+          VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 1);
           constexpr int CH = D / 8;
           for (int e = sm_tid; e < 64 * CH; e += 256) {
             const int c = e / CH, ch = e % CH;
@@ -810,7 +814,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dk) + idx) = *reinterpret_cast<const uint4*>(st_k + c * D + ch * 8);
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dv) + idx) = *reinterpret_cast<const uint4*>(st_v + c * D + ch * 8);
           }
-          tc::named_bar_sync(1, 256);
+          VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 2);
         }
       }
       if (k > 0) ++n_items;

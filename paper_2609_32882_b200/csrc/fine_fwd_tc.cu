@@ -50,6 +50,7 @@ struct FwdMisc {
   uint64_t s_full[kFwdSBufs], s_free[kFwdSBufs];
   uint64_t p_ready[2], p_free[2];
   ItemQueue items;                 // work items of this CTA (see tc_attn.cuh)
+  uint64_t wg_sync[2], all_sync;   // group barriers of one softmax warpgroup (128 threads) and of both (256)
   uint32_t tmem_base;
   int abort_flag;
   int rescue_flag;
@@ -124,6 +125,9 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
       tc::mbar_init(&misc->p_ready[s], 128);
       tc::mbar_init(&misc->p_free[s], 1);
     }
+    tc::mbar_init(&misc->wg_sync[0], 128);
+    tc::mbar_init(&misc->wg_sync[1], 128);
+    tc::mbar_init(&misc->all_sync, 256);
     item_queue_init(&misc->items, 2 + 4 + 256);     // lane 0 of the producers, four issuers, the softmax threads
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
@@ -282,7 +286,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     CubePos cpos;
     cpos.init(g, row & 63);
     const int blk = row >> 6;
-    uint32_t tg = 0, n_items = 0, n_all = 0;
+    uint32_t tg = 0, n_items = 0, n_all = 0, wg_phase = 0, all_phase = 0;
     for (;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
       const int i = item % g.N, bhq = item / g.N;
@@ -328,14 +332,14 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           const int cb = warp_reduce_col(lane);
           misc->red[quad][cb] = mx[0];
           misc->red[quad][cb + 1] = mx[1];
-          tc::named_bar_sync(1 + wg, 128);
+          VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
           if (sm_tid < 64) {
             const float m4 = fmaxf(fmaxf(misc->red[0][sm_tid], misc->red[1][sm_tid]), fmaxf(misc->red[2][sm_tid], misc->red[3][sm_tid]));
             misc->m_ref[sm_tid] = (m4 > -INFINITY) ? m4 * c2 : 0.f;
           }
         }
       }
-      tc::named_bar_sync(3, 256);       // tables and reference exponents visible to both warpgroups
+      VSA2_GROUP_SYNC(&misc->all_sync, all_phase);       // tables and reference exponents visible to both warpgroups
 
       if (k > 0) {
         // first own tile of this query block and the KV block of this thread's key row in it
@@ -402,7 +406,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           misc->red[sm_warp][cb] = l_part[0];
           misc->red[sm_warp][cb + 1] = l_part[1];
         }
-        tc::named_bar_sync(3, 256);
+        VSA2_GROUP_SYNC(&misc->all_sync, all_phase);
         if (wg == 0 && sm_tid < 64) {
           float l = 0.f;
 #pragma unroll
@@ -415,7 +419,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
-        tc::named_bar_sync(3, 256);
+        VSA2_GROUP_SYNC(&misc->all_sync, all_phase);
       }
 
       // O[l, d] = (O_even^T + O_odd^T)[d, q] / l[q] + gate[q] * O_c[d]; this warpgroup owns 32 query columns
@@ -467,7 +471,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
               st_r[qi * D + row] = __float2bfloat16_rn(val - __bfloat162float(vb));
             }
           }
-          tc::named_bar_sync(3, 256);
+          VSA2_GROUP_SYNC(&misc->all_sync, all_phase);
           constexpr int CH = D / 8;                                      // 16-byte chunks per token row
           const int t256 = tid - 256;
           for (int e = t256; e < 64 * CH; e += 256) {
@@ -478,7 +482,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.o) + idx) = *reinterpret_cast<const uint4*>(st_o + qi * D + ch * 8);
             *reinterpret_cast<uint4*>(a.o_res + idx) = *reinterpret_cast<const uint4*>(st_r + qi * D + ch * 8);
           }
-          tc::named_bar_sync(3, 256);        // staging buffers free before the next query block writes P^T
+          VSA2_GROUP_SYNC(&misc->all_sync, all_phase);        // staging buffers free before the next query block writes P^T
         }
       }
       if (k == 0 && wg == 0 && sm_tid < 64 && misc->tok[tb][sm_tid] >= 0)

@@ -168,6 +168,22 @@ __device__ __forceinline__ int item_get(ItemQueue* q, uint32_t seq, volatile int
   do {                                                                 \
     if (!tc::mbar_wait((bar), (parity), &misc->abort_flag)) goto done; \
   } while (0)
+// Barrier among a fixed group of threads, built on an mbarrier (arrival count = size of the group) so that its wait is
+// bounded like every other wait of these kernels: a thread parked in bar.sync could never leave once a partner had
+// given up after a timed-out wait.  PHASE is a per-thread counter of the syncs done on that barrier.
+#define VSA2_GROUP_SYNC(bar, PHASE)                \
+  do {                                             \
+    tc::mbar_arrive(bar);                          \
+    VSA2_WAIT((bar), (PHASE) & 1u);                \
+    ++(PHASE);                                     \
+  } while (0)
+// The same with the index of the sync (0, 1, 2, ... on that barrier) computed by the caller instead of counted.
+#define VSA2_GROUP_SYNC_AT(bar, INDEX)             \
+  do {                                             \
+    tc::mbar_arrive(bar);                          \
+    VSA2_WAIT((bar), (INDEX) & 1u);                \
+  } while (0)
+
 #define VSA2_WAIT_PARKED(bar, parity)                                         \
   do {                                                                        \
     if (!tc::mbar_wait_parked((bar), (parity), &misc->abort_flag)) goto done; \
