@@ -6,18 +6,19 @@
 //     O^T [D,      64 q] += V_pair^T [D, 128] * P^T       (M = D channels,    N = 64 queries, K = 128 keys)
 // K and V tiles arrive by 5-D TMA straight from the raster tensors (one box = one cube, zero-filled outside
 // the grid) into 128-byte-swizzled shared memory; the same V tile that TMA wrote row-per-key is read as an
-// MN-major operand, so nothing is transposed in memory.  Accumulators live in tensor memory: two S^T
-// buffers (64 columns each) and O^T (64 columns).
+// MN-major operand, so nothing is transposed in memory.  Accumulators live in tensor memory: four S^T
+// buffers (64 columns each) and two O^T accumulators (even and odd tiles, summed in the epilogue).
 //
 // Softmax.  One thread owns one key row of S^T, so a query's maximum would need a reduction across 128
 // threads per tile.  Instead each query column keeps a fixed reference M (the exact column maximum of the
 // first tile, in log2 units): P = 2^(s*scale*log2e - M).  Any reference gives the same softmax as long as
 // nothing overflows; the row sums are checked at the end of the query block and a block whose sums left
 // the safe range is recomputed by the exact-maximum kernel (see fine_fwd.cu).  Row sums are accumulated per
-// thread and reduced across the 128 key rows once per query block, deterministically.
+// thread and reduced across the key rows once per query block, deterministically.
 //
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (one elected lane each), warps 2..5 =
-// softmax + epilogue (each owns the tensor-memory lane quadrant warp % 4).  Every wait is bounded.
+// Roles (512 threads): two TMA producer warps, four MMA issuer warps, two softmax + epilogue warpgroups (see the
+// comment above the kernel).  Persistent CTAs draw their query blocks from a global counter (ItemQueue).  Every wait
+// is bounded.
 #include "tc_attn.cuh"
 
 namespace vsa2 {
