@@ -3,7 +3,7 @@
 // Q_r K_r^T * scale, pass 2 recomputes the scores, applies the softmax and pools G x G sub-blocks on chip.
 //
 // A CTA owns 128 consecutive pooled queries (128/G query cubes) of one head and streams the head's pooled
-// keys in tiles of 128 through a TMA ring; S [128 q, 128 keys] lands in tensor memory (two buffers).
+// keys in tiles of 128 through a TMA ring; S [128 q, 128 keys] lands in tensor memory (four buffers).
 // Four compute threads own each query row, 32 key columns of every tile each (a single warp per scheduler keeps
 // the exponential unit only half busy); pass 1 merges their running (max, sum) pairs once per item.  The G
 // rows of a query cube sit in G adjacent lanes: their pooled sums are combined with warp shuffles.
@@ -16,6 +16,7 @@ constexpr int kRtParts = 4;        // compute threads per pooled query row (each
 constexpr int kRtThreads = 64 + 128 * kRtParts;    // TMA warp, MMA warp, 4 * kRtParts compute warps
 constexpr int kRtSlots = 4;
 constexpr int kRtTile = 128;
+constexpr int kRtBufs = 4;         // score tiles in tensor memory (4 x 128 columns = all of it)
 
 template <int D>
 struct RouterTc {
@@ -31,7 +32,7 @@ struct RouterTc {
 struct RouterMisc {
   uint64_t q_full, q_empty;
   uint64_t k_full[kRtSlots], k_empty[kRtSlots];
-  uint64_t s_full[2], s_free[2];
+  uint64_t s_full[kRtBufs], s_free[kRtBufs];
   uint64_t part_ready, part_free;   // pass 1: hand-over of part_stats
   uint32_t tmem_base;
   int abort_flag;
@@ -94,7 +95,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       tc::mbar_init(&misc->k_full[s], 1);
       tc::mbar_init(&misc->k_empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kRtBufs; ++s) {
       tc::mbar_init(&misc->s_full[s], 1);
       tc::mbar_init(&misc->s_free[s], 128 * kRtParts);
     }
@@ -105,7 +106,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     tc::prefetch_tmap(&tm_k);
   }
   if (warp == 1) {
-    tc::tmem_alloc(&misc->tmem_base, 256);
+    tc::tmem_alloc(&misc->tmem_base, 128 * kRtBufs);
     tc::tmem_relinquish();
   }
   tc::tc_fence_before();
@@ -139,9 +140,9 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++n_items) {
         VSA2_WAIT(&misc->q_full, n_items & 1);
         for (int kt = 0; kt < row_tiles; ++kt, ++seq) {
-          const uint32_t slot = seq % kRtSlots, buf = seq & 1;
+          const uint32_t slot = seq % kRtSlots, buf = seq % kRtBufs;
           VSA2_WAIT(&misc->k_full[slot], (seq / kRtSlots) & 1);
-          VSA2_WAIT(&misc->s_free[buf], ((seq >> 1) & 1) ^ 1);
+          VSA2_WAIT(&misc->s_free[buf], ((seq / kRtBufs) & 1) ^ 1);
           tc::tc_fence_after();
           const uint32_t k_addr = slot0 + slot * C::TILE;
 #pragma unroll
@@ -177,8 +178,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       const int qi = r / G;                                       // query cube of this row
       for (int kt = 0; kt < row_tiles; ++kt, ++seq) {
-        const uint32_t buf = seq & 1;
-        VSA2_WAIT(&misc->s_full[buf], (seq >> 1) & 1);
+        const uint32_t buf = seq % kRtBufs;
+        VSA2_WAIT(&misc->s_full[buf], (seq / kRtBufs) & 1);
         tc::tc_fence_after();
 #pragma unroll
         for (int ch = part * (4 / kRtParts); ch < (part + 1) * (4 / kRtParts); ++ch) {
@@ -266,7 +267,7 @@ done:
     }
     __syncthreads();
   }
-  if (warp == 1) tc::tmem_dealloc(tmem_base, 256);
+  if (warp == 1) tc::tmem_dealloc(tmem_base, 128 * kRtBufs);
 }
 
 bool router_tc_supported(const Geo& g) { return g.G == 8 || g.G == 16; }
