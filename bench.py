@@ -41,10 +41,12 @@ NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.498845e9 + 0.294212e9), "fine
                                 "fine_bwd_dkv": 5 * (0.776757e9 + 0.304371e9)}
 
 
-def workload(config: int, heads: int = 0) -> syn.Workload:
+def workload(config: int, heads: int = 0, topk: int = 0) -> syn.Workload:
     wl = syn.CONFIGS[config]
     if heads:
         wl = wl.replace(heads_q=heads, heads_kv=max(1, heads * wl.heads_kv // wl.heads_q), name=f"{wl.name}_{heads}heads")
+    if topk:
+        wl = wl.replace(topk=topk, name=f"{wl.name}_top{topk}")
     return wl
 
 
@@ -177,7 +179,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = workload(args.config, args.heads)
+    wl = workload(args.config, args.heads, args.topk)
     hd = head_inputs(wl, 0, 0)
     flops = flop_counts(wl, 0)
     for _ in range(args.warmup):
@@ -228,7 +230,7 @@ def run_ours(args):
     vb._lib()
 
     # every rank runs its own replica of the workload (heads are independent: no data-path collective)
-    wl = workload(args.config, args.heads)
+    wl = workload(args.config, args.heads, args.topk)
     wl = wl.replace(seed=replicas.replica_seed(wl.seed, rank))
     t_gen = time.time()
     data = syn.make_inputs(wl, threads=max(1, min(32, cpu_cores() // max(1, world))))
@@ -257,6 +259,8 @@ def run_ours(args):
     def step():
         attn.route(dev["q"], dev["k"], budgets)
         attn.forward(dev["q"], dev["k"], dev["v"], dev["gate"], o=o, lse=lse)
+        if args.forward_only:
+            return
         attn.backward(dev["q"], dev["k"], dev["v"], dev["gate"], o, lse, dev["do"], dq=dq, dk=dk, dv=dv, dgate=dgate)
 
     # End to end: every step copies its inputs from pinned host memory and its results back, inside the timed region.
@@ -291,8 +295,9 @@ def run_ours(args):
                 stream.wait_event(ev_out[n - 2])             # the result set has been read back
             attn.route(d["q"], d["k"], budgets)
             attn.forward(d["q"], d["k"], d["v"], d["gate"], o=r["o"], lse=r["lse"])
-            attn.backward(d["q"], d["k"], d["v"], d["gate"], r["o"], r["lse"], d["do"], dq=r["dq"], dk=r["dk"], dv=r["dv"],
-                          dgate=r["dgate"])
+            if not args.forward_only:
+                attn.backward(d["q"], d["k"], d["v"], d["gate"], r["o"], r["lse"], d["do"], dq=r["dq"], dk=r["dk"],
+                              dv=r["dv"], dgate=r["dgate"])
             ev_comp[n].record(stream)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_comp[n])
@@ -362,6 +367,9 @@ def run_ours(args):
         return
 
     flops = flop_counts(wl, nnz_total)
+    if args.forward_only:
+        flops["dense_equiv_fwd_bwd"] = flops["dense_equiv_fwd"]
+        flops["fine_bwd_dq_executed"] = flops["fine_bwd_dkv_executed"] = 0.0
     ms_step = ms_total / args.steps
     ms_step_e2e = ms_e2e / args.steps
     value = replicas.whole_job_throughput(flops["dense_equiv_fwd_bwd"], world, ms_step * 1e-3) / 1e12
@@ -377,7 +385,7 @@ def run_ours(args):
     achieved = kernel_flops[dominant] / (kernel_ms[dominant] * 1e-3) / 1e12
     roofline = {"kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved / peak_tf,
-                "traffic": NCU_TRAFFIC_BYTES_720P_TOP64.get(dominant) if (args.config == 3 and not args.heads) else None,
+                "traffic": NCU_TRAFFIC_BYTES_720P_TOP64.get(dominant) if (args.config == 3 and not args.heads and not args.topk) else None,
                 "peak_kind": pk_kind + " sustained bf16",
                 "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant]}
     fine_fwd_tf = flops["fine_fwd"] / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
@@ -403,7 +411,7 @@ def run_ours(args):
         "data": "synthetic",
         "config": {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
                    "head_dim": wl.head_dim, "cube": list(wl.cube), "rpool": list(wl.rpool), "select_mode": wl.select_mode,
-                   "topk": wl.topk, "selected_pairs": nnz_total, "replicas": world,
+                   "topk": wl.topk, "selected_pairs": nnz_total, "replicas": world, "forward_only": bool(args.forward_only),
                    "l2": "inputs (Q,K,V,dO: 3.1 GB) far larger than the 126 MB L2; no explicit flush",
                    "input_gen_s": round(t_gen, 1)},
         "clocks": clocks,
@@ -435,6 +443,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=1440, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
+    ap.add_argument("--topk", type=int, default=0, help="override the TopK of the configuration (context rows: top-128)")
+    ap.add_argument("--forward-only", action="store_true", help="route + forward only (context rows: inference)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small cases for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
