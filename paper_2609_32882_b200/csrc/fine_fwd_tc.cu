@@ -539,6 +539,13 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
   if (g.N > kFwdMaxCubes) return cudaErrorInvalidValue;
+  // The softmax warpgroups raise their register count to 200 with the registers the service warpgroups give up
+  // (setmaxnreg); that request would block for ever if the launch allocation were smaller than 128 per thread.
+  {
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, g.D == 128 ? (const void*)fine_fwd_tc_kernel<128> : (const void*)fine_fwd_tc_kernel<64>)) != cudaSuccess) return e;
+    if (fa.numRegs * kFwdThreads < 256 * 56 + 256 * 200) return cudaErrorLaunchOutOfResources;
+  }
   if (g.D == 128) {
     const size_t smb = FwdTc<128>::smem_bytes(g.N);
     if ((e = cudaFuncSetAttribute(fine_fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
