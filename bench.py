@@ -41,8 +41,12 @@ NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.498845e9 + 0.294212e9), "fine
                                 "fine_bwd_dkv": 5 * (0.776757e9 + 0.304371e9)}
 
 
-def workload(config: int, heads: int = 0, topk: int = 0) -> syn.Workload:
+def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None) -> syn.Workload:
     wl = syn.CONFIGS[config]
+    if grid:
+        wl = wl.replace(grid=tuple(grid), name=f"{wl.name}_grid{'x'.join(map(str, grid))}")
+    if cube:
+        wl = wl.replace(cube=tuple(cube), name=f"{wl.name}_cube{'x'.join(map(str, cube))}")
     if heads:
         wl = wl.replace(heads_q=heads, heads_kv=max(1, heads * wl.heads_kv // wl.heads_q), name=f"{wl.name}_{heads}heads")
     if topk:
@@ -52,8 +56,8 @@ def workload(config: int, heads: int = 0, topk: int = 0) -> syn.Workload:
 
 def flop_counts(wl: syn.Workload, nnz_total: int) -> dict:
     """Algorithmic work of one step.  nnz_total = selected (query block, KV block) pairs over all heads."""
-    B, D = 64, wl.head_dim
-    L, Hq, N, G = wl.L, wl.heads_q * wl.batch, wl.n_cubes, 8
+    B, D = int(np.prod(wl.cube)), wl.head_dim
+    L, Hq, N, G = wl.L, wl.heads_q * wl.batch, wl.n_cubes, int(np.prod(wl.cube)) // int(np.prod(wl.rpool))
     pair = B * B * D
     return {
         "dense_equiv_fwd": 4.0 * L * L * D * Hq,
@@ -179,7 +183,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = workload(args.config, args.heads, args.topk)
+    wl = workload(args.config, args.heads, args.topk, args.grid, args.cube)
     hd = head_inputs(wl, 0, 0)
     flops = flop_counts(wl, 0)
     for _ in range(args.warmup):
@@ -230,7 +234,7 @@ def run_ours(args):
     vb._lib()
 
     # every rank runs its own replica of the workload (heads are independent: no data-path collective)
-    wl = workload(args.config, args.heads, args.topk)
+    wl = workload(args.config, args.heads, args.topk, args.grid, args.cube)
     wl = wl.replace(seed=replicas.replica_seed(wl.seed, rank))
     t_gen = time.time()
     data = syn.make_inputs(wl, threads=max(1, min(32, cpu_cores() // max(1, world))))
@@ -385,7 +389,7 @@ def run_ours(args):
     achieved = kernel_flops[dominant] / (kernel_ms[dominant] * 1e-3) / 1e12
     roofline = {"kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved / peak_tf,
-                "traffic": NCU_TRAFFIC_BYTES_720P_TOP64.get(dominant) if (args.config == 3 and not args.heads and not args.topk) else None,
+                "traffic": NCU_TRAFFIC_BYTES_720P_TOP64.get(dominant) if (args.config == 3 and not (args.heads or args.topk or args.grid or args.cube)) else None,
                 "peak_kind": pk_kind + " sustained bf16",
                 "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant]}
     fine_fwd_tf = flops["fine_fwd"] / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
@@ -412,7 +416,8 @@ def run_ours(args):
         "config": {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
                    "head_dim": wl.head_dim, "cube": list(wl.cube), "rpool": list(wl.rpool), "select_mode": wl.select_mode,
                    "topk": wl.topk, "selected_pairs": nnz_total, "replicas": world, "forward_only": bool(args.forward_only),
-                   "l2": "inputs (Q,K,V,dO: 3.1 GB) far larger than the 126 MB L2; no explicit flush",
+                   "l2": f"inputs (Q,K,V,dO: {sum(host[k].numel() * 2 for k in ('q', 'k', 'v', 'do')) / 1e9:.1f} GB) far larger than the "
+                         "126 MB L2; no explicit flush",
                    "input_gen_s": round(t_gen, 1)},
         "clocks": clocks,
         "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_step_e2e, "h2d_bytes_per_step": bytes_in,
@@ -445,6 +450,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     ap.add_argument("--topk", type=int, default=0, help="override the TopK of the configuration (context rows: top-128)")
     ap.add_argument("--forward-only", action="store_true", help="route + forward only (context rows: inference)")
+    triple = lambda t: tuple(int(x) for x in t.split(","))
+    ap.add_argument("--grid", type=triple, default=None, help="override the latent grid T,H,W (context rows: the paper's 61,45,80)")
+    ap.add_argument("--cube", type=triple, default=None, help="override the cube, e.g. 4,4,8 (128 tokens; context rows)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small cases for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -40,7 +40,11 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   if (p->topk < 0 || p->nnz_cap < 0 || !(p->softmax_scale >= 0.f)) return VSA2_ERR_INVALID_ARG;
   if (p->cube_t % p->rpool_t || p->cube_h % p->rpool_h || p->cube_w % p->rpool_w) return VSA2_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return VSA2_ERR_UNSUPPORTED;
-  if ((long long)p->cube_t * p->cube_h * p->cube_w != kBlockTokens) return VSA2_ERR_UNSUPPORTED;
+  // 64-token cubes, or 128-token cubes that split along w into two 64-token halves the router pooling respects
+  const long long cube_tokens = (long long)p->cube_t * p->cube_h * p->cube_w;
+  const bool wide = cube_tokens == 2 * kBlockTokens;
+  if (cube_tokens != kBlockTokens && !wide) return VSA2_ERR_UNSUPPORTED;
+  if (wide && (p->cube_w % 2 || (p->cube_w / 2) % p->rpool_w)) return VSA2_ERR_UNSUPPORTED;
   if (p->batch > 65535 || p->heads_q > 65535 || p->heads_q / p->heads_kv > 16) return VSA2_ERR_UNSUPPORTED;
   g->batch = p->batch; g->Hq = p->heads_q; g->Hkv = p->heads_kv; g->rep = p->heads_q / p->heads_kv; g->D = p->head_dim;
   g->T = p->grid_t; g->H = p->grid_h; g->W = p->grid_w;
@@ -53,7 +57,9 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   g->Rt = p->rpool_t; g->Rh = p->rpool_h; g->Rw = p->rpool_w;
   g->Gt = g->Bt / g->Rt; g->Gh = g->Bh / g->Rh; g->Gw = g->Bw / g->Rw;
   g->G = g->Gt * g->Gh * g->Gw;
-  if (128 % g->G) return VSA2_ERR_UNSUPPORTED;
+  if (128 % (wide ? g->G / 2 : g->G)) return VSA2_ERR_UNSUPPORTED;
+  // the second half of the last cube along w must hold at least one grid column (no empty half-cubes)
+  if (wide && (2 * g->Nw - 1) * (g->Bw / 2) >= g->W) return VSA2_ERR_UNSUPPORTED;
   int K = p->topk;
   if (K == 0) {
     if (!(p->keep_fraction > 0.f) || p->keep_fraction > 1.f) {
@@ -116,7 +122,67 @@ BwdLayout bwd_layout(const Geo& g) {
 
 // [StatusBlock + rescue list of the fine forward][scratch of the coarse branch on the pooled grid]
 size_t fwd_pooled_offset() { return align_up(fine_fwd_tc_workspace_bytes(), 256); }
-size_t fwd_workspace_bytes(const Geo& g) { return fwd_pooled_offset() + pooled_layout(g, false).total; }
+
+// 128-token cubes: the regions above are laid out for the half-cube problem (`n` = narrow_geo), followed by what
+// links the two levels: cube-level router scores, half-cube copies of the coarse tensors and of the block map.
+struct WideRouteLayout {
+  RouteLayout narrow;      // status, qr, kr, lse_r, pr (half-cube scores); its selection scratch is unused
+  RouteLayout cube;        // selection scratch and pr at cube level, offsets relative to `cube_base`
+  size_t cube_base, total;
+};
+WideRouteLayout wide_route_layout(const Geo& g) {
+  WideRouteLayout r;
+  r.narrow = route_layout(narrow_geo(g));
+  r.cube = route_layout(g);
+  r.cube_base = align_up(r.narrow.hist, 256);     // everything from the half-cube histograms on is not needed
+  r.total = r.cube_base + r.cube.total;
+  return r;
+}
+struct WideFwdLayout {
+  size_t pooled, x64, oc_hat64, ptr64, idx64, total;
+};
+WideFwdLayout wide_fwd_layout(const Geo& g) {
+  const Geo n = narrow_geo(g);
+  WideFwdLayout r;
+  Carver c;
+  const size_t BHq = (size_t)g.batch * g.Hq;
+  c.take(fine_fwd_tc_workspace_bytes());
+  r.pooled = c.take(pooled_layout(g, false).total);
+  r.x64 = c.take(BHq * n.N * n.D * sizeof(float));
+  r.oc_hat64 = c.take(BHq * n.N * n.D * sizeof(float));
+  r.ptr64 = c.take(BHq * (n.N + 1) * sizeof(int));
+  r.idx64 = c.take(BHq * (size_t)n.nnz_cap * sizeof(int));
+  r.total = c.off;
+  return r;
+}
+struct WideBwdLayout {
+  BwdLayout narrow;        // status, delta, d_oc_hat, dqc, dkc, dvc at half-cube level (delta_c and pooled unused)
+  BwdLayout cube;          // d_oc_hat, delta_c, dqc, dkc, dvc, pooled at cube level, offsets relative to `cube_base`
+  size_t cube_base, oc_hat64, ptr64, idx64, cptr64, ridx64, total;
+};
+WideBwdLayout wide_bwd_layout(const Geo& g) {
+  const Geo n = narrow_geo(g);
+  WideBwdLayout r;
+  r.narrow = bwd_layout(n);
+  r.cube = bwd_layout(g);
+  r.cube_base = align_up(r.narrow.pooled, 256);
+  Carver c;
+  c.off = r.cube_base + r.cube.total;
+  const size_t BHq = (size_t)g.batch * g.Hq;
+  r.oc_hat64 = c.take(BHq * n.N * n.D * sizeof(float));
+  r.ptr64 = c.take(BHq * (n.N + 1) * sizeof(int));
+  r.idx64 = c.take(BHq * (size_t)n.nnz_cap * sizeof(int));
+  r.cptr64 = c.take(BHq * (n.N + 1) * sizeof(int));
+  r.ridx64 = c.take(BHq * (size_t)n.nnz_cap * sizeof(int));
+  r.total = c.off;
+  return r;
+}
+
+size_t route_workspace_bytes(const Geo& g) { return wide_cube(g) ? wide_route_layout(g).total : route_layout(g).total; }
+size_t fwd_workspace_bytes(const Geo& g) {
+  return wide_cube(g) ? wide_fwd_layout(g).total : fwd_pooled_offset() + pooled_layout(g, false).total;
+}
+size_t bwd_workspace_bytes(const Geo& g) { return wide_cube(g) ? wide_bwd_layout(g).total : bwd_layout(g).total; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -176,7 +242,7 @@ int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
   memset(out, 0, sizeof(*out));
   out->n_cubes = g.N;
   out->n_subcubes = g.G;
-  out->block_tokens = kBlockTokens;
+  out->block_tokens = g.Bt * g.Bh * g.Bw;
   out->topk_eff = g.K;
   out->seq_len = g.L;
   out->nnz_cap = g.nnz_cap;
@@ -187,9 +253,9 @@ int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
   out->pooled_kv_elems = BHk * g.N * g.D;
   out->lse_c_elems = BHq * g.N;
   out->o_res_elems = g.out_f32 ? 0 : BHq * (long long)g.L * g.D;
-  out->route_workspace_bytes = route_layout(g).total;
+  out->route_workspace_bytes = route_workspace_bytes(g);
   out->fwd_workspace_bytes = fwd_workspace_bytes(g);
-  out->bwd_workspace_bytes = bwd_layout(g).total;
+  out->bwd_workspace_bytes = bwd_workspace_bytes(g);
   return VSA2_OK;
 }
 
@@ -202,24 +268,42 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
     return VSA2_ERR_INVALID_ARG;
   if (g.mode == VSA2_PER_QUERY_BUDGET && budgets == nullptr) return VSA2_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned256(workspace)) return VSA2_ERR_MISALIGNED;
-  const RouteLayout lay = route_layout(g);
-  if (workspace_bytes < lay.total) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < route_workspace_bytes(g)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
   if ((rc = check_device()) != VSA2_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  StatusBlock* status = at<StatusBlock>(workspace, lay.status);
+  // 128-token cubes: sub-cube means and router scores at half-cube level (`r`), folded to cube scores; the
+  // selection then runs on the cube-level matrix
+  const bool wide = wide_cube(g);
+  const Geo r = wide ? narrow_geo(g) : g;
+  const RouteLayout rl = route_layout(r);
+  RouteLayout lay = rl;
+  unsigned char* sel_base = reinterpret_cast<unsigned char*>(workspace);
+  if (wide) {
+    const WideRouteLayout wl = wide_route_layout(g);
+    lay = wl.cube;
+    sel_base += wl.cube_base;
+  }
+  StatusBlock* status = at<StatusBlock>(workspace, rl.status);
   VSA2_CUDA(cudaMemsetAsync(status, 0, sizeof(StatusBlock), st));
-  bf16* qr = at<bf16>(workspace, lay.qr);
-  bf16* kr = at<bf16>(workspace, lay.kr);
+  bf16* qr = at<bf16>(workspace, rl.qr);
+  bf16* kr = at<bf16>(workspace, rl.kr);
   {
     ProfScope ps(VSA2_KERNEL_POOL, st, 2);
-    VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(q), g.Hq, qr, nullptr, st));
-    VSA2_CUDA(launch_pool(g, reinterpret_cast<const bf16*>(k), g.Hkv, kr, nullptr, st));
+    VSA2_CUDA(launch_pool(r, reinterpret_cast<const bf16*>(q), r.Hq, qr, nullptr, st));
+    VSA2_CUDA(launch_pool(r, reinterpret_cast<const bf16*>(k), r.Hkv, kr, nullptr, st));
   }
-  float* pr = at<float>(workspace, lay.pr);
-  if (router_tc_supported(g) && !(g.flags & VSA2_FLAG_SIMPLE_ROUTER))
-    VSA2_CUDA(launch_router_scores_tc(g, qr, kr, at<float>(workspace, lay.lse_r), pr, status, st));
+  float* pr = at<float>(workspace, rl.pr);
+  if (router_tc_supported(r) && !(g.flags & VSA2_FLAG_SIMPLE_ROUTER))
+    VSA2_CUDA(launch_router_scores_tc(r, qr, kr, at<float>(workspace, rl.lse_r), pr, status, st));
   else
-    VSA2_CUDA(launch_router_scores(g, qr, kr, at<float>(workspace, lay.lse_r), pr, st));
+    VSA2_CUDA(launch_router_scores(r, qr, kr, at<float>(workspace, rl.lse_r), pr, st));
+  if (wide) {
+    g_launches += 1;
+    float* pr_cube = at<float>(sel_base, lay.pr);
+    VSA2_CUDA(launch_fold_scores(r, pr, pr_cube, st));
+    pr = pr_cube;
+  }
+  workspace = sel_base;
   SelectScratch s;
   s.hist = at<unsigned>(workspace, lay.hist);
   s.state = at<unsigned>(workspace, lay.state);
@@ -240,7 +324,12 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
 const float* vsa2_route_scores(const vsa2_params* p, const void* workspace) {
   Geo g;
   if (workspace == nullptr || fill_geo(p, &g) != VSA2_OK) return nullptr;
-  return reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(workspace) + route_layout(g).pr);
+  size_t off = route_layout(g).pr;
+  if (wide_cube(g)) {
+    const WideRouteLayout wl = wide_route_layout(g);
+    off = wl.cube_base + wl.cube.pr;
+  }
+  return reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(workspace) + off);
 }
 
 int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
@@ -262,32 +351,62 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
   const bf16* qb = reinterpret_cast<const bf16*>(q);
   const bf16* kb = reinterpret_cast<const bf16*>(k);
   const bf16* vb = reinterpret_cast<const bf16*>(v);
+  // 128-token cubes: the fine kernels run on the half-cube problem `n` with the expanded map; the coarse branch
+  // runs at cube level from folded half-cube means
+  const bool wide = wide_cube(g);
+  const Geo n = wide ? narrow_geo(g) : g;
+  const WideFwdLayout wl = wide ? wide_fwd_layout(g) : WideFwdLayout();
+  const size_t pooled_off = wide ? wl.pooled : fwd_pooled_offset();
+  const int* row_ptr = map->row_ptr;
+  const int* col_idx = map->col_idx;
+  const float* oc_hat = coarse ? saved->oc_hat : nullptr;
   if (coarse) {
     {
-      ProfScope ps(VSA2_KERNEL_POOL, st, 3);
-      VSA2_CUDA(launch_pool(g, qb, g.Hq, nullptr, saved->qc, st));
-      VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
-      VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
+      ProfScope ps(VSA2_KERNEL_POOL, st, wide ? 6 : 3);
+      if (!wide) {
+        VSA2_CUDA(launch_pool(g, qb, g.Hq, nullptr, saved->qc, st));
+        VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
+        VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
+      } else {
+        float* x64 = at<float>(workspace, wl.x64);
+        VSA2_CUDA(launch_pool(n, qb, n.Hq, nullptr, x64, st));
+        VSA2_CUDA(launch_fold_mean(n, n.Hq, x64, saved->qc, st));
+        VSA2_CUDA(launch_pool(n, kb, n.Hkv, nullptr, x64, st));
+        VSA2_CUDA(launch_fold_mean(n, n.Hkv, x64, saved->kc, st));
+        VSA2_CUDA(launch_pool(n, vb, n.Hkv, nullptr, x64, st));
+        VSA2_CUDA(launch_fold_mean(n, n.Hkv, x64, saved->vc, st));
+      }
     }
-    ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, (g.flags & VSA2_FLAG_BF16_COARSE_FWD) && !(g.flags & VSA2_FLAG_SIMPLE_COARSE) ? 6 : 1);
-    if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
-      VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
-    else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
-      VSA2_CUDA(launch_coarse_fwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
-    else
-      VSA2_CUDA(launch_coarse_fwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c,
-                                         at<unsigned char>(workspace, fwd_pooled_offset()), st));
+    {
+      ProfScope ps(VSA2_KERNEL_COARSE_FWD, st,
+                   ((g.flags & VSA2_FLAG_BF16_COARSE_FWD) && !(g.flags & VSA2_FLAG_SIMPLE_COARSE) ? 6 : 1) + (wide ? 1 : 0));
+      if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
+        VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+      else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
+        VSA2_CUDA(launch_coarse_fwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+      else
+        VSA2_CUDA(launch_coarse_fwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c,
+                                           at<unsigned char>(workspace, pooled_off), st));
+      if (wide) {
+        VSA2_CUDA(launch_expand_rows(n, n.Hq, false, saved->oc_hat, at<float>(workspace, wl.oc_hat64), st));
+        oc_hat = at<float>(workspace, wl.oc_hat64);
+      }
+    }
+  }
+  if (wide) {
+    g_launches += 1;
+    VSA2_CUDA(launch_expand_map(n, map->row_ptr, map->col_idx, at<int>(workspace, wl.ptr64), at<int>(workspace, wl.idx64), st));
+    row_ptr = at<int>(workspace, wl.ptr64);
+    col_idx = at<int>(workspace, wl.idx64);
   }
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
   if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
   {
     ProfScope ps(VSA2_KERNEL_FINE_FWD, st, (g.flags & VSA2_FLAG_EXACT_MAX_FWD) ? 1 : 2);
     if (g.flags & VSA2_FLAG_EXACT_MAX_FWD)
-      VSA2_CUDA(launch_fine_fwd(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
-                                coarse ? saved->oc_hat : nullptr, o, o_res, lse, st));
+      VSA2_CUDA(launch_fine_fwd(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse, st));
     else
-      VSA2_CUDA(launch_fine_fwd_tc(g, qb, kb, vb, coarse ? gate : nullptr, map->row_ptr, map->col_idx,
-                                   coarse ? saved->oc_hat : nullptr, o, o_res, lse,
+      VSA2_CUDA(launch_fine_fwd_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                    reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;
@@ -309,11 +428,18 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
       !aligned16(dk) || !aligned16(dv) || !aligned256(workspace))
     return VSA2_ERR_MISALIGNED;
-  const BwdLayout lay = bwd_layout(g);
-  if (workspace_bytes < lay.total) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < bwd_workspace_bytes(g)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
   if ((rc = check_device()) != VSA2_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   VSA2_CUDA(cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), st));
+  // 128-token cubes: preprocess and the fine passes run on the half-cube problem `n` (regions `lay`), the coarse
+  // backward at cube level (regions `cl` behind `cube_ws`); folds and expansions link the two
+  const bool wide = wide_cube(g);
+  const Geo n = wide ? narrow_geo(g) : g;
+  const WideBwdLayout wl = wide ? wide_bwd_layout(g) : WideBwdLayout();
+  const BwdLayout lay = wide ? wl.narrow : bwd_layout(g);
+  const BwdLayout cl = wide ? wl.cube : lay;
+  void* cube_ws = wide ? at<unsigned char>(workspace, wl.cube_base) : workspace;
   const bf16* qb = reinterpret_cast<const bf16*>(q);
   const bf16* kb = reinterpret_cast<const bf16*>(k);
   const bf16* vb = reinterpret_cast<const bf16*>(v);
@@ -323,46 +449,73 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   float* dqc = at<float>(workspace, lay.dqc);
   float* dkc = at<float>(workspace, lay.dkc);
   float* dvc = at<float>(workspace, lay.dvc);
+  float* d_oc_hat_cube = at<float>(cube_ws, cl.d_oc_hat);
+  float* dqc_cube = at<float>(cube_ws, cl.dqc);
+  float* dkc_cube = at<float>(cube_ws, cl.dkc);
+  float* dvc_cube = at<float>(cube_ws, cl.dvc);
+  const int* row_ptr = map->row_ptr;
+  const int* col_idx = map->col_idx;
+  const int* col_ptr = map->col_ptr;
+  const int* row_idx = map->row_idx;
+  const float* oc_hat = coarse ? saved->oc_hat : nullptr;
+  if (wide) {
+    g_launches += 2;
+    VSA2_CUDA(launch_expand_map(n, map->row_ptr, map->col_idx, at<int>(workspace, wl.ptr64), at<int>(workspace, wl.idx64), st));
+    VSA2_CUDA(launch_expand_map(n, map->col_ptr, map->row_idx, at<int>(workspace, wl.cptr64), at<int>(workspace, wl.ridx64), st));
+    row_ptr = at<int>(workspace, wl.ptr64);
+    col_idx = at<int>(workspace, wl.idx64);
+    col_ptr = at<int>(workspace, wl.cptr64);
+    row_idx = at<int>(workspace, wl.ridx64);
+    if (coarse) {
+      g_launches += 1;
+      VSA2_CUDA(launch_expand_rows(n, n.Hq, false, saved->oc_hat, at<float>(workspace, wl.oc_hat64), st));
+      oc_hat = at<float>(workspace, wl.oc_hat64);
+    }
+  }
   if (!coarse && dgate != nullptr)
     VSA2_CUDA(cudaMemsetAsync(dgate, 0, (size_t)g.batch * g.Hq * g.L * sizeof(float), st));
   const bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<const bf16*>(saved->o_res) : nullptr;
   {
     ProfScope ps(VSA2_KERNEL_BWD_PRE, st, 1);
-    VSA2_CUDA(launch_bwd_preprocess(g, dob, o, o_res, coarse ? gate : nullptr, coarse ? saved->oc_hat : nullptr,
-                                    delta, coarse ? dgate : nullptr, d_oc_hat, st));
+    VSA2_CUDA(launch_bwd_preprocess(n, dob, o, o_res, coarse ? gate : nullptr, oc_hat, delta, coarse ? dgate : nullptr,
+                                    d_oc_hat, st));
   }
   if (coarse) {
     // SIMT / TF32: two kernels; pooled grid: four casts, the dense map, the pooled preprocess, dQ, dK/dV (+ two group spreads)
     const bool pooled_bwd = !(g.flags & (VSA2_FLAG_SIMPLE_COARSE | VSA2_FLAG_TF32_COARSE));
-    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, pooled_bwd ? 8 + (g.rep > 1 ? 2 : 0) : 2);
+    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, (pooled_bwd ? 8 + (g.rep > 1 ? 2 : 0) : 2) + (wide ? 4 : 0));
+    if (wide) VSA2_CUDA(launch_fold_sum(n, n.Hq, d_oc_hat, d_oc_hat_cube, st));
     if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
-      VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
-                                  at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
+      VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
+                                  at<float>(cube_ws, cl.delta_c), dqc_cube, dkc_cube, dvc_cube, st));
     else if (g.flags & VSA2_FLAG_TF32_COARSE)
-      VSA2_CUDA(launch_coarse_bwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat,
-                                     at<float>(workspace, lay.delta_c), dqc, dkc, dvc, st));
+      VSA2_CUDA(launch_coarse_bwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
+                                     at<float>(cube_ws, cl.delta_c), dqc_cube, dkc_cube, dvc_cube, st));
     else
-      VSA2_CUDA(launch_coarse_bwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat, dqc,
-                                         dkc, dvc, at<unsigned char>(workspace, lay.pooled), st));
+      VSA2_CUDA(launch_coarse_bwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
+                                         dqc_cube, dkc_cube, dvc_cube, at<unsigned char>(cube_ws, cl.pooled), st));
+    if (wide) {
+      VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dqc_cube, dqc, st));
+      VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dkc_cube, dkc, st));
+      VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dvc_cube, dvc, st));
+    }
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
     if (g.flags & VSA2_FLAG_SIMPLE_BWD)
-      VSA2_CUDA(launch_fine_bwd_dq(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx,
-                                   coarse ? dqc : nullptr, dq, st));
+      VSA2_CUDA(launch_fine_bwd_dq(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq, st));
     else
-      VSA2_CUDA(launch_fine_bwd_dq_tc(g, qb, kb, vb, dob, lse, delta, map->row_ptr, map->col_idx,
-                                      coarse ? dqc : nullptr, dq, reinterpret_cast<StatusBlock*>(workspace), st));
+      VSA2_CUDA(launch_fine_bwd_dq_tc(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
+                                      reinterpret_cast<StatusBlock*>(workspace), st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
     if (g.flags & VSA2_FLAG_SIMPLE_BWD)
-      VSA2_CUDA(launch_fine_bwd_dkv(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx,
-                                    coarse ? dkc : nullptr, coarse ? dvc : nullptr, dk, dv, st));
+      VSA2_CUDA(launch_fine_bwd_dkv(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
+                                    coarse ? dvc : nullptr, dk, dv, st));
     else
-      VSA2_CUDA(launch_fine_bwd_dkv_tc(g, qb, kb, vb, dob, lse, delta, map->col_ptr, map->row_idx,
-                                       coarse ? dkc : nullptr, coarse ? dvc : nullptr, dk, dv,
-                                       reinterpret_cast<StatusBlock*>(workspace), st));
+      VSA2_CUDA(launch_fine_bwd_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
+                                       coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;
 }

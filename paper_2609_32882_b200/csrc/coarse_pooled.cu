@@ -9,7 +9,7 @@ namespace vsa2 {
 
 // geometry of the pooled problem: tokens = cubes of g, cubes of 4 x 4 x 4 pooled tokens, every block selected
 Geo pooled_geo(const Geo& g) {
-  Geo p = g;
+  Geo p = wide_cube(g) ? narrow_geo(g) : g;      // the kernels' blocks are 64 pooled tokens whatever the caller's cube
   p.T = g.Nt; p.H = g.Nh; p.W = g.Nw;
   p.L = g.N;
   p.Nt = (p.T + p.Bt - 1) / p.Bt; p.Nh = (p.H + p.Bh - 1) / p.Bh; p.Nw = (p.W + p.Bw - 1) / p.Bw;

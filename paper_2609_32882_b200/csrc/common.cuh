@@ -11,7 +11,7 @@ namespace vsa2 {
 
 typedef __nv_bfloat16 bf16;
 
-constexpr int kBlockTokens = 64;   // B: tokens per cube handled by the kernels
+constexpr int kBlockTokens = 64;   // tokens per block handled by the kernels (a 128-token cube runs as two)
 
 // Everything a kernel needs to know about the problem; passed by value.
 struct Geo {
@@ -175,6 +175,17 @@ cudaError_t launch_coarse_fwd_pooled(const Geo& g, const float* qc, const float*
 cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
                                      const float* lse_c, const float* d_oc_hat, float* dqc, float* dkc, float* dvc,
                                      void* workspace, cudaStream_t st);
+
+// cubes of 128 tokens as pairs of 64-token half-cubes (wide_cube.cu); `narrow` is narrow_geo() of the problem
+bool wide_cube(const Geo& g);
+Geo narrow_geo(const Geo& g);
+cudaError_t launch_fold_scores(const Geo& narrow, const float* pr64, float* pr, cudaStream_t st);
+cudaError_t launch_fold_mean(const Geo& narrow, int heads, const float* x64, float* x, cudaStream_t st);
+cudaError_t launch_fold_sum(const Geo& narrow, int heads, const float* x64, float* x, cudaStream_t st);
+cudaError_t launch_expand_rows(const Geo& narrow, int heads, bool by_count, const float* x, float* x64,
+                               cudaStream_t st);
+cudaError_t launch_expand_map(const Geo& narrow, const int* ptr, const int* idx, int* ptr64, int* idx64,
+                              cudaStream_t st);
 
 // tensor-core forward (fine_fwd_tc.cu); `status` heads a workspace of fine_fwd_tc_workspace_bytes()
 size_t fine_fwd_tc_workspace_bytes();

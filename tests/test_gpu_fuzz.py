@@ -11,27 +11,40 @@ from test_gpu_parity import full_parity
 pytestmark = pytest.mark.gpu
 
 
-def random_workload(case: int) -> tuple:
-    rng = np.random.default_rng(1000 + case)
+def random_workload(case: int, wide: bool = False) -> tuple:
+    rng = np.random.default_rng((3000 if wide else 1000) + case)
     grid = (int(rng.integers(3, 10)), int(rng.integers(4, 15)), int(rng.integers(4, 19)))
+    cube = (4, 4, 4)
+    if wide:
+        # cubes of 128 tokens: the last cube along w must reach into its second half (w mod 8 in {0, 5, 6, 7})
+        cube = (4, 4, 8)
+        grid = (grid[0], grid[1], int(rng.choice([w for w in range(5, 34) if w % 8 in (0, 5, 6, 7)])))
     heads_kv = int(rng.integers(1, 4))
     rep = int(rng.choice([1, 1, 2, 4]))
     head_dim = int(rng.choice([64, 128]))
     mode = int(rng.choice([syn.PER_SEQUENCE, syn.PER_QUERY, syn.PER_QUERY_BUDGET]))
-    n_cubes = int(np.prod([-(-g // 4) for g in grid]))
+    n_cubes = int(np.prod([-(-g // c) for g, c in zip(grid, cube)]))
     topk = 0 if mode == syn.PER_QUERY_BUDGET else int(rng.integers(1, max(2, min(n_cubes, 12))))
     batch = int(rng.choice([1, 1, 2]))
-    wl = syn.Workload(f"fuzz_{case}", batch, heads_kv * rep, heads_kv, head_dim, grid, select_mode=mode, topk=topk,
-                      seed=500 + case)
+    wl = syn.Workload(f"fuzz_{case}", batch, heads_kv * rep, heads_kv, head_dim, grid, cube=cube, select_mode=mode,
+                      topk=topk, seed=500 + case)
     out_dtype = vb.F32 if rng.integers(0, 2) else vb.BF16
     return wl, out_dtype
 
 
-@pytest.mark.parametrize("case", range(24))
-def test_random_geometry_full_parity(case):
-    wl, out_dtype = random_workload(case)
+def run_case(wl, out_dtype):
     data = syn.make_inputs(wl)
     nnz_cap = 0
     if wl.select_mode == syn.PER_QUERY_BUDGET:
         nnz_cap = int(np.minimum(data["budgets"], wl.n_cubes).sum(axis=-1).max())
     full_parity(wl, data, out_dtype=out_dtype, nnz_cap=nnz_cap)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_geometry_full_parity(case):
+    run_case(*random_workload(case))
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_random_geometry_cubes_of_128_tokens(case):
+    run_case(*random_workload(case, wide=True))

@@ -1,0 +1,66 @@
+"""GPU parity for cubes of 128 tokens (4 x 4 x 8, router pooling 2 x 2 x 2, G = 16): the CUDA path runs them as pairs
+of 64-token half-cubes; the oracle computes them directly from the definitions."""
+import numpy as np
+import pytest
+
+from paper_2609_32882_b200 import binding as vb
+from paper_2609_32882_b200 import inputs as syn
+from test_gpu_parity import full_parity
+
+pytestmark = pytest.mark.gpu
+
+WIDE = dict(cube=(4, 4, 8), rpool=(2, 2, 2))
+WIDE_SEQ = syn.Workload("wide_per_sequence", 1, 2, 2, 128, (8, 8, 32), select_mode=syn.PER_SEQUENCE, topk=4, seed=61, **WIDE)
+WIDE_RAGGED = syn.Workload("wide_ragged_gqa", 1, 4, 2, 64, (7, 10, 29), select_mode=syn.PER_QUERY, topk=3, seed=62, **WIDE)
+WIDE_BUDGET = syn.Workload("wide_budget", 2, 2, 1, 128, (5, 6, 13), select_mode=syn.PER_QUERY_BUDGET, seed=63, **WIDE)
+WIDE_TILES = syn.Workload("wide_several_tiles", 1, 2, 2, 128, (8, 16, 62), select_mode=syn.PER_SEQUENCE, topk=8, seed=64, **WIDE)
+
+
+def test_wide_cube_per_sequence_full_parity():
+    run = full_parity(WIDE_SEQ, syn.make_inputs(WIDE_SEQ))
+    assert run.attn.sizes.block_tokens == 128 and run.attn.sizes.n_subcubes == 16
+    assert (run.mask.sum(axis=(-1, -2)) == run.N * 4).all()
+
+
+def test_wide_cube_ragged_grid_gqa_full_parity():
+    full_parity(WIDE_RAGGED, syn.make_inputs(WIDE_RAGGED))
+
+
+def test_wide_cube_fp32_outputs():
+    full_parity(WIDE_RAGGED, syn.make_inputs(WIDE_RAGGED), out_dtype=vb.F32, check_route=False)
+
+
+def test_wide_cube_budget_mode_with_empty_rows():
+    wl = WIDE_BUDGET
+    data = syn.make_inputs(wl)
+    N = wl.n_cubes
+    rng = np.random.default_rng(7)
+    data["budgets"] = rng.integers(0, N + 2, size=(wl.batch, wl.heads_q, N), dtype=np.int32)
+    cap = int(np.minimum(data["budgets"], N).sum(axis=-1).max())
+    run = full_parity(wl, data, nnz_cap=cap)
+    assert np.array_equal(run.mask.sum(axis=-1), np.minimum(data["budgets"], N))
+
+
+def test_wide_cube_several_tiles_per_sequence():
+    full_parity(WIDE_TILES, syn.make_inputs(WIDE_TILES))
+
+
+@pytest.mark.parametrize("flags", [vb.FLAG_TF32_COARSE, vb.FLAG_SIMPLE_COARSE | vb.FLAG_SIMPLE_BWD | vb.FLAG_SIMPLE_ROUTER
+                                   | vb.FLAG_EXACT_MAX_FWD])
+def test_wide_cube_alternative_kernels(flags):
+    from oracle import vsa2_oracle as orc
+    from vsa2_testlib import CudaPath, assert_close, oracle_arrays
+    wl = WIDE_RAGGED
+    data = syn.make_inputs(wl)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    a = oracle_arrays(data)
+    run = CudaPath(wl, data, flags=flags)
+    gmask = run.route()
+    O, _ = run.forward()
+    O_ref, _ = orc.forward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale)
+    assert_close("O", O, O_ref, bf16_storage=True)
+    got = run.backward()
+    want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
+    for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
+        assert_close(name, x, y, tol_abs=2e-2 * np.sqrt(2), bf16_storage=name != "dGate")

@@ -60,10 +60,23 @@ def test_topk_is_clamped_and_keep_fraction_is_honoured():
     assert s.topk_eff == 78                                     # 87.5 % block sparsity of 624 cubes
 
 
+def test_query_sizes_for_cubes_of_128_tokens():
+    s = vb.vsa2_query_sizes(vb.make_params(batch=1, heads_q=4, heads_kv=2, head_dim=128, grid=(7, 10, 29),
+                                           cube=(4, 4, 8), topk=5))
+    assert (s.n_cubes, s.n_subcubes, s.block_tokens, s.topk_eff) == (2 * 3 * 4, 16, 128, 5)
+    assert s.nnz_cap == 24 * 5 and s.ptr_elems == 4 * 25 and s.idx_elems == 4 * 24 * 5
+    narrow = vb.vsa2_query_sizes(vb.make_params(batch=1, heads_q=4, heads_kv=2, head_dim=128, grid=(7, 10, 29), topk=10))
+    assert narrow.n_cubes == 2 * s.n_cubes
+    # the wide problem carries the half-cube problem's scratch plus the cube-level link tensors
+    assert s.route_workspace_bytes > 4 * 48 * 48 * 4 and s.bwd_workspace_bytes > narrow.bwd_workspace_bytes // 2
+
+
 @pytest.mark.parametrize("kw,code", [
     (dict(heads_kv=5), vb.ERR_INVALID_ARG),                       # heads_q % heads_kv
     (dict(head_dim=96), vb.ERR_UNSUPPORTED),
-    (dict(cube=(4, 4, 8)), vb.ERR_UNSUPPORTED),                   # B = 128 not built yet
+    (dict(cube=(4, 8, 8)), vb.ERR_UNSUPPORTED),                   # 256 tokens per cube
+    (dict(cube=(4, 4, 8), rpool=(2, 2, 8)), vb.ERR_UNSUPPORTED),  # router pooling straddles the two half-cubes
+    (dict(cube=(4, 4, 8), grid=(8, 16, 20)), vb.ERR_UNSUPPORTED), # last cube's second half lies outside the grid
     (dict(rpool=(3, 2, 2)), vb.ERR_INVALID_ARG),                  # must divide the cube
     (dict(select_mode=7), vb.ERR_INVALID_ARG),
     (dict(topk=0, keep_fraction=0.0), vb.ERR_INVALID_ARG),
