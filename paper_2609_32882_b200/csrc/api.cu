@@ -58,8 +58,6 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   g->Gt = g->Bt / g->Rt; g->Gh = g->Bh / g->Rh; g->Gw = g->Bw / g->Rw;
   g->G = g->Gt * g->Gh * g->Gw;
   if (128 % (wide ? g->G / 2 : g->G)) return VSA2_ERR_UNSUPPORTED;
-  // the second half of the last cube along w must hold at least one grid column (no empty half-cubes)
-  if (wide && (2 * g->Nw - 1) * (g->Bw / 2) >= g->W) return VSA2_ERR_UNSUPPORTED;
   int K = p->topk;
   if (K == 0) {
     if (!(p->keep_fraction > 0.f) || p->keep_fraction > 1.f) {

@@ -90,11 +90,11 @@ __device__ __forceinline__ unsigned long long cube_valid_mask(const Geo& g, int 
   return m;
 }
 
-// number of valid tokens of cube n
+// number of valid tokens of cube n (0 only for the empty trailing half-cubes of a 128-token-cube problem)
 __device__ __forceinline__ int cube_count(const Geo& g, int n) {
   int nt, nh, nw;
   cube_coords(g, n, nt, nh, nw);
-  int ct = min(g.Bt, g.T - nt * g.Bt), ch = min(g.Bh, g.H - nh * g.Bh), cw = min(g.Bw, g.W - nw * g.Bw);
+  int ct = min(g.Bt, g.T - nt * g.Bt), ch = min(g.Bh, g.H - nh * g.Bh), cw = max(0, min(g.Bw, g.W - nw * g.Bw));
   return ct * ch * cw;
 }
 

@@ -327,7 +327,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             VSA2_WAIT(&misc->s_full[s], par);
             tc::tc_fence_after();
             // (the K slot of the tile, and with it its edge flags, stays until the tile's dQ^T product is done)
-            const bool valid = !dup && cpos.valid(misc->edge[tg % kRingA][blk]);
+            const bool valid = !dup && cpos.valid(misc->edge[tg % kRingA][blk], g);
             tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
             tc::tmem_ld_wait();
             tc::tc_fence_before();

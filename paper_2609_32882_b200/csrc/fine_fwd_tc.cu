@@ -316,7 +316,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         if (wg == first_wg) {
           // reference exponent of every query column = exact column maximum of the first tile
           const uint32_t buf = tg % kFwdSBufs;
-          const bool valid = !((blk == 1) && k < 2) && cpos.valid(edge[cols[(blk == 1 && k > 1) ? 1 : 0]]);
+          const bool valid = !((blk == 1) && k < 2) && cpos.valid(edge[cols[(blk == 1 && k > 1) ? 1 : 0]], g);
           VSA2_WAIT(&misc->s_full[buf], (tg / kFwdSBufs) & 1);
           tc::tc_fence_after();
           uint32_t s0[32], s1[32];
@@ -350,7 +350,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int t = t_own; t < nt; t += 2) {
           const uint32_t tgt = tg0 + t, buf = tgt % kFwdSBufs;
           const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          const bool valid = !dup && cpos.valid(edge[j_next]);
+          const bool valid = !dup && cpos.valid(edge[j_next], g);
           if (t + 2 < nt) j_next = cols[(blk == 1 && 2 * t + 5 < k) ? 2 * t + 5 : 2 * t + 4];   // next own tile, fetched early
           const bool all_valid = __all_sync(0xffffffffu, valid);
           VSA2_WAIT(&misc->s_full[buf], (tgt / kFwdSBufs) & 1);

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(256) pool_kernel(const bf16* __restrict__ x, i
       float s = 0.f;
 #pragma unroll 8
       for (int p = 0; p < kBlockTokens; ++p) s += tile[p][d];
-      xc[(bh * g.N + n) * D + d] = s / cnt;
+      xc[(bh * g.N + n) * D + d] = cnt > 0.f ? s / cnt : 0.f;
     }
   }
   if (xr != nullptr) {

@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(256) router_kernel(const bf16* __restrict__ qr
           const float* srow = S + (ci * g.G + a) * SM::LDS + cj * g.G;
           for (int c = 0; c < g.G; ++c) acc += srow[c];
         }
-        pr[((size_t)(b * g.Hq + hq) * g.N + qi) * g.N + kj] = acc / ((float)gi * (float)g.G);
+        pr[((size_t)(b * g.Hq + hq) * g.N + qi) * g.N + kj] = gi > 0 ? acc / ((float)gi * (float)g.G) : 0.f;
       }
     }
   }

@@ -67,11 +67,13 @@ __device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_sl
 }
 
 // Which cubes are cut by the grid boundary: bit 0 / 1 / 2 = last cube along t / h / w with a partial extent.
+// In the half-cube grid of a 128-token-cube problem the last column of blocks along w may lie outside the grid
+// altogether (extent <= 0, still bit 2); the column before it can then be the partial one (bit 3).
 __device__ __forceinline__ unsigned cube_edge_flags_at(const Geo& g, int nt, int nh, int nw) {
   unsigned f = 0;
   if (nt == g.Nt - 1 && g.T % g.Bt) f |= 1u;
   if (nh == g.Nh - 1 && g.H % g.Bh) f |= 2u;
-  if (nw == g.Nw - 1 && g.W % g.Bw) f |= 4u;
+  if ((nw + 1) * g.Bw > g.W) f |= (nw == g.Nw - 1) ? 4u : 8u;
   return f;
 }
 __device__ __forceinline__ unsigned cube_edge_flags(const Geo& g, int n) {
@@ -92,8 +94,8 @@ struct CubePos {
     lh = g.H - (g.Nh - 1) * g.Bh;
     lw = g.W - (g.Nw - 1) * g.Bw;
   }
-  __device__ __forceinline__ bool valid(unsigned f) const {
-    return (!(f & 1u) || bt < lt) && (!(f & 2u) || bh < lh) && (!(f & 4u) || bw < lw);
+  __device__ __forceinline__ bool valid(unsigned f, const Geo& g) const {
+    return (!(f & 1u) || bt < lt) && (!(f & 2u) || bh < lh) && (!(f & 4u) || bw < lw) && (!(f & 8u) || bw < lw + g.Bw);
   }
 };
 

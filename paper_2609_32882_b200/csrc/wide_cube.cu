@@ -1,7 +1,10 @@
 // Cubes of 128 tokens (the 4 x 4 x 8 cube with 2 x 2 x 2 router pooling, G = 16) on top of the 64-token kernels.
 //
 // A cube of 128 tokens whose w extent is even is two 64-token half-cubes that are neighbours along w, and in the
-// half-cube grid (same Nt, Nh; twice Nw) cube c is exactly the half-cubes 2c and 2c+1.  Every quantity of the
+// half-cube grid (same Nt, Nh; twice Nw) cube c is exactly the half-cubes 2c and 2c+1.  When the grid's last cube
+// along w reaches no further than its first half, its second half-cube is EMPTY: it stays in the half-cube grid so
+// that the 2c, 2c+1 numbering holds, has no valid token or router sub-cube, contributes zero weight to every fold,
+// and the fine kernels treat it like the padding of any ragged cube (keys masked, nothing stored).  Every quantity of the
 // method at cube level follows from the half-cube quantities without touching the tokens again:
 //   * router (Eq. 5-7): the 2 x 2 x 2 sub-cubes of a cube are the sub-cubes of its two halves, so the router
 //     softmax over all sub-cube keys is the same matrix, and the cube-level score is the mean over a 16 x 16
@@ -62,7 +65,9 @@ __global__ void __launch_bounds__(256) fold_mean_kernel(Geo n, const float* __re
     const int d = (int)(e % D);
     const int c = (int)(row % (n.N / 2));
     const float c0 = (float)cube_count(n, 2 * c), c1 = (float)cube_count(n, 2 * c + 1);
-    x[e] = (x64[(2 * row) * D + d] * c0 + x64[(2 * row + 1) * D + d] * c1) / (c0 + c1);
+    float v = x64[(2 * row) * D + d] * c0;
+    if (c1 > 0.f) v += x64[(2 * row + 1) * D + d] * c1;       // an empty second half (beyond the grid) has no mean
+    x[e] = v / (c0 + c1);
   }
 }
 

@@ -13,6 +13,8 @@ WIDE = dict(cube=(4, 4, 8), rpool=(2, 2, 2))
 WIDE_SEQ = syn.Workload("wide_per_sequence", 1, 2, 2, 128, (8, 8, 32), select_mode=syn.PER_SEQUENCE, topk=4, seed=61, **WIDE)
 WIDE_RAGGED = syn.Workload("wide_ragged_gqa", 1, 4, 2, 64, (7, 10, 29), select_mode=syn.PER_QUERY, topk=3, seed=62, **WIDE)
 WIDE_BUDGET = syn.Workload("wide_budget", 2, 2, 1, 128, (5, 6, 13), select_mode=syn.PER_QUERY_BUDGET, seed=63, **WIDE)
+WIDE_EMPTY_HALF = syn.Workload("wide_empty_second_half", 1, 4, 2, 128, (7, 10, 28), select_mode=syn.PER_SEQUENCE, topk=5, seed=65, **WIDE)
+WIDE_ONE_COLUMN = syn.Workload("wide_one_column_over", 2, 2, 2, 64, (5, 6, 9), select_mode=syn.PER_QUERY, topk=2, seed=66, **WIDE)
 WIDE_TILES = syn.Workload("wide_several_tiles", 1, 2, 2, 128, (8, 16, 62), select_mode=syn.PER_SEQUENCE, topk=8, seed=64, **WIDE)
 
 
@@ -24,6 +26,13 @@ def test_wide_cube_per_sequence_full_parity():
 
 def test_wide_cube_ragged_grid_gqa_full_parity():
     full_parity(WIDE_RAGGED, syn.make_inputs(WIDE_RAGGED))
+
+
+@pytest.mark.parametrize("wl", [WIDE_EMPTY_HALF, WIDE_ONE_COLUMN], ids=lambda w: w.name)
+def test_wide_cube_whose_last_second_half_lies_outside_the_grid(wl):
+    """w = 28 or 9: the last cube along w holds columns of its first half only (second half-cube empty)."""
+    full_parity(wl, syn.make_inputs(wl))
+    full_parity(wl, syn.make_inputs(wl), out_dtype=vb.F32, check_route=False)
 
 
 def test_wide_cube_fp32_outputs():
@@ -47,10 +56,10 @@ def test_wide_cube_several_tiles_per_sequence():
 
 @pytest.mark.parametrize("flags", [vb.FLAG_TF32_COARSE, vb.FLAG_SIMPLE_COARSE | vb.FLAG_SIMPLE_BWD | vb.FLAG_SIMPLE_ROUTER
                                    | vb.FLAG_EXACT_MAX_FWD])
-def test_wide_cube_alternative_kernels(flags):
+@pytest.mark.parametrize("wl", [WIDE_RAGGED, WIDE_EMPTY_HALF], ids=lambda w: w.name)
+def test_wide_cube_alternative_kernels(flags, wl):
     from oracle import vsa2_oracle as orc
     from vsa2_testlib import CudaPath, assert_close, oracle_arrays
-    wl = WIDE_RAGGED
     data = syn.make_inputs(wl)
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
     scale = 1.0 / np.sqrt(wl.head_dim)

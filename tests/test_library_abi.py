@@ -76,7 +76,6 @@ def test_query_sizes_for_cubes_of_128_tokens():
     (dict(head_dim=96), vb.ERR_UNSUPPORTED),
     (dict(cube=(4, 8, 8)), vb.ERR_UNSUPPORTED),                   # 256 tokens per cube
     (dict(cube=(4, 4, 8), rpool=(2, 2, 8)), vb.ERR_UNSUPPORTED),  # router pooling straddles the two half-cubes
-    (dict(cube=(4, 4, 8), grid=(8, 16, 20)), vb.ERR_UNSUPPORTED), # last cube's second half lies outside the grid
     (dict(rpool=(3, 2, 2)), vb.ERR_INVALID_ARG),                  # must divide the cube
     (dict(select_mode=7), vb.ERR_INVALID_ARG),
     (dict(topk=0, keep_fraction=0.0), vb.ERR_INVALID_ARG),
