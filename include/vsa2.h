@@ -77,7 +77,11 @@ enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward w
 typedef struct vsa2_params {
   int32_t batch, heads_q, heads_kv, head_dim;  /* head_dim in {64, 128}; heads_q % heads_kv == 0, ratio <= 16 */
   int32_t grid_t, grid_h, grid_w;              /* valid latent grid */
-  int32_t cube_t, cube_h, cube_w;              /* cube (block) shape, product must be 64 */
+  int32_t cube_t, cube_h, cube_w;              /* cube (block) shape: 64 tokens (e.g. 4,4,4), or 128 tokens with cube_w even
+                                                  and rpool_w dividing cube_w/2 (the paper's 4,4,8 with R = 2,2,2: G = 16);
+                                                  N, K, budgets and the block map are then in cubes of 128 tokens, and the
+                                                  library computes on the cube's two 64-token halves along w
+                                                  (Sec. 2.2 "Permutation", Eq. 5-7, Eq. 12) */
   int32_t rpool_t, rpool_h, rpool_w;           /* router pooling R, each divides the cube dimension */
   int32_t select_mode;                         /* VSA2_PER_* */
   int32_t topk;                                /* K in blocks (clamped to N); if 0, K = max(1, round(keep_fraction*N)) */

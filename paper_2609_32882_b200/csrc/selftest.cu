@@ -119,6 +119,7 @@ extern "C" int vsa2_selftest_umma(const vsa2_params* p, const void* q, const voi
   vsa2_sizes sz;
   int rc = vsa2_query_sizes(p, &sz);
   if (rc != VSA2_OK) return rc;
+  if (sz.block_tokens != kBlockTokens) return VSA2_ERR_UNSUPPORTED;      // the self-test addresses 64-token tiles
   if (!q || !k || !v || !p_t || !s_t_out || !o_t_out || !k_tile_dump || !status) return VSA2_ERR_INVALID_ARG;
   Geo g = {};
   g.batch = p->batch; g.Hq = p->heads_q; g.Hkv = p->heads_kv; g.rep = g.Hq / g.Hkv; g.D = p->head_dim;
