@@ -119,3 +119,43 @@ def test_config4_gqa_sparsity_levels():
         sampled_attention_parity(w, data, run, gmask, q_heads=(13,), rows=(640,), kv_groups=(3,), kv_cubes=(900,))
         del run
         torch.cuda.empty_cache()
+
+
+WIDE = dict(cube=(4, 4, 8), rpool=(2, 2, 2))
+
+
+def test_config3_720p_cubes_of_128_tokens():
+    """The 720p workload with the paper's 4 x 4 x 8 cube (N = 720 cubes of 128 tokens, G = 16), per-sequence top-64."""
+    base, data = inputs_for(3)
+    wl = base.replace(**WIDE)
+    run = CudaPath(wl, data)
+    gmask = run.route()
+    N = wl.n_cubes
+    assert N == 720 and run.attn.sizes.block_tokens == 128
+    assert (gmask.sum(axis=(-1, -2)) == N * 64).all()
+    for hq in (0, 39):
+        om, P = oracle_route_head(wl, data, 0, hq, syn.PER_SEQUENCE, 64)
+        check_routing(gmask[0, hq], om, P, syn.PER_SEQUENCE)
+    run.forward()
+    run.backward()
+    heavy = int(np.argmax(gmask[0, 17].sum(axis=0)))
+    sampled_attention_parity(wl, data, run, gmask, q_heads=(0, 39), rows=(3, 350, N - 1),
+                             kv_groups=(17,), kv_cubes=(heavy, N - 1))
+
+
+def test_config2_480p_gqa_cubes_of_128_tokens_with_empty_half_cubes():
+    """480p: w = 52 = 6 * 8 + 4, so the last cube along w holds its first half only; t and h are ragged too; GQA 4:1."""
+    base, data = inputs_for(2)
+    wl = base.replace(topk=42, **WIDE)
+    run = CudaPath(wl, data)
+    gmask = run.route()
+    N = wl.n_cubes
+    assert N == 6 * 8 * 7 and (gmask.sum(axis=-1) == 42).all()
+    for hq in (0, 11):
+        om, P = oracle_route_head(wl, data, 0, hq, wl.select_mode, wl.topk)
+        check_routing(gmask[0, hq], om, P, wl.select_mode)
+    run.forward()
+    run.backward()
+    sampled_attention_parity(wl, data, run, gmask, q_heads=(1, 10), rows=(0, 6, 160, N - 1),
+                             kv_groups=(0, 2), kv_cubes=(6, N - 1))         # cubes 6 and N-1 end beyond the grid along w
+    assert torch.isfinite(run.o.float()).all() and torch.isfinite(run.dk.float()).all() and torch.isfinite(run.dq.float()).all()
