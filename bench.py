@@ -268,47 +268,67 @@ def run_ours(args):
         attn.backward(dev["q"], dev["k"], dev["v"], dev["gate"], o, lse, dev["do"], dq=dq, dk=dk, dv=dv, dgate=dgate)
 
     # End to end: every step copies its inputs from pinned host memory and its results back, inside the timed region.
-    # As a training loop would, the copies run on side streams and overlap the kernels: the inputs of step n + 1 are
-    # prefetched while step n computes and the results of step n drain while step n + 1 computes (two device buffer sets).
-    in_sets = [dev, {k: torch.empty_like(v) for k, v in dev.items()}]
-    out_sets = [dict(o=o, lse=lse, dq=dq, dk=dk, dv=dv, dgate=dgate),
-                dict(o=torch.empty_like(o), lse=torch.empty_like(lse), dq=torch.empty_like(dq), dk=torch.empty_like(dk),
-                     dv=torch.empty_like(dv), dgate=torch.empty_like(dgate))]
+    # As a training loop would, the copies run on side streams and overlap the kernels.  Heads are independent, so a
+    # step is cut into head chunks (units) that flow through a two-deep pipeline: the inputs of unit i + 1 load and the
+    # results of unit i - 1 drain while unit i computes; inside a unit the router starts as soon as Q and K have
+    # arrived, the forward when V has, the backward when dO has, and O leaves while the backward runs.
+    chunks = next(c for c in range(args.e2e_chunks, 0, -1) if wl.heads_kv % c == 0) if wl.batch == 1 else 1
+    hq_c, hk_c = wl.heads_q // chunks, wl.heads_kv // chunks
+    attn_e = attn if chunks == 1 else vb.Vsa2Attention(
+        vb.params_from_workload(wl.replace(heads_q=hq_c, heads_kv=hk_c), nnz_cap=nnz_cap))
+    heads_of = {"q": hq_c, "do": hq_c, "gate": hq_c, "k": hk_c, "v": hk_c, "o": hq_c, "dq": hq_c, "dk": hk_c, "dv": hk_c}
+
+    def part(t, name, c):
+        return t if chunks == 1 else t[:, c * heads_of[name]:(c + 1) * heads_of[name]]
+
+    def like(t, name, dtype=None):
+        return torch.empty_like(part(t, name, 0), dtype=dtype or t.dtype)
+
+    in_sets = [{k: like(dev[k], k) for k in dev} for _ in range(2)]
+    out_sets = [dict(o=like(o, "o"), lse=like(lse, "gate"), dq=like(dq, "dq"), dk=like(dk, "dk"), dv=like(dv, "dv"),
+                     dgate=like(dgate, "gate")) for _ in range(2)]
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
 
     def run_e2e(n_steps):
-        ev_in = [torch.cuda.Event() for _ in range(n_steps)]
-        ev_comp = [torch.cuda.Event() for _ in range(n_steps)]
-        ev_out = [torch.cuda.Event() for _ in range(n_steps)]
+        units = n_steps * chunks
+        ev = {k: [torch.cuda.Event() for _ in range(units)] for k in ("qk", "v", "do", "fwd", "comp", "out")}
 
-        def h2d(n):
+        def h2d(i):
+            c, d = i % chunks, in_sets[i % 2]
             with torch.cuda.stream(s_in):
-                if n >= 2:
-                    s_in.wait_event(ev_comp[n - 2])          # the buffer set is free once step n - 2 has computed
-                for k in ("q", "k", "v", "do", "gate"):
-                    in_sets[n % 2][k].copy_(host[k], non_blocking=True)
-                ev_in[n].record(s_in)
+                if i >= 2:
+                    s_in.wait_event(ev["comp"][i - 2])       # the buffer set is free once unit i - 2 has computed
+                for names, mark in ((("q", "k"), "qk"), (("gate", "v"), "v"), (("do",), "do")):
+                    for k in names:
+                        d[k].copy_(part(host[k], k, c), non_blocking=True)
+                    ev[mark][i].record(s_in)
 
         h2d(0)
-        for n in range(n_steps):
-            if n + 1 < n_steps:
-                h2d(n + 1)
-            d, r = in_sets[n % 2], out_sets[n % 2]
-            stream.wait_event(ev_in[n])
-            if n >= 2:
-                stream.wait_event(ev_out[n - 2])             # the result set has been read back
-            attn.route(d["q"], d["k"], budgets)
-            attn.forward(d["q"], d["k"], d["v"], d["gate"], o=r["o"], lse=r["lse"])
-            if not args.forward_only:
-                attn.backward(d["q"], d["k"], d["v"], d["gate"], r["o"], r["lse"], d["do"], dq=r["dq"], dk=r["dk"],
-                              dv=r["dv"], dgate=r["dgate"])
-            ev_comp[n].record(stream)
+        for i in range(units):
+            if i + 1 < units:
+                h2d(i + 1)
+            c, d, r = i % chunks, in_sets[i % 2], out_sets[i % 2]
+            stream.wait_event(ev["qk"][i])
+            if i >= 2:
+                stream.wait_event(ev["out"][i - 2])          # the result set has been read back
+            attn_e.route(d["q"], d["k"], None if budgets is None else part(budgets, "q", c))
+            stream.wait_event(ev["v"][i])
+            attn_e.forward(d["q"], d["k"], d["v"], d["gate"], o=r["o"], lse=r["lse"])
+            ev["fwd"][i].record(stream)
             with torch.cuda.stream(s_out):
-                s_out.wait_event(ev_comp[n])
-                for k in ("o", "dq", "dk", "dv"):
-                    host_out[k].copy_(r[k], non_blocking=True)
-                ev_out[n].record(s_out)
-        stream.wait_event(ev_out[n_steps - 1])               # the timed region ends when the last result is on the host
+                s_out.wait_event(ev["fwd"][i])
+                part(host_out["o"], "o", c).copy_(r["o"], non_blocking=True)
+            if not args.forward_only:
+                stream.wait_event(ev["do"][i])
+                attn_e.backward(d["q"], d["k"], d["v"], d["gate"], r["o"], r["lse"], d["do"], dq=r["dq"], dk=r["dk"],
+                                dv=r["dv"], dgate=r["dgate"])
+            ev["comp"][i].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev["comp"][i])
+                for k in (() if args.forward_only else ("dq", "dk", "dv")):
+                    part(host_out[k], k, c).copy_(r[k], non_blocking=True)
+                ev["out"][i].record(s_out)
+        stream.wait_event(ev["out"][units - 1])              # the timed region ends when the last result is on the host
 
     def barrier():
         if world > 1:
@@ -394,7 +414,7 @@ def run_ours(args):
                 "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant]}
     fine_fwd_tf = flops["fine_fwd"] / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
     bytes_in = sum(host[k].numel() * host[k].element_size() for k in host)
-    bytes_out = sum(t.numel() * t.element_size() for t in host_out.values())
+    bytes_out = sum(t.numel() * t.element_size() for k, t in host_out.items() if k == "o" or not args.forward_only)
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -423,7 +443,8 @@ def run_ours(args):
         "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_step_e2e, "h2d_bytes_per_step": bytes_in,
                 "d2h_bytes_per_step": bytes_out,
                 "how": "pinned host -> device copies of Q,K,V,dO,gate and device -> host copies of O,dQ,dK,dV of every step inside "
-                       "the timed region, on side streams: step n+1's inputs load and step n-1's results drain while step n computes"},
+                       f"the timed region, on side streams, each step cut into {chunks} head chunk(s): the next chunk's inputs load "
+                       "and the previous chunk's results drain while a chunk computes"},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "cpu_baseline": cpu_baseline,
@@ -447,6 +468,7 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="index into the five baseline configurations (3 = 720p top-64)")
     ap.add_argument("--ref-rows", type=int, default=1440, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-chunks", type=int, default=8, help="upper limit of head chunks per step in the end-to-end pipeline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     ap.add_argument("--topk", type=int, default=0, help="override the TopK of the configuration (context rows: top-128)")
     ap.add_argument("--forward-only", action="store_true", help="route + forward only (context rows: inference)")
