@@ -250,7 +250,7 @@ def run_ours(args):
     nnz_cap = 0
     if budgets is not None:
         nnz_cap = int(np.minimum(data["budgets"], wl.n_cubes).sum(axis=-1).max())
-    p = vb.params_from_workload(wl, nnz_cap=nnz_cap)
+    p = vb.params_from_workload(wl, nnz_cap=nnz_cap, flags=args.flags)
     attn = vb.Vsa2Attention(p)
     odt = attn.out_torch_dtype
     o = torch.empty_like(dev["q"], dtype=odt)
@@ -275,7 +275,7 @@ def run_ours(args):
     chunks = next(c for c in range(args.e2e_chunks, 0, -1) if wl.heads_kv % c == 0) if wl.batch == 1 else 1
     hq_c, hk_c = wl.heads_q // chunks, wl.heads_kv // chunks
     attn_e = attn if chunks == 1 else vb.Vsa2Attention(
-        vb.params_from_workload(wl.replace(heads_q=hq_c, heads_kv=hk_c), nnz_cap=nnz_cap))
+        vb.params_from_workload(wl.replace(heads_q=hq_c, heads_kv=hk_c), nnz_cap=nnz_cap, flags=args.flags))
     heads_of = {"q": hq_c, "do": hq_c, "gate": hq_c, "k": hk_c, "v": hk_c, "o": hq_c, "dq": hq_c, "dk": hk_c, "dv": hk_c}
 
     def part(t, name, c):
@@ -468,6 +468,7 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="index into the five baseline configurations (3 = 720p top-64)")
     ap.add_argument("--ref-rows", type=int, default=1440, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="VSA2_FLAG_* bits passed to the library (kernel variants)")
     ap.add_argument("--e2e-chunks", type=int, default=8, help="upper limit of head chunks per step in the end-to-end pipeline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")
     ap.add_argument("--topk", type=int, default=0, help="override the TopK of the configuration (context rows: top-128)")

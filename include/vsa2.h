@@ -69,6 +69,8 @@ enum { VSA2_FLAG_TF32_COARSE = 32 };  /* validation aid: coarse backward with th
 enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
                                          (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
+enum { VSA2_FLAG_HALF_CUBE_FWD = 128 };/* 128-token cubes only: fine forward with the 64-query kernel on the two half-cubes
+                                         separately instead of the 128-query kernel (validation aid, same results) */
 enum { VSA2_FLAG_SIMPLE_COARSE = 16 };/* validation aid: coarse branch (forward and backward) with the fp32 SIMT kernels
                                          instead of the TF32 tensor-core ones */
 enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */

@@ -403,6 +403,9 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     ProfScope ps(VSA2_KERNEL_FINE_FWD, st, (g.flags & VSA2_FLAG_EXACT_MAX_FWD) ? 1 : 2);
     if (g.flags & VSA2_FLAG_EXACT_MAX_FWD)
       VSA2_CUDA(launch_fine_fwd(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse, st));
+    else if (wide && !(g.flags & VSA2_FLAG_HALF_CUBE_FWD))
+      VSA2_CUDA(launch_fine_fwd_wide_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
+                                        reinterpret_cast<StatusBlock*>(workspace), st));
     else
       VSA2_CUDA(launch_fine_fwd_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                    reinterpret_cast<StatusBlock*>(workspace), st));

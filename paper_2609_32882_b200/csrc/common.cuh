@@ -193,6 +193,12 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
                                const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                float* lse, StatusBlock* status, cudaStream_t st);
 
+// tensor-core forward for 128-token cubes (fine_fwd_wide_tc.cu): both halves of a query cube on the same operand tiles;
+// `g`, the map and oc_hat are those of the half-cube problem, the workspace is the one of launch_fine_fwd_tc
+cudaError_t launch_fine_fwd_wide_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                                    const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                                    float* lse, StatusBlock* status, cudaStream_t st);
+
 // tensor-core backward passes (fine_bwd_tc.cu)
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                   const float* lse, const float* delta, const int* row_ptr, const int* col_idx,

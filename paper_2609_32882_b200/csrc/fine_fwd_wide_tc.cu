@@ -1,0 +1,551 @@
+// Fine branch forward (paper Eq. 12) + gated merge (Eq. 14) for cubes of 128 tokens, on the Blackwell tensor cores.
+//
+// A query cube of 128 tokens is two 64-token half-cubes that keep the same KV cubes, so both halves ride on the same
+// operand tiles: the products of fine_fwd_tc.cu are taken with N = 128 query columns,
+//     S^T [128 kv, 128 q] = K_pair [128, D] * Q_pair^T        (M = 128 keys,   N = 128 queries, K = D)
+//     O^T [D,      128 q] += V_pair^T [D, 128] * P^T          (M = D channels, N = 128 queries, K = 128 keys)
+// where K_pair / V_pair are the two halves of ONE key cube and Q_pair the two halves of the query cube.  Per FLOP this
+// halves the TMA traffic into shared memory and cuts the operand fetches of the MMAs by a third against the N = 64
+// kernel, which is bound by exactly that traffic.
+//
+// The kernel works on the half-cube problem (geometry, expanded block map, per-half coarse rows) that the library
+// builds for 128-token cubes: row 2c of the expanded map lists the half-cubes (2j, 2j+1, ...) of query cube c.
+//
+// Roles (512 threads): warp 0 = TMA producer of the K pairs and the Q pair (lane 0 is also the CTA's scheduler), warp 1
+// = TMA producer of the V pairs, warp 2 = issuer of S^T, warp 4 = issuer of O^T, warpgroups 2 and 3 = softmax +
+// epilogue: warpgroup w owns query half w (columns 64w .. 64w+63) of EVERY tile, so each keeps its own reference
+// exponents, row sums and output rows and the two only meet at the operand barriers.  Softmax as in fine_fwd_tc.cu:
+// fixed reference exponent per query column (exact column maximum of the first tile), row sums checked at the end, a
+// half-cube whose sums left the safe range goes to the exact-maximum kernel.  Every wait is bounded.
+#include "tc_attn.cuh"
+
+namespace vsa2 {
+
+constexpr int kFwwThreads = 512;
+constexpr int kFwwKSlots = 2;
+constexpr int kFwwVSlots = 2;
+constexpr int kFwwSBufs = 2;          // S^T buffers of 128 columns
+constexpr int kFwwRescueCap = 16384;  // must match the list the N = 64 launcher sizes (fine_fwd_tc_workspace_bytes)
+constexpr int kFwwMaxCubes = 12288;
+
+template <int D>
+struct FwdWide {
+  static constexpr int DH = D / 64;
+  static constexpr uint32_t SLAB = kSlab;
+  static constexpr uint32_t SLOT = 2 * DH * SLAB;    // a K, V or Q pair: [channel half][block A | block B]
+  static constexpr uint32_t PBYTES = 128 * 128;      // P^T of one query half: 128 key rows x 64 queries bf16
+  static constexpr uint32_t OFF_Q = (kFwwKSlots + kFwwVSlots) * SLOT;
+  static constexpr uint32_t OFF_P = OFF_Q + SLOT;
+  static constexpr uint32_t OFF_MISC = OFF_P + 2 * PBYTES;
+  static constexpr uint32_t MISC_BYTES = 6144;
+  static size_t smem_bytes(int n_half_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_half_cubes + 15) / 16 * 16 + 1024; }
+};
+
+struct FwdWideMisc {
+  uint64_t q_full, q_empty, o_full, o_empty;
+  uint64_t k_full[kFwwKSlots], k_empty[kFwwKSlots];
+  uint64_t v_full[kFwwVSlots], v_empty[kFwwVSlots];
+  uint64_t s_full[kFwwSBufs], s_free[kFwwSBufs];
+  uint64_t p_ready, p_free;
+  ItemQueue items;
+  uint64_t wg_sync[2];             // group barrier of one softmax warpgroup (128 threads)
+  uint32_t tmem_base;
+  int abort_flag;
+  int rescue_flag[2];
+  alignas(16) float m_ref[2][64];  // per query half and column: reference exponent (log2 units)
+  alignas(16) float l_inv[2][64];
+  alignas(16) float red[8][64];    // per-warp partial column reductions (warps 4w .. 4w+3 belong to query half w)
+  int tok[2][2][64];               // [item parity][query half][position]: raster token (-1 = padding)
+  float gate[2][2][64];
+};
+static_assert(sizeof(FwdWideMisc) <= 6144, "misc region too small");
+
+struct FwdWideArgs {
+  int* item_counter;    // global, zero before the launch
+  const float* gate;
+  const int* row_ptr;   // expanded map (half-cube level)
+  const int* col_idx;
+  const float* oc_hat;  // per half-cube
+  void* o;
+  bf16* o_res;
+  float* lse;
+  StatusBlock* status;
+  int* rescue_count;
+  int* rescue_items;
+};
+
+// acc[128, 128] = A_pair[128, D] * B_pair[128, D]^T, both operands in the [channel half][block A | block B] layout
+template <int D>
+__device__ __forceinline__ void mma_pair_pair_kmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_slot) {
+  constexpr uint32_t idesc = tc::idesc_bf16(128, 128, false, false);
+  const uint64_t da = tc::smem_desc_sw128(a_slot, 16, 1024), db = tc::smem_desc_sw128(b_slot, 16, 1024);
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    const uint64_t off = (uint64_t)(((ks / 4) * 2 * kSlab + (ks % 4) * 32) >> 4);
+    tc::mma_ss(tm_acc, da + off, db + off, idesc, ks > 0);
+  }
+}
+
+// acc[D, 128] (+)= A_pair^T[D, 128] * B[128, 128]: A_pair a slot (rows = the 128 keys), B two 128-row swizzled tiles of
+// 64 query columns each, `b_stride` bytes apart
+template <int D>
+__device__ __forceinline__ void mma_pairT_wide_mnmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, uint32_t b_stride,
+                                                       bool accumulate_first) {
+  constexpr uint32_t idesc = tc::idesc_bf16(128, 128, true, true);
+  constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;
+  const uint64_t da = tc::smem_desc_sw128(a_slot, lbo, 1024), db = tc::smem_desc_sw128(b_tile, b_stride, 1024);
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const uint64_t oa = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 2048) >> 4);
+    const uint64_t ob = (uint64_t)((ks * 2048) >> 4);
+    tc::mma_ss(tm_acc, da + oa, db + ob, idesc, accumulate_first || (ks > 0));
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kFwwThreads, 1)
+fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, Geo g, FwdWideArgs a) {
+  using C = FwdWide<D>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* q_tile = smem + C::OFF_Q;
+  unsigned char* p_tile = smem + C::OFF_P;
+  FwdWideMisc* misc = reinterpret_cast<FwdWideMisc*>(smem + C::OFF_MISC);
+  unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;      // edge flags of every half-cube
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_cubes = g.N / 2;                                   // g is the half-cube geometry
+  const int total_items = g.batch * g.Hq * n_cubes;
+  const float c2 = g.scale * 1.4426950408889634f;
+
+  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
+  if (tid == 0) {
+    misc->abort_flag = 0;
+    tc::mbar_init(&misc->q_full, 1);
+    tc::mbar_init(&misc->q_empty, 1);
+    tc::mbar_init(&misc->o_full, 1);
+    tc::mbar_init(&misc->o_empty, 256);
+    for (int s = 0; s < kFwwKSlots; ++s) {
+      tc::mbar_init(&misc->k_full[s], 1);
+      tc::mbar_init(&misc->k_empty[s], 1);
+    }
+    for (int s = 0; s < kFwwVSlots; ++s) {
+      tc::mbar_init(&misc->v_full[s], 1);
+      tc::mbar_init(&misc->v_empty[s], 1);
+    }
+    for (int s = 0; s < kFwwSBufs; ++s) {
+      tc::mbar_init(&misc->s_full[s], 1);
+      tc::mbar_init(&misc->s_free[s], 256);
+    }
+    tc::mbar_init(&misc->p_ready, 256);
+    tc::mbar_init(&misc->p_free, 1);
+    tc::mbar_init(&misc->wg_sync[0], 128);
+    tc::mbar_init(&misc->wg_sync[1], 128);
+    item_queue_init(&misc->items, 2 + 2 + 256);     // lane 0 of the producers, two issuers, the softmax threads
+    tc::fence_barrier_init();
+    tc::prefetch_tmap(&tm_q);
+    tc::prefetch_tmap(&tm_k);
+    tc::prefetch_tmap(&tm_v);
+  }
+  if (warp == 2) {
+    tc::tmem_alloc(&misc->tmem_base, 512);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_base;
+  // tensor-memory columns: S^T buffers at 0 and 128; O^T at 256 .. 383
+
+  if (warp < 8) {
+    tc::reg_dec<56>();
+    if (warp < 2) {
+      // ---------------------------------------------------------------- TMA producers
+      const int which = warp;                               // 0: K ring (+ Q pair), 1: V ring
+      const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+      const uint32_t nslots = which == 0 ? kFwwKSlots : kFwwVSlots;
+      uint64_t* full = which == 0 ? misc->k_full : misc->v_full;
+      uint64_t* empty = which == 0 ? misc->k_empty : misc->v_empty;
+      unsigned char* ring = smem + (which == 0 ? 0 : kFwwKSlots * C::SLOT);
+      const int my_h = lane >> 1, my_blk = lane & 1;
+      const bool issuer = lane < 2 * C::DH;
+      uint32_t tg = 0, n_items = 0, published = 0;
+      for (uint32_t seq = 0;; ++seq) {
+        int item = 0;
+        if (lane == 0) {
+          if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
+          else item = item_get(&misc->items, seq, &misc->abort_flag);
+        }
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item == -2) goto done;
+        if (item < 0) break;
+        const int c = item % n_cubes, bhq = item / n_cubes;
+        const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
+        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c], end = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1];
+        const int nt = (end - beg) >> 1;                    // the expanded list holds both halves of every key cube
+        if (nt == 0) continue;
+        const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+        if (which == 0) {
+          int it_, ih_, iw_;
+          cube_coords(g, 2 * c + my_blk, it_, ih_, iw_);
+          int ok = 1;
+          if (lane == 0) {
+            ok = tc::mbar_wait(&misc->q_empty, (n_items & 1) ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&misc->q_full, C::SLOT);
+          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+          if (issuer)
+            tc::tma_load_5d(q_tile + (2 * my_h + my_blk) * C::SLAB, &tm_q, &misc->q_full, my_h * 64, iw_ * g.Bw, ih_ * g.Bh,
+                            it_ * g.Bt, bhq);
+        }
+        ++n_items;
+        int j = cols[my_blk];
+        for (int t = 0; t < nt; ++t, ++tg) {
+          int jt, jh, jw;
+          cube_coords(g, j, jt, jh, jw);
+          if (t + 1 < nt) j = cols[2 * t + 2 + my_blk];        // next tile, fetched early
+          const uint32_t slot = tg % nslots, par = (tg / nslots) & 1;
+          int ok = 1;
+          if (lane == 0) {
+            ok = tc::mbar_wait(&empty[slot], par ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&full[slot], C::SLOT);
+          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+          if (issuer)
+            tc::tma_load_5d(ring + slot * C::SLOT + (2 * my_h + my_blk) * C::SLAB, tm, &full[slot], my_h * 64,
+                            jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
+        }
+      }
+    } else if (warp == 2) {
+      // ---------------------------------------------------------------- issuer of S^T(t) = K_pair * Q_pair^T
+      if (lane == 0) {
+        const uint32_t q_addr = tc::smem_u32(q_tile), slot0 = tc::smem_u32(smem);
+        uint32_t tg = 0, n_items = 0;
+        for (uint32_t seq = 0;; ++seq) {
+          VSA2_NEXT_ITEM(item, seq);
+          const int c = item % n_cubes, bhq = item / n_cubes;
+          const int nt = (a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c]) >> 1;
+          if (nt == 0) continue;
+          VSA2_WAIT(&misc->q_full, n_items & 1);
+          for (int t = 0; t < nt; ++t, ++tg) {
+            const uint32_t slot = tg % kFwwKSlots, buf = tg % kFwwSBufs;
+            VSA2_WAIT(&misc->k_full[slot], (tg / kFwwKSlots) & 1);
+            VSA2_WAIT(&misc->s_free[buf], ((tg / kFwwSBufs) & 1) ^ 1);
+            tc::tc_fence_after();
+            mma_pair_pair_kmajor<D>(tmem_base + buf * 128, slot0 + slot * C::SLOT, q_addr);
+            tc::mma_commit(&misc->s_full[buf]);
+            tc::mma_commit(&misc->k_empty[slot]);
+          }
+          tc::mma_commit(&misc->q_empty);          // the Q pair may be replaced once these products are done
+          ++n_items;
+        }
+      }
+    } else if (warp == 4) {
+      // ---------------------------------------------------------------- issuer of O^T += V_pair^T * P^T
+      if (lane == 0) {
+        const uint32_t p_addr = tc::smem_u32(p_tile), slot0 = tc::smem_u32(smem);
+        const uint32_t tm_o = tmem_base + 256;
+        uint32_t tg = 0, n_items = 0;
+        for (uint32_t seq = 0;; ++seq) {
+          VSA2_NEXT_ITEM(item, seq);
+          const int c = item % n_cubes, bhq = item / n_cubes;
+          const int nt = (a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c]) >> 1;
+          if (nt == 0) continue;
+          VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous cube's accumulator was read out
+          for (int t = 0; t < nt; ++t, ++tg) {
+            const uint32_t slot = tg % kFwwVSlots;
+            VSA2_WAIT(&misc->v_full[slot], (tg / kFwwVSlots) & 1);
+            VSA2_WAIT(&misc->p_ready, tg & 1);
+            tc::tc_fence_after();
+            mma_pairT_wide_mnmajor<D>(tm_o, slot0 + (kFwwKSlots + slot) * C::SLOT, p_addr, C::PBYTES, t > 0);
+            tc::mma_commit(&misc->v_empty[slot]);
+            tc::mma_commit(&misc->p_free);
+          }
+          tc::mma_commit(&misc->o_full);
+          ++n_items;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
+    tc::reg_inc<200>();
+    const int wg = (warp >> 2) - 2;              // query half owned by this warpgroup
+    const int quad = warp & 3;
+    const int row = (quad << 5) | lane;          // tensor-memory lane: key row in S^T, channel in O^T
+    const int sm_tid = tid & 127;
+    const int sm_warp = warp - 8;                // 4 * wg + quad
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
+    unsigned char* my_p = p_tile + wg * C::PBYTES;
+    CubePos cpos;
+    cpos.init(g, row & 63);
+    const int blk = row >> 6;                    // which half of the key cube this thread's row belongs to
+    uint32_t tg = 0, n_items = 0, n_all = 0, wg_phase = 0;
+    for (;; ++n_all) {
+      VSA2_NEXT_ITEM(item, n_all);
+      const int c = item % n_cubes, bhq = item / n_cubes;
+      const int i = 2 * c + wg;                  // this warpgroup's query half-cube
+      const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c], end = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1];
+      const int nt = (end - beg) >> 1;
+      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+      const int tb = n_all & 1;
+      if (sm_tid < 64) {
+        int it_, ih_, iw_;
+        cube_coords(g, i, it_, ih_, iw_);
+        const int l = cube_token(g, it_, ih_, iw_, sm_tid);
+        misc->tok[tb][wg][sm_tid] = l;
+        misc->gate[tb][wg][sm_tid] = (coarse && l >= 0) ? a.gate[(size_t)bhq * g.L + l] : 0.f;
+      }
+      const float oc_d = (coarse && row < D) ? a.oc_hat[((size_t)bhq * g.N + i) * D + row] : 0.f;
+      if (sm_tid == 0) misc->rescue_flag[wg] = 0;
+
+      float l_part[64];
+#pragma unroll
+      for (int cc = 0; cc < 64; ++cc) l_part[cc] = 0.f;
+      const uint32_t tg0 = tg;
+      if (nt > 0) {
+        // reference exponent of every query column of this half = exact column maximum of the first tile
+        const uint32_t buf = tg % kFwwSBufs;
+        const bool valid = cpos.valid(edge[cols[blk]], g);
+        VSA2_WAIT(&misc->s_full[buf], (tg / kFwwSBufs) & 1);
+        tc::tc_fence_after();
+        uint32_t s0[32], s1[32];
+        tc::tmem_ld32(lane_addr + buf * 128 + wg * 64, s0);
+        tc::tmem_ld32(lane_addr + buf * 128 + wg * 64 + 32, s1);
+        tc::tmem_ld_wait();
+        float mx[64];
+#pragma unroll
+        for (int cc = 0; cc < 32; ++cc) {
+          mx[cc] = valid ? __uint_as_float(s0[cc]) : -INFINITY;
+          mx[cc + 32] = valid ? __uint_as_float(s1[cc]) : -INFINITY;
+        }
+        warp_reduce_cols64<true>(mx, lane);
+        const int cb = warp_reduce_col(lane);
+        misc->red[sm_warp][cb] = mx[0];
+        misc->red[sm_warp][cb + 1] = mx[1];
+        VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
+        if (sm_tid < 64) {
+          const float m4 = fmaxf(fmaxf(misc->red[4 * wg][sm_tid], misc->red[4 * wg + 1][sm_tid]),
+                                 fmaxf(misc->red[4 * wg + 2][sm_tid], misc->red[4 * wg + 3][sm_tid]));
+          misc->m_ref[wg][sm_tid] = (m4 > -INFINITY) ? m4 * c2 : 0.f;
+        }
+      }
+      VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);       // tables and reference exponents visible to the warpgroup
+
+      if (nt > 0) {
+        int j_next = cols[blk];
+        for (int t = 0; t < nt; ++t) {
+          const uint32_t tgt = tg0 + t, buf = tgt % kFwwSBufs;
+          const bool valid = cpos.valid(edge[j_next], g);
+          if (t + 1 < nt) j_next = cols[2 * t + 2 + blk];
+          const bool all_valid = __all_sync(0xffffffffu, valid);
+          VSA2_WAIT(&misc->s_full[buf], (tgt / kFwwSBufs) & 1);
+          tc::tc_fence_after();
+          uint32_t sa[32], sb[32];
+          tc::tmem_ld32(lane_addr + buf * 128 + wg * 64, sa);
+          tc::tmem_ld32(lane_addr + buf * 128 + wg * 64 + 32, sb);
+          tc::tmem_ld_wait();
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->s_free[buf]);
+          uint32_t packed[32];
+          const float4* mref4 = reinterpret_cast<const float4*>(misc->m_ref[wg]);
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 m = mref4[c4];
+            float p0 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 0]), c2, -m.x));
+            float p1 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 1]), c2, -m.y));
+            float p2 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 2]), c2, -m.z));
+            float p3 = ex2_approx(fmaf(__uint_as_float(sa[4 * c4 + 3]), c2, -m.w));
+            if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
+            l_part[4 * c4 + 0] += p0;
+            l_part[4 * c4 + 1] += p1;
+            l_part[4 * c4 + 2] += p2;
+            l_part[4 * c4 + 3] += p3;
+            packed[2 * c4] = pack_bf16x2(p0, p1);
+            packed[2 * c4 + 1] = pack_bf16x2(p2, p3);
+          }
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            const float4 m = mref4[8 + c4];
+            float p0 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 0]), c2, -m.x));
+            float p1 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 1]), c2, -m.y));
+            float p2 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 2]), c2, -m.z));
+            float p3 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 3]), c2, -m.w));
+            if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
+            l_part[32 + 4 * c4 + 0] += p0;
+            l_part[32 + 4 * c4 + 1] += p1;
+            l_part[32 + 4 * c4 + 2] += p2;
+            l_part[32 + 4 * c4 + 3] += p3;
+            packed[16 + 2 * c4] = pack_bf16x2(p0, p1);
+            packed[16 + 2 * c4 + 1] = pack_bf16x2(p2, p3);
+          }
+          VSA2_WAIT(&misc->p_free, (tgt & 1) ^ 1);           // the previous tile's O^T product has read P^T
+          store_row_sw128(my_p, row, packed);
+          tc::fence_proxy_async_smem();
+          tc::mbar_arrive(&misc->p_ready);
+        }
+        tg += nt;
+
+        // ---- epilogue of this query half: row sums over the 128 key rows x tiles
+        warp_reduce_cols64<false>(l_part, lane);
+        {
+          const int cb = warp_reduce_col(lane);
+          misc->red[sm_warp][cb] = l_part[0];
+          misc->red[sm_warp][cb + 1] = l_part[1];
+        }
+        VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
+        if (sm_tid < 64) {
+          const float l = (misc->red[4 * wg][sm_tid] + misc->red[4 * wg + 1][sm_tid]) +
+                          (misc->red[4 * wg + 2][sm_tid] + misc->red[4 * wg + 3][sm_tid]);
+          if (!(l > 1e-30f && l < 1e30f)) misc->rescue_flag[wg] = 1;
+          misc->l_inv[wg][sm_tid] = 1.f / l;
+          const int tk = misc->tok[tb][wg][sm_tid];
+          if (tk >= 0) a.lse[(size_t)bhq * g.L + tk] = (misc->m_ref[wg][sm_tid] + __log2f(l)) * 0.6931471805599453f;
+        }
+        VSA2_WAIT(&misc->o_full, n_items & 1);
+        tc::tc_fence_after();
+        VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
+      }
+
+      // O[l, d] = O^T[d, q] / l[q] + gate[q] * O_c[d] for the 64 queries of this half
+      {
+        float acc[64];
+        if (nt > 0) {
+          uint32_t o0[32], o1[32];
+          tc::tmem_ld32(lane_addr + 256 + wg * 64, o0);
+          tc::tmem_ld32(lane_addr + 256 + wg * 64 + 32, o1);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int cc = 0; cc < 32; ++cc) {
+            acc[cc] = __uint_as_float(o0[cc]);
+            acc[cc + 32] = __uint_as_float(o1[cc]);
+          }
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->o_empty);
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < 64; ++cc) acc[cc] = 0.f;
+        }
+        if (row < D) {
+#pragma unroll
+          for (int qq = 0; qq < 64; ++qq)
+            acc[qq] = fmaf(misc->gate[tb][wg][qq], oc_d, nt > 0 ? acc[qq] * misc->l_inv[wg][qq] : 0.f);
+        }
+        if (g.out_f32 || a.o_res == nullptr) {
+          // plain stores (validation paths): one element per thread and query
+          if (row < D) {
+#pragma unroll
+            for (int qq = 0; qq < 64; ++qq) {
+              const int l = misc->tok[tb][wg][qq];
+              if (l < 0) continue;
+              const size_t idx = ((size_t)bhq * g.L + l) * D + row;
+              store_out(a.o, idx, acc[qq], g.out_f32);
+              if (a.o_res != nullptr) a.o_res[idx] = __float2bfloat16_rn(acc[qq] - __bfloat162float(__float2bfloat16_rn(acc[qq])));
+            }
+          }
+        } else {
+          // bf16 output, then its rounding residual: transpose through this half's P^T buffer (idle now: every product
+          // of the cube has completed), 16-byte stores
+          bf16* st = reinterpret_cast<bf16*>(my_p);                      // [64 q][D]
+          constexpr int CH = D / 8;                                      // 16-byte chunks per token row
+#pragma unroll 1
+          for (int round = 0; round < 2; ++round) {
+            if (row < D) {
+#pragma unroll
+              for (int qq = 0; qq < 64; ++qq) {
+                const bf16 vb = __float2bfloat16_rn(acc[qq]);
+                st[qq * D + row] = round == 0 ? vb : __float2bfloat16_rn(acc[qq] - __bfloat162float(vb));
+              }
+            }
+            VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
+            bf16* dst = round == 0 ? reinterpret_cast<bf16*>(a.o) : a.o_res;
+            for (int e = sm_tid; e < 64 * CH; e += 128) {
+              const int qi = e / CH, ch = e % CH;
+              const int l = misc->tok[tb][wg][qi];
+              if (l < 0) continue;
+              *reinterpret_cast<uint4*>(dst + ((size_t)bhq * g.L + l) * D + ch * 8) =
+                  *reinterpret_cast<const uint4*>(st + qi * D + ch * 8);
+            }
+            VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);    // staging buffer free before it is rewritten
+          }
+        }
+      }
+      if (nt == 0 && sm_tid < 64 && misc->tok[tb][wg][sm_tid] >= 0)
+        a.lse[(size_t)bhq * g.L + misc->tok[tb][wg][sm_tid]] = -INFINITY;
+      if (nt > 0 && sm_tid == 0 && misc->rescue_flag[wg]) {
+        int slot = atomicAdd(a.rescue_count, 1);
+        if (slot < kFwwRescueCap) a.rescue_items[slot] = bhq * g.N + i;      // half-cube item of the N = 64 numbering
+        else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
+      }
+      if (nt > 0) ++n_items;
+    }
+  }
+
+done:
+  tc::tc_fence_before();
+  __syncthreads();
+  if (misc->abort_flag) {
+    if (tid == 0) atomicExch(&a.status->status, VSA2_ERR_DEVICE_TIMEOUT);
+    // let copies that are still in flight land before the CTA's shared memory is released
+    if (tid == 0) {
+      const unsigned long long t0 = tc::global_timer_ns();
+      while (tc::global_timer_ns() - t0 < 200000ull) {
+      }
+    }
+    __syncthreads();
+  }
+  if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
+}
+
+cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
+                                 const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
+                                 const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
+
+// `g`: half-cube geometry; row_ptr / col_idx: the expanded map; oc_hat: per half-cube.  workspace as for the N = 64 launcher.
+cudaError_t launch_fine_fwd_wide_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                                    const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                                    float* lse, StatusBlock* status, cudaStream_t st) {
+  CUtensorMap tq, tk, tv;
+  if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv))
+    return cudaErrorInvalidValue;
+  int dev = 0, sms = 0;
+  cudaError_t e;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if (fine_fwd_tc_workspace_bytes() < 256 + (size_t)kFwwRescueCap * sizeof(int)) return cudaErrorInvalidValue;
+  FwdWideArgs a;
+  a.gate = gate; a.row_ptr = row_ptr; a.col_idx = col_idx; a.oc_hat = oc_hat; a.o = o; a.o_res = o_res; a.lse = lse;
+  a.status = status;
+  a.rescue_count = &status->pad[0];
+  a.item_counter = &status->pad[1];
+  a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
+  const int total = g.batch * g.Hq * (g.N / 2);
+  const int grid = total < sms ? total : sms;
+  if (g.N > kFwwMaxCubes || (g.N & 1)) return cudaErrorInvalidValue;
+  // the softmax warpgroups raise their register count to 200 with what the service warpgroups give up (setmaxnreg);
+  // that request would block for ever if the launch allocation were smaller than 128 registers per thread
+  {
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, g.D == 128 ? (const void*)fine_fwd_wide_tc_kernel<128>
+                                                   : (const void*)fine_fwd_wide_tc_kernel<64>)) != cudaSuccess)
+      return e;
+    if (fa.numRegs * kFwwThreads < 256 * 56 + 256 * 200) return cudaErrorLaunchOutOfResources;
+  }
+  if (g.D == 128) {
+    const size_t smb = FwdWide<128>::smem_bytes(g.N);
+    if (smb > 227 * 1024) return cudaErrorInvalidValue;
+    if ((e = cudaFuncSetAttribute(fine_fwd_wide_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_wide_tc_kernel<128><<<grid, kFwwThreads, smb, st>>>(tq, tk, tv, g, a);
+  } else {
+    const size_t smb = FwdWide<64>::smem_bytes(g.N);
+    if (smb > 227 * 1024) return cudaErrorInvalidValue;
+    if ((e = cudaFuncSetAttribute(fine_fwd_wide_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_wide_tc_kernel<64><<<grid, kFwwThreads, smb, st>>>(tq, tk, tv, g, a);
+  }
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  // half-cubes whose row sums left the safe range are redone with the exact running maximum
+  return launch_fine_fwd_list(g, a.rescue_count, a.rescue_items, q, k, v, gate, row_ptr, col_idx, oc_hat, o, o_res, lse, st);
+}
+
+}  // namespace vsa2

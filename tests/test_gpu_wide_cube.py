@@ -54,7 +54,7 @@ def test_wide_cube_several_tiles_per_sequence():
     full_parity(WIDE_TILES, syn.make_inputs(WIDE_TILES))
 
 
-@pytest.mark.parametrize("flags", [vb.FLAG_TF32_COARSE, vb.FLAG_SIMPLE_COARSE | vb.FLAG_SIMPLE_BWD | vb.FLAG_SIMPLE_ROUTER
+@pytest.mark.parametrize("flags", [vb.FLAG_TF32_COARSE, vb.FLAG_HALF_CUBE_FWD, vb.FLAG_SIMPLE_COARSE | vb.FLAG_SIMPLE_BWD | vb.FLAG_SIMPLE_ROUTER
                                    | vb.FLAG_EXACT_MAX_FWD])
 @pytest.mark.parametrize("wl", [WIDE_RAGGED, WIDE_EMPTY_HALF], ids=lambda w: w.name)
 def test_wide_cube_alternative_kernels(flags, wl):
