@@ -11,17 +11,23 @@
 // The kernel works on the half-cube problem (geometry, expanded block map, per-half coarse rows) that the library
 // builds for 128-token cubes: row 2c of the expanded map lists the half-cubes (2j, 2j+1, ...) of query cube c.
 //
-// Roles (512 threads): warp 0 = TMA producer of the K pairs and the Q pair (lane 0 is also the CTA's scheduler), warp 1
-// = TMA producer of the V pairs, warp 2 = issuer of S^T, warp 4 = issuer of O^T, warpgroups 2 and 3 = softmax +
-// epilogue: warpgroup w owns query half w (columns 64w .. 64w+63) of EVERY tile, so each keeps its own reference
-// exponents, row sums and output rows and the two only meet at the operand barriers.  Softmax as in fine_fwd_tc.cu:
-// fixed reference exponent per query column (exact column maximum of the first tile), row sums checked at the end, a
-// half-cube whose sums left the safe range goes to the exact-maximum kernel.  Every wait is bounded.
+// Roles (640 threads): warp 0 = TMA producer of the K pairs and the Q pair (lane 0 is also the CTA's scheduler), warp 1
+// = TMA producer of the V pairs, warp 2 = issuer of S^T, warp 3 = issuer of O^T, then four softmax + epilogue
+// warpgroups: warpgroup w owns query columns 32w .. 32w+31 of EVERY tile (its thread r holds key row r of them), so
+// each keeps its own reference exponents, row sums and output rows and they meet only at the operand barriers and once
+// per cube.  With 32 columns per thread the role fits the 96 registers a 640-thread CTA gets, so no register
+// re-balancing is needed.  Softmax as in fine_fwd_tc.cu: fixed reference exponent per query column (exact column
+// maximum of the first tile), row sums checked at the end, a half-cube whose sums left the safe range goes to the
+// exact-maximum kernel.  (One reference for all columns would save re-reading 4 KB of references per warp and tile
+// from shared memory, 5 % of the time; but with its own maximum as reference a column's largest P of the first tile
+// is exactly 1, while any other reference rounds it to bf16 and scales the whole output row of a sharply peaked query
+// by up to 2^-9 against its fp32 row sum, which the backward amplifies: measured dK error 5e-2 instead of 1e-2.)
+// Every wait is bounded.
 #include "tc_attn.cuh"
 
 namespace vsa2 {
 
-constexpr int kFwwThreads = 512;
+constexpr int kFwwThreads = 640;      // 4 service warps + 4 softmax warpgroups
 constexpr int kFwwKSlots = 2;
 constexpr int kFwwVSlots = 2;
 constexpr int kFwwSBufs = 2;          // S^T buffers of 128 columns
@@ -48,15 +54,15 @@ struct FwdWideMisc {
   uint64_t s_full[kFwwSBufs], s_free[kFwwSBufs];
   uint64_t p_ready, p_free;
   ItemQueue items;
-  uint64_t wg_sync[2];             // group barrier of one softmax warpgroup (128 threads)
+  uint64_t wg_sync[4], all_sync;   // group barriers of one softmax warpgroup (128 threads) and of all four (512)
   uint32_t tmem_base;
   int abort_flag;
-  int rescue_flag[2];
-  alignas(16) float m_ref[2][64];  // per query half and column: reference exponent (log2 units)
-  alignas(16) float l_inv[2][64];
-  alignas(16) float red[8][64];    // per-warp partial column reductions (warps 4w .. 4w+3 belong to query half w)
-  int tok[2][2][64];               // [item parity][query half][position]: raster token (-1 = padding)
-  float gate[2][2][64];
+  int rescue_flag[4];
+  alignas(16) float m_ref[128];    // per query column of the cube: reference exponent (log2 units)
+  alignas(16) float l_inv[128];
+  alignas(16) float red[16][32];   // per-warp partial column reductions (warps 4w .. 4w+3 belong to warpgroup w)
+  int tok[2][128];                 // [item parity][query column]: raster token (-1 = padding)
+  float gate[2][128];
 };
 static_assert(sizeof(FwdWideMisc) <= 6144, "misc region too small");
 
@@ -125,7 +131,7 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     tc::mbar_init(&misc->q_full, 1);
     tc::mbar_init(&misc->q_empty, 1);
     tc::mbar_init(&misc->o_full, 1);
-    tc::mbar_init(&misc->o_empty, 256);
+    tc::mbar_init(&misc->o_empty, 512);
     for (int s = 0; s < kFwwKSlots; ++s) {
       tc::mbar_init(&misc->k_full[s], 1);
       tc::mbar_init(&misc->k_empty[s], 1);
@@ -136,13 +142,13 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     }
     for (int s = 0; s < kFwwSBufs; ++s) {
       tc::mbar_init(&misc->s_full[s], 1);
-      tc::mbar_init(&misc->s_free[s], 256);
+      tc::mbar_init(&misc->s_free[s], 512);
     }
-    tc::mbar_init(&misc->p_ready, 256);
+    tc::mbar_init(&misc->p_ready, 512);
     tc::mbar_init(&misc->p_free, 1);
-    tc::mbar_init(&misc->wg_sync[0], 128);
-    tc::mbar_init(&misc->wg_sync[1], 128);
-    item_queue_init(&misc->items, 2 + 2 + 256);     // lane 0 of the producers, two issuers, the softmax threads
+    for (int s = 0; s < 4; ++s) tc::mbar_init(&misc->wg_sync[s], 128);
+    tc::mbar_init(&misc->all_sync, 512);
+    item_queue_init(&misc->items, 2 + 2 + 512);     // lane 0 of the producers, two issuers, the softmax threads
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -158,8 +164,7 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   const uint32_t tmem_base = misc->tmem_base;
   // tensor-memory columns: S^T buffers at 0 and 128; O^T at 256 .. 383
 
-  if (warp < 8) {
-    tc::reg_dec<56>();
+  if (warp < 4) {
     if (warp < 2) {
       // ---------------------------------------------------------------- TMA producers
       const int which = warp;                               // 0: K ring (+ Q pair), 1: V ring
@@ -241,8 +246,8 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           ++n_items;
         }
       }
-    } else if (warp == 4) {
-      // ---------------------------------------------------------------- issuer of O^T += V_pair^T * P^T
+    } else {
+      // ---------------------------------------------------------------- issuer of O^T += V_pair^T * P^T (warp 3)
       if (lane == 0) {
         const uint32_t p_addr = tc::smem_u32(p_tile), slot0 = tc::smem_u32(smem);
         const uint32_t tm_o = tmem_base + 256;
@@ -268,16 +273,18 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
-    tc::reg_inc<200>();
-    const int wg = (warp >> 2) - 2;              // query half owned by this warpgroup
+    // ------------------------------------------------------------------ softmax + epilogue (4 x 128 threads)
+    const int wg = (warp - 4) >> 2;              // warpgroup 0..3: query columns 32 wg .. 32 wg + 31 of every tile
+    const int half = wg >> 1;                    // the query half-cube those columns belong to
     const int quad = warp & 3;
     const int row = (quad << 5) | lane;          // tensor-memory lane: key row in S^T, channel in O^T
-    const int sm_tid = tid & 127;
-    const int sm_warp = warp - 8;                // 4 * wg + quad
+    const int sm_tid = (tid - 128) & 127;
+    const int sm_warp = warp - 4;                // 4 * wg + quad
+    const int q0 = 32 * wg;                      // first query column (0..127 over the cube) of this warpgroup
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
-    unsigned char* my_p = p_tile + wg * C::PBYTES;
+    unsigned char* p_row = p_tile + half * C::PBYTES + row * 128;   // this thread's key row of P^T of its query half
+    const int chunk0 = (wg & 1) * 4;             // its 32 queries are the 16-byte chunks chunk0 .. chunk0 + 3 of that row
     CubePos cpos;
     cpos.init(g, row & 63);
     const int blk = row >> 6;                    // which half of the key cube this thread's row belongs to
@@ -285,50 +292,44 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     for (;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
       const int c = item % n_cubes, bhq = item / n_cubes;
-      const int i = 2 * c + wg;                  // this warpgroup's query half-cube
+      const int i = 2 * c + half;                // query half-cube of this warpgroup
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c], end = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1];
       const int nt = (end - beg) >> 1;
       const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
       const int tb = n_all & 1;
-      if (sm_tid < 64) {
+      if (sm_tid < 32) {
         int it_, ih_, iw_;
         cube_coords(g, i, it_, ih_, iw_);
-        const int l = cube_token(g, it_, ih_, iw_, sm_tid);
-        misc->tok[tb][wg][sm_tid] = l;
-        misc->gate[tb][wg][sm_tid] = (coarse && l >= 0) ? a.gate[(size_t)bhq * g.L + l] : 0.f;
+        const int l = cube_token(g, it_, ih_, iw_, (q0 + sm_tid) & 63);
+        misc->tok[tb][q0 + sm_tid] = l;
+        misc->gate[tb][q0 + sm_tid] = (coarse && l >= 0) ? a.gate[(size_t)bhq * g.L + l] : 0.f;
       }
       const float oc_d = (coarse && row < D) ? a.oc_hat[((size_t)bhq * g.N + i) * D + row] : 0.f;
       if (sm_tid == 0) misc->rescue_flag[wg] = 0;
 
-      float l_part[64];
+      float l_part[32];
 #pragma unroll
-      for (int cc = 0; cc < 64; ++cc) l_part[cc] = 0.f;
+      for (int cc = 0; cc < 32; ++cc) l_part[cc] = 0.f;
       const uint32_t tg0 = tg;
       if (nt > 0) {
-        // reference exponent of every query column of this half = exact column maximum of the first tile
+        // reference exponent of this warpgroup's query columns = exact column maximum of the first tile
         const uint32_t buf = tg % kFwwSBufs;
         const bool valid = cpos.valid(edge[cols[blk]], g);
         VSA2_WAIT(&misc->s_full[buf], (tg / kFwwSBufs) & 1);
         tc::tc_fence_after();
-        uint32_t s0[32], s1[32];
-        tc::tmem_ld32(lane_addr + buf * 128 + wg * 64, s0);
-        tc::tmem_ld32(lane_addr + buf * 128 + wg * 64 + 32, s1);
+        uint32_t s0[32];
+        tc::tmem_ld32(lane_addr + buf * 128 + q0, s0);
         tc::tmem_ld_wait();
-        float mx[64];
+        float mx[32];
 #pragma unroll
-        for (int cc = 0; cc < 32; ++cc) {
-          mx[cc] = valid ? __uint_as_float(s0[cc]) : -INFINITY;
-          mx[cc + 32] = valid ? __uint_as_float(s1[cc]) : -INFINITY;
-        }
-        warp_reduce_cols64<true>(mx, lane);
-        const int cb = warp_reduce_col(lane);
-        misc->red[sm_warp][cb] = mx[0];
-        misc->red[sm_warp][cb + 1] = mx[1];
+        for (int cc = 0; cc < 32; ++cc) mx[cc] = valid ? __uint_as_float(s0[cc]) : -INFINITY;
+        warp_reduce_cols32<true>(mx, lane);
+        misc->red[sm_warp][lane] = mx[0];
         VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
-        if (sm_tid < 64) {
+        if (sm_tid < 32) {
           const float m4 = fmaxf(fmaxf(misc->red[4 * wg][sm_tid], misc->red[4 * wg + 1][sm_tid]),
                                  fmaxf(misc->red[4 * wg + 2][sm_tid], misc->red[4 * wg + 3][sm_tid]));
-          misc->m_ref[wg][sm_tid] = (m4 > -INFINITY) ? m4 * c2 : 0.f;
+          misc->m_ref[q0 + sm_tid] = (m4 > -INFINITY) ? m4 * c2 : 0.f;
         }
       }
       VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);       // tables and reference exponents visible to the warpgroup
@@ -342,14 +343,13 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           const bool all_valid = __all_sync(0xffffffffu, valid);
           VSA2_WAIT(&misc->s_full[buf], (tgt / kFwwSBufs) & 1);
           tc::tc_fence_after();
-          uint32_t sa[32], sb[32];
-          tc::tmem_ld32(lane_addr + buf * 128 + wg * 64, sa);
-          tc::tmem_ld32(lane_addr + buf * 128 + wg * 64 + 32, sb);
+          uint32_t sa[32];
+          tc::tmem_ld32(lane_addr + buf * 128 + q0, sa);
           tc::tmem_ld_wait();
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->s_free[buf]);
-          uint32_t packed[32];
-          const float4* mref4 = reinterpret_cast<const float4*>(misc->m_ref[wg]);
+          uint32_t packed[16];
+          const float4* mref4 = reinterpret_cast<const float4*>(misc->m_ref + q0);
 #pragma unroll
           for (int c4 = 0; c4 < 8; ++c4) {
             const float4 m = mref4[c4];
@@ -365,79 +365,59 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             packed[2 * c4] = pack_bf16x2(p0, p1);
             packed[2 * c4 + 1] = pack_bf16x2(p2, p3);
           }
-#pragma unroll
-          for (int c4 = 0; c4 < 8; ++c4) {
-            const float4 m = mref4[8 + c4];
-            float p0 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 0]), c2, -m.x));
-            float p1 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 1]), c2, -m.y));
-            float p2 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 2]), c2, -m.z));
-            float p3 = ex2_approx(fmaf(__uint_as_float(sb[4 * c4 + 3]), c2, -m.w));
-            if (!all_valid) { p0 = valid ? p0 : 0.f; p1 = valid ? p1 : 0.f; p2 = valid ? p2 : 0.f; p3 = valid ? p3 : 0.f; }
-            l_part[32 + 4 * c4 + 0] += p0;
-            l_part[32 + 4 * c4 + 1] += p1;
-            l_part[32 + 4 * c4 + 2] += p2;
-            l_part[32 + 4 * c4 + 3] += p3;
-            packed[16 + 2 * c4] = pack_bf16x2(p0, p1);
-            packed[16 + 2 * c4 + 1] = pack_bf16x2(p2, p3);
-          }
           VSA2_WAIT(&misc->p_free, (tgt & 1) ^ 1);           // the previous tile's O^T product has read P^T
-          store_row_sw128(my_p, row, packed);
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch)
+            *reinterpret_cast<uint4*>(p_row + (((chunk0 + ch) ^ (row & 7)) << 4)) =
+                make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
           tc::fence_proxy_async_smem();
           tc::mbar_arrive(&misc->p_ready);
         }
         tg += nt;
 
-        // ---- epilogue of this query half: row sums over the 128 key rows x tiles
-        warp_reduce_cols64<false>(l_part, lane);
-        {
-          const int cb = warp_reduce_col(lane);
-          misc->red[sm_warp][cb] = l_part[0];
-          misc->red[sm_warp][cb + 1] = l_part[1];
-        }
+        // ---- epilogue of these 32 query columns: row sums over the 128 key rows x tiles
+        warp_reduce_cols32<false>(l_part, lane);
+        misc->red[sm_warp][lane] = l_part[0];
         VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
-        if (sm_tid < 64) {
+        if (sm_tid < 32) {
           const float l = (misc->red[4 * wg][sm_tid] + misc->red[4 * wg + 1][sm_tid]) +
                           (misc->red[4 * wg + 2][sm_tid] + misc->red[4 * wg + 3][sm_tid]);
           if (!(l > 1e-30f && l < 1e30f)) misc->rescue_flag[wg] = 1;
-          misc->l_inv[wg][sm_tid] = 1.f / l;
-          const int tk = misc->tok[tb][wg][sm_tid];
-          if (tk >= 0) a.lse[(size_t)bhq * g.L + tk] = (misc->m_ref[wg][sm_tid] + __log2f(l)) * 0.6931471805599453f;
+          misc->l_inv[q0 + sm_tid] = 1.f / l;
+          const int tk = misc->tok[tb][q0 + sm_tid];
+          if (tk >= 0) a.lse[(size_t)bhq * g.L + tk] = (misc->m_ref[q0 + sm_tid] + __log2f(l)) * 0.6931471805599453f;
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
         VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
       }
 
-      // O[l, d] = O^T[d, q] / l[q] + gate[q] * O_c[d] for the 64 queries of this half
+      // O[l, d] = O^T[d, q] / l[q] + gate[q] * O_c[d] for the 32 queries of this warpgroup
       {
-        float acc[64];
+        float acc[32];
         if (nt > 0) {
-          uint32_t o0[32], o1[32];
-          tc::tmem_ld32(lane_addr + 256 + wg * 64, o0);
-          tc::tmem_ld32(lane_addr + 256 + wg * 64 + 32, o1);
+          uint32_t o0[32];
+          tc::tmem_ld32(lane_addr + 256 + q0, o0);
           tc::tmem_ld_wait();
 #pragma unroll
-          for (int cc = 0; cc < 32; ++cc) {
-            acc[cc] = __uint_as_float(o0[cc]);
-            acc[cc + 32] = __uint_as_float(o1[cc]);
-          }
+          for (int cc = 0; cc < 32; ++cc) acc[cc] = __uint_as_float(o0[cc]);
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->o_empty);
         } else {
 #pragma unroll
-          for (int cc = 0; cc < 64; ++cc) acc[cc] = 0.f;
+          for (int cc = 0; cc < 32; ++cc) acc[cc] = 0.f;
         }
         if (row < D) {
 #pragma unroll
-          for (int qq = 0; qq < 64; ++qq)
-            acc[qq] = fmaf(misc->gate[tb][wg][qq], oc_d, nt > 0 ? acc[qq] * misc->l_inv[wg][qq] : 0.f);
+          for (int qq = 0; qq < 32; ++qq)
+            acc[qq] = fmaf(misc->gate[tb][q0 + qq], oc_d, nt > 0 ? acc[qq] * misc->l_inv[q0 + qq] : 0.f);
         }
         if (g.out_f32 || a.o_res == nullptr) {
           // plain stores (validation paths): one element per thread and query
           if (row < D) {
 #pragma unroll
-            for (int qq = 0; qq < 64; ++qq) {
-              const int l = misc->tok[tb][wg][qq];
+            for (int qq = 0; qq < 32; ++qq) {
+              const int l = misc->tok[tb][q0 + qq];
               if (l < 0) continue;
               const size_t idx = ((size_t)bhq * g.L + l) * D + row;
               store_out(a.o, idx, acc[qq], g.out_f32);
@@ -445,24 +425,24 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             }
           }
         } else {
-          // bf16 output, then its rounding residual: transpose through this half's P^T buffer (idle now: every product
-          // of the cube has completed), 16-byte stores
-          bf16* st = reinterpret_cast<bf16*>(my_p);                      // [64 q][D]
+          // bf16 output, then its rounding residual: transpose through this warpgroup's quarter of the P^T region (idle
+          // now: every product of the cube has completed), 16-byte stores
+          bf16* st = reinterpret_cast<bf16*>(p_tile) + (size_t)wg * 32 * D;      // [32 q][D]
           constexpr int CH = D / 8;                                      // 16-byte chunks per token row
 #pragma unroll 1
           for (int round = 0; round < 2; ++round) {
             if (row < D) {
 #pragma unroll
-              for (int qq = 0; qq < 64; ++qq) {
+              for (int qq = 0; qq < 32; ++qq) {
                 const bf16 vb = __float2bfloat16_rn(acc[qq]);
                 st[qq * D + row] = round == 0 ? vb : __float2bfloat16_rn(acc[qq] - __bfloat162float(vb));
               }
             }
             VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);
             bf16* dst = round == 0 ? reinterpret_cast<bf16*>(a.o) : a.o_res;
-            for (int e = sm_tid; e < 64 * CH; e += 128) {
+            for (int e = sm_tid; e < 32 * CH; e += 128) {
               const int qi = e / CH, ch = e % CH;
-              const int l = misc->tok[tb][wg][qi];
+              const int l = misc->tok[tb][q0 + qi];
               if (l < 0) continue;
               *reinterpret_cast<uint4*>(dst + ((size_t)bhq * g.L + l) * D + ch * 8) =
                   *reinterpret_cast<const uint4*>(st + qi * D + ch * 8);
@@ -471,14 +451,17 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           }
         }
       }
-      if (nt == 0 && sm_tid < 64 && misc->tok[tb][wg][sm_tid] >= 0)
-        a.lse[(size_t)bhq * g.L + misc->tok[tb][wg][sm_tid]] = -INFINITY;
+      if (nt == 0 && sm_tid < 32 && misc->tok[tb][q0 + sm_tid] >= 0)
+        a.lse[(size_t)bhq * g.L + misc->tok[tb][q0 + sm_tid]] = -INFINITY;
       if (nt > 0 && sm_tid == 0 && misc->rescue_flag[wg]) {
         int slot = atomicAdd(a.rescue_count, 1);
         if (slot < kFwwRescueCap) a.rescue_items[slot] = bhq * g.N + i;      // half-cube item of the N = 64 numbering
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
       }
       if (nt > 0) ++n_items;
+      // a warpgroup's staging quarter lies inside the P^T half that two warpgroups write: nobody starts the next
+      // cube's P^T before every warpgroup has drained its staging area
+      VSA2_GROUP_SYNC_AT(&misc->all_sync, n_all);
     }
   }
 
@@ -523,15 +506,6 @@ cudaError_t launch_fine_fwd_wide_tc(const Geo& g, const bf16* q, const bf16* k, 
   const int total = g.batch * g.Hq * (g.N / 2);
   const int grid = total < sms ? total : sms;
   if (g.N > kFwwMaxCubes || (g.N & 1)) return cudaErrorInvalidValue;
-  // the softmax warpgroups raise their register count to 200 with what the service warpgroups give up (setmaxnreg);
-  // that request would block for ever if the launch allocation were smaller than 128 registers per thread
-  {
-    cudaFuncAttributes fa;
-    if ((e = cudaFuncGetAttributes(&fa, g.D == 128 ? (const void*)fine_fwd_wide_tc_kernel<128>
-                                                   : (const void*)fine_fwd_wide_tc_kernel<64>)) != cudaSuccess)
-      return e;
-    if (fa.numRegs * kFwwThreads < 256 * 56 + 256 * 200) return cudaErrorLaunchOutOfResources;
-  }
   if (g.D == 128) {
     const size_t smb = FwdWide<128>::smem_bytes(g.N);
     if (smb > 227 * 1024) return cudaErrorInvalidValue;

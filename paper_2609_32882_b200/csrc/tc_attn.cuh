@@ -116,6 +116,21 @@ __device__ __forceinline__ void warp_reduce_cols64(float (&v)[64], int lane) {
     }
   }
 }
+// The same for a 32-wide vector (31 shuffles): afterwards v[0] holds the reduction over all lanes of column `lane`.
+template <bool IS_MAX>
+__device__ __forceinline__ void warp_reduce_cols32(float (&v)[32], int lane) {
+#pragma unroll
+  for (int n = 16, off = 16; off >= 1; n >>= 1, off >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < n; ++i) {
+      const float send = upper ? v[i] : v[i + n];
+      const float keep = upper ? v[i + n] : v[i];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, off);
+      v[i] = IS_MAX ? fmaxf(keep, recv) : keep + recv;
+    }
+  }
+}
 __device__ __forceinline__ int warp_reduce_col(int lane) {
   return ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
 }
