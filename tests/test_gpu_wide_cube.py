@@ -73,3 +73,34 @@ def test_wide_cube_alternative_kernels(flags, wl):
     want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
     for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
         assert_close(name, x, y, tol_abs=2e-2 * np.sqrt(2), bf16_storage=name != "dGate")
+
+
+def test_wide_cube_forward_survives_a_late_dominant_key_cube():
+    """As for 64-token cubes: the first key cube scores tiny, a later one hundreds of nats higher for one query cube, so
+    the fixed softmax references of the 128-query kernel overflow there and both halves of that query cube must come back
+    correct through the exact-maximum fallback (which works on half-cube items)."""
+    import torch
+    from oracle import vsa2_oracle as orc
+    from vsa2_testlib import CudaPath, assert_close, assert_lse_close, oracle_arrays
+    wl = syn.Workload("wide_late_max", 1, 1, 1, 128, (4, 8, 32), select_mode=syn.PER_QUERY, topk=8, kind="iid", seed=42, **WIDE)
+    data = syn.make_inputs(wl)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    assert geo.N == 8
+    q = syn.bf16_bits_to_f32(data["q"]).copy()
+    k = syn.bf16_bits_to_f32(data["k"]).copy()
+    k *= 0.01
+    big = geo.cube_tokens[7]
+    k[0, 0, big] = 8.0 * np.sign(q[0, 0, big[0]])                  # last key cube: huge, aligned keys
+    q[0, 0, geo.cube_tokens[2]] = 8.0 * np.sign(q[0, 0, big[0]])   # one query cube points at them
+    data["q"], data["k"] = syn.f32_to_bf16_bits(q), syn.f32_to_bf16_bits(k)
+    a = oracle_arrays(data)
+    run = CudaPath(wl, data, flags=vb.FLAG_NO_COARSE, out_dtype=vb.F32)
+    gmask = run.route()
+    assert gmask.all()
+    O, lse = run.forward()
+    O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], np.zeros_like(a["gate"]), gmask, geo, 1 / np.sqrt(128))
+    assert lse_ref.max() > 300
+    assert_close("O", O, O_ref)
+    assert_lse_close(lse, lse_ref)
+    rescued = int(run.attn.ws_fwd[8:12].view(torch.int32).item())
+    assert rescued >= 2                                            # both halves of the query cube (one entry per warpgroup that saw it)

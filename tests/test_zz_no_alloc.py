@@ -28,7 +28,8 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     from vsa2_testlib import dev_bf16
     big = syn.CONFIGS[1]                                                              # per-query TopK, 1.8 MiB
     small = syn.Workload("mini_seq", 2, 3, 3, 64, (6, 9, 10), select_mode=syn.PER_SEQUENCE, topk=4, seed=22)
-    for wl in (big, small, big):                 # the second and third calls run over the previous call's leftovers
+    wide = syn.Workload("mini_wide", 1, 4, 2, 128, (7, 10, 28), cube=(4, 4, 8), select_mode=syn.PER_SEQUENCE, topk=5, seed=65)
+    for wl in (big, small, wide, big):           # every call after the first runs over the previous call's leftovers
         data = syn.make_inputs(wl, with_grad=False)
         p = vb.params_from_workload(wl)
         q, k = dev_bf16(data["q"]), dev_bf16(data["k"])
