@@ -13,7 +13,7 @@ cudaEvent_t g_prof_stop[VSA2_KERNEL_COUNT];
 long long g_launches = 0;
 
 struct RouteLayout {
-  size_t status, qr, kr, lse_r, pr, hist, state, row_tau, row_eq_take, row_cnt, row_gt, row_eq, bitmap, total;
+  size_t status, qr, kr, lse_r, pr, hist, state, row_tau, row_eq_take, row_cnt, row_gt, row_eq, bitmap, bitmap_t, total;
   int words;
 };
 struct BwdLayout {
@@ -98,6 +98,7 @@ RouteLayout route_layout(const Geo& g) {
   r.row_gt = c.take(BHq * g.N * sizeof(int));
   r.row_eq = c.take(BHq * g.N * sizeof(int));
   r.bitmap = c.take(BHq * (size_t)g.N * r.words * sizeof(unsigned));
+  r.bitmap_t = c.take(BHq * (size_t)g.N * r.words * sizeof(unsigned));
   r.total = c.off;
   return r;
 }
@@ -311,9 +312,10 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
   s.row_gt = at<int>(workspace, lay.row_gt);
   s.row_eq = at<int>(workspace, lay.row_eq);
   s.bitmap = at<unsigned>(workspace, lay.bitmap);
+  s.bitmap_t = at<unsigned>(workspace, lay.bitmap_t);
   s.words = lay.words;
   {
-    ProfScope ps(VSA2_KERNEL_SELECT, st, g.mode == VSA2_PER_SEQUENCE ? 13 : 6);
+    ProfScope ps(VSA2_KERNEL_SELECT, st, g.mode == VSA2_PER_SEQUENCE ? 14 : 7);
     VSA2_CUDA(launch_select(g, pr, budgets, s, map->row_ptr, map->col_idx, map->col_ptr, map->row_idx, status, st));
   }
   return VSA2_OK;

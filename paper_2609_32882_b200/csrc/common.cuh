@@ -142,7 +142,8 @@ struct SelectScratch {
   int* row_cnt;          // [BH][N]
   int* row_gt;           // [BH][N]
   int* row_eq;           // [BH][N]
-  unsigned* bitmap;      // [BH][N][words]
+  unsigned* bitmap;      // [BH][N][words]   rows x column words
+  unsigned* bitmap_t;    // [BH][N][words]   columns x row words
   int words;             // ceil(N/32)
 };
 cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, const SelectScratch& s,

@@ -47,26 +47,51 @@ __global__ void __launch_bounds__(256) sel_hist_kernel(const float* __restrict__
     if (sh[i]) atomicAdd(&dst[i], sh[i]);
 }
 
-__global__ void sel_pick_kernel(unsigned* state, const unsigned* hist, int pass) {
-  const int bh = blockIdx.x;
-  if (threadIdx.x != 0) return;
+// One warp per (batch, head): finds the digit whose bin holds the `remaining`-th largest entry.  Lane l owns the bins
+// [l * nb/32, (l+1) * nb/32); a suffix sum over the lanes locates the lane, a short serial walk the bin.
+__global__ void __launch_bounds__(32) sel_pick_kernel(unsigned* state, const unsigned* hist, int pass) {
+  const int bh = blockIdx.x, lane = threadIdx.x;
   const unsigned* hsrc = hist + ((size_t)bh * 3 + pass) * kHistBins;
-  unsigned remaining = state[bh * 8 + 2];
-  const int nb = (int)seq_mask(pass) + 1;
-  int bin = 0;
-  for (int d = nb - 1; d >= 0; --d) {
-    unsigned c = hsrc[d];
-    if (c >= remaining) { bin = d; break; }
-    remaining -= c;
+  const unsigned remaining0 = state[bh * 8 + 2];
+  const int nb = (int)seq_mask(pass) + 1, per = nb / 32;
+  unsigned mine = 0u;
+  for (int d = lane * per; d < (lane + 1) * per; ++d) mine += hsrc[d];
+  // above = entries in the bins of all higher lanes
+  unsigned incl = mine;
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned up = __shfl_down_sync(0xffffffffu, incl, o);
+    if (lane + o < 32) incl += up;
   }
-  const int shift = seq_shift(pass);
-  unsigned prefix = state[bh * 8 + 0] | ((unsigned)bin << shift);
-  state[bh * 8 + 0] = prefix;
-  state[bh * 8 + 1] |= seq_mask(pass) << shift;
-  state[bh * 8 + 2] = remaining;
-  if (pass == 2) {
-    state[bh * 8 + 3] = prefix;      // tau: the smallest kept value
-    state[bh * 8 + 4] = remaining;   // how many entries equal to tau are kept
+  const unsigned above = incl - mine;
+  // the threshold bin lies in the highest lane whose suffix count reaches `remaining0`
+  const bool here = above < remaining0 && incl >= remaining0;
+  const unsigned vote = __ballot_sync(0xffffffffu, here);
+  if (vote == 0u) {                    // fewer entries than requested (cannot happen for keep <= N*N): keep everything
+    if (lane == 0) {
+      const int shift = seq_shift(pass);
+      state[bh * 8 + 1] |= seq_mask(pass) << shift;
+      state[bh * 8 + 2] = remaining0 - incl;      // lane 0's inclusive suffix = all entries
+      if (pass == 2) { state[bh * 8 + 3] = state[bh * 8 + 0]; state[bh * 8 + 4] = state[bh * 8 + 2]; }
+    }
+    return;
+  }
+  if (lane == 31 - __clz(vote)) {
+    unsigned remaining = remaining0 - above;
+    int bin = lane * per;
+    for (int d = (lane + 1) * per - 1; d >= lane * per; --d) {
+      const unsigned c = hsrc[d];
+      if (c >= remaining) { bin = d; break; }
+      remaining -= c;
+    }
+    const int shift = seq_shift(pass);
+    const unsigned prefix = state[bh * 8 + 0] | ((unsigned)bin << shift);
+    state[bh * 8 + 0] = prefix;
+    state[bh * 8 + 1] |= seq_mask(pass) << shift;
+    state[bh * 8 + 2] = remaining;
+    if (pass == 2) {
+      state[bh * 8 + 3] = prefix;      // tau: the smallest kept value
+      state[bh * 8 + 4] = remaining;   // how many entries equal to tau are kept
+    }
   }
 }
 
@@ -246,15 +271,38 @@ __global__ void __launch_bounds__(256) sel_emit_rows_kernel(const float* __restr
   }
 }
 
-// thread per column: count set bits down the rows.  grid (ceil(N/256), BH)
-__global__ void __launch_bounds__(256) sel_col_count_kernel(const unsigned* __restrict__ bitmap, int N, int words,
+// bitmap [BH][N rows][words] -> bitmap_t [BH][N columns][words] (bit i of row-word set <-> bit of column-word set):
+// one warp per 32 x 32 bit tile, transposed with 32 ballots.  grid (words, ceil(words/8), BH), 256 threads
+__global__ void __launch_bounds__(256) sel_transpose_bitmap_kernel(const unsigned* __restrict__ bitmap, int N, int words,
+                                                                   unsigned* __restrict__ bitmap_t) {
+  const int lane = threadIdx.x & 31;
+  const int wj = blockIdx.x;                                   // word column of the source: columns 32 wj .. 32 wj + 31
+  const int wi = blockIdx.y * 8 + (threadIdx.x >> 5);          // word row of the source: rows 32 wi .. 32 wi + 31
+  const int bh = blockIdx.z;
+  if (wi >= words) return;
+  const int i = wi * 32 + lane;
+  const unsigned v = i < N ? __ldg(bitmap + ((size_t)bh * N + i) * words + wj) : 0u;
+  unsigned mine = 0u;
+#pragma unroll
+  for (int bit = 0; bit < 32; ++bit) {
+    const unsigned col_word = __ballot_sync(0xffffffffu, (v >> bit) & 1u);   // rows 32 wi .. of column 32 wj + bit
+    if (lane == bit) mine = col_word;
+  }
+  const int j = wj * 32 + lane;
+  if (j < N) bitmap_t[((size_t)bh * N + j) * words + wi] = mine;
+}
+
+// one warp per column: number of kept rows.  grid (ceil(N/8), BH), 256 threads
+__global__ void __launch_bounds__(256) sel_col_count_kernel(const unsigned* __restrict__ bitmap_t, int N, int words,
                                                             int* col_cnt) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x, bh = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + (threadIdx.x >> 5), bh = blockIdx.y;
   if (j >= N) return;
-  const unsigned* bm = bitmap + (size_t)bh * N * words + (j >> 5);
+  const unsigned* bm = bitmap_t + ((size_t)bh * N + j) * words;
   int c = 0;
-  for (int i = 0; i < N; ++i) c += (__ldg(bm + (size_t)i * words) >> (j & 31)) & 1u;
-  col_cnt[(size_t)bh * N + j] = c;
+  for (int w = lane; w < words; w += 32) c += __popc(__ldg(bm + w));
+  for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if (lane == 0) col_cnt[(size_t)bh * N + j] = c;
 }
 
 __global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* __restrict__ col_cnt, int* col_ptr) {
@@ -272,19 +320,24 @@ __global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* _
   if (threadIdx.x == 0) col_ptr[(size_t)bh * (N + 1) + N] = carry;
 }
 
-__global__ void __launch_bounds__(256) sel_emit_cols_kernel(const unsigned* __restrict__ bitmap, int N, int words,
+// one warp per column: ordered emission of the rows that keep it.  grid (ceil(N/8), BH), 256 threads
+__global__ void __launch_bounds__(256) sel_emit_cols_kernel(const unsigned* __restrict__ bitmap_t, int N, int words,
                                                             const int* __restrict__ col_ptr, int* row_idx,
                                                             long long nnz_cap) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x, bh = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + (threadIdx.x >> 5), bh = blockIdx.y;
   if (j >= N) return;
-  const unsigned* bm = bitmap + (size_t)bh * N * words + (j >> 5);
+  const unsigned* bm = bitmap_t + ((size_t)bh * N + j) * words;
   int pos = col_ptr[(size_t)bh * (N + 1) + j];
   int* out = row_idx + (size_t)bh * nnz_cap;
-  for (int i = 0; i < N; ++i) {
-    if ((__ldg(bm + (size_t)i * words) >> (j & 31)) & 1u) {
-      if (pos < nnz_cap) out[pos] = i;
-      ++pos;
+  const unsigned lt = (1u << lane) - 1u;
+  for (int w = 0; w < words; ++w) {
+    const unsigned word = __ldg(bm + w);
+    if ((word >> lane) & 1u) {
+      const int p = pos + __popc(word & lt);
+      if (p < nnz_cap) out[p] = w * 32 + lane;
     }
+    pos += __popc(word);
   }
 }
 
@@ -311,10 +364,11 @@ cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, con
                                             s.row_eq_take, s.row_cnt, row_ptr, g.nnz_cap, status);
   sel_emit_rows_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(pr, N, s.words, s.row_tau, s.row_eq_take, row_ptr,
                                                               col_idx, s.bitmap, g.nnz_cap);
-  // the column counts reuse row_gt as scratch
-  sel_col_count_kernel<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(s.bitmap, N, s.words, s.row_gt);
+  // columns: transposed bitmap, then counts (row_gt reused as scratch), scan, ordered emission
+  sel_transpose_bitmap_kernel<<<dim3(s.words, (s.words + 7) / 8, BH), 256, 0, st>>>(s.bitmap, N, s.words, s.bitmap_t);
+  sel_col_count_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(s.bitmap_t, N, s.words, s.row_gt);
   sel_scan_cols_kernel<<<BH, 1024, 0, st>>>(N, s.row_gt, col_ptr);
-  sel_emit_cols_kernel<<<dim3((N + 255) / 256, BH), 256, 0, st>>>(s.bitmap, N, s.words, col_ptr, row_idx, g.nnz_cap);
+  sel_emit_cols_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(s.bitmap_t, N, s.words, col_ptr, row_idx, g.nnz_cap);
   return cudaGetLastError();
 }
 
