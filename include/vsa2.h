@@ -65,7 +65,8 @@ enum { VSA2_FLAG_SIMPLE_ROUTER = 8 }; /* validation aid: router scores with the 
  * needs that precision); backward by running the tcgen05 fine-branch kernels on the pooled grid with the means rounded
  * to bf16 (its results enter dQ, dK, dV divided by the cube size, where bf16 operand rounding is far below the error
  * bounds). */
-enum { VSA2_FLAG_TF32_COARSE = 32 };  /* validation aid: coarse backward with the TF32 kernels too */
+enum { VSA2_FLAG_TF32_COARSE = 32 };  /* validation aid: coarse forward and backward with the TF32 tile kernels
+                                         that stage their accumulators in shared memory */
 enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
                                          (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */

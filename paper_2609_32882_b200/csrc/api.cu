@@ -382,8 +382,10 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
                    ((g.flags & VSA2_FLAG_BF16_COARSE_FWD) && !(g.flags & VSA2_FLAG_SIMPLE_COARSE) ? 6 : 1) + (wide ? 1 : 0));
       if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
         VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
-      else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
+      else if (g.flags & VSA2_FLAG_TF32_COARSE)
         VSA2_CUDA(launch_coarse_fwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
+      else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
+        VSA2_CUDA(launch_coarse_fwd_mma(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
       else
         VSA2_CUDA(launch_coarse_fwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c,
                                            at<unsigned char>(workspace, pooled_off), st));

@@ -157,6 +157,9 @@ cudaError_t launch_coarse_bwd(const Geo& g, const float* qc, const float* kc, co
                               float* dvc, cudaStream_t st);
 cudaError_t launch_coarse_fwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
                                  float* lse_c, cudaStream_t st);
+// the same product with register-resident accumulators (coarse_fwd_mma.cu): the default forward
+cudaError_t launch_coarse_fwd_mma(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
+                                  float* lse_c, cudaStream_t st);
 cudaError_t launch_coarse_bwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
                                  const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
                                  float* dvc, cudaStream_t st);
