@@ -14,7 +14,7 @@ What the paper fixes and where (section / equation of the VSA2 paper):
 * router: mean-pool over R sub-cubes, softmax, G x G mean-pool           -- Sec. 2.2 Eq. 5-7
 * per-sequence TopK over the flattened N*N scores, N*K blocks kept       -- Sec. 2.2 Eq. 8-9
 * fine branch: block-sparse attention over the kept pairs                -- Sec. 2.2 Eq. 12
-* gated merge O = G * O_c + O_f                                          -- Sec. 2.2 Eq. 13-14
+* gated merge O = G * O_c + O_f, gate G = tanh(X W_g)                    -- Sec. 2.2 Eq. 13-14
 * padding to whole cubes, padded tokens masked                           -- Sec. 2.2 "Kernel Implementation"
 * the routing decision carries no gradient                               -- Sec. 2.1 (last paragraph)
 
@@ -29,6 +29,9 @@ Readings taken where the paper is silent (each listed in the design notes):
 * ties in TopK go to the lower flat index i*N + j.            PARITY UNPINNED
 * a query block with no selected KV block gets O_f = 0 and lse = -inf.
                                                               PARITY UNPINNED
+* gate projection: X [L, C] are the layer's hidden states (C = model width) and
+  W_g has one column per query head, W_g [C, H_q], so that G [H_q, L] holds the
+  per-token per-head gate of Eq. 13 (the paper writes one head: W_g in R^{D x 1}).
 Everything else is pinned by tests/test_oracle_pins.py.
 """
 from __future__ import annotations
@@ -434,6 +437,22 @@ def backward(Q, K, V, gate, masks, geo: Geometry, scale, dO):
 # ----------------------------------------------------------------------------
 # Appendix "Sparsity Computation", Eq. 15-16
 # ----------------------------------------------------------------------------
+# ----------------------------------------------------------------------------
+# Eq. 13: the gate projection and its backward
+# ----------------------------------------------------------------------------
+def gate_forward(X: np.ndarray, Wg: np.ndarray) -> np.ndarray:
+    """X [L, C] hidden states, W_g [C, H] -> gate [H, L] = tanh(X W_g)^T (Eq. 13, one column of W_g per head)."""
+    return np.tanh(X @ Wg).T
+
+
+def gate_backward(X: np.ndarray, Wg: np.ndarray, dgate: np.ndarray):
+    """dgate [H, L] -> (dX [L, C], dW_g [C, H]).  With z = X W_g and gate = tanh(z): dz = dgate * (1 - gate^2),
+    dX = dz W_g^T, dW_g = X^T dz."""
+    gate = np.tanh(X @ Wg)                 # [L, H]
+    dz = dgate.T * (1.0 - gate * gate)     # [L, H]
+    return dz @ Wg.T, X.T @ dz
+
+
 def fine_cost_fraction(K, B, L):
     """Fine-branch cost relative to dense attention: N K B^2 / L^2 = K B / L (Eq. 15)."""
     return K * B / L

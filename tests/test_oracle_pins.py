@@ -461,3 +461,39 @@ def test_input_generators_are_seeded_and_structured():
     assert np.all(syn.head_gate(syn.CONFIGS[0], 0, 0) == 0.5)
     bud = syn.head_budgets(syn.CONFIGS[4], 0, 0)
     assert bud.shape == (1440,) and bud.min() >= 16 and bud.max() <= 256
+
+
+def test_gate_projection_matches_autograd_and_its_special_cases():
+    """Eq. 13: gate = tanh(X W_g).  Pinned against torch's tanh / matmul / autograd (library routines), the
+    zero-initialised projection of the paper's recipe (W_g = 0 => gate = 0 => O = O_f), saturation and oddness."""
+    rng = np.random.default_rng(17)
+    L, C, H = 37, 24, 5
+    X = rng.standard_normal((L, C))
+    Wg = rng.standard_normal((C, H)) * 0.3
+    dgate = rng.standard_normal((H, L))
+    gate = orc.gate_forward(X, Wg)
+    assert gate.shape == (H, L)
+    xt = torch.tensor(X, requires_grad=True)
+    wt = torch.tensor(Wg, requires_grad=True)
+    gt = torch.tanh(xt @ wt).T
+    np.testing.assert_allclose(gate, gt.detach().numpy(), rtol=1e-13, atol=1e-15)
+    gt.backward(torch.tensor(dgate))
+    dX, dW = orc.gate_backward(X, Wg, dgate)
+    np.testing.assert_allclose(dX, xt.grad.numpy(), rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(dW, wt.grad.numpy(), rtol=1e-12, atol=1e-14)
+    # W_g = 0: gate = 0 everywhere, dX = 0, dW_g = X^T dgate^T
+    z = np.zeros_like(Wg)
+    assert not orc.gate_forward(X, z).any()
+    dX0, dW0 = orc.gate_backward(X, z, dgate)
+    assert not dX0.any()
+    np.testing.assert_allclose(dW0, X.T @ dgate.T, rtol=1e-13)
+    # odd in X, bounded by 1, saturating
+    np.testing.assert_allclose(orc.gate_forward(-X, Wg), -gate, rtol=1e-13)
+    assert np.abs(orc.gate_forward(50.0 * X, Wg)).max() <= 1.0
+    # central finite difference of sum(gate * dgate) w.r.t. one weight and one hidden state
+    f = lambda Xv, Wv: float((orc.gate_forward(Xv, Wv) * dgate).sum())
+    h = 1e-6
+    Wp, Wm = Wg.copy(), Wg.copy(); Wp[3, 2] += h; Wm[3, 2] -= h
+    assert abs((f(X, Wp) - f(X, Wm)) / (2 * h) - dW[3, 2]) < 1e-6
+    Xp, Xm = X.copy(), X.copy(); Xp[11, 7] += h; Xm[11, 7] -= h
+    assert abs((f(Xp, Wg) - f(Xm, Wg)) / (2 * h) - dX[11, 7]) < 1e-6
