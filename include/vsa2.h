@@ -199,6 +199,27 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
                   const void* d_o, void* dq, void* dk, void* dv, float* dgate,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Gate projection of the gated merge (Sec. 2.2 "Gated Merge", Eq. 13): gate[b, h, l] = tanh(sum_c x[b, l, c] * w_g[c, h]),
+ * one column of W_g per query head.  The layer that owns the hidden states calls this before vsa2_attn_fwd (which takes
+ * the gate as an input) and vsa2_gate_bwd after vsa2_attn_bwd (which returns dgate).
+ *   x     [batch, L, hidden]      bf16, device, 16-byte aligned; tokens in raster order, L = grid_t * grid_h * grid_w
+ *   w_g   [hidden, heads_q]       bf16, device
+ *   gate  [batch, heads_q, L]     fp32, device (written)
+ * hidden must be a positive multiple of 8 and heads_q <= 64, else VSA2_ERR_UNSUPPORTED.  Only batch, heads_q and the grid of
+ * `p` are used.  Allocates nothing; enqueues on `cuda_stream`. */
+int vsa2_gate_fwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, float* gate, void* cuda_stream);
+
+/* Backward of vsa2_gate_fwd.  With dz = dgate * (1 - gate^2):
+ *   d_w_g [hidden, heads_q]       fp32, device (written): sum over batch and tokens of x[b, l, c] * dz[b, h, l]
+ *   dx    [batch, L, hidden]      p->out_dtype, device, 16-byte aligned (written): sum_h dz[b, h, l] * w_g[c, h]
+ *   gate, dgate [batch, heads_q, L] fp32, device: the output of vsa2_gate_fwd and the dgate of vsa2_attn_bwd
+ *   workspace: device, 256-byte aligned, at least vsa2_gate_bwd_workspace_bytes(p, hidden) (partial sums of d_w_g, which
+ *   are added in a fixed order: results are bitwise reproducible).  Errors as for vsa2_gate_fwd, plus
+ *   VSA2_ERR_WORKSPACE_TOO_SMALL / VSA2_ERR_MISALIGNED. */
+size_t vsa2_gate_bwd_workspace_bytes(const vsa2_params* p, int32_t hidden);
+int vsa2_gate_bwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, const float* gate,
+                  const float* dgate, float* d_w_g, void* dx, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Synchronises `cuda_stream`, reads the status word at the start of `workspace` and stores it in
  * *status_out (host): VSA2_OK, VSA2_ERR_DEVICE_TIMEOUT or VSA2_ERR_MAP_OVERFLOW. */
 int vsa2_device_status(const void* workspace, void* cuda_stream, int32_t* status_out);

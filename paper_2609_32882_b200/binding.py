@@ -32,7 +32,8 @@ ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_MAP_OVERFLOW = -5, -6, -7
 ERR_STATIC_SCRATCH = -8
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
-           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc", "vsa2_last_cuda_error")
+           "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc", "vsa2_last_cuda_error",
+           "vsa2_gate_fwd", "vsa2_gate_bwd", "vsa2_gate_bwd_workspace_bytes")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv")
@@ -90,6 +91,10 @@ def _lib():
         lib.vsa2_query_sizes.argtypes = [C.POINTER(Params), C.POINTER(Sizes)]
         lib.vsa2_route.argtypes = [C.POINTER(Params), vp, vp, vp, C.POINTER(Map), vp, sz, vp]
         lib.vsa2_route_noalloc.argtypes = [C.POINTER(Params), vp, vp, vp, C.POINTER(Map), vp, vp]
+        lib.vsa2_gate_fwd.argtypes = [C.POINTER(Params), C.c_int32, vp, vp, vp, vp]
+        lib.vsa2_gate_bwd_workspace_bytes.argtypes = [C.POINTER(Params), C.c_int32]
+        lib.vsa2_gate_bwd_workspace_bytes.restype = C.c_size_t
+        lib.vsa2_gate_bwd.argtypes = [C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.vsa2_route_scores.argtypes = [C.POINTER(Params), vp]
         lib.vsa2_route_scores.restype = vp
         lib.vsa2_attn_fwd.argtypes = [C.POINTER(Params), vp, vp, vp, vp, C.POINTER(Map), vp, vp, C.POINTER(Saved), vp, sz, vp]
@@ -172,6 +177,22 @@ def vsa2_route_noalloc(p, q, k, budgets, vmap: Map, device_status=None, stream=N
     Vsa2Error(ERR_STATIC_SCRATCH).  `device_status`: optional int32 CUDA tensor receiving the status word."""
     _check(_lib().vsa2_route_noalloc(C.byref(p), _ptr(q), _ptr(k), _ptr(budgets), C.byref(vmap), _ptr(device_status),
                                      _stream(stream)), "vsa2_route_noalloc")
+
+
+def vsa2_gate_fwd(p, hidden, x, w_g, gate, stream=None):
+    """gate[b, h, l] = tanh(sum_c x[b, l, c] w_g[c, h]) (Eq. 13); x [B, L, hidden] bf16, w_g [hidden, Hq] bf16, gate [B, Hq, L] fp32."""
+    _check(_lib().vsa2_gate_fwd(C.byref(p), hidden, _ptr(x), _ptr(w_g), _ptr(gate), _stream(stream)), "vsa2_gate_fwd")
+
+
+def vsa2_gate_bwd_workspace_bytes(p, hidden) -> int:
+    return int(_lib().vsa2_gate_bwd_workspace_bytes(C.byref(p), hidden))
+
+
+def vsa2_gate_bwd(p, hidden, x, w_g, gate, dgate, d_w_g, dx, workspace, stream=None):
+    """Backward of vsa2_gate_fwd: d_w_g [hidden, Hq] fp32 and dx [B, L, hidden] (the params' output dtype)."""
+    nbytes = workspace.numel() * workspace.element_size()
+    _check(_lib().vsa2_gate_bwd(C.byref(p), hidden, _ptr(x), _ptr(w_g), _ptr(gate), _ptr(dgate), _ptr(d_w_g), _ptr(dx),
+                                _ptr(workspace), nbytes, _stream(stream)), "vsa2_gate_bwd")
 
 
 def vsa2_route_scores(p, workspace) -> int:

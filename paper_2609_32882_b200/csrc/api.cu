@@ -525,6 +525,43 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   return VSA2_OK;
 }
 
+int vsa2_gate_fwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, float* gate, void* cuda_stream) {
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  if (!x || !w_g || !gate) return VSA2_ERR_INVALID_ARG;
+  if (!gate_supported(hidden, g.Hq)) return VSA2_ERR_UNSUPPORTED;
+  if (!aligned16(x)) return VSA2_ERR_MISALIGNED;
+  if ((rc = check_device()) != VSA2_OK) return rc;
+  g_launches += 1;
+  VSA2_CUDA(launch_gate_fwd(g.batch, g.L, hidden, g.Hq, reinterpret_cast<const bf16*>(x), reinterpret_cast<const bf16*>(w_g),
+                            gate, reinterpret_cast<cudaStream_t>(cuda_stream)));
+  return VSA2_OK;
+}
+
+size_t vsa2_gate_bwd_workspace_bytes(const vsa2_params* p, int32_t hidden) {
+  Geo g;
+  if (fill_geo(p, &g) != VSA2_OK || !gate_supported(hidden, g.Hq)) return 0;
+  return gate_bwd_workspace_bytes(g.batch, hidden, g.Hq);
+}
+
+int vsa2_gate_bwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, const float* gate,
+                  const float* dgate, float* d_w_g, void* dx, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  if (!x || !w_g || !gate || !dgate || !d_w_g || !dx || !workspace) return VSA2_ERR_INVALID_ARG;
+  if (!gate_supported(hidden, g.Hq)) return VSA2_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(dx) || !aligned256(workspace)) return VSA2_ERR_MISALIGNED;
+  if (workspace_bytes < gate_bwd_workspace_bytes(g.batch, hidden, g.Hq)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if ((rc = check_device()) != VSA2_OK) return rc;
+  g_launches += 3;
+  VSA2_CUDA(launch_gate_bwd(g.batch, g.L, hidden, g.Hq, g.out_f32, reinterpret_cast<const bf16*>(x),
+                            reinterpret_cast<const bf16*>(w_g), gate, dgate, d_w_g, dx, reinterpret_cast<float*>(workspace),
+                            reinterpret_cast<cudaStream_t>(cuda_stream)));
+  return VSA2_OK;
+}
+
 int vsa2_device_status(const void* workspace, void* cuda_stream, int32_t* status_out) {
   if (workspace == nullptr || status_out == nullptr) return VSA2_ERR_INVALID_ARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);

@@ -120,3 +120,17 @@ def test_binding_refuses_host_tensors():
     import torch
     with pytest.raises(ValueError):
         vb._ptr(torch.zeros(4))
+
+
+def test_gate_entry_points_reject_unsupported_shapes_before_any_cuda_call():
+    lib = vb._lib()                                  # the handle with argument types (size_t arguments)
+    p = vb.make_params(batch=1, heads_q=8, heads_kv=8, head_dim=64, grid=(2, 4, 8), topk=1)
+    one = ctypes.c_void_p(256)
+    assert lib.vsa2_gate_fwd(ctypes.byref(p), 60, one, one, one, None) == vb.ERR_UNSUPPORTED          # hidden % 8
+    assert lib.vsa2_gate_fwd(ctypes.byref(p), 64, None, one, one, None) == vb.ERR_INVALID_ARG
+    assert lib.vsa2_gate_fwd(ctypes.byref(p), 64, ctypes.c_void_p(8), one, one, None) == vb.ERR_MISALIGNED
+    many = vb.make_params(batch=1, heads_q=80, heads_kv=80, head_dim=64, grid=(2, 4, 8), topk=1)
+    assert lib.vsa2_gate_fwd(ctypes.byref(many), 64, one, one, one, None) == vb.ERR_UNSUPPORTED       # more than 64 heads
+    assert vb.vsa2_gate_bwd_workspace_bytes(many, 64) == 0
+    assert vb.vsa2_gate_bwd_workspace_bytes(p, 64) == 16 * 64 * 8 * 4
+    assert lib.vsa2_gate_bwd(ctypes.byref(p), 64, one, one, one, one, one, one, one, 100, None) == vb.ERR_WORKSPACE_TOO_SMALL
