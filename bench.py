@@ -429,6 +429,32 @@ def run_ours(args):
                                    f"{r['measured_s']:.1f} s measured, extrapolated to the whole step "
                                    f"({r['t_step_extrapolated_s']:.0f} s)")}
 
+    gate_info = None
+    if args.gate_hidden:
+        # context only: the projection that produces the gate (Eq. 13) and its backward, device-resident operands
+        hid = args.gate_hidden
+        gx = torch.randn(wl.batch, wl.L, hid, device="cuda").to(torch.bfloat16)
+        gw = (torch.randn(hid, wl.heads_q, device="cuda") / hid ** 0.5).to(torch.bfloat16)
+        gg = torch.empty(wl.batch, wl.heads_q, wl.L, dtype=torch.float32, device="cuda")
+        gdw = torch.empty(hid, wl.heads_q, dtype=torch.float32, device="cuda")
+        gdx = torch.empty_like(gx)
+        gws = torch.empty(max(256, vb.vsa2_gate_bwd_workspace_bytes(p, hid)), dtype=torch.uint8, device="cuda")
+        times = []
+        for fn in (lambda: vb.vsa2_gate_fwd(p, hid, gx, gw, gg),
+                   lambda: vb.vsa2_gate_bwd(p, hid, gx, gw, gg, dgate, gdw, gdx, gws)):
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(5):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) / 5)
+        xbytes = gx.numel() * 2
+        gate_info = {"hidden": hid, "fwd_ms": times[0], "bwd_ms": times[1], "x_bytes": xbytes,
+                     "fwd_gbs": xbytes / times[0] / 1e6, "bwd_gbs": 2 * xbytes / times[1] / 1e6}
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -452,6 +478,7 @@ def run_ours(args):
         "fine_fwd": {"ms": kernel_ms["fine_fwd"], "tflops": fine_fwd_tf, "frac_of_sustained_peak": fine_fwd_tf / peak_tf,
                      "frac_of_burst_peak": fine_fwd_tf / pk["bf16_tflops"], "frac_of_nominal_2250": fine_fwd_tf / 2250.0},
         "kernel_ms": kernel_ms,
+        "gate": gate_info,
         "paper_context": "paper reports 8.9x attention speed-up over FlashAttention-3 on one H800 at 220K tokens (not comparable)",
     }
     print(json.dumps(line), flush=True)
@@ -468,6 +495,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="index into the five baseline configurations (3 = 720p top-64)")
     ap.add_argument("--ref-rows", type=int, default=1440, help="query blocks the CPU oracle computes in its sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gate-hidden", type=int, default=0,
+                    help="also time the gate projection tanh(X W_g) and its backward for this hidden width (context: 'gate' key)")
     ap.add_argument("--flags", type=int, default=0, help="VSA2_FLAG_* bits passed to the library (kernel variants)")
     ap.add_argument("--e2e-chunks", type=int, default=8, help="upper limit of head chunks per step in the end-to-end pipeline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end loop (profiling runs)")

@@ -213,8 +213,8 @@ int vsa2_gate_fwd(const vsa2_params* p, int32_t hidden, const void* x, const voi
  *   d_w_g [hidden, heads_q]       fp32, device (written): sum over batch and tokens of x[b, l, c] * dz[b, h, l]
  *   dx    [batch, L, hidden]      p->out_dtype, device, 16-byte aligned (written): sum_h dz[b, h, l] * w_g[c, h]
  *   gate, dgate [batch, heads_q, L] fp32, device: the output of vsa2_gate_fwd and the dgate of vsa2_attn_bwd
- *   workspace: device, 256-byte aligned, at least vsa2_gate_bwd_workspace_bytes(p, hidden) (partial sums of d_w_g, which
- *   are added in a fixed order: results are bitwise reproducible).  Errors as for vsa2_gate_fwd, plus
+ *   workspace: device, 256-byte aligned, at least vsa2_gate_bwd_workspace_bytes(p, hidden) (dz in bf16 and the
+ *   partial sums of d_w_g, which are added in a fixed order: results are bitwise reproducible).  Errors as for vsa2_gate_fwd, plus
  *   VSA2_ERR_WORKSPACE_TOO_SMALL / VSA2_ERR_MISALIGNED. */
 size_t vsa2_gate_bwd_workspace_bytes(const vsa2_params* p, int32_t hidden);
 int vsa2_gate_bwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, const float* gate,

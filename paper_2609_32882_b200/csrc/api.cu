@@ -542,7 +542,7 @@ int vsa2_gate_fwd(const vsa2_params* p, int32_t hidden, const void* x, const voi
 size_t vsa2_gate_bwd_workspace_bytes(const vsa2_params* p, int32_t hidden) {
   Geo g;
   if (fill_geo(p, &g) != VSA2_OK || !gate_supported(hidden, g.Hq)) return 0;
-  return gate_bwd_workspace_bytes(g.batch, hidden, g.Hq);
+  return gate_bwd_workspace_bytes(g.batch, g.L, hidden, g.Hq);
 }
 
 int vsa2_gate_bwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, const float* gate,
@@ -553,11 +553,11 @@ int vsa2_gate_bwd(const vsa2_params* p, int32_t hidden, const void* x, const voi
   if (!x || !w_g || !gate || !dgate || !d_w_g || !dx || !workspace) return VSA2_ERR_INVALID_ARG;
   if (!gate_supported(hidden, g.Hq)) return VSA2_ERR_UNSUPPORTED;
   if (!aligned16(x) || !aligned16(dx) || !aligned256(workspace)) return VSA2_ERR_MISALIGNED;
-  if (workspace_bytes < gate_bwd_workspace_bytes(g.batch, hidden, g.Hq)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < gate_bwd_workspace_bytes(g.batch, g.L, hidden, g.Hq)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
   if ((rc = check_device()) != VSA2_OK) return rc;
-  g_launches += 3;
+  g_launches += 4;
   VSA2_CUDA(launch_gate_bwd(g.batch, g.L, hidden, g.Hq, g.out_f32, reinterpret_cast<const bf16*>(x),
-                            reinterpret_cast<const bf16*>(w_g), gate, dgate, d_w_g, dx, reinterpret_cast<float*>(workspace),
+                            reinterpret_cast<const bf16*>(w_g), gate, dgate, d_w_g, dx, workspace,
                             reinterpret_cast<cudaStream_t>(cuda_stream)));
   return VSA2_OK;
 }

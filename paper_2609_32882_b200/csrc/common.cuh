@@ -193,10 +193,10 @@ cudaError_t launch_expand_map(const Geo& narrow, const int* ptr, const int* idx,
 
 // gate projection and its backward (gate.cu)
 bool gate_supported(int hidden, int heads);
-size_t gate_bwd_workspace_bytes(int batch, int hidden, int heads);
+size_t gate_bwd_workspace_bytes(int batch, int L, int hidden, int heads);
 cudaError_t launch_gate_fwd(int batch, int L, int C, int Hq, const bf16* x, const bf16* w, float* gate, cudaStream_t st);
 cudaError_t launch_gate_bwd(int batch, int L, int C, int Hq, int out_f32, const bf16* x, const bf16* w, const float* gate,
-                            const float* dgate, float* d_w, void* dx, float* partial, cudaStream_t st);
+                            const float* dgate, float* d_w, void* dx, void* workspace, cudaStream_t st);
 
 // tensor-core forward (fine_fwd_tc.cu); `status` heads a workspace of fine_fwd_tc_workspace_bytes()
 size_t fine_fwd_tc_workspace_bytes();

@@ -32,6 +32,11 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"((uint32_t)__cvta_generic_to_shared(smem_row)));
 }
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t& r0, uint32_t& r1, const void* smem_row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
+               : "=r"(r0), "=r"(r1)
+               : "r"((uint32_t)__cvta_generic_to_shared(smem_row)));
+}
 __device__ __forceinline__ uint32_t lds32(const bf16* p) { return *reinterpret_cast<const uint32_t*>(p); }
 
 // X tile: rows l0 .. l0 + 63 of one batch entry, channels c0 .. c0 + 127 -> xs[64][LDX] (zero outside L x C)
@@ -45,17 +50,34 @@ __device__ __forceinline__ void load_x_tile(bf16* xs, const bf16* x, int l0, int
   }
 }
 
-// dz tile: dz[h][tl] = dgate (1 - gate^2) for heads 0 .. HP - 1 (zero beyond Hq) and tokens l0 .. l0 + 63 -> bf16
-__device__ __forceinline__ void load_dz_tile(bf16* dz, int ld, int HP, const float* gate, const float* dgate, int Hq, int l0,
-                                             int L) {
+// dz = dgate (1 - gate^2) in bf16, once per backward, in the two layouts its products read:
+//   dz_hm [batch][HP][Lp]  head-major  (HP = heads rounded up to 16, Lp = tokens rounded up to 64; zero padding)
+//   dz_tm [batch][Lp][HP]  token-major
+// grid (Lp / 64, batch)
+__global__ void __launch_bounds__(kGtThreads) gate_dz_kernel(const float* __restrict__ gate, const float* __restrict__ dgate,
+                                                             int L, int Lp, int Hq, int HP, bf16* __restrict__ dz_hm,
+                                                             bf16* __restrict__ dz_tm) {
+  extern __shared__ __align__(16) unsigned char gate_dz_smem[];
+  bf16* tile = reinterpret_cast<bf16*>(gate_dz_smem);          // [HP][64 + 8]
+  constexpr int LD = kGtTok + 8;
+  const int l0 = blockIdx.x * kGtTok, b = blockIdx.y;
+  const float* gb = gate + (size_t)b * Hq * L;
+  const float* db = dgate + (size_t)b * Hq * L;
   for (int e = threadIdx.x; e < HP * kGtTok; e += kGtThreads) {
     const int h = e / kGtTok, tl = e % kGtTok;
     float v = 0.f;
     if (h < Hq && l0 + tl < L) {
-      const float g = gate[(size_t)h * L + l0 + tl];
-      v = dgate[(size_t)h * L + l0 + tl] * (1.f - g * g);
+      const float g = gb[(size_t)h * L + l0 + tl];
+      v = db[(size_t)h * L + l0 + tl] * (1.f - g * g);
     }
-    dz[h * ld + tl] = __float2bfloat16_rn(v);
+    const bf16 vb = __float2bfloat16_rn(v);
+    tile[h * LD + tl] = vb;
+    dz_hm[((size_t)b * HP + h) * Lp + l0 + tl] = vb;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < kGtTok * HP; e += kGtThreads) {
+    const int tl = e / HP, h = e % HP;
+    dz_tm[((size_t)b * Lp + l0 + tl) * HP + h] = tile[h * LD + tl];
   }
 }
 
@@ -64,20 +86,32 @@ __device__ __forceinline__ void load_dz_tile(bf16* dz, int ld, int HP, const flo
 template <int NT>
 __global__ void __launch_bounds__(kGtThreads) gate_fwd_kernel(const bf16* __restrict__ x, const bf16* __restrict__ w, int L,
                                                               int C, int Hq, float* __restrict__ gate) {
+  constexpr int LDW = NT * 8 + 8;                           // 16-byte aligned rows, eight rows on different banks
   __shared__ __align__(16) bf16 xs[kGtTok * kLdx];
-  __shared__ __align__(16) bf16 wt[NT * 8 * kLdx];          // W chunk transposed: [head][channel]
+  __shared__ __align__(16) bf16 ws[kGtCh * LDW];            // W chunk as stored: [channel][head]; read by ldmatrix.trans
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int l0 = blockIdx.x * kGtTok, b = blockIdx.y;
   const bf16* xb = x + (size_t)b * L * C;
+  const bool w_vec = Hq % 8 == 0 && (reinterpret_cast<uintptr_t>(w) & 15u) == 0;
   float acc[NT][4];
 #pragma unroll
   for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
   for (int c0 = 0; c0 < C; c0 += kGtCh) {
     __syncthreads();
     load_x_tile(xs, xb, l0, L, c0, C);
-    for (int e = threadIdx.x; e < kGtCh * NT * 8; e += kGtThreads) {
-      const int c = e / (NT * 8), h = e % (NT * 8);
-      wt[h * kLdx + c] = (h < Hq && c0 + c < C) ? w[(size_t)(c0 + c) * Hq + h] : __float2bfloat16_rn(0.f);
+    if (w_vec && c0 + kGtCh <= C) {
+      // rows of W are whole 16-byte vectors and the chunk is contiguous: copy as such, then clear the padding heads
+      const int vec = Hq / 8;
+      const uint4* src = reinterpret_cast<const uint4*>(w + (size_t)c0 * Hq);
+      for (int e = threadIdx.x; e < kGtCh * vec; e += kGtThreads)
+        *reinterpret_cast<uint4*>(ws + (e / vec) * LDW + (e % vec) * 8) = __ldg(src + e);
+      for (int e = threadIdx.x; e < kGtCh * (NT * 8 - Hq); e += kGtThreads)
+        ws[(e / (NT * 8 - Hq)) * LDW + Hq + e % (NT * 8 - Hq)] = __float2bfloat16_rn(0.f);
+    } else {
+      for (int e = threadIdx.x; e < kGtCh * NT * 8; e += kGtThreads) {
+        const int c = e / (NT * 8), h = e % (NT * 8);
+        ws[c * LDW + h] = (h < Hq && c0 + c < C) ? w[(size_t)(c0 + c) * Hq + h] : __float2bfloat16_rn(0.f);
+      }
     }
     __syncthreads();
     const bf16* xr = xs + (warp * 16 + g) * kLdx + 2 * t;
@@ -87,8 +121,10 @@ __global__ void __launch_bounds__(kGtThreads) gate_fwd_kernel(const bf16* __rest
                        lds32(xr + 8 * kLdx + ks * 16 + 8)};
 #pragma unroll
       for (int n = 0; n < NT; ++n) {
-        const bf16* wr = wt + (n * 8 + g) * kLdx + ks * 16 + 2 * t;
-        mma_bf16(acc[n], a, lds32(wr), lds32(wr + 8));
+        // B fragment (k = channels, n = heads) from the [channel][head] tile: two stored 8 x 8 blocks, transposed
+        uint32_t b0, b1;
+        ldmatrix_x2_trans(b0, b1, ws + (ks * 16 + (lane & 15)) * LDW + n * 8);
+        mma_bf16(acc[n], a, b0, b1);
       }
     }
   }
@@ -111,9 +147,9 @@ __global__ void __launch_bounds__(kGtThreads) gate_fwd_kernel(const bf16* __rest
 // ---------------------------------------------------------------------------------------------- dX
 // grid (ceil(L / 64), batch); KT = head tiles of 16 (the contraction)
 template <int KT>
-__global__ void __launch_bounds__(kGtThreads) gate_bwd_dx_kernel(const bf16* __restrict__ w, const float* __restrict__ gate,
-                                                                 const float* __restrict__ dgate, int L, int C, int Hq,
-                                                                 int out_f32, void* __restrict__ dx) {
+__global__ void __launch_bounds__(kGtThreads) gate_bwd_dx_kernel(const bf16* __restrict__ w, const bf16* __restrict__ dz_tm,
+                                                                 int L, int Lp, int C, int Hq, int out_f32,
+                                                                 void* __restrict__ dx) {
   constexpr int LDZ = KT * 16 + 8;
   constexpr int LDO = kDxCh + 4;
   __shared__ __align__(16) bf16 az[kGtTok * LDZ];            // dz^T: [token][head]
@@ -121,16 +157,13 @@ __global__ void __launch_bounds__(kGtThreads) gate_bwd_dx_kernel(const bf16* __r
   __shared__ __align__(16) float st[kGtTok * LDO];           // output tile, for coalesced stores
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int l0 = blockIdx.x * kGtTok, b = blockIdx.y;
-  const float* gb = gate + (size_t)b * Hq * L;
-  const float* db = dgate + (size_t)b * Hq * L;
-  for (int e = threadIdx.x; e < KT * 16 * kGtTok; e += kGtThreads) {
-    const int h = e / kGtTok, tl = e % kGtTok;
-    float v = 0.f;
-    if (h < Hq && l0 + tl < L) {
-      const float gg = gb[(size_t)h * L + l0 + tl];
-      v = db[(size_t)h * L + l0 + tl] * (1.f - gg * gg);
+  {
+    // the tile's 64 rows of dz_tm are contiguous: 16-byte loads
+    const uint4* src = reinterpret_cast<const uint4*>(dz_tm + ((size_t)b * Lp + l0) * (KT * 16));
+    for (int e = threadIdx.x; e < kGtTok * KT * 2; e += kGtThreads) {
+      const int tl = e / (KT * 2), ch = e % (KT * 2);
+      *reinterpret_cast<uint4*>(az + tl * LDZ + ch * 8) = __ldg(src + e);
     }
-    az[tl * LDZ + h] = __float2bfloat16_rn(v);
   }
   __syncthreads();
   uint32_t a[KT][4];
@@ -146,9 +179,23 @@ __global__ void __launch_bounds__(kGtThreads) gate_bwd_dx_kernel(const bf16* __r
   }
   for (int c0 = 0; c0 < C; c0 += kDxCh) {
     __syncthreads();                                           // previous chunk's stores have read st, its products ws
-    for (int e = threadIdx.x; e < kDxCh * KT * 16; e += kGtThreads) {
-      const int c = e / (KT * 16), h = e % (KT * 16);
-      ws[c * LDZ + h] = (h < Hq && c0 + c < C) ? w[(size_t)(c0 + c) * Hq + h] : __float2bfloat16_rn(0.f);
+    if (Hq % 8 == 0 && c0 + kDxCh <= C && (reinterpret_cast<uintptr_t>(w) & 15u) == 0) {
+      // rows of W are whole 16-byte vectors: copy them as such, then clear the padding heads
+      const int vec = Hq / 8;
+      const uint4* src = reinterpret_cast<const uint4*>(w + (size_t)c0 * Hq);
+      for (int e = threadIdx.x; e < kDxCh * vec; e += kGtThreads) {
+        const int c = e / vec, v = e % vec;
+        *reinterpret_cast<uint4*>(ws + c * LDZ + v * 8) = __ldg(src + e);
+      }
+      for (int e = threadIdx.x; e < kDxCh * (KT * 16 - Hq); e += kGtThreads) {
+        const int c = e / (KT * 16 - Hq), h = Hq + e % (KT * 16 - Hq);
+        ws[c * LDZ + h] = __float2bfloat16_rn(0.f);
+      }
+    } else {
+      for (int e = threadIdx.x; e < kDxCh * KT * 16; e += kGtThreads) {
+        const int c = e / (KT * 16), h = e % (KT * 16);
+        ws[c * LDZ + h] = (h < Hq && c0 + c < C) ? w[(size_t)(c0 + c) * Hq + h] : __float2bfloat16_rn(0.f);
+      }
     }
     __syncthreads();
 #pragma unroll 4
@@ -185,8 +232,8 @@ __global__ void __launch_bounds__(kGtThreads) gate_bwd_dx_kernel(const bf16* __r
 // ---------------------------------------------------------------------------------------------- dW_g
 // grid (ceil(C / 128), splits, batch): partial[(b * splits + s)][c][h] = sum over the split's tokens of X[l, c] dz[l, h]
 template <int NT>
-__global__ void __launch_bounds__(kGtThreads) gate_bwd_dw_kernel(const bf16* __restrict__ x, const float* __restrict__ gate,
-                                                                 const float* __restrict__ dgate, int L, int C, int Hq,
+__global__ void __launch_bounds__(kGtThreads) gate_bwd_dw_kernel(const bf16* __restrict__ x, const bf16* __restrict__ dz_hm,
+                                                                 int L, int Lp, int C, int Hq, int HP,
                                                                  float* __restrict__ partial) {
   constexpr int LDZ = kGtTok + 8;
   __shared__ __align__(16) bf16 xs[kGtTok * kLdx];           // [token][channel]; read transposed by ldmatrix
@@ -196,8 +243,7 @@ __global__ void __launch_bounds__(kGtThreads) gate_bwd_dw_kernel(const bf16* __r
   const int per = ((L + splits - 1) / splits + kGtTok - 1) / kGtTok * kGtTok;      // tokens per split, whole tiles
   const int l_beg = s * per, l_end = min(L, l_beg + per);
   const bf16* xb = x + (size_t)b * L * C;
-  const float* gb = gate + (size_t)b * Hq * L;
-  const float* db = dgate + (size_t)b * Hq * L;
+  const bf16* zb = dz_hm + (size_t)b * HP * Lp;
   float acc[2][NT][4];                                        // this warp: channels 32 warp .. + 31 (two tiles of 16)
 #pragma unroll
   for (int m = 0; m < 2; ++m)
@@ -206,7 +252,12 @@ __global__ void __launch_bounds__(kGtThreads) gate_bwd_dw_kernel(const bf16* __r
   for (int l0 = l_beg; l0 < l_end; l0 += kGtTok) {
     __syncthreads();
     load_x_tile(xs, xb, l0, L, c0, C);
-    load_dz_tile(dz, LDZ, NT * 8, gb, db, Hq, l0, L);
+    for (int e = threadIdx.x; e < NT * 8 * (kGtTok / 8); e += kGtThreads) {
+      const int h = e / (kGtTok / 8), ch = e % (kGtTok / 8);
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (h < HP) v = __ldg(reinterpret_cast<const uint4*>(zb + (size_t)h * Lp + l0 + ch * 8));
+      *reinterpret_cast<uint4*>(dz + h * LDZ + ch * 8) = v;
+    }
     __syncthreads();
 #pragma unroll
     for (int ks = 0; ks < kGtTok / 16; ++ks) {
@@ -257,8 +308,15 @@ __global__ void gate_reduce_dw_kernel(const float* __restrict__ partial, int par
 
 bool gate_supported(int hidden, int heads) { return hidden > 0 && hidden % 8 == 0 && heads > 0 && heads <= 64; }
 
-size_t gate_bwd_workspace_bytes(int batch, int hidden, int heads) {
-  return (size_t)batch * kGtSplits * hidden * heads * sizeof(float);
+namespace {
+int padded_heads(int heads) { return (heads + 15) / 16 * 16; }
+int padded_tokens(int L) { return (L + kGtTok - 1) / kGtTok * kGtTok; }
+size_t dz_bytes(int batch, int L, int heads) { return align_up((size_t)batch * padded_tokens(L) * padded_heads(heads) * sizeof(bf16), 256); }
+}  // namespace
+
+// [partial sums of dW_g][dz head-major][dz token-major]
+size_t gate_bwd_workspace_bytes(int batch, int L, int hidden, int heads) {
+  return align_up((size_t)batch * kGtSplits * hidden * heads * sizeof(float), 256) + 2 * dz_bytes(batch, L, heads);
 }
 
 cudaError_t launch_gate_fwd(int batch, int L, int C, int Hq, const bf16* x, const bf16* w, float* gate, cudaStream_t st) {
@@ -276,11 +334,18 @@ cudaError_t launch_gate_fwd(int batch, int L, int C, int Hq, const bf16* x, cons
 }
 
 cudaError_t launch_gate_bwd(int batch, int L, int C, int Hq, int out_f32, const bf16* x, const bf16* w, const float* gate,
-                            const float* dgate, float* d_w, void* dx, float* partial, cudaStream_t st) {
+                            const float* dgate, float* d_w, void* dx, void* workspace, cudaStream_t st) {
+  const int HP = padded_heads(Hq), Lp = padded_tokens(L);
+  float* partial = reinterpret_cast<float*>(workspace);
+  unsigned char* wsb = reinterpret_cast<unsigned char*>(workspace);
+  bf16* dz_hm = reinterpret_cast<bf16*>(wsb + align_up((size_t)batch * kGtSplits * C * Hq * sizeof(float), 256));
+  bf16* dz_tm = reinterpret_cast<bf16*>(reinterpret_cast<unsigned char*>(dz_hm) + dz_bytes(batch, L, Hq));
+  gate_dz_kernel<<<dim3(Lp / kGtTok, batch), kGtThreads, (size_t)HP * (kGtTok + 8) * sizeof(bf16), st>>>(gate, dgate, L, Lp, Hq,
+                                                                                                   HP, dz_hm, dz_tm);
   {
     dim3 grid((L + kGtTok - 1) / kGtTok, batch);
     const int kt = (Hq + 15) / 16;
-#define VSA2_GATE_DX(KT_) gate_bwd_dx_kernel<KT_><<<grid, kGtThreads, 0, st>>>(w, gate, dgate, L, C, Hq, out_f32, dx)
+#define VSA2_GATE_DX(KT_) gate_bwd_dx_kernel<KT_><<<grid, kGtThreads, 0, st>>>(w, dz_tm, L, Lp, C, Hq, out_f32, dx)
     if (kt <= 1) VSA2_GATE_DX(1);
     else if (kt <= 2) VSA2_GATE_DX(2);
     else if (kt <= 3) VSA2_GATE_DX(3);
@@ -290,7 +355,7 @@ cudaError_t launch_gate_bwd(int batch, int L, int C, int Hq, int out_f32, const 
   {
     dim3 grid((C + kGtCh - 1) / kGtCh, kGtSplits, batch);
     const int nt = (Hq + 7) / 8;
-#define VSA2_GATE_DW(NT_) gate_bwd_dw_kernel<NT_><<<grid, kGtThreads, 0, st>>>(x, gate, dgate, L, C, Hq, partial)
+#define VSA2_GATE_DW(NT_) gate_bwd_dw_kernel<NT_><<<grid, kGtThreads, 0, st>>>(x, dz_hm, L, Lp, C, Hq, HP, partial)
     if (nt <= 1) VSA2_GATE_DW(1);
     else if (nt <= 2) VSA2_GATE_DW(2);
     else if (nt <= 4) VSA2_GATE_DW(4);

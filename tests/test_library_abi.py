@@ -132,5 +132,5 @@ def test_gate_entry_points_reject_unsupported_shapes_before_any_cuda_call():
     many = vb.make_params(batch=1, heads_q=80, heads_kv=80, head_dim=64, grid=(2, 4, 8), topk=1)
     assert lib.vsa2_gate_fwd(ctypes.byref(many), 64, one, one, one, None) == vb.ERR_UNSUPPORTED       # more than 64 heads
     assert vb.vsa2_gate_bwd_workspace_bytes(many, 64) == 0
-    assert vb.vsa2_gate_bwd_workspace_bytes(p, 64) == 16 * 64 * 8 * 4
+    assert vb.vsa2_gate_bwd_workspace_bytes(p, 64) == 16 * 64 * 8 * 4 + 2 * 64 * 16 * 2      # dW_g partials + dz in two layouts
     assert lib.vsa2_gate_bwd(ctypes.byref(p), 64, one, one, one, one, one, one, one, 100, None) == vb.ERR_WORKSPACE_TOO_SMALL
