@@ -80,16 +80,6 @@ __device__ __forceinline__ int cube_token(const Geo& g, int nt, int nh, int nw, 
   return cube_token_at(g, nt, nh, nw, bt, bh, bw);
 }
 
-// 64-bit mask of the valid positions of cube n
-__device__ __forceinline__ unsigned long long cube_valid_mask(const Geo& g, int n) {
-  int nt, nh, nw;
-  cube_coords(g, n, nt, nh, nw);
-  unsigned long long m = 0ull;
-  for (int p = 0; p < kBlockTokens; ++p)
-    if (cube_token(g, nt, nh, nw, p) >= 0) m |= 1ull << p;
-  return m;
-}
-
 // number of valid tokens of cube n (0 only for the empty trailing half-cubes of a 128-token-cube problem)
 __device__ __forceinline__ int cube_count(const Geo& g, int n) {
   int nt, nh, nw;
@@ -114,11 +104,6 @@ __device__ __forceinline__ int subcube_count(const Geo& g, int n, int gsub) {
 __device__ __forceinline__ void store_out(void* base, size_t idx, float v, int out_f32) {
   if (out_f32) reinterpret_cast<float*>(base)[idx] = v;
   else reinterpret_cast<bf16*>(base)[idx] = __float2bfloat16_rn(v);
-}
-
-__device__ __forceinline__ float load_out(const void* base, size_t idx, int out_f32) {
-  return out_f32 ? reinterpret_cast<const float*>(base)[idx]
-                 : __bfloat162float(reinterpret_cast<const bf16*>(base)[idx]);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -18,15 +18,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
-// swizzled index into a 128 x 64 fp32 reduction scratch (row r written by one thread, column c read by one)
-__device__ __forceinline__ int scratch_idx(int r, int c) { return r * 64 + (c ^ (r & 31)); }
-
-__device__ __forceinline__ bool pos_valid(const Geo& g, int n, int pos) {
-  int nt, nh, nw;
-  cube_coords(g, n, nt, nh, nw);
-  return cube_token(g, nt, nh, nw, pos) >= 0;
-}
-
 // 64 bf16 (32 packed words) -> one 128-byte row of a swizzled operand tile: 16-byte chunk c lands at c ^ (row & 7)
 __device__ __forceinline__ void store_row_sw128(unsigned char* tile, int row, const uint32_t (&packed)[32]) {
   unsigned char* prow = tile + row * 128;
