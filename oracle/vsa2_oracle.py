@@ -378,16 +378,22 @@ def head_backward(Q, K, V, gate, mask, geo: Geometry, scale, dO, fwd=None):
 # ----------------------------------------------------------------------------
 # multi-head wrappers ([B, H, L, D] arrays; query head hq uses KV head hq // (Hq/Hkv))
 # ----------------------------------------------------------------------------
-def route(Q, K, geo: Geometry, scale, mode, topk=0, budgets=None, return_scores=False):
+def route(Q, K, geo: Geometry, scale, mode, topk=0, budgets=None, return_scores=False, share_group=False):
     """Q [B, Hq, L, D], K [B, Hkv, L, D] -> mask [B, Hq, N, N] (and P_r if asked).
 
     Each query head routes on its own against its KV head's pooled keys; the
     budget N*K holds per (batch, query head).
+
+    share_group: the "group head" pattern of the ablation in Sec. 4 -- the query
+    heads of one KV group share one map.  The block scores of the group's heads
+    are added (the paper does not say how the heads are combined; the sum, or
+    equivalently the mean, is the reading taken) and the TopK runs once per
+    group; the scores returned are then the group sums, repeated per head.
     """
     Bn, Hq = Q.shape[:2]
     rep = Hq // K.shape[1]
     masks = np.zeros((Bn, Hq, geo.N, geo.N), dtype=bool)
-    scores = np.zeros((Bn, Hq, geo.N, geo.N), dtype=np.float64) if return_scores else None
+    scores = np.zeros((Bn, Hq, geo.N, geo.N), dtype=np.float64)
     for b in range(Bn):
         kr_cache = {}
         for hq in range(Hq):
@@ -396,11 +402,16 @@ def route(Q, K, geo: Geometry, scale, mode, topk=0, budgets=None, return_scores=
                 kr_cache[hk] = mean_pool_router(K[b, hk], geo)
             Kr, kv = kr_cache[hk]
             Qr, qv = mean_pool_router(Q[b, hq], geo)
-            P_r = router_block_scores(Qr, Kr, qv, kv, scale)
+            scores[b, hq] = router_block_scores(Qr, Kr, qv, kv, scale)
+        if share_group:
+            if budgets is not None:
+                raise ValueError("per-row budgets belong to single heads: not defined for shared maps")
+            for hk in range(Hq // rep):
+                grp = slice(hk * rep, (hk + 1) * rep)
+                scores[b, grp] = scores[b, grp].sum(axis=0, keepdims=True)
+        for hq in range(Hq):
             bud = None if budgets is None else budgets[b, hq]
-            masks[b, hq] = select_blocks(P_r, mode, topk, bud)
-            if return_scores:
-                scores[b, hq] = P_r
+            masks[b, hq] = select_blocks(scores[b, hq], mode, topk, bud)
     return (masks, scores) if return_scores else masks
 
 

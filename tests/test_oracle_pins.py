@@ -497,3 +497,27 @@ def test_gate_projection_matches_autograd_and_its_special_cases():
     assert abs((f(X, Wp) - f(X, Wm)) / (2 * h) - dW[3, 2]) < 1e-6
     Xp, Xm = X.copy(), X.copy(); Xp[11, 7] += h; Xm[11, 7] -= h
     assert abs((f(Xp, Wg) - f(Xm, Wg)) / (2 * h) - dX[11, 7]) < 1e-6
+
+
+def test_group_shared_routing_is_the_topk_of_the_summed_head_scores():
+    """Sec. 4 "Group Head": the query heads of a KV group share one map.  Pins: identical masks inside a group, equal to the
+    brute-force TopK of the summed per-head scores; one head per group changes nothing; other groups are untouched."""
+    rng = np.random.default_rng(23)
+    geo = orc.Geometry((4, 8, 8), (4, 4, 4), (2, 2, 2))
+    L, D, Hq, Hkv = geo.L, 16, 4, 2
+    Q = rng.standard_normal((1, Hq, L, D)).astype(np.float32).astype(np.float64)
+    K = rng.standard_normal((1, Hkv, L, D)).astype(np.float32).astype(np.float64)
+    own, P = orc.route(Q, K, geo, 0.25, orc.PER_SEQUENCE, 2, return_scores=True)
+    shared, Pg = orc.route(Q, K, geo, 0.25, orc.PER_SEQUENCE, 2, return_scores=True, share_group=True)
+    for hk in range(Hkv):
+        a, b = 2 * hk, 2 * hk + 1
+        assert np.array_equal(shared[0, a], shared[0, b])
+        summed = (P[0, a] + P[0, b]).astype(np.float32)
+        np.testing.assert_allclose(Pg[0, a], P[0, a] + P[0, b], rtol=1e-14)
+        keep = _brute_topk(summed.reshape(-1), geo.N * 2)
+        assert set(np.nonzero(shared[0, a].reshape(-1))[0].tolist()) == keep
+        assert shared[0, a].sum() == geo.N * 2
+    assert not np.array_equal(own[0, 0], own[0, 1])                      # the heads would have chosen differently
+    # a group of one head is the ordinary routing
+    same = orc.route(Q[:, :2], K, geo, 0.25, orc.PER_QUERY, 3, share_group=True)
+    assert np.array_equal(same, orc.route(Q[:, :2], K, geo, 0.25, orc.PER_QUERY, 3))
