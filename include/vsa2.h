@@ -72,6 +72,10 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
 enum { VSA2_FLAG_HALF_CUBE_FWD = 128 };/* 128-token cubes only: fine forward with the 64-query kernel on the two half-cubes
                                          separately instead of the 128-query kernel (validation aid, same results) */
+enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV group share one block map ("group head", Sec. 4
+                                         ablation): the block scores of the group's heads are added before the TopK, so
+                                         the maps written for those heads are identical.  Not with VSA2_PER_QUERY_BUDGET
+                                         (budgets belong to single heads): VSA2_ERR_UNSUPPORTED */
 enum { VSA2_FLAG_SIMPLE_COARSE = 16 };/* validation aid: coarse branch (forward and backward) with the fp32 SIMT kernels
                                          instead of the TF32 tensor-core ones */
 enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */

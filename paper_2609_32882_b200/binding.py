@@ -25,6 +25,7 @@ FLAG_SIMPLE_COARSE = 16
 FLAG_TF32_COARSE = 32
 FLAG_BF16_COARSE_FWD = 64
 FLAG_HALF_CUBE_FWD = 128
+FLAG_GROUP_ROUTING = 256
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4

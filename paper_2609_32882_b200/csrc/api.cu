@@ -266,6 +266,7 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
   if (!q || !k || !map || !workspace || !map->row_ptr || !map->col_idx || !map->col_ptr || !map->row_idx)
     return VSA2_ERR_INVALID_ARG;
   if (g.mode == VSA2_PER_QUERY_BUDGET && budgets == nullptr) return VSA2_ERR_INVALID_ARG;
+  if (g.mode == VSA2_PER_QUERY_BUDGET && (g.flags & VSA2_FLAG_GROUP_ROUTING)) return VSA2_ERR_UNSUPPORTED;
   if (!aligned16(q) || !aligned16(k) || !aligned256(workspace)) return VSA2_ERR_MISALIGNED;
   if (workspace_bytes < route_workspace_bytes(g)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
   if ((rc = check_device()) != VSA2_OK) return rc;
@@ -301,6 +302,10 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
     float* pr_cube = at<float>(sel_base, lay.pr);
     VSA2_CUDA(launch_fold_scores(r, pr, pr_cube, st));
     pr = pr_cube;
+  }
+  if ((g.flags & VSA2_FLAG_GROUP_ROUTING) && g.rep > 1) {
+    g_launches += 1;
+    VSA2_CUDA(launch_group_sum_scores(g, pr, st));
   }
   workspace = sel_base;
   SelectScratch s;

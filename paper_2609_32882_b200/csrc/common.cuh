@@ -169,6 +169,8 @@ cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float*
 bool wide_cube(const Geo& g);
 Geo narrow_geo(const Geo& g);
 cudaError_t launch_fold_scores(const Geo& narrow, const float* pr64, float* pr, cudaStream_t st);
+// "group head" routing: replaces every block score by the sum over the query heads of its KV group (in place)
+cudaError_t launch_group_sum_scores(const Geo& g, float* pr, cudaStream_t st);
 cudaError_t launch_fold_mean(const Geo& narrow, int heads, const float* x64, float* x, cudaStream_t st);
 cudaError_t launch_fold_sum(const Geo& narrow, int heads, const float* x64, float* x, cudaStream_t st);
 cudaError_t launch_expand_rows(const Geo& narrow, int heads, bool by_count, const float* x, float* x64,

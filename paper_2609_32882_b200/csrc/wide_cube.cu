@@ -123,12 +123,31 @@ __global__ void __launch_bounds__(128) expand_map_kernel(int N, int Hq, long lon
   }
 }
 
+// "group head" routing: the query heads of a KV group share one map.  pr [batch, Hq, N, N]: every entry is replaced by
+// the sum over the heads of its group (added in head order), so the selection that follows picks the same set for each
+__global__ void __launch_bounds__(256) group_sum_scores_kernel(float* __restrict__ pr, int rep, size_t per_head, size_t groups) {
+  const size_t total = groups * per_head;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t grp = e / per_head, off = e % per_head;
+    float* base = pr + grp * rep * per_head + off;
+    float sum = 0.f;
+    for (int r = 0; r < rep; ++r) sum += base[(size_t)r * per_head];
+    for (int r = 0; r < rep; ++r) base[(size_t)r * per_head] = sum;
+  }
+}
+
 int grid_for(size_t total) {
   size_t blocks = (total + 255) / 256;
   return (int)(blocks < 148 * 16 ? (blocks ? blocks : 1) : 148 * 16);
 }
 
 }  // namespace
+
+cudaError_t launch_group_sum_scores(const Geo& g, float* pr, cudaStream_t st) {
+  const size_t per_head = (size_t)g.N * g.N, groups = (size_t)g.batch * g.Hkv;
+  group_sum_scores_kernel<<<grid_for(groups * per_head), 256, 0, st>>>(pr, g.rep, per_head, groups);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_fold_scores(const Geo& narrow, const float* pr64, float* pr, cudaStream_t st) {
   const int N = narrow.N / 2;

@@ -257,3 +257,46 @@ def test_bf16_coarse_forward_flag_keeps_the_output_bound():
         O, lse = run.forward()
         assert_close("O", O, O_ref)
         assert_lse_close(lse, lse_ref)
+
+
+@pytest.mark.parametrize("wl", [
+    syn.Workload("shared_gqa", 1, 8, 2, 128, (5, 6, 9), select_mode=syn.PER_SEQUENCE, topk=3, seed=31),
+    syn.Workload("shared_gqa_rows", 2, 4, 2, 64, (6, 9, 10), select_mode=syn.PER_QUERY, topk=4, seed=32),
+    syn.Workload("shared_gqa_wide", 1, 4, 2, 128, (7, 10, 28), cube=(4, 4, 8), select_mode=syn.PER_SEQUENCE, topk=8, seed=33),
+], ids=lambda w: w.name)
+def test_group_shared_routing(wl):
+    """VSA2_FLAG_GROUP_ROUTING: one map per KV group, selected on the summed scores of the group's heads; the attention
+    forward and backward then run on those maps as on any other."""
+    data = syn.make_inputs(wl)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    a = oracle_arrays(data)
+    run = CudaPath(wl, data, flags=vb.FLAG_GROUP_ROUTING)
+    gmask = run.route()
+    omask, P = orc.route(a["q"], a["k"], geo, scale, wl.select_mode, wl.topk, return_scores=True, share_group=True)
+    rep = wl.heads_q // wl.heads_kv
+    for b in range(wl.batch):
+        for h in range(wl.heads_q):
+            assert np.array_equal(gmask[b, h], gmask[b, h - h % rep])            # identical inside a group
+            check_routing(gmask[b, h], omask[b, h], P[b, h], wl.select_mode)
+    pr_gpu = to_f64(run.attn.scores())
+    assert np.abs(pr_gpu - P).max() <= 1e-4 * P.max()
+    O, lse = run.forward()
+    O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale)
+    assert_close("O", O, O_ref, bf16_storage=True)
+    assert_lse_close(lse, lse_ref)
+    got = run.backward()
+    want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
+    for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
+        tol = TOL_ABS * (np.sqrt(rep) if name in ("dK", "dV") else 1.0)
+        assert_close(name, x, y, tol_abs=tol, bf16_storage=name != "dGate")
+
+
+def test_group_shared_routing_is_refused_for_per_row_budgets():
+    wl = MINI_BUDGET
+    data = syn.make_inputs(wl)
+    data["budgets"] = np.full((1, 2, wl.n_cubes), 2, dtype=np.int32)
+    run = CudaPath(wl, data, flags=vb.FLAG_GROUP_ROUTING, nnz_cap=2 * wl.n_cubes)
+    with pytest.raises(vb.Vsa2Error) as e:
+        run.route()
+    assert e.value.code == vb.ERR_UNSUPPORTED
