@@ -75,7 +75,9 @@ enum { VSA2_FLAG_HALF_CUBE_FWD = 128 };/* 128-token cubes only: fine forward wit
 enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV group share one block map ("group head", Sec. 4
                                          ablation): the block scores of the group's heads are added before the TopK, so
                                          the maps written for those heads are identical.  Not with VSA2_PER_QUERY_BUDGET
-                                         (budgets belong to single heads): VSA2_ERR_UNSUPPORTED */
+                                         (budgets belong to single heads): VSA2_ERR_UNSUPPORTED.
+                                         vsa2_attn_fwd with this flag RELIES on that: with an even number of query heads
+                                         per KV head it reads the map of the first head of each pair of heads only */
 enum { VSA2_FLAG_SIMPLE_COARSE = 16 };/* validation aid: coarse branch (forward and backward) with the fp32 SIMT kernels
                                          instead of the TF32 tensor-core ones */
 enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */

@@ -67,6 +67,8 @@ struct FwdWideMisc {
 static_assert(sizeof(FwdWideMisc) <= 6144, "misc region too small");
 
 struct FwdWideArgs {
+  int pair_heads;       // 0: an item is a query cube of 128 tokens (two half-cubes of one head); 1: an item is one query
+                        // block of two consecutive query heads of a KV group whose maps are identical
   int* item_counter;    // global, zero before the launch
   const float* gate;
   const int* row_ptr;   // expanded map (half-cube level)
@@ -79,6 +81,27 @@ struct FwdWideArgs {
   int* rescue_count;
   int* rescue_items;
 };
+
+// The two "members" of an item share their list of key blocks: member m is query block i0 + m * di of head bhq0 + m * dh;
+// the list is row i0 of head bhq0.
+struct WideItem {
+  int bhq0, i0, dh, di;
+};
+__device__ __forceinline__ WideItem decode_item(const Geo& g, int pair_heads, int item) {
+  WideItem w;
+  if (pair_heads) {
+    w.i0 = item % g.N;
+    w.bhq0 = (item / g.N) * 2;
+    w.dh = 1;
+    w.di = 0;
+  } else {
+    w.i0 = (item % (g.N / 2)) * 2;
+    w.bhq0 = item / (g.N / 2);
+    w.dh = 0;
+    w.di = 1;
+  }
+  return w;
+}
 
 // acc[128, 128] = A_pair[128, D] * B_pair[128, D]^T, both operands in the [channel half][block A | block B] layout
 template <int D>
@@ -121,8 +144,7 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;      // edge flags of every half-cube
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_cubes = g.N / 2;                                   // g is the half-cube geometry
-  const int total_items = g.batch * g.Hq * n_cubes;
+  const int total_items = g.batch * g.Hq * g.N / 2;              // pairs of query blocks either way
   const float c2 = g.scale * 1.4426950408889634f;
 
   for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
@@ -185,15 +207,17 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         item = __shfl_sync(0xffffffffu, item, 0);
         if (item == -2) goto done;
         if (item < 0) break;
-        const int c = item % n_cubes, bhq = item / n_cubes;
+        const WideItem wi = decode_item(g, a.pair_heads, item);
+        const int bhq = wi.bhq0;
         const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
-        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c], end = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1];
-        const int nt = (end - beg) >> 1;                    // the expanded list holds both halves of every key cube
+        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + wi.i0], end = a.row_ptr[(size_t)bhq * (g.N + 1) + wi.i0 + 1];
+        const int k = end - beg;
+        const int nt = (k + 1) >> 1;                        // two key blocks per tile (an odd list repeats its last block)
         if (nt == 0) continue;
         const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
         if (which == 0) {
           int it_, ih_, iw_;
-          cube_coords(g, 2 * c + my_blk, it_, ih_, iw_);
+          cube_coords(g, wi.i0 + my_blk * wi.di, it_, ih_, iw_);
           int ok = 1;
           if (lane == 0) {
             ok = tc::mbar_wait(&misc->q_empty, (n_items & 1) ^ 1, &misc->abort_flag);
@@ -202,14 +226,14 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
           if (issuer)
             tc::tma_load_5d(q_tile + (2 * my_h + my_blk) * C::SLAB, &tm_q, &misc->q_full, my_h * 64, iw_ * g.Bw, ih_ * g.Bh,
-                            it_ * g.Bt, bhq);
+                            it_ * g.Bt, bhq + my_blk * wi.dh);
         }
         ++n_items;
-        int j = cols[my_blk];
+        int j = cols[(my_blk == 1 && k > 1) ? 1 : 0];
         for (int t = 0; t < nt; ++t, ++tg) {
           int jt, jh, jw;
           cube_coords(g, j, jt, jh, jw);
-          if (t + 1 < nt) j = cols[2 * t + 2 + my_blk];        // next tile, fetched early
+          if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];   // next tile, fetched early
           const uint32_t slot = tg % nslots, par = (tg / nslots) & 1;
           int ok = 1;
           if (lane == 0) {
@@ -229,8 +253,8 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         uint32_t tg = 0, n_items = 0;
         for (uint32_t seq = 0;; ++seq) {
           VSA2_NEXT_ITEM(item, seq);
-          const int c = item % n_cubes, bhq = item / n_cubes;
-          const int nt = (a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c]) >> 1;
+          const WideItem wi = decode_item(g, a.pair_heads, item);
+          const int nt = (a.row_ptr[(size_t)wi.bhq0 * (g.N + 1) + wi.i0 + 1] - a.row_ptr[(size_t)wi.bhq0 * (g.N + 1) + wi.i0] + 1) >> 1;
           if (nt == 0) continue;
           VSA2_WAIT(&misc->q_full, n_items & 1);
           for (int t = 0; t < nt; ++t, ++tg) {
@@ -254,8 +278,8 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         uint32_t tg = 0, n_items = 0;
         for (uint32_t seq = 0;; ++seq) {
           VSA2_NEXT_ITEM(item, seq);
-          const int c = item % n_cubes, bhq = item / n_cubes;
-          const int nt = (a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c]) >> 1;
+          const WideItem wi = decode_item(g, a.pair_heads, item);
+          const int nt = (a.row_ptr[(size_t)wi.bhq0 * (g.N + 1) + wi.i0 + 1] - a.row_ptr[(size_t)wi.bhq0 * (g.N + 1) + wi.i0] + 1) >> 1;
           if (nt == 0) continue;
           VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous cube's accumulator was read out
           for (int t = 0; t < nt; ++t, ++tg) {
@@ -291,11 +315,13 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     uint32_t tg = 0, n_items = 0, n_all = 0, wg_phase = 0;
     for (;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
-      const int c = item % n_cubes, bhq = item / n_cubes;
-      const int i = 2 * c + half;                // query half-cube of this warpgroup
-      const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c], end = a.row_ptr[(size_t)bhq * (g.N + 1) + 2 * c + 1];
-      const int nt = (end - beg) >> 1;
-      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+      const WideItem wi = decode_item(g, a.pair_heads, item);
+      const int bhq = wi.bhq0 + half * wi.dh;    // head and query block of this warpgroup's member
+      const int i = wi.i0 + half * wi.di;
+      const int beg = a.row_ptr[(size_t)wi.bhq0 * (g.N + 1) + wi.i0], end = a.row_ptr[(size_t)wi.bhq0 * (g.N + 1) + wi.i0 + 1];
+      const int k = end - beg;
+      const int nt = (k + 1) >> 1;
+      const int* cols = a.col_idx + (size_t)wi.bhq0 * g.nnz_cap + beg;
       const int tb = n_all & 1;
       if (sm_tid < 32) {
         int it_, ih_, iw_;
@@ -314,7 +340,7 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       if (nt > 0) {
         // reference exponent of this warpgroup's query columns = exact column maximum of the first tile
         const uint32_t buf = tg % kFwwSBufs;
-        const bool valid = cpos.valid(edge[cols[blk]], g);
+        const bool valid = !((blk == 1) && k < 2) && cpos.valid(edge[cols[(blk == 1 && k > 1) ? 1 : 0]], g);
         VSA2_WAIT(&misc->s_full[buf], (tg / kFwwSBufs) & 1);
         tc::tc_fence_after();
         uint32_t s0[32];
@@ -335,11 +361,12 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       VSA2_GROUP_SYNC(&misc->wg_sync[wg], wg_phase);       // tables and reference exponents visible to the warpgroup
 
       if (nt > 0) {
-        int j_next = cols[blk];
+        int j_next = cols[(blk == 1 && k > 1) ? 1 : 0];
         for (int t = 0; t < nt; ++t) {
           const uint32_t tgt = tg0 + t, buf = tgt % kFwwSBufs;
-          const bool valid = cpos.valid(edge[j_next], g);
-          if (t + 1 < nt) j_next = cols[2 * t + 2 + blk];
+          const bool dup = (blk == 1) && (2 * t + 1 >= k);       // odd list: the last tile holds one key block twice
+          const bool valid = !dup && cpos.valid(edge[j_next], g);
+          if (t + 1 < nt) j_next = cols[(blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
           const bool all_valid = __all_sync(0xffffffffu, valid);
           VSA2_WAIT(&misc->s_full[buf], (tgt / kFwwSBufs) & 1);
           tc::tc_fence_after();
@@ -485,8 +512,10 @@ cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* item
                                  const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
                                  const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
 
-// `g`: half-cube geometry; row_ptr / col_idx: the expanded map; oc_hat: per half-cube.  workspace as for the N = 64 launcher.
-cudaError_t launch_fine_fwd_wide_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+// pair_heads = false: `g` is the half-cube geometry of a 128-token-cube problem, row_ptr / col_idx the expanded map, oc_hat per
+// half-cube.  pair_heads = true: `g` is an ordinary 64-token-cube problem with an even number of query heads per KV head whose
+// maps are identical inside each group (group-shared routing); consecutive heads are paired.  Workspace as for the N = 64 launcher.
+cudaError_t launch_fine_fwd_wide_tc(const Geo& g, bool pair_heads, const bf16* q, const bf16* k, const bf16* v, const float* gate,
                                     const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                     float* lse, StatusBlock* status, cudaStream_t st) {
   CUtensorMap tq, tk, tv;
@@ -498,14 +527,15 @@ cudaError_t launch_fine_fwd_wide_tc(const Geo& g, const bf16* q, const bf16* k, 
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   if (fine_fwd_tc_workspace_bytes() < 256 + (size_t)kFwwRescueCap * sizeof(int)) return cudaErrorInvalidValue;
   FwdWideArgs a;
+  a.pair_heads = pair_heads ? 1 : 0;
   a.gate = gate; a.row_ptr = row_ptr; a.col_idx = col_idx; a.oc_hat = oc_hat; a.o = o; a.o_res = o_res; a.lse = lse;
   a.status = status;
   a.rescue_count = &status->pad[0];
   a.item_counter = &status->pad[1];
   a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
-  const int total = g.batch * g.Hq * (g.N / 2);
+  const int total = g.batch * g.Hq * g.N / 2;         // pairs of query blocks (Hq or N is even)
   const int grid = total < sms ? total : sms;
-  if (g.N > kFwwMaxCubes || (g.N & 1)) return cudaErrorInvalidValue;
+  if (g.N > kFwwMaxCubes || (pair_heads ? (g.rep & 1) : (g.N & 1))) return cudaErrorInvalidValue;
   if (g.D == 128) {
     const size_t smb = FwdWide<128>::smem_bytes(g.N);
     if (smb > 227 * 1024) return cudaErrorInvalidValue;
