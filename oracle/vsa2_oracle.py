@@ -107,6 +107,28 @@ class Geometry:
 
 
 # ----------------------------------------------------------------------------
+# Sec. 2.2 "Permutation": cube-major token order
+# ----------------------------------------------------------------------------
+def to_cube_major(X: np.ndarray, geo: Geometry, fill=0.0) -> np.ndarray:
+    """X [L, D] in raster order -> [N * B, D]: cube n occupies rows n*B .. n*B + B - 1, its tokens in (b_t, b_h, b_w)
+    order; positions outside the grid hold `fill`."""
+    Y = np.full((geo.N * geo.B, X.shape[1]), fill, dtype=X.dtype)
+    l = np.arange(geo.L)
+    t, h, w = l // (geo.H * geo.W), (l // geo.W) % geo.H, l % geo.W
+    pos = ((t % geo.Bt) * geo.Bh + (h % geo.Bh)) * geo.Bw + (w % geo.Bw)
+    Y[geo.cube_of * geo.B + pos] = X
+    return Y
+
+
+def from_cube_major(Y: np.ndarray, geo: Geometry) -> np.ndarray:
+    """Inverse of to_cube_major on the valid tokens: [N * B, D] -> [L, D]."""
+    l = np.arange(geo.L)
+    t, h, w = l // (geo.H * geo.W), (l // geo.W) % geo.H, l % geo.W
+    pos = ((t % geo.Bt) * geo.Bh + (h % geo.Bh)) * geo.Bw + (w % geo.Bw)
+    return Y[geo.cube_of * geo.B + pos]
+
+
+# ----------------------------------------------------------------------------
 # Eq. 1: coarse mean pooling over cubes
 # ----------------------------------------------------------------------------
 def mean_pool_cube(X: np.ndarray, geo: Geometry) -> np.ndarray:

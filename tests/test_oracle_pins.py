@@ -521,3 +521,19 @@ def test_group_shared_routing_is_the_topk_of_the_summed_head_scores():
     # a group of one head is the ordinary routing
     same = orc.route(Q[:, :2], K, geo, 0.25, orc.PER_QUERY, 3, share_group=True)
     assert np.array_equal(same, orc.route(Q[:, :2], K, geo, 0.25, orc.PER_QUERY, 3))
+
+
+@pytest.mark.parametrize("grid,cube", [((4, 8, 8), (4, 4, 4)), ((5, 6, 9), (4, 4, 4)), ((3, 5, 13), (2, 4, 8))])
+def test_cube_major_permutation_matches_a_reshape_of_the_padded_volume(grid, cube):
+    """Sec. 2.2 "Permutation": (T, H, W) -> (N_t N_h N_w) x (B_t B_h B_w).  Pinned against a reshape / transpose of the
+    zero-padded volume (numpy routines), the cube token lists, and its own inverse."""
+    geo = orc.Geometry(grid, cube, (1, 1, 1))
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((geo.L, 6))
+    Y = orc.to_cube_major(X, geo, fill=0.0)
+    vol = pad_volume(X, grid, cube)
+    np.testing.assert_array_equal(Y, to_cube_major(vol, cube).reshape(geo.N * geo.B, 6))
+    for n in (0, geo.N - 1):
+        rows = Y[n * geo.B:(n + 1) * geo.B]
+        np.testing.assert_array_equal(rows[np.abs(rows).sum(axis=1) > 0], X[geo.cube_tokens[n]])
+    np.testing.assert_array_equal(orc.from_cube_major(Y, geo), X)
