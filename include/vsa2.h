@@ -205,6 +205,16 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
                   const void* d_o, void* dq, void* dk, void* dv, float* dgate,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Cube-major copy of a tensor (Sec. 2.2 "Permutation": (T, H, W) -> (N_t N_h N_w) x (B_t B_h B_w)), for callers whose
+ * surrounding code works in that layout; the entry points above take the raster layout and never need it.
+ *   inverse == 0: src [batch, heads, L, D] raster -> dst [batch, heads, N * B, D]; cube n occupies rows n*B .. n*B+B-1, its
+ *                 tokens in (b_t, b_h, b_w) order, positions outside the grid are written as zero
+ *   inverse != 0: src [batch, heads, N * B, D] -> dst [batch, heads, L, D] (positions outside the grid are dropped)
+ * Both bf16, device, 16-byte aligned; `heads` is heads_q or heads_kv of `p`; N and B as in vsa2_query_sizes.  Allocates
+ * nothing; enqueues on `cuda_stream`. */
+int vsa2_permute_cube_major(const vsa2_params* p, int32_t heads, int32_t inverse, const void* src, void* dst,
+                            void* cuda_stream);
+
 /* Gate projection of the gated merge (Sec. 2.2 "Gated Merge", Eq. 13): gate[b, h, l] = tanh(sum_c x[b, l, c] * w_g[c, h]),
  * one column of W_g per query head.  The layer that owns the hidden states calls this before vsa2_attn_fwd (which takes
  * the gate as an input) and vsa2_gate_bwd after vsa2_attn_bwd (which returns dgate).

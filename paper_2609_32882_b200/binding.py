@@ -34,7 +34,7 @@ ERR_STATIC_SCRATCH = -8
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
            "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc", "vsa2_last_cuda_error",
-           "vsa2_gate_fwd", "vsa2_gate_bwd", "vsa2_gate_bwd_workspace_bytes")
+           "vsa2_gate_fwd", "vsa2_gate_bwd", "vsa2_gate_bwd_workspace_bytes", "vsa2_permute_cube_major")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv")
@@ -92,6 +92,7 @@ def _lib():
         lib.vsa2_query_sizes.argtypes = [C.POINTER(Params), C.POINTER(Sizes)]
         lib.vsa2_route.argtypes = [C.POINTER(Params), vp, vp, vp, C.POINTER(Map), vp, sz, vp]
         lib.vsa2_route_noalloc.argtypes = [C.POINTER(Params), vp, vp, vp, C.POINTER(Map), vp, vp]
+        lib.vsa2_permute_cube_major.argtypes = [C.POINTER(Params), C.c_int32, C.c_int32, vp, vp, vp]
         lib.vsa2_gate_fwd.argtypes = [C.POINTER(Params), C.c_int32, vp, vp, vp, vp]
         lib.vsa2_gate_bwd_workspace_bytes.argtypes = [C.POINTER(Params), C.c_int32]
         lib.vsa2_gate_bwd_workspace_bytes.restype = C.c_size_t
@@ -178,6 +179,12 @@ def vsa2_route_noalloc(p, q, k, budgets, vmap: Map, device_status=None, stream=N
     Vsa2Error(ERR_STATIC_SCRATCH).  `device_status`: optional int32 CUDA tensor receiving the status word."""
     _check(_lib().vsa2_route_noalloc(C.byref(p), _ptr(q), _ptr(k), _ptr(budgets), C.byref(vmap), _ptr(device_status),
                                      _stream(stream)), "vsa2_route_noalloc")
+
+
+def vsa2_permute_cube_major(p, heads, src, dst, inverse=False, stream=None):
+    """Raster [B, heads, L, D] -> cube-major [B, heads, N*B, D] (zero padding), or back with inverse=True; bf16."""
+    _check(_lib().vsa2_permute_cube_major(C.byref(p), heads, 1 if inverse else 0, _ptr(src), _ptr(dst), _stream(stream)),
+           "vsa2_permute_cube_major")
 
 
 def vsa2_gate_fwd(p, hidden, x, w_g, gate, stream=None):

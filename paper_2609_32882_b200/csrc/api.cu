@@ -531,6 +531,20 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   return VSA2_OK;
 }
 
+int vsa2_permute_cube_major(const vsa2_params* p, int32_t heads, int32_t inverse, const void* src, void* dst,
+                            void* cuda_stream) {
+  Geo g;
+  int rc = fill_geo(p, &g);
+  if (rc != VSA2_OK) return rc;
+  if (!src || !dst || heads <= 0 || heads > 65535) return VSA2_ERR_INVALID_ARG;
+  if (!aligned16(src) || !aligned16(dst)) return VSA2_ERR_MISALIGNED;
+  if ((rc = check_device()) != VSA2_OK) return rc;
+  g_launches += 1;
+  VSA2_CUDA(launch_permute(g, reinterpret_cast<const bf16*>(src), heads, inverse != 0, reinterpret_cast<bf16*>(dst),
+                           reinterpret_cast<cudaStream_t>(cuda_stream)));
+  return VSA2_OK;
+}
+
 int vsa2_gate_fwd(const vsa2_params* p, int32_t hidden, const void* x, const void* w_g, float* gate, void* cuda_stream) {
   Geo g;
   int rc = fill_geo(p, &g);

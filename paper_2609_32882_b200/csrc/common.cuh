@@ -111,6 +111,9 @@ __device__ __forceinline__ void store_out(void* base, size_t idx, float v, int o
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_pool(const Geo& g, const bf16* x, int heads, bf16* xr, float* xc, cudaStream_t st);
 
+// raster <-> cube-major copy of a [batch, heads, L or N*B, D] bf16 tensor (pool.cu)
+cudaError_t launch_permute(const Geo& g, const bf16* src, int heads, bool inverse, bf16* dst, cudaStream_t st);
+
 cudaError_t launch_router_scores(const Geo& g, const bf16* qr, const bf16* kr, float* lse_r, float* pr,
                                  cudaStream_t st);
 

@@ -77,6 +77,42 @@ __global__ void __launch_bounds__(256) pool_kernel(const bf16* __restrict__ x, i
   }
 }
 
+// Cube-major copy of a raster tensor (paper Sec. 2.2 "Permutation") and back.  One CTA per (cube, head, batch):
+//   forward: y[b, h, n * B + p, :] = x[b, h, token(n, p), :], zero where position p of cube n lies outside the grid
+//   inverse: x[b, h, token(n, p), :] = y[b, h, n * B + p, :] for the positions inside the grid
+// The attention kernels never need this copy (they address cubes through tensor maps over the raster layout); it is for
+// callers whose surrounding code works in the cube-major layout.
+template <int D>
+__global__ void __launch_bounds__(256) permute_kernel(const bf16* __restrict__ src, int heads, Geo g, int inverse,
+                                                      bf16* __restrict__ dst) {
+  const int n = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const size_t bh = (size_t)b * heads + h;
+  const int B = g.Bt * g.Bh * g.Bw;
+  int nt, nh, nw;
+  cube_coords(g, n, nt, nh, nw);
+  constexpr int CH = D / 8;
+  for (int c = threadIdx.x; c < B * CH; c += blockDim.x) {
+    const int p = c / CH, ch = c % CH;
+    const int l = cube_token(g, nt, nh, nw, p);
+    const size_t raster = (bh * g.L + (size_t)max(l, 0)) * D + ch * 8;
+    const size_t cubed = ((bh * g.N + n) * B + p) * (size_t)D + ch * 8;
+    if (!inverse) {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (l >= 0) v = __ldg(reinterpret_cast<const uint4*>(src + raster));
+      *reinterpret_cast<uint4*>(dst + cubed) = v;
+    } else if (l >= 0) {
+      *reinterpret_cast<uint4*>(dst + raster) = __ldg(reinterpret_cast<const uint4*>(src + cubed));
+    }
+  }
+}
+
+cudaError_t launch_permute(const Geo& g, const bf16* src, int heads, bool inverse, bf16* dst, cudaStream_t st) {
+  dim3 grid(g.N, heads, g.batch);
+  if (g.D == 128) permute_kernel<128><<<grid, 256, 0, st>>>(src, heads, g, inverse ? 1 : 0, dst);
+  else permute_kernel<64><<<grid, 256, 0, st>>>(src, heads, g, inverse ? 1 : 0, dst);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_pool(const Geo& g, const bf16* x, int heads, bf16* xr, float* xc, cudaStream_t st) {
   dim3 grid(g.N, heads, g.batch);
   if (g.D == 128) pool_kernel<128><<<grid, 256, 0, st>>>(x, heads, g, xr, xc);
