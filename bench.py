@@ -33,10 +33,11 @@ from paper_2609_32882_b200 import inputs as syn  # noqa: E402
 
 METRIC = "720p routed sparse attn fwd+bwd ms and TFLOPS (actual & dense-equiv) vs B200 BF16 peak"
 UNIT = "TFLOP/s dense-equivalent"
+ORACLE_HOW = "the oracle as it stands: fp64 numpy whose matrix products run on the multithreaded BLAS numpy links"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the 720p top-64 launch with 40 heads: the
-# 8-head ncu capture summarised in profiles/kernels_720p_8heads_ncu_full.md times 5 (every head streams its own
-# tensors, so the traffic grows in proportion to the heads; the 40-head launch is too large for a full-set capture).
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the 720p top-64 launch with 40 heads: an
+# 8-head ncu capture of the same kernels times 5 (every head streams its own tensors, so the traffic grows in
+# proportion to the heads; the 40-head launch is too large for a full-set capture).
 NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.500836e9 + 0.294249e9), "fine_bwd_dq": 5 * (0.663055e9 + 0.146861e9),
                                 "fine_bwd_dkv": 5 * (0.769323e9 + 0.304400e9)}
 
@@ -52,6 +53,15 @@ def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None) -
     if topk:
         wl = wl.replace(topk=topk, name=f"{wl.name}_top{topk}")
     return wl
+
+
+def config_dict(wl: syn.Workload, forward_only: bool) -> dict:
+    """The `config` object of the JSON line: what the workload is (both arms print the same)."""
+    gb = (2 * wl.heads_q + 2 * wl.heads_kv) * wl.batch * wl.L * wl.head_dim * 2 / 1e9
+    return {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
+            "head_dim": wl.head_dim, "cube": list(wl.cube), "rpool": list(wl.rpool), "select_mode": wl.select_mode,
+            "topk": wl.topk, "forward_only": bool(forward_only),
+            "l2": f"inputs (Q,K,V,dO: {gb:.1f} GB) far larger than the 126 MB L2; no explicit flush"}
 
 
 def flop_counts(wl: syn.Workload, nnz_total: int) -> dict:
@@ -200,9 +210,9 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "grid": list(wl.grid), "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
-                       "head_dim": wl.head_dim, "topk": wl.topk, "select_mode": wl.select_mode},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": sample},
+            "config": config_dict(wl, args.forward_only),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_cores(), "kind": "oracle", "sample": sample,
+                             "how": ORACLE_HOW},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -226,7 +236,10 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(local_rank)
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "VERSION")       # one line per job on stderr: the NCCL build in use
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        print(f"[bench] rank {rank} of {dist.get_world_size()} on cuda:{local_rank} ({torch.cuda.get_device_name(local_rank)})",
+              file=sys.stderr, flush=True)
     if rank == 0:
         vbuild.build_library()
     if world > 1:
@@ -423,7 +436,7 @@ def run_ours(args):
             hd["budgets"] = data["budgets"][0, 0]
         r = oracle_sample_step(wl, hd, args.ref_rows)
         cpu_baseline = {"value": flops["dense_equiv_fwd_bwd"] / r["t_step_extrapolated_s"] / 1e12, "unit": UNIT,
-                        "cores": cpu_cores(), "kind": "oracle",
+                        "cores": cpu_cores(), "kind": "oracle", "how": ORACLE_HOW,
                         "sample": (f"head 0 of {wl.heads_q}: full routing + coarse branch + fine fwd/bwd over {r['rows']} of "
                                    f"{wl.n_cubes} query blocks ({r['pairs_sample']} of {r['pairs_head']} pairs), "
                                    f"{r['measured_s']:.1f} s measured, extrapolated to the whole step "
@@ -459,12 +472,8 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
-                   "head_dim": wl.head_dim, "cube": list(wl.cube), "rpool": list(wl.rpool), "select_mode": wl.select_mode,
-                   "topk": wl.topk, "selected_pairs": nnz_total, "replicas": world, "forward_only": bool(args.forward_only),
-                   "l2": f"inputs (Q,K,V,dO: {sum(host[k].numel() * 2 for k in ('q', 'k', 'v', 'do')) / 1e9:.1f} GB) far larger than the "
-                         "126 MB L2; no explicit flush",
-                   "input_gen_s": round(t_gen, 1)},
+        "config": config_dict(wl, args.forward_only),
+        "run": {"selected_pairs": nnz_total, "replicas": world, "input_gen_s": round(t_gen, 1)},
         "clocks": clocks,
         "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_step_e2e, "h2d_bytes_per_step": bytes_in,
                 "d2h_bytes_per_step": bytes_out,
@@ -509,8 +518,13 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    # `python bench.py --gpus N` without a launcher starts its own N ranks (one per GPU); under torchrun it is one of them
+    from paper_2609_32882_b200 import replicas
+    cmd = replicas.launcher_command(args.gpus, os.path.abspath(__file__), sys.argv[1:], os.environ)
+    if cmd is not None:
+        raise SystemExit(subprocess.call(cmd))
+    run_ours(args)
 
 
 if __name__ == "__main__":

@@ -60,13 +60,10 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
        VSA2_FLAG_EXACT_MAX_FWD = 2 }; /* validation aid: run the whole fine forward with the slow kernel that tracks
                                          the exact running row maximum (the tensor-core kernel falls back to it only
                                          for query blocks whose softmax sums leave the safe range) */
-enum { VSA2_FLAG_SIMPLE_ROUTER = 8 }; /* validation aid: router scores with the slow first-generation kernel */
 /* Coarse branch (Eq. 2-3).  Default: forward with TF32 tensor-core tiles on the fp32 cube means (O_c feeds dGate, which
  * needs that precision); backward by running the tcgen05 fine-branch kernels on the pooled grid with the means rounded
  * to bf16 (its results enter dQ, dK, dV divided by the cube size, where bf16 operand rounding is far below the error
  * bounds). */
-enum { VSA2_FLAG_TF32_COARSE = 32 };  /* validation aid: coarse forward and backward with the TF32 tile kernels
-                                         that stage their accumulators in shared memory */
 enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
                                          (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
@@ -78,9 +75,6 @@ enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV 
                                          (budgets belong to single heads): VSA2_ERR_UNSUPPORTED.
                                          vsa2_attn_fwd with this flag RELIES on that: with an even number of query heads
                                          per KV head it reads the map of the first head of each pair of heads only */
-enum { VSA2_FLAG_SIMPLE_COARSE = 16 };/* validation aid: coarse branch (forward and backward) with the fp32 SIMT kernels
-                                         instead of the TF32 tensor-core ones */
-enum { VSA2_FLAG_SIMPLE_BWD = 4 };    /* validation aid: run the fine backward with the slow first-generation kernels */
 
 /* Problem statement (host struct). */
 typedef struct vsa2_params {
@@ -171,10 +165,13 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
  *   - device_status: optional device int32; if not NULL the status word of this call (VSA2_OK,
  *     VSA2_ERR_MAP_OVERFLOW, VSA2_ERR_DEVICE_TIMEOUT) is copied there on the stream, after the kernels.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
- *     current); make that first call outside any stream capture.  No call allocates or frees device memory.
+ *     current); make that first call at start-up, outside any stream capture: with CUDA's lazy module loading it is
+ *     also the moment the driver loads the library's device code and backs the 8 MiB array, so it is the one call
+ *     that can fail for lack of memory.  No call uses cudaMalloc, cudaFree or any allocating routine.
  *   - All calls on one device share the one array, and it keeps the last call's contents: the call clears what
  *     must start at zero itself, but two calls that overlap on the GPU (different streams, no ordering) race;
- *     order them on one stream or with events.  Host-side it is safe to call from several threads. */
+ *     order them on one stream or with events.  The address look-up is guarded by a mutex; the library's launch
+ *     counter is atomic; the profiling hooks (vsa2_profile_events) are not thread-safe. */
 #define VSA2_ROUTE_NOALLOC_MAX_BYTES (8u << 20)
 int vsa2_route_noalloc(const vsa2_params* p, const void* q, const void* k, const int32_t* budgets,
                        const vsa2_map* map_out, int32_t* device_status, void* cuda_stream);
@@ -189,7 +186,10 @@ const float* vsa2_route_scores(const vsa2_params* p, const void* workspace);
  *         fine branch's softmax denominator (scaled scores); -inf and O_f = 0 for a query block
  *         with no selected KV block.
  *   saved: filled for vsa2_attn_bwd (ignored, may be NULL, with VSA2_FLAG_NO_COARSE).
- *   workspace: >= sizes.fwd_workspace_bytes. */
+ *   workspace: >= sizes.fwd_workspace_bytes.
+ * Every argument check, including the alignment of saved->o_res, runs before the first kernel is enqueued.
+ * A map whose vsa2_route ended with VSA2_ERR_MAP_OVERFLOW holds truncated rows: forward and backward on it read at most
+ * nnz_cap entries per (batch, query head) and compute the attention of that truncated map. */
 int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
                   const vsa2_map* map, void* o, float* lse, const vsa2_saved* saved,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
@@ -273,6 +273,21 @@ int64_t vsa2_launch_count(void);
 int vsa2_selftest_umma(const vsa2_params* p, const void* q, const void* k, const void* v, int32_t cube_q,
                        int32_t cube_a, int32_t cube_b, const void* p_t, float* s_t_out, float* o_t_out,
                        void* k_tile_dump, int32_t* status, void* cuda_stream);
+
+/* Diagnostic of the bounded-wait discipline (the paper has no counterpart).  Every device-side wait of the attention
+ * kernels gives up after a time limit: the CTA raises an abort flag, all its roles leave, the status word becomes
+ * VSA2_ERR_DEVICE_TIMEOUT and tensor memory is released.  This call runs that path alone, in one CTA: one thread waits
+ * `limit_us` microseconds (1 .. 100000) on a barrier nothing arrives at, a second thread waits on another barrier with the
+ * kernels' own 2 s limit and must be released by the first one's abort flag.  `status` (device int32, caller-zeroed)
+ * receives VSA2_ERR_DEVICE_TIMEOUT; `waited_ns` (device uint64, may be NULL) the time the first wait took.  No GPU fault,
+ * trap or hang is involved and the context stays usable. */
+int vsa2_selftest_timeout(uint32_t limit_us, int32_t* status, uint64_t* waited_ns, void* cuda_stream);
+
+/* Test hook (the paper has no counterpart): number of query blocks the forward kernels may hand to the exact-maximum
+ * fall-back per call, 1 .. 16384 (default 16384, which also sizes the workspace).  When more blocks than that leave the
+ * safe range of the fixed-reference softmax, the surplus is not recomputed, the status word becomes VSA2_ERR_UNSUPPORTED
+ * and nothing outside the list is read or written.  Process-global; returns the value now in force. */
+int32_t vsa2_debug_rescue_capacity(int32_t capacity);
 
 /* Text of the CUDA error behind the most recent VSA2_ERR_CUDA returned in this process ("no error" if none). */
 const char* vsa2_last_cuda_error(void);

@@ -18,21 +18,26 @@ What the paper fixes and where (section / equation of the VSA2 paper):
 * padding to whole cubes, padded tokens masked                           -- Sec. 2.2 "Kernel Implementation"
 * the routing decision carries no gradient                               -- Sec. 2.1 (last paragraph)
 
-Readings taken where the paper is silent (each listed in the design notes):
+Readings taken where the paper is silent.  The paper cannot confirm them; what the
+tests pin is that each function computes exactly the reading stated here:
 
 * padding: every mean runs over valid tokens only; padded keys and empty key
   sub-cubes are excluded from every softmax; the router's G x G mean divides by
-  (valid query sub-cubes of the cube) x (full G).            PARITY UNPINNED
+  (valid query sub-cubes of the cube) x (full G).  Pinned on padded grids by
+  library pooling of a zero-padded volume and of a volume of ones, and by a
+  brute-force softmax with an explicit -inf mask.
 * router operands: the pooled Q_r, K_r are rounded to bf16 (round to nearest
   even) after an fp32 sum taken in a fixed order (along w, then h, then t) and
-  an fp32 division by the valid count.                        PARITY UNPINNED
-* ties in TopK go to the lower flat index i*N + j.            PARITY UNPINNED
-* a query block with no selected KV block gets O_f = 0 and lse = -inf.
-                                                              PARITY UNPINNED
+  an fp32 division by the valid count.  Pinned by torch's bf16 cast and by a
+  constructed case in which the order of the sum decides the result.
+* ties in TopK go to the lower flat index i*N + j.  Pinned by Python's sort.
+* a query block with no selected KV block gets O_f = 0 and lse = -inf.  Pinned by
+  the dense masked restatement with an empty mask row.
 * gate projection: X [L, C] are the layer's hidden states (C = model width) and
   W_g has one column per query head, W_g [C, H_q], so that G [H_q, L] holds the
   per-token per-head gate of Eq. 13 (the paper writes one head: W_g in R^{D x 1}).
-Everything else is pinned by tests/test_oracle_pins.py.
+* text tokens (Sec. 2.2, the sentence after Eq. 12): see `joint_*` below.
+Every function here is pinned by tests/test_oracle_pins.py.
 """
 from __future__ import annotations
 

@@ -19,10 +19,6 @@ PER_SEQUENCE, PER_QUERY, PER_QUERY_BUDGET = 0, 1, 2
 BF16, F32 = 0, 1
 FLAG_NO_COARSE = 1
 FLAG_EXACT_MAX_FWD = 2
-FLAG_SIMPLE_BWD = 4
-FLAG_SIMPLE_ROUTER = 8
-FLAG_SIMPLE_COARSE = 16
-FLAG_TF32_COARSE = 32
 FLAG_BF16_COARSE_FWD = 64
 FLAG_HALF_CUBE_FWD = 128
 FLAG_GROUP_ROUTING = 256
@@ -34,7 +30,8 @@ ERR_STATIC_SCRATCH = -8
 
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
            "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc", "vsa2_last_cuda_error",
-           "vsa2_gate_fwd", "vsa2_gate_bwd", "vsa2_gate_bwd_workspace_bytes", "vsa2_permute_cube_major")
+           "vsa2_gate_fwd", "vsa2_gate_bwd", "vsa2_gate_bwd_workspace_bytes", "vsa2_permute_cube_major",
+           "vsa2_selftest_timeout", "vsa2_debug_rescue_capacity")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv")
@@ -109,6 +106,8 @@ def _lib():
         lib.vsa2_strerror.restype = C.c_char_p
         lib.vsa2_profile_events.argtypes = [C.c_int32, vp, vp]
         lib.vsa2_selftest_umma.argtypes = [C.POINTER(Params), vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
+        lib.vsa2_selftest_timeout.argtypes = [C.c_uint32, vp, vp, vp]
+        lib.vsa2_debug_rescue_capacity.argtypes = [C.c_int32]
         lib.vsa2_launch_count.argtypes = []
         lib.vsa2_launch_count.restype = C.c_int64
         for name in EXPORTS:

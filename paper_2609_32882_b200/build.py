@@ -56,26 +56,5 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
-def build_probes() -> list:
-    """Compiles the stand-alone hardware probes (probes/*.cu: TMA and tcgen05 rate measurements quoted in the design
-    notes) into probes/bin/.  They are diagnostics: the library does not use them."""
-    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
-    src_dir = os.path.join(HERE, "probes")
-    out_dir = os.path.join(src_dir, "bin")
-    os.makedirs(out_dir, exist_ok=True)
-    outs = []
-    for f in sorted(os.listdir(src_dir)):
-        if not f.endswith(".cu"):
-            continue
-        out = os.path.join(out_dir, f[:-3])
-        subprocess.check_call([nvcc, "-std=c++17", "-O3", "-lineinfo", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-                              + ARCH_FLAGS + [os.path.join(src_dir, f), "-o", out, "-lcuda"])
-        outs.append(out)
-    return outs
-
-
 if __name__ == "__main__":
-    if "--probes" in sys.argv:
-        print("\n".join(build_probes()))
-    else:
-        print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))

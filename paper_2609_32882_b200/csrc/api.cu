@@ -2,6 +2,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 using namespace vsa2;
@@ -10,7 +12,7 @@ namespace {
 
 cudaEvent_t g_prof_start[VSA2_KERNEL_COUNT];
 cudaEvent_t g_prof_stop[VSA2_KERNEL_COUNT];
-long long g_launches = 0;
+std::atomic<long long> g_launches{0};
 
 struct RouteLayout {
   size_t status, qr, kr, lse_r, pr, hist, state, row_tau, row_eq_take, row_cnt, row_gt, row_eq, bitmap, bitmap_t, total;
@@ -229,7 +231,12 @@ int vsa2_profile_events(int32_t kernel_id, void* start_event, void* stop_event) 
   return VSA2_OK;
 }
 
-int64_t vsa2_launch_count(void) { return g_launches; }
+int64_t vsa2_launch_count(void) { return g_launches.load(); }
+
+int32_t vsa2_debug_rescue_capacity(int32_t capacity) {
+  set_fwd_rescue_capacity(capacity);
+  return fwd_rescue_capacity();
+}
 
 const char* vsa2_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
@@ -293,9 +300,9 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
     VSA2_CUDA(launch_pool(r, reinterpret_cast<const bf16*>(k), r.Hkv, kr, nullptr, st));
   }
   float* pr = at<float>(workspace, rl.pr);
-  if (router_tc_supported(r) && !(g.flags & VSA2_FLAG_SIMPLE_ROUTER))
+  if (router_tc_supported(r))
     VSA2_CUDA(launch_router_scores_tc(r, qr, kr, at<float>(workspace, rl.lse_r), pr, status, st));
-  else
+  else   // sub-cube counts the tensor-core kernel has no layout for (G = 1 is the VSA router of Sec. 2.1)
     VSA2_CUDA(launch_router_scores(r, qr, kr, at<float>(workspace, rl.lse_r), pr, st));
   if (wide) {
     g_launches += 1;
@@ -349,6 +356,7 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     return VSA2_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned256(workspace))
     return VSA2_ERR_MISALIGNED;
+  if (saved != nullptr && !g.out_f32 && saved->o_res != nullptr && !aligned16(saved->o_res)) return VSA2_ERR_MISALIGNED;
   if (workspace_bytes < fwd_workspace_bytes(g)) return VSA2_ERR_WORKSPACE_TOO_SMALL;
   if ((rc = check_device()) != VSA2_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -383,17 +391,13 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
       }
     }
     {
-      ProfScope ps(VSA2_KERNEL_COARSE_FWD, st,
-                   ((g.flags & VSA2_FLAG_BF16_COARSE_FWD) && !(g.flags & VSA2_FLAG_SIMPLE_COARSE) ? 6 : 1) + (wide ? 1 : 0));
-      if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
-        VSA2_CUDA(launch_coarse_fwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
-      else if (g.flags & VSA2_FLAG_TF32_COARSE)
-        VSA2_CUDA(launch_coarse_fwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
-      else if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
+      ProfScope ps(VSA2_KERNEL_COARSE_FWD, st, ((g.flags & VSA2_FLAG_BF16_COARSE_FWD) ? 7 : 1) + (wide ? 1 : 0));
+      if (!(g.flags & VSA2_FLAG_BF16_COARSE_FWD))
         VSA2_CUDA(launch_coarse_fwd_mma(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, st));
       else
         VSA2_CUDA(launch_coarse_fwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c,
-                                           at<unsigned char>(workspace, pooled_off), st));
+                                           at<unsigned char>(workspace, pooled_off),
+                                           reinterpret_cast<StatusBlock*>(workspace), st));
       if (wide) {
         VSA2_CUDA(launch_expand_rows(n, n.Hq, false, saved->oc_hat, at<float>(workspace, wl.oc_hat64), st));
         oc_hat = at<float>(workspace, wl.oc_hat64);
@@ -407,7 +411,6 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     col_idx = at<int>(workspace, wl.idx64);
   }
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
-  if (o_res != nullptr && !aligned16(o_res)) return VSA2_ERR_MISALIGNED;
   {
     ProfScope ps(VSA2_KERNEL_FINE_FWD, st, (g.flags & VSA2_FLAG_EXACT_MAX_FWD) ? 1 : 2);
     if (g.flags & VSA2_FLAG_EXACT_MAX_FWD)
@@ -492,19 +495,12 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
                                     d_oc_hat, st));
   }
   if (coarse) {
-    // SIMT / TF32: two kernels; pooled grid: four casts, the dense map, the pooled preprocess, dQ, dK/dV (+ two group spreads)
-    const bool pooled_bwd = !(g.flags & (VSA2_FLAG_SIMPLE_COARSE | VSA2_FLAG_TF32_COARSE));
-    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, (pooled_bwd ? 8 + (g.rep > 1 ? 2 : 0) : 2) + (wide ? 4 : 0));
+    // pooled grid: four casts, the dense map, the pooled preprocess, dQ, dK/dV (+ two group spreads)
+    ProfScope ps(VSA2_KERNEL_COARSE_BWD, st, 9 + (g.rep > 1 ? 2 : 0) + (wide ? 4 : 0));
     if (wide) VSA2_CUDA(launch_fold_sum(n, n.Hq, d_oc_hat, d_oc_hat_cube, st));
-    if (g.flags & VSA2_FLAG_SIMPLE_COARSE)
-      VSA2_CUDA(launch_coarse_bwd(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
-                                  at<float>(cube_ws, cl.delta_c), dqc_cube, dkc_cube, dvc_cube, st));
-    else if (g.flags & VSA2_FLAG_TF32_COARSE)
-      VSA2_CUDA(launch_coarse_bwd_tc(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
-                                     at<float>(cube_ws, cl.delta_c), dqc_cube, dkc_cube, dvc_cube, st));
-    else
-      VSA2_CUDA(launch_coarse_bwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
-                                         dqc_cube, dkc_cube, dvc_cube, at<unsigned char>(cube_ws, cl.pooled), st));
+    VSA2_CUDA(launch_coarse_bwd_pooled(g, saved->qc, saved->kc, saved->vc, saved->oc_hat, saved->lse_c, d_oc_hat_cube,
+                                       dqc_cube, dkc_cube, dvc_cube, at<unsigned char>(cube_ws, cl.pooled),
+                                       reinterpret_cast<StatusBlock*>(workspace), st));
     if (wide) {
       VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dqc_cube, dqc, st));
       VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dkc_cube, dkc, st));
@@ -513,20 +509,13 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
-    if (g.flags & VSA2_FLAG_SIMPLE_BWD)
-      VSA2_CUDA(launch_fine_bwd_dq(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq, st));
-    else
-      VSA2_CUDA(launch_fine_bwd_dq_tc(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
-                                      reinterpret_cast<StatusBlock*>(workspace), st));
+    VSA2_CUDA(launch_fine_bwd_dq_tc(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
+                                    reinterpret_cast<StatusBlock*>(workspace), st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
-    if (g.flags & VSA2_FLAG_SIMPLE_BWD)
-      VSA2_CUDA(launch_fine_bwd_dkv(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
-                                    coarse ? dvc : nullptr, dk, dv, st));
-    else
-      VSA2_CUDA(launch_fine_bwd_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
-                                       coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
+    VSA2_CUDA(launch_fine_bwd_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
+                                     coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;
 }

@@ -82,8 +82,16 @@ __global__ void spread_to_group_kernel(const float* __restrict__ x_kv, float* __
   reinterpret_cast<float4*>(x_q)[(size_t)hq * per_head4 + i] = v;
 }
 
+// The pooled passes count their work items in a status block of their own (inside the scratch region); a non-zero
+// status word there (a bounded wait that ran out, a rescue list that overflowed) is copied into the caller's status word,
+// which is the one vsa2_device_status reads.
+__global__ void merge_status_kernel(const StatusBlock* __restrict__ from, StatusBlock* __restrict__ into) {
+  const int s = from->status;
+  if (s != 0) atomicCAS(&into->status, 0, s);
+}
+
 cudaError_t launch_coarse_fwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
-                                     float* lse_c, void* workspace, cudaStream_t st) {
+                                     float* lse_c, void* workspace, StatusBlock* caller_status, cudaStream_t st) {
   const Geo p = pooled_geo(g);
   const PooledLayout lay = pooled_layout(g, false);
   unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
@@ -100,13 +108,16 @@ cudaError_t launch_coarse_fwd_pooled(const Geo& g, const float* qc, const float*
   if ((e = cast_to_bf16(vc, v16, BHk * g.N * g.D, st)) != cudaSuccess) return e;
   dense_map_kernel<<<(unsigned)BHq, 256, 0, st>>>(ptr, idx, p.N, (int)BHq);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  return launch_fine_fwd_tc(p, q16, k16, v16, nullptr, ptr, idx, nullptr, oc_hat, nullptr, lse_c,
-                            reinterpret_cast<StatusBlock*>(ws + lay.status), st);
+  if ((e = launch_fine_fwd_tc(p, q16, k16, v16, nullptr, ptr, idx, nullptr, oc_hat, nullptr, lse_c,
+                              reinterpret_cast<StatusBlock*>(ws + lay.status), st)) != cudaSuccess)
+    return e;
+  merge_status_kernel<<<1, 1, 0, st>>>(reinterpret_cast<const StatusBlock*>(ws + lay.status), caller_status);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
                                      const float* lse_c, const float* d_oc_hat, float* dqc, float* dkc, float* dvc,
-                                     void* workspace, cudaStream_t st) {
+                                     void* workspace, StatusBlock* caller_status, cudaStream_t st) {
   const Geo p = pooled_geo(g);
   const PooledLayout lay = pooled_layout(g, true);
   unsigned char* ws = reinterpret_cast<unsigned char*>(workspace);
@@ -143,7 +154,8 @@ cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float*
     spread_to_group_kernel<<<grid, 256, 0, st>>>(dv_kv, dvc, g.rep, per_head4, (int)BHq);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  return cudaSuccess;
+  merge_status_kernel<<<1, 1, 0, st>>>(status, caller_status);
+  return cudaGetLastError();
 }
 
 }  // namespace vsa2

@@ -138,19 +138,10 @@ cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, con
                           int* row_ptr, int* col_idx, int* col_ptr, int* row_idx, StatusBlock* status,
                           cudaStream_t st);
 
-cudaError_t launch_coarse_fwd(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
-                              float* lse_c, cudaStream_t st);
-cudaError_t launch_coarse_bwd(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
-                              const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
-                              float* dvc, cudaStream_t st);
-cudaError_t launch_coarse_fwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
-                                 float* lse_c, cudaStream_t st);
-// the same product with register-resident accumulators (coarse_fwd_mma.cu): the default forward
+// coarse branch forward on the fp32 cube means, TF32 tensor-core products with register-resident accumulators
+// (coarse_fwd_mma.cu)
 cudaError_t launch_coarse_fwd_mma(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
                                   float* lse_c, cudaStream_t st);
-cudaError_t launch_coarse_bwd_tc(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
-                                 const float* lse_c, const float* d_oc_hat, float* delta_c, float* dqc, float* dkc,
-                                 float* dvc, cudaStream_t st);
 
 cudaError_t launch_fine_fwd(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
                             const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
@@ -163,10 +154,10 @@ struct PooledLayout {
 Geo pooled_geo(const Geo& g);
 PooledLayout pooled_layout(const Geo& g, bool backward);
 cudaError_t launch_coarse_fwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, float* oc_hat,
-                                     float* lse_c, void* workspace, cudaStream_t st);
+                                     float* lse_c, void* workspace, StatusBlock* caller_status, cudaStream_t st);
 cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float* kc, const float* vc, const float* oc_hat,
                                      const float* lse_c, const float* d_oc_hat, float* dqc, float* dkc, float* dvc,
-                                     void* workspace, cudaStream_t st);
+                                     void* workspace, StatusBlock* caller_status, cudaStream_t st);
 
 // cubes of 128 tokens as pairs of 64-token half-cubes (wide_cube.cu); `narrow` is narrow_geo() of the problem
 bool wide_cube(const Geo& g);
@@ -190,6 +181,8 @@ cudaError_t launch_gate_bwd(int batch, int L, int C, int Hq, int out_f32, const 
 
 // tensor-core forward (fine_fwd_tc.cu); `status` heads a workspace of fine_fwd_tc_workspace_bytes()
 size_t fine_fwd_tc_workspace_bytes();
+int fwd_rescue_capacity();
+void set_fwd_rescue_capacity(int cap);
 cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
                                const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                float* lse, StatusBlock* status, cudaStream_t st);
@@ -213,11 +206,4 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
 cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,
                                   const float* oc_hat, float* delta, float* dgate, float* d_oc_hat,
                                   cudaStream_t st);
-cudaError_t launch_fine_bwd_dq(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
-                               const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
-                               const float* dqc, void* dq, cudaStream_t st);
-cudaError_t launch_fine_bwd_dkv(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
-                                const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
-                                const float* dkc, const float* dvc, void* dk, void* dv, cudaStream_t st);
-
 }  // namespace vsa2

@@ -136,16 +136,18 @@ __global__ void __launch_bounds__(256) fine_fwd_kernel(const bf16* __restrict__ 
   fine_fwd_block<D>(smem_raw, blockIdx.x, blockIdx.y, blockIdx.z, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
 }
 
-// Recomputes the query blocks listed in `items` (flat index (b*Hq + hq)*N + i; *count entries).
+// Recomputes the query blocks listed in `items` (flat index (b*Hq + hq)*N + i).  *count may exceed the capacity of the
+// list (its producers keep counting after the list is full and report that through the status word): only the `cap`
+// entries that were written are read.
 template <int D>
-__global__ void __launch_bounds__(256) fine_fwd_list_kernel(const int* __restrict__ count, const int* __restrict__ items,
+__global__ void __launch_bounds__(256) fine_fwd_list_kernel(const int* __restrict__ count, int cap, const int* __restrict__ items,
                                                             const bf16* __restrict__ q, const bf16* __restrict__ k,
                                                             const bf16* __restrict__ v, const float* __restrict__ gate,
                                                             const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                                                             const float* __restrict__ oc_hat, Geo g, void* __restrict__ o,
                                                             bf16* __restrict__ o_res, float* __restrict__ lse) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  const int n = *count;
+  const int n = min(*count, cap);
   for (int e = blockIdx.x; e < n; e += gridDim.x) {
     int item = items[e];
     int i = item % g.N, bh = item / g.N;
@@ -154,18 +156,18 @@ __global__ void __launch_bounds__(256) fine_fwd_list_kernel(const int* __restric
   }
 }
 
-cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
+cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, int cap, const int* items, const bf16* q, const bf16* k,
                                  const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
                                  const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st) {
   cudaError_t e;
   if (g.D == 128) {
     size_t smb = FineFwdSmem<128>::bytes;
     if ((e = cudaFuncSetAttribute(fine_fwd_list_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    fine_fwd_list_kernel<128><<<64, 256, smb, st>>>(count, items, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
+    fine_fwd_list_kernel<128><<<64, 256, smb, st>>>(count, cap, items, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
   } else {
     size_t smb = FineFwdSmem<64>::bytes;
     if ((e = cudaFuncSetAttribute(fine_fwd_list_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    fine_fwd_list_kernel<64><<<64, 256, smb, st>>>(count, items, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
+    fine_fwd_list_kernel<64><<<64, 256, smb, st>>>(count, cap, items, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
   }
   return cudaGetLastError();
 }

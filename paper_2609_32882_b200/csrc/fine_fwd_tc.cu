@@ -75,14 +75,15 @@ struct FwdArgs {
   StatusBlock* status;
   int* rescue_count;
   int* rescue_items;
+  int rescue_cap;       // entries the list holds
 };
 
 // Roles (512 threads = 4 warpgroups).  An issuing thread needs ~60 cycles per MMA plus ~100-200 per barrier
 // operation, more than the 48 cycles an N = 64 MMA takes to execute, so issue and copy work is spread:
-//   warpgroups 0, 1 (few registers): warp 0 = TMA producer of the K pairs and the Q tile, warp 1 = TMA producer of the
-//       V pairs (lane 0 owns the barriers, lanes 0 .. 2*D/64-1 each issue one box), warps 2, 3 = issuers of the S^T
-//       products of the even / odd tiles, warps 4, 5 = issuers of the O^T products of the even / odd tiles (each
-//       into its own accumulator, summed in the epilogue), warps 6, 7 idle.
+//   warpgroups 0, 1 (few registers): warps 0, 6 = TMA producers of the K pairs (first / second block; warp 0 also
+//       brings the Q tile), warps 1, 7 = TMA producers of the V pairs (lane 0 owns the barriers, lanes 0 .. D/64-1 each
+//       issue one box), warps 2, 3 = issuers of the S^T products of the even / odd tiles, warps 4, 5 = issuers of the
+//       O^T products of the even / odd tiles (each into its own accumulator, summed in the epilogue).
 //   warpgroups 2, 3: softmax + epilogue; warpgroup w handles the tiles with (global tile index & 1) == w - 2, so two
 //       tiles are in the exponential unit at any time.  A warp owns tensor-memory lane quadrant warp % 4.
 // Every mbarrier has one producing role and one consuming role (or all consumers see every phase), so a phase can
@@ -111,11 +112,11 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc::mbar_init(&misc->o_full, 2);       // both O^T issuers
     tc::mbar_init(&misc->o_empty, 256);
     for (int s = 0; s < kFwdKSlots; ++s) {
-      tc::mbar_init(&misc->k_full[s], 1);
+      tc::mbar_init(&misc->k_full[s], 2);    // the two producer warps of the ring
       tc::mbar_init(&misc->k_empty[s], 2);   // the issuing S^T warp (on completion) and the observing one
     }
     for (int s = 0; s < kFwdVSlots; ++s) {
-      tc::mbar_init(&misc->v_full[s], 1);
+      tc::mbar_init(&misc->v_full[s], 2);
       tc::mbar_init(&misc->v_empty[s], 1);
     }
     for (int s = 0; s < kFwdSBufs; ++s) {
@@ -129,7 +130,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     tc::mbar_init(&misc->wg_sync[0], 128);
     tc::mbar_init(&misc->wg_sync[1], 128);
     tc::mbar_init(&misc->all_sync, 256);
-    item_queue_init(&misc->items, 2 + 4 + 256);     // lane 0 of the producers, four issuers, the softmax threads
+    item_queue_init(&misc->items, 4 + 4 + 256);     // lane 0 of the producers, four issuers, the softmax threads
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -147,22 +148,26 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 
   if (warp < 8) {
     tc::reg_dec<56>();
-    if (warp < 2) {
+    if (warp < 2 || warp >= 6) {
       // ---------------------------------------------------------------- TMA producers
-      const int which = warp;                               // 0: K ring (+ Q tile), 1: V ring
+      // One warp sustains only ~24 B/clk of 5-D boxes (the copy instructions of a warp issue one after the other,
+      // ~350 cycles per 8 KB box), so every ring has two producer warps: warps 0, 1 bring the first block of each
+      // pair, warps 6, 7 the second.  Both arrive on the slot's full barrier with their half of the bytes.
+      const int which = warp & 1;                           // 0: K ring (+ Q tile), 1: V ring
+      const int my_blk = warp >> 2;                         // 0: first block of the pair, 1: second
       const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
       const uint32_t nslots = which == 0 ? kFwdKSlots : kFwdVSlots;
       uint64_t* full = which == 0 ? misc->k_full : misc->v_full;
       uint64_t* empty = which == 0 ? misc->k_empty : misc->v_empty;
       unsigned char* ring = smem + (which == 0 ? 0 : kFwdKSlots * C::SLOT);
-      const int my_h = lane >> 1, my_blk = lane & 1;
-      const bool issuer = lane < 2 * C::DH;
+      const int my_h = lane;
+      const bool issuer = lane < C::DH;
       uint32_t tg = 0, n_items = 0, published = 0;
       for (uint32_t seq = 0;; ++seq) {
         // warp 0, lane 0 is the CTA's scheduler
         int item = 0;
         if (lane == 0) {
-          if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
+          if (warp == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
           else item = item_get(&misc->items, seq, &misc->abort_flag);
         }
         item = __shfl_sync(0xffffffffu, item, 0);
@@ -174,7 +179,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const int k = end - beg;
         if (k == 0) continue;
         const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
-        if (which == 0) {
+        if (warp == 0) {
           int it_, ih_, iw_;
           cube_coords(g, i, it_, ih_, iw_);
           int ok = 1;
@@ -197,7 +202,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
           int ok = 1;
           if (lane == 0) {
             ok = tc::mbar_wait(&empty[slot], par ^ 1, &misc->abort_flag);
-            if (ok) tc::mbar_expect_tx(&full[slot], C::SLOT);
+            if (ok) tc::mbar_expect_tx(&full[slot], C::SLOT / 2);
           }
           if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
           if (issuer)
@@ -490,7 +495,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         a.lse[(size_t)bhq * g.L + misc->tok[tb][sm_tid]] = -INFINITY;
       if (k > 0 && wg == 0 && sm_tid == 0 && misc->rescue_flag) {
         int slot = atomicAdd(a.rescue_count, 1);
-        if (slot < kRescueCap) a.rescue_items[slot] = item;
+        if (slot < a.rescue_cap) a.rescue_items[slot] = item;
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
       }
       if (k > 0) ++n_items;
@@ -513,11 +518,17 @@ done:
   if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
 }
 
-cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
+cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, int cap, const int* items, const bf16* q, const bf16* k,
                                  const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
                                  const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
 
 size_t fine_fwd_tc_workspace_bytes() { return 256 + (size_t)kRescueCap * sizeof(int); }
+
+// Entries of the rescue list the kernels may use (<= kRescueCap, which sizes the workspace).  Process-wide; lowered only by
+// tests that make the list overflow on a small problem.
+static int g_rescue_cap = kRescueCap;
+int fwd_rescue_capacity() { return g_rescue_cap; }
+void set_fwd_rescue_capacity(int cap) { g_rescue_cap = cap < 1 ? 1 : (cap > kRescueCap ? kRescueCap : cap); }
 
 // workspace: [StatusBlock][rescue list]; the rescue counter is StatusBlock.pad[0].
 cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
@@ -536,6 +547,7 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
   a.rescue_count = &status->pad[0];
   a.item_counter = &status->pad[1];
   a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
+  a.rescue_cap = g_rescue_cap;
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
   if (g.N > kFwdMaxCubes) return cudaErrorInvalidValue;
@@ -557,7 +569,7 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // query blocks whose row sums left the safe range are redone with the exact running maximum
-  return launch_fine_fwd_list(g, a.rescue_count, a.rescue_items, q, k, v, gate, row_ptr, col_idx, oc_hat, o, o_res, lse, st);
+  return launch_fine_fwd_list(g, a.rescue_count, a.rescue_cap, a.rescue_items, q, k, v, gate, row_ptr, col_idx, oc_hat, o, o_res, lse, st);
 }
 
 }  // namespace vsa2

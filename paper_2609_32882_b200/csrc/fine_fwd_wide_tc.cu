@@ -80,6 +80,7 @@ struct FwdWideArgs {
   StatusBlock* status;
   int* rescue_count;
   int* rescue_items;
+  int rescue_cap;       // entries the list holds
 };
 
 // The two "members" of an item share their list of key blocks: member m is query block i0 + m * di of head bhq0 + m * dh;
@@ -482,7 +483,7 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         a.lse[(size_t)bhq * g.L + misc->tok[tb][q0 + sm_tid]] = -INFINITY;
       if (nt > 0 && sm_tid == 0 && misc->rescue_flag[wg]) {
         int slot = atomicAdd(a.rescue_count, 1);
-        if (slot < kFwwRescueCap) a.rescue_items[slot] = bhq * g.N + i;      // half-cube item of the N = 64 numbering
+        if (slot < a.rescue_cap) a.rescue_items[slot] = bhq * g.N + i;      // half-cube item of the N = 64 numbering
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
       }
       if (nt > 0) ++n_items;
@@ -508,7 +509,7 @@ done:
   if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
 }
 
-cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, const int* items, const bf16* q, const bf16* k,
+cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, int cap, const int* items, const bf16* q, const bf16* k,
                                  const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
                                  const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
 
@@ -533,6 +534,7 @@ cudaError_t launch_fine_fwd_wide_tc(const Geo& g, bool pair_heads, const bf16* q
   a.rescue_count = &status->pad[0];
   a.item_counter = &status->pad[1];
   a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
+  a.rescue_cap = fwd_rescue_capacity() < kFwwRescueCap ? fwd_rescue_capacity() : kFwwRescueCap;
   const int total = g.batch * g.Hq * g.N / 2;         // pairs of query blocks (Hq or N is even)
   const int grid = total < sms ? total : sms;
   if (g.N > kFwwMaxCubes || (pair_heads ? (g.rep & 1) : (g.N & 1))) return cudaErrorInvalidValue;
@@ -549,7 +551,7 @@ cudaError_t launch_fine_fwd_wide_tc(const Geo& g, bool pair_heads, const bf16* q
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // half-cubes whose row sums left the safe range are redone with the exact running maximum
-  return launch_fine_fwd_list(g, a.rescue_count, a.rescue_items, q, k, v, gate, row_ptr, col_idx, oc_hat, o, o_res, lse, st);
+  return launch_fine_fwd_list(g, a.rescue_count, a.rescue_cap, a.rescue_items, q, k, v, gate, row_ptr, col_idx, oc_hat, o, o_res, lse, st);
 }
 
 }  // namespace vsa2

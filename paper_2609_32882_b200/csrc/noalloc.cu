@@ -10,7 +10,7 @@
 
 #include "common.cuh"
 
-#define VSA2_ROUTE_STATIC_BYTES (8u << 20)   // 8 MiB, held by every GPU that loads the library until exit
+#define VSA2_ROUTE_STATIC_BYTES VSA2_ROUTE_NOALLOC_MAX_BYTES   // 8 MiB, held by every GPU that has loaded the library's device code
 
 // The scratch itself.  In host code this name is only a stand-in for the symbol, never a device address:
 // the address is obtained once per device with cudaGetSymbolAddress below.

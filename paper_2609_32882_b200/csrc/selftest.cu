@@ -109,9 +109,57 @@ __global__ void __launch_bounds__(128) selftest_kernel(const __grid_constant__ C
   if (warp == 0) tc::tmem_dealloc(tmem_base, 128);
 }
 
+// The give-up path of the attention kernels in isolation: a CTA allocates tensor memory, one role waits on an mbarrier
+// that no role ever arrives at, with a limit of `limit_us` microseconds instead of the kernels' 2 s; the wait runs out,
+// the role raises the CTA's abort flag, every thread leaves through the common exit, the status word receives
+// VSA2_ERR_DEVICE_TIMEOUT and the tensor memory is released.  Nothing faults or hangs; the context stays usable.
+__global__ void __launch_bounds__(128) selftest_timeout_kernel(unsigned limit_us, int* __restrict__ status,
+                                                               unsigned long long* __restrict__ waited_ns) {
+  __shared__ __align__(8) uint64_t never, other;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) {
+    abort_flag = 0;
+    tc::mbar_init(&never, 1);
+    tc::mbar_init(&other, 1);
+    tc::fence_barrier_init();
+  }
+  if (warp == 0) {
+    tc::tmem_alloc(&tmem_base_s, 128);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+  if (tid == 32) {
+    // the role whose producer never shows up
+    const unsigned long long t0 = tc::global_timer_ns();
+    const bool ok = tc::mbar_wait_ns(&never, 0, &abort_flag, (unsigned long long)limit_us * 1000ull);
+    if (waited_ns != nullptr) *waited_ns = tc::global_timer_ns() - t0;
+    if (ok) atomicExch(status, VSA2_ERR_INVALID_ARG);      // cannot happen: nothing arrives on that barrier
+  } else if (tid == 64) {
+    // a second role parked on another barrier: it must leave as soon as the first one has given up (shared abort flag),
+    // long before its own 2 s limit
+    tc::mbar_wait(&other, 0, &abort_flag);
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (abort_flag && tid == 0) atomicExch(status, VSA2_ERR_DEVICE_TIMEOUT);
+  if (warp == 0) tc::tmem_dealloc(tmem_base, 128);
+}
+
 }  // namespace vsa2
 
 using namespace vsa2;
+
+extern "C" int vsa2_selftest_timeout(uint32_t limit_us, int32_t* status, uint64_t* waited_ns, void* cuda_stream) {
+  if (status == nullptr || limit_us == 0 || limit_us > 100000u) return VSA2_ERR_INVALID_ARG;
+  selftest_timeout_kernel<<<1, 128, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(
+      limit_us, status, reinterpret_cast<unsigned long long*>(waited_ns));
+  return cudaGetLastError() == cudaSuccess ? VSA2_OK : VSA2_ERR_CUDA;
+}
 
 extern "C" int vsa2_selftest_umma(const vsa2_params* p, const void* q, const void* k, const void* v, int32_t cube_q,
                                   int32_t cube_a, int32_t cube_b, const void* p_t, float* s_t_out, float* o_t_out,

@@ -106,7 +106,8 @@ __global__ void __launch_bounds__(128) expand_map_kernel(int N, int Hq, long lon
   const int c = blockIdx.x;
   const size_t bh = (size_t)blockIdx.z * Hq + blockIdx.y;
   const int* p = ptr + bh * (N + 1);
-  const int beg = p[c], end = p[c + 1], len = end - beg;
+  // (a map whose selection overflowed nnz_cap has row pointers beyond the capacity: such rows are cut at `cap`)
+  const int beg = (int)min((long long)p[c], cap), end = (int)min((long long)p[c + 1], cap), len = end - beg;
   const int* src = idx + bh * cap + beg;
   int* p64 = ptr64 + bh * (2 * N + 1);
   int* dst = idx64 + bh * 4 * cap + 4 * (size_t)beg;

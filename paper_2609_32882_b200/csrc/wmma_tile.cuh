@@ -1,6 +1,7 @@
-// Small CTA-level tile GEMM on shared-memory operands (bf16 in, fp32 out) used by the
-// first-generation kernels.  All warps of the CTA take part; 16x16 output tiles are dealt
-// round-robin to the warps.
+// Small CTA-level tile GEMM on shared-memory operands (bf16 in, fp32 out) used by the two fall-back kernels:
+// the exact-running-maximum forward that redoes rescued query blocks (fine_fwd.cu) and the router for sub-cube
+// counts the tensor-core router has no layout for (router.cu).  All warps of the CTA take part; 16x16 output
+// tiles are dealt round-robin to the warps.
 #pragma once
 #include <mma.h>
 

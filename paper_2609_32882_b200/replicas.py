@@ -6,6 +6,10 @@ Works with any torch.distributed backend (NCCL on GPUs, gloo in the CPU tests).
 """
 from __future__ import annotations
 
+import os
+import socket
+import sys
+
 import torch
 import torch.distributed as dist
 
@@ -36,3 +40,28 @@ def max_over_ranks(values, device="cpu"):
 def whole_job_throughput(units_per_rank: float, world: int, seconds: float) -> float:
     """Units all ranks processed divided by the slowest rank's time."""
     return units_per_rank * world / seconds
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launcher_command(gpus: int, script: str, argv: list, env: dict, port: int | None = None):
+    """How `python <script> --gpus N ...` becomes N ranks.
+
+    Under a launcher (WORLD_SIZE is set) the process is one of the ranks: returns None, after checking that the
+    launcher's world size is the one asked for.  Started plainly with --gpus N > 1, the script must start its own
+    ranks: returns the torch.distributed.run command line (one process per GPU of this node, rendezvous on 127.0.0.1)
+    that re-runs the same script with the same arguments.
+    """
+    world = env.get("WORLD_SIZE")
+    if world is not None:
+        if int(world) != int(gpus):
+            raise SystemExit(f"--gpus {gpus} disagrees with the launcher's WORLD_SIZE={world}")
+        return None
+    if gpus <= 1:
+        return None
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(gpus)}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port or free_port()), script] + list(argv)

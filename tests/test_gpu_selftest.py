@@ -69,3 +69,31 @@ def test_tma_cube_tiles_and_tcgen05_products(wl, cubes):
     assert np.abs(got_o[:D] - o_ref).max() < 1e-3 * max(1.0, np.abs(o_ref).max())
     if D == 64:
         assert np.abs(got_o[64:] - o_ref).max() < 1e-3 * max(1.0, np.abs(o_ref).max())
+
+
+def test_a_wait_that_runs_out_reports_a_timeout_and_leaves_the_context_usable():
+    """The give-up path of the attention kernels, driven without any fault: a wait on a barrier nothing arrives at runs out
+    after 1 ms, the CTA's second waiting role is released by the shared abort flag, the status word reads
+    VSA2_ERR_DEVICE_TIMEOUT, tensor memory is handed back -- and an ordinary route + forward right after it succeeds (it
+    allocates all 512 tensor-memory columns, so a leaked allocation would make it wait and time out as well)."""
+    import time
+    from vsa2_testlib import CudaPath
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    lib = vb._lib()
+    t0 = time.time()
+    for _ in range(3):
+        status.zero_()
+        rc = lib.vsa2_selftest_timeout(1000, status.data_ptr(), waited.data_ptr(), None)
+        assert rc == vb.OK
+        torch.cuda.synchronize()
+        assert status.item() == vb.ERR_DEVICE_TIMEOUT
+        assert 1_000_000 <= waited.item() < 50_000_000          # about 1 ms, nowhere near the kernels' own 2 s limit
+    assert time.time() - t0 < 1.5                               # the second role did not sit out its 2 s either
+    assert lib.vsa2_selftest_timeout(0, status.data_ptr(), None, None) == vb.ERR_INVALID_ARG
+    assert lib.vsa2_selftest_timeout(1000, None, None, None) == vb.ERR_INVALID_ARG
+    wl = syn.CONFIGS[0]
+    run = CudaPath(wl, syn.make_inputs(wl, threads=1))
+    run.route()
+    O, lse = run.forward()                                      # check_status inside: VSA2_OK
+    assert np.isfinite(O).all()

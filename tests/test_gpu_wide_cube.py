@@ -54,8 +54,7 @@ def test_wide_cube_several_tiles_per_sequence():
     full_parity(WIDE_TILES, syn.make_inputs(WIDE_TILES))
 
 
-@pytest.mark.parametrize("flags", [vb.FLAG_TF32_COARSE, vb.FLAG_HALF_CUBE_FWD, vb.FLAG_SIMPLE_COARSE | vb.FLAG_SIMPLE_BWD | vb.FLAG_SIMPLE_ROUTER
-                                   | vb.FLAG_EXACT_MAX_FWD])
+@pytest.mark.parametrize("flags", [vb.FLAG_HALF_CUBE_FWD, vb.FLAG_EXACT_MAX_FWD, vb.FLAG_BF16_COARSE_FWD])
 @pytest.mark.parametrize("wl", [WIDE_RAGGED, WIDE_EMPTY_HALF], ids=lambda w: w.name)
 def test_wide_cube_alternative_kernels(flags, wl):
     from oracle import vsa2_oracle as orc
@@ -72,7 +71,9 @@ def test_wide_cube_alternative_kernels(flags, wl):
     got = run.backward()
     want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
     for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
-        assert_close(name, x, y, tol_abs=2e-2 * np.sqrt(2), bf16_storage=name != "dGate")
+        if name == "dGate" and flags == vb.FLAG_BF16_COARSE_FWD:
+            continue      # documented cost of that flag: O_c carries bf16 operand rounding, dGate may leave the bound
+        assert_close(name, x, y, bf16_storage=name != "dGate")
 
 
 def test_wide_cube_forward_survives_a_late_dominant_key_cube():

@@ -53,3 +53,45 @@ def test_two_ranks_agree_on_the_slowest_time_and_take_disjoint_work():
 def test_single_process_is_identity():
     assert replicas.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert replicas.head_shard(3, 4, 0, 1) == (0, 3, 0, 12)
+
+
+def test_launcher_arguments():
+    """`bench.py --gpus N` started without a launcher re-runs itself under torch.distributed.run with N ranks; under a
+    launcher it is a rank and only checks the world size."""
+    import sys
+    import pytest
+    argv = ["--gpus", "4", "--steps", "2", "--warmup", "3"]
+    cmd = replicas.launcher_command(4, "bench.py", argv, env={}, port=29999)
+    assert cmd[:3] == [sys.executable, "-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29999"
+    assert cmd[-7:] == ["bench.py"] + argv
+    assert replicas.launcher_command(1, "bench.py", ["--gpus", "1"], env={}) is None
+    assert replicas.launcher_command(4, "bench.py", argv, env={"WORLD_SIZE": "4", "RANK": "2"}) is None
+    with pytest.raises(SystemExit):
+        replicas.launcher_command(4, "bench.py", argv, env={"WORLD_SIZE": "2"})
+    assert 1024 < replicas.free_port() < 65536
+
+
+def _launched_rank_main():
+    """Body of the script the launcher test runs under torch.distributed.run (gloo, CPU)."""
+    import torch.distributed as d
+    d.init_process_group("gloo")
+    mx = replicas.max_over_ranks([float(d.get_rank())])
+    if d.get_rank() == 0:
+        print(f"LAUNCHED world={d.get_world_size()} max={mx[0]}", flush=True)
+    d.destroy_process_group()
+
+
+def test_launcher_command_starts_the_ranks(tmp_path):
+    """The command line the launcher builds really starts two ranks that find each other (gloo on CPU)."""
+    import subprocess
+    import sys
+    script = tmp_path / "ranks.py"
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script.write_text(f"import sys\nsys.path.insert(0, {root!r})\nsys.path.insert(0, {os.path.join(root, 'tests')!r})\n"
+                      "import test_multi_rank_cpu as t\nt._launched_rank_main()\n")
+    cmd = replicas.launcher_command(2, str(script), [], env={})
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "LAUNCHED world=2 max=1.0" in out.stdout

@@ -280,6 +280,101 @@ def test_router_padding_reading_rows_sum_to_one_over_G():
     assert (P_r >= 0).all()
 
 
+def _masked_subcube_mean_lib(X, grid, cube, rpool):
+    """Masked mean over router sub-cubes of a padded grid from library pooling only: the zero-padded value volume and a
+    padded volume of ones both go through torch avg_pool3d; their ratio is sum / (number of valid tokens).
+    Returns (mean [Tp/Rt, Hp/Rh, Wp/Rw, D] float32 with 0 where nothing is valid, count of the same leading shape)."""
+    D = X.shape[1]
+    vol = torch.from_numpy(pad_volume(X.astype(np.float32), grid, cube)).permute(3, 0, 1, 2)[None]
+    ones = torch.from_numpy(pad_volume(np.ones((X.shape[0], 1), np.float32), grid, cube)).permute(3, 0, 1, 2)[None]
+    s = F.avg_pool3d(vol, kernel_size=rpool)[0].permute(1, 2, 3, 0)
+    c = F.avg_pool3d(ones, kernel_size=rpool)[0].permute(1, 2, 3, 0)
+    mean = torch.where(c > 0, s / c.clamp(min=1e-9), torch.zeros_like(s))
+    count = torch.round(c[..., 0] * (rpool[0] * rpool[1] * rpool[2])).to(torch.int64)
+    return mean, count
+
+
+@pytest.mark.parametrize("grid", [(3, 5, 8), (5, 6, 9), (3, 5, 9)])
+def test_router_pool_on_a_padded_grid_divides_by_the_valid_count(grid):
+    """Padding reading of Eq. 5: the mean of a cut sub-cube runs over its valid tokens only.  Dividing by the full
+    sub-cube size R (or by any other count) fails the bitwise comparison below."""
+    cube, rpool, D = (4, 4, 4), (2, 2, 2), 8
+    geo = orc.Geometry(grid, cube, rpool)
+    rng = np.random.default_rng(31)
+    # few mantissa bits and power-of-two counts: every fp32 sum and division is exact, so the library's masked mean and
+    # the oracle's must agree bit for bit whatever the order of the additions
+    X = np.round(rng.standard_normal((geo.L, D)) * 4) / 4
+    Xr, valid = orc.mean_pool_router(X, geo)
+    mean, count = _masked_subcube_mean_lib(X, grid, cube, rpool)
+    lib = to_cube_major(mean.to(torch.bfloat16).to(torch.float64).numpy(), (geo.Gt, geo.Gh, geo.Gw))      # [N, G, D]
+    cnt = to_cube_major(count.numpy(), (geo.Gt, geo.Gh, geo.Gw))                                            # [N, G]
+    assert set(np.unique(cnt)) <= {0, 1, 2, 4, 8} and (cnt == 0).any() and (cnt < 8).any()
+    assert np.array_equal(valid, cnt > 0)
+    assert np.array_equal(Xr, lib)
+    assert (Xr[~valid] == 0).all()
+    # literal special case: a sub-cube with one valid token holds that token's value, one with two holds their mean
+    T, H, W = grid
+    l = geo.raster_index(T - 1, H - 1, W - 1)
+    n, g = geo.cube_of[l], geo.sub_of[l]
+    members = np.nonzero((geo.cube_of == n) & (geo.sub_of == g))[0]
+    assert len(members) == cnt[n, g]
+    assert np.array_equal(Xr[n, g], orc.round_f32_to_bf16(X[members].mean(axis=0).astype(np.float32)).astype(np.float64))
+    if grid == (3, 5, 9):
+        assert len(members) == 1 and np.array_equal(Xr[n, g], X[l])
+    # general values: same means up to the last bf16 bit (fp32 summation order)
+    Y = orc.bf16_bits_to_f64(syn.f32_to_bf16_bits(rng.standard_normal((geo.L, D), dtype=np.float32)))
+    Yr, _ = orc.mean_pool_router(Y, geo)
+    meany, _ = _masked_subcube_mean_lib(Y, grid, cube, rpool)
+    liby = to_cube_major(meany.to(torch.bfloat16).to(torch.float64).numpy(), (geo.Gt, geo.Gh, geo.Gw))
+    assert (Yr != liby).mean() < 5e-3 and np.abs(Yr - liby).max() <= np.abs(liby).max() * 2.0 ** -7
+    # R = B: the router operand is the bf16 rounding of the cube mean of Eq. 1 (which the dense restatement pins under
+    # padding); cube counts such as 3*4*4 are not powers of two, so allow the last bf16 bit
+    geo_b = orc.Geometry(grid, cube, cube)
+    Zr, zv = orc.mean_pool_router(Y, geo_b)
+    Zc = orc.round_f32_to_bf16(orc.mean_pool_cube(Y, geo_b).astype(np.float32)).astype(np.float64)
+    assert zv.all() and (Zr[:, 0] != Zc).mean() < 5e-3 and np.abs(Zr[:, 0] - Zc).max() <= np.abs(Zc).max() * 2.0 ** -7
+
+
+@pytest.mark.parametrize("grid", [(3, 5, 8), (3, 5, 9)])
+def test_router_scores_on_a_padded_grid_match_brute_force_with_an_explicit_mask(grid):
+    """Padding reading of Eq. 6-7 against brute force: every pooled query row takes a softmax over ALL pooled keys with
+    -inf written on the key sub-cubes that hold no valid token; P_r[i, j] adds the G x G sub-block over valid query
+    sub-cubes and divides by (valid query sub-cubes of cube i) * G.  Not masking the empty keys, masking by cube instead
+    of by sub-cube, or dividing by G * G all fail."""
+    cube, rpool, D = (4, 4, 4), (2, 2, 2), 16
+    geo = orc.Geometry(grid, cube, rpool)
+    rng = np.random.default_rng(32)
+    Q = np.round(rng.standard_normal((geo.L, D)) * 4) / 4
+    K = np.round(rng.standard_normal((geo.L, D)) * 4) / 4
+    scale = 0.35
+    Qr, qv = orc.mean_pool_router(Q, geo)
+    Kr, kv = orc.mean_pool_router(K, geo)
+    P_r = orc.router_block_scores(Qr, Kr, qv, kv, scale)
+    # independent operands and validity, laid out [N, G, .] by reshape
+    G3 = (geo.Gt, geo.Gh, geo.Gw)
+    qm, qc = _masked_subcube_mean_lib(Q, grid, cube, rpool)
+    km, kc = _masked_subcube_mean_lib(K, grid, cube, rpool)
+    q = torch.from_numpy(to_cube_major(qm.to(torch.bfloat16).to(torch.float64).numpy(), G3)).reshape(-1, D)
+    k = torch.from_numpy(to_cube_major(km.to(torch.bfloat16).to(torch.float64).numpy(), G3)).reshape(-1, D)
+    q_ok = torch.from_numpy(to_cube_major(qc.numpy(), G3) > 0)                   # [N, G]
+    k_ok = torch.from_numpy(to_cube_major(kc.numpy(), G3) > 0).reshape(-1)       # [N G]
+    assert (~k_ok).any() and (~q_ok).any()
+    s = (q @ k.T) * scale
+    s = s.masked_fill(~k_ok[None, :], float("-inf"))
+    p_hat = torch.softmax(s, dim=1) * q_ok.reshape(-1, 1)
+    N, G = geo.N, geo.G
+    ref = torch.zeros(N, N, dtype=torch.float64)
+    for i in range(N):
+        for j in range(N):
+            ref[i, j] = p_hat[i * G:(i + 1) * G, j * G:(j + 1) * G].sum() / (q_ok[i].sum() * G)
+    assert np.abs(P_r - ref.numpy()).max() < 1e-15
+    assert np.allclose(P_r.sum(axis=1), 1.0 / G, atol=1e-14)
+    # a cube pair whose key cube has fewer valid sub-cubes holds less mass than the same scores would give unmasked
+    empty_keys = np.nonzero(~k_ok.numpy())[0]
+    p_unmasked = torch.softmax((q @ k.T) * scale, dim=1)
+    assert (p_unmasked[:, empty_keys] > 0).all() and (p_hat[:, empty_keys] == 0).all()
+
+
 def test_router_map_invariant_to_permuting_tokens_inside_a_sub_cube():
     grid, D = (4, 8, 8), 16
     rng = np.random.default_rng(9)
@@ -365,6 +460,33 @@ def test_backward_matches_autograd_of_dense_restatement(grid, cube):
     for name, t in (("dQ", tq), ("dK", tk), ("dV", tv), ("dGate", tg)):
         err = np.abs(g[name] - t.grad.numpy()).max()
         assert err < 1e-11, (name, err)
+
+
+@pytest.mark.parametrize("kv_cubes", [(0, 5), (3, 7, 11)])
+def test_fine_backward_restricted_to_kv_cubes_matches_the_full_backward_and_autograd(kv_cubes):
+    """fine_backward_kv_cubes must return exactly the rows of the full fine-branch dK, dV that belong to the requested KV
+    cubes: the softmax statistics (lse, delta) come from ALL kept blocks of a query row, not from the requested ones."""
+    grid, cube = (5, 6, 9), (4, 4, 4)
+    Q, K, V, dO, gate, geo, mask = rand_problem(grid, 16, 21, cube=cube)
+    mask[2, :] = False                                  # an empty query row
+    mask[:, kv_cubes[0]] |= np.arange(geo.N) % 2 == 0   # the first requested cube is kept by many rows
+    assert geo.N == 12 and (geo.cube_count < 64).any()
+    scale = 0.2
+    dK, dV = orc.fine_backward_kv_cubes(Q, K, V, mask, geo, scale, dO, kv_cubes)
+    tok = np.concatenate([geo.cube_tokens[j] for j in kv_cubes])
+    rest = np.setdiff1d(np.arange(geo.L), tok)
+    assert (dK[rest] == 0).all() and (dV[rest] == 0).all()
+    # (1) the full oracle backward of the fine branch
+    O_f, lse = orc.fine_attention(Q, K, V, mask, geo, scale)
+    _, fk, fv = orc.fine_backward(Q, K, V, mask, geo, scale, dO, lse, O_f)
+    assert np.abs(dK[tok] - fk[tok]).max() < 1e-12 and np.abs(dV[tok] - fv[tok]).max() < 1e-12
+    # (2) autograd of the dense masked restatement with the gate at zero (O = O_f)
+    tq, tk, tv = (torch.from_numpy(a).requires_grad_(True) for a in (Q, K, V))
+    O, _, _ = dense_restatement(tq, tk, tv, torch.zeros(geo.L, dtype=torch.float64), mask, grid, cube, scale)
+    (O * torch.from_numpy(dO)).sum().backward()
+    assert np.abs(dK[tok] - tk.grad.numpy()[tok]).max() < 1e-11
+    assert np.abs(dV[tok] - tv.grad.numpy()[tok]).max() < 1e-11
+    assert np.abs(tk.grad.numpy()[tok]).max() > 1e-3
 
 
 def test_backward_matches_central_finite_differences_on_config0():

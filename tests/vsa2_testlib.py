@@ -5,12 +5,10 @@ Tolerances (fp32 comparison against the fp64 oracle):
   outputs and gradients: max abs err <= 2e-2 and mean rel err <= 5e-3, where
                          mean rel err = mean|a - b| / mean|b| over the tensor;
   lse:                   max abs err <= 1e-3 where finite, -inf must match -inf;
-                         When the library stores a tensor in bf16 (out_dtype BF16) the storage rounding,
-                         up to 2^-8 |x| per element (half an ulp at the bottom of a binade), comes on top: the
-                         elementwise bound is then 2e-2 + 2^-8 |ref|; runs with fp32 outputs are held to the plain 2e-2.
-                         dK and dV of a GQA group are sums over the group's `rep` query heads, each within
-                         the bound above; independent rounding noise adds in quadrature, so group-summed dK, dV are
-                         held to sqrt(rep) * 2e-2 (rep = 1 for MHA: unchanged).
+                         Runs with fp32 outputs (out_dtype F32) are held to exactly these bounds, MHA and GQA alike.
+                         When the library stores a tensor in bf16 (out_dtype BF16) the storage rounding alone,
+                         up to 2^-8 |x| per element (half an ulp at the bottom of a binade), can exceed 2e-2 for
+                         |x| > 5: the elementwise bound of such runs is 2e-2 + 2^-8 |ref|.
   routing:               the map must equal the oracle's except at entries whose oracle score lies
                          within 1e-3 * tau (relative) of the threshold tau = smallest kept score of
                          that (batch, head) [per-sequence] or row [per-query]; counts must be exact.
@@ -140,12 +138,20 @@ def sampled_attention_parity(wl, data, run, gmask, q_heads, rows, kv_groups=(), 
     """Oracle vs GPU on sampled outputs of a full-size run (the full oracle would take hours):
     O, lse, dQ, dGate on the tokens of the query cubes `rows` of the query heads `q_heads`; dK, dV on the tokens
     of `kv_cubes` for the KV heads `kv_groups` (all query heads of the group, all query blocks that keep the cube).
-    `run` must have executed forward (and backward).  bf16 outputs are assumed."""
+    `run` is a CudaPath that has executed forward (and backward), or a list of them over the same inputs and map (e.g.
+    one with bf16 and one with fp32 outputs): the oracle's sample is computed once and every run is held to the bound
+    of its own output dtype.  Returns {tensor name: (max abs err, mean rel err)} of the last run."""
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
     scale = 1.0 / np.sqrt(wl.head_dim)
     rep = wl.heads_q // wl.heads_kv
-    o_gpu, lse_gpu = run.o, run.lse
+    runs = list(run) if isinstance(run, (list, tuple)) else [run]
     stats = {}
+
+    def check(name, field, idx, ref, plain=False):
+        for r in runs:
+            st = (not plain) and r.p.out_dtype == vb.BF16
+            stats[name] = assert_close(f"{name} ({'bf16' if r.p.out_dtype == vb.BF16 else 'fp32'} outputs)",
+                                       to_f64(getattr(r, field)[idx[0], idx[1]][idx[2]]), ref, bf16_storage=st)
 
     def head_arrays(b, hq):
         hk = hq // rep
@@ -165,13 +171,14 @@ def sampled_attention_parity(wl, data, run, gmask, q_heads, rows, kv_groups=(), 
         toks = np.concatenate([geo.cube_tokens[i] for i in rows])
         O_f, lse = orc.fine_attention(Q, K, V, gmask[b, hq], geo, scale, rows=rows)
         O_ref = gate[toks, None] * fwd["Oc_hat"][geo.cube_of[toks]] + O_f[toks]
-        stats[f"O_h{hq}"] = assert_close(f"O head {hq}", to_f64(o_gpu[b, hq][toks]), O_ref, bf16_storage=True)
-        assert_lse_close(to_f64(lse_gpu[b, hq][toks]), lse[toks])
+        check(f"O_h{hq}", "o", (b, hq, toks), O_ref)
+        for r in runs:
+            assert_lse_close(to_f64(r.lse[b, hq][toks]), lse[toks])
         if backward:
             c = orc.coarse_path_backward(Q, K, V, gate, geo, scale, dO, fwd)
             fq, _, _ = orc.fine_backward(Q, K, V, gmask[b, hq], geo, scale, dO, lse, O_f, rows=rows)
-            stats[f"dQ_h{hq}"] = assert_close(f"dQ head {hq}", to_f64(run.dq[b, hq][toks]), (c["dQ"] + fq)[toks], bf16_storage=True)
-            assert_close(f"dGate head {hq}", to_f64(run.dgate[b, hq][toks]), c["dGate"][toks])
+            check(f"dQ_h{hq}", "dq", (b, hq, toks), (c["dQ"] + fq)[toks])
+            check(f"dGate_h{hq}", "dgate", (b, hq, toks), c["dGate"][toks], plain=True)
     if backward:
         for hk in kv_groups:
             toks = np.concatenate([geo.cube_tokens[j] for j in kv_cubes])
@@ -184,7 +191,6 @@ def sampled_attention_parity(wl, data, run, gmask, q_heads, rows, kv_groups=(), 
                 fk, fv = orc.fine_backward_kv_cubes(Q, K, V, gmask[b, hq], geo, scale, dO, kv_cubes)
                 dK_ref += (c["dK"] + fk)[toks]
                 dV_ref += (c["dV"] + fv)[toks]
-            tol = TOL_ABS * np.sqrt(rep)
-            stats[f"dK_g{hk}"] = assert_close(f"dK kv head {hk}", to_f64(run.dk[b, hk][toks]), dK_ref, tol_abs=tol, bf16_storage=True)
-            stats[f"dV_g{hk}"] = assert_close(f"dV kv head {hk}", to_f64(run.dv[b, hk][toks]), dV_ref, tol_abs=tol, bf16_storage=True)
+            check(f"dK_g{hk}", "dk", (b, hk, toks), dK_ref)
+            check(f"dV_g{hk}", "dv", (b, hk, toks), dV_ref)
     return stats
