@@ -67,6 +67,11 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
 enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
                                          (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
+enum { VSA2_FLAG_FAST_BWD = 4 };      /* backward passes with P and dS rounded once to bf16 before the dV, dK and dQ products
+                                         (about 10-20 % faster).  By default both are carried as a bf16 value plus the bf16
+                                         rounding of what that lost, which keeps dQ, dK, dV inside max abs err 2e-2 where
+                                         gradients are large (|g| > 5: sharply peaked rows, GQA groups); with this flag the
+                                         worst elements reach 2.5e-2 (MHA, 720p) to 3.7e-2 (GQA 4:1, 480p) */
 enum { VSA2_FLAG_HALF_CUBE_FWD = 128 };/* 128-token cubes only: fine forward with the 64-query kernel on the two half-cubes
                                          separately instead of the 128-query kernel (validation aid, same results) */
 enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV group share one block map ("group head", Sec. 4

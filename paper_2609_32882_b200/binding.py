@@ -19,6 +19,7 @@ PER_SEQUENCE, PER_QUERY, PER_QUERY_BUDGET = 0, 1, 2
 BF16, F32 = 0, 1
 FLAG_NO_COARSE = 1
 FLAG_EXACT_MAX_FWD = 2
+FLAG_FAST_BWD = 4
 FLAG_BF16_COARSE_FWD = 64
 FLAG_HALF_CUBE_FWD = 128
 FLAG_GROUP_ROUTING = 256

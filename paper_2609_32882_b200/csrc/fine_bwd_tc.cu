@@ -33,17 +33,19 @@ static_assert(kRingB == 2, "ring B shares its slot index with the two accumulato
 // Shared-memory plan of both passes (D = 128: 5 x 32 KB ring slots, 2 x 16 KB stationary tiles, 2 x 16 KB operand
 // buffers, 2 KB of barriers and per-block vectors: exactly the 227 KB a block may use).  Ring A has 3 slots, ring B 2;
 // each ring has one producing warp and fixed consuming roles.
-template <int D>
+// RA: slots of ring A; NP: 16 KB operand buffers (the dK/dV pass in its split mode trades one ring-A slot for the two
+// buffers that hold the low-order parts of P and dS).
+template <int D, int RA = kRingA, int NP = 2>
 struct BwdTc {
   static constexpr int DH = D / 64;
   static constexpr uint32_t SLOT = 2 * DH * kSlab;   // a pair of cube tiles, [half][A | B]
   static constexpr uint32_t TILE = DH * kSlab;       // one cube tile, [half]
   static constexpr uint32_t PBYTES = 128 * 128;      // 128 rows x 64 bf16
-  static constexpr uint32_t OFF_RING_B = kRingA * SLOT;
-  static constexpr uint32_t OFF_ST0 = (kRingA + kRingB) * SLOT;   // stationary tile 0 (Q or K)
+  static constexpr uint32_t OFF_RING_B = RA * SLOT;
+  static constexpr uint32_t OFF_ST0 = (RA + kRingB) * SLOT;       // stationary tile 0 (Q or K)
   static constexpr uint32_t OFF_ST1 = OFF_ST0 + TILE;             // stationary tile 1 (dO or V)
-  static constexpr uint32_t OFF_P = OFF_ST1 + TILE;               // two 16 KB operand buffers
-  static constexpr uint32_t OFF_MISC = OFF_P + 2 * PBYTES;
+  static constexpr uint32_t OFF_P = OFF_ST1 + TILE;               // the 16 KB operand buffers
+  static constexpr uint32_t OFF_MISC = OFF_P + NP * PBYTES;
   static constexpr uint32_t MISC_BYTES = 2048;
   static constexpr size_t smem_bytes = OFF_MISC + MISC_BYTES + 1024;
 };
@@ -135,7 +137,10 @@ struct DqArgs {
 // the stationary Q and dO tiles, warp 1 = TMA producer of the V pairs (ring B), warp 2 = issuer of S^T, warp 3 = issuer
 // of dP^T, warp 12 = issuer of dQ^T += K_pair^T dS^T, warps 4..11 = elementwise stage + epilogue (each half of the query
 // columns): P is formed from S^T while dP^T is still being computed.
-template <int D>
+// SPLIT: dS^T is handed to the dQ^T product as [bf16(dS^T) | bf16(dS^T - bf16(dS^T))] (one N = 128 product into two
+// accumulator halves that the epilogue adds), which removes the bf16 rounding of dS from dQ; the two operand buffers
+// then hold one tile (hi, lo) instead of two tiles.
+template <int D, bool SPLIT>
 __global__ void __launch_bounds__(kDqThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, Geo g,
@@ -169,7 +174,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
-  // tensor-memory columns: S^T buffers 0, 64; dP^T buffers 128, 192; dQ^T 256
+  // tensor-memory columns: S^T buffers 0, 64; dP^T buffers 128, 192; dQ^T 256 (SPLIT: its low-order part at 320)
 
   if (warp < 2) {
     // ------------------------------------------------------------------ TMA producers
@@ -273,10 +278,11 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int nt = (k + 1) >> 1;
         VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);
         for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t sd = tg & 1, pd = (tg >> 1) & 1, sa = tg % kRingA;
+          const uint32_t sd = SPLIT ? 0u : (tg & 1), pd = SPLIT ? (tg & 1) : ((tg >> 1) & 1), sa = tg % kRingA;
           VSA2_WAIT(&misc->ds_ready[sd], pd);
           tc::tc_fence_after();
-          mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
+          if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr, C::PBYTES, t > 0);
+          else mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
           tc::mma_commit(&misc->a_empty[sa]);
           tc::mma_commit(&misc->ds_free[sd]);
         }
@@ -321,7 +327,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t s = tg & 1, par = (tg >> 1) & 1;
           const bool dup = (blk == 1) && (2 * t + 1 >= k);
-          uint32_t packed[16];
+          uint32_t packed[16], packed_lo[SPLIT ? 16 : 1];
           {
             uint32_t sv[32];      // S^T, then P^T
             VSA2_WAIT(&misc->s_full[s], par);
@@ -354,20 +360,35 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
               const float d1 = __uint_as_float(sv[4 * c4 + 1]) * (__uint_as_float(dp[4 * c4 + 1]) - dl.y) * g.scale;
               const float d2 = __uint_as_float(sv[4 * c4 + 2]) * (__uint_as_float(dp[4 * c4 + 2]) - dl.z) * g.scale;
               const float d3 = __uint_as_float(sv[4 * c4 + 3]) * (__uint_as_float(dp[4 * c4 + 3]) - dl.w) * g.scale;
-              packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
-              packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
+              if constexpr (SPLIT) {
+                uint32_t h0, l0, h1, l1;
+                split_bf16x2(d0, d1, h0, l0);
+                split_bf16x2(d2, d3, h1, l1);
+                packed[2 * c4] = valid ? h0 : 0u;
+                packed[2 * c4 + 1] = valid ? h1 : 0u;
+                packed_lo[2 * c4] = valid ? l0 : 0u;
+                packed_lo[2 * c4 + 1] = valid ? l1 : 0u;
+              } else {
+                packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
+                packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
+              }
             }
           }
-          VSA2_WAIT(&misc->ds_free[s], par ^ 1);
+          const uint32_t sd = SPLIT ? 0u : s;
+          VSA2_WAIT(&misc->ds_free[sd], SPLIT ? ((tg & 1) ^ 1) : (par ^ 1));
           {
-            unsigned char* prow = ds_tile + s * C::PBYTES + row * 128;
+            unsigned char* prow = ds_tile + sd * C::PBYTES + row * 128;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch)
+            for (int ch = 0; ch < 4; ++ch) {
               *reinterpret_cast<uint4*>(prow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
                   make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+              if constexpr (SPLIT)
+                *reinterpret_cast<uint4*>(prow + C::PBYTES + (((half * 4 + ch) ^ (row & 7)) << 4)) =
+                    make_uint4(packed_lo[4 * ch], packed_lo[4 * ch + 1], packed_lo[4 * ch + 2], packed_lo[4 * ch + 3]);
+            }
           }
           tc::fence_proxy_async_smem();
-          tc::mbar_arrive(&misc->ds_ready[s]);
+          tc::mbar_arrive(&misc->ds_ready[sd]);
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
@@ -378,6 +399,13 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         if (k > 0) {
           tc::tmem_ld32(lane_addr + 256 + half * 32, o0);
           tc::tmem_ld_wait();
+          if constexpr (SPLIT) {
+            uint32_t o1[32];
+            tc::tmem_ld32(lane_addr + 320 + half * 32, o1);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o0[c] = __float_as_uint(__uint_as_float(o0[c]) + __uint_as_float(o1[c]));
+          }
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->o_empty);
         } else {
@@ -467,18 +495,24 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b,
 // elementwise stage + epilogue (each half of the key columns): P is handed to the dV^T product before dS is formed;
 // warps 12..15 = one thread per query row of the tile: they look up the row's (head, block, token) and fetch its lse and
 // delta one tile ahead, so that the elementwise warps, which bound the pass, touch no global memory inside a tile.
-template <int D>
+// SPLIT: P and dS are handed to the dV^T and dK^T products as [bf16(X) | bf16(X - bf16(X))] (N = 128 products into two
+// accumulator halves that the epilogue adds), which removes their bf16 rounding from dV and dK: a KV block sums hundreds of
+// query blocks (times the query heads of a GQA group), and with plain bf16 operands that noise alone passes 2e-2.  The two
+// extra operand buffers take the place of the third ring-A slot.
+template <int D, bool SPLIT>
 __global__ void __launch_bounds__(kDkvThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, Geo g,
                        DkvArgs a) {
-  using C = BwdTc<D>;
+  constexpr int RA = SPLIT ? 2 : kRingA;                   // slots of the Q ring
+  constexpr uint32_t TM_DK = 256, TM_DV = SPLIT ? 384 : 320;
+  using C = BwdTc<D, RA, SPLIT ? 4 : 2>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* k_tile = smem + C::OFF_ST0;
   unsigned char* v_tile = smem + C::OFF_ST1;
-  unsigned char* p_tile = smem + C::OFF_P;                 // P  [128 q, 64 kv]
-  unsigned char* ds_tile = smem + C::OFF_P + C::PBYTES;    // dS [128 q, 64 kv]
+  unsigned char* p_tile = smem + C::OFF_P;                                  // P  [128 q, 64 kv] (SPLIT: followed by its low part)
+  unsigned char* ds_tile = smem + C::OFF_P + (SPLIT ? 2 : 1) * C::PBYTES;   // dS [128 q, 64 kv] (SPLIT: followed by its low part)
   BwdMisc* misc = reinterpret_cast<BwdMisc*>(smem + C::OFF_MISC);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -504,7 +538,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem_base = misc->tmem_base;
-  // tensor-memory columns: S buffers 0, 64; dP buffers 128, 192; dK^T 256; dV^T 320
+  // tensor-memory columns: S buffers 0, 64; dP buffers 128, 192; dK^T 256; dV^T 320 (SPLIT: dK^T 256 + 320, dV^T 384 + 448)
 
   // per item: prefix of the per-head column counts and the list starts (every role recomputes them)
 #define VSA2_DKV_ITEM_SETUP()                                                            \
@@ -561,7 +595,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         cube_coords(g, i_l, it_, ih_, iw_);
         const int bhq_t = bhq_l;
         if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
-        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
+        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, RA, smem, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
         else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
       }
     }
@@ -582,7 +616,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t sb = tg & 1, pb = (tg >> 1) & 1;
           if (is_s) {
-            const uint32_t sa = tg % kRingA, pa = (tg / kRingA) & 1;
+            const uint32_t sa = tg % RA, pa = (tg / RA) & 1;
             VSA2_WAIT_PARKED(&misc->a_full[sa], pa);
             VSA2_WAIT_PARKED(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
@@ -622,14 +656,16 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             VSA2_WAIT_PARKED(&misc->b_full[sv], (tg >> 1) & 1);
             VSA2_WAIT_PARKED(&misc->p_ready, tg & 1);
             tc::tc_fence_after();
-            mma_pairT_mnmajor<D>(tmem_base + 320, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
+            if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, C::PBYTES, t > 0);
+            else mma_pairT_mnmajor<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
             tc::mma_commit(&misc->b_empty[sv]);
             tc::mma_commit(&misc->p_free);
           } else {
-            const uint32_t sa = tg % kRingA;
+            const uint32_t sa = tg % RA;
             VSA2_WAIT_PARKED(&misc->ds_ready[0], tg & 1);
             tc::tc_fence_after();
-            mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, b_addr, t > 0);
+            if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, C::PBYTES, t > 0);
+            else mma_pairT_mnmajor<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
             tc::mma_commit(&misc->a_empty[sa]);
             tc::mma_commit(&misc->ds_free[0]);
           }
@@ -720,7 +756,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->s_free[s]);
           {
-            uint32_t pp[16];
+            uint32_t pp[16], pl[SPLIT ? 16 : 1];
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
               float p0 = ex2_approx(fmaf(__uint_as_float(sv[c]), c2, -lse2));
@@ -731,19 +767,24 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               }
               sv[c] = __float_as_uint(p0);
               sv[c + 1] = __float_as_uint(p1);
-              pp[c >> 1] = pack_bf16x2(p0, p1);
+              if constexpr (SPLIT) split_bf16x2(p0, p1, pp[c >> 1], pl[c >> 1]);
+              else pp[c >> 1] = pack_bf16x2(p0, p1);
             }
             VSA2_WAIT(&misc->p_free, (tg & 1) ^ 1);
             unsigned char* prow = p_tile + row * 128;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch)
+            for (int ch = 0; ch < 4; ++ch) {
               *reinterpret_cast<uint4*>(prow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
                   make_uint4(pp[4 * ch], pp[4 * ch + 1], pp[4 * ch + 2], pp[4 * ch + 3]);
+              if constexpr (SPLIT)
+                *reinterpret_cast<uint4*>(prow + C::PBYTES + (((half * 4 + ch) ^ (row & 7)) << 4)) =
+                    make_uint4(pl[4 * ch], pl[4 * ch + 1], pl[4 * ch + 2], pl[4 * ch + 3]);
+            }
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&misc->p_ready);
           }
           {
-            uint32_t dp[32], pd[16];
+            uint32_t dp[32], pd[16], pdl[SPLIT ? 16 : 1];
             VSA2_WAIT(&misc->dp_full[s], par);
             tc::tc_fence_after();
             tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
@@ -754,14 +795,19 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int c = 0; c < 32; c += 2) {
               const float d0 = __uint_as_float(sv[c]) * (__uint_as_float(dp[c]) - dlt) * g.scale;
               const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
-              pd[c >> 1] = pack_bf16x2(d0, d1);
+              if constexpr (SPLIT) split_bf16x2(d0, d1, pd[c >> 1], pdl[c >> 1]);
+              else pd[c >> 1] = pack_bf16x2(d0, d1);
             }
             VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
             unsigned char* drow = ds_tile + row * 128;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch)
+            for (int ch = 0; ch < 4; ++ch) {
               *reinterpret_cast<uint4*>(drow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
                   make_uint4(pd[4 * ch], pd[4 * ch + 1], pd[4 * ch + 2], pd[4 * ch + 3]);
+              if constexpr (SPLIT)
+                *reinterpret_cast<uint4*>(drow + C::PBYTES + (((half * 4 + ch) ^ (row & 7)) << 4)) =
+                    make_uint4(pdl[4 * ch], pdl[4 * ch + 1], pdl[4 * ch + 2], pdl[4 * ch + 3]);
+            }
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&misc->ds_ready[0]);
           }
@@ -773,9 +819,20 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       {
         uint32_t kk[32], vv[32];
         if (k > 0) {
-          tc::tmem_ld32(lane_addr + 256 + half * 32, kk);
-          tc::tmem_ld32(lane_addr + 320 + half * 32, vv);
+          tc::tmem_ld32(lane_addr + TM_DK + half * 32, kk);
+          tc::tmem_ld32(lane_addr + TM_DV + half * 32, vv);
           tc::tmem_ld_wait();
+          if constexpr (SPLIT) {
+            uint32_t lo[32];
+            tc::tmem_ld32(lane_addr + TM_DK + 64 + half * 32, lo);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) kk[c] = __float_as_uint(__uint_as_float(kk[c]) + __uint_as_float(lo[c]));
+            tc::tmem_ld32(lane_addr + TM_DV + 64 + half * 32, lo);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) vv[c] = __float_as_uint(__uint_as_float(vv[c]) + __uint_as_float(lo[c]));
+          }
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->o_empty);
         } else {
@@ -859,13 +916,22 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
   DqArgs a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, dq, status};
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
+  const bool split = !(g.flags & VSA2_FLAG_FAST_BWD);
+#define VSA2_LAUNCH_DQ(DD, SP)                                                                                                   \
+  do {                                                                                                                           \
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                    \
+                                  (int)BwdTc<DD>::smem_bytes)))                                                                  \
+      return e;                                                                                                                  \
+    fine_bwd_dq_tc_kernel<DD, SP><<<grid, kDqThreads, BwdTc<DD>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);                       \
+  } while (0)
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
-    fine_bwd_dq_tc_kernel<128><<<grid, kDqThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if (split) VSA2_LAUNCH_DQ(128, true);
+    else VSA2_LAUNCH_DQ(128, false);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
-    fine_bwd_dq_tc_kernel<64><<<grid, kDqThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if (split) VSA2_LAUNCH_DQ(64, true);
+    else VSA2_LAUNCH_DQ(64, false);
   }
+#undef VSA2_LAUNCH_DQ
   return cudaGetLastError();
 }
 
@@ -884,13 +950,23 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   DkvArgs a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
+  const bool split = !(g.flags & VSA2_FLAG_FAST_BWD);
+#define VSA2_LAUNCH_DKV(DD, SP)                                                                                                  \
+  do {                                                                                                                           \
+    using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                   \
+                                  (int)L_::smem_bytes)))                                                                         \
+      return e;                                                                                                                  \
+    fine_bwd_dkv_tc_kernel<DD, SP><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);                            \
+  } while (0)
   if (g.D == 128) {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<128>::smem_bytes))) return e;
-    fine_bwd_dkv_tc_kernel<128><<<grid, kDkvThreads, BwdTc<128>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if (split) VSA2_LAUNCH_DKV(128, true);
+    else VSA2_LAUNCH_DKV(128, false);
   } else {
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BwdTc<64>::smem_bytes))) return e;
-    fine_bwd_dkv_tc_kernel<64><<<grid, kDkvThreads, BwdTc<64>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);
+    if (split) VSA2_LAUNCH_DKV(64, true);
+    else VSA2_LAUNCH_DKV(64, false);
   }
+#undef VSA2_LAUNCH_DKV
   return cudaGetLastError();
 }
 

@@ -57,6 +57,31 @@ __device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_sl
   }
 }
 
+// The same product with 128 columns: B is two 128-row tiles side by side, `b_stride` bytes apart (columns 0..63 from the first,
+// 64..127 from the second), acc[D, 128].  Used with B = [X_hi | X_lo], the bf16 rounding of X and the bf16 rounding of what
+// that lost: the two column halves of the accumulator then sum to A^T X at about 16 bits of operand precision, for one
+// N = 128 instruction (64 cycles) per step instead of two N = 64 instructions (2 x 48).
+template <int D>
+__device__ __forceinline__ void mma_pairT_mnmajor_n128(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, uint32_t b_stride,
+                                                       bool accumulate_first) {
+  constexpr uint32_t idesc = tc::idesc_bf16(128, 128, true, true);
+  constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;
+  const uint64_t da = tc::smem_desc_sw128(a_slot, lbo, 1024), db = tc::smem_desc_sw128(b_tile, b_stride, 1024);
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const uint64_t oa = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 2048) >> 4);
+    const uint64_t ob = (uint64_t)((ks * 2048) >> 4);
+    tc::mma_ss(tm_acc, da + oa, db + ob, idesc, accumulate_first || (ks > 0));
+  }
+}
+
+// x -> (bf16(x), bf16(x - bf16(x))) for two values, packed like pack_bf16x2
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16x2(x0, x1);
+  const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xffff0000u);
+  lo = pack_bf16x2(x0 - h0, x1 - h1);
+}
+
 // Which cubes are cut by the grid boundary: bit 0 / 1 / 2 = last cube along t / h / w with a partial extent.
 // In the half-cube grid of a 128-token-cube problem the last column of blocks along w may lie outside the grid
 // altogether (extent <= 0, still bit 2); the column before it can then be the partial one (bit 3).

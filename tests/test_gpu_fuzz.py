@@ -48,3 +48,33 @@ def test_random_geometry_full_parity(case):
 @pytest.mark.parametrize("case", range(16))
 def test_random_geometry_cubes_of_128_tokens(case):
     run_case(*random_workload(case, wide=True))
+
+
+@pytest.mark.parametrize("case,wide", [(186, False), (102, True), (187, True), (189, True)])
+def test_geometries_with_sharply_peaked_rows(case, wide):
+    """Four geometries of a wider sweep (cases 100-219) whose rows keep one to seven blocks: the softmax is sharply peaked,
+    gradients reach |g| = 5..30, and with P and dS rounded once to bf16 the worst element of dV or dQ missed 2e-2
+    (2.2e-2 .. 2.8e-2).  They pass since the backward carries P and dS as a bf16 pair (high part + rounding residual)."""
+    run_case(*random_workload(case, wide))
+
+
+def test_fast_backward_flag_stays_close():
+    """VSA2_FLAG_FAST_BWD (P and dS rounded once to bf16): same results within the looser figure its documentation states."""
+    from oracle import vsa2_oracle as orc
+    from vsa2_testlib import CudaPath, oracle_arrays
+    wl, _ = random_workload(3)
+    data = syn.make_inputs(wl)
+    nnz_cap = int(np.minimum(data["budgets"], wl.n_cubes).sum(axis=-1).max()) if wl.select_mode == syn.PER_QUERY_BUDGET else 0
+    outs = []
+    for flags in (0, vb.FLAG_FAST_BWD):
+        run = CudaPath(wl, data, out_dtype=vb.F32, flags=flags, nnz_cap=nnz_cap)
+        run.route()
+        run.forward()
+        outs.append(run.backward())
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    a = oracle_arrays(data)
+    want = orc.backward(a["q"], a["k"], a["v"], a["gate"], run.mask, geo, 1.0 / np.sqrt(wl.head_dim), a["do"])
+    for name, precise, fast, ref in zip(("dQ", "dK", "dV"), outs[0], outs[1], want):
+        e_p, e_f = np.abs(precise - ref).max(), np.abs(fast - ref).max()
+        assert e_p <= 2e-2 and e_f <= 4e-2, (name, e_p, e_f)
+        assert e_p <= e_f + 1e-6, (name, e_p, e_f)           # the split never makes things worse
