@@ -36,7 +36,9 @@ tests pin is that each function computes exactly the reading stated here:
 * gate projection: X [L, C] are the layer's hidden states (C = model width) and
   W_g has one column per query head, W_g [C, H_q], so that G [H_q, L] holds the
   per-token per-head gate of Eq. 13 (the paper writes one head: W_g in R^{D x 1}).
-* text tokens (Sec. 2.2, the sentence after Eq. 12): see `joint_*` below.
+* text tokens (Sec. 2.2, the sentence after Eq. 12): one softmax per row over the kept video blocks plus all text
+  keys (video queries) or over everything (text queries); see `joint_*` below.  Pinned by SDPA over the
+  concatenated sequence, by the log-sum-exp merge identity and by autograd.
 Every function here is pinned by tests/test_oracle_pins.py.
 """
 from __future__ import annotations
@@ -297,6 +299,122 @@ def fine_attention(Q, K, V, mask, geo: Geometry, scale, rows=None):
         O_f[qt] = (e / l) @ V[kt]
         lse[qt] = (m + np.log(l))[:, 0]
     return O_f, lse
+
+
+# ----------------------------------------------------------------------------
+# Sec. 2.2 "Fine Branch", the sentence after Eq. 12: text tokens (MMDiT)
+# ----------------------------------------------------------------------------
+# Video and text tokens share one attention space.  Reading taken (the paper gives one sentence): the block map M
+# covers video-video pairs only; every video query additionally attends ALL text keys, and every text query attends
+# all video keys and all text keys, each row with ONE softmax over its whole key set.  Text tokens take no part in
+# the coarse branch, the router or the gate: a text query's output is its fine-branch output.
+def joint_fine_attention(Q, K, V, Qt, Kt, Vt, mask, geo: Geometry, scale, rows=None, text_rows=None):
+    """Video Q, K, V [L, D], text Qt, Kt, Vt [Lt, D], mask [N, N] -> (O_f [L, D], lse [L], O_t [Lt, D], lse_t [Lt]).
+
+    Video queries of cube i: softmax over the valid tokens of the kept cubes of row i followed by all text tokens.
+    Text queries: softmax over all video tokens followed by all text tokens.  `rows` / `text_rows` restrict the work to
+    some video query cubes / text query tokens (the others stay 0 / -inf).
+    """
+    L, D = Q.shape
+    Lt = Qt.shape[0]
+    O_f = np.zeros((L, D), dtype=np.float64)
+    lse = np.full(L, -np.inf, dtype=np.float64)
+    for i in (range(geo.N) if rows is None else rows):
+        cols = np.nonzero(mask[i])[0]
+        qt = geo.cube_tokens[i]
+        kt = np.concatenate([geo.cube_tokens[j] for j in cols] + [np.zeros(0, np.int64)]).astype(np.int64)
+        Kk = np.concatenate([K[kt], Kt])
+        Vv = np.concatenate([V[kt], Vt])
+        if Kk.shape[0] == 0:
+            continue
+        s = (Q[qt] @ Kk.T) * scale
+        m = s.max(axis=1, keepdims=True)
+        e = np.exp(s - m)
+        l = e.sum(axis=1, keepdims=True)
+        O_f[qt] = (e / l) @ Vv
+        lse[qt] = (m + np.log(l))[:, 0]
+    O_t = np.zeros((Lt, D), dtype=np.float64)
+    lse_t = np.full(Lt, -np.inf, dtype=np.float64)
+    tr = np.arange(Lt) if text_rows is None else np.asarray(text_rows, dtype=np.int64)
+    if tr.size:
+        Kk = np.concatenate([K, Kt])
+        Vv = np.concatenate([V, Vt])
+        s = (Qt[tr] @ Kk.T) * scale
+        m = s.max(axis=1, keepdims=True)
+        e = np.exp(s - m)
+        l = e.sum(axis=1, keepdims=True)
+        O_t[tr] = (e / l) @ Vv
+        lse_t[tr] = (m + np.log(l))[:, 0]
+    return O_f, lse, O_t, lse_t
+
+
+def joint_fine_backward(Q, K, V, Qt, Kt, Vt, mask, geo: Geometry, scale, dO, dOt, lse, O_f, lse_t, O_t,
+                        rows=None, text_rows=None):
+    """Backward of joint_fine_attention for the video query cubes in `rows` and the text queries in `text_rows` (all if
+    None).  Same formulas as fine_backward, over each row's whole key set.  Returns dQ, dK, dV [L, D] and dQt, dKt, dVt
+    [Lt, D] (the key / value gradients hold only the contributions of the visited queries)."""
+    dQ, dK, dV = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)
+    dQt, dKt, dVt = np.zeros_like(Qt), np.zeros_like(Kt), np.zeros_like(Vt)
+    delta = (dO * O_f).sum(axis=1)
+    for i in (range(geo.N) if rows is None else rows):
+        cols = np.nonzero(mask[i])[0]
+        qt = geo.cube_tokens[i]
+        kt = np.concatenate([geo.cube_tokens[j] for j in cols] + [np.zeros(0, np.int64)]).astype(np.int64)
+        nv = kt.size
+        Kk = np.concatenate([K[kt], Kt])
+        Vv = np.concatenate([V[kt], Vt])
+        if Kk.shape[0] == 0:
+            continue
+        s = (Q[qt] @ Kk.T) * scale
+        P = np.exp(s - lse[qt][:, None])
+        dVv = P.T @ dO[qt]
+        dP = dO[qt] @ Vv.T
+        dS = P * (dP - delta[qt][:, None])
+        dQ[qt] += (dS @ Kk) * scale
+        dKk = (dS.T @ Q[qt]) * scale
+        dK[kt] += dKk[:nv]
+        dV[kt] += dVv[:nv]
+        dKt += dKk[nv:]
+        dVt += dVv[nv:]
+    tr = np.arange(Qt.shape[0]) if text_rows is None else np.asarray(text_rows, dtype=np.int64)
+    if tr.size:
+        L = K.shape[0]
+        Kk = np.concatenate([K, Kt])
+        Vv = np.concatenate([V, Vt])
+        delta_t = (dOt[tr] * O_t[tr]).sum(axis=1)
+        s = (Qt[tr] @ Kk.T) * scale
+        P = np.exp(s - lse_t[tr][:, None])
+        dVv = P.T @ dOt[tr]
+        dP = dOt[tr] @ Vv.T
+        dS = P * (dP - delta_t[:, None])
+        dQt[tr] += (dS @ Kk) * scale
+        dKk = (dS.T @ Qt[tr]) * scale
+        dK += dKk[:L]
+        dV += dVv[:L]
+        dKt += dKk[L:]
+        dVt += dVv[L:]
+    return dQ, dK, dV, dQt, dKt, dVt
+
+
+def joint_head_forward(Q, K, V, Qt, Kt, Vt, gate, mask, geo: Geometry, scale):
+    """The whole operator with text tokens for one head: coarse branch and merge on the video tokens as in head_forward
+    (Eq. 1-4, 14), fine branch by joint_fine_attention.  Returns the dict of head_forward plus O_t, lse_t."""
+    Qc, Kc, Vc = mean_pool_cube(Q, geo), mean_pool_cube(K, geo), mean_pool_cube(V, geo)
+    Oc_hat, lse_c = coarse_attention(Qc, Kc, Vc, scale)
+    O_f, lse, O_t, lse_t = joint_fine_attention(Q, K, V, Qt, Kt, Vt, mask, geo, scale)
+    O = gate[:, None] * Oc_hat[geo.cube_of] + O_f
+    return dict(O=O, O_f=O_f, lse=lse, O_t=O_t, lse_t=lse_t, Oc_hat=Oc_hat, lse_c=lse_c, Qc=Qc, Kc=Kc, Vc=Vc)
+
+
+def joint_head_backward(Q, K, V, Qt, Kt, Vt, gate, mask, geo: Geometry, scale, dO, dOt, fwd=None):
+    """Gradients of sum(O * dO) + sum(O_t * dOt) for one head given the block mask: coarse path as in head_backward,
+    fine path by joint_fine_backward.  Returns dQ, dK, dV, dGate (video) and dQt, dKt, dVt (text)."""
+    if fwd is None:
+        fwd = joint_head_forward(Q, K, V, Qt, Kt, Vt, gate, mask, geo, scale)
+    c = coarse_path_backward(Q, K, V, gate, geo, scale, dO, fwd)
+    fq, fk, fv, tq, tk, tv = joint_fine_backward(Q, K, V, Qt, Kt, Vt, mask, geo, scale, dO, dOt, fwd["lse"], fwd["O_f"],
+                                                 fwd["lse_t"], fwd["O_t"])
+    return dict(dQ=c["dQ"] + fq, dK=c["dK"] + fk, dV=c["dV"] + fv, dGate=c["dGate"], dQt=tq, dKt=tk, dVt=tv)
 
 
 # ----------------------------------------------------------------------------

@@ -419,6 +419,9 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
       // 128 query columns per tile: the halves of a 128-token cube, or two heads of a group that share their map
       VSA2_CUDA(launch_fine_fwd_wide_tc(n, !wide, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                         reinterpret_cast<StatusBlock*>(workspace), st));
+    else if (fine_fwd_rows_supported(n) && !(g.flags & 512))
+      VSA2_CUDA(launch_fine_fwd_rows_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
+                                        reinterpret_cast<StatusBlock*>(workspace), st));
     else
       VSA2_CUDA(launch_fine_fwd_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                    reinterpret_cast<StatusBlock*>(workspace), st));

@@ -187,6 +187,12 @@ cudaError_t launch_fine_fwd_tc(const Geo& g, const bf16* q, const bf16* k, const
                                const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                float* lse, StatusBlock* status, cudaStream_t st);
 
+// tensor-core forward with the queries in the accumulator rows (fine_fwd_rows_tc.cu); same workspace as launch_fine_fwd_tc
+bool fine_fwd_rows_supported(const Geo& g);
+cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                                    const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                                    float* lse, StatusBlock* status, cudaStream_t st);
+
 // tensor-core forward with 128 query columns (fine_fwd_wide_tc.cu): two query blocks that keep the same key blocks on the
 // same operand tiles -- the two halves of a 128-token query cube (`g`, the map and oc_hat are those of the half-cube problem)
 // or, with pair_heads, one query block of two query heads that share their map; the workspace is the one of launch_fine_fwd_tc

@@ -1,0 +1,577 @@
+// Fine branch forward (paper Eq. 12) + gated merge (Eq. 14) on the Blackwell tensor cores, queries in the lanes.
+//
+// Formulation.  A query block has B = 64 tokens.  Both products keep the 64 queries in the rows of the accumulator (M = 64)
+// and stack two selected KV blocks per tile:
+//     S [64 q, 128 kv] = Q [64, D] * K_pair^T            (A = Q from shared memory,  B = K_pair, N = 128 keys)
+//     O [64 q, D]     += P [64, 128 kv] * V_pair         (A = P from TENSOR MEMORY,  B = V_pair, N = D)
+// M = 64 runs the tensor pipe at half rate, but every K / V tile is fetched from shared memory exactly once per tile and P
+// never touches shared memory: per tile 64 KB of TMA writes + 64 KB of B fetches + 16 KB of Q, against 176 KB for the
+// transposed M = 128, N = 64 products, which were bound by that traffic.  K and V tiles arrive by 5-D TMA straight from the
+// raster tensors (one box = one cube, zero-filled outside the grid); the V tile that TMA wrote row-per-key is read as an
+// MN-major B operand, so nothing is transposed in memory.
+//
+// Tensor memory (512 columns): two S buffers (2 x 128 fp32 columns), two P buffers (2 x 64 columns of bf16 pairs) and the O
+// accumulator (D columns).  An M = 64 accumulator keeps row m in lane (m % 16) + 32 (m / 16); the softmax warps read S with
+// 16-lane loads that give a thread two query rows x 32 key columns, and the bf16 pairs it forms from neighbouring columns
+// are exactly the words its 16-lane store writes into the P operand.
+//
+// Softmax.  Four threads share a query row.  Each row keeps a fixed reference M (the exact row maximum of the block's first
+// tile, log2 units): P = 2^(s*scale*log2e - M); any reference gives the same softmax unless something overflows, the row
+// sums are checked at the end of the query block and a block outside the safe range is redone by the exact-maximum kernel
+// (fine_fwd.cu).  Two sums are kept per row: the fp32 sum of the exponentials, which gives the log-sum-exp, and the sum of
+// their bf16 roundings, which is what the P V product really adds up -- the output is normalised by the latter, so the
+// weights sum to one and the rounding of a dominant P cancels instead of scaling the whole output row (that scaling,
+// 2^-9 relative, reached the backward through delta = rowsum(dO * O) and was its largest error on sharply peaked rows).
+//
+// Roles (512 threads): warps 0..3 = TMA producers (K / V ring x first / second block of a pair; warp 0 also brings the Q
+// tile and schedules the CTA's work items), warp 4 = issuer of S, warp 5 = issuer of O, warps 8..15 = two softmax +
+// epilogue warpgroups that alternate tiles.  Persistent CTAs draw query blocks from a global counter.  Every wait is bounded.
+#include "tc_attn.cuh"
+
+namespace vsa2 {
+
+constexpr int kFrThreads = 512;
+constexpr int kFrKSlots = 3;
+constexpr int kFrVSlots = 2;
+constexpr int kFrMaxCubes = 8192;      // edge-flag table in shared memory: one byte per cube
+
+template <int D>
+struct FwdRows {
+  static constexpr int DH = D / 64;
+  static constexpr uint32_t SLOT = 2 * DH * kSlab;     // a K pair or a V pair, [half][A | B]
+  static constexpr uint32_t QBYTES = DH * kSlab;
+  static constexpr uint32_t PITCH = D * 2 + 16;        // bytes per staged output row (odd multiple of 16: no bank conflicts)
+  static constexpr uint32_t STAGE = 64 * PITCH;
+  static constexpr uint32_t OFF_Q = (kFrKSlots + kFrVSlots) * SLOT;
+  static constexpr uint32_t OFF_STAGE = OFF_Q + QBYTES;
+  static constexpr uint32_t OFF_MISC = OFF_STAGE + 2 * STAGE;
+  static constexpr uint32_t MISC_BYTES = 4096;
+  static constexpr uint32_t TM_S = 0, TM_P = 256, TM_O = 384;
+  static size_t smem_bytes(int n_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_cubes + 15) / 16 * 16 + 1024; }
+};
+
+struct FwdRowsMisc {
+  uint64_t q_full, q_empty, o_full, o_empty;
+  uint64_t k_full[kFrKSlots], k_empty[kFrKSlots];
+  uint64_t v_full[kFrVSlots], v_empty[kFrVSlots];
+  uint64_t s_full[2], s_free[2];
+  uint64_t p_ready[2], p_free[2];
+  ItemQueue items;
+  uint64_t all_sync;               // group barrier of the 256 softmax threads
+  uint32_t tmem_base;
+  int abort_flag;
+  int rescue_flag;
+  unsigned short vmask[16][4];     // [edge flags][lane % 4]: which of a thread's 16 key columns of a block are valid tokens
+  alignas(16) float m_ref[64];     // per query row: reference exponent (log2 units)
+  float red[2][2][64];             // [warpgroup][exact sum | sum of the bf16 roundings][query row]
+  alignas(16) float oc[128];       // coarse output row of the query cube
+  int tok[2][64];                  // raster token of each query row (-1 = padding), by item parity
+  float gate[2][64];
+};
+static_assert(sizeof(FwdRowsMisc) <= 4096, "misc region too small");
+
+struct FwdRowsArgs {
+  int* item_counter;    // global, zero before the launch
+  const float* gate;
+  const int* row_ptr;
+  const int* col_idx;
+  const float* oc_hat;
+  void* o;
+  bf16* o_res;
+  float* lse;
+  StatusBlock* status;
+  int* rescue_count;
+  int* rescue_items;
+  int rescue_cap;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kFrThreads, 1)
+fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, Geo g, FwdRowsArgs a) {
+  using C = FwdRows<D>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* q_tile = smem + C::OFF_Q;
+  unsigned char* stage = smem + C::OFF_STAGE;
+  FwdRowsMisc* misc = reinterpret_cast<FwdRowsMisc*>(smem + C::OFF_MISC);
+  unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;      // edge flags of every cube
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int total_items = g.batch * g.Hq * g.N;
+  const float c2 = g.scale * 1.4426950408889634f;
+
+  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
+  if (tid < 64) {
+    // validity of key columns 8n + 2c + e (n = 0..7, e = 0, 1) of a 64-token block with edge flags f, for lane % 4 == c
+    const unsigned f = tid >> 2, c = tid & 3;
+    unsigned m = 0;
+    for (int n = 0; n < 8; ++n)
+      for (int e = 0; e < 2; ++e) {
+        CubePos cp;
+        cp.init(g, 8 * n + 2 * (int)c + e);
+        if (cp.valid(f, g)) m |= 1u << (2 * n + e);
+      }
+    misc->vmask[f][c] = (unsigned short)m;
+  }
+  if (tid == 0) {
+    misc->abort_flag = 0;
+    tc::mbar_init(&misc->q_full, 1);
+    tc::mbar_init(&misc->q_empty, 1);
+    tc::mbar_init(&misc->o_full, 1);
+    tc::mbar_init(&misc->o_empty, 256);
+    for (int s = 0; s < kFrKSlots; ++s) {
+      tc::mbar_init(&misc->k_full[s], 2);    // the two producer warps of the ring
+      tc::mbar_init(&misc->k_empty[s], 1);
+    }
+    for (int s = 0; s < kFrVSlots; ++s) {
+      tc::mbar_init(&misc->v_full[s], 2);
+      tc::mbar_init(&misc->v_empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(&misc->s_full[s], 1);
+      tc::mbar_init(&misc->s_free[s], 128);
+      tc::mbar_init(&misc->p_ready[s], 128);
+      tc::mbar_init(&misc->p_free[s], 1);
+    }
+    tc::mbar_init(&misc->all_sync, 256);
+    item_queue_init(&misc->items, 4 + 2 + 256);     // lane 0 of the producers, two issuers, the softmax threads
+    tc::fence_barrier_init();
+    tc::prefetch_tmap(&tm_q);
+    tc::prefetch_tmap(&tm_k);
+    tc::prefetch_tmap(&tm_v);
+  }
+  if (warp == 4) {
+    tc::tmem_alloc(&misc->tmem_base, 512);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = misc->tmem_base;
+
+  if (warp < 8) {
+    tc::reg_dec<56>();
+    if (warp < 4) {
+      // ---------------------------------------------------------------- TMA producers
+      // One warp sustains only ~24 B/clk of 5-D boxes (the copy instructions of a warp issue one after the other), so every
+      // ring has two producer warps, one per block of a pair; both arrive on the slot's full barrier with half the bytes.
+      const int which = warp & 1;                           // 0: K ring (+ Q tile), 1: V ring
+      const int my_blk = warp >> 1;                         // 0: first block of the pair, 1: second
+      const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+      const uint32_t nslots = which == 0 ? kFrKSlots : kFrVSlots;
+      uint64_t* full = which == 0 ? misc->k_full : misc->v_full;
+      uint64_t* empty = which == 0 ? misc->k_empty : misc->v_empty;
+      unsigned char* ring = smem + (which == 0 ? 0 : kFrKSlots * C::SLOT);
+      const int my_h = lane;
+      const bool issuer = lane < C::DH;
+      uint32_t tg = 0, n_items = 0, published = 0;
+      for (uint32_t seq = 0;; ++seq) {
+        // warp 0, lane 0 is the CTA's scheduler
+        int item = 0;
+        if (lane == 0) {
+          if (warp == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
+          else item = item_get(&misc->items, seq, &misc->abort_flag);
+        }
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item == -2) goto done;
+        if (item < 0) break;
+        const int i = item % g.N, bhq = item / g.N;
+        const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
+        const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
+        const int k = end - beg;
+        if (k == 0) continue;
+        const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+        if (warp == 0) {
+          int it_, ih_, iw_;
+          cube_coords(g, i, it_, ih_, iw_);
+          int ok = 1;
+          if (lane == 0) {
+            ok = tc::mbar_wait(&misc->q_empty, (n_items & 1) ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&misc->q_full, C::QBYTES);
+          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+          if (lane < C::DH)
+            tc::tma_load_5d(q_tile + lane * kSlab, &tm_q, &misc->q_full, lane * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+        }
+        ++n_items;
+        const int nt = (k + 1) >> 1;
+        int j = cols[(my_blk == 1 && k > 1) ? 1 : 0];           // this warp's KV block of tile 0
+        for (int t = 0; t < nt; ++t, ++tg) {
+          int jt, jh, jw;
+          cube_coords(g, j, jt, jh, jw);
+          if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];   // next tile, fetched early
+          const uint32_t slot = tg % nslots, par = (tg / nslots) & 1;
+          int ok = 1;
+          if (lane == 0) {
+            ok = tc::mbar_wait(&empty[slot], par ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&full[slot], C::SLOT / 2);
+          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
+          if (issuer)
+            tc::tma_load_5d(ring + slot * C::SLOT + (2 * my_h + my_blk) * kSlab, tm, &full[slot], my_h * 64,
+                            jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
+        }
+      }
+    } else if (warp == 4) {
+      // ---------------------------------------------------------------- issuer of S(t) = Q * K_pair^T
+      if (lane == 0) {
+        constexpr uint32_t idesc = tc::idesc_bf16(64, 128, false, false);
+        const uint64_t dq = tc::smem_desc_sw128(tc::smem_u32(q_tile), 16, 1024);
+        const uint32_t slot0 = tc::smem_u32(smem);
+        uint32_t tg = 0, n_items = 0;
+        for (uint32_t seq = 0;; ++seq) {
+          VSA2_NEXT_ITEM(item, seq);
+          const int i = item % g.N, bhq = item / g.N;
+          const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+          if (k == 0) continue;
+          const int nt = (k + 1) >> 1;
+          VSA2_WAIT(&misc->q_full, n_items & 1);
+          for (int t = 0; t < nt; ++t, ++tg) {
+            const uint32_t slot = tg % kFrKSlots, buf = tg & 1;
+            VSA2_WAIT(&misc->k_full[slot], (tg / kFrKSlots) & 1);
+            VSA2_WAIT(&misc->s_free[buf], ((tg >> 1) & 1) ^ 1);
+            tc::tc_fence_after();
+            const uint64_t dk = tc::smem_desc_sw128(slot0 + slot * C::SLOT, 16, 1024);
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+              const uint64_t oa = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 32) >> 4);
+              const uint64_t ob = (uint64_t)(((ks / 4) * 2 * kSlab + (ks % 4) * 32) >> 4);
+              tc::mma_ss(tmem_base + C::TM_S + buf * 128, dq + oa, dk + ob, idesc, ks > 0);
+            }
+            tc::mma_commit(&misc->s_full[buf]);
+            tc::mma_commit(&misc->k_empty[slot]);
+          }
+          tc::mma_commit(&misc->q_empty);          // the Q tile may be replaced once the last S of the block is done
+          ++n_items;
+        }
+      }
+    } else if (warp == 5) {
+      // ---------------------------------------------------------------- issuer of O += P(t) * V_pair
+      if (lane == 0) {
+        constexpr uint32_t idesc = tc::idesc_bf16(64, D, false, true);
+        constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;       // distance between the two 64-channel halves of V
+        const uint32_t slot0 = tc::smem_u32(smem) + kFrKSlots * C::SLOT;
+        uint32_t tg = 0, n_items = 0;
+        for (uint32_t seq = 0;; ++seq) {
+          VSA2_NEXT_ITEM(item, seq);
+          const int i = item % g.N, bhq = item / g.N;
+          const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+          if (k == 0) continue;
+          const int nt = (k + 1) >> 1;
+          VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous query block's accumulator was read out
+          for (int t = 0; t < nt; ++t, ++tg) {
+            const uint32_t slot = tg % kFrVSlots, buf = tg & 1;
+            VSA2_WAIT(&misc->v_full[slot], (tg / kFrVSlots) & 1);
+            VSA2_WAIT(&misc->p_ready[buf], (tg >> 1) & 1);
+            tc::tc_fence_after();
+            const uint64_t dv = tc::smem_desc_sw128(slot0 + slot * C::SLOT, lbo, 1024);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint64_t ob = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 2048) >> 4);
+              tc::mma_ts(tmem_base + C::TM_O, tmem_base + C::TM_P + buf * 64 + ks * 8, dv + ob, idesc, t > 0 || ks > 0);
+            }
+            tc::mma_commit(&misc->v_empty[slot]);
+            tc::mma_commit(&misc->p_free[buf]);
+          }
+          tc::mma_commit(&misc->o_full);
+          ++n_items;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
+    tc::reg_inc<200>();
+    const int wg = (warp >> 2) - 2;              // 0 or 1: the tiles with (global tile index & 1) == wg
+    const int quad = warp & 3;
+    const int cq = lane & 3;
+    const int row_a = quad * 16 + (lane >> 2), row_b = row_a + 8;     // the two query rows of this thread
+    const int sm_tid = tid & 127;
+    const int t256 = tid - 256;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
+    constexpr int COLS = D / 2;                  // output columns per warpgroup in the epilogue
+    uint32_t tg = 0, n_items = 0, all_phase = 0;
+    for (uint32_t n_all = 0;; ++n_all) {
+      VSA2_NEXT_ITEM(item, n_all);
+      const int i = item % g.N, bhq = item / g.N;
+      const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
+      const int k = end - beg;
+      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
+      const int tb = n_all & 1;
+      if (wg == 0 && sm_tid < 64) {
+        int it_, ih_, iw_;
+        cube_coords(g, i, it_, ih_, iw_);
+        const int l = cube_token(g, it_, ih_, iw_, sm_tid);
+        misc->tok[tb][sm_tid] = l;
+        misc->gate[tb][sm_tid] = (coarse && l >= 0) ? a.gate[(size_t)bhq * g.L + l] : 0.f;
+      }
+      if (wg == 1 && sm_tid < D) misc->oc[sm_tid] = coarse ? a.oc_hat[((size_t)bhq * g.N + i) * D + sm_tid] : 0.f;
+      if (wg == 0 && sm_tid == 0) misc->rescue_flag = 0;
+
+      const int nt = (k + 1) >> 1;
+      const uint32_t tg0 = tg;
+      uint32_t sv[64];
+      bool have_first = false;
+      if (k > 0 && (tg & 1) == (uint32_t)wg) {
+        // this warpgroup owns tile 0: reference exponent of every query row = exact row maximum of that tile
+        const uint32_t buf = tg & 1;
+        VSA2_WAIT(&misc->s_full[buf], (tg >> 1) & 1);
+        tc::tc_fence_after();
+        tc::tmem_ld_16x256b_x16(lane_addr + C::TM_S + buf * 128, sv);
+        tc::tmem_ld_wait();
+        tc::tc_fence_before();
+        tc::mbar_arrive(&misc->s_free[buf]);
+        have_first = true;
+        const unsigned ma = misc->vmask[edge[cols[0]]][cq];
+        const unsigned mb = k > 1 ? misc->vmask[edge[cols[1]]][cq] : 0u;
+        float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+          const unsigned m = (n < 8 ? ma : mb) >> (2 * (n & 7));
+          if (m & 1u) { mx_a = fmaxf(mx_a, __uint_as_float(sv[4 * n])); mx_b = fmaxf(mx_b, __uint_as_float(sv[4 * n + 2])); }
+          if (m & 2u) { mx_a = fmaxf(mx_a, __uint_as_float(sv[4 * n + 1])); mx_b = fmaxf(mx_b, __uint_as_float(sv[4 * n + 3])); }
+        }
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+        if (cq == 0) {
+          misc->m_ref[row_a] = (mx_a > -INFINITY) ? mx_a * c2 : 0.f;
+          misc->m_ref[row_b] = (mx_b > -INFINITY) ? mx_b * c2 : 0.f;
+        }
+      }
+      VSA2_GROUP_SYNC(&misc->all_sync, all_phase);       // tables and reference exponents visible to both warpgroups
+
+      float l_a = 0.f, l_b = 0.f, r_a = 0.f, r_b = 0.f;   // exact sums and sums of the bf16 roundings of the two rows
+      float m_a = 0.f, m_b = 0.f;
+      if (k > 0) {
+        m_a = misc->m_ref[row_a];
+        m_b = misc->m_ref[row_b];
+        for (int t = ((tg0 & 1) == (uint32_t)wg) ? 0 : 1; t < nt; t += 2) {
+          const uint32_t tgt = tg0 + t, buf = tgt & 1;
+          const bool dup = 2 * t + 1 >= k;
+          const unsigned ma = misc->vmask[edge[cols[2 * t]]][cq];
+          const unsigned mb = dup ? 0u : misc->vmask[edge[cols[2 * t + 1]]][cq];
+          if (!(have_first && t == 0)) {
+            VSA2_WAIT(&misc->s_full[buf], (tgt >> 1) & 1);
+            tc::tc_fence_after();
+            tc::tmem_ld_16x256b_x16(lane_addr + C::TM_S + buf * 128, sv);
+            tc::tmem_ld_wait();
+            tc::tc_fence_before();
+            tc::mbar_arrive(&misc->s_free[buf]);
+          }
+          uint32_t pk[32];
+          if ((ma & mb) == 0xffffu) {
+#pragma unroll
+            for (int n = 0; n < 16; ++n) {
+              const float p0 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 0]), c2, -m_a));
+              const float p1 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 1]), c2, -m_a));
+              const float p2 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 2]), c2, -m_b));
+              const float p3 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 3]), c2, -m_b));
+              l_a += p0 + p1;
+              l_b += p2 + p3;
+              const uint32_t wa = pack_bf16x2(p0, p1), wb = pack_bf16x2(p2, p3);
+              r_a += __uint_as_float(wa << 16) + __uint_as_float(wa & 0xffff0000u);
+              r_b += __uint_as_float(wb << 16) + __uint_as_float(wb & 0xffff0000u);
+              pk[2 * n] = wa;
+              pk[2 * n + 1] = wb;
+            }
+          } else {
+#pragma unroll
+            for (int n = 0; n < 16; ++n) {
+              const unsigned m = (n < 8 ? ma : mb) >> (2 * (n & 7));
+              float p0 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 0]), c2, -m_a));
+              float p1 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 1]), c2, -m_a));
+              float p2 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 2]), c2, -m_b));
+              float p3 = ex2_approx(fmaf(__uint_as_float(sv[4 * n + 3]), c2, -m_b));
+              if (!(m & 1u)) { p0 = 0.f; p2 = 0.f; }
+              if (!(m & 2u)) { p1 = 0.f; p3 = 0.f; }
+              l_a += p0 + p1;
+              l_b += p2 + p3;
+              const uint32_t wa = pack_bf16x2(p0, p1), wb = pack_bf16x2(p2, p3);
+              r_a += __uint_as_float(wa << 16) + __uint_as_float(wa & 0xffff0000u);
+              r_b += __uint_as_float(wb << 16) + __uint_as_float(wb & 0xffff0000u);
+              pk[2 * n] = wa;
+              pk[2 * n + 1] = wb;
+            }
+          }
+          VSA2_WAIT(&misc->p_free[buf], ((tgt >> 1) & 1) ^ 1);
+          tc::tmem_st_16x128b_x16(lane_addr + C::TM_P + buf * 64, pk);
+          tc::tmem_st_wait();
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->p_ready[buf]);
+        }
+        tg += nt;
+        // row sums: over the four threads of a row here, over the two warpgroups through shared memory
+        l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
+        l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
+        r_a += __shfl_xor_sync(0xffffffffu, r_a, 1);
+        r_b += __shfl_xor_sync(0xffffffffu, r_b, 1);
+        l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+        l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
+        r_a += __shfl_xor_sync(0xffffffffu, r_a, 2);
+        r_b += __shfl_xor_sync(0xffffffffu, r_b, 2);
+        if (cq == 0) {
+          misc->red[wg][0][row_a] = l_a;
+          misc->red[wg][0][row_b] = l_b;
+          misc->red[wg][1][row_a] = r_a;
+          misc->red[wg][1][row_b] = r_b;
+        }
+      }
+      VSA2_GROUP_SYNC(&misc->all_sync, all_phase);
+      float inv_a = 0.f, inv_b = 0.f;
+      if (k > 0) {
+        const float la = misc->red[0][0][row_a] + misc->red[1][0][row_a], lb = misc->red[0][0][row_b] + misc->red[1][0][row_b];
+        const float ra = misc->red[0][1][row_a] + misc->red[1][1][row_a], rb = misc->red[0][1][row_b] + misc->red[1][1][row_b];
+        inv_a = 1.f / ra;
+        inv_b = 1.f / rb;
+        if (wg == 0 && cq == 0) {
+          // sums outside the safe range (overflow, NaN or total underflow): hand the block to the exact kernel
+          if (!(la > 1e-30f && la < 1e30f && ra > 1e-30f) || !(lb > 1e-30f && lb < 1e30f && rb > 1e-30f)) misc->rescue_flag = 1;
+          const int ta = misc->tok[tb][row_a], tk_b = misc->tok[tb][row_b];
+          if (ta >= 0) a.lse[(size_t)bhq * g.L + ta] = (m_a + __log2f(la)) * 0.6931471805599453f;
+          if (tk_b >= 0) a.lse[(size_t)bhq * g.L + tk_b] = (m_b + __log2f(lb)) * 0.6931471805599453f;
+        }
+        VSA2_WAIT(&misc->o_full, n_items & 1);
+        tc::tc_fence_after();
+      } else if (wg == 0 && cq == 0) {
+        const int ta = misc->tok[tb][row_a], tk_b = misc->tok[tb][row_b];
+        if (ta >= 0) a.lse[(size_t)bhq * g.L + ta] = -INFINITY;
+        if (tk_b >= 0) a.lse[(size_t)bhq * g.L + tk_b] = -INFINITY;
+      }
+
+      // O[l, d] = O_acc[q, d] / (rounded row sum) + gate[q] * O_c[d]; this warpgroup owns COLS output columns
+      {
+        constexpr int NR = COLS / 2;              // registers per thread: 2 rows x COLS / 4 columns
+        uint32_t acc[NR];
+        if (k > 0) {
+          if constexpr (D == 128) tc::tmem_ld_16x256b_x8(lane_addr + C::TM_O + wg * COLS, acc);
+          else tc::tmem_ld_16x256b_x4(lane_addr + C::TM_O + wg * COLS, acc);
+          tc::tmem_ld_wait();
+          tc::tc_fence_before();
+          tc::mbar_arrive(&misc->o_empty);
+        } else {
+#pragma unroll
+          for (int c = 0; c < NR; ++c) acc[c] = 0u;
+        }
+        const float ga = misc->gate[tb][row_a], gb = misc->gate[tb][row_b];
+        const int ta = misc->tok[tb][row_a], tk_b = misc->tok[tb][row_b];
+        if (g.out_f32) {
+#pragma unroll
+          for (int n = 0; n < COLS / 8; ++n) {
+            const int col = wg * COLS + 8 * n + 2 * cq;
+            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[col]);
+            if (ta >= 0)
+              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.L + ta) * D + col) =
+                  make_float2(fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a));
+            if (tk_b >= 0)
+              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.L + tk_b) * D + col) =
+                  make_float2(fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b));
+          }
+        } else {
+          // bf16 output and rounding residual: through shared memory, then 16-byte stores
+          unsigned char* st_o = stage;
+          unsigned char* st_r = stage + C::STAGE;
+#pragma unroll
+          for (int n = 0; n < COLS / 8; ++n) {
+            const int col = wg * COLS + 8 * n + 2 * cq;
+            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[col]);
+            const float v0 = fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), v1 = fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a);
+            const float v2 = fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), v3 = fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b);
+            uint32_t ha, la2, hb, lb2;
+            split_bf16x2(v0, v1, ha, la2);
+            split_bf16x2(v2, v3, hb, lb2);
+            *reinterpret_cast<uint32_t*>(st_o + row_a * C::PITCH + col * 2) = ha;
+            *reinterpret_cast<uint32_t*>(st_o + row_b * C::PITCH + col * 2) = hb;
+            *reinterpret_cast<uint32_t*>(st_r + row_a * C::PITCH + col * 2) = la2;
+            *reinterpret_cast<uint32_t*>(st_r + row_b * C::PITCH + col * 2) = lb2;
+          }
+          VSA2_GROUP_SYNC(&misc->all_sync, all_phase);
+          constexpr int CH = D / 8;                                      // 16-byte chunks per token row
+          for (int e = t256; e < 64 * CH; e += 256) {
+            const int qi = e / CH, ch = e % CH;
+            const int l = misc->tok[tb][qi];
+            if (l < 0) continue;
+            const size_t idx = ((size_t)bhq * g.L + l) * D + ch * 8;
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.o) + idx) = *reinterpret_cast<const uint4*>(st_o + qi * C::PITCH + ch * 16);
+            if (a.o_res != nullptr)
+              *reinterpret_cast<uint4*>(a.o_res + idx) = *reinterpret_cast<const uint4*>(st_r + qi * C::PITCH + ch * 16);
+          }
+          VSA2_GROUP_SYNC(&misc->all_sync, all_phase);        // staging rows free before the next query block writes them
+        }
+      }
+      if (k > 0 && wg == 0 && sm_tid == 0 && misc->rescue_flag) {
+        int slot = atomicAdd(a.rescue_count, 1);
+        if (slot < a.rescue_cap) a.rescue_items[slot] = item;
+        else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
+      }
+      if (k > 0) ++n_items;
+    }
+  }
+
+done:
+  tc::tc_fence_before();
+  __syncthreads();
+  if (misc->abort_flag) {
+    if (tid == 0) atomicExch(&a.status->status, VSA2_ERR_DEVICE_TIMEOUT);
+    // let copies that are still in flight land before the CTA's shared memory is released
+    if (tid == 0) {
+      const unsigned long long t0 = tc::global_timer_ns();
+      while (tc::global_timer_ns() - t0 < 200000ull) {
+      }
+    }
+    __syncthreads();
+  }
+  if (warp == 4) tc::tmem_dealloc(tmem_base, 512);
+}
+
+cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, int cap, const int* items, const bf16* q, const bf16* k,
+                                 const bf16* v, const float* gate, const int* row_ptr, const int* col_idx,
+                                 const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
+
+bool fine_fwd_rows_supported(const Geo& g) { return g.N <= kFrMaxCubes; }
+
+// workspace: [StatusBlock][rescue list] as for launch_fine_fwd_tc; the rescue counter is StatusBlock.pad[0].
+cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                                    const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                                    float* lse, StatusBlock* status, cudaStream_t st) {
+  CUtensorMap tq, tk, tv;
+  if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv))
+    return cudaErrorInvalidValue;
+  int dev = 0, sms = 0;
+  cudaError_t e;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if (g.N > kFrMaxCubes) return cudaErrorInvalidValue;
+  FwdRowsArgs a;
+  a.gate = gate; a.row_ptr = row_ptr; a.col_idx = col_idx; a.oc_hat = oc_hat; a.o = o; a.o_res = o_res; a.lse = lse;
+  a.status = status;
+  a.rescue_count = &status->pad[0];
+  a.item_counter = &status->pad[1];
+  a.rescue_items = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(status) + 256);
+  a.rescue_cap = fwd_rescue_capacity();
+  const int total = g.batch * g.Hq * g.N;
+  const int grid = total < sms ? total : sms;
+  // The softmax warpgroups raise their register count to 200 with the registers the service warpgroups give up
+  // (setmaxnreg); that request would block for ever if the launch allocation were smaller than 128 per thread.
+  {
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, g.D == 128 ? (const void*)fine_fwd_rows_tc_kernel<128> : (const void*)fine_fwd_rows_tc_kernel<64>)) != cudaSuccess) return e;
+    if (fa.numRegs * kFrThreads < 256 * 56 + 256 * 200) return cudaErrorLaunchOutOfResources;
+  }
+  if (g.D == 128) {
+    const size_t smb = FwdRows<128>::smem_bytes(g.N);
+    if ((e = cudaFuncSetAttribute(fine_fwd_rows_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_rows_tc_kernel<128><<<grid, kFrThreads, smb, st>>>(tq, tk, tv, g, a);
+  } else {
+    const size_t smb = FwdRows<64>::smem_bytes(g.N);
+    if ((e = cudaFuncSetAttribute(fine_fwd_rows_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
+    fine_fwd_rows_tc_kernel<64><<<grid, kFrThreads, smb, st>>>(tq, tk, tv, g, a);
+  }
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  // query blocks whose row sums left the safe range are redone with the exact running maximum
+  return launch_fine_fwd_list(g, a.rescue_count, a.rescue_cap, a.rescue_items, q, k, v, gate, row_ptr, col_idx, oc_hat, o, o_res, lse, st);
+}
+
+}  // namespace vsa2

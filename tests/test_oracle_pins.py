@@ -659,3 +659,91 @@ def test_cube_major_permutation_matches_a_reshape_of_the_padded_volume(grid, cub
         rows = Y[n * geo.B:(n + 1) * geo.B]
         np.testing.assert_array_equal(rows[np.abs(rows).sum(axis=1) > 0], X[geo.cube_tokens[n]])
     np.testing.assert_array_equal(orc.from_cube_major(Y, geo), X)
+
+
+# ---------------------------------------------------------------------------
+# Sec. 2.2, the sentence after Eq. 12: text tokens share the attention space (MMDiT)
+# ---------------------------------------------------------------------------
+def rand_text(Lt, D, seed):
+    rng = np.random.default_rng(seed)
+    return tuple(orc.bf16_bits_to_f64(syn.f32_to_bf16_bits(rng.standard_normal((Lt, D), dtype=np.float32))) for _ in range(4))
+
+
+@pytest.mark.parametrize("grid,Lt", [((4, 8, 8), 37), ((5, 6, 9), 70)])
+def test_text_tokens_with_all_blocks_kept_are_dense_attention_over_the_concatenation(grid, Lt):
+    D, scale = 16, 0.3
+    Q, K, V, dO, gate, geo, mask = rand_problem(grid, D, 41)
+    Qt, Kt, Vt, dOt = rand_text(Lt, D, 42)
+    mask[:] = True
+    O_f, lse, O_t, lse_t = orc.joint_fine_attention(Q, K, V, Qt, Kt, Vt, mask, geo, scale)
+    qc, kc, vc = (torch.from_numpy(np.concatenate(p)) for p in ((Q, Qt), (K, Kt), (V, Vt)))
+    ref = F.scaled_dot_product_attention(qc[None], kc[None], vc[None], scale=scale)[0].numpy()
+    ref_lse = torch.logsumexp(qc @ kc.T * scale, dim=1).numpy()
+    assert np.abs(np.concatenate((O_f, O_t)) - ref).max() < 1e-12
+    assert np.abs(np.concatenate((lse, lse_t)) - ref_lse).max() < 1e-12
+    # without text tokens the joint functions are the plain ones
+    e = np.zeros((0, D))
+    O0, l0, Ot0, lt0 = orc.joint_fine_attention(Q, K, V, e, e, e, mask, geo, scale)
+    O1, l1 = orc.fine_attention(Q, K, V, mask, geo, scale)
+    assert np.array_equal(O0, O1) and np.array_equal(l0, l1) and Ot0.shape == (0, D)
+
+
+def test_text_tokens_merge_with_the_video_part_by_log_sum_exp():
+    """A video query's joint softmax over (kept video blocks, text) is the log-sum-exp merge of the block-sparse result
+    (pinned above) with a library softmax attention over the text keys alone; an empty video row leaves the text part."""
+    grid, D, Lt, scale = (5, 6, 9), 16, 45, 0.25
+    Q, K, V, dO, gate, geo, mask = rand_problem(grid, D, 43, density=0.3)
+    mask[3, :] = False
+    Qt, Kt, Vt, dOt = rand_text(Lt, D, 44)
+    O_f, lse, O_t, lse_t = orc.joint_fine_attention(Q, K, V, Qt, Kt, Vt, mask, geo, scale)
+    O_vv, lse_vv = orc.fine_attention(Q, K, V, mask, geo, scale)
+    st = torch.from_numpy(Q @ Kt.T * scale)
+    lse_vt = torch.logsumexp(st, dim=1).numpy()
+    O_vt = (torch.softmax(st, dim=1) @ torch.from_numpy(Vt)).numpy()
+    tot = np.logaddexp(lse_vv, lse_vt)
+    merged = np.exp(lse_vv - tot)[:, None] * O_vv + np.exp(lse_vt - tot)[:, None] * O_vt
+    assert np.abs(lse - tot).max() < 1e-12 and np.abs(O_f - merged).max() < 1e-12
+    rows3 = geo.cube_tokens[3]
+    assert np.abs(O_f[rows3] - O_vt[rows3]).max() < 1e-12
+    # text queries: dense over everything (library)
+    kc, vc = torch.from_numpy(np.concatenate((K, Kt))), torch.from_numpy(np.concatenate((V, Vt)))
+    ref_t = F.scaled_dot_product_attention(torch.from_numpy(Qt)[None], kc[None], vc[None], scale=scale)[0].numpy()
+    assert np.abs(O_t - ref_t).max() < 1e-12
+    # restricting the rows computes the same values on those rows
+    Of2, l2, Ot2, lt2 = orc.joint_fine_attention(Q, K, V, Qt, Kt, Vt, mask, geo, scale, rows=(1, 3), text_rows=(0, 44))
+    sel = np.concatenate([geo.cube_tokens[1], geo.cube_tokens[3]])
+    assert np.array_equal(Of2[sel], O_f[sel]) and np.array_equal(Ot2[[0, 44]], O_t[[0, 44]]) and (Ot2[1:44] == 0).all()
+
+
+def test_text_tokens_backward_matches_autograd_of_a_dense_masked_restatement():
+    grid, cube, D, Lt, scale = (5, 6, 9), (4, 4, 4), 16, 21, 0.2
+    Q, K, V, dO, gate, geo, mask = rand_problem(grid, D, 45, cube=cube, density=0.4)
+    mask[2, :] = False
+    Qt, Kt, Vt, dOt = rand_text(Lt, D, 46)
+    g = orc.joint_head_backward(Q, K, V, Qt, Kt, Vt, gate, mask, geo, scale, dO, dOt)
+    # restatement: one [L + Lt] x [L + Lt] score matrix in raster order, boolean mask built from the cube index of every
+    # token by reshape (never the oracle's index formula), library softmax; coarse branch from dense_restatement
+    L = geo.L
+    cube_of = to_cube_major(pad_volume(np.arange(L), grid, cube, fill=-1), cube)          # [N, B] raster ids
+    tok_cube = np.zeros(L, dtype=np.int64)
+    for n in range(cube_of.shape[0]):
+        ids = cube_of[n][cube_of[n] >= 0]
+        tok_cube[ids] = n
+    allow = np.ones((L + Lt, L + Lt), dtype=bool)
+    allow[:L, :L] = mask[tok_cube][:, tok_cube]
+    t = {n: torch.from_numpy(a).requires_grad_(True) for n, a in
+         (("q", Q), ("k", K), ("v", V), ("qt", Qt), ("kt", Kt), ("vt", Vt), ("gate", gate))}
+    s = torch.cat((t["q"], t["qt"])) @ torch.cat((t["k"], t["kt"])).T * scale
+    s = s.masked_fill(~torch.from_numpy(allow), float("-inf"))
+    O_all = torch.softmax(s, dim=1) @ torch.cat((t["v"], t["vt"]))
+    _, _, coarse = dense_restatement(t["q"], t["k"], t["v"], t["gate"], mask, grid, cube, scale)
+    B = cube[0] * cube[1] * cube[2]
+    flat = torch.from_numpy(cube_of.reshape(-1))
+    O_c = torch.zeros(L, D, dtype=torch.float64).index_put((flat[flat >= 0],), coarse["Oc_hat"].repeat_interleave(B, dim=0)[flat >= 0])
+    O = t["gate"][:, None] * O_c + O_all[:L]
+    ((O * torch.from_numpy(dO)).sum() + (O_all[L:] * torch.from_numpy(dOt)).sum()).backward()
+    for name, key in (("dQ", "q"), ("dK", "k"), ("dV", "v"), ("dQt", "qt"), ("dKt", "kt"), ("dVt", "vt"), ("dGate", "gate")):
+        err = np.abs(g[name] - t[key].grad.numpy()).max()
+        assert err < 1e-11, (name, err)
+    fwd = orc.joint_head_forward(Q, K, V, Qt, Kt, Vt, gate, mask, geo, scale)
+    assert np.abs(fwd["O"] - O.detach().numpy()).max() < 1e-12 and np.abs(fwd["O_t"] - O_all[L:].detach().numpy()).max() < 1e-12
