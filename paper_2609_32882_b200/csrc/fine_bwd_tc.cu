@@ -231,13 +231,14 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     }
   } else if (warp == 2 || warp == 3) {
     // ------------------------------------------------------------------ issuers of S^T = K_pair Q^T (warp 2) and
-    // dP^T = V_pair dO^T (warp 3)
-    if (lane == 0) {
+    // dP^T = V_pair dO^T (warp 3).  The whole warp runs the loop and one elected lane issues: a converged warp keeps the
+    // descriptors in uniform registers, and a tcgen05.mma then issues every ~74 cycles instead of ~117 from a lone lane.
+    {
       const bool is_s = warp == 2;
       const uint32_t b_addr = tc::smem_u32(is_s ? q_tile : do_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (uint32_t seq = 0;; ++seq) {
-        VSA2_NEXT_ITEM(item, seq);
+        VSA2_NEXT_ITEM_WARP(item, seq);
         const int i = item % g.N, bhq = item / g.N;
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
@@ -250,28 +251,34 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             VSA2_WAIT(&misc->a_full[sa], pa);
             VSA2_WAIT(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
-            mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
-            tc::mma_commit(&misc->s_full[sb]);
+            if (tc::elect_one()) {
+              mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+              tc::mma_commit(&misc->s_full[sb]);
+              if (t == nt - 1) tc::mma_commit(&misc->st_empty);
+            }
           } else {
             VSA2_WAIT(&misc->b_full[sb], pb);
             VSA2_WAIT(&misc->dp_free[sb], pb ^ 1);
             tc::tc_fence_after();
-            mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
-            tc::mma_commit(&misc->dp_full[sb]);
-            tc::mma_commit(&misc->b_empty[sb]);
+            if (tc::elect_one()) {
+              mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
+              tc::mma_commit(&misc->dp_full[sb]);
+              tc::mma_commit(&misc->b_empty[sb]);
+              if (t == nt - 1) tc::mma_commit(&misc->st_empty);
+            }
           }
+          __syncwarp();
         }
-        tc::mma_commit(&misc->st_empty);
         ++n_items;
       }
     }
   } else if (warp == 12) {
     // ------------------------------------------------------------------ issuer of dQ^T += K_pair^T dS^T
-    if (lane == 0) {
+    {
       const uint32_t ds_addr = tc::smem_u32(ds_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (uint32_t seq = 0;; ++seq) {
-        VSA2_NEXT_ITEM(item, seq);
+        VSA2_NEXT_ITEM_WARP(item, seq);
         const int i = item % g.N, bhq = item / g.N;
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
@@ -281,12 +288,15 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           const uint32_t sd = SPLIT ? 0u : (tg & 1), pd = SPLIT ? (tg & 1) : ((tg >> 1) & 1), sa = tg % kRingA;
           VSA2_WAIT(&misc->ds_ready[sd], pd);
           tc::tc_fence_after();
-          if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr, C::PBYTES, t > 0);
-          else mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
-          tc::mma_commit(&misc->a_empty[sa]);
-          tc::mma_commit(&misc->ds_free[sd]);
+          if (tc::elect_one()) {
+            if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr, C::PBYTES, t > 0);
+            else mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
+            tc::mma_commit(&misc->a_empty[sa]);
+            tc::mma_commit(&misc->ds_free[sd]);
+            if (t == nt - 1) tc::mma_commit(&misc->o_full);
+          }
+          __syncwarp();
         }
-        tc::mma_commit(&misc->o_full);
         ++n_items;
       }
     }
@@ -601,13 +611,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
   } else if (warp == 2 || warp == 3) {
     // ------------------------------------------------------------------ issuers of S = Q_pair K^T (warp 2) and
-    // dP = dO_pair V^T (warp 3)
-    if (lane == 0) {
+    // dP = dO_pair V^T (warp 3); whole warp in the loop, one elected lane issues (see the dQ pass)
+    {
       const bool is_s = warp == 2;
       const uint32_t b_addr = tc::smem_u32(is_s ? k_tile : v_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (uint32_t seq = 0;; ++seq) {
-        VSA2_NEXT_ITEM(item, seq);
+        VSA2_NEXT_ITEM_WARP(item, seq);
         VSA2_DKV_ITEM_SETUP();
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
@@ -620,30 +630,36 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             VSA2_WAIT_PARKED(&misc->a_full[sa], pa);
             VSA2_WAIT_PARKED(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
-            mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
-            tc::mma_commit(&misc->s_full[sb]);
+            if (tc::elect_one()) {
+              mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+              tc::mma_commit(&misc->s_full[sb]);
+              if (t == nt - 1) tc::mma_commit(&misc->st_empty);
+            }
           } else {
             VSA2_WAIT_PARKED(&misc->b_full[sb], pb);
             VSA2_WAIT_PARKED(&misc->dp_free[sb], pb ^ 1);
             tc::tc_fence_after();
-            mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
-            tc::mma_commit(&misc->dp_full[sb]);
-            tc::mma_commit(&misc->b_empty[sb]);
+            if (tc::elect_one()) {
+              mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
+              tc::mma_commit(&misc->dp_full[sb]);
+              tc::mma_commit(&misc->b_empty[sb]);
+              if (t == nt - 1) tc::mma_commit(&misc->st_empty);
+            }
           }
+          __syncwarp();
         }
-        tc::mma_commit(&misc->st_empty);
         ++n_items;
       }
     }
   } else if (warp == 16 || warp == 17) {
     // ------------------------------------------------------------------ issuers of dV^T += dO_pair^T P (warp 16) and
-    // dK^T += Q_pair^T dS (warp 17)
-    if (lane == 0) {
+    // dK^T += Q_pair^T dS (warp 17); whole warp in the loop, one elected lane issues
+    {
       const bool is_v = warp == 16;
       const uint32_t b_addr = tc::smem_u32(is_v ? p_tile : ds_tile), base = tc::smem_u32(smem);
       uint32_t tg = 0, n_items = 0;
       for (uint32_t seq = 0;; ++seq) {
-        VSA2_NEXT_ITEM(item, seq);
+        VSA2_NEXT_ITEM_WARP(item, seq);
         VSA2_DKV_ITEM_SETUP();
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
         if (k == 0) continue;
@@ -656,21 +672,27 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             VSA2_WAIT_PARKED(&misc->b_full[sv], (tg >> 1) & 1);
             VSA2_WAIT_PARKED(&misc->p_ready, tg & 1);
             tc::tc_fence_after();
-            if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, C::PBYTES, t > 0);
-            else mma_pairT_mnmajor<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
-            tc::mma_commit(&misc->b_empty[sv]);
-            tc::mma_commit(&misc->p_free);
+            if (tc::elect_one()) {
+              if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, C::PBYTES, t > 0);
+              else mma_pairT_mnmajor<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
+              tc::mma_commit(&misc->b_empty[sv]);
+              tc::mma_commit(&misc->p_free);
+              if (t == nt - 1) tc::mma_commit(&misc->o_full);
+            }
           } else {
             const uint32_t sa = tg % RA;
             VSA2_WAIT_PARKED(&misc->ds_ready[0], tg & 1);
             tc::tc_fence_after();
-            if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, C::PBYTES, t > 0);
-            else mma_pairT_mnmajor<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
-            tc::mma_commit(&misc->a_empty[sa]);
-            tc::mma_commit(&misc->ds_free[0]);
+            if (tc::elect_one()) {
+              if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, C::PBYTES, t > 0);
+              else mma_pairT_mnmajor<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
+              tc::mma_commit(&misc->a_empty[sa]);
+              tc::mma_commit(&misc->ds_free[0]);
+              if (t == nt - 1) tc::mma_commit(&misc->o_full);
+            }
           }
+          __syncwarp();
         }
-        tc::mma_commit(&misc->o_full);
         ++n_items;
       }
     }

@@ -32,7 +32,7 @@ namespace vsa2 {
 
 constexpr int kFrThreads = 512;
 constexpr int kFrKSlots = 3;
-constexpr int kFrVSlots = 2;
+constexpr int kFrVSlots = 3;
 constexpr int kFrMaxCubes = 8192;      // edge-flag table in shared memory: one byte per cube
 
 template <int D>
@@ -40,18 +40,17 @@ struct FwdRows {
   static constexpr int DH = D / 64;
   static constexpr uint32_t SLOT = 2 * DH * kSlab;     // a K pair or a V pair, [half][A | B]
   static constexpr uint32_t QBYTES = DH * kSlab;
-  static constexpr uint32_t PITCH = D * 2 + 16;        // bytes per staged output row (odd multiple of 16: no bank conflicts)
-  static constexpr uint32_t STAGE = 64 * PITCH;
+  static constexpr int NQ = 1;                                            // Q tiles (by item parity if 2)
   static constexpr uint32_t OFF_Q = (kFrKSlots + kFrVSlots) * SLOT;
-  static constexpr uint32_t OFF_STAGE = OFF_Q + QBYTES;
-  static constexpr uint32_t OFF_MISC = OFF_STAGE + 2 * STAGE;
+  static constexpr uint32_t OFF_MISC = OFF_Q + NQ * QBYTES;
   static constexpr uint32_t MISC_BYTES = 4096;
   static constexpr uint32_t TM_S = 0, TM_P = 256, TM_O = 384;
   static size_t smem_bytes(int n_cubes) { return OFF_MISC + MISC_BYTES + ((size_t)n_cubes + 15) / 16 * 16 + 1024; }
 };
 
 struct FwdRowsMisc {
-  uint64_t q_full, q_empty, o_full, o_empty;
+  uint64_t q_full[2], q_empty[2], o_full, o_empty;
+  uint64_t tab_full[2], tab_free[2];   // per-item tables (tok, gate, oc) of the item with that parity
   uint64_t k_full[kFrKSlots], k_empty[kFrKSlots];
   uint64_t v_full[kFrVSlots], v_empty[kFrVSlots];
   uint64_t s_full[2], s_free[2];
@@ -64,11 +63,20 @@ struct FwdRowsMisc {
   unsigned short vmask[16][4];     // [edge flags][lane % 4]: which of a thread's 16 key columns of a block are valid tokens
   alignas(16) float m_ref[64];     // per query row: reference exponent (log2 units)
   float red[2][2][64];             // [warpgroup][exact sum | sum of the bf16 roundings][query row]
-  alignas(16) float oc[128];       // coarse output row of the query cube
+  alignas(16) float oc[2][128];    // coarse output row of the query cube, by item parity
   int tok[2][64];                  // raster token of each query row (-1 = padding), by item parity
   float gate[2][64];
+  int list_k[2], list_beg[2];      // length and start of the item's list of KV blocks
+  int list_head[2][4];             // its first four entries (tiles 0 and 1)
 };
 static_assert(sizeof(FwdRowsMisc) <= 4096, "misc region too small");
+
+#ifdef VSA2_TRACE
+__device__ long long g_fr_trace[4 * 256 * 8];
+#define FR_TR(role, tile, slot) do { if (blockIdx.x == 0 && (tile) < 256u) g_fr_trace[((role) * 256 + (tile)) * 8 + (slot)] = clock64(); } while (0)
+#else
+#define FR_TR(role, tile, slot) do {} while (0)
+#endif
 
 struct FwdRowsArgs {
   int* item_counter;    // global, zero before the launch
@@ -93,7 +101,6 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* q_tile = smem + C::OFF_Q;
-  unsigned char* stage = smem + C::OFF_STAGE;
   FwdRowsMisc* misc = reinterpret_cast<FwdRowsMisc*>(smem + C::OFF_MISC);
   unsigned char* edge = smem + C::OFF_MISC + C::MISC_BYTES;      // edge flags of every cube
 
@@ -116,8 +123,12 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   }
   if (tid == 0) {
     misc->abort_flag = 0;
-    tc::mbar_init(&misc->q_full, 1);
-    tc::mbar_init(&misc->q_empty, 1);
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(&misc->q_full[s], 1);
+      tc::mbar_init(&misc->q_empty[s], 1);
+      tc::mbar_init(&misc->tab_full[s], 32);
+      tc::mbar_init(&misc->tab_free[s], 256);
+    }
     tc::mbar_init(&misc->o_full, 1);
     tc::mbar_init(&misc->o_empty, 256);
     for (int s = 0; s < kFrKSlots; ++s) {
@@ -135,7 +146,7 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       tc::mbar_init(&misc->p_free[s], 1);
     }
     tc::mbar_init(&misc->all_sync, 256);
-    item_queue_init(&misc->items, 4 + 2 + 256);     // lane 0 of the producers, two issuers, the softmax threads
+    item_queue_init(&misc->items, 4 + 2 + 1 + 256); // lane 0 of the producers, of the two issuers and of the table loader, the softmax threads
     tc::fence_barrier_init();
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
@@ -186,13 +197,15 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           int it_, ih_, iw_;
           cube_coords(g, i, it_, ih_, iw_);
           int ok = 1;
+          const uint32_t qb = n_items % C::NQ;
           if (lane == 0) {
-            ok = tc::mbar_wait(&misc->q_empty, (n_items & 1) ^ 1, &misc->abort_flag);
-            if (ok) tc::mbar_expect_tx(&misc->q_full, C::QBYTES);
+            ok = tc::mbar_wait(&misc->q_empty[qb], ((n_items / C::NQ) & 1) ^ 1, &misc->abort_flag);
+            if (ok) tc::mbar_expect_tx(&misc->q_full[qb], C::QBYTES);
           }
           if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
           if (lane < C::DH)
-            tc::tma_load_5d(q_tile + lane * kSlab, &tm_q, &misc->q_full, lane * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+            tc::tma_load_5d(q_tile + qb * C::QBYTES + lane * kSlab, &tm_q, &misc->q_full[qb], lane * 64, iw_ * g.Bw, ih_ * g.Bh,
+                            it_ * g.Bt, bhq);
         }
         ++n_items;
         const int nt = (k + 1) >> 1;
@@ -215,23 +228,33 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       }
     } else if (warp == 4) {
       // ---------------------------------------------------------------- issuer of S(t) = Q * K_pair^T
-      if (lane == 0) {
-        constexpr uint32_t idesc = tc::idesc_bf16(64, 128, false, false);
-        const uint64_t dq = tc::smem_desc_sw128(tc::smem_u32(q_tile), 16, 1024);
-        const uint32_t slot0 = tc::smem_u32(smem);
-        uint32_t tg = 0, n_items = 0;
-        for (uint32_t seq = 0;; ++seq) {
-          VSA2_NEXT_ITEM(item, seq);
-          const int i = item % g.N, bhq = item / g.N;
-          const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
-          if (k == 0) continue;
-          const int nt = (k + 1) >> 1;
-          VSA2_WAIT(&misc->q_full, n_items & 1);
-          for (int t = 0; t < nt; ++t, ++tg) {
-            const uint32_t slot = tg % kFrKSlots, buf = tg & 1;
-            VSA2_WAIT(&misc->k_full[slot], (tg / kFrKSlots) & 1);
-            VSA2_WAIT(&misc->s_free[buf], ((tg >> 1) & 1) ^ 1);
-            tc::tc_fence_after();
+      // The whole warp runs the loop and one elected lane issues: with the warp converged the compiler keeps the
+      // descriptors in uniform registers, and a tcgen05.mma then issues every ~74 cycles instead of ~117 from a lone lane.
+      constexpr uint32_t idesc = tc::idesc_bf16(64, 128, false, false);
+      const uint32_t slot0 = tc::smem_u32(smem);
+      uint32_t tg = 0, n_items = 0;
+      for (uint32_t seq = 0;; ++seq) {
+        int item = 0;
+        if (lane == 0) item = item_get(&misc->items, seq, &misc->abort_flag);
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item == -2) goto done;
+        if (item < 0) break;
+        const int i = item % g.N, bhq = item / g.N;
+        const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+        if (k == 0) continue;
+        const int nt = (k + 1) >> 1;
+        const uint32_t qb = n_items % C::NQ;
+        const uint64_t dq = tc::smem_desc_sw128(tc::smem_u32(q_tile) + qb * C::QBYTES, 16, 1024);
+        VSA2_WAIT(&misc->q_full[qb], (n_items / C::NQ) & 1);
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t slot = tg % kFrKSlots, buf = tg & 1;
+          if (lane == 0) FR_TR(0, tg, 0);
+          VSA2_WAIT(&misc->k_full[slot], (tg / kFrKSlots) & 1);
+          if (lane == 0) FR_TR(0, tg, 1);
+          VSA2_WAIT(&misc->s_free[buf], ((tg >> 1) & 1) ^ 1);
+          if (lane == 0) FR_TR(0, tg, 2);
+          tc::tc_fence_after();
+          if (tc::elect_one()) {
             const uint64_t dk = tc::smem_desc_sw128(slot0 + slot * C::SLOT, 16, 1024);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
@@ -241,30 +264,39 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             }
             tc::mma_commit(&misc->s_full[buf]);
             tc::mma_commit(&misc->k_empty[slot]);
+            if (t == nt - 1) tc::mma_commit(&misc->q_empty[qb]);   // the Q tile may be replaced once the last S of the block is done
           }
-          tc::mma_commit(&misc->q_empty);          // the Q tile may be replaced once the last S of the block is done
-          ++n_items;
+          __syncwarp();
+          if (lane == 0) FR_TR(0, tg, 3);
         }
+        ++n_items;
       }
     } else if (warp == 5) {
       // ---------------------------------------------------------------- issuer of O += P(t) * V_pair
-      if (lane == 0) {
-        constexpr uint32_t idesc = tc::idesc_bf16(64, D, false, true);
-        constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;       // distance between the two 64-channel halves of V
-        const uint32_t slot0 = tc::smem_u32(smem) + kFrKSlots * C::SLOT;
-        uint32_t tg = 0, n_items = 0;
-        for (uint32_t seq = 0;; ++seq) {
-          VSA2_NEXT_ITEM(item, seq);
-          const int i = item % g.N, bhq = item / g.N;
-          const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
-          if (k == 0) continue;
-          const int nt = (k + 1) >> 1;
-          VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous query block's accumulator was read out
-          for (int t = 0; t < nt; ++t, ++tg) {
-            const uint32_t slot = tg % kFrVSlots, buf = tg & 1;
-            VSA2_WAIT(&misc->v_full[slot], (tg / kFrVSlots) & 1);
-            VSA2_WAIT(&misc->p_ready[buf], (tg >> 1) & 1);
-            tc::tc_fence_after();
+      constexpr uint32_t idesc = tc::idesc_bf16(64, D, false, true);
+      constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;       // distance between the two 64-channel halves of V
+      const uint32_t slot0 = tc::smem_u32(smem) + kFrKSlots * C::SLOT;
+      uint32_t tg = 0, n_items = 0;
+      for (uint32_t seq = 0;; ++seq) {
+        int item = 0;
+        if (lane == 0) item = item_get(&misc->items, seq, &misc->abort_flag);
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item == -2) goto done;
+        if (item < 0) break;
+        const int i = item % g.N, bhq = item / g.N;
+        const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
+        if (k == 0) continue;
+        const int nt = (k + 1) >> 1;
+        VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous query block's accumulator was read out
+        for (int t = 0; t < nt; ++t, ++tg) {
+          const uint32_t slot = tg % kFrVSlots, buf = tg & 1;
+          if (lane == 0) FR_TR(1, tg, 0);
+          VSA2_WAIT(&misc->v_full[slot], (tg / kFrVSlots) & 1);
+          if (lane == 0) FR_TR(1, tg, 1);
+          VSA2_WAIT(&misc->p_ready[buf], (tg >> 1) & 1);
+          if (lane == 0) FR_TR(1, tg, 2);
+          tc::tc_fence_after();
+          if (tc::elect_one()) {
             const uint64_t dv = tc::smem_desc_sw128(slot0 + slot * C::SLOT, lbo, 1024);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
@@ -273,10 +305,53 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             }
             tc::mma_commit(&misc->v_empty[slot]);
             tc::mma_commit(&misc->p_free[buf]);
+            if (t == nt - 1) tc::mma_commit(&misc->o_full);
           }
-          tc::mma_commit(&misc->o_full);
-          ++n_items;
+          __syncwarp();
+          if (lane == 0) FR_TR(1, tg, 3);
         }
+        ++n_items;
+      }
+    } else if (warp == 6) {
+      // ---------------------------------------------------------------- per-item tables, one item ahead of the softmax warps:
+      // raster token and gate of every query row, coarse output row of the cube (global loads kept off their critical path)
+      const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
+      for (uint32_t seq = 0;; ++seq) {
+        int item = 0;
+        if (lane == 0) item = item_get(&misc->items, seq, &misc->abort_flag);
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item == -2) goto done;
+        if (item < 0) break;
+        const int i = item % g.N, bhq = item / g.N;
+        const uint32_t tb = seq & 1;
+        int it_, ih_, iw_;
+        cube_coords(g, i, it_, ih_, iw_);
+        const int beg_ = a.row_ptr[(size_t)bhq * (g.N + 1) + i], k_ = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - beg_;
+        const int head_ = (lane < 4 && lane < k_) ? a.col_idx[(size_t)bhq * g.nnz_cap + beg_ + lane] : 0;
+        int l2[2];
+        float g2[2], oc4[4];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          l2[r] = cube_token(g, it_, ih_, iw_, lane + 32 * r);
+          g2[r] = (coarse && l2[r] >= 0) ? a.gate[(size_t)bhq * g.L + l2[r]] : 0.f;
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+          oc4[r] = (coarse && lane + 32 * r < D) ? a.oc_hat[((size_t)bhq * g.N + i) * D + lane + 32 * r] : 0.f;
+        VSA2_WAIT_PARKED(&misc->tab_free[tb], ((seq >> 1) & 1) ^ 1);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          misc->tok[tb][lane + 32 * r] = l2[r];
+          misc->gate[tb][lane + 32 * r] = g2[r];
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) misc->oc[tb][lane + 32 * r] = oc4[r];
+        if (lane < 4) misc->list_head[tb][lane] = head_;
+        if (lane == 0) {
+          misc->list_k[tb] = k_;
+          misc->list_beg[tb] = beg_;
+        }
+        tc::mbar_arrive(&misc->tab_full[tb]);
       }
     }
   } else {
@@ -287,26 +362,18 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const int cq = lane & 3;
     const int row_a = quad * 16 + (lane >> 2), row_b = row_a + 8;     // the two query rows of this thread
     const int sm_tid = tid & 127;
-    const int t256 = tid - 256;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && a.gate != nullptr;
     constexpr int COLS = D / 2;                  // output columns per warpgroup in the epilogue
     uint32_t tg = 0, n_items = 0, all_phase = 0;
     for (uint32_t n_all = 0;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
       const int i = item % g.N, bhq = item / g.N;
-      const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
-      const int k = end - beg;
-      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
       const int tb = n_all & 1;
-      if (wg == 0 && sm_tid < 64) {
-        int it_, ih_, iw_;
-        cube_coords(g, i, it_, ih_, iw_);
-        const int l = cube_token(g, it_, ih_, iw_, sm_tid);
-        misc->tok[tb][sm_tid] = l;
-        misc->gate[tb][sm_tid] = (coarse && l >= 0) ? a.gate[(size_t)bhq * g.L + l] : 0.f;
-      }
-      if (wg == 1 && sm_tid < D) misc->oc[sm_tid] = coarse ? a.oc_hat[((size_t)bhq * g.N + i) * D + sm_tid] : 0.f;
+      VSA2_WAIT(&misc->tab_full[tb], (n_all >> 1) & 1);  // the item's tables (loaded one item ahead by warp 6)
+      const int k = misc->list_k[tb];
+      const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + misc->list_beg[tb];
+      const int* head = misc->list_head[tb];
+      (void)i;
       if (wg == 0 && sm_tid == 0) misc->rescue_flag = 0;
 
       const int nt = (k + 1) >> 1;
@@ -323,8 +390,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         tc::tc_fence_before();
         tc::mbar_arrive(&misc->s_free[buf]);
         have_first = true;
-        const unsigned ma = misc->vmask[edge[cols[0]]][cq];
-        const unsigned mb = k > 1 ? misc->vmask[edge[cols[1]]][cq] : 0u;
+        const unsigned ma = misc->vmask[edge[head[0]]][cq];
+        const unsigned mb = k > 1 ? misc->vmask[edge[head[1]]][cq] : 0u;
         float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
         for (int n = 0; n < 16; ++n) {
@@ -341,26 +408,36 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           misc->m_ref[row_b] = (mx_b > -INFINITY) ? mx_b * c2 : 0.f;
         }
       }
-      VSA2_GROUP_SYNC(&misc->all_sync, all_phase);       // tables and reference exponents visible to both warpgroups
+      VSA2_GROUP_SYNC(&misc->all_sync, all_phase);       // reference exponents visible to both warpgroups
 
       float l_a = 0.f, l_b = 0.f, r_a = 0.f, r_b = 0.f;   // exact sums and sums of the bf16 roundings of the two rows
       float m_a = 0.f, m_b = 0.f;
       if (k > 0) {
         m_a = misc->m_ref[row_a];
         m_b = misc->m_ref[row_b];
-        for (int t = ((tg0 & 1) == (uint32_t)wg) ? 0 : 1; t < nt; t += 2) {
+        const int t_first = ((tg0 & 1) == (uint32_t)wg) ? 0 : 1;
+        // KV blocks of this warpgroup's tiles: the first from the item's table, the others fetched one own tile ahead
+        int ja = head[2 * t_first < k ? 2 * t_first : 0], jb = head[2 * t_first + 1 < k ? 2 * t_first + 1 : 0];
+        for (int t = t_first; t < nt; t += 2) {
           const uint32_t tgt = tg0 + t, buf = tgt & 1;
           const bool dup = 2 * t + 1 >= k;
-          const unsigned ma = misc->vmask[edge[cols[2 * t]]][cq];
-          const unsigned mb = dup ? 0u : misc->vmask[edge[cols[2 * t + 1]]][cq];
+          const unsigned ma = misc->vmask[edge[ja]][cq];
+          const unsigned mb = dup ? 0u : misc->vmask[edge[jb]][cq];
+          if (t + 2 < nt) {
+            ja = cols[2 * t + 4];
+            jb = cols[2 * t + 5 < k ? 2 * t + 5 : 2 * t + 4];
+          }
+          if (sm_tid == 0) FR_TR(2 + wg, tgt, 0);
           if (!(have_first && t == 0)) {
             VSA2_WAIT(&misc->s_full[buf], (tgt >> 1) & 1);
+            if (sm_tid == 0) FR_TR(2 + wg, tgt, 1);
             tc::tc_fence_after();
             tc::tmem_ld_16x256b_x16(lane_addr + C::TM_S + buf * 128, sv);
             tc::tmem_ld_wait();
             tc::tc_fence_before();
             tc::mbar_arrive(&misc->s_free[buf]);
           }
+          if (sm_tid == 0) FR_TR(2 + wg, tgt, 2);
           uint32_t pk[32];
           if ((ma & mb) == 0xffffu) {
 #pragma unroll
@@ -396,11 +473,14 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
               pk[2 * n + 1] = wb;
             }
           }
+          if (sm_tid == 0) FR_TR(2 + wg, tgt, 3);
           VSA2_WAIT(&misc->p_free[buf], ((tgt >> 1) & 1) ^ 1);
+          if (sm_tid == 0) FR_TR(2 + wg, tgt, 4);
           tc::tmem_st_16x128b_x16(lane_addr + C::TM_P + buf * 64, pk);
           tc::tmem_st_wait();
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->p_ready[buf]);
+          if (sm_tid == 0) FR_TR(2 + wg, tgt, 5);
         }
         tg += nt;
         // row sums: over the four threads of a row here, over the two warpgroups through shared memory
@@ -461,7 +541,7 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 #pragma unroll
           for (int n = 0; n < COLS / 8; ++n) {
             const int col = wg * COLS + 8 * n + 2 * cq;
-            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[col]);
+            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[tb][col]);
             if (ta >= 0)
               *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.L + ta) * D + col) =
                   make_float2(fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a));
@@ -470,37 +550,32 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                   make_float2(fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b));
           }
         } else {
-          // bf16 output and rounding residual: through shared memory, then 16-byte stores
-          unsigned char* st_o = stage;
-          unsigned char* st_r = stage + C::STAGE;
+          // bf16 output and its rounding residual: a thread stores bf16 pairs, the four threads of a row 16 contiguous bytes;
+          // the eight column groups of a row complete its 128-byte lines within the same loop, so L2 merges them
+          bf16* ob = reinterpret_cast<bf16*>(a.o);
 #pragma unroll
           for (int n = 0; n < COLS / 8; ++n) {
             const int col = wg * COLS + 8 * n + 2 * cq;
-            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[col]);
+            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[tb][col]);
             const float v0 = fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), v1 = fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a);
             const float v2 = fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), v3 = fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b);
             uint32_t ha, la2, hb, lb2;
             split_bf16x2(v0, v1, ha, la2);
             split_bf16x2(v2, v3, hb, lb2);
-            *reinterpret_cast<uint32_t*>(st_o + row_a * C::PITCH + col * 2) = ha;
-            *reinterpret_cast<uint32_t*>(st_o + row_b * C::PITCH + col * 2) = hb;
-            *reinterpret_cast<uint32_t*>(st_r + row_a * C::PITCH + col * 2) = la2;
-            *reinterpret_cast<uint32_t*>(st_r + row_b * C::PITCH + col * 2) = lb2;
+            if (ta >= 0) {
+              const size_t idx = ((size_t)bhq * g.L + ta) * D + col;
+              *reinterpret_cast<uint32_t*>(ob + idx) = ha;
+              if (a.o_res != nullptr) *reinterpret_cast<uint32_t*>(a.o_res + idx) = la2;
+            }
+            if (tk_b >= 0) {
+              const size_t idx = ((size_t)bhq * g.L + tk_b) * D + col;
+              *reinterpret_cast<uint32_t*>(ob + idx) = hb;
+              if (a.o_res != nullptr) *reinterpret_cast<uint32_t*>(a.o_res + idx) = lb2;
+            }
           }
-          VSA2_GROUP_SYNC(&misc->all_sync, all_phase);
-          constexpr int CH = D / 8;                                      // 16-byte chunks per token row
-          for (int e = t256; e < 64 * CH; e += 256) {
-            const int qi = e / CH, ch = e % CH;
-            const int l = misc->tok[tb][qi];
-            if (l < 0) continue;
-            const size_t idx = ((size_t)bhq * g.L + l) * D + ch * 8;
-            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.o) + idx) = *reinterpret_cast<const uint4*>(st_o + qi * C::PITCH + ch * 16);
-            if (a.o_res != nullptr)
-              *reinterpret_cast<uint4*>(a.o_res + idx) = *reinterpret_cast<const uint4*>(st_r + qi * C::PITCH + ch * 16);
-          }
-          VSA2_GROUP_SYNC(&misc->all_sync, all_phase);        // staging rows free before the next query block writes them
         }
       }
+      tc::mbar_arrive(&misc->tab_free[tb]);
       if (k > 0 && wg == 0 && sm_tid == 0 && misc->rescue_flag) {
         int slot = atomicAdd(a.rescue_count, 1);
         if (slot < a.rescue_cap) a.rescue_items[slot] = item;
@@ -531,6 +606,12 @@ cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, int cap, const 
                                  const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
 
 bool fine_fwd_rows_supported(const Geo& g) { return g.N <= kFrMaxCubes; }
+
+#ifdef VSA2_TRACE
+extern "C" int vsa2_debug_fwd_trace(long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_fr_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -5;
+}
+#endif
 
 // workspace: [StatusBlock][rescue list] as for launch_fine_fwd_tc; the rescue counter is StatusBlock.pad[0].
 cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,

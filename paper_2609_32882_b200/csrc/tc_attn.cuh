@@ -197,6 +197,14 @@ __device__ __forceinline__ int item_get(ItemQueue* q, uint32_t seq, volatile int
   if (ITEM == -2) goto done;                                       \
   if (ITEM < 0) break
 
+// the same for a role whose whole warp runs the loop (lane 0 takes the item, the others receive it by shuffle)
+#define VSA2_NEXT_ITEM_WARP(ITEM, SEQ)                                     \
+  int ITEM = 0;                                                            \
+  if (lane == 0) ITEM = item_get(&misc->items, (SEQ), &misc->abort_flag);  \
+  ITEM = __shfl_sync(0xffffffffu, ITEM, 0);                                \
+  if (ITEM == -2) goto done;                                               \
+  if (ITEM < 0) break
+
 #define VSA2_WAIT(bar, parity)                                         \
   do {                                                                 \
     if (!tc::mbar_wait((bar), (parity), &misc->abort_flag)) goto done; \
