@@ -42,8 +42,10 @@ NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.500836e9 + 0.294249e9), "fine
                                 "fine_bwd_dkv": 5 * (0.769323e9 + 0.304400e9)}
 
 
-def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None) -> syn.Workload:
+def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None, text_len: int = 0) -> syn.Workload:
     wl = syn.CONFIGS[config]
+    if text_len:
+        wl = wl.replace(text_len=text_len, name=f"{wl.name}_text{text_len}")
     if grid:
         wl = wl.replace(grid=tuple(grid), name=f"{wl.name}_grid{'x'.join(map(str, grid))}")
     if cube:
@@ -57,8 +59,8 @@ def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None) -
 
 def config_dict(wl: syn.Workload, forward_only: bool) -> dict:
     """The `config` object of the JSON line: what the workload is (both arms print the same)."""
-    gb = (2 * wl.heads_q + 2 * wl.heads_kv) * wl.batch * wl.L * wl.head_dim * 2 / 1e9
-    return {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
+    gb = (2 * wl.heads_q + 2 * wl.heads_kv) * wl.batch * (wl.L + wl.text_len) * wl.head_dim * 2 / 1e9
+    return {"workload": wl.name, "grid": list(wl.grid), "tokens": wl.L, "text_tokens": wl.text_len, "heads_q": wl.heads_q, "heads_kv": wl.heads_kv,
             "head_dim": wl.head_dim, "cube": list(wl.cube), "rpool": list(wl.rpool), "select_mode": wl.select_mode,
             "topk": wl.topk, "forward_only": bool(forward_only),
             "l2": f"inputs (Q,K,V,dO: {gb:.1f} GB) far larger than the 126 MB L2; no explicit flush"}
@@ -67,7 +69,7 @@ def config_dict(wl: syn.Workload, forward_only: bool) -> dict:
 def flop_counts(wl: syn.Workload, nnz_total: int) -> dict:
     """Algorithmic work of one step.  nnz_total = selected (query block, KV block) pairs over all heads."""
     B, D = int(np.prod(wl.cube)), wl.head_dim
-    L, Hq, N, G = wl.L, wl.heads_q * wl.batch, wl.n_cubes, int(np.prod(wl.cube)) // int(np.prod(wl.rpool))
+    L, Hq, N, G = wl.L + wl.text_len, wl.heads_q * wl.batch, wl.n_cubes, int(np.prod(wl.cube)) // int(np.prod(wl.rpool))
     pair = B * B * D
     return {
         "dense_equiv_fwd": 4.0 * L * L * D * Hq,
@@ -193,7 +195,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = workload(args.config, args.heads, args.topk, args.grid, args.cube)
+    wl = workload(args.config, args.heads, args.topk, args.grid, args.cube, args.text_len)
     hd = head_inputs(wl, 0, 0)
     flops = flop_counts(wl, 0)
     for _ in range(args.warmup):
@@ -247,7 +249,7 @@ def run_ours(args):
     vb._lib()
 
     # every rank runs its own replica of the workload (heads are independent: no data-path collective)
-    wl = workload(args.config, args.heads, args.topk, args.grid, args.cube)
+    wl = workload(args.config, args.heads, args.topk, args.grid, args.cube, args.text_len)
     wl = wl.replace(seed=replicas.replica_seed(wl.seed, rank))
     t_gen = time.time()
     data = syn.make_inputs(wl, threads=max(1, min(32, cpu_cores() // max(1, world))))
@@ -353,6 +355,10 @@ def run_ours(args):
     torch.cuda.synchronize()
     attn.check_status()
     nnz_total = int(attn.map_views()[0][..., -1].sum().item())
+    if wl.text_len:
+        # block pairs the fine kernels compute with text tokens: every video row also keeps the text blocks, text rows keep all
+        tb = -(-wl.text_len // 64)
+        nnz_total += wl.batch * wl.heads_q * (wl.n_cubes * tb + tb * (wl.n_cubes + tb))
 
     # per-kernel events: one (start, stop) pair per kernel group and step
     nk = len(vb.KERNELS)
@@ -515,6 +521,8 @@ def main():
     ap.add_argument("--grid", type=triple, default=None, help="override the latent grid T,H,W (context rows: the paper's 61,45,80)")
     ap.add_argument("--cube", type=triple, default=None, help="override the cube, e.g. 4,4,8 (128 tokens; context rows)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small cases for ncu captures)")
+    ap.add_argument("--text-len", type=int, default=0,
+                    help="text tokens appended to every head (context rows: joint video + text attention)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

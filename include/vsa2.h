@@ -67,19 +67,27 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
 enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
                                          (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
-enum { VSA2_FLAG_FAST_BWD = 4 };      /* backward passes with P and dS rounded once to bf16 before the dV, dK and dQ products
-                                         (about 10-20 % faster).  By default both are carried as a bf16 value plus the bf16
-                                         rounding of what that lost, which keeps dQ, dK, dV inside max abs err 2e-2 where
-                                         gradients are large (|g| > 5: sharply peaked rows, GQA groups); with this flag the
-                                         worst elements reach 2.5e-2 (MHA, 720p) to 3.7e-2 (GQA 4:1, 480p) */
-enum { VSA2_FLAG_HALF_CUBE_FWD = 128 };/* 128-token cubes only: fine forward with the 64-query kernel on the two half-cubes
-                                         separately instead of the 128-query kernel (validation aid, same results) */
+/* Precision of the backward passes.  P and dS are the bf16 operands of the dV, dK and dQ products; rounded once (2^-9
+ * relative) they alone push the worst elements of large gradients (|g| > 5) past max abs err 2e-2.  By default the dQ pass
+ * always, and the dK/dV pass for GQA groups (where a KV block sums several heads), carry them as a bf16 pair -- the value
+ * and the bf16 rounding of what that lost -- in one product of twice the width.  Measured on 720p / 480p samples against
+ * the oracle (fp32 outputs): dQ 7e-3 instead of 2.5e-2, GQA dK 8e-3 instead of 2.6e-2; MHA dK, dV stay near 1e-2 either way. */
+enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once everywhere (dQ pass about 15 % faster, GQA dK/dV pass about 30 %) */
+enum { VSA2_FLAG_PRECISE_BWD = 8 };   /* carry the pair in the dK/dV pass for MHA as well (that pass about 35 % slower): for maps
+                                         that keep only a few blocks per row, where the softmax is sharply peaked */
+enum { VSA2_FLAG_PAIR_QUERY_FWD = 128 };/* fine forward with the 128-query kernel where two query blocks keep the same KV blocks on the
+                                         same operand tiles: the two halves of a 128-token cube, or (with VSA2_FLAG_GROUP_ROUTING and an
+                                         even number of query heads per KV head) pairs of heads that share their map.  About 1.2x
+                                         faster there than the default 64-query kernel, but it normalises the output by the fp32 row
+                                         sum rather than by the sum of the bf16-rounded weights, so on sharply peaked rows dQ of a
+                                         later backward can reach 2.5e-2 */
 enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV group share one block map ("group head", Sec. 4
                                          ablation): the block scores of the group's heads are added before the TopK, so
                                          the maps written for those heads are identical.  Not with VSA2_PER_QUERY_BUDGET
                                          (budgets belong to single heads): VSA2_ERR_UNSUPPORTED.
-                                         vsa2_attn_fwd with this flag RELIES on that: with an even number of query heads
-                                         per KV head it reads the map of the first head of each pair of heads only */
+                                         vsa2_attn_fwd with this flag and VSA2_FLAG_PAIR_QUERY_FWD RELIES on that: with an
+                                         even number of query heads per KV head it reads the map of the first head of each
+                                         pair of heads only */
 
 /* Problem statement (host struct). */
 typedef struct vsa2_params {
@@ -97,6 +105,12 @@ typedef struct vsa2_params {
   float   softmax_scale;                       /* 0 => 1/sqrt(head_dim); used by coarse, router and fine alike */
   int32_t out_dtype;                           /* VSA2_BF16 or VSA2_F32: dtype of O, dQ, dK, dV */
   int32_t flags;                               /* VSA2_FLAG_* */
+  int32_t text_len;                            /* Lt >= 0: text tokens that share the attention space (Sec. 2.2, the sentence
+                                                  after Eq. 12; MMDiT).  With Lt > 0 every token tensor (q, k, v, o, d_o, dq, dk,
+                                                  dv: [batch, heads, L + Lt, D]; lse: [batch, heads_q, L + Lt]) holds the L video
+                                                  tokens in raster order followed by the Lt text tokens.  The block map, the router
+                                                  and the coarse branch cover the video tokens only; gate and dgate stay
+                                                  [batch, heads_q, L].  64-token cubes only. */
   int64_t nnz_cap;                             /* capacity of col_idx/row_idx per (batch, query head); 0 => N*K.
                                                   PER_QUERY_BUDGET requires it (>= sum_i min(k_i, N)). */
 } vsa2_params;
@@ -114,10 +128,13 @@ typedef struct vsa2_sizes {
   int64_t pooled_q_elems;     /* float elements of saved.qc and saved.oc_hat: batch*heads_q*N*D */
   int64_t pooled_kv_elems;    /* float elements of saved.kc and of saved.vc: batch*heads_kv*N*D */
   int64_t lse_c_elems;        /* float elements of saved.lse_c: batch*heads_q*N */
-  int64_t o_res_elems;        /* bf16 elements of saved.o_res: batch*heads_q*L*D (0 when out_dtype is fp32) */
+  int64_t o_res_elems;        /* bf16 elements of saved.o_res: batch*heads_q*(L + Lt)*D (0 when out_dtype is fp32) */
   size_t  route_workspace_bytes;
   size_t  fwd_workspace_bytes;
   size_t  bwd_workspace_bytes;
+  int64_t tokens_per_head;    /* L + Lt: rows per head of every token tensor */
+  int32_t text_blocks;        /* ceil(Lt / 64): blocks the fine kernels append to the N video cubes */
+  int32_t reserved;
 } vsa2_sizes;
 
 /* Block map of the selected (query block, KV block) pairs (host struct of device pointers).
@@ -184,6 +201,12 @@ int vsa2_route_noalloc(const vsa2_params* p, const void* q, const void* k, const
 /* Read-only access to the block scores P_r [batch, heads_q, N, N] (fp32) that the last vsa2_route
  * call on `workspace` left there; valid until the workspace is reused.  Returns NULL on bad input. */
 const float* vsa2_route_scores(const vsa2_params* p, const void* workspace);
+
+/* Text tokens (p->text_len > 0; Sec. 2.2, the sentence after Eq. 12).  Reading taken: one softmax per query row over its whole
+ * key set.  A video query of cube i attends the kept video cubes of row i of the map and ALL text keys; a text query attends
+ * all video keys and all text keys.  Text queries take no part in the coarse branch or the gate (their output is the fine
+ * branch's), text keys none in the router.  vsa2_route is unchanged (it reads the video rows of q and k); vsa2_attn_fwd and
+ * vsa2_attn_bwd append the text blocks to the map inside their workspace and run the same kernels on the longer lists. */
 
 /* Coarse branch (Eq. 1-4), fine branch (Eq. 12) and merge (Eq. 14).
  *   gate: fp32 [batch, heads_q, L] (the caller's tanh(X W_g), Eq. 13); NULL means gate = 0.

@@ -20,8 +20,9 @@ BF16, F32 = 0, 1
 FLAG_NO_COARSE = 1
 FLAG_EXACT_MAX_FWD = 2
 FLAG_FAST_BWD = 4
+FLAG_PRECISE_BWD = 8
 FLAG_BF16_COARSE_FWD = 64
-FLAG_HALF_CUBE_FWD = 128
+FLAG_PAIR_QUERY_FWD = 128
 FLAG_GROUP_ROUTING = 256
 
 OK = 0
@@ -53,7 +54,7 @@ class Params(C.Structure):
                 ("cube_t", C.c_int32), ("cube_h", C.c_int32), ("cube_w", C.c_int32),
                 ("rpool_t", C.c_int32), ("rpool_h", C.c_int32), ("rpool_w", C.c_int32),
                 ("select_mode", C.c_int32), ("topk", C.c_int32), ("keep_fraction", C.c_float),
-                ("softmax_scale", C.c_float), ("out_dtype", C.c_int32), ("flags", C.c_int32),
+                ("softmax_scale", C.c_float), ("out_dtype", C.c_int32), ("flags", C.c_int32), ("text_len", C.c_int32),
                 ("nnz_cap", C.c_int64)]
 
 
@@ -63,7 +64,8 @@ class Sizes(C.Structure):
                 ("ptr_elems", C.c_int64), ("idx_elems", C.c_int64), ("pooled_q_elems", C.c_int64),
                 ("pooled_kv_elems", C.c_int64), ("lse_c_elems", C.c_int64), ("o_res_elems", C.c_int64),
                 ("route_workspace_bytes", C.c_size_t), ("fwd_workspace_bytes", C.c_size_t),
-                ("bwd_workspace_bytes", C.c_size_t)]
+                ("bwd_workspace_bytes", C.c_size_t), ("tokens_per_head", C.c_int64), ("text_blocks", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class Map(C.Structure):
@@ -145,14 +147,15 @@ def _check(code, where):
 
 def make_params(batch, heads_q, heads_kv, head_dim, grid, cube=(4, 4, 4), rpool=(2, 2, 2),
                 select_mode=PER_SEQUENCE, topk=0, keep_fraction=0.0, softmax_scale=0.0, out_dtype=BF16,
-                flags=0, nnz_cap=0) -> Params:
+                flags=0, nnz_cap=0, text_len=0) -> Params:
     return Params(batch, heads_q, heads_kv, head_dim, *grid, *cube, *rpool, select_mode, topk, keep_fraction,
-                  softmax_scale, out_dtype, flags, nnz_cap)
+                  softmax_scale, out_dtype, flags, text_len, nnz_cap)
 
 
 def params_from_workload(wl, **overrides) -> Params:
     kw = dict(batch=wl.batch, heads_q=wl.heads_q, heads_kv=wl.heads_kv, head_dim=wl.head_dim, grid=wl.grid,
-              cube=wl.cube, rpool=wl.rpool, select_mode=wl.select_mode, topk=wl.topk)
+              cube=wl.cube, rpool=wl.rpool, select_mode=wl.select_mode, topk=wl.topk,
+              text_len=getattr(wl, "text_len", 0))
     kw.update(overrides)
     return make_params(**kw)
 
@@ -318,8 +321,8 @@ class Vsa2Attention:
             dk = torch.empty(k.shape, dtype=self.out_torch_dtype, device=q.device)
         if dv is None:
             dv = torch.empty(v.shape, dtype=self.out_torch_dtype, device=q.device)
-        if dgate is None:
-            dgate = torch.empty(q.shape[:-1], dtype=torch.float32, device=q.device)
+        if dgate is None:      # video tokens only (text tokens have no gate)
+            dgate = torch.empty(q.shape[:-2] + (self.sizes.seq_len,), dtype=torch.float32, device=q.device)
         vsa2_attn_bwd(p, q, k, v, gate, self.map, o, lse, self.saved, d_o, dq, dk, dv, dgate, self.ws_bwd, stream=stream)
         return dq, dk, dv, dgate
 

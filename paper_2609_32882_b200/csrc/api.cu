@@ -39,7 +39,7 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   if (p->heads_q % p->heads_kv) return VSA2_ERR_INVALID_ARG;
   if (p->select_mode < VSA2_PER_SEQUENCE || p->select_mode > VSA2_PER_QUERY_BUDGET) return VSA2_ERR_INVALID_ARG;
   if (p->out_dtype != VSA2_BF16 && p->out_dtype != VSA2_F32) return VSA2_ERR_INVALID_ARG;
-  if (p->topk < 0 || p->nnz_cap < 0 || !(p->softmax_scale >= 0.f)) return VSA2_ERR_INVALID_ARG;
+  if (p->topk < 0 || p->nnz_cap < 0 || !(p->softmax_scale >= 0.f) || p->text_len < 0) return VSA2_ERR_INVALID_ARG;
   if (p->cube_t % p->rpool_t || p->cube_h % p->rpool_h || p->cube_w % p->rpool_w) return VSA2_ERR_INVALID_ARG;
   if (p->head_dim != 64 && p->head_dim != 128) return VSA2_ERR_UNSUPPORTED;
   // 64-token cubes, or 128-token cubes that split along w into two 64-token halves the router pooling respects
@@ -47,15 +47,19 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   const bool wide = cube_tokens == 2 * kBlockTokens;
   if (cube_tokens != kBlockTokens && !wide) return VSA2_ERR_UNSUPPORTED;
   if (wide && (p->cube_w % 2 || (p->cube_w / 2) % p->rpool_w)) return VSA2_ERR_UNSUPPORTED;
+  if (wide && p->text_len > 0) return VSA2_ERR_UNSUPPORTED;
   if (p->batch > 65535 || p->heads_q > 65535 || p->heads_q / p->heads_kv > 16) return VSA2_ERR_UNSUPPORTED;
   g->batch = p->batch; g->Hq = p->heads_q; g->Hkv = p->heads_kv; g->rep = p->heads_q / p->heads_kv; g->D = p->head_dim;
   g->T = p->grid_t; g->H = p->grid_h; g->W = p->grid_w;
   long long L = (long long)g->T * g->H * g->W;
-  if (L > 0x7fffffffLL / 128) return VSA2_ERR_UNSUPPORTED;
+  if (L + p->text_len > 0x7fffffffLL / 128) return VSA2_ERR_UNSUPPORTED;
   g->L = (int)L;
+  g->Lt = p->text_len;
+  g->S = (int)L + p->text_len;
   g->Bt = p->cube_t; g->Bh = p->cube_h; g->Bw = p->cube_w;
   g->Nt = (g->T + g->Bt - 1) / g->Bt; g->Nh = (g->H + g->Bh - 1) / g->Bh; g->Nw = (g->W + g->Bw - 1) / g->Bw;
   g->N = g->Nt * g->Nh * g->Nw;
+  g->Nvid = g->N;
   g->Rt = p->rpool_t; g->Rh = p->rpool_h; g->Rw = p->rpool_w;
   g->Gt = g->Bt / g->Rt; g->Gh = g->Bh / g->Rh; g->Gw = g->Bw / g->Rw;
   g->G = g->Gt * g->Gh * g->Gw;
@@ -80,6 +84,35 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   else if (p->select_mode == VSA2_PER_QUERY_BUDGET) return VSA2_ERR_INVALID_ARG;
   else g->nnz_cap = (long long)g->N * K;
   return VSA2_OK;
+}
+
+// Block problem of the fine kernels with text tokens: the N video cubes followed by ceil(Lt / 64) text blocks; its maps
+// are the video maps with the text blocks appended to every row and one dense row per text block.
+int text_blocks(const Geo& g) { return (g.Lt + kBlockTokens - 1) / kBlockTokens; }
+Geo text_geo(const Geo& g) {
+  Geo x = g;
+  const int tb = text_blocks(g);
+  x.N = g.Nvid + tb;
+  x.nnz_cap = g.nnz_cap + (long long)g.Nvid * tb + (long long)tb * x.N;
+  return x;
+}
+struct TextMapLayout {
+  size_t ptr, idx, cptr, ridx, total;     // offsets behind the call's other workspace regions
+};
+TextMapLayout text_map_layout(const Geo& g, bool with_csc) {
+  TextMapLayout r = {};
+  if (g.Lt == 0) return r;
+  const Geo x = text_geo(g);
+  Carver c;
+  const size_t BHq = (size_t)g.batch * g.Hq;
+  r.ptr = c.take(BHq * (x.N + 1) * sizeof(int));
+  r.idx = c.take(BHq * (size_t)x.nnz_cap * sizeof(int));
+  if (with_csc) {
+    r.cptr = c.take(BHq * (x.N + 1) * sizeof(int));
+    r.ridx = c.take(BHq * (size_t)x.nnz_cap * sizeof(int));
+  }
+  r.total = c.off;
+  return r;
 }
 
 RouteLayout route_layout(const Geo& g) {
@@ -110,7 +143,7 @@ BwdLayout bwd_layout(const Geo& g) {
   Carver c;
   const size_t BHq = (size_t)g.batch * g.Hq;
   r.status = c.take(sizeof(StatusBlock));
-  r.delta = c.take(BHq * g.L * sizeof(float));
+  r.delta = c.take(BHq * g.S * sizeof(float));
   r.d_oc_hat = c.take(BHq * g.N * g.D * sizeof(float));
   r.delta_c = c.take(BHq * g.N * sizeof(float));
   r.dqc = c.take(BHq * g.N * g.D * sizeof(float));
@@ -180,10 +213,12 @@ WideBwdLayout wide_bwd_layout(const Geo& g) {
 }
 
 size_t route_workspace_bytes(const Geo& g) { return wide_cube(g) ? wide_route_layout(g).total : route_layout(g).total; }
-size_t fwd_workspace_bytes(const Geo& g) {
-  return wide_cube(g) ? wide_fwd_layout(g).total : fwd_pooled_offset() + pooled_layout(g, false).total;
+size_t fwd_base_bytes(const Geo& g) {
+  return wide_cube(g) ? wide_fwd_layout(g).total : align_up(fwd_pooled_offset() + pooled_layout(g, false).total, 256);
 }
-size_t bwd_workspace_bytes(const Geo& g) { return wide_cube(g) ? wide_bwd_layout(g).total : bwd_layout(g).total; }
+size_t bwd_base_bytes(const Geo& g) { return wide_cube(g) ? wide_bwd_layout(g).total : align_up(bwd_layout(g).total, 256); }
+size_t fwd_workspace_bytes(const Geo& g) { return fwd_base_bytes(g) + text_map_layout(g, false).total; }
+size_t bwd_workspace_bytes(const Geo& g) { return bwd_base_bytes(g) + text_map_layout(g, true).total; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -258,7 +293,9 @@ int vsa2_query_sizes(const vsa2_params* p, vsa2_sizes* out) {
   out->pooled_q_elems = BHq * g.N * g.D;
   out->pooled_kv_elems = BHk * g.N * g.D;
   out->lse_c_elems = BHq * g.N;
-  out->o_res_elems = g.out_f32 ? 0 : BHq * (long long)g.L * g.D;
+  out->o_res_elems = g.out_f32 ? 0 : BHq * (long long)g.S * g.D;
+  out->tokens_per_head = g.S;
+  out->text_blocks = text_blocks(g);
   out->route_workspace_bytes = route_workspace_bytes(g);
   out->fwd_workspace_bytes = fwd_workspace_bytes(g);
   out->bwd_workspace_bytes = bwd_workspace_bytes(g);
@@ -411,16 +448,29 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     col_idx = at<int>(workspace, wl.idx64);
   }
   bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<bf16*>(saved->o_res) : nullptr;
+  Geo fx = n;                                   // geometry of the fine kernels' block problem
+  if (g.Lt > 0) {
+    // text tokens: append the text blocks to the map (in the workspace) and run the kernels on the block problem
+    const TextMapLayout tl = text_map_layout(g, false);
+    unsigned char* tbase = at<unsigned char>(workspace, fwd_base_bytes(g));
+    fx = text_geo(g);
+    if (!fine_fwd_rows_supported(fx)) return VSA2_ERR_UNSUPPORTED;
+    g_launches += 1;
+    VSA2_CUDA(launch_extend_map(g, text_blocks(g), map->row_ptr, map->col_idx, at<int>(tbase, tl.ptr), at<int>(tbase, tl.idx),
+                                fx.nnz_cap, st));
+    row_ptr = at<int>(tbase, tl.ptr);
+    col_idx = at<int>(tbase, tl.idx);
+  }
   {
     ProfScope ps(VSA2_KERNEL_FINE_FWD, st, (g.flags & VSA2_FLAG_EXACT_MAX_FWD) ? 1 : 2);
     if (g.flags & VSA2_FLAG_EXACT_MAX_FWD)
-      VSA2_CUDA(launch_fine_fwd(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse, st));
-    else if (!(g.flags & VSA2_FLAG_HALF_CUBE_FWD) && (wide || ((g.flags & VSA2_FLAG_GROUP_ROUTING) && g.rep % 2 == 0)))
+      VSA2_CUDA(launch_fine_fwd(fx, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse, st));
+    else if (g.Lt == 0 && (g.flags & VSA2_FLAG_PAIR_QUERY_FWD) && (wide || ((g.flags & VSA2_FLAG_GROUP_ROUTING) && g.rep % 2 == 0)))
       // 128 query columns per tile: the halves of a 128-token cube, or two heads of a group that share their map
       VSA2_CUDA(launch_fine_fwd_wide_tc(n, !wide, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                         reinterpret_cast<StatusBlock*>(workspace), st));
-    else if (fine_fwd_rows_supported(n) && !(g.flags & 512))
-      VSA2_CUDA(launch_fine_fwd_rows_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
+    else if (fine_fwd_rows_supported(fx) && !(g.flags & 512))
+      VSA2_CUDA(launch_fine_fwd_rows_tc(fx, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                         reinterpret_cast<StatusBlock*>(workspace), st));
     else
       VSA2_CUDA(launch_fine_fwd_tc(n, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
@@ -489,12 +539,27 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
       oc_hat = at<float>(workspace, wl.oc_hat64);
     }
   }
+  Geo fx = n;                                   // geometry of the fine kernels' block problem
+  if (g.Lt > 0) {
+    const TextMapLayout tl = text_map_layout(g, true);
+    unsigned char* tbase = at<unsigned char>(workspace, bwd_base_bytes(g));
+    fx = text_geo(g);
+    g_launches += 2;
+    VSA2_CUDA(launch_extend_map(g, text_blocks(g), map->row_ptr, map->col_idx, at<int>(tbase, tl.ptr), at<int>(tbase, tl.idx),
+                                fx.nnz_cap, st));
+    VSA2_CUDA(launch_extend_map(g, text_blocks(g), map->col_ptr, map->row_idx, at<int>(tbase, tl.cptr), at<int>(tbase, tl.ridx),
+                                fx.nnz_cap, st));
+    row_ptr = at<int>(tbase, tl.ptr);
+    col_idx = at<int>(tbase, tl.idx);
+    col_ptr = at<int>(tbase, tl.cptr);
+    row_idx = at<int>(tbase, tl.ridx);
+  }
   if (!coarse && dgate != nullptr)
     VSA2_CUDA(cudaMemsetAsync(dgate, 0, (size_t)g.batch * g.Hq * g.L * sizeof(float), st));
   const bf16* o_res = (saved != nullptr && !g.out_f32) ? reinterpret_cast<const bf16*>(saved->o_res) : nullptr;
   {
     ProfScope ps(VSA2_KERNEL_BWD_PRE, st, 1);
-    VSA2_CUDA(launch_bwd_preprocess(n, dob, o, o_res, coarse ? gate : nullptr, oc_hat, delta, coarse ? dgate : nullptr,
+    VSA2_CUDA(launch_bwd_preprocess(fx, dob, o, o_res, coarse ? gate : nullptr, oc_hat, delta, coarse ? dgate : nullptr,
                                     d_oc_hat, st));
   }
   if (coarse) {
@@ -512,12 +577,12 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
-    VSA2_CUDA(launch_fine_bwd_dq_tc(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
+    VSA2_CUDA(launch_fine_bwd_dq_tc(fx, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
                                     reinterpret_cast<StatusBlock*>(workspace), st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
-    VSA2_CUDA(launch_fine_bwd_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
+    VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                      coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;

@@ -24,20 +24,19 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restr
   __shared__ float ocs[D];
   const int i = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const size_t bhq = (size_t)b * g.Hq + hq;
-  const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr;
+  // text blocks (i >= Nvid) take no part in the coarse branch or the gate: only delta is formed for them
+  const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr && !block_is_text(g, i);
   const int r = threadIdx.x >> 2, qd = threadIdx.x & 3;
   constexpr int NCH = D / 32;          // 16-byte chunks (8 channels) per thread
-  int nt, nh, nw;
-  cube_coords(g, i, nt, nh, nw);
-  const int l = cube_token(g, nt, nh, nw, r);
+  const int l = block_token(g, i, r);
   if (coarse)
-    for (int d = threadIdx.x; d < D; d += blockDim.x) ocs[d] = oc_hat[(bhq * g.N + i) * D + d];
+    for (int d = threadIdx.x; d < D; d += blockDim.x) ocs[d] = oc_hat[(bhq * g.Nvid + i) * D + d];
   float s_oo = 0.f, s_oc = 0.f;
   const float gt = (coarse && l >= 0) ? gate[bhq * g.L + l] : 0.f;
   uint4 dv[NCH], ob[NCH], rb[NCH];
   float4 of[NCH][2];
   if (l >= 0) {
-    const size_t base = (bhq * g.L + l) * D;
+    const size_t base = (bhq * g.S + l) * D;
 #pragma unroll
     for (int k = 0; k < NCH; ++k) {
       const int d0 = (4 * k + qd) * 8;
@@ -102,8 +101,8 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restr
   s_oc += __shfl_xor_sync(0xffffffffu, s_oc, 1);
   s_oc += __shfl_xor_sync(0xffffffffu, s_oc, 2);
   if (qd == 0 && l >= 0) {
-    delta[bhq * g.L + l] = s_oo - gt * s_oc;     // rowsum(dO * (O - gate*O_c)) = rowsum(dO * O_f)
-    if (dgate != nullptr) dgate[bhq * g.L + l] = s_oc;
+    delta[bhq * g.S + l] = s_oo - gt * s_oc;     // rowsum(dO * (O - gate*O_c)) = rowsum(dO * O_f)
+    if (dgate != nullptr && coarse) dgate[bhq * g.L + l] = s_oc;
   }
   if (coarse) {
     __syncthreads();
@@ -120,7 +119,7 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(const bf16* __restr
       float tot = 0.f;
 #pragma unroll
       for (int q = 0; q < PARTS; ++q) tot += gdo[q * LD + threadIdx.x];
-      d_oc_hat[(bhq * g.N + i) * D + threadIdx.x] = tot;
+      d_oc_hat[(bhq * g.Nvid + i) * D + threadIdx.x] = tot;
     }
   }
 }

@@ -25,6 +25,11 @@ struct Geo {
   int flags;
   float scale;      // softmax scale
   long long nnz_cap;
+  // Text tokens (the sentence after Eq. 12): every token tensor holds S = L + Lt rows per head, the L video tokens in raster
+  // order followed by Lt text tokens.  The routing and coarse kernels see the video part only (N = Nvid cubes).  The fine
+  // kernels and the backward preprocess run on the BLOCK problem: N = Nvid + ceil(Lt / 64) blocks, block j < Nvid is video
+  // cube j, block j >= Nvid holds text tokens 64 (j - Nvid) .. ; their maps are the block maps extended by the text blocks.
+  int Nvid, Lt, S;
 };
 
 // Status block at the start of every workspace.
@@ -101,6 +106,40 @@ __device__ __forceinline__ int subcube_count(const Geo& g, int n, int gsub) {
   return ct * ch * cw;
 }
 
+// ---- blocks of the fine kernels: video cubes followed by text blocks ---------------------------------------------------
+__device__ __forceinline__ bool block_is_text(const Geo& g, int j) { return j >= g.Nvid; }
+// TMA box coordinates (dimensions 1..3 of the 5-D maps) of block j: a video cube in the raster map, or 64 rows of the text map
+__device__ __forceinline__ void block_box(const Geo& g, int j, int& c1, int& c2, int& c3) {
+  if (j < g.Nvid) {
+    int jt, jh, jw;
+    cube_coords(g, j, jt, jh, jw);
+    c1 = jw * g.Bw; c2 = jh * g.Bh; c3 = jt * g.Bt;
+  } else {
+    c1 = (j - g.Nvid) * kBlockTokens; c2 = 0; c3 = 0;
+  }
+}
+// position p of block j -> row of the token tensors (0 .. S-1), or -1 if padding
+__device__ __forceinline__ int block_token(const Geo& g, int j, int p) {
+  if (j < g.Nvid) {
+    int jt, jh, jw;
+    cube_coords(g, j, jt, jh, jw);
+    return cube_token(g, jt, jh, jw, p);
+  }
+  const int t = (j - g.Nvid) * kBlockTokens + p;
+  return t < g.Lt ? g.L + t : -1;
+}
+// valid tokens of block j
+__device__ __forceinline__ int block_count(const Geo& g, int j) {
+  if (j < g.Nvid) return cube_count(g, j);
+  return min(kBlockTokens, g.Lt - (j - g.Nvid) * kBlockTokens);
+}
+// work item -> (batch * heads index, block).  Blocks are handed out in descending order inside a head, so that the text
+// blocks (whose lists are the longest by far) start first and the persistent CTAs do not end on them.
+__device__ __forceinline__ void item_block(const Geo& g, int item, int& bh, int& i) {
+  bh = item / g.N;
+  i = g.N - 1 - (item - bh * g.N);
+}
+
 __device__ __forceinline__ void store_out(void* base, size_t idx, float v, int out_f32) {
   if (out_f32) reinterpret_cast<float*>(base)[idx] = v;
   else reinterpret_cast<bf16*>(base)[idx] = __float2bfloat16_rn(v);
@@ -170,6 +209,10 @@ cudaError_t launch_fold_sum(const Geo& narrow, int heads, const float* x64, floa
 cudaError_t launch_expand_rows(const Geo& narrow, int heads, bool by_count, const float* x, float* x64,
                                cudaStream_t st);
 cudaError_t launch_expand_map(const Geo& narrow, const int* ptr, const int* idx, int* ptr64, int* idx64,
+                              cudaStream_t st);
+// block map of the video cubes (g: the video problem) -> block map with `text_blocks` text blocks appended to every row and
+// all-ones text rows; capx = capacity per (batch, head) of idxx
+cudaError_t launch_extend_map(const Geo& g, int text_blocks, const int* ptr, const int* idx, int* ptrx, int* idxx, long long capx,
                               cudaStream_t st);
 
 // gate projection and its backward (gate.cu)

@@ -100,7 +100,7 @@ __device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
 }
 
 // One warp streams pairs of cube tiles into a ring of NS slots: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one
-// box each (half h = lane / 2 of block lane & 1).  `coord_*`: cube coordinates of this lane's block, `bh`: its head.
+// box each (half h = lane / 2 of block lane & 1).  C3, C2, C1: box coordinates of this lane's block in map TMAP, `bh`: its head.
 // `LANE0_PRE`: statement lane 0 runs once the slot is free, before the loads are armed (may use slot_).
 #define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH, LANE0_PRE, WAITFN)                  \
   do {                                                                                                            \
@@ -116,7 +116,7 @@ __device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
     if (!__shfl_sync(0xffffffffu, ok_, 0)) goto done;                                                             \
     if (lane < 2 * C::DH)                                                                                         \
       tc::tma_load_5d((RING_BASE) + slot_ * C::SLOT + (2 * (lane >> 1) + (lane & 1)) * kSlab, (TMAP), &(FULL)[slot_], \
-                      (lane >> 1) * 64, (CW) * g.Bw, (CH) * g.Bh, (CT) * g.Bt, (BH));                             \
+                      (lane >> 1) * 64, (CW), (CH), (CT), (BH));                                                  \
   } while (0)
 
 // ================================================================================================
@@ -143,7 +143,9 @@ struct DqArgs {
 template <int D, bool SPLIT>
 __global__ void __launch_bounds__(kDqThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, Geo g,
+                      const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                      const __grid_constant__ CUtensorMap tm_qt, const __grid_constant__ CUtensorMap tm_kt,
+                      const __grid_constant__ CUtensorMap tm_vt, const __grid_constant__ CUtensorMap tm_dot, Geo g,
                       DqArgs a) {
   using C = BwdTc<D>;
   extern __shared__ unsigned char smem_raw[];
@@ -180,6 +182,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     // ------------------------------------------------------------------ TMA producers
     const int which = warp;                               // 0: K pairs (ring A) + Q, dO tiles; 1: V pairs (ring B)
     const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+    const CUtensorMap* tm_text = which == 0 ? &tm_kt : &tm_vt;
     const int my_blk = lane & 1;
     uint32_t tg = 0, n_items = 0, published = 0;
     for (uint32_t seq = 0;; ++seq) {
@@ -192,15 +195,17 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       item = __shfl_sync(0xffffffffu, item, 0);
       if (item == -2) goto done;
       if (item < 0) break;
-      const int i = item % g.N, bhq = item / g.N;
+      int i, bhq;
+      item_block(g, item, bhq, i);
       const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
       if (k == 0) continue;
       const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
       if (which == 0) {
-        int it_, ih_, iw_;
-        cube_coords(g, i, it_, ih_, iw_);
+        int c1, c2, c3;
+        block_box(g, i, c1, c2, c3);
+        const bool qtext = block_is_text(g, i);
         int ok = 1;
         if (lane == 0) {
           ok = tc::mbar_wait(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
@@ -209,23 +214,25 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
         if (lane < 2 * C::DH) {
           const int h = lane >> 1;
-          if (lane & 1) tc::tma_load_5d(do_tile + h * kSlab, &tm_do, &misc->st_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
-          else tc::tma_load_5d(q_tile + h * kSlab, &tm_q, &misc->st_full, h * 64, iw_ * g.Bw, ih_ * g.Bh, it_ * g.Bt, bhq);
+          if (lane & 1) tc::tma_load_5d(do_tile + h * kSlab, qtext ? &tm_dot : &tm_do, &misc->st_full, h * 64, c1, c2, c3, bhq);
+          else tc::tma_load_5d(q_tile + h * kSlab, qtext ? &tm_qt : &tm_q, &misc->st_full, h * 64, c1, c2, c3, bhq);
         }
       }
       ++n_items;
       const int nt = (k + 1) >> 1;
       int j = cols[(my_blk == 1 && k > 1) ? 1 : 0];
       for (int t = 0; t < nt; ++t, ++tg) {
-        int jt, jh, jw;
-        cube_coords(g, j, jt, jh, jw);
+        int c1, c2, c3;
+        block_box(g, j, c1, c2, c3);
+        const CUtensorMap* tm_j = block_is_text(g, j) ? tm_text : tm;
+        const unsigned ef0 = block_edge_flags(g, j);
         if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];
         if (which == 0) {
-          const unsigned ef0 = cube_edge_flags_at(g, jt, jh, jw), ef1 = __shfl_sync(0xffffffffu, ef0, 1);
-          VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm, tg, jt, jh, jw, bhk,
+          const unsigned ef1 = __shfl_sync(0xffffffffu, ef0, 1);
+          VSA2_RING_LOAD(misc->a_full, misc->a_empty, kRingA, smem, tm_j, tg, c3, c2, c1, bhk,
                          { misc->edge[slot_][0] = (unsigned char)ef0; misc->edge[slot_][1] = (unsigned char)ef1; }, mbar_wait);
         } else {
-          VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, jt, jh, jw, bhk, {}, mbar_wait);
+          VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm_j, tg, c3, c2, c1, bhk, {}, mbar_wait);
         }
       }
     }
@@ -239,7 +246,8 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       uint32_t tg = 0, n_items = 0;
       for (uint32_t seq = 0;; ++seq) {
         VSA2_NEXT_ITEM_WARP(item, seq);
-        const int i = item % g.N, bhq = item / g.N;
+        int i, bhq;
+        item_block(g, item, bhq, i);
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
@@ -279,7 +287,8 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       uint32_t tg = 0, n_items = 0;
       for (uint32_t seq = 0;; ++seq) {
         VSA2_NEXT_ITEM_WARP(item, seq);
-        const int i = item % g.N, bhq = item / g.N;
+        int i, bhq;
+        item_block(g, item, bhq, i);
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
@@ -314,21 +323,20 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     uint32_t tg = 0, n_items = 0;
     for (uint32_t n_all = 0;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
-      const int i = item % g.N, bhq = item / g.N;
+      int i, bhq;
+      item_block(g, item, bhq, i);
       const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
       const int k = end - beg;
       const int tb = n_all & 1;
       const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
       if (sm_tid < 64) {
-        int it_, ih_, iw_;
-        cube_coords(g, i, it_, ih_, iw_);
-        const int l = cube_token(g, it_, ih_, iw_, sm_tid);
+        const int l = block_token(g, i, sm_tid);
         misc->tok[tb][sm_tid] = l;
-        misc->stats[tb * 64 + sm_tid] = l >= 0 ? a.lse[(size_t)bhq * g.L + l] * 1.4426950408889634f : INFINITY;
-        misc->stats[128 + tb * 64 + sm_tid] = l >= 0 ? a.delta[(size_t)bhq * g.L + l] : 0.f;
+        misc->stats[tb * 64 + sm_tid] = l >= 0 ? a.lse[(size_t)bhq * g.S + l] * 1.4426950408889634f : INFINITY;
+        misc->stats[128 + tb * 64 + sm_tid] = l >= 0 ? a.delta[(size_t)bhq * g.S + l] : 0.f;
       }
-      const float coarse_d = (a.dqc != nullptr && row < D)
-                                 ? a.dqc[((size_t)bhq * g.N + i) * D + row] / (float)cube_count(g, i) : 0.f;
+      const float coarse_d = (a.dqc != nullptr && row < D && !block_is_text(g, i))
+                                 ? a.dqc[((size_t)bhq * g.Nvid + i) * D + row] / (float)cube_count(g, i) : 0.f;
       VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0);
       if (k > 0) {
         const int nt = (k + 1) >> 1;
@@ -428,7 +436,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int c = 0; c < 32; ++c) {
               const int l = misc->tok[tb][half * 32 + c];
               if (l < 0) continue;
-              store_out(a.dq, ((size_t)bhq * g.L + l) * D + row, __uint_as_float(o0[c]) + coarse_d, 1);
+              store_out(a.dq, ((size_t)bhq * g.S + l) * D + row, __uint_as_float(o0[c]) + coarse_d, 1);
             }
           }
         } else {
@@ -445,7 +453,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const int qi = e / CH, ch = e % CH;
             const int l = misc->tok[tb][qi];
             if (l < 0) continue;
-            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dq) + ((size_t)bhq * g.L + l) * D + ch * 8) =
+            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dq) + ((size_t)bhq * g.S + l) * D + ch * 8) =
                 *reinterpret_cast<const uint4*>(st + qi * D + ch * 8);
           }
           VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 2);
@@ -512,7 +520,9 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b,
 template <int D, bool SPLIT>
 __global__ void __launch_bounds__(kDkvThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, Geo g,
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                       const __grid_constant__ CUtensorMap tm_qt, const __grid_constant__ CUtensorMap tm_kt,
+                       const __grid_constant__ CUtensorMap tm_vt, const __grid_constant__ CUtensorMap tm_dot, Geo g,
                        DkvArgs a) {
   constexpr int RA = SPLIT ? 2 : kRingA;                   // slots of the Q ring
   constexpr uint32_t TM_DK = 256, TM_DV = SPLIT ? 384 : 320;
@@ -552,7 +562,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
   // per item: prefix of the per-head column counts and the list starts (every role recomputes them)
 #define VSA2_DKV_ITEM_SETUP()                                                            \
-  const int j = item % g.N, bhk = item / g.N;                                            \
+  int j, bhk;                                                                            \
+  item_block(g, item, bhk, j);                                                           \
   const int b = bhk / g.Hkv, hk = bhk % g.Hkv;                                           \
   int cnt_prefix[kMaxRep + 1], col_beg[kMaxRep];                                         \
   cnt_prefix[0] = 0;                                                                     \
@@ -567,6 +578,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // ------------------------------------------------------------------ TMA producers
     const int which = warp;                               // 0: Q pairs (ring A) + K, V tiles; 1: dO pairs (ring B)
     const CUtensorMap* tm = which == 0 ? &tm_q : &tm_do;
+    const CUtensorMap* tm_text = which == 0 ? &tm_qt : &tm_dot;
     const int my_blk = lane & 1;
     uint32_t tg = 0, n_items = 0, published = 0;
     for (uint32_t seq = 0;; ++seq) {
@@ -582,8 +594,9 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       VSA2_DKV_ITEM_SETUP();
       if (k == 0) continue;
       if (which == 0) {
-        int jt, jh, jw;
-        cube_coords(g, j, jt, jh, jw);
+        int c1, c2, c3;
+        block_box(g, j, c1, c2, c3);
+        const bool ktext = block_is_text(g, j);
         int ok = 1;
         if (lane == 0) {
           ok = tc::mbar_wait_parked(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
@@ -592,8 +605,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
         if (lane < 2 * C::DH) {
           const int h = lane >> 1;
-          if (lane & 1) tc::tma_load_5d(v_tile + h * kSlab, &tm_v, &misc->st_full, h * 64, jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
-          else tc::tma_load_5d(k_tile + h * kSlab, &tm_k, &misc->st_full, h * 64, jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
+          if (lane & 1) tc::tma_load_5d(v_tile + h * kSlab, ktext ? &tm_vt : &tm_v, &misc->st_full, h * 64, c1, c2, c3, bhk);
+          else tc::tma_load_5d(k_tile + h * kSlab, ktext ? &tm_kt : &tm_k, &misc->st_full, h * 64, c1, c2, c3, bhk);
         }
       }
       ++n_items;
@@ -601,12 +614,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       int bhq_l, i_l;           // this lane's entry of the tile, fetched one tile ahead of the slot wait
       dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && k > 1) ? 1 : 0, bhq_l, i_l);
       for (int t = 0; t < nt; ++t, ++tg) {
-        int it_, ih_, iw_;
-        cube_coords(g, i_l, it_, ih_, iw_);
+        int c1, c2, c3;
+        block_box(g, i_l, c1, c2, c3);
+        const CUtensorMap* tm_i = block_is_text(g, i_l) ? tm_text : tm;
         const int bhq_t = bhq_l;
         if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
-        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, RA, smem, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
-        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm, tg, it_, ih_, iw_, bhq_t, {}, mbar_wait_parked);
+        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, RA, smem, tm_i, tg, c3, c2, c1, bhq_t, {}, mbar_wait_parked);
+        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm_i, tg, c3, c2, c1, bhq_t, {}, mbar_wait_parked);
       }
     }
   } else if (warp == 2 || warp == 3) {
@@ -700,8 +714,6 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // ------------------------------------------------------------------ row statistics of the tiles (128 threads)
     const int r = tid - 384;                 // query row of the tile
     const int blk = r >> 6;
-    CubePos cpos;
-    cpos.init(g, r & 63);
     float2* rowstat = reinterpret_cast<float2*>(misc->stats);
     uint32_t tg = 0;
     for (uint32_t seq = 0;; ++seq) {
@@ -713,11 +725,9 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       int bhq_n, i_n;
       dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
       for (int t = 0; t < nt; ++t, ++tg) {
-        int it_, ih_, iw_;
-        cube_coords(g, i_n, it_, ih_, iw_);
         const bool dup = (blk == 1) && (2 * t + 1 >= k);
-        const int l = dup ? -1 : cube_token_at(g, it_, ih_, iw_, cpos.bt, cpos.bh, cpos.bw);
-        const size_t idx = l >= 0 ? (size_t)bhq_n * g.L + l : 0;
+        const int l = dup ? -1 : block_token(g, i_n, r & 63);
+        const size_t idx = l >= 0 ? (size_t)bhq_n * g.S + l : 0;
         const float lse_raw = a.lse[idx], dlt_raw = a.delta[idx];
         if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
         VSA2_WAIT_PARKED(&misc->stat_free, (tg & 1) ^ 1);
@@ -740,19 +750,17 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       (void)col_beg;
       const int tb = n_all & 1;
       const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
-      int jt, jh, jw;
-      cube_coords(g, j, jt, jh, jw);
-      if (sm_tid < 64) misc->tok[tb][sm_tid] = cube_token(g, jt, jh, jw, sm_tid);
+      if (sm_tid < 64) misc->tok[tb][sm_tid] = block_token(g, j, sm_tid);
       uint32_t kvmask = 0xffffffffu;           // validity of this thread's 32 key columns
-      if (k > 0 && cube_edge_flags(g, j) != 0) {
+      if (k > 0 && block_count(g, j) < kBlockTokens) {
         kvmask = 0u;
         for (int p = 0; p < 32; ++p)
-          if (cube_token(g, jt, jh, jw, half * 32 + p) >= 0) kvmask |= 1u << p;
+          if (block_token(g, j, half * 32 + p) >= 0) kvmask |= 1u << p;
       }
       float coarse_k = 0.f, coarse_v = 0.f;
-      if (a.dkc != nullptr && row < D) {
+      if (a.dkc != nullptr && row < D && !block_is_text(g, j)) {
         for (int hh = 0; hh < g.rep; ++hh) {
-          const size_t cidx = ((size_t)(b * g.Hq + hk * g.rep + hh) * g.N + j) * D + row;
+          const size_t cidx = ((size_t)(b * g.Hq + hk * g.rep + hh) * g.Nvid + j) * D + row;
           coarse_k += a.dkc[cidx];
           coarse_v += a.dvc[cidx];
         }
@@ -867,7 +875,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int c = 0; c < 32; ++c) {
               const int l = misc->tok[tb][half * 32 + c];
               if (l < 0) continue;
-              const size_t idx = ((size_t)bhk * g.L + l) * D + row;
+              const size_t idx = ((size_t)bhk * g.S + l) * D + row;
               store_out(a.dk, idx, __uint_as_float(kk[c]) + coarse_k, 1);
               store_out(a.dv, idx, __uint_as_float(vv[c]) + coarse_v, 1);
             }
@@ -889,7 +897,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const int c = e / CH, ch = e % CH;
             const int l = misc->tok[tb][c];
             if (l < 0) continue;
-            const size_t idx = ((size_t)bhk * g.L + l) * D + ch * 8;
+            const size_t idx = ((size_t)bhk * g.S + l) * D + ch * 8;
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dk) + idx) = *reinterpret_cast<const uint4*>(st_k + c * D + ch * 8);
             *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dv) + idx) = *reinterpret_cast<const uint4*>(st_v + c * D + ch * 8);
           }
@@ -928,9 +936,10 @@ static cudaError_t sm_count(int* sms) {
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                   const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
                                   const float* dqc, void* dq, StatusBlock* status, cudaStream_t st) {
-  CUtensorMap tq, tk, tv, tdo;
+  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
-      !make_cube_tmap(&tdo, d_o, g, g.Hq))
+      !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) ||
+      !make_text_tmap(&tvt, v, g, g.Hkv) || !make_text_tmap(&tdot, d_o, g, g.Hq))
     return cudaErrorInvalidValue;
   int sms = 0;
   cudaError_t e;
@@ -944,7 +953,7 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
     if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                    \
                                   (int)BwdTc<DD>::smem_bytes)))                                                                  \
       return e;                                                                                                                  \
-    fine_bwd_dq_tc_kernel<DD, SP><<<grid, kDqThreads, BwdTc<DD>::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);                       \
+    fine_bwd_dq_tc_kernel<DD, SP><<<grid, kDqThreads, BwdTc<DD>::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                       \
   } while (0)
   if (g.D == 128) {
     if (split) VSA2_LAUNCH_DQ(128, true);
@@ -962,9 +971,10 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
                                    cudaStream_t st) {
   if (g.rep > kMaxRep) return cudaErrorInvalidValue;
-  CUtensorMap tq, tk, tv, tdo;
+  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
-      !make_cube_tmap(&tdo, d_o, g, g.Hq))
+      !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) ||
+      !make_text_tmap(&tvt, v, g, g.Hkv) || !make_text_tmap(&tdot, d_o, g, g.Hq))
     return cudaErrorInvalidValue;
   int sms = 0;
   cudaError_t e;
@@ -972,14 +982,15 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   DkvArgs a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
-  const bool split = !(g.flags & VSA2_FLAG_FAST_BWD);
+  // a KV block of a GQA group sums rep times as many query blocks: there the plain bf16 rounding of P and dS passes 2e-2
+  const bool split = (g.flags & VSA2_FLAG_PRECISE_BWD) || (g.rep > 1 && !(g.flags & VSA2_FLAG_FAST_BWD));
 #define VSA2_LAUNCH_DKV(DD, SP)                                                                                                  \
   do {                                                                                                                           \
     using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
     if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                   \
                                   (int)L_::smem_bytes)))                                                                         \
       return e;                                                                                                                  \
-    fine_bwd_dkv_tc_kernel<DD, SP><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, g, a);                            \
+    fine_bwd_dkv_tc_kernel<DD, SP><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                            \
   } while (0)
   if (g.D == 128) {
     if (split) VSA2_LAUNCH_DKV(128, true);

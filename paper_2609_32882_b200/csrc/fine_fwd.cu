@@ -39,9 +39,9 @@ __device__ __forceinline__ void fine_fwd_block(unsigned char* smem_raw, int i, i
 
   const int hk = hq / g.rep;
   const size_t bhq = (size_t)b * g.Hq + hq, bhk = (size_t)b * g.Hkv + hk;
-  const bf16* qh = q + bhq * g.L * D;
-  const bf16* kh = k + bhk * g.L * D;
-  const bf16* vh = v + bhk * g.L * D;
+  const bf16* qh = q + bhq * g.S * D;
+  const bf16* kh = k + bhk * g.S * D;
+  const bf16* vh = v + bhk * g.S * D;
   const int* cols = col_idx + bhq * g.nnz_cap;
   const int beg = row_ptr[bhq * (g.N + 1) + i], end = row_ptr[bhq * (g.N + 1) + i + 1];
 
@@ -56,11 +56,7 @@ __device__ __forceinline__ void fine_fwd_block(unsigned char* smem_raw, int i, i
     __syncthreads();
     load_cube_tile<D>(Ks, SM::LDX, kh, g, j);
     load_cube_tile<D>(Vs, SM::LDX, vh, g, j);
-    if (threadIdx.x < 64) {
-      int nt, nh, nw;
-      cube_coords(g, j, nt, nh, nw);
-      kvalid[threadIdx.x] = cube_token(g, nt, nh, nw, threadIdx.x) >= 0;
-    }
+    if (threadIdx.x < 64) kvalid[threadIdx.x] = block_token(g, j, threadIdx.x) >= 0;
     __syncthreads();
     tile_gemm<64, 64, D, false, true, false>(Qs, SM::LDX, Ks, SM::LDX, S, SM::LDS);
     __syncthreads();
@@ -100,16 +96,14 @@ __device__ __forceinline__ void fine_fwd_block(unsigned char* smem_raw, int i, i
   }
   __syncthreads();
   // epilogue: normalise, merge with the coarse branch, write valid tokens only
-  int nt, nh, nw;
-  cube_coords(g, i, nt, nh, nw);
-  const int l = cube_token(g, nt, nh, nw, r);
+  const int l = block_token(g, i, r);
   if (l >= 0) {
     const float denom = row_l[r];
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
-    const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr;
+    const bool coarse = !(g.flags & VSA2_FLAG_NO_COARSE) && gate != nullptr && !block_is_text(g, i);
     const float gt = coarse ? gate[bhq * g.L + l] : 0.f;
-    const float* oc = oc_hat + (bhq * g.N + i) * D;
-    const size_t obase = (bhq * g.L + l) * D;
+    const float* oc = oc_hat + (bhq * g.Nvid + i) * D;
+    const size_t obase = (bhq * g.S + l) * D;
     for (int c = 0; c < OC; ++c) {
       int d = qd * OC + c;
       float val = O[r * SM::LDO + d] * inv;
@@ -121,7 +115,7 @@ __device__ __forceinline__ void fine_fwd_block(unsigned char* smem_raw, int i, i
         o_res[obase + d] = __float2bfloat16_rn(val - rounded);
       }
     }
-    if (qd == 0) lse[bhq * g.L + l] = denom > 0.f ? row_m[r] + __logf(denom) : -INFINITY;
+    if (qd == 0) lse[bhq * g.S + l] = denom > 0.f ? row_m[r] + __logf(denom) : -INFINITY;
   }
 }
 
@@ -150,7 +144,8 @@ __global__ void __launch_bounds__(256) fine_fwd_list_kernel(const int* __restric
   const int n = min(*count, cap);
   for (int e = blockIdx.x; e < n; e += gridDim.x) {
     int item = items[e];
-    int i = item % g.N, bh = item / g.N;
+    int i, bh;
+    item_block(g, item, bh, i);
     __syncthreads();
     fine_fwd_block<D>(smem_raw, i, bh % g.Hq, bh / g.Hq, q, k, v, gate, row_ptr, col_idx, oc_hat, g, o, o_res, lse);
   }

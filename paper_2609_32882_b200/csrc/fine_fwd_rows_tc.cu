@@ -96,7 +96,9 @@ struct FwdRowsArgs {
 template <int D>
 __global__ void __launch_bounds__(kFrThreads, 1)
 fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                        const __grid_constant__ CUtensorMap tm_v, Geo g, FwdRowsArgs a) {
+                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_qt,
+                        const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt, Geo g,
+                        FwdRowsArgs a) {
   using C = FwdRows<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -108,7 +110,7 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   const int total_items = g.batch * g.Hq * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
 
-  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)cube_edge_flags(g, n);
+  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)block_edge_flags(g, n);
   if (tid < 64) {
     // validity of key columns 8n + 2c + e (n = 0..7, e = 0, 1) of a 64-token block with edge flags f, for lane % 4 == c
     const unsigned f = tid >> 2, c = tid & 3;
@@ -151,6 +153,11 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     tc::prefetch_tmap(&tm_q);
     tc::prefetch_tmap(&tm_k);
     tc::prefetch_tmap(&tm_v);
+    if (g.Lt > 0) {
+      tc::prefetch_tmap(&tm_qt);
+      tc::prefetch_tmap(&tm_kt);
+      tc::prefetch_tmap(&tm_vt);
+    }
   }
   if (warp == 4) {
     tc::tmem_alloc(&misc->tmem_base, 512);
@@ -170,6 +177,7 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       const int which = warp & 1;                           // 0: K ring (+ Q tile), 1: V ring
       const int my_blk = warp >> 1;                         // 0: first block of the pair, 1: second
       const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+      const CUtensorMap* tm_text = which == 0 ? &tm_kt : &tm_vt;
       const uint32_t nslots = which == 0 ? kFrKSlots : kFrVSlots;
       uint64_t* full = which == 0 ? misc->k_full : misc->v_full;
       uint64_t* empty = which == 0 ? misc->k_empty : misc->v_empty;
@@ -187,15 +195,16 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         item = __shfl_sync(0xffffffffu, item, 0);
         if (item == -2) goto done;
         if (item < 0) break;
-        const int i = item % g.N, bhq = item / g.N;
+        int i, bhq;
+        item_block(g, item, bhq, i);
         const int b = bhq / g.Hq, hq = bhq % g.Hq, bhk = b * g.Hkv + hq / g.rep;
         const int beg = a.row_ptr[(size_t)bhq * (g.N + 1) + i], end = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1];
         const int k = end - beg;
         if (k == 0) continue;
         const int* cols = a.col_idx + (size_t)bhq * g.nnz_cap + beg;
         if (warp == 0) {
-          int it_, ih_, iw_;
-          cube_coords(g, i, it_, ih_, iw_);
+          int c1, c2, c3;
+          block_box(g, i, c1, c2, c3);
           int ok = 1;
           const uint32_t qb = n_items % C::NQ;
           if (lane == 0) {
@@ -204,15 +213,16 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           }
           if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
           if (lane < C::DH)
-            tc::tma_load_5d(q_tile + qb * C::QBYTES + lane * kSlab, &tm_q, &misc->q_full[qb], lane * 64, iw_ * g.Bw, ih_ * g.Bh,
-                            it_ * g.Bt, bhq);
+            tc::tma_load_5d(q_tile + qb * C::QBYTES + lane * kSlab, block_is_text(g, i) ? &tm_qt : &tm_q, &misc->q_full[qb],
+                            lane * 64, c1, c2, c3, bhq);
         }
         ++n_items;
         const int nt = (k + 1) >> 1;
         int j = cols[(my_blk == 1 && k > 1) ? 1 : 0];           // this warp's KV block of tile 0
         for (int t = 0; t < nt; ++t, ++tg) {
-          int jt, jh, jw;
-          cube_coords(g, j, jt, jh, jw);
+          int c1, c2, c3;
+          block_box(g, j, c1, c2, c3);
+          const CUtensorMap* tm_j = block_is_text(g, j) ? tm_text : tm;
           if (t + 1 < nt) j = cols[(my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2];   // next tile, fetched early
           const uint32_t slot = tg % nslots, par = (tg / nslots) & 1;
           int ok = 1;
@@ -222,8 +232,7 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           }
           if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
           if (issuer)
-            tc::tma_load_5d(ring + slot * C::SLOT + (2 * my_h + my_blk) * kSlab, tm, &full[slot], my_h * 64,
-                            jw * g.Bw, jh * g.Bh, jt * g.Bt, bhk);
+            tc::tma_load_5d(ring + slot * C::SLOT + (2 * my_h + my_blk) * kSlab, tm_j, &full[slot], my_h * 64, c1, c2, c3, bhk);
         }
       }
     } else if (warp == 4) {
@@ -239,7 +248,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         item = __shfl_sync(0xffffffffu, item, 0);
         if (item == -2) goto done;
         if (item < 0) break;
-        const int i = item % g.N, bhq = item / g.N;
+        int i, bhq;
+        item_block(g, item, bhq, i);
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
@@ -283,7 +293,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         item = __shfl_sync(0xffffffffu, item, 0);
         if (item == -2) goto done;
         if (item < 0) break;
-        const int i = item % g.N, bhq = item / g.N;
+        int i, bhq;
+        item_block(g, item, bhq, i);
         const int k = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - a.row_ptr[(size_t)bhq * (g.N + 1) + i];
         if (k == 0) continue;
         const int nt = (k + 1) >> 1;
@@ -322,22 +333,22 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         item = __shfl_sync(0xffffffffu, item, 0);
         if (item == -2) goto done;
         if (item < 0) break;
-        const int i = item % g.N, bhq = item / g.N;
+        int i, bhq;
+        item_block(g, item, bhq, i);
         const uint32_t tb = seq & 1;
-        int it_, ih_, iw_;
-        cube_coords(g, i, it_, ih_, iw_);
+        const bool video = !block_is_text(g, i);      // text queries take no part in the coarse branch or the gate
         const int beg_ = a.row_ptr[(size_t)bhq * (g.N + 1) + i], k_ = a.row_ptr[(size_t)bhq * (g.N + 1) + i + 1] - beg_;
         const int head_ = (lane < 4 && lane < k_) ? a.col_idx[(size_t)bhq * g.nnz_cap + beg_ + lane] : 0;
         int l2[2];
         float g2[2], oc4[4];
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-          l2[r] = cube_token(g, it_, ih_, iw_, lane + 32 * r);
-          g2[r] = (coarse && l2[r] >= 0) ? a.gate[(size_t)bhq * g.L + l2[r]] : 0.f;
+          l2[r] = block_token(g, i, lane + 32 * r);
+          g2[r] = (coarse && video && l2[r] >= 0) ? a.gate[(size_t)bhq * g.L + l2[r]] : 0.f;
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r)
-          oc4[r] = (coarse && lane + 32 * r < D) ? a.oc_hat[((size_t)bhq * g.N + i) * D + lane + 32 * r] : 0.f;
+          oc4[r] = (coarse && video && lane + 32 * r < D) ? a.oc_hat[((size_t)bhq * g.Nvid + i) * D + lane + 32 * r] : 0.f;
         VSA2_WAIT_PARKED(&misc->tab_free[tb], ((seq >> 1) & 1) ^ 1);
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -364,10 +375,23 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const int sm_tid = tid & 127;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     constexpr int COLS = D / 2;                  // output columns per warpgroup in the epilogue
+    // which of this thread's 16 key columns of a block with edge flags f hold tokens
+    auto kv_mask = [&](unsigned f) -> unsigned {
+      if (!(f & kTextBlockFlag)) return misc->vmask[f][cq];
+      const int cnt = (int)(f & 0x7fu) + 1;
+      if (cnt == kBlockTokens) return 0xffffu;
+      unsigned m = 0;
+      for (int n = 0; n < 8; ++n) {
+        if (8 * n + 2 * cq < cnt) m |= 1u << (2 * n);
+        if (8 * n + 2 * cq + 1 < cnt) m |= 2u << (2 * n);
+      }
+      return m;
+    };
     uint32_t tg = 0, n_items = 0, all_phase = 0;
     for (uint32_t n_all = 0;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
-      const int i = item % g.N, bhq = item / g.N;
+      int i, bhq;
+      item_block(g, item, bhq, i);
       const int tb = n_all & 1;
       VSA2_WAIT(&misc->tab_full[tb], (n_all >> 1) & 1);  // the item's tables (loaded one item ahead by warp 6)
       const int k = misc->list_k[tb];
@@ -390,8 +414,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         tc::tc_fence_before();
         tc::mbar_arrive(&misc->s_free[buf]);
         have_first = true;
-        const unsigned ma = misc->vmask[edge[head[0]]][cq];
-        const unsigned mb = k > 1 ? misc->vmask[edge[head[1]]][cq] : 0u;
+        const unsigned ma = kv_mask(edge[head[0]]);
+        const unsigned mb = k > 1 ? kv_mask(edge[head[1]]) : 0u;
         float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
         for (int n = 0; n < 16; ++n) {
@@ -421,8 +445,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         for (int t = t_first; t < nt; t += 2) {
           const uint32_t tgt = tg0 + t, buf = tgt & 1;
           const bool dup = 2 * t + 1 >= k;
-          const unsigned ma = misc->vmask[edge[ja]][cq];
-          const unsigned mb = dup ? 0u : misc->vmask[edge[jb]][cq];
+          const unsigned ma = kv_mask(edge[ja]);
+          const unsigned mb = dup ? 0u : kv_mask(edge[jb]);
           if (t + 2 < nt) {
             ja = cols[2 * t + 4];
             jb = cols[2 * t + 5 < k ? 2 * t + 5 : 2 * t + 4];
@@ -510,15 +534,15 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           // sums outside the safe range (overflow, NaN or total underflow): hand the block to the exact kernel
           if (!(la > 1e-30f && la < 1e30f && ra > 1e-30f) || !(lb > 1e-30f && lb < 1e30f && rb > 1e-30f)) misc->rescue_flag = 1;
           const int ta = misc->tok[tb][row_a], tk_b = misc->tok[tb][row_b];
-          if (ta >= 0) a.lse[(size_t)bhq * g.L + ta] = (m_a + __log2f(la)) * 0.6931471805599453f;
-          if (tk_b >= 0) a.lse[(size_t)bhq * g.L + tk_b] = (m_b + __log2f(lb)) * 0.6931471805599453f;
+          if (ta >= 0) a.lse[(size_t)bhq * g.S + ta] = (m_a + __log2f(la)) * 0.6931471805599453f;
+          if (tk_b >= 0) a.lse[(size_t)bhq * g.S + tk_b] = (m_b + __log2f(lb)) * 0.6931471805599453f;
         }
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
       } else if (wg == 0 && cq == 0) {
         const int ta = misc->tok[tb][row_a], tk_b = misc->tok[tb][row_b];
-        if (ta >= 0) a.lse[(size_t)bhq * g.L + ta] = -INFINITY;
-        if (tk_b >= 0) a.lse[(size_t)bhq * g.L + tk_b] = -INFINITY;
+        if (ta >= 0) a.lse[(size_t)bhq * g.S + ta] = -INFINITY;
+        if (tk_b >= 0) a.lse[(size_t)bhq * g.S + tk_b] = -INFINITY;
       }
 
       // O[l, d] = O_acc[q, d] / (rounded row sum) + gate[q] * O_c[d]; this warpgroup owns COLS output columns
@@ -543,10 +567,10 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             const int col = wg * COLS + 8 * n + 2 * cq;
             const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[tb][col]);
             if (ta >= 0)
-              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.L + ta) * D + col) =
+              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.S + ta) * D + col) =
                   make_float2(fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a));
             if (tk_b >= 0)
-              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.L + tk_b) * D + col) =
+              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.S + tk_b) * D + col) =
                   make_float2(fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b));
           }
         } else {
@@ -563,12 +587,12 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             split_bf16x2(v0, v1, ha, la2);
             split_bf16x2(v2, v3, hb, lb2);
             if (ta >= 0) {
-              const size_t idx = ((size_t)bhq * g.L + ta) * D + col;
+              const size_t idx = ((size_t)bhq * g.S + ta) * D + col;
               *reinterpret_cast<uint32_t*>(ob + idx) = ha;
               if (a.o_res != nullptr) *reinterpret_cast<uint32_t*>(a.o_res + idx) = la2;
             }
             if (tk_b >= 0) {
-              const size_t idx = ((size_t)bhq * g.L + tk_b) * D + col;
+              const size_t idx = ((size_t)bhq * g.S + tk_b) * D + col;
               *reinterpret_cast<uint32_t*>(ob + idx) = hb;
               if (a.o_res != nullptr) *reinterpret_cast<uint32_t*>(a.o_res + idx) = lb2;
             }
@@ -617,8 +641,9 @@ extern "C" int vsa2_debug_fwd_trace(long long* host_out) {
 cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,
                                     const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                     float* lse, StatusBlock* status, cudaStream_t st) {
-  CUtensorMap tq, tk, tv;
-  if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv))
+  CUtensorMap tq, tk, tv, tqt, tkt, tvt;
+  if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
+      !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) || !make_text_tmap(&tvt, v, g, g.Hkv))
     return cudaErrorInvalidValue;
   int dev = 0, sms = 0;
   cudaError_t e;
@@ -644,11 +669,11 @@ cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, 
   if (g.D == 128) {
     const size_t smb = FwdRows<128>::smem_bytes(g.N);
     if ((e = cudaFuncSetAttribute(fine_fwd_rows_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    fine_fwd_rows_tc_kernel<128><<<grid, kFrThreads, smb, st>>>(tq, tk, tv, g, a);
+    fine_fwd_rows_tc_kernel<128><<<grid, kFrThreads, smb, st>>>(tq, tk, tv, tqt, tkt, tvt, g, a);
   } else {
     const size_t smb = FwdRows<64>::smem_bytes(g.N);
     if ((e = cudaFuncSetAttribute(fine_fwd_rows_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smb))) return e;
-    fine_fwd_rows_tc_kernel<64><<<grid, kFrThreads, smb, st>>>(tq, tk, tv, g, a);
+    fine_fwd_rows_tc_kernel<64><<<grid, kFrThreads, smb, st>>>(tq, tk, tv, tqt, tkt, tvt, g, a);
   }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // query blocks whose row sums left the safe range are redone with the exact running maximum

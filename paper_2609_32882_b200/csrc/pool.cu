@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(256) pool_kernel(const bf16* __restrict__ x, i
   __shared__ float tile[kBlockTokens][D];
   const int n = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const size_t bh = (size_t)b * heads + h;
-  const bf16* base = x + bh * (size_t)g.L * D;
+  const bf16* base = x + bh * (size_t)g.S * D;
   int nt, nh, nw;
   cube_coords(g, n, nt, nh, nw);
   constexpr int CH = D / 8;
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(256) permute_kernel(const bf16* __restrict__ s
   for (int c = threadIdx.x; c < B * CH; c += blockDim.x) {
     const int p = c / CH, ch = c % CH;
     const int l = cube_token(g, nt, nh, nw, p);
-    const size_t raster = (bh * g.L + (size_t)max(l, 0)) * D + ch * 8;
+    const size_t raster = (bh * g.S + (size_t)max(l, 0)) * D + ch * 8;
     const size_t cubed = ((bh * g.N + n) * B + p) * (size_t)D + ch * 8;
     if (!inverse) {
       uint4 v = make_uint4(0, 0, 0, 0);

@@ -82,6 +82,12 @@ __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, u
   lo = pack_bf16x2(x0 - h0, x1 - h1);
 }
 
+__device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
 // Which cubes are cut by the grid boundary: bit 0 / 1 / 2 = last cube along t / h / w with a partial extent.
 // In the half-cube grid of a 128-token-cube problem the last column of blocks along w may lie outside the grid
 // altogether (extent <= 0, still bit 2); the column before it can then be the partial one (bit 3).
@@ -97,11 +103,19 @@ __device__ __forceinline__ unsigned cube_edge_flags(const Geo& g, int n) {
   cube_coords(g, n, nt, nh, nw);
   return cube_edge_flags_at(g, nt, nh, nw);
 }
+// The same for a block of the fine kernels: a text block carries bit 7 and, in its low bits, its number of tokens - 1.
+constexpr unsigned kTextBlockFlag = 0x80u;
+__device__ __forceinline__ unsigned block_edge_flags(const Geo& g, int j) {
+  if (j < g.Nvid) return cube_edge_flags(g, j);
+  return kTextBlockFlag | (unsigned)(block_count(g, j) - 1);
+}
 
 // Position of a token inside its cube and the test "is this position inside the valid grid for a cube with edge flags f".
 struct CubePos {
   int bt, bh, bw, lt, lh, lw;   // coordinates of the position; valid extents of the last cube along each axis
-  __device__ __forceinline__ void init(const Geo& g, int pos) {
+  int pos;                      // the position itself (text blocks: row of the block)
+  __device__ __forceinline__ void init(const Geo& g, int pos_) {
+    pos = pos_;
     bw = pos % g.Bw;
     int r = pos / g.Bw;
     bh = r % g.Bh;
@@ -111,6 +125,7 @@ struct CubePos {
     lw = g.W - (g.Nw - 1) * g.Bw;
   }
   __device__ __forceinline__ bool valid(unsigned f, const Geo& g) const {
+    if (f & kTextBlockFlag) return pos <= (int)(f & 0x7fu);
     return (!(f & 1u) || bt < lt) && (!(f & 2u) || bh < lh) && (!(f & 4u) || bw < lw) && (!(f & 8u) || bw < lw + g.Bw);
   }
 };

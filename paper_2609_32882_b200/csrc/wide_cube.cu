@@ -25,6 +25,7 @@ Geo narrow_geo(const Geo& g) {
   n.Bw = g.Bw / 2;
   n.Nw = g.Nw * 2;
   n.N = g.N * 2;
+  n.Nvid = n.N;
   n.Gw = n.Bw / n.Rw;
   n.G = n.Gt * n.Gh * n.Gw;
   n.nnz_cap = g.nnz_cap * 4;
@@ -124,6 +125,36 @@ __global__ void __launch_bounds__(128) expand_map_kernel(int N, int Hq, long lon
   }
 }
 
+// Block map of the video cubes -> block map of the block problem with text tokens (Sec. 2.2, the sentence after Eq. 12): every
+// video row (or column) additionally keeps all NtB text blocks, and every text row (column) keeps all Nvid + NtB blocks.
+// ptr [BH, Nvid+1], idx [BH, cap] -> ptrx [BH, Nx+1], idxx [BH, capx] with Nx = Nvid + NtB, capx = cap + Nvid NtB + NtB Nx.
+// The same rule serves the CSR and the CSC map (the extension is symmetric).
+__global__ void __launch_bounds__(128) extend_map_kernel(int Nvid, int NtB, int Hq, long long cap, long long capx,
+                                                         const int* __restrict__ ptr, const int* __restrict__ idx,
+                                                         int* __restrict__ ptrx, int* __restrict__ idxx) {
+  const int r = blockIdx.x, Nx = Nvid + NtB;
+  const size_t bh = (size_t)blockIdx.z * Hq + blockIdx.y;
+  const int* p = ptr + bh * (Nvid + 1);
+  int* px = ptrx + bh * (Nx + 1);
+  int* dst = idxx + bh * capx;
+  if (r < Nvid) {
+    const int beg = (int)min((long long)p[r], cap), end = (int)min((long long)p[r + 1], cap), len = end - beg;
+    const int start = beg + r * NtB;
+    if (threadIdx.x == 0) px[r] = start;
+    const int* src = idx + bh * cap + beg;
+    for (int e = threadIdx.x; e < len; e += blockDim.x) dst[start + e] = src[e];
+    for (int e = threadIdx.x; e < NtB; e += blockDim.x) dst[start + len + e] = Nvid + e;
+  } else {
+    const int t = r - Nvid;
+    const int start = (int)min((long long)p[Nvid], cap) + Nvid * NtB + t * Nx;
+    if (threadIdx.x == 0) {
+      px[r] = start;
+      if (r == Nx - 1) px[Nx] = start + Nx;
+    }
+    for (int e = threadIdx.x; e < Nx; e += blockDim.x) dst[start + e] = e;
+  }
+}
+
 // "group head" routing: the query heads of a KV group share one map.  pr [batch, Hq, N, N]: every entry is replaced by
 // the sum over the heads of its group (added in head order), so the selection that follows picks the same set for each
 __global__ void __launch_bounds__(256) group_sum_scores_kernel(float* __restrict__ pr, int rep, size_t per_head, size_t groups) {
@@ -180,6 +211,13 @@ cudaError_t launch_expand_map(const Geo& narrow, const int* ptr, const int* idx,
                               cudaStream_t st) {
   dim3 grid(narrow.N / 2, narrow.Hq, narrow.batch);
   expand_map_kernel<<<grid, 128, 0, st>>>(narrow.N / 2, narrow.Hq, narrow.nnz_cap / 4, ptr, idx, ptr64, idx64);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_extend_map(const Geo& g, int text_blocks, const int* ptr, const int* idx, int* ptrx, int* idxx, long long capx,
+                              cudaStream_t st) {
+  dim3 grid(g.Nvid + text_blocks, g.Hq, g.batch);
+  extend_map_kernel<<<grid, 128, 0, st>>>(g.Nvid, text_blocks, g.Hq, g.nnz_cap, capx, ptr, idx, ptrx, idxx);
   return cudaGetLastError();
 }
 

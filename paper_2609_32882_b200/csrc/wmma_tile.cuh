@@ -55,16 +55,14 @@ __device__ __forceinline__ void tile_gemm(const bf16* A, int lda, const bf16* B,
   }
 }
 
-// Loads the 64 x D bf16 tile of cube n of one head (raster layout in global memory) into shared
+// Loads the 64 x D bf16 tile of block n of one head (a video cube of the raster layout, or a text block) into shared
 // memory [64][ld]; padding positions are zero-filled.
 template <int D>
 __device__ __forceinline__ void load_cube_tile(bf16* dst, int ld, const bf16* head_base, const Geo& g, int n) {
-  int nt, nh, nw;
-  cube_coords(g, n, nt, nh, nw);
   constexpr int CH = D / 8;
   for (int c = threadIdx.x; c < kBlockTokens * CH; c += blockDim.x) {
     int p = c / CH, ch = c % CH;
-    int l = cube_token(g, nt, nh, nw, p);
+    int l = block_token(g, n, p);
     uint4 v = make_uint4(0, 0, 0, 0);
     if (l >= 0) v = __ldg(reinterpret_cast<const uint4*>(head_base + (size_t)l * D + ch * 8));
     *reinterpret_cast<uint4*>(dst + (size_t)p * ld + ch * 8) = v;

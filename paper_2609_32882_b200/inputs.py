@@ -44,6 +44,7 @@ class Workload:
     kind: str = "locality"
     seed: int = 0
     gate_const: float | None = None
+    text_len: int = 0    # text tokens appended to every head's token rows (MMDiT joint attention)
 
     @property
     def L(self):
@@ -83,7 +84,16 @@ def _rng(seed, name, b, h):
 
 
 def head_tensor(wl: Workload, name: str, b: int, h: int) -> np.ndarray:
-    """One head of q, k, v or do as bf16 bit patterns, shape [L, D]."""
+    """One head of q, k, v or do as bf16 bit patterns, shape [L + text_len, D]: the video tokens in raster order, then the
+    text tokens (i.i.d. N(0,1): text embeddings carry no spatial structure)."""
+    x = _head_video(wl, name, b, h)
+    if wl.text_len:
+        rng = np.random.default_rng([int(wl.seed), _TENSOR_ID[name], int(b), int(h), 7])
+        x = np.concatenate([x, f32_to_bf16_bits(rng.standard_normal((wl.text_len, wl.head_dim), dtype=np.float32))])
+    return x
+
+
+def _head_video(wl: Workload, name: str, b: int, h: int) -> np.ndarray:
     rng = _rng(wl.seed, name, b, h)
     t, hh, w = wl.grid
     d = wl.head_dim

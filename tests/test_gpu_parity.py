@@ -17,10 +17,10 @@ MINI_COARSE = syn.Workload("mini_two_coarse_tiles", 1, 2, 1, 128, (8, 24, 28), s
 MINI_BUDGET = syn.Workload("mini_budget", 1, 2, 1, 128, (8, 8, 12), select_mode=syn.PER_QUERY_BUDGET, seed=23)
 
 
-def full_parity(wl, data, out_dtype=vb.BF16, nnz_cap=0, check_route=True):
+def full_parity(wl, data, out_dtype=vb.BF16, nnz_cap=0, check_route=True, flags=0):
     geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
     scale = 1.0 / np.sqrt(wl.head_dim)
-    run = CudaPath(wl, data, out_dtype=out_dtype, nnz_cap=nnz_cap)
+    run = CudaPath(wl, data, out_dtype=out_dtype, nnz_cap=nnz_cap, flags=flags)
     a = oracle_arrays(data)
     gmask = run.route()
     if check_route:
@@ -220,13 +220,14 @@ def test_rescue_list_overflow_is_reported_and_stays_inside_the_list():
         n_over = int(words[2])
         assert n_over >= 3                                                 # at least the three aimed blocks were counted
         assert 0 <= words[64] < geo.N                                      # one was listed and redone
+        redone = geo.N - 1 - int(words[64])                                # (items count the blocks of a head downwards)
         assert (words[65:65 + 4096] == 0x5A5A5A5A).all()                   # nothing written behind the capacity
         O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], np.zeros_like(a["gate"]), gmask, geo, 1 / np.sqrt(128))
         O = to_f64(o)
         # blocks whose scores stay small never left the safe range; the listed one was redone: those must be right
         calm = [i for i in range(geo.N) if lse_ref[0, 0, geo.cube_tokens[i]].max() < 40]
         assert len(calm) >= geo.N - n_over
-        fine = np.concatenate([geo.cube_tokens[i] for i in calm] + [geo.cube_tokens[int(words[64])]])
+        fine = np.concatenate([geo.cube_tokens[i] for i in calm] + [geo.cube_tokens[redone]])
         assert np.abs(O[0, 0, fine] - O_ref[0, 0, fine]).max() <= TOL_ABS
     finally:
         assert vb._lib().vsa2_debug_rescue_capacity(16384) == 16384
@@ -306,6 +307,12 @@ def test_group_shared_routing(wl):
     want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
     for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
         assert_close(name, x, y, bf16_storage=name != "dGate")
+    # the same maps through the 128-query forward, which stacks pairs of heads (or the halves of a 128-token cube)
+    pair = CudaPath(wl, data, flags=vb.FLAG_GROUP_ROUTING | vb.FLAG_PAIR_QUERY_FWD)
+    assert np.array_equal(pair.route(), gmask)
+    O2, lse2 = pair.forward()
+    assert_close("O (128-query forward)", O2, O_ref, bf16_storage=True)
+    assert_lse_close(lse2, lse_ref)
 
 
 def test_group_shared_routing_is_refused_for_per_row_budgets():
