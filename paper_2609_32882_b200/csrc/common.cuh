@@ -133,12 +133,14 @@ __device__ __forceinline__ int block_count(const Geo& g, int j) {
   if (j < g.Nvid) return cube_count(g, j);
   return min(kBlockTokens, g.Lt - (j - g.Nvid) * kBlockTokens);
 }
-// work item -> (batch * heads index, block).  Blocks are handed out in descending order inside a head, so that the text
-// blocks (whose lists are the longest by far) start first and the persistent CTAs do not end on them.
+// work item -> (batch * heads index, block).  With text tokens the blocks of a head are handed out in descending order, so
+// that the text blocks (whose lists are the longest by far) start first and the persistent CTAs do not end on them.
 __device__ __forceinline__ void item_block(const Geo& g, int item, int& bh, int& i) {
   bh = item / g.N;
-  i = g.N - 1 - (item - bh * g.N);
+  const int r = item - bh * g.N;
+  i = g.Lt > 0 ? g.N - 1 - r : r;
 }
+__device__ __forceinline__ int block_item(const Geo& g, int bh, int i) { return bh * g.N + (g.Lt > 0 ? g.N - 1 - i : i); }
 
 __device__ __forceinline__ void store_out(void* base, size_t idx, float v, int out_f32) {
   if (out_f32) reinterpret_cast<float*>(base)[idx] = v;

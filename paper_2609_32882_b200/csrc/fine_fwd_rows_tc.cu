@@ -60,7 +60,7 @@ struct FwdRowsMisc {
   uint32_t tmem_base;
   int abort_flag;
   int rescue_flag;
-  unsigned short vmask[16][4];     // [edge flags][lane % 4]: which of a thread's 16 key columns of a block are valid tokens
+  unsigned short vmask[17][4];     // [table row of the block][lane % 4]: which of a thread's 16 key columns are valid tokens
   alignas(16) float m_ref[64];     // per query row: reference exponent (log2 units)
   float red[2][2][64];             // [warpgroup][exact sum | sum of the bf16 roundings][query row]
   alignas(16) float oc[2][128];    // coarse output row of the query cube, by item parity
@@ -110,16 +110,22 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   const int total_items = g.batch * g.Hq * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
 
-  for (int n = tid; n < g.N; n += blockDim.x) edge[n] = (unsigned char)block_edge_flags(g, n);
-  if (tid < 64) {
-    // validity of key columns 8n + 2c + e (n = 0..7, e = 0, 1) of a 64-token block with edge flags f, for lane % 4 == c
+  // per block: the row of the validity table below -- the edge flags of a video cube (0 = nothing cut), 0 for a full text
+  // block, 16 for the ragged last text block
+  for (int n = tid; n < g.N; n += blockDim.x)
+    edge[n] = (unsigned char)(n < g.Nvid ? cube_edge_flags(g, n) : (block_count(g, n) == kBlockTokens ? 0 : 16));
+  if (tid < 68) {
+    // validity of key columns 8n + 2c + e (n = 0..7, e = 0, 1) of a 64-token block, for lane % 4 == c: rows 0..15 by the
+    // edge flags of a video cube, row 16 for the last text block when it holds fewer than 64 tokens
     const unsigned f = tid >> 2, c = tid & 3;
+    const int text_tail = g.Lt % kBlockTokens;
     unsigned m = 0;
     for (int n = 0; n < 8; ++n)
       for (int e = 0; e < 2; ++e) {
+        const int pos = 8 * n + 2 * (int)c + e;
         CubePos cp;
-        cp.init(g, 8 * n + 2 * (int)c + e);
-        if (cp.valid(f, g)) m |= 1u << (2 * n + e);
+        cp.init(g, pos);
+        if (f < 16 ? cp.valid(f, g) : pos < text_tail) m |= 1u << (2 * n + e);
       }
     misc->vmask[f][c] = (unsigned short)m;
   }
@@ -375,18 +381,6 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const int sm_tid = tid & 127;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     constexpr int COLS = D / 2;                  // output columns per warpgroup in the epilogue
-    // which of this thread's 16 key columns of a block with edge flags f hold tokens
-    auto kv_mask = [&](unsigned f) -> unsigned {
-      if (!(f & kTextBlockFlag)) return misc->vmask[f][cq];
-      const int cnt = (int)(f & 0x7fu) + 1;
-      if (cnt == kBlockTokens) return 0xffffu;
-      unsigned m = 0;
-      for (int n = 0; n < 8; ++n) {
-        if (8 * n + 2 * cq < cnt) m |= 1u << (2 * n);
-        if (8 * n + 2 * cq + 1 < cnt) m |= 2u << (2 * n);
-      }
-      return m;
-    };
     uint32_t tg = 0, n_items = 0, all_phase = 0;
     for (uint32_t n_all = 0;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
@@ -414,8 +408,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         tc::tc_fence_before();
         tc::mbar_arrive(&misc->s_free[buf]);
         have_first = true;
-        const unsigned ma = kv_mask(edge[head[0]]);
-        const unsigned mb = k > 1 ? kv_mask(edge[head[1]]) : 0u;
+        const unsigned ma = misc->vmask[edge[head[0]]][cq];
+        const unsigned mb = k > 1 ? misc->vmask[edge[head[1]]][cq] : 0u;
         float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
         for (int n = 0; n < 16; ++n) {
@@ -445,8 +439,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         for (int t = t_first; t < nt; t += 2) {
           const uint32_t tgt = tg0 + t, buf = tgt & 1;
           const bool dup = 2 * t + 1 >= k;
-          const unsigned ma = kv_mask(edge[ja]);
-          const unsigned mb = dup ? 0u : kv_mask(edge[jb]);
+          const unsigned ma = misc->vmask[edge[ja]][cq];
+          const unsigned mb = dup ? 0u : misc->vmask[edge[jb]][cq];
           if (t + 2 < nt) {
             ja = cols[2 * t + 4];
             jb = cols[2 * t + 5 < k ? 2 * t + 5 : 2 * t + 4];

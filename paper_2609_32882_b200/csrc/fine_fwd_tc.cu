@@ -495,7 +495,7 @@ fine_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         a.lse[(size_t)bhq * g.L + misc->tok[tb][sm_tid]] = -INFINITY;
       if (k > 0 && wg == 0 && sm_tid == 0 && misc->rescue_flag) {
         int slot = atomicAdd(a.rescue_count, 1);
-        if (slot < a.rescue_cap) a.rescue_items[slot] = bhq * g.N + (g.N - 1 - i);   // the list kernel's item numbering
+        if (slot < a.rescue_cap) a.rescue_items[slot] = block_item(g, bhq, i);   // the list kernel's item numbering
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
       }
       if (k > 0) ++n_items;

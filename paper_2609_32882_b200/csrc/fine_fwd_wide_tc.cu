@@ -483,7 +483,7 @@ fine_fwd_wide_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         a.lse[(size_t)bhq * g.L + misc->tok[tb][q0 + sm_tid]] = -INFINITY;
       if (nt > 0 && sm_tid == 0 && misc->rescue_flag[wg]) {
         int slot = atomicAdd(a.rescue_count, 1);
-        if (slot < a.rescue_cap) a.rescue_items[slot] = bhq * g.N + (g.N - 1 - i);      // half-cube item in the list kernel's numbering
+        if (slot < a.rescue_cap) a.rescue_items[slot] = block_item(g, bhq, i);      // half-cube item in the list kernel's numbering
         else atomicExch(&a.status->status, VSA2_ERR_UNSUPPORTED);
       }
       if (nt > 0) ++n_items;

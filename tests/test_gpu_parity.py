@@ -220,7 +220,7 @@ def test_rescue_list_overflow_is_reported_and_stays_inside_the_list():
         n_over = int(words[2])
         assert n_over >= 3                                                 # at least the three aimed blocks were counted
         assert 0 <= words[64] < geo.N                                      # one was listed and redone
-        redone = geo.N - 1 - int(words[64])                                # (items count the blocks of a head downwards)
+        redone = int(words[64])
         assert (words[65:65 + 4096] == 0x5A5A5A5A).all()                   # nothing written behind the capacity
         O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], np.zeros_like(a["gate"]), gmask, geo, 1 / np.sqrt(128))
         O = to_f64(o)
