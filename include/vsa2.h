@@ -75,19 +75,13 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
 enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once everywhere (dQ pass about 15 % faster, GQA dK/dV pass about 30 %) */
 enum { VSA2_FLAG_PRECISE_BWD = 8 };   /* carry the pair in the dK/dV pass for MHA as well (that pass about 35 % slower): for maps
                                          that keep only a few blocks per row, where the softmax is sharply peaked */
-enum { VSA2_FLAG_PAIR_QUERY_FWD = 128 };/* fine forward with the 128-query kernel where two query blocks keep the same KV blocks on the
-                                         same operand tiles: the two halves of a 128-token cube, or (with VSA2_FLAG_GROUP_ROUTING and an
-                                         even number of query heads per KV head) pairs of heads that share their map.  About 1.2x
-                                         faster there than the default 64-query kernel, but it normalises the output by the fp32 row
-                                         sum rather than by the sum of the bf16-rounded weights, so on sharply peaked rows dQ of a
-                                         later backward can reach 2.5e-2 */
 enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV group share one block map ("group head", Sec. 4
                                          ablation): the block scores of the group's heads are added before the TopK, so
                                          the maps written for those heads are identical.  Not with VSA2_PER_QUERY_BUDGET
                                          (budgets belong to single heads): VSA2_ERR_UNSUPPORTED.
-                                         vsa2_attn_fwd with this flag and VSA2_FLAG_PAIR_QUERY_FWD RELIES on that: with an
-                                         even number of query heads per KV head it reads the map of the first head of each
-                                         pair of heads only */
+                                         vsa2_attn_fwd with this flag RELIES on that: with an even number of query heads per
+                                         KV head it stacks pairs of heads in the 128 rows of one tile (the same K/V tiles
+                                         serve both) and reads the map of the first head of each pair only */
 
 /* Problem statement (host struct). */
 typedef struct vsa2_params {

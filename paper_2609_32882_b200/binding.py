@@ -22,7 +22,6 @@ FLAG_EXACT_MAX_FWD = 2
 FLAG_FAST_BWD = 4
 FLAG_PRECISE_BWD = 8
 FLAG_BF16_COARSE_FWD = 64
-FLAG_PAIR_QUERY_FWD = 128
 FLAG_GROUP_ROUTING = 256
 
 OK = 0

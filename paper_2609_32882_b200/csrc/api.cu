@@ -465,11 +465,11 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
     ProfScope ps(VSA2_KERNEL_FINE_FWD, st, (g.flags & VSA2_FLAG_EXACT_MAX_FWD) ? 1 : 2);
     if (g.flags & VSA2_FLAG_EXACT_MAX_FWD)
       VSA2_CUDA(launch_fine_fwd(fx, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse, st));
-    else if (g.Lt == 0 && (g.flags & VSA2_FLAG_PAIR_QUERY_FWD) && (wide || ((g.flags & VSA2_FLAG_GROUP_ROUTING) && g.rep % 2 == 0)))
-      // 128 query columns per tile: the halves of a 128-token cube, or two heads of a group that share their map
-      VSA2_CUDA(launch_fine_fwd_wide_tc(n, !wide, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
-                                        reinterpret_cast<StatusBlock*>(workspace), st));
-    else if (fine_fwd_rows_supported(fx) && !(g.flags & 512))
+    else if ((wide || (g.flags & VSA2_FLAG_GROUP_ROUTING)) && fine_fwd_rows2_supported(n, !wide))
+      // 128 query rows per tile: the halves of a 128-token cube, or two heads of a group that share their map
+      VSA2_CUDA(launch_fine_fwd_rows2_tc(n, !wide, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
+                                         reinterpret_cast<StatusBlock*>(workspace), st));
+    else if (fine_fwd_rows_supported(fx))
       VSA2_CUDA(launch_fine_fwd_rows_tc(fx, qb, kb, vb, coarse ? gate : nullptr, row_ptr, col_idx, oc_hat, o, o_res, lse,
                                         reinterpret_cast<StatusBlock*>(workspace), st));
     else

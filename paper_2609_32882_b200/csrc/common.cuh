@@ -238,12 +238,13 @@ cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, 
                                     const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                     float* lse, StatusBlock* status, cudaStream_t st);
 
-// tensor-core forward with 128 query columns (fine_fwd_wide_tc.cu): two query blocks that keep the same key blocks on the
-// same operand tiles -- the two halves of a 128-token query cube (`g`, the map and oc_hat are those of the half-cube problem)
-// or, with pair_heads, one query block of two query heads that share their map; the workspace is the one of launch_fine_fwd_tc
-cudaError_t launch_fine_fwd_wide_tc(const Geo& g, bool pair_heads, const bf16* q, const bf16* k, const bf16* v, const float* gate,
-                                    const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
-                                    float* lse, StatusBlock* status, cudaStream_t st);
+// tensor-core forward with two query blocks (128 rows) per tile (fine_fwd_rows2_tc.cu): the halves of a 128-token cube, or one
+// block of two heads that share their map.  `g`, the map and oc_hat are those of the half-cube problem (or, with pair_heads,
+// of the ordinary 64-token problem); the workspace is the one of launch_fine_fwd_tc
+bool fine_fwd_rows2_supported(const Geo& g, bool pair_heads);
+cudaError_t launch_fine_fwd_rows2_tc(const Geo& g, bool pair_heads, const bf16* q, const bf16* k, const bf16* v, const float* gate,
+                                     const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
+                                     float* lse, StatusBlock* status, cudaStream_t st);
 
 // tensor-core backward passes (fine_bwd_tc.cu)
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,

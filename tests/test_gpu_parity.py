@@ -307,12 +307,6 @@ def test_group_shared_routing(wl):
     want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, scale, a["do"])
     for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
         assert_close(name, x, y, bf16_storage=name != "dGate")
-    # the same maps through the 128-query forward, which stacks pairs of heads (or the halves of a 128-token cube)
-    pair = CudaPath(wl, data, flags=vb.FLAG_GROUP_ROUTING | vb.FLAG_PAIR_QUERY_FWD)
-    assert np.array_equal(pair.route(), gmask)
-    O2, lse2 = pair.forward()
-    assert_close("O (128-query forward)", O2, O_ref, bf16_storage=True)
-    assert_lse_close(lse2, lse_ref)
 
 
 def test_group_shared_routing_is_refused_for_per_row_budgets():

@@ -29,7 +29,7 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     big = syn.CONFIGS[1]                                                              # per-query TopK, 1.8 MiB
     small = syn.Workload("mini_seq", 2, 3, 3, 64, (6, 9, 10), select_mode=syn.PER_SEQUENCE, topk=4, seed=22)
     wide = syn.Workload("mini_wide", 1, 4, 2, 128, (7, 10, 28), cube=(4, 4, 8), select_mode=syn.PER_SEQUENCE, topk=5, seed=65)
-    for wl in (big, small, wide, big):           # every call after the first runs over the previous call's leftovers
+    for n_call, wl in enumerate((big, small, wide, big)):   # every call after the first runs over the previous call's leftovers
         data = syn.make_inputs(wl, with_grad=False)
         p = vb.params_from_workload(wl)
         q, k = dev_bf16(data["q"]), dev_bf16(data["k"])
@@ -41,8 +41,12 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
                 for n in (s.ptr_elems, s.idx_elems, s.ptr_elems, s.idx_elems)]
         status = torch.full((1,), 123, dtype=torch.int32, device="cuda")
         m = vb.Map(*(b.data_ptr() for b in bufs))
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         vb.vsa2_route_noalloc(p, q, k, None, m, status)
         torch.cuda.synchronize()
+        if n_call > 0:       # (the first call on a device may make the driver load the library's device code and back the array)
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
         assert status.item() == vb.OK
         for got, want in zip(bufs, (ref.row_ptr, ref.col_idx, ref.col_ptr, ref.row_idx)):
             assert torch.equal(got, want[:got.numel()])
