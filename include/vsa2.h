@@ -264,7 +264,7 @@ int vsa2_device_status(const void* workspace, void* cuda_stream, int32_t* status
 
 /* Kernel groups, for timing from outside (e.g. a benchmark) without a profiler. */
 enum {
-  VSA2_KERNEL_POOL = 0,         /* mean pooling (Eq. 1, Eq. 5) */
+  VSA2_KERNEL_POOL = 0,         /* vsa2_attn_fwd: cube means of Q, K, V (Eq. 1) */
   VSA2_KERNEL_ROUTER_LSE = 1,   /* router pass 1: row log-sum-exp (Eq. 6) */
   VSA2_KERNEL_ROUTER_POOL = 2,  /* router pass 2: softmax + G x G pooling (Eq. 6-7) */
   VSA2_KERNEL_SELECT = 3,       /* TopK + CSR/CSC (Eq. 8-9) */
@@ -274,7 +274,8 @@ enum {
   VSA2_KERNEL_COARSE_BWD = 7,
   VSA2_KERNEL_FINE_BWD_DQ = 8,
   VSA2_KERNEL_FINE_BWD_DKV = 9,
-  VSA2_KERNEL_COUNT = 10
+  VSA2_KERNEL_POOL_ROUTER = 10, /* vsa2_route: sub-cube means of Q, K (Eq. 5) */
+  VSA2_KERNEL_COUNT = 11
 };
 
 /* Asks the library to record `start_event` before and `stop_event` after the launches of one kernel

@@ -35,7 +35,7 @@ EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd
            "vsa2_selftest_timeout", "vsa2_debug_rescue_capacity")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
-           "fine_bwd_dq", "fine_bwd_dkv")
+           "fine_bwd_dq", "fine_bwd_dkv", "pool_router")
 
 
 class Vsa2Error(RuntimeError):

@@ -59,6 +59,7 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   g->Bt = p->cube_t; g->Bh = p->cube_h; g->Bw = p->cube_w;
   g->Nt = (g->T + g->Bt - 1) / g->Bt; g->Nh = (g->H + g->Bh - 1) / g->Bh; g->Nw = (g->W + g->Bw - 1) / g->Bw;
   g->N = g->Nt * g->Nh * g->Nw;
+  geo_set_magics(*g);
   g->Nvid = g->N;
   g->Rt = p->rpool_t; g->Rh = p->rpool_h; g->Rw = p->rpool_w;
   g->Gt = g->Bt / g->Rt; g->Gh = g->Bh / g->Rh; g->Gw = g->Bw / g->Rw;
@@ -332,9 +333,8 @@ int vsa2_route(const vsa2_params* p, const void* q, const void* k, const int32_t
   bf16* qr = at<bf16>(workspace, rl.qr);
   bf16* kr = at<bf16>(workspace, rl.kr);
   {
-    ProfScope ps(VSA2_KERNEL_POOL, st, 2);
-    VSA2_CUDA(launch_pool(r, reinterpret_cast<const bf16*>(q), r.Hq, qr, nullptr, st));
-    VSA2_CUDA(launch_pool(r, reinterpret_cast<const bf16*>(k), r.Hkv, kr, nullptr, st));
+    ProfScope ps(VSA2_KERNEL_POOL_ROUTER, st, 1);
+    VSA2_CUDA(launch_pool_router(r, reinterpret_cast<const bf16*>(q), reinterpret_cast<const bf16*>(k), qr, kr, st));
   }
   float* pr = at<float>(workspace, rl.pr);
   if (router_tc_supported(r))
@@ -412,11 +412,9 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
   const float* oc_hat = coarse ? saved->oc_hat : nullptr;
   if (coarse) {
     {
-      ProfScope ps(VSA2_KERNEL_POOL, st, wide ? 6 : 3);
+      ProfScope ps(VSA2_KERNEL_POOL, st, wide ? 6 : 1);
       if (!wide) {
-        VSA2_CUDA(launch_pool(g, qb, g.Hq, nullptr, saved->qc, st));
-        VSA2_CUDA(launch_pool(g, kb, g.Hkv, nullptr, saved->kc, st));
-        VSA2_CUDA(launch_pool(g, vb, g.Hkv, nullptr, saved->vc, st));
+        VSA2_CUDA(launch_pool_coarse(g, qb, kb, vb, saved->qc, saved->kc, saved->vc, st));
       } else {
         float* x64 = at<float>(workspace, wl.x64);
         VSA2_CUDA(launch_pool(n, qb, n.Hq, nullptr, x64, st));
@@ -575,15 +573,25 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
       VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dvc_cube, dvc, st));
     }
   }
+  // cubes of 128 tokens: both passes on 128 x 128 tiles (temporary switch: flag 2048 keeps the 64-token kernels)
+  const bool wide128 = wide && g.Lt == 0 && fine_bwd128_supported(n) && !(g.flags & 2048);
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
-    VSA2_CUDA(launch_fine_bwd_dq_tc(fx, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
-                                    reinterpret_cast<StatusBlock*>(workspace), st));
+    if (wide128)
+      VSA2_CUDA(launch_fine_bwd128_dq_tc(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
+                                         reinterpret_cast<StatusBlock*>(workspace), st));
+    else
+      VSA2_CUDA(launch_fine_bwd_dq_tc(fx, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
+                                      reinterpret_cast<StatusBlock*>(workspace), st));
   }
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
-    VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
-                                     coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
+    if (wide128 && !fine_bwd_dkv_wants_pair(n))
+      VSA2_CUDA(launch_fine_bwd128_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
+                                          coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
+    else
+      VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
+                                       coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
   }
   return VSA2_OK;
 }

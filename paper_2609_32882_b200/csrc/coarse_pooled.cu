@@ -14,6 +14,7 @@ Geo pooled_geo(const Geo& g) {
   p.L = g.N;
   p.Nt = (p.T + p.Bt - 1) / p.Bt; p.Nh = (p.H + p.Bh - 1) / p.Bh; p.Nw = (p.W + p.Bw - 1) / p.Bw;
   p.N = p.Nt * p.Nh * p.Nw;
+  geo_set_magics(p);
   p.Nvid = p.N; p.Lt = 0; p.S = p.L;
   p.K = p.N;
   p.mode = VSA2_PER_QUERY;

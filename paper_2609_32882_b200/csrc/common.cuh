@@ -30,7 +30,18 @@ struct Geo {
   // kernels and the backward preprocess run on the BLOCK problem: N = Nvid + ceil(Lt / 64) blocks, block j < Nvid is video
   // cube j, block j >= Nvid holds text tokens 64 (j - Nvid) .. ; their maps are the block maps extended by the text blocks.
   int Nvid, Lt, S;
+  // ceil(2^32 / d) for d = Nw, Nh, Bw, Bh (geo_set_magics): the index arithmetic of the kernels divides by these with one
+  // multiply instead of a reciprocal, which would run on the unit the softmax exponentials need
+  unsigned mNw, mNh, mBw, mBh;
 };
+inline unsigned div_magic(int d) { return d <= 1 ? 0u : (unsigned)((0x100000000ull + (unsigned)d - 1ull) / (unsigned)d); }
+// to be called wherever Nw, Nh, Bw or Bh of a Geo are set
+inline void geo_set_magics(Geo& g) {
+  g.mNw = div_magic(g.Nw);
+  g.mNh = div_magic(g.Nh);
+  g.mBw = div_magic(g.Bw);
+  g.mBh = div_magic(g.Bh);
+}
 
 // Status block at the start of every workspace.
 struct StatusBlock {
@@ -49,25 +60,19 @@ struct ProfScope {
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// q = n / d, r = n % d for 0 <= n < 2^22 and 0 < d, through one reciprocal and a fix-up (exact).  The tensor-core
-// kernels decode cube and token indices several times per tile, and a 32-bit integer division costs tens of instructions.
-__device__ __forceinline__ void fast_divmod(int n, int d, int& q, int& r) {
-  q = __float2int_rz(__fdividef((float)n, (float)d));
+// q = n / d, r = n % d for 0 <= n < 2^22 and 0 < d < 2^10 with m = ceil(2^32 / d) (0 for d = 1): floor(n m / 2^32) is exact
+// while n d < 2^32.  The tensor-core kernels decode cube and token indices several times per tile; a 32-bit integer division
+// costs tens of instructions and a reciprocal on the special-function unit.
+__device__ __forceinline__ void fast_divmod(int n, int d, unsigned m, int& q, int& r) {
+  q = m == 0u ? n : (int)__umulhi((unsigned)n, m);
   r = n - q * d;
-  if (r < 0) {
-    --q;
-    r += d;
-  } else if (r >= d) {
-    ++q;
-    r -= d;
-  }
 }
 
 // cube n -> (nt, nh, nw);  n = (nt*Nh + nh)*Nw + nw
 __device__ __forceinline__ void cube_coords(const Geo& g, int n, int& nt, int& nh, int& nw) {
   int r;
-  fast_divmod(n, g.Nw, r, nw);
-  fast_divmod(r, g.Nh, nt, nh);
+  fast_divmod(n, g.Nw, g.mNw, r, nw);
+  fast_divmod(r, g.Nh, g.mNh, nt, nh);
 }
 
 // position (bt, bh, bw) inside cube (nt, nh, nw) -> raster token index, or -1 if padding
@@ -80,8 +85,8 @@ __device__ __forceinline__ int cube_token_at(const Geo& g, int nt, int nh, int n
 // position p in [0, B) inside a cube, ordered (bt, bh, bw) -> raster token index, or -1 if padding
 __device__ __forceinline__ int cube_token(const Geo& g, int nt, int nh, int nw, int p) {
   int bw, bh, bt, r;
-  fast_divmod(p, g.Bw, r, bw);
-  fast_divmod(r, g.Bh, bt, bh);
+  fast_divmod(p, g.Bw, g.mBw, r, bw);
+  fast_divmod(r, g.Bh, g.mBh, bt, bh);
   return cube_token_at(g, nt, nh, nw, bt, bh, bw);
 }
 
@@ -151,6 +156,9 @@ __device__ __forceinline__ void store_out(void* base, size_t idx, float v, int o
 // launchers implemented in the .cu files (all enqueue on `st`, return cudaGetLastError())
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_pool(const Geo& g, const bf16* x, int heads, bf16* xr, float* xc, cudaStream_t st);
+cudaError_t launch_pool_router(const Geo& g, const bf16* q, const bf16* k, bf16* qr, bf16* kr, cudaStream_t st);
+cudaError_t launch_pool_coarse(const Geo& g, const bf16* q, const bf16* k, const bf16* v, float* qc, float* kc, float* vc,
+                               cudaStream_t st);
 
 // raster <-> cube-major copy of a [batch, heads, L or N*B, D] bf16 tensor (pool.cu)
 cudaError_t launch_permute(const Geo& g, const bf16* src, int heads, bool inverse, bf16* dst, cudaStream_t st);
@@ -245,6 +253,17 @@ bool fine_fwd_rows2_supported(const Geo& g, bool pair_heads);
 cudaError_t launch_fine_fwd_rows2_tc(const Geo& g, bool pair_heads, const bf16* q, const bf16* k, const bf16* v, const float* gate,
                                      const int* row_ptr, const int* col_idx, const float* oc_hat, void* o, bf16* o_res,
                                      float* lse, StatusBlock* status, cudaStream_t st);
+
+// tensor-core backward passes for cubes of 128 tokens (fine_bwd128_tc.cu): `g` and the maps are those of the half-cube problem
+bool fine_bwd128_supported(const Geo& g);
+bool fine_bwd_dkv_wants_pair(const Geo& g);
+cudaError_t launch_fine_bwd128_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                                     const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
+                                     const float* dqc, void* dq, StatusBlock* status, cudaStream_t st);
+cudaError_t launch_fine_bwd128_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
+                                      const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
+                                      const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
+                                      cudaStream_t st);
 
 // tensor-core backward passes (fine_bwd_tc.cu)
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,

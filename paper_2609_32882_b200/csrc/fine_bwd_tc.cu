@@ -982,8 +982,7 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   DkvArgs a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
-  // a KV block of a GQA group sums rep times as many query blocks: there the plain bf16 rounding of P and dS passes 2e-2
-  const bool split = (g.flags & VSA2_FLAG_PRECISE_BWD) || (g.rep > 1 && !(g.flags & VSA2_FLAG_FAST_BWD));
+  const bool split = fine_bwd_dkv_wants_pair(g);
 #define VSA2_LAUNCH_DKV(DD, SP)                                                                                                  \
   do {                                                                                                                           \
     using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \

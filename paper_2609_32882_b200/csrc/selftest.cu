@@ -175,6 +175,7 @@ extern "C" int vsa2_selftest_umma(const vsa2_params* p, const void* q, const voi
   g.Bt = p->cube_t; g.Bh = p->cube_h; g.Bw = p->cube_w;
   g.Nt = (g.T + g.Bt - 1) / g.Bt; g.Nh = (g.H + g.Bh - 1) / g.Bh; g.Nw = (g.W + g.Bw - 1) / g.Bw; g.N = sz.n_cubes;
   g.Nvid = g.N; g.Lt = 0; g.S = g.L;
+  geo_set_magics(g);
   if (cube_q < 0 || cube_q >= g.N || cube_a < 0 || cube_a >= g.N || cube_b < 0 || cube_b >= g.N) return VSA2_ERR_INVALID_ARG;
   CUtensorMap tq, tk, tv;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv))

@@ -24,6 +24,7 @@ Geo narrow_geo(const Geo& g) {
   Geo n = g;
   n.Bw = g.Bw / 2;
   n.Nw = g.Nw * 2;
+  geo_set_magics(n);
   n.N = g.N * 2;
   n.Nvid = n.N;
   n.Gw = n.Bw / n.Rw;
