@@ -60,12 +60,27 @@ struct ProfScope {
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// q = n / d, r = n % d for 0 <= n < 2^22 and 0 < d < 2^10 with m = ceil(2^32 / d) (0 for d = 1): floor(n m / 2^32) is exact
-// while n d < 2^32.  The tensor-core kernels decode cube and token indices several times per tile; a 32-bit integer division
-// costs tens of instructions and a reciprocal on the special-function unit.
+// q = n / d, r = n % d for 0 <= n < 2^22 and 0 < d < 2^10 with m = ceil(2^32 / d) (0 for d = 1): floor(n m / 2^32), exact
+// while n d < 2^32 -- one multiply.  The tensor-core kernels decode cube and token indices several times per tile; the
+// earlier form (a reciprocal and a fix-up) runs on the special-function unit, behind the exponentials of the softmax warps,
+// which cost a service warp of the 128-token backward 4000 cycles per tile.  A translation unit that defines
+// VSA2_RECIPROCAL_DIVMOD before including this header keeps the reciprocal form (where that measured faster).
 __device__ __forceinline__ void fast_divmod(int n, int d, unsigned m, int& q, int& r) {
+#ifdef VSA2_RECIPROCAL_DIVMOD
+  (void)m;
+  q = __float2int_rz(__fdividef((float)n, (float)d));
+  r = n - q * d;
+  if (r < 0) {
+    --q;
+    r += d;
+  } else if (r >= d) {
+    ++q;
+    r -= d;
+  }
+#else
   q = m == 0u ? n : (int)__umulhi((unsigned)n, m);
   r = n - q * d;
+#endif
 }
 
 // cube n -> (nt, nh, nw);  n = (nt*Nh + nh)*Nw + nw

@@ -54,13 +54,6 @@ struct Bwd128Misc {
 };
 static_assert(sizeof(Bwd128Misc) <= 2048, "misc region too small");
 
-#ifdef VSA2_TRACE
-__device__ long long g_w2_trace[2 * 6 * 256 * 8];
-#define W2_TR(role, tile, slot) do { if (blockIdx.x == 0 && (tile) < 256u) g_w2_trace[((PASS * 6 + (role)) * 256 + (tile)) * 8 + (slot)] = clock64(); } while (0)
-#else
-#define W2_TR(role, tile, slot) do {} while (0)
-#endif
-
 struct Bwd128Args {
   int* item_counter;    // global, zero before the launch
   const float* lse;
@@ -302,10 +295,8 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
             if (t + 1 < nt_l) j = ent[2 * t + 2 + my_blk];        // the next entry is on its way while this warp waits
             const uint32_t slot = tg % nslots, par = (tg / nslots) & 1;
             int ok = 1;
-            if (lane == 0 && warp < 2) W2_TR(4 + warp, tg, 0);
             if (lane == 0) {
               ok = tc::mbar_wait_parked(&empty[slot], par ^ 1, &misc->abort_flag);
-              if (warp < 2) W2_TR(4 + warp, tg, 1);
               if (ok) {
                 if (PASS == 0 && which == 0) misc->edge[slot][my_blk] = (unsigned char)ef;
                 tc::mbar_expect_tx(&full[slot], C::SLOT / 2);
@@ -334,20 +325,16 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
         VSA2_WAIT(&misc->st_full, n_items & 1);
         VSA2_W2_TILES_BEGIN
           uint32_t slot;
-          if (lane == 0) W2_TR(is_s ? 0 : 1, tg, 0);
           if (is_s) {
             slot = tg % kW2RingA;
             VSA2_WAIT(&misc->a_full[slot], (tg / kW2RingA) & 1);
-            if (lane == 0) W2_TR(0, tg, 1);
             VSA2_WAIT(&misc->s_free, (tg & 1) ^ 1);
           } else {
             slot = tg % kW2RingB;
             VSA2_WAIT(&misc->b_full[slot], (tg / kW2RingB) & 1);
-            if (lane == 0) W2_TR(1, tg, 1);
             if (PASS == 0) VSA2_WAIT(&misc->dp_free[tg % NDP], ((tg / NDP) & 1) ^ 1);
             else VSA2_WAIT(&misc->s_loaded, tg & 1);        // S^T of this tile has left the staging columns
           }
-          if (lane == 0) W2_TR(is_s ? 0 : 1, tg, 2);
           tc::tc_fence_after();
           if (tc::elect_one()) {
             const uint64_t dy = tc::smem_desc_sw128(ring0 + slot * C::SLOT, 16, 1024);
@@ -366,7 +353,6 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
             if (tt == nt_all - 1) tc::mma_commit(&misc->st_empty);
           }
           __syncwarp();
-          if (lane == 0) W2_TR(is_s ? 0 : 1, tg, 3);
         VSA2_W2_TILES_END
         ++n_items;
       }
@@ -385,10 +371,8 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
           const uint32_t sa = tg % kW2RingA, sb = tg % kW2RingB;
           if (PASS == 1) {
             // dV += P^T dO_i: P depends on S only, so it can be ready before the dO pair of the tile has landed
-            if (lane == 0) W2_TR(2, tg, 0);
             VSA2_WAIT(&misc->b_full[sb], (tg / kW2RingB) & 1);
             VSA2_WAIT(&misc->p_ready, tg & 1);
-            if (lane == 0) W2_TR(2, tg, 1);
             tc::tc_fence_after();
             if (tc::elect_one()) {
               mma_out_ts<D, SPLIT, true>(tmem_base + TM_ACC1, tmem_base + TM_P, ring_b + sb * C::SLOT, tt > 0);
@@ -397,11 +381,8 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
               if (tt == nt_all - 1) tc::mma_commit(&misc->o_full);
             }
             __syncwarp();
-            if (lane == 0) W2_TR(2, tg, 2);
           }
-          if (lane == 0) W2_TR(2, tg, 3);
           VSA2_WAIT(&misc->ds_ready, tg & 1);
-          if (lane == 0) W2_TR(2, tg, 4);
           tc::tc_fence_after();
           if (tc::elect_one()) {
             if (PASS == 0) mma_out_ts<D, SPLIT, false>(tmem_base + TM_ACC0, tmem_base + TM_DP + (tg % NDP) * 128, ring_a + sa * C::SLOT, tt > 0);
@@ -411,7 +392,6 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
             if (tt == nt_all - 1) tc::mma_commit(&misc->o_full);
           }
           __syncwarp();
-          if (lane == 0) W2_TR(2, tg, 5);
         VSA2_W2_TILES_END
         ++n_items;
       }
@@ -506,16 +486,12 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
       cur_fl = nxt_fl;                                                                                        \
       entry_geo(ent[min(2 * t0 + 32 + lane, n_ent - 1)], nxt_base, nxt_fl);                                   \
     }                                                                                                         \
-    if (lane == 0) W2_TR(5, tg, 4);                                                                           \
     if ((T) + 2 < nt_l) {                                                                                     \
       int b0_, f0_, b1_, f1_;                                                                                 \
       VSA2_W2_ENTRY((T) + 2, b0_, f0_, b1_, f1_)                                                              \
-      if (lane == 0) W2_TR(5, tg, 5);                                                                         \
       load_stats(mh, b0_, f0_, b1_, f1_, FREE##_ls, FREE##_dl, FREE##_ok);                                    \
     }                                                                                                         \
-    if (lane == 0) W2_TR(5, tg, 2);                                                                           \
     VSA2_WAIT_PARKED(&misc->stat_free, (tg & 1) ^ 1);                                                         \
-    if (lane == 0) W2_TR(5, tg, 3);                                                                           \
     _Pragma("unroll") for (int u = 0; u < 4; ++u)                                                             \
         misc->lse2[lane + 32 * u] = ((CUR##_ok >> u) & 1u) ? CUR##_ls[u] * 1.4426950408889634f : INFINITY;    \
     tc::mbar_arrive(&misc->stat_full);                                                                        \
@@ -561,24 +537,18 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
         VSA2_W2_TILES_BEGIN
           const uint32_t dpb = (tg % NDP) * 128;
           uint32_t pf[64];                 // S, then P (as float bits) of this thread's 64 columns
-          if (tid == 256) W2_TR(3, tg, 0);
           VSA2_WAIT(&misc->s_full, tg & 1);
-          if (tid == 256) W2_TR(3, tg, 1);
           tc::tc_fence_after();
-          if (PASS == 1 && tid == 256) W2_TR(3, tg, 0);
           unsigned long long vm = ~0ull;
           if (PASS == 0) vm = misc->vmask[misc->edge[tg % kW2RingA][half]];
           else VSA2_WAIT(&misc->stat_full, tg & 1);
-          if (tid == 256) W2_TR(3, tg, 5);
           tc::tmem_ld32(lane_addr + TM_S + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(&pf[0]));
           tc::tmem_ld32(lane_addr + TM_S + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(&pf[32]));
           if (PASS == 0) {
             // dP of this tile is normally there already (two buffers): fetch it together with S, then one pass over the
             // registers: P = exp2(S c2 - lse), dS = P (dP - delta); the factor `scale` goes into the epilogue
             uint32_t dp[64];
-            if (tid == 256) W2_TR(3, tg, 2);
             VSA2_WAIT(&misc->dp_full[tg % NDP], (tg / NDP) & 1);
-            if (tid == 256) W2_TR(3, tg, 3);
             tc::tc_fence_after();
             tc::tmem_ld32(lane_addr + TM_DP + dpb + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
             tc::tmem_ld32(lane_addr + TM_DP + dpb + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
@@ -601,7 +571,6 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
             tc::tmem_ld_wait();
             tc::tc_fence_before();
             tc::mbar_arrive(&misc->s_loaded);        // S^T is in registers: dP^T may take the staging columns
-            if (tid == 256) W2_TR(3, tg, 6);
             VSA2_WAIT(&misc->p_free, (tg & 1) ^ 1);  // dV of the previous tile has read its P^T
             tc::tc_fence_after();
             uint32_t dp[64];
@@ -623,9 +592,7 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
               if (c == 0) {
                 // half way through the exponentials dP^T of this tile is complete: pull it into registers now, so that
                 // S^T of the next tile can be computed while this stage finishes the tile
-                if (tid == 256) W2_TR(3, tg, 7);
                 VSA2_WAIT(&misc->dp_full[0], tg & 1);
-                if (tid == 256) W2_TR(3, tg, 3);
                 tc::tc_fence_after();
                 tc::tmem_ld32(lane_addr + TM_DP + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
                 tc::tmem_ld32(lane_addr + TM_DP + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
@@ -638,7 +605,6 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
             tc::tmem_st_wait();
             tc::tc_fence_before();
             tc::mbar_arrive(&misc->p_ready);
-            if (tid == 256) W2_TR(3, tg, 2);
             VSA2_WAIT(&misc->dlt_full, tg & 1);
             VSA2_WAIT(&misc->ds_free, (tg & 1) ^ 1); // dK of the previous tile has read its dS^T
             tc::tc_fence_after();
@@ -662,7 +628,6 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
           tc::tmem_st_wait();
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->ds_ready);
-          if (tid == 256) W2_TR(3, tg, 4);
         VSA2_W2_TILES_END
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
@@ -744,12 +709,6 @@ done:
   }
   if (warp == 4) tc::tmem_dealloc(tmem_base, 512);
 }
-
-#ifdef VSA2_TRACE
-extern "C" int vsa2_debug_bwd128_trace(long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_w2_trace, sizeof(long long) * 2 * 6 * 256 * 8) == cudaSuccess ? 0 : -5;
-}
-#endif
 
 // A KV cube of a GQA group sums rep times as many query cubes: there the plain bf16 rounding of P and dS passes 2e-2 and
 // the dK/dV pass carries them as bf16 pairs, which only the 64-token kernel has room for.

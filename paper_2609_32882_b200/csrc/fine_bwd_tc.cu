@@ -20,104 +20,9 @@
 // Accumulators stay in tensor memory for the whole list of a block, so every output element is written
 // once, by one thread, in a fixed order: no floating-point atomics, bitwise reproducible.
 // The pooling backward of the coarse branch (Eq. 1) is added in the epilogues.
-#include "tc_attn.cuh"
+#include "fine_bwd_tc.cuh"
 
 namespace vsa2 {
-
-constexpr int kDqThreads = 416;    // dQ pass: 4 service warps, 2 x 4 elementwise warps, 1 more issuer warp
-constexpr int kDkvThreads = 576;   // dK/dV pass: 4 service warps, 2 x 4 elementwise warps, 4 row-statistics warps, 2 issuer warps
-constexpr int kRingA = 3;          // slots of the ring whose tiles are also an operand of the last product of a tile
-constexpr int kRingB = 2;          // (the ring-B slot of a tile is also the index of its tensor-memory buffers)
-static_assert(kRingB == 2, "ring B shares its slot index with the two accumulator buffers");
-
-// Shared-memory plan of both passes (D = 128: 5 x 32 KB ring slots, 2 x 16 KB stationary tiles, 2 x 16 KB operand
-// buffers, 2 KB of barriers and per-block vectors: exactly the 227 KB a block may use).  Ring A has 3 slots, ring B 2;
-// each ring has one producing warp and fixed consuming roles.
-// RA: slots of ring A; NP: 16 KB operand buffers (the dK/dV pass in its split mode trades one ring-A slot for the two
-// buffers that hold the low-order parts of P and dS).
-template <int D, int RA = kRingA, int NP = 2>
-struct BwdTc {
-  static constexpr int DH = D / 64;
-  static constexpr uint32_t SLOT = 2 * DH * kSlab;   // a pair of cube tiles, [half][A | B]
-  static constexpr uint32_t TILE = DH * kSlab;       // one cube tile, [half]
-  static constexpr uint32_t PBYTES = 128 * 128;      // 128 rows x 64 bf16
-  static constexpr uint32_t OFF_RING_B = RA * SLOT;
-  static constexpr uint32_t OFF_ST0 = (RA + kRingB) * SLOT;       // stationary tile 0 (Q or K)
-  static constexpr uint32_t OFF_ST1 = OFF_ST0 + TILE;             // stationary tile 1 (dO or V)
-  static constexpr uint32_t OFF_P = OFF_ST1 + TILE;               // the 16 KB operand buffers
-  static constexpr uint32_t OFF_MISC = OFF_P + NP * PBYTES;
-  static constexpr uint32_t MISC_BYTES = 2048;
-  static constexpr size_t smem_bytes = OFF_MISC + MISC_BYTES + 1024;
-};
-
-struct BwdMisc {
-  uint64_t st_full, st_empty, o_full, o_empty;
-  uint64_t a_full[kRingA], a_empty[kRingA], b_full[kRingB], b_empty[kRingB];
-  uint64_t s_full[2], s_free[2], dp_full[2], dp_free[2];   // the two score / dP accumulators in tensor memory
-  uint64_t p_ready, p_free;                                 // dK/dV pass: the P operand buffer
-  uint64_t ds_ready[2], ds_free[2];                         // dS operand buffers (the dK/dV pass has one)
-  uint64_t stat_full, stat_free;                            // dK/dV pass: the per-row statistics of a tile
-  ItemQueue items;                                          // work items of this CTA (see tc_attn.cuh)
-  uint64_t e_sync;                                          // group barrier of the 256 elementwise threads
-  uint32_t tmem_base;
-  int abort_flag;
-  unsigned char edge[kRingA][2];   // dQ pass: edge flags of the two key cubes in each ring-A slot (written by its producer)
-  // dQ pass: lse2[tb][c] = stats[tb * 64 + c], delta[tb][c] = stats[128 + tb * 64 + c]: per query column of the item with
-  // parity tb, lse * log2(e) (+inf for padding) and delta.  dK/dV pass: (lse * log2(e), delta) of the 128 query rows of
-  // the current tile, interleaved.
-  alignas(16) float stats[256];
-  int tok[2][64];
-};
-static_assert(sizeof(BwdMisc) <= 2048, "misc region too small");
-
-__device__ __forceinline__ void bwd_init_barriers(BwdMisc* misc) {
-  misc->abort_flag = 0;
-  tc::mbar_init(&misc->st_full, 1);
-  tc::mbar_init(&misc->st_empty, 2);     // both first-stage issuers
-  tc::mbar_init(&misc->o_full, 1);       // re-initialised to 2 by the dK/dV pass (two last-stage issuers)
-  tc::mbar_init(&misc->o_empty, 256);
-  for (int s = 0; s < kRingA; ++s) {
-    tc::mbar_init(&misc->a_full[s], 1);
-    tc::mbar_init(&misc->a_empty[s], 1);
-  }
-  for (int s = 0; s < kRingB; ++s) {
-    tc::mbar_init(&misc->b_full[s], 1);
-    tc::mbar_init(&misc->b_empty[s], 1);
-  }
-  for (int s = 0; s < 2; ++s) {
-    tc::mbar_init(&misc->s_full[s], 1);
-    tc::mbar_init(&misc->s_free[s], 256);
-    tc::mbar_init(&misc->dp_full[s], 1);
-    tc::mbar_init(&misc->dp_free[s], 256);
-    tc::mbar_init(&misc->ds_ready[s], 256);
-    tc::mbar_init(&misc->ds_free[s], 1);
-  }
-  tc::mbar_init(&misc->p_ready, 256);
-  tc::mbar_init(&misc->e_sync, 256);
-  tc::mbar_init(&misc->p_free, 1);
-  tc::mbar_init(&misc->stat_full, 128);
-  tc::mbar_init(&misc->stat_free, 256);
-}
-
-// One warp streams pairs of cube tiles into a ring of NS slots: lane 0 owns the barriers, lanes 0 .. 2*DH-1 issue one
-// box each (half h = lane / 2 of block lane & 1).  C3, C2, C1: box coordinates of this lane's block in map TMAP, `bh`: its head.
-// `LANE0_PRE`: statement lane 0 runs once the slot is free, before the loads are armed (may use slot_).
-#define VSA2_RING_LOAD(FULL, EMPTY, NS, RING_BASE, TMAP, SEQ, CT, CH, CW, BH, LANE0_PRE, WAITFN)                  \
-  do {                                                                                                            \
-    const uint32_t slot_ = (SEQ) % (NS), par_ = ((SEQ) / (NS)) & 1;                                               \
-    int ok_ = 1;                                                                                                  \
-    if (lane == 0) {                                                                                              \
-      ok_ = tc::WAITFN(&(EMPTY)[slot_], par_ ^ 1, &misc->abort_flag);                                             \
-      if (ok_) {                                                                                                  \
-        LANE0_PRE;                                                                                                \
-        tc::mbar_expect_tx(&(FULL)[slot_], C::SLOT);                                                              \
-      }                                                                                                           \
-    }                                                                                                             \
-    if (!__shfl_sync(0xffffffffu, ok_, 0)) goto done;                                                             \
-    if (lane < 2 * C::DH)                                                                                         \
-      tc::tma_load_5d((RING_BASE) + slot_ * C::SLOT + (2 * (lane >> 1) + (lane & 1)) * kSlab, (TMAP), &(FULL)[slot_], \
-                      (lane >> 1) * 64, (CW), (CH), (CT), (BH));                                                  \
-  } while (0)
 
 // ================================================================================================
 // dQ pass
@@ -479,460 +384,8 @@ done:
 }
 
 // ================================================================================================
-// dK/dV pass
+// launcher
 // ================================================================================================
-struct DkvArgs {
-  int* item_counter;    // global, zero before the launch
-  const float* lse;
-  const float* delta;
-  const int* col_ptr;
-  const int* row_idx;
-  const float* dkc;     // [B, Hq, N, D] per query head, or null
-  const float* dvc;
-  void* dk;
-  void* dv;
-  StatusBlock* status;
-};
-
-constexpr int kMaxRep = 16;   // query heads per KV head the dK/dV pass supports
-
-// entry e of the concatenated column lists of the group's query heads -> (query head, query block)
-// (`cnt_prefix`, `col_beg`: per-head counts prefix and list starts of the item, read once per item so that this lookup
-// costs a single global load)
-__device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b, int hk, const int* cnt_prefix,
-                                          const int* col_beg, int e, int& bhq, int& i) {
-  int hh = 0;
-  while (hh + 1 < g.rep && e >= cnt_prefix[hh + 1]) ++hh;
-  bhq = b * g.Hq + hk * g.rep + hh;
-  i = a.row_idx[(size_t)bhq * g.nnz_cap + col_beg[hh] + (e - cnt_prefix[hh])];
-}
-
-// Roles: warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA producer of the
-// dO pairs (ring B), warp 2 = issuer of S = Q_pair K^T, warp 3 = issuer of dP = dO_pair V^T, warp 16 = issuer of
-// dV^T += dO_pair^T P (frees the dO slot), warp 17 = issuer of dK^T += Q_pair^T dS (frees the Q slot), warps 4..11 =
-// elementwise stage + epilogue (each half of the key columns): P is handed to the dV^T product before dS is formed;
-// warps 12..15 = one thread per query row of the tile: they look up the row's (head, block, token) and fetch its lse and
-// delta one tile ahead, so that the elementwise warps, which bound the pass, touch no global memory inside a tile.
-// SPLIT: P and dS are handed to the dV^T and dK^T products as [bf16(X) | bf16(X - bf16(X))] (N = 128 products into two
-// accumulator halves that the epilogue adds), which removes their bf16 rounding from dV and dK: a KV block sums hundreds of
-// query blocks (times the query heads of a GQA group), and with plain bf16 operands that noise alone passes 2e-2.  The two
-// extra operand buffers take the place of the third ring-A slot.
-template <int D, bool SPLIT>
-__global__ void __launch_bounds__(kDkvThreads, 1)
-fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                       const __grid_constant__ CUtensorMap tm_qt, const __grid_constant__ CUtensorMap tm_kt,
-                       const __grid_constant__ CUtensorMap tm_vt, const __grid_constant__ CUtensorMap tm_dot, Geo g,
-                       DkvArgs a) {
-  constexpr int RA = SPLIT ? 2 : kRingA;                   // slots of the Q ring
-  constexpr uint32_t TM_DK = 256, TM_DV = SPLIT ? 384 : 320;
-  using C = BwdTc<D, RA, SPLIT ? 4 : 2>;
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
-  unsigned char* k_tile = smem + C::OFF_ST0;
-  unsigned char* v_tile = smem + C::OFF_ST1;
-  unsigned char* p_tile = smem + C::OFF_P;                                  // P  [128 q, 64 kv] (SPLIT: followed by its low part)
-  unsigned char* ds_tile = smem + C::OFF_P + (SPLIT ? 2 : 1) * C::PBYTES;   // dS [128 q, 64 kv] (SPLIT: followed by its low part)
-  BwdMisc* misc = reinterpret_cast<BwdMisc*>(smem + C::OFF_MISC);
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int total_items = g.batch * g.Hkv * g.N;
-  const float c2 = g.scale * 1.4426950408889634f;
-
-  if (tid == 0) {
-    bwd_init_barriers(misc);
-    tc::mbar_init(&misc->o_full, 2);                                          // two last-stage issuers
-    item_queue_init(&misc->items, 2 + 4 + 256 + 128);
-    for (int s = 0; s < kRingB; ++s) tc::mbar_init(&misc->b_empty[s], 2);     // a dO slot is read by dP and by dV^T
-    tc::fence_barrier_init();
-    tc::prefetch_tmap(&tm_q);
-    tc::prefetch_tmap(&tm_k);
-    tc::prefetch_tmap(&tm_v);
-    tc::prefetch_tmap(&tm_do);
-  }
-  if (warp == 2) {
-    tc::tmem_alloc(&misc->tmem_base, 512);
-    tc::tmem_relinquish();
-  }
-  tc::tc_fence_before();
-  __syncthreads();
-  tc::tc_fence_after();
-  const uint32_t tmem_base = misc->tmem_base;
-  // tensor-memory columns: S buffers 0, 64; dP buffers 128, 192; dK^T 256; dV^T 320 (SPLIT: dK^T 256 + 320, dV^T 384 + 448)
-
-  // per item: prefix of the per-head column counts and the list starts (every role recomputes them)
-#define VSA2_DKV_ITEM_SETUP()                                                            \
-  int j, bhk;                                                                            \
-  item_block(g, item, bhk, j);                                                           \
-  const int b = bhk / g.Hkv, hk = bhk % g.Hkv;                                           \
-  int cnt_prefix[kMaxRep + 1], col_beg[kMaxRep];                                         \
-  cnt_prefix[0] = 0;                                                                     \
-  for (int hh = 0; hh < g.rep; ++hh) {                                                   \
-    const size_t base_ = (size_t)(b * g.Hq + hk * g.rep + hh) * (g.N + 1) + j;           \
-    col_beg[hh] = a.col_ptr[base_];                                                      \
-    cnt_prefix[hh + 1] = cnt_prefix[hh] + (a.col_ptr[base_ + 1] - col_beg[hh]);          \
-  }                                                                                      \
-  const int k = cnt_prefix[g.rep];
-
-  if (warp < 2) {
-    // ------------------------------------------------------------------ TMA producers
-    const int which = warp;                               // 0: Q pairs (ring A) + K, V tiles; 1: dO pairs (ring B)
-    const CUtensorMap* tm = which == 0 ? &tm_q : &tm_do;
-    const CUtensorMap* tm_text = which == 0 ? &tm_qt : &tm_dot;
-    const int my_blk = lane & 1;
-    uint32_t tg = 0, n_items = 0, published = 0;
-    for (uint32_t seq = 0;; ++seq) {
-      // warp 0, lane 0 is the CTA's scheduler
-      int item = 0;
-      if (lane == 0) {
-        if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
-        else item = item_get(&misc->items, seq, &misc->abort_flag);
-      }
-      item = __shfl_sync(0xffffffffu, item, 0);
-      if (item == -2) goto done;
-      if (item < 0) break;
-      VSA2_DKV_ITEM_SETUP();
-      if (k == 0) continue;
-      if (which == 0) {
-        int c1, c2, c3;
-        block_box(g, j, c1, c2, c3);
-        const bool ktext = block_is_text(g, j);
-        int ok = 1;
-        if (lane == 0) {
-          ok = tc::mbar_wait_parked(&misc->st_empty, (n_items & 1) ^ 1, &misc->abort_flag);
-          if (ok) tc::mbar_expect_tx(&misc->st_full, 2 * C::TILE);
-        }
-        if (!__shfl_sync(0xffffffffu, ok, 0)) goto done;
-        if (lane < 2 * C::DH) {
-          const int h = lane >> 1;
-          if (lane & 1) tc::tma_load_5d(v_tile + h * kSlab, ktext ? &tm_vt : &tm_v, &misc->st_full, h * 64, c1, c2, c3, bhk);
-          else tc::tma_load_5d(k_tile + h * kSlab, ktext ? &tm_kt : &tm_k, &misc->st_full, h * 64, c1, c2, c3, bhk);
-        }
-      }
-      ++n_items;
-      const int nt = (k + 1) >> 1;
-      int bhq_l, i_l;           // this lane's entry of the tile, fetched one tile ahead of the slot wait
-      dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && k > 1) ? 1 : 0, bhq_l, i_l);
-      for (int t = 0; t < nt; ++t, ++tg) {
-        int c1, c2, c3;
-        block_box(g, i_l, c1, c2, c3);
-        const CUtensorMap* tm_i = block_is_text(g, i_l) ? tm_text : tm;
-        const int bhq_t = bhq_l;
-        if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
-        if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, RA, smem, tm_i, tg, c3, c2, c1, bhq_t, {}, mbar_wait_parked);
-        else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm_i, tg, c3, c2, c1, bhq_t, {}, mbar_wait_parked);
-      }
-    }
-  } else if (warp == 2 || warp == 3) {
-    // ------------------------------------------------------------------ issuers of S = Q_pair K^T (warp 2) and
-    // dP = dO_pair V^T (warp 3); whole warp in the loop, one elected lane issues (see the dQ pass)
-    {
-      const bool is_s = warp == 2;
-      const uint32_t b_addr = tc::smem_u32(is_s ? k_tile : v_tile), base = tc::smem_u32(smem);
-      uint32_t tg = 0, n_items = 0;
-      for (uint32_t seq = 0;; ++seq) {
-        VSA2_NEXT_ITEM_WARP(item, seq);
-        VSA2_DKV_ITEM_SETUP();
-        (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
-        if (k == 0) continue;
-        const int nt = (k + 1) >> 1;
-        VSA2_WAIT_PARKED(&misc->st_full, n_items & 1);
-        for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t sb = tg & 1, pb = (tg >> 1) & 1;
-          if (is_s) {
-            const uint32_t sa = tg % RA, pa = (tg / RA) & 1;
-            VSA2_WAIT_PARKED(&misc->a_full[sa], pa);
-            VSA2_WAIT_PARKED(&misc->s_free[sb], pb ^ 1);
-            tc::tc_fence_after();
-            if (tc::elect_one()) {
-              mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
-              tc::mma_commit(&misc->s_full[sb]);
-              if (t == nt - 1) tc::mma_commit(&misc->st_empty);
-            }
-          } else {
-            VSA2_WAIT_PARKED(&misc->b_full[sb], pb);
-            VSA2_WAIT_PARKED(&misc->dp_free[sb], pb ^ 1);
-            tc::tc_fence_after();
-            if (tc::elect_one()) {
-              mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
-              tc::mma_commit(&misc->dp_full[sb]);
-              tc::mma_commit(&misc->b_empty[sb]);
-              if (t == nt - 1) tc::mma_commit(&misc->st_empty);
-            }
-          }
-          __syncwarp();
-        }
-        ++n_items;
-      }
-    }
-  } else if (warp == 16 || warp == 17) {
-    // ------------------------------------------------------------------ issuers of dV^T += dO_pair^T P (warp 16) and
-    // dK^T += Q_pair^T dS (warp 17); whole warp in the loop, one elected lane issues
-    {
-      const bool is_v = warp == 16;
-      const uint32_t b_addr = tc::smem_u32(is_v ? p_tile : ds_tile), base = tc::smem_u32(smem);
-      uint32_t tg = 0, n_items = 0;
-      for (uint32_t seq = 0;; ++seq) {
-        VSA2_NEXT_ITEM_WARP(item, seq);
-        VSA2_DKV_ITEM_SETUP();
-        (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
-        if (k == 0) continue;
-        const int nt = (k + 1) >> 1;
-        VSA2_WAIT_PARKED(&misc->o_empty, (n_items & 1) ^ 1);
-        for (int t = 0; t < nt; ++t, ++tg) {
-          if (is_v) {
-            // P depends on S only, so it can be ready before the dO pair of the tile has landed: wait for that too
-            const uint32_t sv = tg & 1;
-            VSA2_WAIT_PARKED(&misc->b_full[sv], (tg >> 1) & 1);
-            VSA2_WAIT_PARKED(&misc->p_ready, tg & 1);
-            tc::tc_fence_after();
-            if (tc::elect_one()) {
-              if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, C::PBYTES, t > 0);
-              else mma_pairT_mnmajor<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
-              tc::mma_commit(&misc->b_empty[sv]);
-              tc::mma_commit(&misc->p_free);
-              if (t == nt - 1) tc::mma_commit(&misc->o_full);
-            }
-          } else {
-            const uint32_t sa = tg % RA;
-            VSA2_WAIT_PARKED(&misc->ds_ready[0], tg & 1);
-            tc::tc_fence_after();
-            if (tc::elect_one()) {
-              if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, C::PBYTES, t > 0);
-              else mma_pairT_mnmajor<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
-              tc::mma_commit(&misc->a_empty[sa]);
-              tc::mma_commit(&misc->ds_free[0]);
-              if (t == nt - 1) tc::mma_commit(&misc->o_full);
-            }
-          }
-          __syncwarp();
-        }
-        ++n_items;
-      }
-    }
-  } else if (warp >= 12 && warp < 16) {
-    // ------------------------------------------------------------------ row statistics of the tiles (128 threads)
-    const int r = tid - 384;                 // query row of the tile
-    const int blk = r >> 6;
-    float2* rowstat = reinterpret_cast<float2*>(misc->stats);
-    uint32_t tg = 0;
-    for (uint32_t seq = 0;; ++seq) {
-      VSA2_NEXT_ITEM(item, seq);
-      VSA2_DKV_ITEM_SETUP();
-      (void)j; (void)bhk;
-      if (k == 0) continue;
-      const int nt = (k + 1) >> 1;
-      int bhq_n, i_n;
-      dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
-      for (int t = 0; t < nt; ++t, ++tg) {
-        const bool dup = (blk == 1) && (2 * t + 1 >= k);
-        const int l = dup ? -1 : block_token(g, i_n, r & 63);
-        const size_t idx = l >= 0 ? (size_t)bhq_n * g.S + l : 0;
-        const float lse_raw = a.lse[idx], dlt_raw = a.delta[idx];
-        if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
-        VSA2_WAIT_PARKED(&misc->stat_free, (tg & 1) ^ 1);
-        rowstat[r] = make_float2(l >= 0 ? lse_raw * 1.4426950408889634f : INFINITY, l >= 0 ? dlt_raw : 0.f);
-        tc::mbar_arrive(&misc->stat_full);
-      }
-    }
-  } else if (warp >= 4 && warp < 12) {
-    // ------------------------------------------------------------------ elementwise stage + epilogue (256 threads):
-    // warps 4..7 take key columns 0..31 of every tile, warps 8..11 columns 32..63
-    const int quad = warp & 3;
-    const int half = (warp - 4) >> 2;
-    const int row = (quad << 5) | lane;      // query row of the tile (S, dP) / channel (dK^T, dV^T)
-    const int sm_tid = tid - 128;            // 0..255
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint32_t tg = 0, n_items = 0;
-    for (uint32_t n_all = 0;; ++n_all) {
-      VSA2_NEXT_ITEM(item, n_all);
-      VSA2_DKV_ITEM_SETUP();
-      (void)col_beg;
-      const int tb = n_all & 1;
-      const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
-      if (sm_tid < 64) misc->tok[tb][sm_tid] = block_token(g, j, sm_tid);
-      uint32_t kvmask = 0xffffffffu;           // validity of this thread's 32 key columns
-      if (k > 0 && block_count(g, j) < kBlockTokens) {
-        kvmask = 0u;
-        for (int p = 0; p < 32; ++p)
-          if (block_token(g, j, half * 32 + p) >= 0) kvmask |= 1u << p;
-      }
-      float coarse_k = 0.f, coarse_v = 0.f;
-      if (a.dkc != nullptr && row < D && !block_is_text(g, j)) {
-        for (int hh = 0; hh < g.rep; ++hh) {
-          const size_t cidx = ((size_t)(b * g.Hq + hk * g.rep + hh) * g.Nvid + j) * D + row;
-          coarse_k += a.dkc[cidx];
-          coarse_v += a.dvc[cidx];
-        }
-        const float inv_cnt = 1.f / (float)cube_count(g, j);
-        coarse_k *= inv_cnt;
-        coarse_v *= inv_cnt;
-      }
-      VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0);
-      if (k > 0) {
-        const int nt = (k + 1) >> 1;
-        const float2* rowstat = reinterpret_cast<const float2*>(misc->stats);
-        for (int t = 0; t < nt; ++t, ++tg) {
-          const uint32_t s = tg & 1, par = (tg >> 1) & 1;
-          VSA2_WAIT(&misc->stat_full, tg & 1);
-          const float2 rs = rowstat[row];
-          tc::mbar_arrive(&misc->stat_free);
-          const float lse2 = rs.x, dlt = rs.y;
-          uint32_t sv[32];      // S, then P
-          VSA2_WAIT(&misc->s_full[s], par);
-          tc::tc_fence_after();
-          tc::tmem_ld32(lane_addr + s * 64 + half * 32, sv);
-          tc::tmem_ld_wait();
-          tc::tc_fence_before();
-          tc::mbar_arrive(&misc->s_free[s]);
-          {
-            uint32_t pp[16], pl[SPLIT ? 16 : 1];
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              float p0 = ex2_approx(fmaf(__uint_as_float(sv[c]), c2, -lse2));
-              float p1 = ex2_approx(fmaf(__uint_as_float(sv[c + 1]), c2, -lse2));
-              if (kvmask != 0xffffffffu) {
-                p0 = ((kvmask >> c) & 1u) ? p0 : 0.f;
-                p1 = ((kvmask >> (c + 1)) & 1u) ? p1 : 0.f;
-              }
-              sv[c] = __float_as_uint(p0);
-              sv[c + 1] = __float_as_uint(p1);
-              if constexpr (SPLIT) split_bf16x2(p0, p1, pp[c >> 1], pl[c >> 1]);
-              else pp[c >> 1] = pack_bf16x2(p0, p1);
-            }
-            VSA2_WAIT(&misc->p_free, (tg & 1) ^ 1);
-            unsigned char* prow = p_tile + row * 128;
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              *reinterpret_cast<uint4*>(prow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
-                  make_uint4(pp[4 * ch], pp[4 * ch + 1], pp[4 * ch + 2], pp[4 * ch + 3]);
-              if constexpr (SPLIT)
-                *reinterpret_cast<uint4*>(prow + C::PBYTES + (((half * 4 + ch) ^ (row & 7)) << 4)) =
-                    make_uint4(pl[4 * ch], pl[4 * ch + 1], pl[4 * ch + 2], pl[4 * ch + 3]);
-            }
-            tc::fence_proxy_async_smem();
-            tc::mbar_arrive(&misc->p_ready);
-          }
-          {
-            uint32_t dp[32], pd[16], pdl[SPLIT ? 16 : 1];
-            VSA2_WAIT(&misc->dp_full[s], par);
-            tc::tc_fence_after();
-            tc::tmem_ld32(lane_addr + 128 + s * 64 + half * 32, dp);
-            tc::tmem_ld_wait();
-            tc::tc_fence_before();
-            tc::mbar_arrive(&misc->dp_free[s]);
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              const float d0 = __uint_as_float(sv[c]) * (__uint_as_float(dp[c]) - dlt) * g.scale;
-              const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
-              if constexpr (SPLIT) split_bf16x2(d0, d1, pd[c >> 1], pdl[c >> 1]);
-              else pd[c >> 1] = pack_bf16x2(d0, d1);
-            }
-            VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
-            unsigned char* drow = ds_tile + row * 128;
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              *reinterpret_cast<uint4*>(drow + (((half * 4 + ch) ^ (row & 7)) << 4)) =
-                  make_uint4(pd[4 * ch], pd[4 * ch + 1], pd[4 * ch + 2], pd[4 * ch + 3]);
-              if constexpr (SPLIT)
-                *reinterpret_cast<uint4*>(drow + C::PBYTES + (((half * 4 + ch) ^ (row & 7)) << 4)) =
-                    make_uint4(pdl[4 * ch], pdl[4 * ch + 1], pdl[4 * ch + 2], pdl[4 * ch + 3]);
-            }
-            tc::fence_proxy_async_smem();
-            tc::mbar_arrive(&misc->ds_ready[0]);
-          }
-        }
-        VSA2_WAIT(&misc->o_full, n_items & 1);
-        tc::tc_fence_after();
-      }
-      // epilogue: dK[l, d] = dK^T[d, kv] + sum_heads dK_c[j, d] / count(j), same for dV; this thread owns 32 key columns
-      {
-        uint32_t kk[32], vv[32];
-        if (k > 0) {
-          tc::tmem_ld32(lane_addr + TM_DK + half * 32, kk);
-          tc::tmem_ld32(lane_addr + TM_DV + half * 32, vv);
-          tc::tmem_ld_wait();
-          if constexpr (SPLIT) {
-            uint32_t lo[32];
-            tc::tmem_ld32(lane_addr + TM_DK + 64 + half * 32, lo);
-            tc::tmem_ld_wait();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) kk[c] = __float_as_uint(__uint_as_float(kk[c]) + __uint_as_float(lo[c]));
-            tc::tmem_ld32(lane_addr + TM_DV + 64 + half * 32, lo);
-            tc::tmem_ld_wait();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) vv[c] = __float_as_uint(__uint_as_float(vv[c]) + __uint_as_float(lo[c]));
-          }
-          tc::tc_fence_before();
-          tc::mbar_arrive(&misc->o_empty);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) { kk[c] = 0u; vv[c] = 0u; }
-        }
-        if (g.out_f32) {
-          if (row < D) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int l = misc->tok[tb][half * 32 + c];
-              if (l < 0) continue;
-              const size_t idx = ((size_t)bhk * g.S + l) * D + row;
-              store_out(a.dk, idx, __uint_as_float(kk[c]) + coarse_k, 1);
-              store_out(a.dv, idx, __uint_as_float(vv[c]) + coarse_v, 1);
-            }
-          }
-        } else {
-          // bf16: transpose through shared memory (the P and dS buffers are idle now), then 16-byte stores
-          bf16* st_k = reinterpret_cast<bf16*>(p_tile);       // [64 kv][D]
-          bf16* st_v = reinterpret_cast<bf16*>(ds_tile);      // [64 kv][D]
-          if (row < D) {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              st_k[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(kk[c]) + coarse_k);
-              st_v[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(vv[c]) + coarse_v);
-            }
-          }
-          VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 1);
-          constexpr int CH = D / 8;
-          for (int e = sm_tid; e < 64 * CH; e += 256) {
-            const int c = e / CH, ch = e % CH;
-            const int l = misc->tok[tb][c];
-            if (l < 0) continue;
-            const size_t idx = ((size_t)bhk * g.S + l) * D + ch * 8;
-            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dk) + idx) = *reinterpret_cast<const uint4*>(st_k + c * D + ch * 8);
-            *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.dv) + idx) = *reinterpret_cast<const uint4*>(st_v + c * D + ch * 8);
-          }
-          VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 2);
-        }
-      }
-      if (k > 0) ++n_items;
-    }
-  }
-
-done:
-  tc::tc_fence_before();
-  __syncthreads();
-  if (misc->abort_flag) {
-    if (tid == 0) {
-      atomicExch(&a.status->status, VSA2_ERR_DEVICE_TIMEOUT);
-      const unsigned long long t0 = tc::global_timer_ns();
-      while (tc::global_timer_ns() - t0 < 200000ull) {
-      }
-    }
-    __syncthreads();
-  }
-  if (warp == 2) tc::tmem_dealloc(tmem_base, 512);
-}
-
-// ================================================================================================
-// launchers
-// ================================================================================================
-static cudaError_t sm_count(int* sms) {
-  int dev = 0;
-  cudaError_t e;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  return cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
-}
-
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                   const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
                                   const float* dqc, void* dq, StatusBlock* status, cudaStream_t st) {
@@ -943,7 +396,7 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
     return cudaErrorInvalidValue;
   int sms = 0;
   cudaError_t e;
-  if ((e = sm_count(&sms)) != cudaSuccess) return e;
+  if ((e = bwd_sm_count(&sms)) != cudaSuccess) return e;
   DqArgs a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, dq, status};
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
@@ -963,42 +416,6 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
     else VSA2_LAUNCH_DQ(64, false);
   }
 #undef VSA2_LAUNCH_DQ
-  return cudaGetLastError();
-}
-
-cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
-                                   const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
-                                   const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                   cudaStream_t st) {
-  if (g.rep > kMaxRep) return cudaErrorInvalidValue;
-  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
-  if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
-      !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) ||
-      !make_text_tmap(&tvt, v, g, g.Hkv) || !make_text_tmap(&tdot, d_o, g, g.Hq))
-    return cudaErrorInvalidValue;
-  int sms = 0;
-  cudaError_t e;
-  if ((e = sm_count(&sms)) != cudaSuccess) return e;
-  DkvArgs a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
-  const int total = g.batch * g.Hkv * g.N;
-  const int grid = total < sms ? total : sms;
-  const bool split = fine_bwd_dkv_wants_pair(g);
-#define VSA2_LAUNCH_DKV(DD, SP)                                                                                                  \
-  do {                                                                                                                           \
-    using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                   \
-                                  (int)L_::smem_bytes)))                                                                         \
-      return e;                                                                                                                  \
-    fine_bwd_dkv_tc_kernel<DD, SP><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                            \
-  } while (0)
-  if (g.D == 128) {
-    if (split) VSA2_LAUNCH_DKV(128, true);
-    else VSA2_LAUNCH_DKV(128, false);
-  } else {
-    if (split) VSA2_LAUNCH_DKV(64, true);
-    else VSA2_LAUNCH_DKV(64, false);
-  }
-#undef VSA2_LAUNCH_DKV
   return cudaGetLastError();
 }
 

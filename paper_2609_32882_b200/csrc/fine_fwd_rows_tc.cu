@@ -71,13 +71,6 @@ struct FwdRowsMisc {
 };
 static_assert(sizeof(FwdRowsMisc) <= 4096, "misc region too small");
 
-#ifdef VSA2_TRACE
-__device__ long long g_fr_trace[4 * 256 * 8];
-#define FR_TR(role, tile, slot) do { if (blockIdx.x == 0 && (tile) < 256u) g_fr_trace[((role) * 256 + (tile)) * 8 + (slot)] = clock64(); } while (0)
-#else
-#define FR_TR(role, tile, slot) do {} while (0)
-#endif
-
 struct FwdRowsArgs {
   int* item_counter;    // global, zero before the launch
   const float* gate;
@@ -264,11 +257,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         VSA2_WAIT(&misc->q_full[qb], (n_items / C::NQ) & 1);
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t slot = tg % kFrKSlots, buf = tg & 1;
-          if (lane == 0) FR_TR(0, tg, 0);
           VSA2_WAIT(&misc->k_full[slot], (tg / kFrKSlots) & 1);
-          if (lane == 0) FR_TR(0, tg, 1);
           VSA2_WAIT(&misc->s_free[buf], ((tg >> 1) & 1) ^ 1);
-          if (lane == 0) FR_TR(0, tg, 2);
           tc::tc_fence_after();
           if (tc::elect_one()) {
             const uint64_t dk = tc::smem_desc_sw128(slot0 + slot * C::SLOT, 16, 1024);
@@ -283,7 +273,6 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             if (t == nt - 1) tc::mma_commit(&misc->q_empty[qb]);   // the Q tile may be replaced once the last S of the block is done
           }
           __syncwarp();
-          if (lane == 0) FR_TR(0, tg, 3);
         }
         ++n_items;
       }
@@ -307,11 +296,8 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         VSA2_WAIT(&misc->o_empty, (n_items & 1) ^ 1);      // the previous query block's accumulator was read out
         for (int t = 0; t < nt; ++t, ++tg) {
           const uint32_t slot = tg % kFrVSlots, buf = tg & 1;
-          if (lane == 0) FR_TR(1, tg, 0);
           VSA2_WAIT(&misc->v_full[slot], (tg / kFrVSlots) & 1);
-          if (lane == 0) FR_TR(1, tg, 1);
           VSA2_WAIT(&misc->p_ready[buf], (tg >> 1) & 1);
-          if (lane == 0) FR_TR(1, tg, 2);
           tc::tc_fence_after();
           if (tc::elect_one()) {
             const uint64_t dv = tc::smem_desc_sw128(slot0 + slot * C::SLOT, lbo, 1024);
@@ -325,7 +311,6 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             if (t == nt - 1) tc::mma_commit(&misc->o_full);
           }
           __syncwarp();
-          if (lane == 0) FR_TR(1, tg, 3);
         }
         ++n_items;
       }
@@ -445,17 +430,14 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             ja = cols[2 * t + 4];
             jb = cols[2 * t + 5 < k ? 2 * t + 5 : 2 * t + 4];
           }
-          if (sm_tid == 0) FR_TR(2 + wg, tgt, 0);
           if (!(have_first && t == 0)) {
             VSA2_WAIT(&misc->s_full[buf], (tgt >> 1) & 1);
-            if (sm_tid == 0) FR_TR(2 + wg, tgt, 1);
             tc::tc_fence_after();
             tc::tmem_ld_16x256b_x16(lane_addr + C::TM_S + buf * 128, sv);
             tc::tmem_ld_wait();
             tc::tc_fence_before();
             tc::mbar_arrive(&misc->s_free[buf]);
           }
-          if (sm_tid == 0) FR_TR(2 + wg, tgt, 2);
           uint32_t pk[32];
           if ((ma & mb) == 0xffffu) {
 #pragma unroll
@@ -491,14 +473,11 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
               pk[2 * n + 1] = wb;
             }
           }
-          if (sm_tid == 0) FR_TR(2 + wg, tgt, 3);
           VSA2_WAIT(&misc->p_free[buf], ((tgt >> 1) & 1) ^ 1);
-          if (sm_tid == 0) FR_TR(2 + wg, tgt, 4);
           tc::tmem_st_16x128b_x16(lane_addr + C::TM_P + buf * 64, pk);
           tc::tmem_st_wait();
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->p_ready[buf]);
-          if (sm_tid == 0) FR_TR(2 + wg, tgt, 5);
         }
         tg += nt;
         // row sums: over the four threads of a row here, over the two warpgroups through shared memory
@@ -624,12 +603,6 @@ cudaError_t launch_fine_fwd_list(const Geo& g, const int* count, int cap, const 
                                  const float* oc_hat, void* o, bf16* o_res, float* lse, cudaStream_t st);
 
 bool fine_fwd_rows_supported(const Geo& g) { return g.N <= kFrMaxCubes; }
-
-#ifdef VSA2_TRACE
-extern "C" int vsa2_debug_fwd_trace(long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_fr_trace, sizeof(long long) * 4 * 256 * 8) == cudaSuccess ? 0 : -5;
-}
-#endif
 
 // workspace: [StatusBlock][rescue list] as for launch_fine_fwd_tc; the rescue counter is StatusBlock.pad[0].
 cudaError_t launch_fine_fwd_rows_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const float* gate,

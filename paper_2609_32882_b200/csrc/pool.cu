@@ -1,5 +1,7 @@
 // Mean pooling over cubes (coarse branch, paper Eq. 1) and over router sub-cubes (Eq. 5).
 // HBM-bound: every token row is read once with 16-byte loads.
+// (one cube decode per thread: this file keeps the reciprocal form of the index divisions, which measured 7 % faster here)
+#define VSA2_RECIPROCAL_DIVMOD 1
 #include "common.cuh"
 
 namespace vsa2 {
