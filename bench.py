@@ -38,8 +38,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the 720p top-64 launch with 40 heads: an
 # 8-head ncu capture of the same kernels times 5 (every head streams its own tensors, so the traffic grows in
 # proportion to the heads; the 40-head launch is too large for a full-set capture).
-NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.500836e9 + 0.294249e9), "fine_bwd_dq": 5 * (0.663055e9 + 0.146861e9),
-                                "fine_bwd_dkv": 5 * (0.769323e9 + 0.304400e9)}
+NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.498373e9 + 0.288805e9), "fine_bwd_dq": 5 * (0.666063e9 + 0.147825e9),
+                                "fine_bwd_dkv": 5 * (0.762483e9 + 0.305517e9)}
 
 
 def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None, text_len: int = 0) -> syn.Workload:

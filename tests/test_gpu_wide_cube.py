@@ -1,5 +1,6 @@
-"""GPU parity for cubes of 128 tokens (4 x 4 x 8, router pooling 2 x 2 x 2, G = 16): the CUDA path runs them as pairs
-of 64-token half-cubes; the oracle computes them directly from the definitions."""
+"""GPU parity for cubes of 128 tokens (4 x 4 x 8, router pooling 2 x 2 x 2, G = 16): the CUDA path routes and pools them as
+pairs of 64-token half-cubes and runs the fine branch on 128 x 128 tiles; the oracle computes them directly from the
+definitions."""
 import numpy as np
 import pytest
 
@@ -37,6 +38,25 @@ def test_wide_cube_whose_last_second_half_lies_outside_the_grid(wl):
 
 def test_wide_cube_fp32_outputs():
     full_parity(WIDE_RAGGED, syn.make_inputs(WIDE_RAGGED), out_dtype=vb.F32, check_route=False)
+
+
+@pytest.mark.parametrize("wl", [WIDE_RAGGED, WIDE_EMPTY_HALF], ids=lambda w: w.name)
+def test_wide_cube_gqa_with_operands_rounded_once(wl):
+    """VSA2_FLAG_FAST_BWD on a GQA problem: the dK/dV pass then runs on 128 x 128 tiles too and walks the transposed lists of
+    all query heads of a KV group in turn (by default a GQA group takes the 64-token dK/dV kernel with its bf16 pairs); the
+    dQ pass runs without the dS pair.  Held to the looser figure the flag states."""
+    from oracle import vsa2_oracle as orc
+    from vsa2_testlib import CudaPath, assert_close, oracle_arrays
+    data = syn.make_inputs(wl)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    a = oracle_arrays(data)
+    run = CudaPath(wl, data, out_dtype=vb.F32, flags=vb.FLAG_FAST_BWD)
+    gmask = run.route()
+    run.forward()
+    got = run.backward()
+    want = orc.backward(a["q"], a["k"], a["v"], a["gate"], gmask, geo, 1.0 / np.sqrt(wl.head_dim), a["do"])
+    for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
+        assert_close(name, x, y, tol_abs=2e-2 if name == "dGate" else 4e-2)
 
 
 def test_wide_cube_budget_mode_with_empty_rows():
