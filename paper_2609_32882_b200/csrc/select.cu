@@ -36,8 +36,24 @@ __global__ void __launch_bounds__(256) sel_hist_kernel(const float* __restrict__
   const int shift = seq_shift(pass);
   const unsigned dmask = seq_mask(pass);
   const unsigned* src = reinterpret_cast<const unsigned*>(pr) + (size_t)bh * n_elems;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_elems;
-       i += (long long)gridDim.x * blockDim.x) {
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x, nthr = (long long)gridDim.x * blockDim.x;
+  long long done = 0;
+  if ((n_elems & 3) == 0) {
+    // 16-byte loads, two in flight per thread (the passes after the first count almost nothing: they are pure streaming reads)
+    const uint4* src4 = reinterpret_cast<const uint4*>(src);
+    const long long n4 = n_elems >> 2;
+    for (long long i = tid; i < n4; i += 2 * nthr) {
+      const uint4 a = __ldg(src4 + i);
+      const bool two = i + nthr < n4;
+      const uint4 b = two ? __ldg(src4 + i + nthr) : make_uint4(0, 0, 0, 0);
+      const unsigned va[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if ((e < 4 || two) && (va[e] & pmask) == prefix) atomicAdd(&sh[(va[e] >> shift) & dmask], 1u);
+    }
+    done = n_elems;
+  }
+  for (long long i = done + tid; i < n_elems; i += nthr) {
     unsigned v = __ldg(src + i);
     if ((v & pmask) == prefix) atomicAdd(&sh[(v >> shift) & dmask], 1u);
   }
@@ -95,28 +111,100 @@ __global__ void __launch_bounds__(32) sel_pick_kernel(unsigned* state, const uns
   }
 }
 
-// per-sequence: count entries above / equal to tau in every row.  grid (N, BH), 128 threads
-__global__ void __launch_bounds__(128) sel_row_stats_kernel(const float* __restrict__ pr, int N,
-                                                            const unsigned* __restrict__ state, int* row_gt, int* row_eq) {
-  const int i = blockIdx.x, bh = blockIdx.y;
+// per-sequence, one read of P_r for both the counts and the emission: one warp per row writes the row's bitmap words of the
+// entries above tau (`bits_gt`) and equal to tau (`bits_eq`) and the two counts.  grid (ceil(N/8), BH), 256 threads
+__global__ void __launch_bounds__(256) sel_row_bits_kernel(const float* __restrict__ pr, int N, int words,
+                                                           const unsigned* __restrict__ state, unsigned* bits_gt,
+                                                           unsigned* bits_eq, int* row_gt, int* row_eq) {
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int bh = blockIdx.y;
+  if (i >= N) return;
   const unsigned tau = state[bh * 8 + 3];
   const unsigned* src = reinterpret_cast<const unsigned*>(pr) + ((size_t)bh * N + i) * N;
   int gt = 0, eq = 0;
-  for (int j = threadIdx.x; j < N; j += blockDim.x) {
-    unsigned v = __ldg(src + j);
-    gt += v > tau;
-    eq += v == tau;
+  constexpr int U = 8;                 // words in flight per warp (the kernel is a pure streaming read)
+  for (int w0 = 0; w0 < words; w0 += U) {
+    unsigned v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int j = (w0 + u) * 32 + lane;
+      v[u] = j < N ? __ldg(src + j) : 0u;      // (scores are non-negative: 0 is never above tau, and equal only if tau = 0
+    }                                          //  -- excluded by the j < N test below)
+    unsigned mine_g = 0u, mine_e = 0u;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int j = (w0 + u) * 32 + lane;
+      const unsigned gb = __ballot_sync(0xffffffffu, j < N && v[u] > tau);
+      const unsigned eb = __ballot_sync(0xffffffffu, j < N && v[u] == tau);
+      if (lane == u) { mine_g = gb; mine_e = eb; }
+      gt += __popc(gb);
+      eq += __popc(eb);
+    }
+    if (lane < U && w0 + lane < words) {       // lanes 0..U-1 write one word each: consecutive addresses
+      bits_gt[((size_t)bh * N + i) * words + w0 + lane] = mine_g;
+      bits_eq[((size_t)bh * N + i) * words + w0 + lane] = mine_e;
+    }
   }
-  __shared__ int sg[4], se[4];
-  for (int o = 16; o; o >>= 1) {
-    gt += __shfl_xor_sync(0xffffffffu, gt, o);
-    eq += __shfl_xor_sync(0xffffffffu, eq, o);
+  if (lane == 0) {
+    row_gt[(size_t)bh * N + i] = gt;
+    row_eq[(size_t)bh * N + i] = eq;
   }
-  if ((threadIdx.x & 31) == 0) { sg[threadIdx.x >> 5] = gt; se[threadIdx.x >> 5] = eq; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    row_gt[(size_t)bh * N + i] = sg[0] + sg[1] + sg[2] + sg[3];
-    row_eq[(size_t)bh * N + i] = se[0] + se[1] + se[2] + se[3];
+}
+
+// inclusive prefix sum over the lanes of a warp
+__device__ __forceinline__ int warp_incl_scan(int v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
+}
+
+// per-sequence: ordered emission of the kept columns from the two bitmaps (`bitmap` holds the entries above tau on entry and
+// the kept entries on return).  One warp per row, one LANE per bitmap word: the lanes count their bits, a warp scan gives every
+// word its position in the row's list, and each lane writes its own few entries (a warp per word spent 30 instructions on
+// every word, 45 words a row).  Ties at tau go to the lower column: a lane keeps the equal entries whose rank in the row is
+// below the row's quota.  grid (ceil(N/8), BH), 256 threads
+__global__ void __launch_bounds__(256) sel_emit_rows_bits_kernel(int N, int words, const unsigned* __restrict__ bits_eq,
+                                                                 const int* __restrict__ row_eq_take,
+                                                                 const int* __restrict__ row_ptr, int* col_idx,
+                                                                 unsigned* bitmap, long long nnz_cap) {
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int bh = blockIdx.y;
+  if (i >= N) return;
+  const int take = row_eq_take[(size_t)bh * N + i];
+  int pos = row_ptr[(size_t)bh * (N + 1) + i];
+  int eq_seen = 0;
+  int* out = col_idx + (size_t)bh * nnz_cap;
+  const size_t base = ((size_t)bh * N + i) * words;
+  for (int w0 = 0; w0 < words; w0 += 32) {
+    const int w = w0 + lane;
+    const unsigned gb = w < words ? bitmap[base + w] : 0u;
+    unsigned eb = w < words ? __ldg(bits_eq + base + w) : 0u;
+    const int ce = __popc(eb);
+    const int ce_incl = warp_incl_scan(ce, lane);
+    int rank = eq_seen + ce_incl - ce;             // equal entries of the row before this word
+    unsigned keep = 0u;
+    while (eb != 0u && rank < take) {
+      keep |= eb & (0u - eb);
+      eb &= eb - 1u;
+      ++rank;
+    }
+    unsigned sel = gb | keep;
+    const int c = __popc(sel);
+    const int c_incl = warp_incl_scan(c, lane);
+    int p = pos + c_incl - c;
+    if (w < words && sel != gb) bitmap[base + w] = sel;
+    while (sel != 0u) {
+      if (p < nnz_cap) out[p] = w * 32 + (__ffs(sel) - 1);
+      sel &= sel - 1u;
+      ++p;
+    }
+    pos += __shfl_sync(0xffffffffu, c_incl, 31);
+    eq_seen += __shfl_sync(0xffffffffu, ce_incl, 31);
   }
 }
 
@@ -320,7 +408,7 @@ __global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* _
   if (threadIdx.x == 0) col_ptr[(size_t)bh * (N + 1) + N] = carry;
 }
 
-// one warp per column: ordered emission of the rows that keep it.  grid (ceil(N/8), BH), 256 threads
+// one warp per column, one lane per bitmap word: ordered emission of the rows that keep it.  grid (ceil(N/8), BH), 256 threads
 __global__ void __launch_bounds__(256) sel_emit_cols_kernel(const unsigned* __restrict__ bitmap_t, int N, int words,
                                                             const int* __restrict__ col_ptr, int* row_idx,
                                                             long long nnz_cap) {
@@ -330,14 +418,18 @@ __global__ void __launch_bounds__(256) sel_emit_cols_kernel(const unsigned* __re
   const unsigned* bm = bitmap_t + ((size_t)bh * N + j) * words;
   int pos = col_ptr[(size_t)bh * (N + 1) + j];
   int* out = row_idx + (size_t)bh * nnz_cap;
-  const unsigned lt = (1u << lane) - 1u;
-  for (int w = 0; w < words; ++w) {
-    const unsigned word = __ldg(bm + w);
-    if ((word >> lane) & 1u) {
-      const int p = pos + __popc(word & lt);
-      if (p < nnz_cap) out[p] = w * 32 + lane;
+  for (int w0 = 0; w0 < words; w0 += 32) {
+    // one lane per word, as in sel_emit_rows_bits_kernel
+    unsigned word = w0 + lane < words ? __ldg(bm + w0 + lane) : 0u;
+    const int c = __popc(word);
+    const int c_incl = warp_incl_scan(c, lane);
+    int p = pos + c_incl - c;
+    while (word != 0u) {
+      if (p < nnz_cap) out[p] = (w0 + lane) * 32 + (__ffs(word) - 1);
+      word &= word - 1u;
+      ++p;
     }
-    pos += __popc(word);
+    pos += __shfl_sync(0xffffffffu, c_incl, 31);
   }
 }
 
@@ -355,15 +447,20 @@ cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, con
       sel_hist_kernel<<<dim3(chunks, BH), 256, 0, st>>>(pr, n_elems, s.state, s.hist, pass);
       sel_pick_kernel<<<BH, 32, 0, st>>>(s.state, s.hist, pass);
     }
-    sel_row_stats_kernel<<<dim3(N, BH), 128, 0, st>>>(pr, N, s.state, s.row_gt, s.row_eq);
+    // counts and bitmaps in one read of P_r (the bitmap of the entries equal to tau borrows the transposed bitmap's space)
+    sel_row_bits_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(pr, N, s.words, s.state, s.bitmap, s.bitmap_t, s.row_gt, s.row_eq);
   } else {
     sel_row_topk_kernel<<<dim3(N, BH), 256, 0, st>>>(pr, N, g.K, g.mode == VSA2_PER_QUERY_BUDGET ? budgets : nullptr,
                                                      s.row_tau, s.row_eq_take, s.row_cnt);
   }
   sel_scan_rows_kernel<<<BH, 1024, 0, st>>>(N, g.mode == VSA2_PER_SEQUENCE, s.state, s.row_gt, s.row_eq, s.row_tau,
                                             s.row_eq_take, s.row_cnt, row_ptr, g.nnz_cap, status);
-  sel_emit_rows_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(pr, N, s.words, s.row_tau, s.row_eq_take, row_ptr,
-                                                              col_idx, s.bitmap, g.nnz_cap);
+  if (g.mode == VSA2_PER_SEQUENCE)
+    sel_emit_rows_bits_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(N, s.words, s.bitmap_t, s.row_eq_take, row_ptr, col_idx,
+                                                                     s.bitmap, g.nnz_cap);
+  else
+    sel_emit_rows_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(pr, N, s.words, s.row_tau, s.row_eq_take, row_ptr,
+                                                                col_idx, s.bitmap, g.nnz_cap);
   // columns: transposed bitmap, then counts (row_gt reused as scratch), scan, ordered emission
   sel_transpose_bitmap_kernel<<<dim3(s.words, (s.words + 7) / 8, BH), 256, 0, st>>>(s.bitmap, N, s.words, s.bitmap_t);
   sel_col_count_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(s.bitmap_t, N, s.words, s.row_gt);
