@@ -306,6 +306,12 @@ int vsa2_selftest_umma(const vsa2_params* p, const void* q, const void* k, const
  * trap or hang is involved and the context stays usable. */
 int vsa2_selftest_timeout(uint32_t limit_us, int32_t* status, uint64_t* waited_ns, void* cuda_stream);
 
+/* Host-only diagnostic (no GPU, no CUDA call; the paper has no counterpart): the kernels decode cube and token indices with
+ * q = floor(n * ceil(2^32 / d) / 2^32) instead of a division.  Checks that quotient against n / d for every 0 <= n <= n_max
+ * and every divisor d_min .. d_exhaustive, and for the divisors up to d_max at every multiple of d and its two neighbours.
+ * Returns the number of wrong quotients (0 for n_max * d_max < 2^32; the library's n stay below 2^22, its d below 2^10). */
+int64_t vsa2_selftest_divmod(int32_t n_max, int32_t d_min, int32_t d_exhaustive, int32_t d_max);
+
 /* Test hook (the paper has no counterpart): number of query blocks the forward kernels may hand to the exact-maximum
  * fall-back per call, 1 .. 16384 (default 16384, which also sizes the workspace).  When more blocks than that leave the
  * safe range of the fixed-reference softmax, the surplus is not recomputed, the status word becomes VSA2_ERR_UNSUPPORTED

@@ -32,7 +32,7 @@ ERR_STATIC_SCRATCH = -8
 EXPORTS = ("vsa2_query_sizes", "vsa2_route", "vsa2_route_scores", "vsa2_attn_fwd", "vsa2_attn_bwd",
            "vsa2_device_status", "vsa2_strerror", "vsa2_profile_events", "vsa2_launch_count", "vsa2_selftest_umma", "vsa2_route_noalloc", "vsa2_last_cuda_error",
            "vsa2_gate_fwd", "vsa2_gate_bwd", "vsa2_gate_bwd_workspace_bytes", "vsa2_permute_cube_major",
-           "vsa2_selftest_timeout", "vsa2_debug_rescue_capacity")
+           "vsa2_selftest_timeout", "vsa2_debug_rescue_capacity", "vsa2_selftest_divmod")
 
 KERNELS = ("pool", "router_lse", "router_pool", "select", "coarse_fwd", "fine_fwd", "bwd_pre", "coarse_bwd",
            "fine_bwd_dq", "fine_bwd_dkv", "pool_router")
@@ -112,8 +112,10 @@ def _lib():
         lib.vsa2_debug_rescue_capacity.argtypes = [C.c_int32]
         lib.vsa2_launch_count.argtypes = []
         lib.vsa2_launch_count.restype = C.c_int64
+        lib.vsa2_selftest_divmod.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32]
+        lib.vsa2_selftest_divmod.restype = C.c_int64
         for name in EXPORTS:
-            if name not in ("vsa2_strerror", "vsa2_route_scores", "vsa2_launch_count", "vsa2_last_cuda_error"):
+            if name not in ("vsa2_strerror", "vsa2_route_scores", "vsa2_launch_count", "vsa2_last_cuda_error", "vsa2_selftest_divmod"):
                 getattr(lib, name).restype = C.c_int
         _LIB = lib
     return _LIB

@@ -65,6 +65,10 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // earlier form (a reciprocal and a fix-up) runs on the special-function unit, behind the exponentials of the softmax warps,
 // which cost a service warp of the 128-token backward 4000 cycles per tile.  A translation unit that defines
 // VSA2_RECIPROCAL_DIVMOD before including this header keeps the reciprocal form (where that measured faster).
+// (host and device: vsa2_selftest_divmod checks the multiply form on the host, exhaustively for small divisors)
+__host__ __device__ __forceinline__ int mulhi_div(int n, unsigned m) {
+  return m == 0u ? n : (int)(((unsigned long long)(unsigned)n * m) >> 32);
+}
 __device__ __forceinline__ void fast_divmod(int n, int d, unsigned m, int& q, int& r) {
 #ifdef VSA2_RECIPROCAL_DIVMOD
   (void)m;
@@ -78,7 +82,7 @@ __device__ __forceinline__ void fast_divmod(int n, int d, unsigned m, int& q, in
     r -= d;
   }
 #else
-  q = m == 0u ? n : (int)__umulhi((unsigned)n, m);
+  q = mulhi_div(n, m);
   r = n - q * d;
 #endif
 }

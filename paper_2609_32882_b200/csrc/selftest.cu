@@ -154,6 +154,26 @@ __global__ void __launch_bounds__(128) selftest_timeout_kernel(unsigned limit_us
 
 using namespace vsa2;
 
+// Host-only check of the index division the kernels use (common.cuh: q = floor(n * ceil(2^32 / d) / 2^32)): every n up to
+// n_max for every divisor d_min .. d_exhaustive, and for the larger divisors up to d_max every multiple of d and its two
+// neighbours.  Returns the number of wrong quotients.
+extern "C" int64_t vsa2_selftest_divmod(int32_t n_max, int32_t d_min, int32_t d_exhaustive, int32_t d_max) {
+  int64_t bad = 0;
+  for (int d = d_min < 1 ? 1 : d_min; d <= d_max; ++d) {
+    const unsigned m = div_magic(d);
+    if (d <= d_exhaustive) {
+      for (int n = 0; n <= n_max; ++n) bad += mulhi_div(n, m) != n / d;
+    } else {
+      for (long long k = 0; k * d <= n_max; ++k)
+        for (int e = -1; e <= 1; ++e) {
+          const long long n = k * d + e;
+          if (n >= 0 && n <= n_max) bad += mulhi_div((int)n, m) != (int)(n / d);
+        }
+    }
+  }
+  return bad;
+}
+
 extern "C" int vsa2_selftest_timeout(uint32_t limit_us, int32_t* status, uint64_t* waited_ns, void* cuda_stream) {
   if (status == nullptr || limit_us == 0 || limit_us > 100000u) return VSA2_ERR_INVALID_ARG;
   selftest_timeout_kernel<<<1, 128, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(

@@ -106,6 +106,15 @@ def test_null_pointers_are_rejected_before_any_cuda_call(lib):
     assert vb._lib().vsa2_query_sizes(None, None) == vb.ERR_INVALID_ARG
 
 
+def test_index_division_by_multiply_is_exact(lib):
+    """Every kernel decodes cube and token indices with floor(n * ceil(2^32 / d) / 2^32); the library checks that form on the
+    host against n / d: all n < 2^22 for the divisors a grid produces most (up to 64), multiples of d and their neighbours
+    for the rest up to 1024."""
+    assert lib.vsa2_selftest_divmod(1 << 22, 1, 64, 1024) == 0
+    # and the check itself bites: far outside the range the form is exact for (n d < 2^32) it reports mismatches
+    assert lib.vsa2_selftest_divmod(0x7fffffff, 1000003, 0, 1000003) > 0
+
+
 def test_strerror_covers_every_code():
     seen = set()
     for code in range(0, -9, -1):
