@@ -71,7 +71,9 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
  * relative) they alone push the worst elements of large gradients (|g| > 5) past max abs err 2e-2.  By default the dQ pass
  * always, and the dK/dV pass for GQA groups (where a KV block sums several heads), carry them as a bf16 pair -- the value
  * and the bf16 rounding of what that lost -- in one product of twice the width.  Measured on 720p / 480p samples against
- * the oracle (fp32 outputs): dQ 7e-3 instead of 2.5e-2, GQA dK 8e-3 instead of 2.6e-2; MHA dK, dV stay near 1e-2 either way. */
+ * the oracle (fp32 outputs): dQ 7e-3 instead of 2.5e-2, GQA dK 8e-3 instead of 2.6e-2; MHA dK, dV stay near 1e-2 either way.
+ * With cubes of 128 tokens the pair of the dQ pass travels along the contraction instead; a dK/dV pass that needs pairs (GQA, or
+ * VSA2_FLAG_PRECISE_BWD) runs on the 64-token halves, the others on 128 x 128 tiles. */
 enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once everywhere (dQ pass about 15 % faster, GQA dK/dV pass about 30 %) */
 enum { VSA2_FLAG_PRECISE_BWD = 8 };   /* carry the pair in the dK/dV pass for MHA as well (that pass about 35 % slower): for maps
                                          that keep only a few blocks per row, where the softmax is sharply peaked */
@@ -90,7 +92,8 @@ typedef struct vsa2_params {
   int32_t cube_t, cube_h, cube_w;              /* cube (block) shape: 64 tokens (e.g. 4,4,4), or 128 tokens with cube_w even
                                                   and rpool_w dividing cube_w/2 (the paper's 4,4,8 with R = 2,2,2: G = 16);
                                                   N, K, budgets and the block map are then in cubes of 128 tokens, and the
-                                                  library computes on the cube's two 64-token halves along w
+                                                  library routes and pools on the cube's two 64-token halves along w
+                                                  and runs the fine branch on 128 x 128 tiles
                                                   (Sec. 2.2 "Permutation", Eq. 5-7, Eq. 12) */
   int32_t rpool_t, rpool_h, rpool_w;           /* router pooling R, each divides the cube dimension */
   int32_t select_mode;                         /* VSA2_PER_* */
@@ -104,7 +107,8 @@ typedef struct vsa2_params {
                                                   dv: [batch, heads, L + Lt, D]; lse: [batch, heads_q, L + Lt]) holds the L video
                                                   tokens in raster order followed by the Lt text tokens.  The block map, the router
                                                   and the coarse branch cover the video tokens only; gate and dgate stay
-                                                  [batch, heads_q, L].  64-token cubes only. */
+                                                  [batch, heads_q, L].  With cubes of 128 tokens the fine branch then runs on the
+                                                  64-token halves (the text blocks are 64 tokens). */
   int64_t nnz_cap;                             /* capacity of col_idx/row_idx per (batch, query head); 0 => N*K.
                                                   PER_QUERY_BUDGET requires it (>= sum_i min(k_i, N)). */
 } vsa2_params;

@@ -47,7 +47,6 @@ int fill_geo(const vsa2_params* p, Geo* g) {
   const bool wide = cube_tokens == 2 * kBlockTokens;
   if (cube_tokens != kBlockTokens && !wide) return VSA2_ERR_UNSUPPORTED;
   if (wide && (p->cube_w % 2 || (p->cube_w / 2) % p->rpool_w)) return VSA2_ERR_UNSUPPORTED;
-  if (wide && p->text_len > 0) return VSA2_ERR_UNSUPPORTED;
   if (p->batch > 65535 || p->heads_q > 65535 || p->heads_q / p->heads_kv > 16) return VSA2_ERR_UNSUPPORTED;
   g->batch = p->batch; g->Hq = p->heads_q; g->Hkv = p->heads_kv; g->rep = p->heads_q / p->heads_kv; g->D = p->head_dim;
   g->T = p->grid_t; g->H = p->grid_h; g->W = p->grid_w;
@@ -103,7 +102,7 @@ struct TextMapLayout {
 TextMapLayout text_map_layout(const Geo& g, bool with_csc) {
   TextMapLayout r = {};
   if (g.Lt == 0) return r;
-  const Geo x = text_geo(g);
+  const Geo x = text_geo(wide_cube(g) ? narrow_geo(g) : g);      // (128-token cubes: the block problem of the half-cubes)
   Carver c;
   const size_t BHq = (size_t)g.batch * g.Hq;
   r.ptr = c.take(BHq * (x.N + 1) * sizeof(int));
@@ -449,12 +448,13 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
   Geo fx = n;                                   // geometry of the fine kernels' block problem
   if (g.Lt > 0) {
     // text tokens: append the text blocks to the map (in the workspace) and run the kernels on the block problem
+    // (with 128-token cubes the half-cube map built above is what gets extended, and the 64-token kernels run)
     const TextMapLayout tl = text_map_layout(g, false);
     unsigned char* tbase = at<unsigned char>(workspace, fwd_base_bytes(g));
-    fx = text_geo(g);
+    fx = text_geo(n);
     if (!fine_fwd_rows_supported(fx)) return VSA2_ERR_UNSUPPORTED;
     g_launches += 1;
-    VSA2_CUDA(launch_extend_map(g, text_blocks(g), map->row_ptr, map->col_idx, at<int>(tbase, tl.ptr), at<int>(tbase, tl.idx),
+    VSA2_CUDA(launch_extend_map(n, text_blocks(g), row_ptr, col_idx, at<int>(tbase, tl.ptr), at<int>(tbase, tl.idx),
                                 fx.nnz_cap, st));
     row_ptr = at<int>(tbase, tl.ptr);
     col_idx = at<int>(tbase, tl.idx);
@@ -541,11 +541,11 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
   if (g.Lt > 0) {
     const TextMapLayout tl = text_map_layout(g, true);
     unsigned char* tbase = at<unsigned char>(workspace, bwd_base_bytes(g));
-    fx = text_geo(g);
+    fx = text_geo(n);
     g_launches += 2;
-    VSA2_CUDA(launch_extend_map(g, text_blocks(g), map->row_ptr, map->col_idx, at<int>(tbase, tl.ptr), at<int>(tbase, tl.idx),
+    VSA2_CUDA(launch_extend_map(n, text_blocks(g), row_ptr, col_idx, at<int>(tbase, tl.ptr), at<int>(tbase, tl.idx),
                                 fx.nnz_cap, st));
-    VSA2_CUDA(launch_extend_map(g, text_blocks(g), map->col_ptr, map->row_idx, at<int>(tbase, tl.cptr), at<int>(tbase, tl.ridx),
+    VSA2_CUDA(launch_extend_map(n, text_blocks(g), col_ptr, row_idx, at<int>(tbase, tl.cptr), at<int>(tbase, tl.ridx),
                                 fx.nnz_cap, st));
     row_ptr = at<int>(tbase, tl.ptr);
     col_idx = at<int>(tbase, tl.idx);

@@ -101,11 +101,17 @@ def test_text_tokens_with_empty_video_rows():
     assert np.array_equal(run.mask.sum(axis=-1), data["budgets"])
 
 
-def test_text_tokens_are_refused_for_cubes_of_128_tokens():
-    with pytest.raises(vb.Vsa2Error) as e:
-        vb.vsa2_query_sizes(vb.make_params(batch=1, heads_q=2, heads_kv=2, head_dim=128, grid=(4, 8, 16), cube=(4, 4, 8), topk=2,
-                                           text_len=10))
-    assert e.value.code == vb.ERR_UNSUPPORTED
+@pytest.mark.parametrize("wl,dt", [
+    (syn.Workload("text_wide_gqa", 1, 4, 2, 128, (7, 10, 29), select_mode=syn.PER_QUERY, topk=3, seed=56, text_len=100,
+                  cube=(4, 4, 8), rpool=(2, 2, 2)), vb.BF16),
+    (syn.Workload("text_wide_per_sequence", 1, 2, 2, 64, (8, 8, 32), select_mode=syn.PER_SEQUENCE, topk=4, seed=57, text_len=70,
+                  cube=(4, 4, 8), rpool=(2, 2, 2)), vb.F32),
+], ids=lambda x: x.name if hasattr(x, "name") else str(x))
+def test_text_tokens_with_cubes_of_128_tokens(wl, dt):
+    """The paper's own cube with text tokens: the map is expanded to the 64-token halves, the text blocks are appended to that
+    block problem, and the 64-token kernels run it."""
+    run = run_case(wl, out_dtype=dt)
+    assert run.attn.sizes.block_tokens == 128
 
 
 def test_zero_text_tokens_is_the_plain_problem():
