@@ -197,12 +197,16 @@ __global__ void __launch_bounds__(256) sel_emit_rows_bits_kernel(int N, int word
     const int c = __popc(sel);
     const int c_incl = warp_incl_scan(c, lane);
     int p = pos + c_incl - c;
-    if (w < words && sel != gb) bitmap[base + w] = sel;
-    while (sel != 0u) {
-      if (p < nnz_cap) out[p] = w * 32 + (__ffs(sel) - 1);
+    unsigned kept = 0u;                              // (entries past the capacity of the map are dropped from the bitmap too,
+    while (sel != 0u) {                              //  so that the transposed map lists exactly the pairs emitted here)
+      if (p < nnz_cap) {
+        out[p] = w * 32 + (__ffs(sel) - 1);
+        kept |= sel & (0u - sel);
+      }
       sel &= sel - 1u;
       ++p;
     }
+    if (w < words && kept != gb) bitmap[base + w] = kept;
     pos += __shfl_sync(0xffffffffu, c_incl, 31);
     eq_seen += __shfl_sync(0xffffffffu, ce_incl, 31);
   }
@@ -315,11 +319,13 @@ __global__ void __launch_bounds__(1024) sel_scan_rows_kernel(int N, int per_sequ
     int c = i < N ? row_cnt[base + i] : 0;
     int tot;
     int pre = carry + block_excl_scan(c, ws, tot);
-    if (i < N) row_ptr[(size_t)bh * (N + 1) + i] = pre;
+    // (an overflowing selection is reported below; its row pointers stop at the capacity, so that every later reader of
+    // the map stays inside col_idx: rows past the capacity are empty, the row that crosses it is cut)
+    if (i < N) row_ptr[(size_t)bh * (N + 1) + i] = (int)min((long long)pre, nnz_cap);
     carry += tot;
   }
   if (threadIdx.x == 0) {
-    row_ptr[(size_t)bh * (N + 1) + N] = carry;
+    row_ptr[(size_t)bh * (N + 1) + N] = (int)min((long long)carry, nnz_cap);
     if ((long long)carry > nnz_cap) atomicExch(&status->status, VSA2_ERR_MAP_OVERFLOW);
   }
 }
@@ -349,13 +355,13 @@ __global__ void __launch_bounds__(256) sel_emit_rows_kernel(const float* __restr
     unsigned eqb = __ballot_sync(0xffffffffu, eq);
     bool sel = gt || (eq && (eq_seen + __popc(eqb & lt)) < take);
     unsigned selb = __ballot_sync(0xffffffffu, sel);
-    if (sel) {
-      int p = pos + __popc(selb & lt);
-      if (p < nnz_cap) out[p] = j;
-    }
+    const int p = pos + __popc(selb & lt);
+    const bool emit = sel && p < nnz_cap;            // (entries past the capacity of the map are dropped from the bitmap too,
+    if (emit) out[p] = j;                            //  so that the transposed map lists exactly the pairs emitted here)
+    const unsigned keptb = __ballot_sync(0xffffffffu, emit);
     pos += __popc(selb);
     eq_seen += __popc(eqb);
-    if (lane == 0) bitmap[((size_t)bh * N + i) * words + w] = selb;
+    if (lane == 0) bitmap[((size_t)bh * N + i) * words + w] = keptb;
   }
 }
 
@@ -393,7 +399,8 @@ __global__ void __launch_bounds__(256) sel_col_count_kernel(const unsigned* __re
   if (lane == 0) col_cnt[(size_t)bh * N + j] = c;
 }
 
-__global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* __restrict__ col_cnt, int* col_ptr) {
+__global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* __restrict__ col_cnt, int* col_ptr,
+                                                             long long nnz_cap) {
   __shared__ int ws[33];
   const int bh = blockIdx.x;
   int carry = 0;
@@ -402,10 +409,10 @@ __global__ void __launch_bounds__(1024) sel_scan_cols_kernel(int N, const int* _
     int c = j < N ? col_cnt[(size_t)bh * N + j] : 0;
     int tot;
     int pre = carry + block_excl_scan(c, ws, tot);
-    if (j < N) col_ptr[(size_t)bh * (N + 1) + j] = pre;
+    if (j < N) col_ptr[(size_t)bh * (N + 1) + j] = (int)min((long long)pre, nnz_cap);      // (as for the rows)
     carry += tot;
   }
-  if (threadIdx.x == 0) col_ptr[(size_t)bh * (N + 1) + N] = carry;
+  if (threadIdx.x == 0) col_ptr[(size_t)bh * (N + 1) + N] = (int)min((long long)carry, nnz_cap);
 }
 
 // one warp per column, one lane per bitmap word: ordered emission of the rows that keep it.  grid (ceil(N/8), BH), 256 threads
@@ -464,7 +471,7 @@ cudaError_t launch_select(const Geo& g, const float* pr, const int* budgets, con
   // columns: transposed bitmap, then counts (row_gt reused as scratch), scan, ordered emission
   sel_transpose_bitmap_kernel<<<dim3(s.words, (s.words + 7) / 8, BH), 256, 0, st>>>(s.bitmap, N, s.words, s.bitmap_t);
   sel_col_count_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(s.bitmap_t, N, s.words, s.row_gt);
-  sel_scan_cols_kernel<<<BH, 1024, 0, st>>>(N, s.row_gt, col_ptr);
+  sel_scan_cols_kernel<<<BH, 1024, 0, st>>>(N, s.row_gt, col_ptr, g.nnz_cap);
   sel_emit_cols_kernel<<<dim3((N + 7) / 8, BH), 256, 0, st>>>(s.bitmap_t, N, s.words, col_ptr, row_idx, g.nnz_cap);
   return cudaGetLastError();
 }

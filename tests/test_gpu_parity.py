@@ -187,6 +187,40 @@ def test_forward_survives_a_late_dominant_key_block():
     assert rescued >= 1
 
 
+def test_map_overflow_is_reported_and_the_truncated_map_stays_inside_its_capacity():
+    """Per-row budgets that need more entries than nnz_cap: vsa2_route reports VSA2_ERR_MAP_OVERFLOW, the row and column
+    pointers stop at the capacity (rows past it are empty, the row that crosses it is cut), and forward + backward on that
+    map compute the attention of exactly the truncated map (CSR and CSC list the same pairs)."""
+    from oracle import vsa2_oracle as orc
+    from vsa2_testlib import CudaPath, assert_close, assert_lse_close, csr_to_mask, oracle_arrays, to_f64
+    wl = MINI_BUDGET
+    data = syn.make_inputs(wl)
+    N = wl.n_cubes
+    data["budgets"] = np.full((wl.batch, wl.heads_q, N), 3, dtype=np.int32)
+    cap = 3 * N - 7                                  # seven entries short
+    run = CudaPath(wl, data, out_dtype=vb.F32, nnz_cap=cap)
+    run.attn.route(run.q, run.k, run.budgets)
+    with pytest.raises(vb.Vsa2Error) as e:
+        run.attn.check_status()
+    assert e.value.code == vb.ERR_MAP_OVERFLOW
+    rp, ci, cp, ri = (t.cpu().numpy() for t in run.attn.map_views())
+    assert rp.max() == cap and cp.max() <= cap and (np.diff(rp, axis=-1) >= 0).all() and (np.diff(cp, axis=-1) >= 0).all()
+    mask = csr_to_mask(rp, ci, N)
+    counts = mask.sum(axis=-1)
+    assert (counts[..., :-3] == 3).all() and counts.sum(axis=-1).max() == cap       # only the last rows are cut
+    O, lse = run.attn.forward(run.q, run.k, run.v, run.gate)
+    a = oracle_arrays(data)
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    O_ref, lse_ref = orc.forward(a["q"], a["k"], a["v"], a["gate"], mask, geo, 1.0 / np.sqrt(wl.head_dim))
+    assert_close("O", to_f64(O), O_ref)
+    assert_lse_close(to_f64(lse), lse_ref)
+    assert np.array_equal(np.swapaxes(csr_to_mask(cp, ri, N), -1, -2), mask), "the transposed map lists other pairs"
+    got = run.attn.backward(run.q, run.k, run.v, run.gate, O, lse, run.do)
+    want = orc.backward(a["q"], a["k"], a["v"], a["gate"], mask, geo, 1.0 / np.sqrt(wl.head_dim), a["do"])
+    for name, x, y in zip(("dQ", "dK", "dV", "dGate"), got, want):
+        assert_close(name, to_f64(x), y)
+
+
 def test_rescue_list_overflow_is_reported_and_stays_inside_the_list():
     """More query blocks leave the safe range of the fixed-reference softmax than the rescue list may hold (capacity
     lowered to 1 through the test hook): the status word reports it, the list holds exactly one entry, the words behind
