@@ -1,9 +1,10 @@
 // dK/dV pass of the backward of the fine branch (gradient of paper Eq. 12) on the Blackwell tensor cores: the formulation,
 // the shared-memory plan and the dQ pass are in fine_bwd_tc.cu / fine_bwd_tc.cuh.
 //
-// This translation unit keeps the reciprocal form of the index divisions (common.cuh): the pass measured 5 % slower with
-// the multiply form (A/B on one GPU at 720p: 18.1 against 19.0 ms), while every other kernel gained from it.
-#define VSA2_RECIPROCAL_DIVMOD 1
+// The pass runs at the edge of the SM's instruction cache (about 32 KB; a miss goes to a cache that the SMs of a GPC share
+// and that saturates): with 87 KB of code its hit rate was 90 % and the time moved by several per cent with any change of
+// the code's size or layout.  What is executed per tile and per item is therefore kept small: one query head per KV head
+// is a template case of its own, the key-column mask comes from the token table, index divisions are multiplies.
 #include "fine_bwd_tc.cuh"
 
 namespace vsa2 {
@@ -29,11 +30,11 @@ constexpr int kMaxRep = 16;   // query heads per KV head the dK/dV pass supports
 // entry e of the concatenated column lists of the group's query heads -> (query head, query block)
 // (`cnt_prefix`, `col_beg`: per-head counts prefix and list starts of the item, read once per item so that this lookup
 // costs a single global load)
-__device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b, int hk, const int* cnt_prefix,
+__device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int rep, int b, int hk, const int* cnt_prefix,
                                           const int* col_beg, int e, int& bhq, int& i) {
   int hh = 0;
-  while (hh + 1 < g.rep && e >= cnt_prefix[hh + 1]) ++hh;
-  bhq = b * g.Hq + hk * g.rep + hh;
+  while (hh + 1 < rep && e >= cnt_prefix[hh + 1]) ++hh;
+  bhq = b * g.Hq + hk * rep + hh;
   i = a.row_idx[(size_t)bhq * g.nnz_cap + col_beg[hh] + (e - cnt_prefix[hh])];
 }
 
@@ -47,7 +48,10 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int b,
 // accumulator halves that the epilogue adds), which removes their bf16 rounding from dV and dK: a KV block sums hundreds of
 // query blocks (times the query heads of a GQA group), and with plain bf16 operands that noise alone passes 2e-2.  The two
 // extra operand buffers take the place of the third ring-A slot.
-template <int D, bool SPLIT>
+// MHA: one query head per KV head (g.rep == 1): the per-head prefix of the column lists and the search in it fold away,
+// which takes several KB out of every role's per-item code and out of the producers' and statistics warps' tile loops
+// (the pass runs at the edge of the SM's instruction cache).
+template <int D, bool SPLIT, bool MHA>
 __global__ void __launch_bounds__(kDkvThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -68,6 +72,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_items = g.batch * g.Hkv * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
+  const int rep = MHA ? 1 : g.rep;
 
   if (tid == 0) {
     bwd_init_barriers(misc);
@@ -95,14 +100,14 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   int j, bhk;                                                                            \
   item_block(g, item, bhk, j);                                                           \
   const int b = bhk / g.Hkv, hk = bhk % g.Hkv;                                           \
-  int cnt_prefix[kMaxRep + 1], col_beg[kMaxRep];                                         \
+  int cnt_prefix[(MHA ? 1 : kMaxRep) + 1], col_beg[MHA ? 1 : kMaxRep];                   \
   cnt_prefix[0] = 0;                                                                     \
-  for (int hh = 0; hh < g.rep; ++hh) {                                                   \
-    const size_t base_ = (size_t)(b * g.Hq + hk * g.rep + hh) * (g.N + 1) + j;           \
+  for (int hh = 0; hh < rep; ++hh) {                                                     \
+    const size_t base_ = (size_t)(b * g.Hq + hk * rep + hh) * (g.N + 1) + j;             \
     col_beg[hh] = a.col_ptr[base_];                                                      \
     cnt_prefix[hh + 1] = cnt_prefix[hh] + (a.col_ptr[base_ + 1] - col_beg[hh]);          \
   }                                                                                      \
-  const int k = cnt_prefix[g.rep];
+  const int k = cnt_prefix[rep];
 
   if (warp < 2) {
     // ------------------------------------------------------------------ TMA producers
@@ -142,13 +147,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       ++n_items;
       const int nt = (k + 1) >> 1;
       int bhq_l, i_l;           // this lane's entry of the tile, fetched one tile ahead of the slot wait
-      dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && k > 1) ? 1 : 0, bhq_l, i_l);
+      dkv_entry(g, a, rep, b, hk, cnt_prefix, col_beg, (my_blk == 1 && k > 1) ? 1 : 0, bhq_l, i_l);
       for (int t = 0; t < nt; ++t, ++tg) {
         int c1, c2, c3;
         block_box(g, i_l, c1, c2, c3);
         const CUtensorMap* tm_i = block_is_text(g, i_l) ? tm_text : tm;
         const int bhq_t = bhq_l;
-        if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
+        if (t + 1 < nt) dkv_entry(g, a, rep, b, hk, cnt_prefix, col_beg, (my_blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_l, i_l);
         if (which == 0) VSA2_RING_LOAD(misc->a_full, misc->a_empty, RA, smem, tm_i, tg, c3, c2, c1, bhq_t, {}, mbar_wait_parked);
         else VSA2_RING_LOAD(misc->b_full, misc->b_empty, kRingB, smem + C::OFF_RING_B, tm_i, tg, c3, c2, c1, bhq_t, {}, mbar_wait_parked);
       }
@@ -253,13 +258,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (k == 0) continue;
       const int nt = (k + 1) >> 1;
       int bhq_n, i_n;
-      dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
+      dkv_entry(g, a, rep, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
       for (int t = 0; t < nt; ++t, ++tg) {
         const bool dup = (blk == 1) && (2 * t + 1 >= k);
         const int l = dup ? -1 : block_token(g, i_n, r & 63);
         const size_t idx = l >= 0 ? (size_t)bhq_n * g.S + l : 0;
         const float lse_raw = a.lse[idx], dlt_raw = a.delta[idx];
-        if (t + 1 < nt) dkv_entry(g, a, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
+        if (t + 1 < nt) dkv_entry(g, a, rep, b, hk, cnt_prefix, col_beg, (blk == 1 && 2 * t + 3 < k) ? 2 * t + 3 : 2 * t + 2, bhq_n, i_n);
         VSA2_WAIT_PARKED(&misc->stat_free, (tg & 1) ^ 1);
         rowstat[r] = make_float2(l >= 0 ? lse_raw * 1.4426950408889634f : INFINITY, l >= 0 ? dlt_raw : 0.f);
         tc::mbar_arrive(&misc->stat_full);
@@ -281,16 +286,10 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const int tb = n_all & 1;
       const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
       if (sm_tid < 64) misc->tok[tb][sm_tid] = block_token(g, j, sm_tid);
-      uint32_t kvmask = 0xffffffffu;           // validity of this thread's 32 key columns
-      if (k > 0 && block_count(g, j) < kBlockTokens) {
-        kvmask = 0u;
-        for (int p = 0; p < 32; ++p)
-          if (block_token(g, j, half * 32 + p) >= 0) kvmask |= 1u << p;
-      }
       float coarse_k = 0.f, coarse_v = 0.f;
       if (a.dkc != nullptr && row < D && !block_is_text(g, j)) {
-        for (int hh = 0; hh < g.rep; ++hh) {
-          const size_t cidx = ((size_t)(b * g.Hq + hk * g.rep + hh) * g.Nvid + j) * D + row;
+        for (int hh = 0; hh < rep; ++hh) {
+          const size_t cidx = ((size_t)(b * g.Hq + hk * rep + hh) * g.Nvid + j) * D + row;
           coarse_k += a.dkc[cidx];
           coarse_v += a.dvc[cidx];
         }
@@ -299,6 +298,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         coarse_v *= inv_cnt;
       }
       VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0);
+      uint32_t kvmask = 0xffffffffu;           // validity of this thread's 32 key columns, from the token table
+      if (k > 0 && block_count(g, j) < kBlockTokens) {
+        kvmask = 0u;
+#pragma unroll 1
+        for (int p = 0; p < 32; ++p)
+          if (misc->tok[tb][half * 32 + p] >= 0) kvmask |= 1u << p;
+      }
       if (k > 0) {
         const int nt = (k + 1) >> 1;
         const float2* rowstat = reinterpret_cast<const float2*>(misc->stats);
@@ -473,20 +479,25 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
   const bool split = fine_bwd_dkv_wants_pair(g);
-#define VSA2_LAUNCH_DKV(DD, SP)                                                                                                  \
+#define VSA2_LAUNCH_DKV(DD, SP, MH)                                                                                                \
   do {                                                                                                                           \
     using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                   \
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize,               \
                                   (int)L_::smem_bytes)))                                                                         \
       return e;                                                                                                                  \
-    fine_bwd_dkv_tc_kernel<DD, SP><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                            \
+    fine_bwd_dkv_tc_kernel<DD, SP, MH><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                        \
   } while (0)
+  const bool mha = g.rep == 1;
   if (g.D == 128) {
-    if (split) VSA2_LAUNCH_DKV(128, true);
-    else VSA2_LAUNCH_DKV(128, false);
+    if (split && mha) VSA2_LAUNCH_DKV(128, true, true);
+    else if (split) VSA2_LAUNCH_DKV(128, true, false);
+    else if (mha) VSA2_LAUNCH_DKV(128, false, true);
+    else VSA2_LAUNCH_DKV(128, false, false);
   } else {
-    if (split) VSA2_LAUNCH_DKV(64, true);
-    else VSA2_LAUNCH_DKV(64, false);
+    if (split && mha) VSA2_LAUNCH_DKV(64, true, true);
+    else if (split) VSA2_LAUNCH_DKV(64, true, false);
+    else if (mha) VSA2_LAUNCH_DKV(64, false, true);
+    else VSA2_LAUNCH_DKV(64, false, false);
   }
 #undef VSA2_LAUNCH_DKV
   return cudaGetLastError();
