@@ -573,8 +573,8 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
       VSA2_CUDA(launch_expand_rows(n, n.Hq, true, dvc_cube, dvc, st));
     }
   }
-  // cubes of 128 tokens: both passes on 128 x 128 tiles (temporary switch: flag 2048 keeps the 64-token kernels)
-  const bool wide128 = wide && g.Lt == 0 && fine_bwd128_supported(n) && !(g.flags & 2048);
+  // cubes of 128 tokens: both passes on 128 x 128 tiles
+  const bool wide128 = wide && g.Lt == 0 && fine_bwd128_supported(n);
   {
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, 1);
     if (wide128)
