@@ -86,6 +86,20 @@ struct FwdRowsArgs {
   int rescue_cap;
 };
 
+// 4 x 4 transpose of 32-bit words among the four lanes of a quad (cq = lane % 4): in, lane c holds x[n] = word c of chunk n;
+// out, lane c holds the four words of chunk c in order.  Two rounds of exchanges (lane distance 1, then 2).
+__device__ __forceinline__ void quad_transpose4(uint32_t (&x)[4], int cq) {
+  const bool b0 = cq & 1, b1 = cq & 2;
+  {
+    const uint32_t r0 = __shfl_xor_sync(0xffffffffu, b0 ? x[0] : x[1], 1), r1 = __shfl_xor_sync(0xffffffffu, b0 ? x[2] : x[3], 1);
+    if (b0) { x[0] = r0; x[2] = r1; } else { x[1] = r0; x[3] = r1; }
+  }
+  {
+    const uint32_t r0 = __shfl_xor_sync(0xffffffffu, b1 ? x[0] : x[2], 2), r1 = __shfl_xor_sync(0xffffffffu, b1 ? x[1] : x[3], 2);
+    if (b1) { x[0] = r0; x[1] = r1; } else { x[2] = r0; x[3] = r1; }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kFrThreads, 1)
 fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -520,54 +534,64 @@ fine_fwd_rows_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 
       // O[l, d] = O_acc[q, d] / (rounded row sum) + gate[q] * O_c[d]; this warpgroup owns COLS output columns
       {
-        constexpr int NR = COLS / 2;              // registers per thread: 2 rows x COLS / 4 columns
-        uint32_t acc[NR];
-        if (k > 0) {
-          if constexpr (D == 128) tc::tmem_ld_16x256b_x8(lane_addr + C::TM_O + wg * COLS, acc);
-          else tc::tmem_ld_16x256b_x4(lane_addr + C::TM_O + wg * COLS, acc);
-          tc::tmem_ld_wait();
-          tc::tc_fence_before();
-          tc::mbar_arrive(&misc->o_empty);
-        } else {
-#pragma unroll
-          for (int c = 0; c < NR; ++c) acc[c] = 0u;
-        }
+        // The accumulator is read in slices of 32 columns inside a rolled loop: what runs once per query block is fetched
+        // from the instruction cache once per query block (the tile loop has evicted it by then).
         const float ga = misc->gate[tb][row_a], gb = misc->gate[tb][row_b];
         const int ta = misc->tok[tb][row_a], tk_b = misc->tok[tb][row_b];
-        if (g.out_f32) {
-#pragma unroll
-          for (int n = 0; n < COLS / 8; ++n) {
-            const int col = wg * COLS + 8 * n + 2 * cq;
-            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[tb][col]);
-            if (ta >= 0)
-              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.S + ta) * D + col) =
-                  make_float2(fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a));
-            if (tk_b >= 0)
-              *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + ((size_t)bhq * g.S + tk_b) * D + col) =
-                  make_float2(fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b));
-          }
-        } else {
-          // bf16 output and its rounding residual: a thread stores bf16 pairs, the four threads of a row 16 contiguous bytes;
-          // the eight column groups of a row complete its 128-byte lines within the same loop, so L2 merges them
-          bf16* ob = reinterpret_cast<bf16*>(a.o);
-#pragma unroll
-          for (int n = 0; n < COLS / 8; ++n) {
-            const int col = wg * COLS + 8 * n + 2 * cq;
-            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[tb][col]);
-            const float v0 = fmaf(ga, oc2.x, __uint_as_float(acc[4 * n]) * inv_a), v1 = fmaf(ga, oc2.y, __uint_as_float(acc[4 * n + 1]) * inv_a);
-            const float v2 = fmaf(gb, oc2.x, __uint_as_float(acc[4 * n + 2]) * inv_b), v3 = fmaf(gb, oc2.y, __uint_as_float(acc[4 * n + 3]) * inv_b);
-            uint32_t ha, la2, hb, lb2;
-            split_bf16x2(v0, v1, ha, la2);
-            split_bf16x2(v2, v3, hb, lb2);
-            if (ta >= 0) {
-              const size_t idx = ((size_t)bhq * g.S + ta) * D + col;
-              *reinterpret_cast<uint32_t*>(ob + idx) = ha;
-              if (a.o_res != nullptr) *reinterpret_cast<uint32_t*>(a.o_res + idx) = la2;
+        bf16* ob = reinterpret_cast<bf16*>(a.o);
+        const size_t base_a = ((size_t)bhq * g.S + (ta >= 0 ? ta : 0)) * D + wg * COLS, base_b = ((size_t)bhq * g.S + (tk_b >= 0 ? tk_b : 0)) * D + wg * COLS;
+#pragma unroll 1
+        for (int n0 = 0; n0 < COLS / 8; n0 += 4) {
+          uint32_t acc[16];
+          if (k > 0) {
+            tc::tmem_ld_16x256b_x4(lane_addr + C::TM_O + wg * COLS + 8 * n0, acc);
+            tc::tmem_ld_wait();
+            if (n0 + 4 >= COLS / 8) {
+              tc::tc_fence_before();
+              tc::mbar_arrive(&misc->o_empty);
             }
-            if (tk_b >= 0) {
-              const size_t idx = ((size_t)bhq * g.S + tk_b) * D + col;
-              *reinterpret_cast<uint32_t*>(ob + idx) = hb;
-              if (a.o_res != nullptr) *reinterpret_cast<uint32_t*>(a.o_res + idx) = lb2;
+          } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) acc[c] = 0u;
+          }
+          float v[16];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float2 oc2 = *reinterpret_cast<const float2*>(&misc->oc[tb][wg * COLS + 8 * (n0 + u) + 2 * cq]);
+            v[4 * u] = fmaf(ga, oc2.x, __uint_as_float(acc[4 * u]) * inv_a);
+            v[4 * u + 1] = fmaf(ga, oc2.y, __uint_as_float(acc[4 * u + 1]) * inv_a);
+            v[4 * u + 2] = fmaf(gb, oc2.x, __uint_as_float(acc[4 * u + 2]) * inv_b);
+            v[4 * u + 3] = fmaf(gb, oc2.y, __uint_as_float(acc[4 * u + 3]) * inv_b);
+          }
+          if (g.out_f32) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int col = 8 * (n0 + u) + 2 * cq;
+              if (ta >= 0) *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + base_a + col) = make_float2(v[4 * u], v[4 * u + 1]);
+              if (tk_b >= 0) *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.o) + base_b + col) = make_float2(v[4 * u + 2], v[4 * u + 3]);
+            }
+          } else {
+            // bf16 output and its rounding residual.  A thread holds bf16 pairs (columns 8n + 2cq, +1 of its two rows); stored
+            // as such, every warp store touched eight lines with 16 bytes each and the 32 stores per thread kept the SM's
+            // store path busy for ~2000 cycles per query block (clock64 trace: 3500 cycles from the last product to the end
+            // of the epilogue).  The four threads of a row transpose 4 x 4 words with shuffles, so that a thread stores 16
+            // contiguous bytes: 8 stores per thread instead of 32.
+            uint32_t ha[4], la4[4], hb[4], lb4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              split_bf16x2(v[4 * u], v[4 * u + 1], ha[u], la4[u]);
+              split_bf16x2(v[4 * u + 2], v[4 * u + 3], hb[u], lb4[u]);
+            }
+            quad_transpose4(ha, cq);
+            quad_transpose4(hb, cq);
+            const int col = 8 * (n0 + cq);
+            if (ta >= 0) *reinterpret_cast<uint4*>(ob + base_a + col) = make_uint4(ha[0], ha[1], ha[2], ha[3]);
+            if (tk_b >= 0) *reinterpret_cast<uint4*>(ob + base_b + col) = make_uint4(hb[0], hb[1], hb[2], hb[3]);
+            if (a.o_res != nullptr) {
+              quad_transpose4(la4, cq);
+              quad_transpose4(lb4, cq);
+              if (ta >= 0) *reinterpret_cast<uint4*>(a.o_res + base_a + col) = make_uint4(la4[0], la4[1], la4[2], la4[3]);
+              if (tk_b >= 0) *reinterpret_cast<uint4*>(a.o_res + base_b + col) = make_uint4(lb4[0], lb4[1], lb4[2], lb4[3]);
             }
           }
         }
