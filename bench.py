@@ -42,6 +42,11 @@ NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.498373e9 + 0.288805e9), "fine
                                 "fine_bwd_dkv": 5 * (0.762483e9 + 0.305517e9)}
 
 
+# L2 -> SM read rate that ncu reports as the sustained peak of this part (derived__lts__lts2xbar_bytes.sum.peak_sustained
+# in the 8-head capture of profiles/kernels_720p_8heads_ncu_full.md, where the fine forward itself reads 12.0 TB/s).
+NCU_L2_TO_SM_PEAK_TBS = 11.776
+
+
 def workload(config: int, heads: int = 0, topk: int = 0, grid=None, cube=None, text_len: int = 0) -> syn.Workload:
     wl = syn.CONFIGS[config]
     if text_len:
@@ -432,6 +437,13 @@ def run_ours(args):
                 "peak_kind": pk_kind + " sustained bf16",
                 "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant]}
     fine_fwd_tf = flops["fine_fwd"] / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
+    # operand bytes the fine forward has to bring into shared memory: a K and a V tile per selected (query block, KV block)
+    # pair and a Q tile per query block, in bf16 -- none of it can be reused between the query blocks of a head, whose
+    # lists differ, so this is the kernel's compulsory L2 -> SM traffic
+    blk = 64
+    q_rows = 128 if (wl.cube[0] * wl.cube[1] * wl.cube[2] == 128 or (args.flags & 256)) else 64   # query rows that share a K / V tile
+    fwd_tile_bytes = nnz_total * 2 * blk * wl.head_dim * 2 * blk // q_rows
+    fwd_l2_tbs = fwd_tile_bytes / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
     bytes_in = sum(host[k].numel() * host[k].element_size() for k in host)
     bytes_out = sum(t.numel() * t.element_size() for k, t in host_out.items() if k == "o" or not args.forward_only)
 
@@ -491,7 +503,12 @@ def run_ours(args):
         "cpu_baseline": cpu_baseline,
         "actual_tflops": executed / (ms_step * 1e-3) / 1e12 * world,
         "fine_fwd": {"ms": kernel_ms["fine_fwd"], "tflops": fine_fwd_tf, "frac_of_sustained_peak": fine_fwd_tf / peak_tf,
-                     "frac_of_burst_peak": fine_fwd_tf / pk["bf16_tflops"], "frac_of_nominal_2250": fine_fwd_tf / 2250.0},
+                     "frac_of_burst_peak": fine_fwd_tf / pk["bf16_tflops"], "frac_of_nominal_2250": fine_fwd_tf / 2250.0,
+                     "l2_to_sm": {"bytes_per_launch": fwd_tile_bytes, "achieved_tbs": fwd_l2_tbs, "peak_tbs": NCU_L2_TO_SM_PEAK_TBS,
+                                  "frac": fwd_l2_tbs / NCU_L2_TO_SM_PEAK_TBS,
+                                  "what": "K and V tiles of every selected block pair (64 FLOP per byte at D = 128 with 64 query rows per tile); "
+                                          "peak = the sustained L2 -> SM rate ncu reports (at the profiled clock, so a run at a higher "
+                                          "clock can read above 1); with 64-token cubes this rate, not the tensor pipe, bounds the kernel"}},
         "kernel_ms": kernel_ms,
         "gate": gate_info,
         "paper_context": "paper reports 8.9x attention speed-up over FlashAttention-3 on one H800 at 220K tokens (not comparable)",
