@@ -359,8 +359,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc::mbar_arrive(&misc->dp_free[s]);
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
-              const float d0 = __uint_as_float(sv[c]) * (__uint_as_float(dp[c]) - dlt) * g.scale;
-              const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt) * g.scale;
+              const float d0 = __uint_as_float(sv[c]) * (__uint_as_float(dp[c]) - dlt);
+              const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt);
               if constexpr (SPLIT) split_bf16x2(d0, d1, pd[c >> 1], pdl[c >> 1]);
               else pd[c >> 1] = pack_bf16x2(d0, d1);
             }
@@ -381,7 +381,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
       }
-      // epilogue: dK[l, d] = dK^T[d, kv] + sum_heads dK_c[j, d] / count(j), same for dV; this thread owns 32 key columns
+      // epilogue: dK[l, d] = scale * dK^T[d, kv] + sum_heads dK_c[j, d] / count(j) (dS goes to its product without the
+      // softmax scale), dV the same without a scale; this thread owns 32 key columns
       {
         uint32_t kk[32], vv[32];
         if (k > 0) {
@@ -412,7 +413,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               const int l = misc->tok[tb][half * 32 + c];
               if (l < 0) continue;
               const size_t idx = ((size_t)bhk * g.S + l) * D + row;
-              store_out(a.dk, idx, __uint_as_float(kk[c]) + coarse_k, 1);
+              store_out(a.dk, idx, fmaf(__uint_as_float(kk[c]), g.scale, coarse_k), 1);
               store_out(a.dv, idx, __uint_as_float(vv[c]) + coarse_v, 1);
             }
           }
@@ -423,7 +424,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
           if (row < D) {
 #pragma unroll
             for (int c = 0; c < 32; ++c) {
-              st_k[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(kk[c]) + coarse_k);
+              st_k[(half * 32 + c) * D + row] = __float2bfloat16_rn(fmaf(__uint_as_float(kk[c]), g.scale, coarse_k));
               st_v[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(vv[c]) + coarse_v);
             }
           }
