@@ -279,10 +279,10 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 #pragma unroll
             for (int c4 = 0; c4 < 8; ++c4) {
               const float4 dl = del4[c4];
-              const float d0 = __uint_as_float(sv[4 * c4 + 0]) * (__uint_as_float(dp[4 * c4 + 0]) - dl.x) * g.scale;
-              const float d1 = __uint_as_float(sv[4 * c4 + 1]) * (__uint_as_float(dp[4 * c4 + 1]) - dl.y) * g.scale;
-              const float d2 = __uint_as_float(sv[4 * c4 + 2]) * (__uint_as_float(dp[4 * c4 + 2]) - dl.z) * g.scale;
-              const float d3 = __uint_as_float(sv[4 * c4 + 3]) * (__uint_as_float(dp[4 * c4 + 3]) - dl.w) * g.scale;
+              const float d0 = __uint_as_float(sv[4 * c4 + 0]) * (__uint_as_float(dp[4 * c4 + 0]) - dl.x);
+              const float d1 = __uint_as_float(sv[4 * c4 + 1]) * (__uint_as_float(dp[4 * c4 + 1]) - dl.y);
+              const float d2 = __uint_as_float(sv[4 * c4 + 2]) * (__uint_as_float(dp[4 * c4 + 2]) - dl.z);
+              const float d3 = __uint_as_float(sv[4 * c4 + 3]) * (__uint_as_float(dp[4 * c4 + 3]) - dl.w);
               if constexpr (SPLIT) {
                 uint32_t h0, l0, h1, l1;
                 split_bf16x2(d0, d1, h0, l0);
@@ -316,7 +316,8 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         VSA2_WAIT(&misc->o_full, n_items & 1);
         tc::tc_fence_after();
       }
-      // epilogue: dQ[l, d] = dQ^T[d, q] + dQ_c[i, d] / count(i); this thread owns 32 query columns of channel `row`
+      // epilogue: dQ[l, d] = scale * dQ^T[d, q] + dQ_c[i, d] / count(i) (dS goes to its product without the softmax scale);
+      // this thread owns 32 query columns of channel `row`
       {
         uint32_t o0[32];
         if (k > 0) {
@@ -341,7 +342,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int c = 0; c < 32; ++c) {
               const int l = misc->tok[tb][half * 32 + c];
               if (l < 0) continue;
-              store_out(a.dq, ((size_t)bhq * g.S + l) * D + row, __uint_as_float(o0[c]) + coarse_d, 1);
+              store_out(a.dq, ((size_t)bhq * g.S + l) * D + row, fmaf(__uint_as_float(o0[c]), g.scale, coarse_d), 1);
             }
           }
         } else {
@@ -350,7 +351,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           if (row < D) {
 #pragma unroll
             for (int c = 0; c < 32; ++c)
-              st[(half * 32 + c) * D + row] = __float2bfloat16_rn(__uint_as_float(o0[c]) + coarse_d);
+              st[(half * 32 + c) * D + row] = __float2bfloat16_rn(fmaf(__uint_as_float(o0[c]), g.scale, coarse_d));
           }
           VSA2_GROUP_SYNC_AT(&misc->e_sync, e_sync0 + 1);
           constexpr int CH = D / 8;
