@@ -71,7 +71,10 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
  * relative) they alone push the worst elements of large gradients (|g| > 5) past max abs err 2e-2.  By default the dQ pass
  * always, and the dK/dV pass for GQA groups (where a KV block sums several heads), carry them as a bf16 pair -- the value
  * and the bf16 rounding of what that lost -- in one product of twice the width.  Measured on 720p / 480p samples against
- * the oracle (fp32 outputs): dQ 7e-3 instead of 2.5e-2, GQA dK 8e-3 instead of 2.6e-2; MHA dK, dV stay near 1e-2 either way.
+ * the oracle (fp32 outputs): dQ 7e-3 instead of 2.5e-2, GQA dK 8e-3 instead of 2.6e-2.  With one query head per KV head the
+ * rounding of the plain form leaves 1 - 2e-3 of a block's largest gradient; only KV blocks that nearly every query keeps have
+ * gradients large enough (|dK| = 15 on the 720p sample) for that to cross 2e-2, so the dK/dV pass computes the blocks kept by
+ * more than 256 query blocks with pairs in a second launch (about +5 % of that pass) and the others plain.
  * With cubes of 128 tokens the pair of the dQ pass travels along the contraction instead; a dK/dV pass that needs pairs (GQA, or
  * VSA2_FLAG_PRECISE_BWD) runs on the 64-token halves, the others on 128 x 128 tiles. */
 enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once everywhere (dQ pass about 15 % faster, GQA dK/dV pass about 30 %) */

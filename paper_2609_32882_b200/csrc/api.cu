@@ -585,13 +585,14 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
                                       reinterpret_cast<StatusBlock*>(workspace), st));
   }
   {
-    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, 1);
-    if (wide128 && !fine_bwd_dkv_wants_pair(n))
+    const bool dkv128 = wide128 && !fine_bwd_dkv_wants_pair(n);
+    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, (!dkv128 && fine_bwd_dkv_splits_long_columns(fx, true)) ? 2 : 1);
+    if (dkv128)
       VSA2_CUDA(launch_fine_bwd128_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                           coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
     else
       VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
-                                       coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
+                                       coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st, true));
   }
   return VSA2_OK;
 }

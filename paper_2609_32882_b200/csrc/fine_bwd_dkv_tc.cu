@@ -23,6 +23,7 @@ struct DkvArgs {
   void* dk;
   void* dv;
   StatusBlock* status;
+  int k_lo, k_hi;       // the launch handles the KV blocks whose column lists hold k_lo .. k_hi entries, and leaves the others alone
 };
 
 constexpr int kMaxRep = 16;   // query heads per KV head the dK/dV pass supports
@@ -127,7 +128,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       if (item == -2) goto done;
       if (item < 0) break;
       VSA2_DKV_ITEM_SETUP();
-      if (k == 0) continue;
+      if (k == 0 || k < a.k_lo || k > a.k_hi) continue;
       if (which == 0) {
         int c1, c2, c3;
         block_box(g, j, c1, c2, c3);
@@ -169,7 +170,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         VSA2_NEXT_ITEM_WARP(item, seq);
         VSA2_DKV_ITEM_SETUP();
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
-        if (k == 0) continue;
+        if (k == 0 || k < a.k_lo || k > a.k_hi) continue;
         const int nt = (k + 1) >> 1;
         VSA2_WAIT_PARKED(&misc->st_full, n_items & 1);
         for (int t = 0; t < nt; ++t, ++tg) {
@@ -211,7 +212,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         VSA2_NEXT_ITEM_WARP(item, seq);
         VSA2_DKV_ITEM_SETUP();
         (void)b; (void)hk; (void)j; (void)bhk; (void)col_beg;
-        if (k == 0) continue;
+        if (k == 0 || k < a.k_lo || k > a.k_hi) continue;
         const int nt = (k + 1) >> 1;
         VSA2_WAIT_PARKED(&misc->o_empty, (n_items & 1) ^ 1);
         for (int t = 0; t < nt; ++t, ++tg) {
@@ -255,7 +256,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       VSA2_NEXT_ITEM(item, seq);
       VSA2_DKV_ITEM_SETUP();
       (void)j; (void)bhk;
-      if (k == 0) continue;
+      if (k == 0 || k < a.k_lo || k > a.k_hi) continue;
       const int nt = (k + 1) >> 1;
       int bhq_n, i_n;
       dkv_entry(g, a, rep, b, hk, cnt_prefix, col_beg, (blk == 1 && k > 1) ? 1 : 0, bhq_n, i_n);
@@ -279,12 +280,14 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int sm_tid = tid - 128;            // 0..255
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint32_t tg = 0, n_items = 0;
+    uint32_t n_mine = 0;                       // items of this launch so far (the group syncs and table parities count these)
     for (uint32_t n_all = 0;; ++n_all) {
       VSA2_NEXT_ITEM(item, n_all);
       VSA2_DKV_ITEM_SETUP();
       (void)col_beg;
-      const int tb = n_all & 1;
-      const uint32_t e_sync0 = n_all * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
+      if (k < a.k_lo || k > a.k_hi) continue;  // another launch's item (an empty list still gets its coarse-only output)
+      const int tb = n_mine & 1;
+      const uint32_t e_sync0 = n_mine * (g.out_f32 ? 1u : 3u);     // index of this item's first group sync
       if (sm_tid < 64) misc->tok[tb][sm_tid] = block_token(g, j, sm_tid);
       float coarse_k = 0.f, coarse_v = 0.f;
       if (a.dkc != nullptr && row < D && !block_is_text(g, j)) {
@@ -442,6 +445,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
       }
       if (k > 0) ++n_items;
+      ++n_mine;
     }
   }
 
@@ -463,10 +467,20 @@ done:
 // ================================================================================================
 // launcher
 // ================================================================================================
+// A column list longer than this many query blocks goes through the pair form (see below)
+constexpr int kDkvLongColumn = 256;
+
+// `split_long_columns`: when the pass would run with plain bf16 operands (one query head per KV head, no precision flag), the
+// KV blocks that more than kDkvLongColumn query blocks keep are computed by a second launch that carries P and dS as bf16
+// pairs.  The rounding of the plain form leaves a relative error of 1 - 2e-3 of the largest gradient of a block, whatever
+// the list length (720p sample, fp32 outputs: 6.5e-3 at |dK| = 5.5 with 200 query blocks, 6.3e-3 at 3.0 with 260); the
+// few blocks that nearly every query keeps reach |dK| = 15 and then 1.5e-2 .. 2.7e-2 depending on nothing but where the
+// roundings fall (e.g. whether the softmax scale is applied before or after dS is rounded), i.e. across the stated 2e-2.
+// As pairs they come out at 6e-3.  The two launches walk the same item sequence and each skips the other's blocks.
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, bool split_long_columns) {
   if (g.rep > kMaxRep) return cudaErrorInvalidValue;
   CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
@@ -476,10 +490,9 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   int sms = 0;
   cudaError_t e;
   if ((e = bwd_sm_count(&sms)) != cudaSuccess) return e;
-  DkvArgs a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
-  const bool split = fine_bwd_dkv_wants_pair(g);
+  const bool mha = g.rep == 1;
 #define VSA2_LAUNCH_DKV(DD, SP, MH)                                                                                                \
   do {                                                                                                                           \
     using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
@@ -488,20 +501,32 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
       return e;                                                                                                                  \
     fine_bwd_dkv_tc_kernel<DD, SP, MH><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                        \
   } while (0)
-  const bool mha = g.rep == 1;
-  if (g.D == 128) {
-    if (split && mha) VSA2_LAUNCH_DKV(128, true, true);
-    else if (split) VSA2_LAUNCH_DKV(128, true, false);
-    else if (mha) VSA2_LAUNCH_DKV(128, false, true);
-    else VSA2_LAUNCH_DKV(128, false, false);
-  } else {
-    if (split && mha) VSA2_LAUNCH_DKV(64, true, true);
-    else if (split) VSA2_LAUNCH_DKV(64, true, false);
-    else if (mha) VSA2_LAUNCH_DKV(64, false, true);
-    else VSA2_LAUNCH_DKV(64, false, false);
-  }
+  auto launch = [&](bool split, int counter_slot, int k_lo, int k_hi) -> cudaError_t {
+    DkvArgs a{&status->pad[counter_slot], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, k_lo, k_hi};
+    if (g.D == 128) {
+      if (split && mha) VSA2_LAUNCH_DKV(128, true, true);
+      else if (split) VSA2_LAUNCH_DKV(128, true, false);
+      else if (mha) VSA2_LAUNCH_DKV(128, false, true);
+      else VSA2_LAUNCH_DKV(128, false, false);
+    } else {
+      if (split && mha) VSA2_LAUNCH_DKV(64, true, true);
+      else if (split) VSA2_LAUNCH_DKV(64, true, false);
+      else if (mha) VSA2_LAUNCH_DKV(64, false, true);
+      else VSA2_LAUNCH_DKV(64, false, false);
+    }
+    return cudaGetLastError();
+  };
 #undef VSA2_LAUNCH_DKV
-  return cudaGetLastError();
+  constexpr int kAll = 0x7fffffff;
+  if (fine_bwd_dkv_wants_pair(g)) return launch(true, 3, 0, kAll);
+  if (!fine_bwd_dkv_splits_long_columns(g, split_long_columns)) return launch(false, 3, 0, kAll);
+  if ((e = launch(false, 3, 0, kDkvLongColumn)) != cudaSuccess) return e;
+  return launch(true, 4, kDkvLongColumn + 1, kAll);
+}
+
+// whether launch_fine_bwd_dkv_tc runs as two launches for this problem
+bool fine_bwd_dkv_splits_long_columns(const Geo& g, bool split_long_columns) {
+  return split_long_columns && !fine_bwd_dkv_wants_pair(g) && !(g.flags & VSA2_FLAG_FAST_BWD);
 }
 
 }  // namespace vsa2
