@@ -212,17 +212,39 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               p[c] = ex2_approx(fmaf(__uint_as_float(s[c]), c2, -my_lse2));
               if (kbits != 0xffffffffu) p[c] = ((kbits >> c) & 1u) ? p[c] : 0.f;
             }
+            // Column sums of the 32 / G key cubes of the chunk, then the sum over the G rows of the query cube, which sit in
+            // G adjacent lanes: a butterfly that halves the values a lane carries at every step (4 shuffles instead of
+            // 3 per key cube; the passes are bound by instruction issue) and leaves each total in one lane.
+            static_assert(G == 8 || G == 16, "router pooling layout");
+            float tv[32 / G];
 #pragma unroll
             for (int cc = 0; cc < 32 / G; ++cc) {
               float tot = 0.f;
 #pragma unroll
               for (int c = 0; c < G; ++c) tot += p[cc * G + c];
-#pragma unroll
-              for (int o = 1; o < G; o <<= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
-              const int kj = (kt * kRtTile + ch * 32) / G + cc;
-              if ((lane & (G - 1)) == (cc & (G - 1)) && qi < g.N && kj < g.N)
-                pr[((size_t)bhq * g.N + qi) * g.N + kj] = tot * inv_norm;
+              tv[cc] = tot;
             }
+            float t;
+            int cc_mine;
+            if constexpr (G == 8) {
+              const bool hi4 = lane & 4, hi2 = lane & 2;
+              const float k0 = hi4 ? tv[2] : tv[0], k1 = hi4 ? tv[3] : tv[1];
+              const float s0 = hi4 ? tv[0] : tv[2], s1 = hi4 ? tv[1] : tv[3];
+              const float u0 = k0 + __shfl_xor_sync(0xffffffffu, s0, 4), u1 = k1 + __shfl_xor_sync(0xffffffffu, s1, 4);
+              t = (hi2 ? u1 : u0) + __shfl_xor_sync(0xffffffffu, hi2 ? u0 : u1, 2);
+              t += __shfl_xor_sync(0xffffffffu, t, 1);
+              cc_mine = (hi4 ? 2 : 0) + (hi2 ? 1 : 0);
+            } else {
+              const bool hi8 = lane & 8;
+              t = (hi8 ? tv[1] : tv[0]) + __shfl_xor_sync(0xffffffffu, hi8 ? tv[0] : tv[1], 8);
+              t += __shfl_xor_sync(0xffffffffu, t, 4);
+              t += __shfl_xor_sync(0xffffffffu, t, 2);
+              t += __shfl_xor_sync(0xffffffffu, t, 1);
+              cc_mine = hi8 ? 1 : 0;
+            }
+            const int kj = (kt * kRtTile + ch * 32) / G + cc_mine;
+            const bool owner = G == 8 ? !(lane & 1) : !(lane & 7);
+            if (owner && qi < g.N && kj < g.N) pr[((size_t)bhq * g.N + qi) * g.N + kj] = t * inv_norm;
           }
         }
         tc::tc_fence_before();
