@@ -174,3 +174,23 @@ def test_config2_480p_gqa_cubes_of_128_tokens_with_empty_half_cubes():
     sampled_attention_parity(wl, data, fp32_twin(wl, data, run), gmask, q_heads=(1, 10), rows=(0, 6, 160, N - 1),
                              kv_groups=(0, 2), kv_cubes=(6, N - 1))         # cubes 6 and N-1 end beyond the grid along w
     assert torch.isfinite(run.o.float()).all() and torch.isfinite(run.dk.float()).all() and torch.isfinite(run.dq.float()).all()
+
+
+def test_dkv_columns_on_both_sides_of_the_pair_threshold():
+    """One query head per KV head: the dK/dV pass gives the KV blocks that more than 256 query blocks keep to its bf16-pair
+    form in a second launch and the others to the plain form.  320 cubes, every query block keeps 256 of them, so the
+    column lists scatter around 256 entries: a block on each side of the threshold, and the longest and shortest lists,
+    against the oracle -- each launch must write its own blocks and leave the other's alone."""
+    wl = syn.Workload("columns_near_256", 1, 1, 1, 128, (20, 32, 32), select_mode=syn.PER_QUERY, topk=256, kind="iid", seed=77)
+    data = syn.make_inputs(wl, threads=16)
+    run = CudaPath(wl, data)
+    gmask = run.route()
+    cnt = gmask[0, 0].sum(axis=0)
+    assert cnt.min() <= 256 < cnt.max()
+    below = int(np.nonzero(cnt == cnt[cnt <= 256].max())[0][0])      # the longest list of the plain launch
+    above = int(np.nonzero(cnt == cnt[cnt > 256].min())[0][0])       # the shortest list of the pair launch
+    run.forward()
+    run.backward()
+    sampled_attention_parity(wl, data, fp32_twin(wl, data, run), gmask, q_heads=(), rows=(),
+                             kv_groups=(0,), kv_cubes=(below, above, int(np.argmax(cnt)), int(np.argmin(cnt))))
+    assert torch.isfinite(run.dk.float()).all() and torch.isfinite(run.dv.float()).all()
