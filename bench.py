@@ -42,6 +42,15 @@ NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.498373e9 + 0.288805e9), "fine
                                 "fine_bwd_dkv": 5 * (0.762483e9 + 0.305517e9)}
 
 
+# What ncu shows as the busiest unit of each tensor kernel at 64-token cubes (8-head capture, profiles/): the roofline
+# below is quoted against the tensor peak as the contract asks, these say what actually holds the kernel there.
+NCU_LIMITER = {
+    "fine_fwd": "L2 -> SM read rate: 12.0 TB/s against 11.8 TB/s sustained peak (tensor pipe 76 % active at the half rate of M = 64)",
+    "fine_bwd_dq": "shared-memory data pipe: tensor-core operand fetches 57 % + thread loads/stores 40 % (tensor pipe 47 %)",
+    "fine_bwd_dkv": "shared-memory data pipe: tensor-core operand fetches 61 % + thread loads/stores 29 % (tensor pipe 46 %)",
+    "router_lse": "exponential unit 76 %, instruction issue 70 %",
+    "router_pool": "exponential unit 76 %, instruction issue 70 %",
+}
 # L2 -> SM read rate that ncu reports as the sustained peak of this part (derived__lts__lts2xbar_bytes.sum.peak_sustained
 # in the 8-head capture of profiles/kernels_720p_8heads_ncu_full.md, where the fine forward itself reads 12.0 TB/s).
 NCU_L2_TO_SM_PEAK_TBS = 11.776
@@ -435,7 +444,8 @@ def run_ours(args):
                 "frac": achieved / peak_tf,
                 "traffic": NCU_TRAFFIC_BYTES_720P_TOP64.get(dominant) if (args.config == 3 and not (args.heads or args.topk or args.grid or args.cube)) else None,
                 "peak_kind": pk_kind + " sustained bf16",
-                "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant]}
+                "flops_per_launch": kernel_flops[dominant], "ms_per_launch": kernel_ms[dominant],
+                "limiter_ncu": NCU_LIMITER.get(dominant) if wl.cube[0] * wl.cube[1] * wl.cube[2] == 64 else None}
     fine_fwd_tf = flops["fine_fwd"] / (kernel_ms["fine_fwd"] * 1e-3) / 1e12
     # operand bytes the fine forward has to bring into shared memory: a K and a V tile per selected (query block, KV block)
     # pair and a Q tile per query block, in bf16 -- none of it can be reused between the query blocks of a head, whose
