@@ -38,18 +38,18 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the 720p top-64 launch with 40 heads: an
 # 8-head ncu capture of the same kernels times 5 (every head streams its own tensors, so the traffic grows in
 # proportion to the heads; the 40-head launch is too large for a full-set capture).
-NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.498373e9 + 0.288805e9), "fine_bwd_dq": 5 * (0.666063e9 + 0.147825e9),
-                                "fine_bwd_dkv": 5 * (0.762483e9 + 0.305517e9)}
+NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.501040e9 + 0.294885e9), "fine_bwd_dq": 5 * (0.663608e9 + 0.147419e9),
+                                "fine_bwd_dkv": 5 * (0.763098e9 + 0.295859e9 + 0.168354e9 + 0.004243e9)}   # both dK/dV launches
 
 
 # What ncu shows as the busiest unit of each tensor kernel at 64-token cubes (8-head capture, profiles/): the roofline
 # below is quoted against the tensor peak as the contract asks, these say what actually holds the kernel there.
 NCU_LIMITER = {
-    "fine_fwd": "L2 -> SM read rate: 12.0 TB/s against 11.8 TB/s sustained peak (tensor pipe 76 % active at the half rate of M = 64)",
-    "fine_bwd_dq": "shared-memory data pipe: tensor-core operand fetches 57 % + thread loads/stores 40 % (tensor pipe 47 %)",
-    "fine_bwd_dkv": "shared-memory data pipe: tensor-core operand fetches 61 % + thread loads/stores 29 % (tensor pipe 46 %)",
-    "router_lse": "exponential unit 76 %, instruction issue 70 %",
-    "router_pool": "exponential unit 76 %, instruction issue 70 %",
+    "fine_fwd": "L2 -> SM read rate: 12.8 TB/s against 11.8 TB/s sustained peak (tensor pipe 82 % active at the half rate of M = 64)",
+    "fine_bwd_dq": "shared-memory data pipe: tensor-core operand fetches 59 % + thread loads/stores 39 % (tensor pipe 48 %)",
+    "fine_bwd_dkv": "shared-memory data pipe: tensor-core operand fetches 69 % + thread loads/stores 31 % (tensor pipe 47 %)",
+    "router_lse": "exponential unit 81 %, instruction issue 65 %",
+    "router_pool": "exponential unit 77 %, instruction issue 69 %",
 }
 # L2 -> SM read rate that ncu reports as the sustained peak of this part (derived__lts__lts2xbar_bytes.sum.peak_sustained
 # in the 8-head capture of profiles/kernels_720p_8heads_ncu_full.md, where the fine forward itself reads 12.0 TB/s).
