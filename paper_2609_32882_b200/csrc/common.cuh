@@ -291,7 +291,7 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                   cudaStream_t st, bool split_long_columns);
+                                   cudaStream_t st, bool split_long_columns, int* item_list);
 bool fine_bwd_dkv_splits_long_columns(const Geo& g, bool split_long_columns);
 
 cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,

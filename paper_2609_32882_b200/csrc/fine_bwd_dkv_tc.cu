@@ -24,6 +24,8 @@ struct DkvArgs {
   void* dv;
   StatusBlock* status;
   int k_lo, k_hi;       // the launch handles the KV blocks whose column lists hold k_lo .. k_hi entries, and leaves the others alone
+  const int* item_list; // null, or [count, item, item, ...]: the items with k_lo .. k_hi entries (the launch then walks this list
+                        // instead of all items: a launch for the few long lists would spend most of its time skipping)
 };
 
 constexpr int kMaxRep = 16;   // query heads per KV head the dK/dV pass supports
@@ -37,6 +39,46 @@ __device__ __forceinline__ void dkv_entry(const Geo& g, const DkvArgs& a, int re
   while (hh + 1 < rep && e >= cnt_prefix[hh + 1]) ++hh;
   bhq = b * g.Hq + hk * rep + hh;
   i = a.row_idx[(size_t)bhq * g.nnz_cap + col_beg[hh] + (e - cnt_prefix[hh])];
+}
+
+// The work items whose column lists hold k_lo .. k_hi entries, appended to list[1 ...] with their count in list[0] (zero
+// before the launch).  The order of the list depends on the run; the results do not (an item is a whole KV block).
+__global__ void __launch_bounds__(256) dkv_list_items_kernel(Geo g, const int* __restrict__ col_ptr, int rep, int total,
+                                                             int k_lo, int k_hi, int* list) {
+  const int item = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
+  bool in = false;
+  if (item < total) {
+    int j, bhk;
+    item_block(g, item, bhk, j);
+    const int b = bhk / g.Hkv, hk = bhk % g.Hkv;
+    int kk = 0;
+    for (int hh = 0; hh < rep; ++hh) {
+      const size_t base = (size_t)(b * g.Hq + hk * rep + hh) * (g.N + 1) + j;
+      kk += col_ptr[base + 1] - col_ptr[base];
+    }
+    in = kk >= k_lo && kk <= k_hi;
+  }
+  const unsigned m = __ballot_sync(0xffffffffu, in);
+  if (m == 0u) return;
+  const int leader = __ffs(m) - 1;
+  int base = 0;
+  if (lane == leader) base = atomicAdd(&list[0], __popc(m));
+  base = __shfl_sync(0xffffffffu, base, leader);
+  if (in) list[1 + base + __popc(m & ((1u << lane) - 1u))] = item;
+}
+
+// scheduler of a launch that walks an item list: publish_ahead of tc_attn.cuh with the list in between
+__device__ __forceinline__ bool dkv_publish_listed(ItemQueue* q, uint32_t seq, uint32_t& published, int* counter,
+                                                   const int* list, volatile int* abort_flag) {
+  while (published <= seq + kItemAhead) {
+    const uint32_t slot = published % kItemSlots, par = ((published / kItemSlots) & 1) ^ 1;
+    if (!tc::mbar_wait_parked(&q->empty[slot], par, abort_flag)) return false;
+    const int it = atomicAdd(counter, 1);
+    q->item[slot] = it < list[0] ? list[1 + it] : -1;
+    tc::mbar_arrive(&q->full[slot]);
+    ++published;
+  }
+  return true;
 }
 
 // Roles: warp 0 = TMA producer of the Q pairs (ring A) and of the stationary K and V tiles, warp 1 = TMA producer of the
@@ -75,6 +117,9 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const float c2 = g.scale * 1.4426950408889634f;
   const int rep = MHA ? 1 : g.rep;
 
+  // the launch of the few long lists lets the launch behind it in the stream (the other lists: disjoint outputs, nothing
+  // read from this one) take the SMs as its CTAs leave them
+  if (SPLIT && a.item_list != nullptr) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) {
     bwd_init_barriers(misc);
     tc::mbar_init(&misc->o_full, 2);                                          // two last-stage issuers
@@ -121,8 +166,14 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       // warp 0, lane 0 is the CTA's scheduler
       int item = 0;
       if (lane == 0) {
-        if (which == 0 && !item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag)) item = -2;
-        else item = item_get(&misc->items, seq, &misc->abort_flag);
+        bool pub_ok = true;
+        if (which == 0) {
+          if (SPLIT && a.item_list != nullptr)
+            pub_ok = dkv_publish_listed(&misc->items, seq, published, a.item_counter, a.item_list, &misc->abort_flag);
+          else
+            pub_ok = item_publish_ahead(&misc->items, seq, published, a.item_counter, total_items, &misc->abort_flag);
+        }
+        item = pub_ok ? item_get(&misc->items, seq, &misc->abort_flag) : -2;
       }
       item = __shfl_sync(0xffffffffu, item, 0);
       if (item == -2) goto done;
@@ -476,11 +527,12 @@ constexpr int kDkvLongColumn = 256;
 // the list length (720p sample, fp32 outputs: 6.5e-3 at |dK| = 5.5 with 200 query blocks, 6.3e-3 at 3.0 with 260); the
 // few blocks that nearly every query keeps reach |dK| = 15 and then 1.5e-2 .. 2.7e-2 depending on nothing but where the
 // roundings fall (e.g. whether the softmax scale is applied before or after dS is rounded), i.e. across the stated 2e-2.
-// As pairs they come out at 6e-3.  The two launches walk the same item sequence and each skips the other's blocks.
+// As pairs they come out at 6e-3.  The first launch walks all items and skips the long lists; the second walks the list of
+// them that a small kernel collects into `item_list` (1 + batch * Hkv * N ints of scratch; null: it walks all items too).
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                   cudaStream_t st, bool split_long_columns) {
+                                   cudaStream_t st, bool split_long_columns, int* item_list) {
   if (g.rep > kMaxRep) return cudaErrorInvalidValue;
   CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
@@ -499,10 +551,23 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
     if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize,               \
                                   (int)L_::smem_bytes)))                                                                         \
       return e;                                                                                                                  \
-    fine_bwd_dkv_tc_kernel<DD, SP, MH><<<grid, kDkvThreads, L_::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                        \
+    cfg.dynamicSmemBytes = L_::smem_bytes;                                                                                       \
+    if ((e = cudaLaunchKernelEx(&cfg, fine_bwd_dkv_tc_kernel<DD, SP, MH>, tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a)))          \
+      return e;                                                                                                                  \
   } while (0)
-  auto launch = [&](bool split, int counter_slot, int k_lo, int k_hi) -> cudaError_t {
-    DkvArgs a{&status->pad[counter_slot], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, k_lo, k_hi};
+  // `overlap`: the launch may start while the launch before it in the stream is still running (programmatic dependent
+  // launch; that one releases it at its start and the two touch disjoint outputs)
+  auto launch = [&](bool split, int counter_slot, int k_lo, int k_hi, const int* list, bool overlap) -> cudaError_t {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kDkvThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    DkvArgs a{&status->pad[counter_slot], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, k_lo, k_hi, list};
     if (g.D == 128) {
       if (split && mha) VSA2_LAUNCH_DKV(128, true, true);
       else if (split) VSA2_LAUNCH_DKV(128, true, false);
@@ -518,10 +583,20 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   };
 #undef VSA2_LAUNCH_DKV
   constexpr int kAll = 0x7fffffff;
-  if (fine_bwd_dkv_wants_pair(g)) return launch(true, 3, 0, kAll);
-  if (!fine_bwd_dkv_splits_long_columns(g, split_long_columns)) return launch(false, 3, 0, kAll);
-  if ((e = launch(false, 3, 0, kDkvLongColumn)) != cudaSuccess) return e;
-  return launch(true, 4, kDkvLongColumn + 1, kAll);
+  if (fine_bwd_dkv_wants_pair(g)) return launch(true, 3, 0, kAll, nullptr, false);
+  if (!fine_bwd_dkv_splits_long_columns(g, split_long_columns)) return launch(false, 3, 0, kAll, nullptr, false);
+  if (item_list == nullptr) {
+    if ((e = launch(false, 3, 0, kDkvLongColumn, nullptr, false)) != cudaSuccess) return e;
+    return launch(true, 4, kDkvLongColumn + 1, kAll, nullptr, false);
+  }
+  // The long lists are a few hundred of the items: a small kernel collects them, the pair launch starts on them at once
+  // (a handful of 0.3 ms items on 148 CTAs: it would end with most SMs idle), and the plain launch fills the SMs as the
+  // pair launch's CTAs leave them.
+  if ((e = cudaMemsetAsync(item_list, 0, sizeof(int), st)) != cudaSuccess) return e;
+  dkv_list_items_kernel<<<(total + 255) / 256, 256, 0, st>>>(g, col_ptr, g.rep, total, kDkvLongColumn + 1, kAll, item_list);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  if ((e = launch(true, 4, kDkvLongColumn + 1, kAll, item_list, false)) != cudaSuccess) return e;
+  return launch(false, 3, 0, kDkvLongColumn, nullptr, true);
 }
 
 // whether launch_fine_bwd_dkv_tc runs as two launches for this problem
