@@ -144,7 +144,7 @@ cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float*
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // delta_c = rowsum(dO_c * O_c) through the preprocess kernel of the pooled problem (no gate: only delta is written)
   if ((e = launch_bwd_preprocess(p, do16, oc_hat, nullptr, nullptr, nullptr, delta, nullptr, nullptr, st)) != cudaSuccess) return e;
-  if ((e = launch_fine_bwd_dq_tc(p, q16, k16, v16, do16, lse_c, delta, ptr, idx, nullptr, dqc, status, st)) != cudaSuccess) return e;
+  if ((e = launch_fine_bwd_dq_tc(p, q16, k16, v16, do16, lse_c, delta, ptr, idx, nullptr, dqc, status, st, nullptr, nullptr)) != cudaSuccess) return e;
   const bool grouped = g.rep > 1;
   if ((e = launch_fine_bwd_dkv_tc(p, q16, k16, v16, do16, lse_c, delta, ptr, idx, nullptr, nullptr, grouped ? dk_kv : dkc,
                                   grouped ? dv_kv : dvc, status, st, false, nullptr)) != cudaSuccess)

@@ -287,7 +287,8 @@ cudaError_t launch_fine_bwd128_dkv_tc(const Geo& g, const bf16* q, const bf16* k
 // tensor-core backward passes (fine_bwd_tc.cu)
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                   const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
-                                  const float* dqc, void* dq, StatusBlock* status, cudaStream_t st);
+                                  const float* dqc, void* dq, StatusBlock* status, cudaStream_t st, void* q16, void* k16);
+bool fine_bwd_dq_uses_f16(const Geo& g);
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,

@@ -36,7 +36,58 @@ struct DqArgs {
   const float* dqc;     // [B, Hq, N, D] or null
   void* dq;
   StatusBlock* status;
+  // fp16 form and its fallback: `range_flag` (zero at first) is set when a value left the fp16 range.  when = 0: the launch
+  // always runs; 1: it runs if the flag is clear (and sets it if a dS saturates); 2: it runs only if the flag is set.
+  int* range_flag;
+  int when;
 };
+
+// Slot of StatusBlock.pad that holds the range flag of the fp16 dQ pass
+constexpr int kRangeFlagSlot = 8;
+
+// fp32 pair -> packed fp16 pair (`lo` in the low half), values beyond the fp16 range clamped to +-65504
+__device__ __forceinline__ uint32_t pack_f16x2_sat(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// Copies of two bf16 tensors in fp16 (8 elements per thread and step).  Every finite bf16 below 65520 in magnitude has an
+// exact fp16 image down to 2^-24 granularity (fp16 keeps more mantissa bits), so products of the copies equal the products
+// of the originals; a finite value beyond that range sets `range_flag` and the caller's fp16 kernels stand back.
+__global__ void __launch_bounds__(256) cast_bf16_to_f16_kernel(const uint4* __restrict__ xa, uint4* __restrict__ ya, size_t na,
+                                                               const uint4* __restrict__ xb, uint4* __restrict__ yb, size_t nb,
+                                                               int* range_flag) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x, n = na + nb;
+  bool bad = false;
+  constexpr int U = 4;      // 16-byte loads in flight per thread (a pure streaming kernel)
+  for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n; i0 += U * stride) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const size_t i = i0 + u * stride;
+      v[u] = i < n ? (i < na ? __ldg(xa + i) : __ldg(xb + (i - na))) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const size_t i = i0 + u * stride;
+      if (i >= n) break;
+      const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+      uint32_t r[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t m0 = w[e] & 0x7fffu, m1 = (w[e] >> 16) & 0x7fffu;     // magnitudes as bf16 bit patterns (0x4780 = 65536)
+        bad |= (m0 >= 0x4780u && m0 < 0x7f80u) || (m1 >= 0x4780u && m1 < 0x7f80u);
+        const __half2 h = __floats2half2_rn(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
+        r[e] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      const uint4 o = make_uint4(r[0], r[1], r[2], r[3]);
+      if (i < na) ya[i] = o;
+      else yb[i - na] = o;
+    }
+  }
+  if (bad) atomicExch(range_flag, 1);
+}
 
 // Roles: warp 0 = TMA producer of the K pairs (ring A; a slot is held until the dQ^T product of its tile is done) and of
 // the stationary Q and dO tiles, warp 1 = TMA producer of the V pairs (ring B), warp 2 = issuer of S^T, warp 3 = issuer
@@ -45,7 +96,11 @@ struct DqArgs {
 // SPLIT: dS^T is handed to the dQ^T product as [bf16(dS^T) | bf16(dS^T - bf16(dS^T))] (one N = 128 product into two
 // accumulator halves that the epilogue adds), which removes the bf16 rounding of dS from dQ; the two operand buffers
 // then hold one tile (hi, lo) instead of two tiles.
-template <int D, bool SPLIT>
+// F16 (without SPLIT): the maps of Q and K point at fp16 copies of the tensors and dS^T is rounded to fp16, so S^T and the
+// dQ^T product are fp16 x fp16 instructions (dP^T stays bf16 x bf16: V and dO are not copied).  S^T comes out as with the
+// bf16 originals (the copies are exact), dS keeps 11 significant bits instead of 8, which is what the pair form is for, at
+// the cost of the plain form.
+template <int D, bool SPLIT, bool F16>
 __global__ void __launch_bounds__(kDqThreads, 1)
 fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -63,6 +118,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int total_items = g.batch * g.Hq * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
+  if (a.when != 0 && ((*a.range_flag != 0) != (a.when == 2))) return;     // (the flag is final before this launch starts)
 
   if (tid == 0) {
     bwd_init_barriers(misc);
@@ -165,7 +221,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             VSA2_WAIT(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
             if (tc::elect_one()) {
-              mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+              mma_pair_kmajor<D, F16>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
               tc::mma_commit(&misc->s_full[sb]);
               if (t == nt - 1) tc::mma_commit(&misc->st_empty);
             }
@@ -204,7 +260,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           tc::tc_fence_after();
           if (tc::elect_one()) {
             if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr, C::PBYTES, t > 0);
-            else mma_pairT_mnmajor<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
+            else mma_pairT_mnmajor<D, F16>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
             tc::mma_commit(&misc->a_empty[sa]);
             tc::mma_commit(&misc->ds_free[sd]);
             if (t == nt - 1) tc::mma_commit(&misc->o_full);
@@ -226,7 +282,15 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     cpos.init(g, row & 63);
     const int blk = row >> 6;
     uint32_t tg = 0, n_items = 0;
+    uint32_t sat = 0u;        // F16: largest magnitudes (as fp16 bit patterns, two lanes) of the dS values this thread rounded
     for (uint32_t n_all = 0;; ++n_all) {
+      if constexpr (F16) {
+        // a dS at the clamp (or not a number): the result of this launch is not to be used, the fallback launch redoes it
+        if ((sat & 0xffffu) >= 0x7bffu || (sat >> 16) >= 0x7bffu) {
+          atomicExch(a.range_flag, 1);
+          sat = 0u;
+        }
+      }
       VSA2_NEXT_ITEM(item, n_all);
       int i, bhq;
       item_block(g, item, bhq, i);
@@ -291,6 +355,10 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 packed[2 * c4 + 1] = valid ? h1 : 0u;
                 packed_lo[2 * c4] = valid ? l0 : 0u;
                 packed_lo[2 * c4 + 1] = valid ? l1 : 0u;
+              } else if constexpr (F16) {
+                packed[2 * c4] = valid ? pack_f16x2_sat(d0, d1) : 0u;
+                packed[2 * c4 + 1] = valid ? pack_f16x2_sat(d2, d3) : 0u;
+                sat = __vmaxu2(sat, __vmaxu2(packed[2 * c4] & 0x7fff7fffu, packed[2 * c4 + 1] & 0x7fff7fffu));
               } else {
                 packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
                 packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
@@ -387,37 +455,65 @@ done:
 // ================================================================================================
 // launcher
 // ================================================================================================
+// `q16`, `k16`: null, or scratch for fp16 copies of Q and K (as many elements as the tensors).  With them the default pass
+// (no precision flag) is: the copy, the fp16 form of the kernel, and a launch of the pair form that does nothing unless the
+// range flag came up (a finite |Q|, |K| >= 65520 or a |dS| >= 65504: the pair form then computes dQ as before).
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                   const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
-                                  const float* dqc, void* dq, StatusBlock* status, cudaStream_t st) {
-  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
-  if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
-      !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) ||
+                                  const float* dqc, void* dq, StatusBlock* status, cudaStream_t st, void* q16, void* k16) {
+  const bool f16 = fine_bwd_dq_uses_f16(g) && q16 != nullptr && k16 != nullptr;
+  const bf16* qa = f16 ? reinterpret_cast<const bf16*>(q16) : q;      // (same element size and layout: the maps only move bytes)
+  const bf16* ka = f16 ? reinterpret_cast<const bf16*>(k16) : k;
+  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot, tq0, tk0, tqt0, tkt0;
+  if (!make_cube_tmap(&tq, qa, g, g.Hq) || !make_cube_tmap(&tk, ka, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
+      !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, qa, g, g.Hq) || !make_text_tmap(&tkt, ka, g, g.Hkv) ||
       !make_text_tmap(&tvt, v, g, g.Hkv) || !make_text_tmap(&tdot, d_o, g, g.Hq))
+    return cudaErrorInvalidValue;
+  if (f16 && (!make_cube_tmap(&tq0, q, g, g.Hq) || !make_cube_tmap(&tk0, k, g, g.Hkv) || !make_text_tmap(&tqt0, q, g, g.Hq) ||
+              !make_text_tmap(&tkt0, k, g, g.Hkv)))
     return cudaErrorInvalidValue;
   int sms = 0;
   cudaError_t e;
   if ((e = bwd_sm_count(&sms)) != cudaSuccess) return e;
-  DqArgs a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, dq, status};
+  int* flag = &status->pad[kRangeFlagSlot];
+  DqArgs a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, dq, status, flag, 0};
   const int total = g.batch * g.Hq * g.N;
   const int grid = total < sms ? total : sms;
   const bool split = !(g.flags & VSA2_FLAG_FAST_BWD);
-#define VSA2_LAUNCH_DQ(DD, SP)                                                                                                   \
+#define VSA2_LAUNCH_DQ(DD, SP, F, TQ, TK, TQT, TKT)                                                                              \
   do {                                                                                                                           \
-    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<DD, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize,                    \
+    if ((e = cudaFuncSetAttribute(fine_bwd_dq_tc_kernel<DD, SP, F>, cudaFuncAttributeMaxDynamicSharedMemorySize,                 \
                                   (int)BwdTc<DD>::smem_bytes)))                                                                  \
       return e;                                                                                                                  \
-    fine_bwd_dq_tc_kernel<DD, SP><<<grid, kDqThreads, BwdTc<DD>::smem_bytes, st>>>(tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a);                       \
+    fine_bwd_dq_tc_kernel<DD, SP, F><<<grid, kDqThreads, BwdTc<DD>::smem_bytes, st>>>(TQ, TK, tv, tdo, TQT, TKT, tvt, tdot, g, a); \
   } while (0)
+  if (f16) {
+    const size_t nq = (size_t)g.batch * g.Hq * g.S * g.D / 8, nk = (size_t)g.batch * g.Hkv * g.S * g.D / 8;
+    cast_bf16_to_f16_kernel<<<sms * 16, 256, 0, st>>>(reinterpret_cast<const uint4*>(q), reinterpret_cast<uint4*>(q16), nq,
+                                                     reinterpret_cast<const uint4*>(k), reinterpret_cast<uint4*>(k16), nk, flag);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    a.when = 1;
+    if (g.D == 128) VSA2_LAUNCH_DQ(128, false, true, tq, tk, tqt, tkt);
+    else VSA2_LAUNCH_DQ(64, false, true, tq, tk, tqt, tkt);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    a.when = 2;
+    a.item_counter = &status->pad[kRangeFlagSlot + 1];     // (its own counter: the fp16 launch has used the other)
+    if (g.D == 128) VSA2_LAUNCH_DQ(128, true, false, tq0, tk0, tqt0, tkt0);
+    else VSA2_LAUNCH_DQ(64, true, false, tq0, tk0, tqt0, tkt0);
+    return cudaGetLastError();
+  }
   if (g.D == 128) {
-    if (split) VSA2_LAUNCH_DQ(128, true);
-    else VSA2_LAUNCH_DQ(128, false);
+    if (split) VSA2_LAUNCH_DQ(128, true, false, tq, tk, tqt, tkt);
+    else VSA2_LAUNCH_DQ(128, false, false, tq, tk, tqt, tkt);
   } else {
-    if (split) VSA2_LAUNCH_DQ(64, true);
-    else VSA2_LAUNCH_DQ(64, false);
+    if (split) VSA2_LAUNCH_DQ(64, true, false, tq, tk, tqt, tkt);
+    else VSA2_LAUNCH_DQ(64, false, false, tq, tk, tqt, tkt);
   }
 #undef VSA2_LAUNCH_DQ
   return cudaGetLastError();
 }
+
+// whether the dQ pass of this problem takes its fp16 form when it is given the scratch for the copies
+bool fine_bwd_dq_uses_f16(const Geo& g) { return !(g.flags & (VSA2_FLAG_FAST_BWD | VSA2_FLAG_PRECISE_BWD)); }
 
 }  // namespace vsa2

@@ -30,9 +30,10 @@ __device__ __forceinline__ void store_row_sw128(unsigned char* tile, int row, co
 // Issues the D/16 (K-major x K-major) instructions of  acc[128, 64] = A_pair[128, D] * B[64, D]^T.
 // A_pair: slot laid out [half][block A | block B] slabs; B: tile laid out [half] slabs.
 // The descriptors are built once and advanced by adding the (16-byte-unit) offset to the address field.
-template <int D>
+// (F16: both operands hold fp16 instead of bf16)
+template <int D, bool F16 = false>
 __device__ __forceinline__ void mma_pair_kmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile) {
-  constexpr uint32_t idesc = tc::idesc_bf16(128, 64, false, false);
+  constexpr uint32_t idesc = F16 ? tc::idesc_f16(128, 64, false, false) : tc::idesc_bf16(128, 64, false, false);
   const uint64_t da = tc::smem_desc_sw128(a_slot, 16, 1024), db = tc::smem_desc_sw128(b_tile, 16, 1024);
 #pragma unroll
   for (int ks = 0; ks < D / 16; ++ks) {
@@ -44,9 +45,9 @@ __device__ __forceinline__ void mma_pair_kmajor(uint32_t tm_acc, uint32_t a_slot
 
 // Issues the 8 (MN-major x MN-major) instructions of  acc[D, 64] (+)= A_pair^T[D, 128] * B[128, 64], where A_pair is a
 // slot in the [half][block A | block B] layout (rows = the 128 contraction indices) and B is a 128-row swizzled tile.
-template <int D>
+template <int D, bool F16 = false>
 __device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, bool accumulate_first) {
-  constexpr uint32_t idesc = tc::idesc_bf16(128, 64, true, true);
+  constexpr uint32_t idesc = F16 ? tc::idesc_f16(128, 64, true, true) : tc::idesc_bf16(128, 64, true, true);
   constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;     // distance between the two 64-channel halves
   const uint64_t da = tc::smem_desc_sw128(a_slot, lbo, 1024), db = tc::smem_desc_sw128(b_tile, 0, 1024);
 #pragma unroll
