@@ -218,10 +218,8 @@ size_t fwd_base_bytes(const Geo& g) {
 }
 size_t bwd_base_bytes(const Geo& g) { return wide_cube(g) ? wide_bwd_layout(g).total : align_up(bwd_layout(g).total, 256); }
 size_t fwd_workspace_bytes(const Geo& g) { return fwd_base_bytes(g) + text_map_layout(g, false).total; }
-// fp16 copies of Q and K for the dQ pass on 64-token blocks (behind the other regions of the backward's workspace)
-bool dq_pass_f16(const Geo& g) {
-  return fine_bwd_dq_uses_f16(g) && !(wide_cube(g) && g.Lt == 0 && fine_bwd128_supported(narrow_geo(g)));
-}
+// fp16 copies of Q and K for the dQ pass (behind the other regions of the backward's workspace)
+bool dq_pass_f16(const Geo& g) { return fine_bwd_dq_uses_f16(g); }
 size_t bwd_f16_offset(const Geo& g) { return align_up(bwd_base_bytes(g) + text_map_layout(g, true).total, 256); }
 size_t bwd_q16_bytes(const Geo& g) { return align_up((size_t)g.batch * g.Hq * g.S * g.D * sizeof(bf16), 256); }
 size_t bwd_k16_bytes(const Geo& g) { return align_up((size_t)g.batch * g.Hkv * g.S * g.D * sizeof(bf16), 256); }
@@ -589,7 +587,9 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
     ProfScope ps(VSA2_KERNEL_FINE_BWD_DQ, st, f16 ? 3 : 1);
     if (wide128)
       VSA2_CUDA(launch_fine_bwd128_dq_tc(n, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
-                                         reinterpret_cast<StatusBlock*>(workspace), st));
+                                         reinterpret_cast<StatusBlock*>(workspace), st,
+                                         f16 ? at<unsigned char>(workspace, bwd_f16_offset(g)) : nullptr,
+                                         f16 ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g)) : nullptr));
     else
       VSA2_CUDA(launch_fine_bwd_dq_tc(fx, qb, kb, vb, dob, lse, delta, row_ptr, col_idx, coarse ? dqc : nullptr, dq,
                                       reinterpret_cast<StatusBlock*>(workspace), st,

@@ -278,7 +278,7 @@ bool fine_bwd128_supported(const Geo& g);
 bool fine_bwd_dkv_wants_pair(const Geo& g);
 cudaError_t launch_fine_bwd128_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                      const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
-                                     const float* dqc, void* dq, StatusBlock* status, cudaStream_t st);
+                                     const float* dqc, void* dq, StatusBlock* status, cudaStream_t st, void* q16, void* k16);
 cudaError_t launch_fine_bwd128_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                       const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                       const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
@@ -289,6 +289,11 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
                                   const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
                                   const float* dqc, void* dq, StatusBlock* status, cudaStream_t st, void* q16, void* k16);
 bool fine_bwd_dq_uses_f16(const Geo& g);
+// Slot of StatusBlock.pad that holds the range flag of the fp16 dQ passes (the slot behind it: the fallback launch's counter)
+constexpr int kRangeFlagSlot = 8;
+// fp16 copies of two bf16 tensors (element counts multiples of 8); a finite value beyond the fp16 range sets *range_flag
+cudaError_t launch_cast_bf16_to_f16(const bf16* a, void* a16, size_t na, const bf16* b, void* b16, size_t nb, int* range_flag,
+                                    cudaStream_t st);
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,

@@ -65,6 +65,8 @@ struct Bwd128Args {
   void* out0;           // dQ / dK
   void* out1;           // dV
   StatusBlock* status;
+  int* range_flag;      // fp16 form of the dQ pass and its fallback: as in DqArgs of the 64-token pass (when = 0: always runs)
+  int when;
 };
 
 // The stationary cube of a work item and the lists of streamed cubes that meet it.
@@ -127,9 +129,10 @@ struct ItemLists {
 // of column chunk c as bf16 pairs in columns 32 c .. 32 c + 15, with SPLIT their low-order parts in 32 c + 16 .. 32 c + 31),
 // Y a ring slot (MN-major B operand).
 // COMPACT (not with SPLIT): the 128 values of a row as 64 consecutive columns of bf16 pairs.
-template <int D, bool SPLIT, bool COMPACT>
+// F16: A and Y hold fp16.
+template <int D, bool SPLIT, bool COMPACT, bool F16 = false>
 __device__ __forceinline__ void mma_out_ts(uint32_t tm_acc, uint32_t tm_a, uint32_t slot_addr, bool accumulate_first) {
-  constexpr uint32_t idesc = tc::idesc_bf16(128, D, false, true);
+  constexpr uint32_t idesc = F16 ? tc::idesc_f16(128, D, false, true) : tc::idesc_bf16(128, D, false, true);
   constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;
   const uint64_t db = tc::smem_desc_sw128(slot_addr, lbo, 1024);
   constexpr int STEPS = SPLIT ? 16 : 8;
@@ -159,17 +162,32 @@ __device__ __forceinline__ void store_operand_chunk(uint32_t taddr, const float 
   }
 }
 
+// the same as fp16 pairs (clamped at the largest fp16 value); `sat` collects the largest magnitudes (fp16 bit patterns, two lanes)
+__device__ __forceinline__ void store_operand_chunk_f16(uint32_t taddr, const float (&v)[32], uint32_t& sat) {
+  uint32_t h[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    h[e] = pack_f16x2_sat(v[2 * e], v[2 * e + 1]);
+    sat = __vmaxu2(sat, h[e] & 0x7fff7fffu);
+  }
+  tc::tmem_st_32x32b_x16(taddr, h);
+}
+
 // Roles (512 threads): warps 0..3 = TMA producers (ring A / ring B x first / second block of a pair; warp 0 also brings the
 // stationary tiles and schedules the CTA's work items), warp 4 = issuer of S, warp 5 = issuer of dP, warp 6 = issuer of
 // the output products, warp 7 = loader of the per-column lse and delta (dK/dV pass), warps 8..15 = elementwise stage +
 // epilogue (thread = row r of the tile x one half of its columns).
-template <int D, int PASS, bool SPLIT>
+// F16 (dQ pass, without SPLIT): the maps of X0 = Q and Y0 = K point at fp16 copies and dS is rounded to fp16, so S and the dQ
+// product are fp16 x fp16 instructions (dP stays bf16 x bf16); see the 64-token dQ pass.
+template <int D, int PASS, bool SPLIT, bool F16 = false>
 __global__ void __launch_bounds__(kW2Threads, 1)
 fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_constant__ CUtensorMap tm_x1,
                       const __grid_constant__ CUtensorMap tm_y0, const __grid_constant__ CUtensorMap tm_y1, Geo g,
                       Bwd128Args a) {
   using C = Bwd128<D>;
   static_assert(PASS == 0 || !SPLIT, "the dK/dV pass has no room for the low-order parts of P and dS");
+  static_assert(!F16 || (PASS == 0 && !SPLIT), "the fp16 form is the dQ pass without pairs");
+  if (a.when != 0 && ((*a.range_flag != 0) != (a.when == 2))) return;     // (the flag is final before this launch starts)
   constexpr uint32_t NDP = PASS == 0 ? 2 : 1;                  // dP buffers
   // dQ pass: S 0; dP buffers 128, 256 (dS overwrites the dP it came from); dQ 384.
   // dK/dV pass: S^T and dP^T take turns in the staging columns 0..127 (each is pulled into registers as soon as it is
@@ -312,7 +330,7 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
       // ---------------------------------------------------------------- issuers of S = X0 Y0^T (warp 4) and dP = X1 Y1^T
       // (warp 5): the whole warp runs the loop, one elected lane issues
       const bool is_s = warp == 4;
-      constexpr uint32_t idesc = tc::idesc_bf16(128, 128, false, false);
+      const uint32_t idesc = (F16 && is_s) ? tc::idesc_f16(128, 128, false, false) : tc::idesc_bf16(128, 128, false, false);
       const uint64_t dx = tc::smem_desc_sw128(tc::smem_u32(is_s ? x0_tile : x1_tile), 16, 1024);
       const uint32_t ring0 = tc::smem_u32(smem) + (is_s ? 0 : C::OFF_RING_B);
       uint32_t tg = 0, n_items = 0;
@@ -385,7 +403,7 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
           VSA2_WAIT(&misc->ds_ready, tg & 1);
           tc::tc_fence_after();
           if (tc::elect_one()) {
-            if (PASS == 0) mma_out_ts<D, SPLIT, false>(tmem_base + TM_ACC0, tmem_base + TM_DP + (tg % NDP) * 128, ring_a + sa * C::SLOT, tt > 0);
+            if (PASS == 0) mma_out_ts<D, SPLIT, false, F16>(tmem_base + TM_ACC0, tmem_base + TM_DP + (tg % NDP) * 128, ring_a + sa * C::SLOT, tt > 0);
             else mma_out_ts<D, SPLIT, true>(tmem_base + TM_ACC0, tmem_base + TM_DS, ring_a + sa * C::SLOT, tt > 0);
             tc::mma_commit(&misc->a_empty[sa]);
             tc::mma_commit(PASS == 0 ? &misc->dp_free[tg % NDP] : &misc->ds_free);
@@ -521,7 +539,15 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
     const int member = row >> 6;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint32_t tg = 0, n_items = 0;
+    uint32_t sat = 0u;        // F16: largest magnitudes of the dS values this thread rounded
     for (uint32_t n_all = 0;; ++n_all) {
+      if constexpr (F16) {
+        // a dS at the clamp (or not a number): the result of this launch is not to be used, the fallback launch redoes it
+        if ((sat & 0xffffu) >= 0x7bffu || (sat >> 16) >= 0x7bffu) {
+          atomicExch(a.range_flag, 1);
+          sat = 0u;
+        }
+      }
       VSA2_NEXT_ITEM(item, n_all);
       ItemLists<PASS> il;
       il.init(g, item);
@@ -565,7 +591,9 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
                 const float d = p * (__uint_as_float(dp[32 * c + e]) - dlt);
                 ds[e] = (full || ((vm >> (32 * c + e)) & 1ull)) ? d : 0.f;
               }
-              store_operand_chunk<SPLIT>(lane_addr + TM_DP + dpb + 64 * half + 32 * c, ds);   // dS over the dP columns it came from
+              // dS over the dP columns it came from
+              if constexpr (F16) store_operand_chunk_f16(lane_addr + TM_DP + dpb + 64 * half + 32 * c, ds, sat);
+              else store_operand_chunk<SPLIT>(lane_addr + TM_DP + dpb + 64 * half + 32 * c, ds);
             }
           } else {
             tc::tmem_ld_wait();
@@ -721,17 +749,17 @@ bool fine_bwd128_supported(const Geo& g) {
   return g.Lt == 0 && g.N % 2 == 0 && g.rep <= 16 && (g.D == 64 || g.D == 128);
 }
 
-template <int D, int PASS, bool SPLIT>
+template <int D, int PASS, bool SPLIT, bool F16 = false>
 static cudaError_t launch_bwd128(const CUtensorMap& x0, const CUtensorMap& x1, const CUtensorMap& y0, const CUtensorMap& y1,
                                  const Geo& g, const Bwd128Args& a, int grid, cudaStream_t st) {
   cudaError_t e;
   cudaFuncAttributes fa;
-  if ((e = cudaFuncGetAttributes(&fa, fine_bwd128_tc_kernel<D, PASS, SPLIT>)) != cudaSuccess) return e;
+  if ((e = cudaFuncGetAttributes(&fa, fine_bwd128_tc_kernel<D, PASS, SPLIT, F16>)) != cudaSuccess) return e;
   if (fa.numRegs * kW2Threads < 256 * 56 + 256 * 200) return cudaErrorLaunchOutOfResources;
-  if ((e = cudaFuncSetAttribute(fine_bwd128_tc_kernel<D, PASS, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if ((e = cudaFuncSetAttribute(fine_bwd128_tc_kernel<D, PASS, SPLIT, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)Bwd128<D>::smem_bytes)))
     return e;
-  fine_bwd128_tc_kernel<D, PASS, SPLIT><<<grid, kW2Threads, Bwd128<D>::smem_bytes, st>>>(x0, x1, y0, y1, g, a);
+  fine_bwd128_tc_kernel<D, PASS, SPLIT, F16><<<grid, kW2Threads, Bwd128<D>::smem_bytes, st>>>(x0, x1, y0, y1, g, a);
   return cudaGetLastError();
 }
 
@@ -739,20 +767,38 @@ static cudaError_t launch_bwd128(const CUtensorMap& x0, const CUtensorMap& x1, c
 // launch_fine_bwd_dq_tc
 cudaError_t launch_fine_bwd128_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                      const float* lse, const float* delta, const int* row_ptr, const int* col_idx,
-                                     const float* dqc, void* dq, StatusBlock* status, cudaStream_t st) {
+                                     const float* dqc, void* dq, StatusBlock* status, cudaStream_t st, void* q16, void* k16) {
   if (!fine_bwd128_supported(g)) return cudaErrorInvalidValue;
-  CUtensorMap tq, tk, tv, tdo;
+  const bool f16 = fine_bwd_dq_uses_f16(g) && q16 != nullptr && k16 != nullptr;
+  CUtensorMap tq, tk, tv, tdo, tq16, tk16;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
       !make_cube_tmap(&tdo, d_o, g, g.Hq))
+    return cudaErrorInvalidValue;
+  if (f16 && (!make_cube_tmap(&tq16, reinterpret_cast<const bf16*>(q16), g, g.Hq) ||      // (same element size and layout)
+              !make_cube_tmap(&tk16, reinterpret_cast<const bf16*>(k16), g, g.Hkv)))
     return cudaErrorInvalidValue;
   int dev = 0, sms = 0;
   cudaError_t e;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  Bwd128Args a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, nullptr, dq, nullptr, status};
+  int* flag = &status->pad[kRangeFlagSlot];
+  Bwd128Args a{&status->pad[2], lse, delta, row_ptr, col_idx, dqc, nullptr, dq, nullptr, status, flag, 0};
   const int total = g.batch * g.Hq * (g.N / 2);
   const int grid = total < sms ? total : sms;
   const bool split = !(g.flags & VSA2_FLAG_FAST_BWD);
+  if (f16) {
+    // the copy, the fp16 form, and the pair form that runs only if the range flag came up (see launch_fine_bwd_dq_tc)
+    if ((e = launch_cast_bf16_to_f16(q, q16, (size_t)g.batch * g.Hq * g.S * g.D, k, k16, (size_t)g.batch * g.Hkv * g.S * g.D, flag,
+                                     st)) != cudaSuccess)
+      return e;
+    a.when = 1;
+    e = g.D == 128 ? launch_bwd128<128, 0, false, true>(tq16, tdo, tk16, tv, g, a, grid, st)
+                   : launch_bwd128<64, 0, false, true>(tq16, tdo, tk16, tv, g, a, grid, st);
+    if (e != cudaSuccess) return e;
+    a.when = 2;
+    a.item_counter = &status->pad[kRangeFlagSlot + 1];
+    return g.D == 128 ? launch_bwd128<128, 0, true>(tq, tdo, tk, tv, g, a, grid, st) : launch_bwd128<64, 0, true>(tq, tdo, tk, tv, g, a, grid, st);
+  }
   if (g.D == 128) return split ? launch_bwd128<128, 0, true>(tq, tdo, tk, tv, g, a, grid, st) : launch_bwd128<128, 0, false>(tq, tdo, tk, tv, g, a, grid, st);
   return split ? launch_bwd128<64, 0, true>(tq, tdo, tk, tv, g, a, grid, st) : launch_bwd128<64, 0, false>(tq, tdo, tk, tv, g, a, grid, st);
 }

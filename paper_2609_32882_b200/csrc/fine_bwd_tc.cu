@@ -42,16 +42,6 @@ struct DqArgs {
   int when;
 };
 
-// Slot of StatusBlock.pad that holds the range flag of the fp16 dQ pass
-constexpr int kRangeFlagSlot = 8;
-
-// fp32 pair -> packed fp16 pair (`lo` in the low half), values beyond the fp16 range clamped to +-65504
-__device__ __forceinline__ uint32_t pack_f16x2_sat(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-
 // Copies of two bf16 tensors in fp16 (8 elements per thread and step).  Every finite bf16 below 65520 in magnitude has an
 // exact fp16 image down to 2^-24 granularity (fp16 keeps more mantissa bits), so products of the copies equal the products
 // of the originals; a finite value beyond that range sets `range_flag` and the caller's fp16 kernels stand back.
@@ -488,10 +478,9 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
     fine_bwd_dq_tc_kernel<DD, SP, F><<<grid, kDqThreads, BwdTc<DD>::smem_bytes, st>>>(TQ, TK, tv, tdo, TQT, TKT, tvt, tdot, g, a); \
   } while (0)
   if (f16) {
-    const size_t nq = (size_t)g.batch * g.Hq * g.S * g.D / 8, nk = (size_t)g.batch * g.Hkv * g.S * g.D / 8;
-    cast_bf16_to_f16_kernel<<<sms * 16, 256, 0, st>>>(reinterpret_cast<const uint4*>(q), reinterpret_cast<uint4*>(q16), nq,
-                                                     reinterpret_cast<const uint4*>(k), reinterpret_cast<uint4*>(k16), nk, flag);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_cast_bf16_to_f16(q, q16, (size_t)g.batch * g.Hq * g.S * g.D, k, k16, (size_t)g.batch * g.Hkv * g.S * g.D, flag,
+                                     st)) != cudaSuccess)
+      return e;
     a.when = 1;
     if (g.D == 128) VSA2_LAUNCH_DQ(128, false, true, tq, tk, tqt, tkt);
     else VSA2_LAUNCH_DQ(64, false, true, tq, tk, tqt, tkt);
@@ -510,6 +499,18 @@ cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, co
     else VSA2_LAUNCH_DQ(64, false, false, tq, tk, tqt, tkt);
   }
 #undef VSA2_LAUNCH_DQ
+  return cudaGetLastError();
+}
+
+cudaError_t launch_cast_bf16_to_f16(const bf16* a, void* a16, size_t na, const bf16* b, void* b16, size_t nb, int* range_flag,
+                                    cudaStream_t st) {
+  int sms = 0;
+  cudaError_t e;
+  if ((e = bwd_sm_count(&sms)) != cudaSuccess) return e;
+  if ((na | nb) & 7) return cudaErrorInvalidValue;
+  cast_bf16_to_f16_kernel<<<sms * 16, 256, 0, st>>>(reinterpret_cast<const uint4*>(a), reinterpret_cast<uint4*>(a16), na / 8,
+                                                     reinterpret_cast<const uint4*>(b), reinterpret_cast<uint4*>(b16), nb / 8,
+                                                     range_flag);
   return cudaGetLastError();
 }
 

@@ -76,6 +76,13 @@ __device__ __forceinline__ void mma_pairT_mnmajor_n128(uint32_t tm_acc, uint32_t
   }
 }
 
+// fp32 pair -> packed fp16 pair (`lo` in the low half), values beyond the fp16 range clamped to +-65504
+__device__ __forceinline__ uint32_t pack_f16x2_sat(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
 // x -> (bf16(x), bf16(x - bf16(x))) for two values, packed like pack_bf16x2
 __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
   hi = pack_bf16x2(x0, x1);

@@ -351,3 +351,39 @@ def test_group_shared_routing_is_refused_for_per_row_budgets():
     with pytest.raises(vb.Vsa2Error) as e:
         run.route()
     assert e.value.code == vb.ERR_UNSUPPORTED
+
+
+def _dq_of(wl, data, flags):
+    run = CudaPath(wl, data, out_dtype=vb.F32, flags=flags)
+    run.route()
+    run.forward()
+    run.backward()
+    return run.dq.clone(), run
+
+
+@pytest.mark.parametrize("what", ["in_range", "large_k", "large_do"])
+def test_dq_pass_leaves_its_fp16_form_when_a_value_leaves_the_fp16_range(what):
+    """The default dQ pass works on fp16 copies of Q and K and rounds dS to fp16.  A finite |K| beyond the fp16 range, or a
+    dS beyond it (here: a large dO), must hand the pass back to the bf16-pair form, whose result VSA2_FLAG_PRECISE_BWD gives
+    directly: the two runs then agree bit for bit.  In range the two forms differ (in the last bits), which shows that the
+    fp16 form is the one that ran, and both sit inside the stated bound."""
+    wl = MINI_SEQ
+    data = syn.make_inputs(wl)
+    if what == "large_k":
+        k = data["k"].copy()
+        k[0, 0, 5, 3] = 0x4780           # bf16 bits of 65536: finite, beyond the largest fp16 value
+        data["k"] = k
+    if what == "large_do":
+        data["do"] = syn.f32_to_bf16_bits(syn.bf16_bits_to_f32(data["do"]) * np.float32(3.0e6))
+    dq_default, run = _dq_of(wl, data, 0)
+    dq_pair, _ = _dq_of(wl, data, vb.FLAG_PRECISE_BWD)
+    assert torch.isfinite(dq_default).all()
+    if what == "in_range":
+        assert not torch.equal(dq_default, dq_pair)
+        geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+        a = oracle_arrays(data)
+        want = orc.backward(a["q"], a["k"], a["v"], a["gate"], run.mask, geo, 1.0 / np.sqrt(wl.head_dim), a["do"])[0]
+        assert_close("dQ (fp16 form)", to_f64(dq_default), want)
+        assert_close("dQ (pair form)", to_f64(dq_pair), want)
+    else:
+        assert torch.equal(dq_default, dq_pair)
