@@ -602,14 +602,16 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
     const size_t list_need = (size_t)fx.batch * fx.Hkv * fx.N + 1, list_have = (size_t)n.batch * n.Hq * n.N * n.D;
     int* item_list = list_need <= list_have ? reinterpret_cast<int*>(d_oc_hat) : nullptr;
     const bool two = !dkv128 && fine_bwd_dkv_splits_long_columns(fx, true);
-    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, two ? (item_list ? 3 : 2) : 1);
+    const bool f16 = two && dq_pass_f16(g) && !wide128;      // the dQ pass has left fp16 copies of Q and K (64-token pass)
+    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, two ? (item_list ? 3 : 2) + (f16 ? 1 : 0) : 1);
     if (dkv128)
       VSA2_CUDA(launch_fine_bwd128_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                           coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
     else
       VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                        coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st, true,
-                                       item_list));
+                                       item_list, f16 ? at<unsigned char>(workspace, bwd_f16_offset(g)) : nullptr,
+                                       f16 ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g)) : nullptr));
   }
   return VSA2_OK;
 }

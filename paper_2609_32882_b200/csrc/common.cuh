@@ -297,7 +297,8 @@ cudaError_t launch_cast_bf16_to_f16(const bf16* a, void* a16, size_t na, const b
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                   cudaStream_t st, bool split_long_columns, int* item_list);
+                                   cudaStream_t st, bool split_long_columns, int* item_list, const void* q16,
+                                   const void* k16);
 bool fine_bwd_dkv_splits_long_columns(const Geo& g, bool split_long_columns);
 
 cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,

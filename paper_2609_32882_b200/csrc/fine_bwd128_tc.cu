@@ -162,13 +162,13 @@ __device__ __forceinline__ void store_operand_chunk(uint32_t taddr, const float 
   }
 }
 
-// the same as fp16 pairs (clamped at the largest fp16 value); `sat` collects the largest magnitudes (fp16 bit patterns, two lanes)
-__device__ __forceinline__ void store_operand_chunk_f16(uint32_t taddr, const float (&v)[32], uint32_t& sat) {
+// the same as fp16 pairs (clamped at the largest fp16 value); `sat` collects the largest magnitude
+__device__ __forceinline__ void store_operand_chunk_f16(uint32_t taddr, const float (&v)[32], float& sat) {
   uint32_t h[16];
 #pragma unroll
   for (int e = 0; e < 16; ++e) {
     h[e] = pack_f16x2_sat(v[2 * e], v[2 * e + 1]);
-    sat = __vmaxu2(sat, h[e] & 0x7fff7fffu);
+    sat = max3_abs(sat, v[2 * e], v[2 * e + 1]);
   }
   tc::tmem_st_32x32b_x16(taddr, h);
 }
@@ -539,13 +539,13 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
     const int member = row >> 6;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint32_t tg = 0, n_items = 0;
-    uint32_t sat = 0u;        // F16: largest magnitudes of the dS values this thread rounded
+    float sat = 0.f;          // F16: largest magnitude of the dS values this thread rounded
     for (uint32_t n_all = 0;; ++n_all) {
       if constexpr (F16) {
-        // a dS at the clamp (or not a number): the result of this launch is not to be used, the fallback launch redoes it
-        if ((sat & 0xffffu) >= 0x7bffu || (sat >> 16) >= 0x7bffu) {
+        // a dS beyond the fp16 range (it was clamped): the result of this launch is not to be used, the fallback launch redoes it
+        if (sat >= 65504.f) {
           atomicExch(a.range_flag, 1);
-          sat = 0u;
+          sat = 0.f;
         }
       }
       VSA2_NEXT_ITEM(item, n_all);

@@ -24,6 +24,8 @@ struct DkvArgs {
   void* dv;
   StatusBlock* status;
   int k_lo, k_hi;       // the launch handles the KV blocks whose column lists hold k_lo .. k_hi entries, and leaves the others alone
+  int* range_flag;      // fp16 form and its fallback, as in DqArgs of the dQ pass (when = 0: the launch always runs)
+  int when;
   const int* item_list; // null, or [count, item, item, ...]: the items with k_lo .. k_hi entries (the launch then walks this list
                         // instead of all items: a launch for the few long lists would spend most of its time skipping)
 };
@@ -94,7 +96,13 @@ __device__ __forceinline__ bool dkv_publish_listed(ItemQueue* q, uint32_t seq, u
 // MHA: one query head per KV head (g.rep == 1): the per-head prefix of the column lists and the search in it fold away,
 // which takes several KB out of every role's per-item code and out of the producers' and statistics warps' tile loops
 // (the pass runs at the edge of the SM's instruction cache).
-template <int D, bool SPLIT, bool MHA>
+// F16 (without SPLIT): the maps of Q and K point at the fp16 copies the dQ pass has made and dS is rounded to fp16, so S and
+// the dK^T product are fp16 x fp16 instructions; dP and the dV^T product keep bf16 operands (V and dO are not copied, P is
+// rounded to bf16).  dK is where the rounding of the plain form shows (|dK| reaches 15 on the blocks most queries keep):
+// with 11 bits in dS it stays below 1e-2 there, and the second launch for the long lists is not needed.  The launch stands
+// back when the range flag is up: the dQ pass, which runs first, forms the same dS values and raises it if one of them (or
+// a value of Q or K) leaves the fp16 range.
+template <int D, bool SPLIT, bool MHA, bool F16>
 __global__ void __launch_bounds__(kDkvThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -116,6 +124,8 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int total_items = g.batch * g.Hkv * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
   const int rep = MHA ? 1 : g.rep;
+  static_assert(!F16 || !SPLIT, "the fp16 form carries no pairs");
+  if (a.when != 0 && ((*a.range_flag != 0) != (a.when == 2))) return;     // (the flag is final before this launch starts)
 
   // the launch of the few long lists lets the launch behind it in the stream (the other lists: disjoint outputs, nothing
   // read from this one) take the SMs as its CTAs leave them
@@ -232,7 +242,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             VSA2_WAIT_PARKED(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
             if (tc::elect_one()) {
-              mma_pair_kmajor<D>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+              mma_pair_kmajor<D, F16>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
               tc::mma_commit(&misc->s_full[sb]);
               if (t == nt - 1) tc::mma_commit(&misc->st_empty);
             }
@@ -286,7 +296,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc::tc_fence_after();
             if (tc::elect_one()) {
               if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, C::PBYTES, t > 0);
-              else mma_pairT_mnmajor<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
+              else mma_pairT_mnmajor<D, F16>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
               tc::mma_commit(&misc->a_empty[sa]);
               tc::mma_commit(&misc->ds_free[0]);
               if (t == nt - 1) tc::mma_commit(&misc->o_full);
@@ -415,8 +425,13 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int c = 0; c < 32; c += 2) {
               const float d0 = __uint_as_float(sv[c]) * (__uint_as_float(dp[c]) - dlt);
               const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt);
-              if constexpr (SPLIT) split_bf16x2(d0, d1, pd[c >> 1], pdl[c >> 1]);
-              else pd[c >> 1] = pack_bf16x2(d0, d1);
+              if constexpr (SPLIT) {
+                split_bf16x2(d0, d1, pd[c >> 1], pdl[c >> 1]);
+              } else if constexpr (F16) {
+                pd[c >> 1] = pack_f16x2_sat(d0, d1);     // (a dS at the clamp: the dQ pass has met the same value and raised the flag)
+              } else {
+                pd[c >> 1] = pack_bf16x2(d0, d1);
+              }
             }
             VSA2_WAIT(&misc->ds_free[0], (tg & 1) ^ 1);
             unsigned char* drow = ds_tile + row * 128;
@@ -532,9 +547,16 @@ constexpr int kDkvLongColumn = 256;
 cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                   cudaStream_t st, bool split_long_columns, int* item_list) {
+                                   cudaStream_t st, bool split_long_columns, int* item_list, const void* q16,
+                                   const void* k16) {
   if (g.rep > kMaxRep) return cudaErrorInvalidValue;
-  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot;
+  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot, tq16, tk16, tqt16, tkt16;
+  const bool f16 = q16 != nullptr && k16 != nullptr && fine_bwd_dkv_splits_long_columns(g, split_long_columns);
+  if (f16 && (!make_cube_tmap(&tq16, reinterpret_cast<const bf16*>(q16), g, g.Hq) ||       // (same element size and layout)
+              !make_cube_tmap(&tk16, reinterpret_cast<const bf16*>(k16), g, g.Hkv) ||
+              !make_text_tmap(&tqt16, reinterpret_cast<const bf16*>(q16), g, g.Hq) ||
+              !make_text_tmap(&tkt16, reinterpret_cast<const bf16*>(k16), g, g.Hkv)))
+    return cudaErrorInvalidValue;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
       !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) ||
       !make_text_tmap(&tvt, v, g, g.Hkv) || !make_text_tmap(&tdot, d_o, g, g.Hq))
@@ -545,19 +567,19 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
   const bool mha = g.rep == 1;
-#define VSA2_LAUNCH_DKV(DD, SP, MH)                                                                                                \
+#define VSA2_LAUNCH_DKV(DD, SP, MH, F, TQ, TK, TQT, TKT)                                                                         \
   do {                                                                                                                           \
     using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
-    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize,               \
+    if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP, MH, F>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
                                   (int)L_::smem_bytes)))                                                                         \
       return e;                                                                                                                  \
     cfg.dynamicSmemBytes = L_::smem_bytes;                                                                                       \
-    if ((e = cudaLaunchKernelEx(&cfg, fine_bwd_dkv_tc_kernel<DD, SP, MH>, tq, tk, tv, tdo, tqt, tkt, tvt, tdot, g, a)))          \
+    if ((e = cudaLaunchKernelEx(&cfg, fine_bwd_dkv_tc_kernel<DD, SP, MH, F>, TQ, TK, tv, tdo, TQT, TKT, tvt, tdot, g, a)))       \
       return e;                                                                                                                  \
   } while (0)
   // `overlap`: the launch may start while the launch before it in the stream is still running (programmatic dependent
-  // launch; that one releases it at its start and the two touch disjoint outputs)
-  auto launch = [&](bool split, int counter_slot, int k_lo, int k_hi, const int* list, bool overlap) -> cudaError_t {
+  // launch; that one releases it at its start and the two touch disjoint outputs).  `when`: see DkvArgs.
+  auto launch = [&](bool split, int counter_slot, int k_lo, int k_hi, const int* list, bool overlap, int when) -> cudaError_t {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kDkvThreads);
@@ -567,27 +589,44 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    DkvArgs a{&status->pad[counter_slot], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, k_lo, k_hi, list};
-    if (g.D == 128) {
-      if (split && mha) VSA2_LAUNCH_DKV(128, true, true);
-      else if (split) VSA2_LAUNCH_DKV(128, true, false);
-      else if (mha) VSA2_LAUNCH_DKV(128, false, true);
-      else VSA2_LAUNCH_DKV(128, false, false);
+    DkvArgs a{&status->pad[counter_slot], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, k_lo, k_hi,
+              &status->pad[kRangeFlagSlot], when, list};
+    if (when == 1) {       // the fp16 form (plain operands, one launch for all lists)
+      if (g.D == 128) {
+        if (mha) VSA2_LAUNCH_DKV(128, false, true, true, tq16, tk16, tqt16, tkt16);
+        else VSA2_LAUNCH_DKV(128, false, false, true, tq16, tk16, tqt16, tkt16);
+      } else {
+        if (mha) VSA2_LAUNCH_DKV(64, false, true, true, tq16, tk16, tqt16, tkt16);
+        else VSA2_LAUNCH_DKV(64, false, false, true, tq16, tk16, tqt16, tkt16);
+      }
+    } else if (g.D == 128) {
+      if (split && mha) VSA2_LAUNCH_DKV(128, true, true, false, tq, tk, tqt, tkt);
+      else if (split) VSA2_LAUNCH_DKV(128, true, false, false, tq, tk, tqt, tkt);
+      else if (mha) VSA2_LAUNCH_DKV(128, false, true, false, tq, tk, tqt, tkt);
+      else VSA2_LAUNCH_DKV(128, false, false, false, tq, tk, tqt, tkt);
     } else {
-      if (split && mha) VSA2_LAUNCH_DKV(64, true, true);
-      else if (split) VSA2_LAUNCH_DKV(64, true, false);
-      else if (mha) VSA2_LAUNCH_DKV(64, false, true);
-      else VSA2_LAUNCH_DKV(64, false, false);
+      if (split && mha) VSA2_LAUNCH_DKV(64, true, true, false, tq, tk, tqt, tkt);
+      else if (split) VSA2_LAUNCH_DKV(64, true, false, false, tq, tk, tqt, tkt);
+      else if (mha) VSA2_LAUNCH_DKV(64, false, true, false, tq, tk, tqt, tkt);
+      else VSA2_LAUNCH_DKV(64, false, false, false, tq, tk, tqt, tkt);
     }
     return cudaGetLastError();
   };
 #undef VSA2_LAUNCH_DKV
   constexpr int kAll = 0x7fffffff;
-  if (fine_bwd_dkv_wants_pair(g)) return launch(true, 3, 0, kAll, nullptr, false);
-  if (!fine_bwd_dkv_splits_long_columns(g, split_long_columns)) return launch(false, 3, 0, kAll, nullptr, false);
+  if (fine_bwd_dkv_wants_pair(g)) return launch(true, 3, 0, kAll, nullptr, false, 0);
+  if (!fine_bwd_dkv_splits_long_columns(g, split_long_columns)) return launch(false, 3, 0, kAll, nullptr, false, 0);
+  // With the fp16 copies of Q and K: one launch in the fp16 form; the two launches below then run only if the range flag
+  // came up (in the dQ pass or in this launch), on counters of their own.
+  int when = 0, slot_plain = 3;
+  if (f16) {
+    if ((e = launch(false, 3, 0, kAll, nullptr, false, 1)) != cudaSuccess) return e;
+    when = 2;
+    slot_plain = 5;
+  }
   if (item_list == nullptr) {
-    if ((e = launch(false, 3, 0, kDkvLongColumn, nullptr, false)) != cudaSuccess) return e;
-    return launch(true, 4, kDkvLongColumn + 1, kAll, nullptr, false);
+    if ((e = launch(false, slot_plain, 0, kDkvLongColumn, nullptr, false, when)) != cudaSuccess) return e;
+    return launch(true, 4, kDkvLongColumn + 1, kAll, nullptr, false, when);
   }
   // The long lists are a few hundred of the items: a small kernel collects them, the pair launch starts on them at once
   // (a handful of 0.3 ms items on 148 CTAs: it would end with most SMs idle), and the plain launch fills the SMs as the
@@ -595,8 +634,8 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   if ((e = cudaMemsetAsync(item_list, 0, sizeof(int), st)) != cudaSuccess) return e;
   dkv_list_items_kernel<<<(total + 255) / 256, 256, 0, st>>>(g, col_ptr, g.rep, total, kDkvLongColumn + 1, kAll, item_list);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  if ((e = launch(true, 4, kDkvLongColumn + 1, kAll, item_list, false)) != cudaSuccess) return e;
-  return launch(false, 3, 0, kDkvLongColumn, nullptr, true);
+  if ((e = launch(true, 4, kDkvLongColumn + 1, kAll, item_list, false, when)) != cudaSuccess) return e;
+  return launch(false, slot_plain, 0, kDkvLongColumn, nullptr, true, when);
 }
 
 // whether launch_fine_bwd_dkv_tc runs as two launches for this problem

@@ -272,13 +272,13 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     cpos.init(g, row & 63);
     const int blk = row >> 6;
     uint32_t tg = 0, n_items = 0;
-    uint32_t sat = 0u;        // F16: largest magnitudes (as fp16 bit patterns, two lanes) of the dS values this thread rounded
+    float sat = 0.f;          // F16: largest magnitude of the dS values this thread rounded
     for (uint32_t n_all = 0;; ++n_all) {
       if constexpr (F16) {
-        // a dS at the clamp (or not a number): the result of this launch is not to be used, the fallback launch redoes it
-        if ((sat & 0xffffu) >= 0x7bffu || (sat >> 16) >= 0x7bffu) {
+        // a dS beyond the fp16 range (it was clamped): the result of this launch is not to be used, the fallback launch redoes it
+        if (sat >= 65504.f) {
           atomicExch(a.range_flag, 1);
-          sat = 0u;
+          sat = 0.f;
         }
       }
       VSA2_NEXT_ITEM(item, n_all);
@@ -348,7 +348,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
               } else if constexpr (F16) {
                 packed[2 * c4] = valid ? pack_f16x2_sat(d0, d1) : 0u;
                 packed[2 * c4 + 1] = valid ? pack_f16x2_sat(d2, d3) : 0u;
-                sat = __vmaxu2(sat, __vmaxu2(packed[2 * c4] & 0x7fff7fffu, packed[2 * c4 + 1] & 0x7fff7fffu));
+                sat = max3_abs(max3_abs(sat, d0, d1), d2, d3);
               } else {
                 packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
                 packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;

@@ -83,6 +83,12 @@ __device__ __forceinline__ uint32_t pack_f16x2_sat(float lo, float hi) {
   return r;
 }
 
+// max(m, |a|, |b|) in one instruction (the three-input maximum of sm_100; the absolute values fold into it)
+__device__ __forceinline__ float max3_abs(float m, float a, float b) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b)));
+  return r;
+}
 // x -> (bf16(x), bf16(x - bf16(x))) for two values, packed like pack_bf16x2
 __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
   hi = pack_bf16x2(x0, x1);
