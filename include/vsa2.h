@@ -67,19 +67,26 @@ enum { VSA2_FLAG_NO_COARSE = 1,       /* skip the coarse branch: O = O_f (the ga
 enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the pooled grid with bf16 operands as well
                                          (about 8x faster; O_c then carries bf16 operand rounding: O stays within the
                                          output bound, dGate of a later backward may exceed 2e-2 by about 2x) */
-/* Precision of the backward passes.  P and dS are the bf16 operands of the dV, dK and dQ products; rounded once (2^-9
- * relative) they alone push the worst elements of large gradients (|g| > 5) past max abs err 2e-2.  By default the dQ pass
- * always, and the dK/dV pass for GQA groups (where a KV block sums several heads), carry them as a bf16 pair -- the value
- * and the bf16 rounding of what that lost -- in one product of twice the width.  Measured on 720p / 480p samples against
- * the oracle (fp32 outputs): dQ 7e-3 instead of 2.5e-2, GQA dK 8e-3 instead of 2.6e-2.  With one query head per KV head the
- * rounding of the plain form leaves 1 - 2e-3 of a block's largest gradient; only KV blocks that nearly every query keeps have
- * gradients large enough (|dK| = 15 on the 720p sample) for that to cross 2e-2, so the dK/dV pass computes the blocks kept by
- * more than 256 query blocks with pairs in a second launch (about +5 % of that pass) and the others plain.
- * With cubes of 128 tokens the pair of the dQ pass travels along the contraction instead; a dK/dV pass that needs pairs (GQA, or
- * VSA2_FLAG_PRECISE_BWD) runs on the 64-token halves, the others on 128 x 128 tiles. */
-enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once everywhere (dQ pass about 15 % faster, GQA dK/dV pass about 30 %) */
-enum { VSA2_FLAG_PRECISE_BWD = 8 };   /* carry the pair in the dK/dV pass for MHA as well (that pass about 35 % slower): for maps
-                                         that keep only a few blocks per row, where the softmax is sharply peaked */
+/* Precision of the backward passes.  P and dS are 16-bit operands of the dV, dK and dQ products; rounded once to bf16 (2^-9
+ * relative) they alone push the worst elements of large gradients (|g| > 5) past max abs err 2e-2 (720p sample, fp32 outputs:
+ * dQ 2.5e-2; with one query head per KV head the KV blocks that nearly every query keeps reach |dK| = 15 and 1.5 - 2.7e-2).
+ * Default: the dQ pass works on fp16 copies of Q and K that it makes in the workspace (every bf16 value inside the fp16
+ * range has an exact fp16 image, so S is unchanged) and rounds dS to fp16, 11 significant bits instead of 8, at the speed
+ * of the once-rounded form; with one query head per KV head the dK/dV pass does the same for S, dS and its dK product (P and
+ * the dV product stay bf16: |dV| is small).  Measured against the oracle (fp32 outputs, 720p sample): dQ 8.7e-3, dK 3.5e-3.
+ * A range flag guards the fp16 forms: a finite |Q| or |K| of 65520 or more, or a |dS| of 65504 or more, and the passes are
+ * redone by the bf16-pair kernels described next (launched behind the fp16 ones, they return at once while the flag is clear).
+ * The pair form carries X as the bf16 value and the bf16 rounding of what that lost, in one product of twice the width: the
+ * dK/dV pass of GQA groups (where a KV block sums several heads) uses it by default (GQA dK 8e-3 instead of 2.6e-2), and the
+ * fallback of the one-head-per-KV-head case uses it for the KV blocks kept by more than 256 query blocks.
+ * With cubes of 128 tokens the dQ pass has the same fp16 form (its pair form, the fallback, travels along the contraction); a
+ * dK/dV pass that needs pairs (GQA, or VSA2_FLAG_PRECISE_BWD) runs on the 64-token halves, the others on 128 x 128 tiles with
+ * bf16 operands. */
+enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once to bf16 everywhere, no fp16 copies (saves the 0.5 ms copy at 720p; GQA
+                                         dK/dV pass about 30 % faster) */
+enum { VSA2_FLAG_PRECISE_BWD = 8 };   /* bf16 pairs in the dQ pass and in the dK/dV pass, for MHA as well (dQ pass about 15 %, dK/dV
+                                         pass about 35 % slower): for maps that keep only a few blocks per row, where the softmax is
+                                         sharply peaked and P itself needs the extra bits */
 enum { VSA2_FLAG_GROUP_ROUTING = 256 };/* vsa2_route: the query heads of one KV group share one block map ("group head", Sec. 4
                                          ablation): the block scores of the group's heads are added before the TopK, so
                                          the maps written for those heads are identical.  Not with VSA2_PER_QUERY_BUDGET
@@ -227,8 +234,8 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
  *   o, lse, saved: as written by the forward call;  d_o: bf16 [batch, heads_q, L, D].
  *   dq [batch, heads_q, L, D], dk, dv [batch, heads_kv, L, D] in p->out_dtype (dk, dv summed over the
  *   query heads of a group); dgate fp32 [batch, heads_q, L] (may be NULL).
- *   workspace: >= sizes.bwd_workspace_bytes.  No floating-point atomics are used: results are
- *   bitwise reproducible run to run. */
+ *   workspace: >= sizes.bwd_workspace_bytes (without a precision flag this includes fp16 copies of Q and K: 2 bytes per
+ *   element of the two tensors).  No floating-point atomics are used: results are bitwise reproducible run to run. */
 int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
                   const vsa2_map* map, const void* o, const float* lse, const vsa2_saved* saved,
                   const void* d_o, void* dq, void* dk, void* dv, float* dgate,
