@@ -76,9 +76,13 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
  * the dV product stay bf16: |dV| is small).  Measured against the oracle (fp32 outputs, 720p sample): dQ 8.7e-3, dK 3.5e-3.
  * A range flag guards the fp16 forms: a finite |Q| or |K| of 65520 or more, or a |dS| of 65504 or more, and the passes are
  * redone by the bf16-pair kernels described next (launched behind the fp16 ones, they return at once while the flag is clear).
+ * GQA groups (a KV block sums the query blocks of several heads) with TopK >= 8: the dK/dV pass makes fp16 copies of V and dO
+ * as well and runs all four products in fp16, P included (480p sample: dK 9.4e-3, dV 2.7e-3; once-rounded bf16 2.2e-2 and
+ * 1.4e-2), about 30 % faster than the pair form.
  * The pair form carries X as the bf16 value and the bf16 rounding of what that lost, in one product of twice the width: the
- * dK/dV pass of GQA groups (where a KV block sums several heads) uses it by default (GQA dK 8e-3 instead of 2.6e-2), and the
- * fallback of the one-head-per-KV-head case uses it for the KV blocks kept by more than 256 query blocks.
+ * dK/dV pass of GQA groups uses it when rows keep fewer than 8 blocks or have per-row budgets (sharply peaked weights, where
+ * 11 bits do not do), and as its fallback; the fallback of the one-head-per-KV-head case uses it for the KV blocks kept by more
+ * than 256 query blocks.
  * With cubes of 128 tokens the dQ pass has the same fp16 form (its pair form, the fallback, travels along the contraction); a
  * dK/dV pass that needs pairs (GQA, or VSA2_FLAG_PRECISE_BWD) runs on the 64-token halves, the others on 128 x 128 tiles with
  * bf16 operands. */
@@ -234,8 +238,8 @@ int vsa2_attn_fwd(const vsa2_params* p, const void* q, const void* k, const void
  *   o, lse, saved: as written by the forward call;  d_o: bf16 [batch, heads_q, L, D].
  *   dq [batch, heads_q, L, D], dk, dv [batch, heads_kv, L, D] in p->out_dtype (dk, dv summed over the
  *   query heads of a group); dgate fp32 [batch, heads_q, L] (may be NULL).
- *   workspace: >= sizes.bwd_workspace_bytes (without a precision flag this includes fp16 copies of Q and K: 2 bytes per
- *   element of the two tensors).  No floating-point atomics are used: results are bitwise reproducible run to run. */
+ *   workspace: >= sizes.bwd_workspace_bytes (without a precision flag this includes fp16 copies of Q and K, for GQA groups
+ *   also of V and dO: 2 bytes per element of those tensors).  No floating-point atomics are used: results are bitwise reproducible run to run. */
 int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void* v, const float* gate,
                   const vsa2_map* map, const void* o, const float* lse, const vsa2_saved* saved,
                   const void* d_o, void* dq, void* dk, void* dv, float* dgate,

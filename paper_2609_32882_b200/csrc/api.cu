@@ -223,8 +223,13 @@ bool dq_pass_f16(const Geo& g) { return fine_bwd_dq_uses_f16(g); }
 size_t bwd_f16_offset(const Geo& g) { return align_up(bwd_base_bytes(g) + text_map_layout(g, true).total, 256); }
 size_t bwd_q16_bytes(const Geo& g) { return align_up((size_t)g.batch * g.Hq * g.S * g.D * sizeof(bf16), 256); }
 size_t bwd_k16_bytes(const Geo& g) { return align_up((size_t)g.batch * g.Hkv * g.S * g.D * sizeof(bf16), 256); }
+// GQA groups: fp16 copies of V and dO as well, for the all-fp16 dK/dV pass (behind the copies of Q and K)
+bool dkv_pass_gqa_f16(const Geo& g) { return dq_pass_f16(g) && fine_bwd_dkv_gqa_uses_f16(g); }
 size_t bwd_workspace_bytes(const Geo& g) {
-  return dq_pass_f16(g) ? bwd_f16_offset(g) + bwd_q16_bytes(g) + bwd_k16_bytes(g) : bwd_base_bytes(g) + text_map_layout(g, true).total;
+  if (!dq_pass_f16(g)) return bwd_base_bytes(g) + text_map_layout(g, true).total;
+  size_t n = bwd_f16_offset(g) + bwd_q16_bytes(g) + bwd_k16_bytes(g);
+  if (dkv_pass_gqa_f16(g)) n += bwd_k16_bytes(g) + bwd_q16_bytes(g);      // V like K, dO like Q
+  return n;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -602,8 +607,10 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
     const size_t list_need = (size_t)fx.batch * fx.Hkv * fx.N + 1, list_have = (size_t)n.batch * n.Hq * n.N * n.D;
     int* item_list = list_need <= list_have ? reinterpret_cast<int*>(d_oc_hat) : nullptr;
     const bool two = !dkv128 && fine_bwd_dkv_splits_long_columns(fx, true);
-    const bool f16 = two && dq_pass_f16(g) && !wide128;      // the dQ pass has left fp16 copies of Q and K (64-token pass)
-    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, two ? (item_list ? 3 : 2) + (f16 ? 1 : 0) : 1);
+    const bool gqa16 = !dkv128 && dkv_pass_gqa_f16(g);    // (the copy of V and dO, the all-fp16 form, the pair form as its fallback)
+    const bool f16 = (two || gqa16) && dq_pass_f16(g);              // the dQ pass has left fp16 copies of Q and K
+    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, two ? (item_list ? 3 : 2) + (f16 ? 1 : 0) : (gqa16 ? 3 : 1));
+    unsigned char* v16 = gqa16 ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g) + bwd_k16_bytes(g)) : nullptr;
     if (dkv128)
       VSA2_CUDA(launch_fine_bwd128_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                           coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
@@ -611,7 +618,8 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
       VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                        coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st, true,
                                        item_list, f16 ? at<unsigned char>(workspace, bwd_f16_offset(g)) : nullptr,
-                                       f16 ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g)) : nullptr));
+                                       f16 ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g)) : nullptr, v16,
+                                       gqa16 ? v16 + bwd_k16_bytes(g) : nullptr));
   }
   return VSA2_OK;
 }

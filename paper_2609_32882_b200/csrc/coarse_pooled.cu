@@ -147,7 +147,7 @@ cudaError_t launch_coarse_bwd_pooled(const Geo& g, const float* qc, const float*
   if ((e = launch_fine_bwd_dq_tc(p, q16, k16, v16, do16, lse_c, delta, ptr, idx, nullptr, dqc, status, st, nullptr, nullptr)) != cudaSuccess) return e;
   const bool grouped = g.rep > 1;
   if ((e = launch_fine_bwd_dkv_tc(p, q16, k16, v16, do16, lse_c, delta, ptr, idx, nullptr, nullptr, grouped ? dk_kv : dkc,
-                                  grouped ? dv_kv : dvc, status, st, false, nullptr, nullptr, nullptr)) != cudaSuccess)
+                                  grouped ? dv_kv : dvc, status, st, false, nullptr, nullptr, nullptr, nullptr, nullptr)) != cudaSuccess)
     return e;
   if (grouped) {
     const size_t per_head4 = (size_t)g.N * g.D / 4;

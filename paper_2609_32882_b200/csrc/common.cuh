@@ -298,7 +298,8 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
                                    cudaStream_t st, bool split_long_columns, int* item_list, const void* q16,
-                                   const void* k16);
+                                   const void* k16, void* v16, void* do16);
+bool fine_bwd_dkv_gqa_uses_f16(const Geo& g);
 bool fine_bwd_dkv_splits_long_columns(const Geo& g, bool split_long_columns);
 
 cudaError_t launch_bwd_preprocess(const Geo& g, const bf16* d_o, const void* o, const bf16* o_res, const float* gate,

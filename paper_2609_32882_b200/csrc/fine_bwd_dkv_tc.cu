@@ -102,7 +102,9 @@ __device__ __forceinline__ bool dkv_publish_listed(ItemQueue* q, uint32_t seq, u
 // with 11 bits in dS it stays below 1e-2 there, and the second launch for the long lists is not needed.  The launch stands
 // back when the range flag is up: the dQ pass, which runs first, forms the same dS values and raises it if one of them (or
 // a value of Q or K) leaves the fp16 range.
-template <int D, bool SPLIT, bool MHA, bool F16>
+// F16 = 2: all four maps point at fp16 copies and P is rounded to fp16 as well (every product fp16 x fp16): the form for GQA
+// groups, where a KV block sums the query blocks of several heads and bf16 P leaves dV at 1.4e-2 (480p sample, |dV| = 11).
+template <int D, bool SPLIT, bool MHA, int F16>
 __global__ void __launch_bounds__(kDkvThreads, 1)
 fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -124,7 +126,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int total_items = g.batch * g.Hkv * g.N;
   const float c2 = g.scale * 1.4426950408889634f;
   const int rep = MHA ? 1 : g.rep;
-  static_assert(!F16 || !SPLIT, "the fp16 form carries no pairs");
+  static_assert(F16 == 0 || !SPLIT, "the fp16 forms carry no pairs");
   if (a.when != 0 && ((*a.range_flag != 0) != (a.when == 2))) return;     // (the flag is final before this launch starts)
 
   // the launch of the few long lists lets the launch behind it in the stream (the other lists: disjoint outputs, nothing
@@ -242,7 +244,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             VSA2_WAIT_PARKED(&misc->s_free[sb], pb ^ 1);
             tc::tc_fence_after();
             if (tc::elect_one()) {
-              mma_pair_kmajor<D, F16>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
+              mma_pair_kmajor<D, F16 != 0>(tmem_base + sb * 64, base + sa * C::SLOT, b_addr);
               tc::mma_commit(&misc->s_full[sb]);
               if (t == nt - 1) tc::mma_commit(&misc->st_empty);
             }
@@ -251,7 +253,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             VSA2_WAIT_PARKED(&misc->dp_free[sb], pb ^ 1);
             tc::tc_fence_after();
             if (tc::elect_one()) {
-              mma_pair_kmajor<D>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
+              mma_pair_kmajor<D, F16 == 2>(tmem_base + 128 + sb * 64, base + C::OFF_RING_B + sb * C::SLOT, b_addr);
               tc::mma_commit(&misc->dp_full[sb]);
               tc::mma_commit(&misc->b_empty[sb]);
               if (t == nt - 1) tc::mma_commit(&misc->st_empty);
@@ -285,7 +287,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc::tc_fence_after();
             if (tc::elect_one()) {
               if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, C::PBYTES, t > 0);
-              else mma_pairT_mnmajor<D>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
+              else mma_pairT_mnmajor<D, F16 == 2>(tmem_base + TM_DV, base + C::OFF_RING_B + sv * C::SLOT, b_addr, t > 0);
               tc::mma_commit(&misc->b_empty[sv]);
               tc::mma_commit(&misc->p_free);
               if (t == nt - 1) tc::mma_commit(&misc->o_full);
@@ -296,7 +298,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc::tc_fence_after();
             if (tc::elect_one()) {
               if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, C::PBYTES, t > 0);
-              else mma_pairT_mnmajor<D, F16>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
+              else mma_pairT_mnmajor<D, F16 != 0>(tmem_base + TM_DK, base + sa * C::SLOT, b_addr, t > 0);
               tc::mma_commit(&misc->a_empty[sa]);
               tc::mma_commit(&misc->ds_free[0]);
               if (t == nt - 1) tc::mma_commit(&misc->o_full);
@@ -398,6 +400,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               sv[c] = __float_as_uint(p0);
               sv[c + 1] = __float_as_uint(p1);
               if constexpr (SPLIT) split_bf16x2(p0, p1, pp[c >> 1], pl[c >> 1]);
+              else if constexpr (F16 == 2) pp[c >> 1] = pack_f16x2_sat(p0, p1);
               else pp[c >> 1] = pack_bf16x2(p0, p1);
             }
             VSA2_WAIT(&misc->p_free, (tg & 1) ^ 1);
@@ -427,7 +430,7 @@ fine_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
               const float d1 = __uint_as_float(sv[c + 1]) * (__uint_as_float(dp[c + 1]) - dlt);
               if constexpr (SPLIT) {
                 split_bf16x2(d0, d1, pd[c >> 1], pdl[c >> 1]);
-              } else if constexpr (F16) {
+              } else if constexpr (F16 != 0) {
                 pd[c >> 1] = pack_f16x2_sat(d0, d1);     // (a dS at the clamp: the dQ pass has met the same value and raised the flag)
               } else {
                 pd[c >> 1] = pack_bf16x2(d0, d1);
@@ -548,10 +551,13 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
                                    const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                    const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
                                    cudaStream_t st, bool split_long_columns, int* item_list, const void* q16,
-                                   const void* k16) {
+                                   const void* k16, void* v16, void* do16) {
   if (g.rep > kMaxRep) return cudaErrorInvalidValue;
-  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot, tq16, tk16, tqt16, tkt16;
-  const bool f16 = q16 != nullptr && k16 != nullptr && fine_bwd_dkv_splits_long_columns(g, split_long_columns);
+  CUtensorMap tq, tk, tv, tdo, tqt, tkt, tvt, tdot, tq16, tk16, tqt16, tkt16, tv16, tdo16, tvt16, tdot16;
+  // GQA groups without a precision flag take the all-fp16 form when they are given scratch for fp16 copies of V and dO as
+  // well (their fallback is the pair form over all lists)
+  const bool gqa16 = fine_bwd_dkv_gqa_uses_f16(g) && split_long_columns && v16 != nullptr && do16 != nullptr;
+  const bool f16 = q16 != nullptr && k16 != nullptr && (gqa16 || fine_bwd_dkv_splits_long_columns(g, split_long_columns));
   if (f16 && (!make_cube_tmap(&tq16, reinterpret_cast<const bf16*>(q16), g, g.Hq) ||       // (same element size and layout)
               !make_cube_tmap(&tk16, reinterpret_cast<const bf16*>(k16), g, g.Hkv) ||
               !make_text_tmap(&tqt16, reinterpret_cast<const bf16*>(q16), g, g.Hq) ||
@@ -561,20 +567,25 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
       !make_cube_tmap(&tdo, d_o, g, g.Hq) || !make_text_tmap(&tqt, q, g, g.Hq) || !make_text_tmap(&tkt, k, g, g.Hkv) ||
       !make_text_tmap(&tvt, v, g, g.Hkv) || !make_text_tmap(&tdot, d_o, g, g.Hq))
     return cudaErrorInvalidValue;
+  if (f16 && gqa16 && (!make_cube_tmap(&tv16, reinterpret_cast<const bf16*>(v16), g, g.Hkv) ||
+                       !make_cube_tmap(&tdo16, reinterpret_cast<const bf16*>(do16), g, g.Hq) ||
+                       !make_text_tmap(&tvt16, reinterpret_cast<const bf16*>(v16), g, g.Hkv) ||
+                       !make_text_tmap(&tdot16, reinterpret_cast<const bf16*>(do16), g, g.Hq)))
+    return cudaErrorInvalidValue;
   int sms = 0;
   cudaError_t e;
   if ((e = bwd_sm_count(&sms)) != cudaSuccess) return e;
   const int total = g.batch * g.Hkv * g.N;
   const int grid = total < sms ? total : sms;
   const bool mha = g.rep == 1;
-#define VSA2_LAUNCH_DKV(DD, SP, MH, F, TQ, TK, TQT, TKT)                                                                         \
+#define VSA2_LAUNCH_DKV(DD, SP, MH, F, TQ, TK, TQT, TKT, TV, TDO, TVT, TDOT)                                                                         \
   do {                                                                                                                           \
     using L_ = BwdTc<DD, SP ? 2 : kRingA, SP ? 4 : 2>;                                                                           \
     if ((e = cudaFuncSetAttribute(fine_bwd_dkv_tc_kernel<DD, SP, MH, F>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
                                   (int)L_::smem_bytes)))                                                                         \
       return e;                                                                                                                  \
     cfg.dynamicSmemBytes = L_::smem_bytes;                                                                                       \
-    if ((e = cudaLaunchKernelEx(&cfg, fine_bwd_dkv_tc_kernel<DD, SP, MH, F>, TQ, TK, tv, tdo, TQT, TKT, tvt, tdot, g, a)))       \
+    if ((e = cudaLaunchKernelEx(&cfg, fine_bwd_dkv_tc_kernel<DD, SP, MH, F>, TQ, TK, TV, TDO, TQT, TKT, TVT, TDOT, g, a)))       \
       return e;                                                                                                                  \
   } while (0)
   // `overlap`: the launch may start while the launch before it in the stream is still running (programmatic dependent
@@ -591,29 +602,34 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
     cfg.numAttrs = overlap ? 1 : 0;
     DkvArgs a{&status->pad[counter_slot], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, k_lo, k_hi,
               &status->pad[kRangeFlagSlot], when, list};
-    if (when == 1) {       // the fp16 form (plain operands, one launch for all lists)
-      if (g.D == 128) {
-        if (mha) VSA2_LAUNCH_DKV(128, false, true, true, tq16, tk16, tqt16, tkt16);
-        else VSA2_LAUNCH_DKV(128, false, false, true, tq16, tk16, tqt16, tkt16);
-      } else {
-        if (mha) VSA2_LAUNCH_DKV(64, false, true, true, tq16, tk16, tqt16, tkt16);
-        else VSA2_LAUNCH_DKV(64, false, false, true, tq16, tk16, tqt16, tkt16);
-      }
+    if (when == 1 && gqa16) {       // every product in fp16
+      if (g.D == 128) VSA2_LAUNCH_DKV(128, false, false, 2, tq16, tk16, tqt16, tkt16, tv16, tdo16, tvt16, tdot16);
+      else VSA2_LAUNCH_DKV(64, false, false, 2, tq16, tk16, tqt16, tkt16, tv16, tdo16, tvt16, tdot16);
+    } else if (when == 1) {         // S and the dK product in fp16 (one query head per KV head)
+      if (g.D == 128) VSA2_LAUNCH_DKV(128, false, true, 1, tq16, tk16, tqt16, tkt16, tv, tdo, tvt, tdot);
+      else VSA2_LAUNCH_DKV(64, false, true, 1, tq16, tk16, tqt16, tkt16, tv, tdo, tvt, tdot);
     } else if (g.D == 128) {
-      if (split && mha) VSA2_LAUNCH_DKV(128, true, true, false, tq, tk, tqt, tkt);
-      else if (split) VSA2_LAUNCH_DKV(128, true, false, false, tq, tk, tqt, tkt);
-      else if (mha) VSA2_LAUNCH_DKV(128, false, true, false, tq, tk, tqt, tkt);
-      else VSA2_LAUNCH_DKV(128, false, false, false, tq, tk, tqt, tkt);
+      if (split && mha) VSA2_LAUNCH_DKV(128, true, true, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
+      else if (split) VSA2_LAUNCH_DKV(128, true, false, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
+      else if (mha) VSA2_LAUNCH_DKV(128, false, true, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
+      else VSA2_LAUNCH_DKV(128, false, false, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
     } else {
-      if (split && mha) VSA2_LAUNCH_DKV(64, true, true, false, tq, tk, tqt, tkt);
-      else if (split) VSA2_LAUNCH_DKV(64, true, false, false, tq, tk, tqt, tkt);
-      else if (mha) VSA2_LAUNCH_DKV(64, false, true, false, tq, tk, tqt, tkt);
-      else VSA2_LAUNCH_DKV(64, false, false, false, tq, tk, tqt, tkt);
+      if (split && mha) VSA2_LAUNCH_DKV(64, true, true, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
+      else if (split) VSA2_LAUNCH_DKV(64, true, false, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
+      else if (mha) VSA2_LAUNCH_DKV(64, false, true, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
+      else VSA2_LAUNCH_DKV(64, false, false, 0, tq, tk, tqt, tkt, tv, tdo, tvt, tdot);
     }
     return cudaGetLastError();
   };
 #undef VSA2_LAUNCH_DKV
   constexpr int kAll = 0x7fffffff;
+  if (f16 && gqa16) {
+    if ((e = launch_cast_bf16_to_f16(v, v16, (size_t)g.batch * g.Hkv * g.S * g.D, d_o, do16, (size_t)g.batch * g.Hq * g.S * g.D,
+                                     &status->pad[kRangeFlagSlot], st)) != cudaSuccess)
+      return e;
+    if ((e = launch(false, 3, 0, kAll, nullptr, false, 1)) != cudaSuccess) return e;
+    return launch(true, 4, 0, kAll, nullptr, false, 2);
+  }
   if (fine_bwd_dkv_wants_pair(g)) return launch(true, 3, 0, kAll, nullptr, false, 0);
   if (!fine_bwd_dkv_splits_long_columns(g, split_long_columns)) return launch(false, 3, 0, kAll, nullptr, false, 0);
   // With the fp16 copies of Q and K: one launch in the fp16 form; the two launches below then run only if the range flag
@@ -636,6 +652,15 @@ cudaError_t launch_fine_bwd_dkv_tc(const Geo& g, const bf16* q, const bf16* k, c
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   if ((e = launch(true, 4, kDkvLongColumn + 1, kAll, item_list, false, when)) != cudaSuccess) return e;
   return launch(false, slot_plain, 0, kDkvLongColumn, nullptr, true, when);
+}
+
+// Whether the dK/dV pass of a GQA problem takes its all-fp16 form when it is given the scratch for the four copies.  Rows that
+// keep only a few blocks have sharply peaked weights and gradients of 10 - 30 per element; a KV block then sums the heads of
+// a group at magnitudes where the 11 bits of fp16 leave 2e-2 (a per-query top-1 case with 12:3 heads: dK 2.08e-2), so those
+// problems (and per-row budgets, whose sizes the host does not know) keep the bf16 pairs.
+constexpr int kGqaF16MinTopk = 8;
+bool fine_bwd_dkv_gqa_uses_f16(const Geo& g) {
+  return g.rep > 1 && !(g.flags & (VSA2_FLAG_FAST_BWD | VSA2_FLAG_PRECISE_BWD)) && g.K >= kGqaF16MinTopk;
 }
 
 // whether launch_fine_bwd_dkv_tc runs as two launches for this problem

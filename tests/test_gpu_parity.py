@@ -353,21 +353,26 @@ def test_group_shared_routing_is_refused_for_per_row_budgets():
     assert e.value.code == vb.ERR_UNSUPPORTED
 
 
-def _dq_of(wl, data, flags):
+MINI_GQA_TOP8 = syn.Workload("mini_gqa_top8", 1, 4, 2, 128, (8, 12, 12), select_mode=syn.PER_QUERY, topk=8, seed=25)
+
+
+def _grads_of(wl, data, flags):
     run = CudaPath(wl, data, out_dtype=vb.F32, flags=flags)
     run.route()
     run.forward()
     run.backward()
-    return run.dq.clone(), run
+    return (run.dq.clone(), run.dk.clone(), run.dv.clone()), run
 
 
 @pytest.mark.parametrize("what", ["in_range", "large_k", "large_do"])
-def test_dq_pass_leaves_its_fp16_form_when_a_value_leaves_the_fp16_range(what):
-    """The default dQ pass works on fp16 copies of Q and K and rounds dS to fp16.  A finite |K| beyond the fp16 range, or a
-    dS beyond it (here: a large dO), must hand the pass back to the bf16-pair form, whose result VSA2_FLAG_PRECISE_BWD gives
-    directly: the two runs then agree bit for bit.  In range the two forms differ (in the last bits), which shows that the
-    fp16 form is the one that ran, and both sit inside the stated bound."""
-    wl = MINI_SEQ
+@pytest.mark.parametrize("wl", [MINI_SEQ, MINI_GQA_TOP8], ids=lambda w: w.name)
+def test_backward_leaves_its_fp16_forms_when_a_value_leaves_the_fp16_range(wl, what):
+    """The default dQ pass works on fp16 copies of Q and K and rounds dS to fp16; the dK/dV pass does the same for its dK
+    product and, for GQA groups that keep 8 blocks or more per row, for all four products.  A finite |K| beyond the fp16
+    range, or a dS beyond it (here: a large dO), must hand the passes back to the bf16-pair forms.  VSA2_FLAG_PRECISE_BWD runs
+    those directly: dQ then agrees bit for bit, and so do dK and dV of the GQA case (with one query head per KV head the
+    fallback of the dK/dV pass takes pairs only for lists longer than 256, so here it must equal the once-rounded form).  In range the
+    forms differ in the last bits, which shows that the fp16 forms are the ones that ran, and all sit inside the stated bound."""
     data = syn.make_inputs(wl)
     if what == "large_k":
         k = data["k"].copy()
@@ -375,15 +380,24 @@ def test_dq_pass_leaves_its_fp16_form_when_a_value_leaves_the_fp16_range(what):
         data["k"] = k
     if what == "large_do":
         data["do"] = syn.f32_to_bf16_bits(syn.bf16_bits_to_f32(data["do"]) * np.float32(3.0e6))
-    dq_default, run = _dq_of(wl, data, 0)
-    dq_pair, _ = _dq_of(wl, data, vb.FLAG_PRECISE_BWD)
-    assert torch.isfinite(dq_default).all()
+    gqa = wl.heads_q != wl.heads_kv
+    got, run = _grads_of(wl, data, 0)
+    pair, _ = _grads_of(wl, data, vb.FLAG_PRECISE_BWD)
+    for t in got:
+        assert torch.isfinite(t).all()
+    geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
+    a = oracle_arrays(data)
+    want = orc.backward(a["q"], a["k"], a["v"], a["gate"], run.mask, geo, 1.0 / np.sqrt(wl.head_dim), a["do"])
     if what == "in_range":
-        assert not torch.equal(dq_default, dq_pair)
-        geo = orc.Geometry(wl.grid, wl.cube, wl.rpool)
-        a = oracle_arrays(data)
-        want = orc.backward(a["q"], a["k"], a["v"], a["gate"], run.mask, geo, 1.0 / np.sqrt(wl.head_dim), a["do"])[0]
-        assert_close("dQ (fp16 form)", to_f64(dq_default), want)
-        assert_close("dQ (pair form)", to_f64(dq_pair), want)
+        assert not torch.equal(got[0], pair[0]) and not torch.equal(got[1], pair[1])
+        for name, x, y, w in zip(("dQ", "dK", "dV"), got, pair, want):
+            assert_close(name + " (fp16 form)", to_f64(x), w)
+            assert_close(name + " (pair form)", to_f64(y), w)
     else:
-        assert torch.equal(dq_default, dq_pair)
+        assert torch.equal(got[0], pair[0])
+        if gqa:
+            assert torch.equal(got[1], pair[1]) and torch.equal(got[2], pair[2])
+        else:
+            # no list of this problem is longer than 256: the fallback is the once-rounded kernel, which FAST_BWD runs directly
+            fast, _ = _grads_of(wl, data, vb.FLAG_FAST_BWD)
+            assert torch.equal(got[1], fast[1]) and torch.equal(got[2], fast[2])
