@@ -83,9 +83,9 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
  * dK/dV pass of GQA groups uses it when rows keep fewer than 8 blocks or have per-row budgets (sharply peaked weights, where
  * 11 bits do not do), and as its fallback; the fallback of the one-head-per-KV-head case uses it for the KV blocks kept by more
  * than 256 query blocks.
- * With cubes of 128 tokens the dQ pass has the same fp16 form (its pair form, the fallback, travels along the contraction); a
- * dK/dV pass that needs pairs (GQA, or VSA2_FLAG_PRECISE_BWD) runs on the 64-token halves, the others on 128 x 128 tiles with
- * bf16 operands. */
+ * With cubes of 128 tokens both passes have the same fp16 forms on 128 x 128 tiles (the pair form of the dQ pass, its fallback,
+ * travels along the contraction; the fallback of the dK/dV pass is its bf16 form); a dK/dV pass for GQA groups or with
+ * VSA2_FLAG_PRECISE_BWD runs on the 64-token halves. */
 enum { VSA2_FLAG_FAST_BWD = 4 };      /* round P and dS once to bf16 everywhere, no fp16 copies (saves the 0.5 ms copy at 720p; GQA
                                          dK/dV pass about 30 % faster) */
 enum { VSA2_FLAG_PRECISE_BWD = 8 };   /* bf16 pairs in the dQ pass and in the dK/dV pass, for MHA as well (dQ pass about 15 %, dK/dV

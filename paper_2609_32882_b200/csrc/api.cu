@@ -609,11 +609,14 @@ int vsa2_attn_bwd(const vsa2_params* p, const void* q, const void* k, const void
     const bool two = !dkv128 && fine_bwd_dkv_splits_long_columns(fx, true);
     const bool gqa16 = !dkv128 && dkv_pass_gqa_f16(g);    // (the copy of V and dO, the all-fp16 form, the pair form as its fallback)
     const bool f16 = (two || gqa16) && dq_pass_f16(g);              // the dQ pass has left fp16 copies of Q and K
-    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, two ? (item_list ? 3 : 2) + (f16 ? 1 : 0) : (gqa16 ? 3 : 1));
+    ProfScope ps(VSA2_KERNEL_FINE_BWD_DKV, st, dkv128 ? (dq_pass_f16(g) ? 2 : 1)
+                                                      : two ? (item_list ? 3 : 2) + (f16 ? 1 : 0) : (gqa16 ? 3 : 1));
     unsigned char* v16 = gqa16 ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g) + bwd_k16_bytes(g)) : nullptr;
     if (dkv128)
       VSA2_CUDA(launch_fine_bwd128_dkv_tc(n, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
-                                          coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st));
+                                          coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st,
+                                          dq_pass_f16(g) ? at<unsigned char>(workspace, bwd_f16_offset(g)) : nullptr,
+                                          dq_pass_f16(g) ? at<unsigned char>(workspace, bwd_f16_offset(g) + bwd_q16_bytes(g)) : nullptr));
     else
       VSA2_CUDA(launch_fine_bwd_dkv_tc(fx, qb, kb, vb, dob, lse, delta, col_ptr, row_idx, coarse ? dkc : nullptr,
                                        coarse ? dvc : nullptr, dk, dv, reinterpret_cast<StatusBlock*>(workspace), st, true,

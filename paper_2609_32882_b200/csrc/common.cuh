@@ -282,7 +282,7 @@ cudaError_t launch_fine_bwd128_dq_tc(const Geo& g, const bf16* q, const bf16* k,
 cudaError_t launch_fine_bwd128_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                       const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                       const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                      cudaStream_t st);
+                                      cudaStream_t st, const void* q16, const void* k16);
 
 // tensor-core backward passes (fine_bwd_tc.cu)
 cudaError_t launch_fine_bwd_dq_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,

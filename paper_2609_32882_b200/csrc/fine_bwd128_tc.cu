@@ -177,8 +177,9 @@ __device__ __forceinline__ void store_operand_chunk_f16(uint32_t taddr, const fl
 // stationary tiles and schedules the CTA's work items), warp 4 = issuer of S, warp 5 = issuer of dP, warp 6 = issuer of
 // the output products, warp 7 = loader of the per-column lse and delta (dK/dV pass), warps 8..15 = elementwise stage +
 // epilogue (thread = row r of the tile x one half of its columns).
-// F16 (dQ pass, without SPLIT): the maps of X0 = Q and Y0 = K point at fp16 copies and dS is rounded to fp16, so S and the dQ
-// product are fp16 x fp16 instructions (dP stays bf16 x bf16); see the 64-token dQ pass.
+// F16 (without SPLIT): the maps of X0 and Y0 (Q and K, in the order of the pass) point at fp16 copies and dS is rounded to fp16,
+// so S and the dQ (dK) product are fp16 x fp16 instructions; dP, P and the dV product stay bf16.  See the 64-token passes; as
+// there, only the dQ pass tracks the magnitude of dS.
 template <int D, int PASS, bool SPLIT, bool F16 = false>
 __global__ void __launch_bounds__(kW2Threads, 1)
 fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_constant__ CUtensorMap tm_x1,
@@ -186,7 +187,7 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
                       Bwd128Args a) {
   using C = Bwd128<D>;
   static_assert(PASS == 0 || !SPLIT, "the dK/dV pass has no room for the low-order parts of P and dS");
-  static_assert(!F16 || (PASS == 0 && !SPLIT), "the fp16 form is the dQ pass without pairs");
+  static_assert(!F16 || !SPLIT, "the fp16 forms carry no pairs");
   if (a.when != 0 && ((*a.range_flag != 0) != (a.when == 2))) return;     // (the flag is final before this launch starts)
   constexpr uint32_t NDP = PASS == 0 ? 2 : 1;                  // dP buffers
   // dQ pass: S 0; dP buffers 128, 256 (dS overwrites the dP it came from); dQ 384.
@@ -404,7 +405,7 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
           tc::tc_fence_after();
           if (tc::elect_one()) {
             if (PASS == 0) mma_out_ts<D, SPLIT, false, F16>(tmem_base + TM_ACC0, tmem_base + TM_DP + (tg % NDP) * 128, ring_a + sa * C::SLOT, tt > 0);
-            else mma_out_ts<D, SPLIT, true>(tmem_base + TM_ACC0, tmem_base + TM_DS, ring_a + sa * C::SLOT, tt > 0);
+            else mma_out_ts<D, SPLIT, true, F16>(tmem_base + TM_ACC0, tmem_base + TM_DS, ring_a + sa * C::SLOT, tt > 0);
             tc::mma_commit(&misc->a_empty[sa]);
             tc::mma_commit(PASS == 0 ? &misc->dp_free[tg % NDP] : &misc->ds_free);
             if (tt == nt_all - 1) tc::mma_commit(&misc->o_full);
@@ -649,7 +650,14 @@ fine_bwd128_tc_kernel(const __grid_constant__ CUtensorMap tm_x0, const __grid_co
                 ds[4 * e4 + 2] = __uint_as_float(pf[32 * c + 4 * e4 + 2]) * (__uint_as_float(dp[32 * c + 4 * e4 + 2]) - dl.z);
                 ds[4 * e4 + 3] = __uint_as_float(pf[32 * c + 4 * e4 + 3]) * (__uint_as_float(dp[32 * c + 4 * e4 + 3]) - dl.w);
               }
-              store_operand_chunk<false>(lane_addr + TM_DS + 32 * half + 16 * c, ds);
+              if constexpr (F16) {     // (a dS at the clamp: the dQ pass has met the same value and raised the flag)
+                uint32_t h[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) h[e] = pack_f16x2_sat(ds[2 * e], ds[2 * e + 1]);
+                tc::tmem_st_32x32b_x16(lane_addr + TM_DS + 32 * half + 16 * c, h);
+              } else {
+                store_operand_chunk<false>(lane_addr + TM_DS + 32 * half + 16 * c, ds);
+              }
             }
           }
           if (PASS == 1) tc::mbar_arrive(&misc->dlt_free);
@@ -807,21 +815,35 @@ cudaError_t launch_fine_bwd128_dq_tc(const Geo& g, const bf16* q, const bf16* k,
 cudaError_t launch_fine_bwd128_dkv_tc(const Geo& g, const bf16* q, const bf16* k, const bf16* v, const bf16* d_o,
                                       const float* lse, const float* delta, const int* col_ptr, const int* row_idx,
                                       const float* dkc, const float* dvc, void* dk, void* dv, StatusBlock* status,
-                                      cudaStream_t st) {
+                                      cudaStream_t st, const void* q16, const void* k16) {
   if (!fine_bwd128_supported(g)) return cudaErrorInvalidValue;
-  CUtensorMap tq, tk, tv, tdo;
+  // `q16`, `k16`: null, or the fp16 copies of Q and K that the dQ pass of the same call has made (and whose range flag it has
+  // settled): the pass then runs in its fp16 form, with the bf16 form behind the flag
+  const bool f16 = fine_bwd_dq_uses_f16(g) && q16 != nullptr && k16 != nullptr;
+  CUtensorMap tq, tk, tv, tdo, tq16, tk16;
   if (!make_cube_tmap(&tq, q, g, g.Hq) || !make_cube_tmap(&tk, k, g, g.Hkv) || !make_cube_tmap(&tv, v, g, g.Hkv) ||
       !make_cube_tmap(&tdo, d_o, g, g.Hq))
+    return cudaErrorInvalidValue;
+  if (f16 && (!make_cube_tmap(&tq16, reinterpret_cast<const bf16*>(q16), g, g.Hq) ||
+              !make_cube_tmap(&tk16, reinterpret_cast<const bf16*>(k16), g, g.Hkv)))
     return cudaErrorInvalidValue;
   int dev = 0, sms = 0;
   cudaError_t e;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  Bwd128Args a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status};
+  Bwd128Args a{&status->pad[3], lse, delta, col_ptr, row_idx, dkc, dvc, dk, dv, status, &status->pad[kRangeFlagSlot], 0};
   const int total = g.batch * g.Hkv * (g.N / 2);
   const int grid = total < sms ? total : sms;
   const bool split = fine_bwd_dkv_wants_pair(g);
   if (split) return cudaErrorInvalidValue;      // (the caller takes the 64-token kernels for that)
+  if (f16) {
+    a.when = 1;
+    e = g.D == 128 ? launch_bwd128<128, 1, false, true>(tk16, tv, tq16, tdo, g, a, grid, st)
+                   : launch_bwd128<64, 1, false, true>(tk16, tv, tq16, tdo, g, a, grid, st);
+    if (e != cudaSuccess) return e;
+    a.when = 2;
+    a.item_counter = &status->pad[5];
+  }
   if (g.D == 128) return launch_bwd128<128, 1, false>(tk, tv, tq, tdo, g, a, grid, st);
   return launch_bwd128<64, 1, false>(tk, tv, tq, tdo, g, a, grid, st);
 }
