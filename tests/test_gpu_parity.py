@@ -354,6 +354,7 @@ def test_group_shared_routing_is_refused_for_per_row_budgets():
 
 
 MINI_GQA_TOP8 = syn.Workload("mini_gqa_top8", 1, 4, 2, 128, (8, 12, 12), select_mode=syn.PER_QUERY, topk=8, seed=25)
+MINI_SEQ_128 = MINI_SEQ.replace(name="mini_per_sequence_cubes_of_128", cube=(4, 4, 8), rpool=(2, 2, 2), topk=3)
 
 
 def _grads_of(wl, data, flags):
@@ -365,13 +366,14 @@ def _grads_of(wl, data, flags):
 
 
 @pytest.mark.parametrize("what", ["in_range", "large_k", "large_do"])
-@pytest.mark.parametrize("wl", [MINI_SEQ, MINI_GQA_TOP8], ids=lambda w: w.name)
+@pytest.mark.parametrize("wl", [MINI_SEQ, MINI_GQA_TOP8, MINI_SEQ_128], ids=lambda w: w.name)
 def test_backward_leaves_its_fp16_forms_when_a_value_leaves_the_fp16_range(wl, what):
     """The default dQ pass works on fp16 copies of Q and K and rounds dS to fp16; the dK/dV pass does the same for its dK
     product and, for GQA groups that keep 8 blocks or more per row, for all four products.  A finite |K| beyond the fp16
     range, or a dS beyond it (here: a large dO), must hand the passes back to the bf16-pair forms.  VSA2_FLAG_PRECISE_BWD runs
     those directly: dQ then agrees bit for bit, and so do dK and dV of the GQA case (with one query head per KV head the
-    fallback of the dK/dV pass takes pairs only for lists longer than 256, so here it must equal the once-rounded form).  In range the
+    fallback of the dK/dV pass takes pairs only for lists longer than 256 -- and none with cubes of 128 tokens --, so here it
+    must equal the once-rounded form).  In range the
     forms differ in the last bits, which shows that the fp16 forms are the ones that ran, and all sit inside the stated bound."""
     data = syn.make_inputs(wl)
     if what == "large_k":
