@@ -74,7 +74,7 @@ enum { VSA2_FLAG_BF16_COARSE_FWD = 64 }; /* forward of the coarse branch on the 
  * range has an exact fp16 image, so S is unchanged) and rounds dS to fp16, 11 significant bits instead of 8, at the speed
  * of the once-rounded form; with one query head per KV head the dK/dV pass does the same for S, dS and its dK product (P and
  * the dV product stay bf16: |dV| is small).  Measured against the oracle (fp32 outputs, 720p sample): dQ 8.7e-3, dK 3.5e-3.
- * A range flag guards the fp16 forms: a finite |Q| or |K| of 65520 or more, or a |dS| of 65504 or more, and the passes are
+ * A range flag guards the fp16 forms: a finite |Q| or |K| of 65520 or more, or a dS beyond the largest fp16 value, and the passes are
  * redone by the bf16-pair kernels described next (launched behind the fp16 ones, they return at once while the flag is clear).
  * GQA groups (a KV block sums the query blocks of several heads) with TopK >= 8: the dK/dV pass makes fp16 copies of V and dO
  * as well and runs all four products in fp16, P included (480p sample: dK 9.4e-3, dV 2.7e-3; once-rounded bf16 2.2e-2 and

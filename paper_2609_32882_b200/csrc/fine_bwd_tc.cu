@@ -272,15 +272,7 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     cpos.init(g, row & 63);
     const int blk = row >> 6;
     uint32_t tg = 0, n_items = 0;
-    float sat = 0.f;          // F16: largest magnitude of the dS values this thread rounded
     for (uint32_t n_all = 0;; ++n_all) {
-      if constexpr (F16) {
-        // a dS beyond the fp16 range (it was clamped): the result of this launch is not to be used, the fallback launch redoes it
-        if (sat >= 65504.f) {
-          atomicExch(a.range_flag, 1);
-          sat = 0.f;
-        }
-      }
       VSA2_NEXT_ITEM(item, n_all);
       int i, bhq;
       item_block(g, item, bhq, i);
@@ -346,9 +338,8 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 packed_lo[2 * c4] = valid ? l0 : 0u;
                 packed_lo[2 * c4 + 1] = valid ? l1 : 0u;
               } else if constexpr (F16) {
-                packed[2 * c4] = valid ? pack_f16x2_sat(d0, d1) : 0u;
-                packed[2 * c4 + 1] = valid ? pack_f16x2_sat(d2, d3) : 0u;
-                sat = max3_abs(max3_abs(sat, d0, d1), d2, d3);
+                packed[2 * c4] = valid ? pack_f16x2(d0, d1) : 0u;      // (beyond the fp16 range: an infinity, which the
+                packed[2 * c4 + 1] = valid ? pack_f16x2(d2, d3) : 0u;  //  epilogue finds in the accumulator)
               } else {
                 packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
                 packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;
@@ -390,6 +381,11 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           }
           tc::tc_fence_before();
           tc::mbar_arrive(&misc->o_empty);
+          // F16: a dS that left the fp16 range went into the product as an infinity and has made every channel of its query
+          // column non-finite: the result of this launch is not to be used, the fallback launch redoes it
+          if constexpr (F16) {
+            if (row < D && any_non_finite32(o0)) atomicExch(a.range_flag, 1);
+          }
         } else {
 #pragma unroll
           for (int c = 0; c < 32; ++c) o0[c] = 0u;

@@ -89,6 +89,19 @@ __device__ __forceinline__ float max3_abs(float m, float a, float b) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b)));
   return r;
 }
+// fp32 pair -> packed fp16 pair (`lo` in the low half); a value beyond the fp16 range becomes an infinity
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// whether one of 32 accumulator values (float bits) is an infinity or not a number: x * 0 is 0 for every finite x
+__device__ __forceinline__ bool any_non_finite32(const uint32_t (&v)[32]) {
+  float t = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; ++e) t = fmaf(__uint_as_float(v[e]), 0.f, t);
+  return t != t;
+}
 // x -> (bf16(x), bf16(x - bf16(x))) for two values, packed like pack_bf16x2
 __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
   hi = pack_bf16x2(x0, x1);
