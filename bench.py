@@ -38,17 +38,17 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the 720p top-64 launch with 40 heads: an
 # 8-head ncu capture of the same kernels times 5 (every head streams its own tensors, so the traffic grows in
 # proportion to the heads; the 40-head launch is too large for a full-set capture).
-NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.501040e9 + 0.294885e9),
-                                "fine_bwd_dq": 5 * (0.666100e9 + 0.148100e9 + 0.309700e9 + 0.262000e9),   # with the fp16 copy of Q, K
-                                "fine_bwd_dkv": 5 * (0.788600e9 + 0.306500e9)}
+NCU_TRAFFIC_BYTES_720P_TOP64 = {"fine_fwd": 5 * (0.504200e9 + 0.295100e9),
+                                "fine_bwd_dq": 5 * (0.663200e9 + 0.147600e9 + 0.309700e9 + 0.262100e9),   # with the fp16 copy of Q, K
+                                "fine_bwd_dkv": 5 * (0.791600e9 + 0.304900e9)}
 
 
 # What ncu shows as the busiest unit of each tensor kernel at 64-token cubes (8-head capture, profiles/): the roofline
 # below is quoted against the tensor peak as the contract asks, these say what actually holds the kernel there.
 NCU_LIMITER = {
-    "fine_fwd": "L2 -> SM read rate: 12.8 TB/s against 11.8 TB/s sustained peak (tensor pipe 82 % active at the half rate of M = 64)",
-    "fine_bwd_dq": "shared-memory data pipe: tensor-core operand fetches 60 % + thread loads/stores 36 % (tensor pipe 41 %)",
-    "fine_bwd_dkv": "shared-memory data pipe: tensor-core operand fetches 67 % + thread loads/stores 31 % (tensor pipe 47 %)",
+    "fine_fwd": "L2 -> SM read rate: 12.9 TB/s against 11.8 TB/s sustained peak (tensor pipe 82 % active at the half rate of M = 64)",
+    "fine_bwd_dq": "shared-memory data pipe: tensor-core operand fetches 62 % + thread loads/stores 38 % (tensor pipe 42 %)",
+    "fine_bwd_dkv": "shared-memory data pipe: tensor-core operand fetches 67 % + thread loads/stores 32 % (tensor pipe 47 %)",
     "router_lse": "exponential unit 81 %, instruction issue 65 %",
     "router_pool": "exponential unit 77 %, instruction issue 69 %",
 }
