@@ -250,7 +250,10 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           tc::tc_fence_after();
           if (tc::elect_one()) {
             if constexpr (SPLIT) mma_pairT_mnmajor_n128<D>(tmem_base + 256, base + sa * C::SLOT, ds_addr, C::PBYTES, t > 0);
-            else mma_pairT_mnmajor<D, F16>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0);
+            // (F16: the second block of an odd list's last tile repeats the first and stays out of the product; the other
+            //  forms zero its dS rows instead)
+            else mma_pairT_mnmajor<D, F16>(tmem_base + 256, base + sa * C::SLOT, ds_addr + sd * C::PBYTES, t > 0,
+                                           (F16 && t == nt - 1 && (k & 1)) ? 4 : 8);
             tc::mma_commit(&misc->a_empty[sa]);
             tc::mma_commit(&misc->ds_free[sd]);
             if (t == nt - 1) tc::mma_commit(&misc->o_full);
@@ -338,8 +341,12 @@ fine_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 packed_lo[2 * c4] = valid ? l0 : 0u;
                 packed_lo[2 * c4 + 1] = valid ? l1 : 0u;
               } else if constexpr (F16) {
-                packed[2 * c4] = valid ? pack_f16x2(d0, d1) : 0u;      // (beyond the fp16 range: an infinity, which the
-                packed[2 * c4 + 1] = valid ? pack_f16x2(d2, d3) : 0u;  //  epilogue finds in the accumulator)
+                // No validity mask in this form: a key row without a token (a position of an edge cube outside the grid, a row
+                // behind the last text token) is a zero row of the K tile and adds nothing to dQ^T whatever its dS, and the
+                // repeated block of an odd list's last tile is left out by the issuer.  (A dS beyond the fp16 range, such a
+                // row's included, becomes an infinity, which the epilogue finds in the accumulator.)
+                packed[2 * c4] = pack_f16x2(d0, d1);
+                packed[2 * c4 + 1] = pack_f16x2(d2, d3);
               } else {
                 packed[2 * c4] = valid ? pack_bf16x2(d0, d1) : 0u;
                 packed[2 * c4 + 1] = valid ? pack_bf16x2(d2, d3) : 0u;

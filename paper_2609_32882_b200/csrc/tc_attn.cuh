@@ -45,8 +45,10 @@ __device__ __forceinline__ void mma_pair_kmajor(uint32_t tm_acc, uint32_t a_slot
 
 // Issues the 8 (MN-major x MN-major) instructions of  acc[D, 64] (+)= A_pair^T[D, 128] * B[128, 64], where A_pair is a
 // slot in the [half][block A | block B] layout (rows = the 128 contraction indices) and B is a 128-row swizzled tile.
+// `ksteps`: 8, or 4 to contract over the first block of the pair only.
 template <int D, bool F16 = false>
-__device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, bool accumulate_first) {
+__device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_slot, uint32_t b_tile, bool accumulate_first,
+                                                  int ksteps = 8) {
   constexpr uint32_t idesc = F16 ? tc::idesc_f16(128, 64, true, true) : tc::idesc_bf16(128, 64, true, true);
   constexpr uint32_t lbo = (D == 128) ? 2 * kSlab : 0;     // distance between the two 64-channel halves
   const uint64_t da = tc::smem_desc_sw128(a_slot, lbo, 1024), db = tc::smem_desc_sw128(b_tile, 0, 1024);
@@ -54,7 +56,7 @@ __device__ __forceinline__ void mma_pairT_mnmajor(uint32_t tm_acc, uint32_t a_sl
   for (int ks = 0; ks < 8; ++ks) {
     const uint64_t oa = (uint64_t)(((ks / 4) * kSlab + (ks % 4) * 2048) >> 4);
     const uint64_t ob = (uint64_t)((ks * 2048) >> 4);
-    tc::mma_ss(tm_acc, da + oa, db + ob, idesc, accumulate_first || (ks > 0));
+    if (ks < ksteps) tc::mma_ss(tm_acc, da + oa, db + ob, idesc, accumulate_first || (ks > 0));
   }
 }
 
