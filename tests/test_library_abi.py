@@ -50,6 +50,29 @@ def test_query_sizes_matches_the_geometry_of_the_five_configs():
         assert s.route_workspace_bytes % 256 == 0 and s.bwd_workspace_bytes % 256 == 0
 
 
+def test_backward_workspace_holds_the_fp16_copies_of_the_default_forms():
+    """Without a precision flag the backward keeps fp16 copies of Q and K in its workspace (2 bytes per element), for GQA
+    groups that keep 8 blocks or more per row also of V and dO; the once-rounded and the pair forms need none."""
+    def up(x):
+        return (x + 255) // 256 * 256
+
+    def bwd_bytes(wl, **kw):
+        return vb.vsa2_query_sizes(vb.params_from_workload(wl, **kw)).bwd_workspace_bytes
+
+    wl = syn.CONFIGS[3]                                    # one query head per KV head
+    q16 = up(wl.batch * wl.heads_q * wl.L * wl.head_dim * 2)
+    k16 = up(wl.batch * wl.heads_kv * wl.L * wl.head_dim * 2)
+    plain = bwd_bytes(wl, flags=vb.FLAG_FAST_BWD)
+    assert bwd_bytes(wl, flags=vb.FLAG_PRECISE_BWD) == plain
+    assert bwd_bytes(wl) == up(plain) + q16 + k16
+    wl = syn.CONFIGS[2]                                    # 12 query heads on 3 KV heads, top-78
+    q16 = up(wl.batch * wl.heads_q * wl.L * wl.head_dim * 2)
+    k16 = up(wl.batch * wl.heads_kv * wl.L * wl.head_dim * 2)
+    plain = bwd_bytes(wl, flags=vb.FLAG_FAST_BWD)
+    assert bwd_bytes(wl) == up(plain) + 2 * (q16 + k16)
+    assert bwd_bytes(wl, topk=4) == up(plain) + q16 + k16  # rows that keep few blocks: the dK/dV pass stays with its pairs
+
+
 def test_topk_is_clamped_and_keep_fraction_is_honoured():
     wl = syn.CONFIGS[1]
     assert vb.vsa2_query_sizes(vb.params_from_workload(wl, topk=1000)).topk_eff == 32
