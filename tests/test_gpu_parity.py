@@ -403,3 +403,25 @@ def test_backward_leaves_its_fp16_forms_when_a_value_leaves_the_fp16_range(wl, w
             # no list of this problem is longer than 256: the fallback is the once-rounded kernel, which FAST_BWD runs directly
             fast, _ = _grads_of(wl, data, vb.FLAG_FAST_BWD)
             assert torch.equal(got[1], fast[1]) and torch.equal(got[2], fast[2])
+
+
+def test_dq_pass_falls_back_when_a_row_without_a_token_overflows():
+    """The fp16 dQ pass does not mask the dS of key rows that hold no token (positions of an edge cube outside the grid): their
+    K rows are zero.  If every score of a query row lies below -88, exp(0 - lse) of such a row overflows, the product turns its
+    query column into NaN, and the pass must notice and hand over to the pair form, which masks.  Here all scores are -128 on a
+    grid with ragged edges: the results must be finite and equal, bit for bit, to the forms the fallback runs (the problem is
+    too ill-conditioned -- all weights equal, gradients from cancellation -- to be compared with the oracle at the usual bound)."""
+    # grid (6, 9, 10): ragged in all three directions; every query keeps all 18 cubes, the cut ones at the edges included
+    wl = MINI_SEQ.replace(name="mini_dense_ragged", select_mode=syn.PER_QUERY, topk=18)
+    data = syn.make_inputs(wl)
+    rng = np.random.default_rng(7)
+    data["q"] = syn.f32_to_bf16_bits(np.full(data["q"].shape, -16.0, dtype=np.float32))
+    data["k"] = syn.f32_to_bf16_bits((1.0 + 0.01 * rng.standard_normal(data["k"].shape)).astype(np.float32))
+    got, run = _grads_of(wl, data, 0)
+    pair, _ = _grads_of(wl, data, vb.FLAG_PRECISE_BWD)
+    fast, _ = _grads_of(wl, data, vb.FLAG_FAST_BWD)
+    for t in got:
+        assert torch.isfinite(t).all()
+    assert run.mask.all()
+    assert torch.equal(got[0], pair[0])
+    assert torch.equal(got[1], fast[1]) and torch.equal(got[2], fast[2])
